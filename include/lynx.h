@@ -1,0 +1,146 @@
+/*
+ * lynx.h -- C interface of the B200 (sm_100a) library for the data-parallel hot path of
+ * Lynx's progressive speculative quantisation of the KV cache.
+ *
+ * The path (paper sections in brackets):
+ *   1. split-quantise: BF16 K or V rows -> 8-bit linear per-group codes (Section 2.3,
+ *      "Standard & Grouped Quantization": Q(X) = round(X/S + Z), S from the group's min-max
+ *      range) split into an Anchor plane (top 4 bits) and a Residual plane (bottom 4 bits),
+ *      two 4-bit values per byte, each stream contiguous, the scalars travelling with the
+ *      Anchor stream (Section 4.1 stage 4; Section "Implementation", Compression Kernel).
+ *   2. anchor attention: decode attention softmax(Q K^T / sqrt(d)) V (Section 2) evaluated on
+ *      the Anchor plane alone, which is what the decode instance has when it starts drafting
+ *      (Section 4.2, Anchor Phase).
+ *   3. merge-verify attention: Anchor and Residual recombined into the full 8-bit state
+ *      Q_full (Section 4.2, Residual Phase), the k drafted positions scored in one pass and the
+ *      longest agreeing prefix reported (Section 4.3).
+ *   4. recombine: the stand-alone Residual-phase refinement to full codes / BF16 pages.
+ *
+ * Group = one token's head vector of 128 elements (a "row").  Per row:
+ *   mn = min, mx = max, range = fl(mx - mn), scale = fl(range/255), inv = fl(255/range),
+ *   zero = mn (with -0 stored as +0); range < 2^-100 -> scale = inv = 0 (constant row);
+ *   code = round-half-even of the exact product fl(x - mn) * inv, in [0, 255];
+ *   anchor nibble a = code >> 4, residual nibble r = code & 15;
+ *   byte j of a plane row = nibble of element 2j (low half) | nibble of element 2j+1 << 4.
+ * Reconstruction: full state x^ = zero + scale * (16 a + r); Anchor-only state
+ * x^ = zero + scale * (16 a + 8) (bucket mid-point).  Inputs must be finite.
+ *
+ * Memory layout of a quantised K (or V) cache of one layer, paged:
+ *   anchor, residual : uint8 [num_blocks][num_kv_heads][block_tokens][64]
+ *   meta             : float [num_blocks][num_kv_heads][block_tokens][2] = {scale, zero}
+ * Token t of sequence b lives in row (t % block_tokens) of block
+ * block_table[b][t / block_tokens].  A contiguous cache is the identity block table.
+ * Several layers may be flattened into the batch dimension (each (layer, sequence) pair is an
+ * independent problem with its own block-table row).
+ *
+ * Conventions for every call:
+ *   - every pointer is a DEVICE pointer owned by the caller unless stated otherwise; the
+ *     library never allocates, frees or synchronises (lynx_check is the one exception);
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream); calls
+ *     only enqueue work and return;
+ *   - arguments are validated on the host before any launch; an invalid call launches
+ *     nothing and returns a status other than LYNX_OK;
+ *   - device code never traps: block ids outside [0, num_blocks) are clamped and recorded in
+ *     the workspace's status word, which lynx_check turns into LYNX_ERR_BAD_BLOCK_TABLE.
+ */
+#ifndef LYNX_H_
+#define LYNX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LYNX_OK = 0,
+  LYNX_ERR_NULL = 1,            /* a required pointer is NULL */
+  LYNX_ERR_SHAPE = 2,           /* negative / zero / inconsistent size */
+  LYNX_ERR_ALIGN = 3,           /* a pointer is not 16-byte aligned */
+  LYNX_ERR_UNSUPPORTED = 4,     /* head_dim != 128, block_tokens % 16 != 0, too many columns */
+  LYNX_ERR_WORKSPACE = 5,       /* workspace too small (see lynx_workspace_bytes) */
+  LYNX_ERR_CUDA = 6,            /* a CUDA runtime call failed */
+  LYNX_ERR_BAD_BLOCK_TABLE = 7, /* (lynx_check) a kernel saw a block id out of range */
+  LYNX_ERR_TIMEOUT = 8          /* (lynx_check) a bounded on-chip wait ran out */
+} lynx_status;
+
+/* One of K or V of one layer (or of several flattened layers), quantised and paged. */
+typedef struct {
+  const uint8_t* anchor;   /* [num_blocks][Hkv][block_tokens][64] */
+  const uint8_t* residual; /* same shape; ignored (may be NULL) by lynx_anchor_attention */
+  const float* meta;       /* [num_blocks][Hkv][block_tokens][2] = {scale, zero} */
+} lynx_plane;
+
+typedef struct {
+  int32_t num_q_heads;        /* Hq, a multiple of num_kv_heads; Hq/Hkv in 1..16 */
+  int32_t num_kv_heads;       /* Hkv */
+  int32_t head_dim;           /* must be 128 */
+  int32_t block_tokens;       /* tokens per block, a multiple of 16 */
+  int32_t num_blocks;         /* blocks in the pool the planes cover */
+  int32_t max_blocks_per_seq; /* row length of block_table */
+} lynx_shape;
+
+/* Steps 1 (Section 2.3 quantiser; Section 4.1 stage 4 split; Compression Kernel packing).
+ * src_bf16 : [n_rows][128] BF16, 16-byte aligned.  Row i of src produces row i of anchor
+ *            ([n_rows][64] u8), residual ([n_rows][64] u8) and meta ([n_rows][2] float).
+ * block_ids: NULL -> all rows 0..n_rows-1 are quantised.  Otherwise int32 [n_block_ids]:
+ *            only rows block_ids[i]*rows_per_block .. +rows_per_block-1 are quantised (newly
+ *            arrived blocks); ids outside [0, n_rows/rows_per_block) are skipped.  n_rows must
+ *            then be a multiple of rows_per_block.
+ * n_rows == 0 (or n_block_ids == 0) is a valid no-op. */
+lynx_status lynx_split_quantize(const void* src_bf16, int64_t n_rows, const int32_t* block_ids,
+                                int32_t n_block_ids, int32_t rows_per_block, uint8_t* anchor,
+                                uint8_t* residual, float* meta, void* stream);
+
+/* Step 4 (Section 4.2 Residual Phase refinement to Q_full).  For each of n_rows rows:
+ * code = (a << 4) | r.  codes_u8 ([n_rows][128] u8) and dequant_bf16 ([n_rows][128] BF16 =
+ * bf16_rne(fl(fma(code, scale, zero)))) are optional outputs; at least one must be given. */
+lynx_status lynx_recombine(const uint8_t* anchor, const uint8_t* residual, const float* meta,
+                           int64_t n_rows, uint8_t* codes_u8, void* dequant_bf16, void* stream);
+
+/* Bytes of workspace the two attention calls need for `batch` sequences, `n_cols_q` query
+ * positions (n_q or k) and sequences of at most max_blocks_per_seq * block_tokens tokens.
+ * Returns 0 for an unsupported shape.  The workspace must be zero-filled once before its first
+ * use (lynx_workspace_init, or cudaMemsetAsync of the whole buffer); each call leaves it ready
+ * for the next.  Calls sharing a workspace must be ordered on one stream. */
+size_t lynx_workspace_bytes(const lynx_shape* shape, int32_t batch, int32_t n_cols_q);
+lynx_status lynx_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Step 2 (Section 2 attention equation on the Anchor-only state of Section 4.2).
+ * q_bf16 : [batch][n_q][Hq][128] BF16; query head h reads KV head h / (Hq/Hkv).
+ * Query j of sequence b attends tokens [0, seq_lens[b]) (causal == 0) or
+ * [0, seq_lens[b] - n_q + j + 1) (causal != 0); a query that sees no token gets zeros.
+ * softmax_scale 0 means 1/sqrt(128).  out : [batch][n_q][Hq][128] float.
+ * n_q * (Hq/Hkv) must be <= 64.  seq_lens[b] is clamped to the table's capacity. */
+lynx_status lynx_anchor_attention(const lynx_shape* shape, const void* q_bf16, int32_t batch,
+                                  int32_t n_q, int32_t causal, lynx_plane K, lynx_plane V,
+                                  const int32_t* block_table, const int32_t* seq_lens,
+                                  float softmax_scale, float* out, void* workspace,
+                                  size_t workspace_bytes, void* stream);
+
+/* Step 3 (Section 4.2 Residual Phase + Section 4.3 verification).  Same attention on the
+ * recombined full codes for the k drafted positions in one pass over the context, then per
+ * sequence   dev[b][j] = max over heads, dims of |out_full - draft| / (atol + rtol*|out_full|)
+ * and first_reject[b] = smallest j with dev[b][j] > 1, or k if none (the longest agreeing
+ * prefix; out_full at that position is the correction).
+ * draft_out : [batch][k][Hq][128] float, the Anchor-state results being verified; may be NULL,
+ * then dev / first_reject are not written (and may be NULL).  out_full : same shape, float. */
+lynx_status lynx_merge_verify_attention(const lynx_shape* shape, const void* q_bf16,
+                                        int32_t batch, int32_t k, int32_t causal, lynx_plane K,
+                                        lynx_plane V, const int32_t* block_table,
+                                        const int32_t* seq_lens, float softmax_scale,
+                                        const float* draft_out, float atol, float rtol,
+                                        float* out_full, int32_t* first_reject, float* dev,
+                                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronises `stream`, reads and clears the workspace's status word.  Test / debug use. */
+lynx_status lynx_check(void* workspace, void* stream);
+
+const char* lynx_status_string(lynx_status s);
+int lynx_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LYNX_H_ */

@@ -1,0 +1,222 @@
+"""Thin Python binding of the Lynx C-ABI CUDA library (sm_100a).
+
+Argument marshalling only: every step of the path runs in the library's kernels.  Torch is
+used for device memory and streams.  There is no CPU fallback: if ``liblynx.so`` is missing
+or a call returns an error status, an exception is raised.
+
+Names mirror ``include/lynx.h``: split_quantize, recombine, anchor_attention,
+merge_verify_attention, workspace_bytes.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "liblynx.so")
+_lib = None
+
+D = 128
+
+
+class LynxError(RuntimeError):
+    pass
+
+
+class _Plane(ctypes.Structure):
+    _fields_ = [("anchor", ctypes.c_void_p), ("residual", ctypes.c_void_p), ("meta", ctypes.c_void_p)]
+
+
+class _Shape(ctypes.Structure):
+    _fields_ = [("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("block_tokens", ctypes.c_int32),
+                ("num_blocks", ctypes.c_int32), ("max_blocks_per_seq", ctypes.c_int32)]
+
+
+EXPORTS = ["lynx_split_quantize", "lynx_recombine", "lynx_workspace_bytes", "lynx_workspace_init",
+           "lynx_anchor_attention", "lynx_merge_verify_attention", "lynx_check",
+           "lynx_status_string", "lynx_version"]
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def load():
+    """Load liblynx.so (built in-tree by paper_2607_01831_b200/build.py). Fails loudly."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise LynxError(f"{_LIB_PATH} is missing: build it with `python -m paper_2607_01831_b200.build` "
+                        "(there is no CPU fallback)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+    lib.lynx_split_quantize.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp, vp]
+    lib.lynx_split_quantize.restype = ctypes.c_int
+    lib.lynx_recombine.argtypes = [vp, vp, vp, i64, vp, vp, vp]
+    lib.lynx_recombine.restype = ctypes.c_int
+    lib.lynx_workspace_bytes.argtypes = [ctypes.POINTER(_Shape), i32, i32]
+    lib.lynx_workspace_bytes.restype = ctypes.c_size_t
+    lib.lynx_workspace_init.argtypes = [vp, ctypes.c_size_t, vp]
+    lib.lynx_workspace_init.restype = ctypes.c_int
+    lib.lynx_anchor_attention.argtypes = [ctypes.POINTER(_Shape), vp, i32, i32, i32, _Plane, _Plane,
+                                          vp, vp, f32, vp, vp, ctypes.c_size_t, vp]
+    lib.lynx_anchor_attention.restype = ctypes.c_int
+    lib.lynx_merge_verify_attention.argtypes = [ctypes.POINTER(_Shape), vp, i32, i32, i32, _Plane,
+                                                _Plane, vp, vp, f32, vp, f32, f32, vp, vp, vp, vp,
+                                                ctypes.c_size_t, vp]
+    lib.lynx_merge_verify_attention.restype = ctypes.c_int
+    lib.lynx_check.argtypes = [vp, vp]
+    lib.lynx_check.restype = ctypes.c_int
+    lib.lynx_status_string.argtypes = [ctypes.c_int]
+    lib.lynx_status_string.restype = ctypes.c_char_p
+    lib.lynx_version.restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _ok(status: int, what: str):
+    if status != 0:
+        msg = load().lynx_status_string(status).decode()
+        raise LynxError(f"{what}: status {status} ({msg})")
+
+
+def _ptr(t: torch.Tensor | None):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise LynxError("device tensors required")
+    if not t.is_contiguous():
+        raise LynxError("contiguous tensors required")
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+@dataclass
+class Planes:
+    """Quantised K or V: anchor / residual u8 [..., 64], meta f32 [..., 2] (device tensors)."""
+    anchor: torch.Tensor
+    residual: torch.Tensor | None
+    meta: torch.Tensor
+
+    def _c(self) -> _Plane:
+        return _Plane(_ptr(self.anchor), _ptr(self.residual), _ptr(self.meta))
+
+
+def alloc_planes(lead_shape, device) -> Planes:
+    lead = tuple(lead_shape)
+    return Planes(torch.empty(lead + (64,), dtype=torch.uint8, device=device),
+                  torch.empty(lead + (64,), dtype=torch.uint8, device=device),
+                  torch.empty(lead + (2,), dtype=torch.float32, device=device))
+
+
+def split_quantize(src: torch.Tensor, out: Planes | None = None, block_ids: torch.Tensor | None = None,
+                   rows_per_block: int = 0) -> Planes:
+    """lynx_split_quantize: src BF16 [..., 128] -> Planes with the same leading shape."""
+    if src.dtype != torch.bfloat16 or src.shape[-1] != D:
+        raise LynxError("src must be BF16 [..., 128]")
+    if out is None:
+        out = alloc_planes(src.shape[:-1], src.device)
+    n_rows = src.numel() // D
+    nb = 0 if block_ids is None else block_ids.numel()
+    _ok(load().lynx_split_quantize(_ptr(src), n_rows, _ptr(block_ids), nb, rows_per_block,
+                                   _ptr(out.anchor), _ptr(out.residual), _ptr(out.meta), _stream()),
+        "lynx_split_quantize")
+    return out
+
+
+def recombine(planes: Planes, want_codes: bool = True, want_bf16: bool = False):
+    """lynx_recombine: returns (codes u8 [...,128] or None, dequantised BF16 [...,128] or None)."""
+    lead = tuple(planes.anchor.shape[:-1])
+    dev = planes.anchor.device
+    codes = torch.empty(lead + (D,), dtype=torch.uint8, device=dev) if want_codes else None
+    deq = torch.empty(lead + (D,), dtype=torch.bfloat16, device=dev) if want_bf16 else None
+    n_rows = planes.anchor.numel() // 64
+    _ok(load().lynx_recombine(_ptr(planes.anchor), _ptr(planes.residual), _ptr(planes.meta), n_rows,
+                              _ptr(codes), _ptr(deq), _stream()), "lynx_recombine")
+    return codes, deq
+
+
+@dataclass
+class Geometry:
+    num_q_heads: int
+    num_kv_heads: int
+    block_tokens: int
+    num_blocks: int
+    max_blocks_per_seq: int
+    head_dim: int = D
+
+    def _c(self) -> _Shape:
+        return _Shape(self.num_q_heads, self.num_kv_heads, self.head_dim, self.block_tokens,
+                      self.num_blocks, self.max_blocks_per_seq)
+
+
+def workspace_bytes(geo: Geometry, batch: int, n_q: int) -> int:
+    return int(load().lynx_workspace_bytes(ctypes.byref(geo._c()), batch, n_q))
+
+
+def make_workspace(geo: Geometry, batch: int, n_q: int, device) -> torch.Tensor:
+    """Allocate and zero a workspace large enough for (batch, n_q) attention calls."""
+    n = workspace_bytes(geo, batch, n_q)
+    if n == 0:
+        raise LynxError("unsupported attention shape")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    _ok(load().lynx_workspace_init(_ptr(ws), n, _stream()), "lynx_workspace_init")
+    return ws
+
+
+def check(workspace: torch.Tensor):
+    """lynx_check: synchronises and raises if a kernel recorded a bad block id or a timeout."""
+    _ok(load().lynx_check(_ptr(workspace), _stream()), "lynx_check")
+
+
+def anchor_attention(geo: Geometry, q: torch.Tensor, K: Planes, V: Planes, block_table: torch.Tensor,
+                     seq_lens: torch.Tensor, workspace: torch.Tensor, causal: bool = False,
+                     softmax_scale: float = 0.0, out: torch.Tensor | None = None) -> torch.Tensor:
+    """lynx_anchor_attention: q BF16 [B][n_q][Hq][128] -> float32 [B][n_q][Hq][128]."""
+    B, n_q, Hq, d = q.shape
+    if q.dtype != torch.bfloat16 or d != D or Hq != geo.num_q_heads:
+        raise LynxError("q must be BF16 [B][n_q][Hq][128]")
+    if out is None:
+        out = torch.empty(B, n_q, Hq, D, dtype=torch.float32, device=q.device)
+    _ok(load().lynx_anchor_attention(ctypes.byref(geo._c()), _ptr(q), B, n_q, int(causal), K._c(),
+                                     V._c(), _ptr(block_table), _ptr(seq_lens), softmax_scale,
+                                     _ptr(out), _ptr(workspace), workspace.numel(), _stream()),
+        "lynx_anchor_attention")
+    return out
+
+
+def merge_verify_attention(geo: Geometry, q: torch.Tensor, K: Planes, V: Planes,
+                           block_table: torch.Tensor, seq_lens: torch.Tensor, workspace: torch.Tensor,
+                           draft_out: torch.Tensor | None = None, atol: float = 0.0, rtol: float = 0.0,
+                           causal: bool = True, softmax_scale: float = 0.0,
+                           out_full: torch.Tensor | None = None, first_reject: torch.Tensor | None = None,
+                           dev: torch.Tensor | None = None):
+    """lynx_merge_verify_attention -> (out_full f32 [B][k][Hq][128], first_reject i32 [B], dev f32 [B][k]).
+    first_reject / dev are None when no draft is given."""
+    B, k, Hq, d = q.shape
+    if q.dtype != torch.bfloat16 or d != D or Hq != geo.num_q_heads:
+        raise LynxError("q must be BF16 [B][k][Hq][128]")
+    if out_full is None:
+        out_full = torch.empty(B, k, Hq, D, dtype=torch.float32, device=q.device)
+    if draft_out is not None:
+        if draft_out.dtype != torch.float32 or tuple(draft_out.shape) != (B, k, Hq, D):
+            raise LynxError("draft_out must be float32 [B][k][Hq][128]")
+        if first_reject is None:
+            first_reject = torch.empty(B, dtype=torch.int32, device=q.device)
+        if dev is None:
+            dev = torch.empty(B, k, dtype=torch.float32, device=q.device)
+    _ok(load().lynx_merge_verify_attention(ctypes.byref(geo._c()), _ptr(q), B, k, int(causal), K._c(),
+                                           V._c(), _ptr(block_table), _ptr(seq_lens), softmax_scale,
+                                           _ptr(draft_out), atol, rtol, _ptr(out_full),
+                                           _ptr(first_reject), _ptr(dev), _ptr(workspace),
+                                           workspace.numel(), _stream()),
+        "lynx_merge_verify_attention")
+    return out_full, first_reject, dev

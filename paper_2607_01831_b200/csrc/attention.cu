@@ -1,0 +1,848 @@
+// lynx_anchor_attention and lynx_merge_verify_attention: split-K decode attention over the
+// packed nibble planes, dequantised in registers (sm_100a).
+//
+// What is computed (Section 2 attention equation on the states of Section 4.2; accept/reject
+// of Section 4.3): for every (sequence, KV head) the G = Hq/Hkv query heads of each of the n_q
+// query positions ("columns", n_q*G of them) share one pass over that head's K and V planes.
+//
+// Per-token groups make dequantisation almost free: with x^ = zero_t + scale_t * level,
+//     q . K^_t        = scale_t * (q . level_t) + zero_t * sum_d q_d
+//     sum_t p_t V^_t  = sum_t (p_t scale_t) level_t + (sum_t p_t zero_t) * 1
+// so the two contractions run on the integer levels, which are exact in FP16, and the scalars
+// are applied per token outside.  Levels are centred (a-8 for the Anchor state, code-128 for
+// the full state) so that no large bias enters the FP32 accumulation.
+//
+// Kernel shape.  Grid = (chunk, KV head, sequence): flash-decoding split-K over the context.
+// A CTA has TW*CG consumer warps and one producer warp.  The producer streams 16-token
+// sub-blocks (1 KiB per plane + 128 B of meta, each contiguous in the paged layout) into a
+// shared-memory ring with cp.async.bulk (TMA, 1-D) completing on mbarriers.  Consumer warp
+// (tw, cg) takes 16-token tile tw of every stage for columns [cg*NT*8, (cg+1)*NT*8):
+//   S^T[16 tok x 8 col] = level(K)[16 x 128] . Q^T        mma.m16n8k16, tokens are M
+//   online softmax with a lazily updated maximum (one warp vote per tile, no shuffles)
+//   P^T -> B operand by movmatrix (8x8 b16 transpose)
+//   O^T[128 dim x 8 col] += level(V)^T[128 x 16 tok] . P^T  mma.m16n8k16, dims are M
+// Operands are built straight from the nibbles with LOP3/PRMT and one FP16 add/fma per pair.
+// Partials (m, l, O) are merged across the CTA's token warps in shared memory, written to the
+// workspace, and the last CTA of a (sequence, KV head) (atomic ticket, no waiting) merges the
+// chunks; for verification the last CTA of a sequence also takes the accept/reject decision.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "lynx_common.cuh"
+
+namespace lynx {
+namespace {
+
+constexpr int kMaxQ = 16;          // query positions per call
+constexpr int kMaxCols = 64;       // n_q * G
+constexpr int kMaxChunkTokens = 8192;
+constexpr int kPartStride = 132;   // floats per (chunk, column) partial: O[128], m, l, pad
+
+struct AttnParams {
+  const __nv_bfloat16* q;
+  const uint8_t *ka, *kr, *va, *vr;
+  const float *km, *vm;
+  const int32_t* block_table;
+  const int32_t* seq_lens;
+  float* out;
+  const float* draft;
+  int32_t* first_reject;
+  float* dev;
+  uint32_t* ws_flags;
+  uint32_t* ws_chunk_ctr;  // [B*Hkv]
+  uint32_t* ws_seq_ctr;    // [B]
+  float* ws_dev;           // [B*Hkv][kMaxQ]
+  float* ws_part;          // [B*Hkv][max_chunks][ncols_pad][kPartStride]
+  float atol, rtol;
+  float sm_log2;           // softmax_scale * log2(e)
+  int B, nq, causal, Hq, Hkv, G, bt, num_blocks, max_blocks, chunk_tokens, max_chunks, ncols;
+};
+
+// ------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: gives up after ~2 s (or as soon as another thread of the CTA gave up), records
+// it in the CTA's abort word and returns false.  Nothing in this kernel waits on another CTA.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_word) {
+  const uint64_t t0 = globaltimer_ns();
+  for (;;) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_word) return false;
+    if (globaltimer_ns() - t0 > 2000000000ull) {
+      *abort_word = 1;
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_word);
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                         uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+__device__ __forceinline__ uint32_t hadd2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("add.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t hfma2(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  return __byte_perm(a, b, sel);
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float2 lds64f(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
+
+// FP16x2 constants
+constexpr uint32_t kMagic = 0x64006400u;      // 1024, 1024
+constexpr uint32_t kNeg1032 = 0xE408E408u;    // -1032
+constexpr uint32_t kSixteenth = 0x2C002C00u;  // 1/16
+constexpr uint32_t kNeg72 = 0xD480D480u;      // -72
+constexpr uint32_t kNeg1152 = 0xE480E480u;    // -1152
+
+// Four FP16 pairs (value - 8) from the low 16 bits of each half of u: nibbles 0..3 of the low
+// half go to the low lanes, nibbles 0..3 of the high half to the high lanes.
+__device__ __forceinline__ void nib4_to_h2(uint32_t u, uint32_t (&r)[4]) {
+  const uint32_t s = u >> 8;
+  r[0] = hadd2((u & 0x000F000Fu) | kMagic, kNeg1032);
+  r[1] = hfma2((u & 0x00F000F0u) | kMagic, kSixteenth, kNeg72);
+  r[2] = hadd2((s & 0x000F000Fu) | kMagic, kNeg1032);
+  r[3] = hfma2((s & 0x00F000F0u) | kMagic, kSixteenth, kNeg72);
+}
+// Full codes of 8 elements from an anchor word and a residual word: ev = codes of elements
+// 0,2,4,6 (one per byte), od = codes of elements 1,3,5,7.
+__device__ __forceinline__ void merge_codes(uint32_t xa, uint32_t xr, uint32_t& ev, uint32_t& od) {
+  ev = ((xa << 4) & 0xF0F0F0F0u) | (xr & 0x0F0F0F0Fu);
+  od = (xa & 0xF0F0F0F0u) | ((xr >> 4) & 0x0F0F0F0Fu);
+}
+// token row permutation inside a 16-token tile (keeps the shared-memory reads of both the
+// K fragments and the V fragments at <= 2-way bank conflicts)
+__device__ __forceinline__ int pi_row(int r) { return r ^ ((r >> 1) & 1); }
+
+template <bool FULL, int NT>
+struct WarpState {
+  uint32_t qf[NT][8][2];  // Q^T B-fragments: [n-tile][k-step][reg]
+  float qs[NT][2];        // sum_d q_d of the thread's two columns (times 2^-e already folded)
+  float m[NT][2];         // running (lazy) maximum, log2 units
+  float l[NT][2];         // partial softmax denominators (this thread's rows only)
+  float zs[NT][2];        // partial sum p * (zero + mid*scale) of V
+  float o[NT][8][4];      // O^T accumulators: [n-tile][m-tile (16 dims)][c-reg]
+  int lim[NT][2];         // exclusive token limit of the thread's two columns
+};
+
+// One 16-token tile.  st = shared address of the stage, tw = tile index within the stage,
+// tile_t0 = absolute index of the tile's first token, masked = some (token, column) of this
+// tile is not visible.
+template <bool FULL, int NT, int ST>
+__device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st, int tw, int tile_t0,
+                                             bool masked, float ca, float cb, int g, int t) {
+  constexpr uint32_t KA = 0, VA = ST * 64, KR = ST * 128, VR = ST * 192;
+  constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
+  constexpr float kMidK = FULL ? 128.0f : 136.0f;
+  constexpr float kLevelScaleV = FULL ? 1.0f : 16.0f;
+  const int r0 = tw * 16 + pi_row(g);  // stage row of S row g; S row g+8 is r0 + 8
+
+  // ---- S^T = level(K) . Q^T ------------------------------------------------------------
+  float s[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s[nt][i] = 0.0f;
+  {
+    const uint4 a_lo = lds128(st + KA + r0 * 64 + t * 16);
+    const uint4 a_hi = lds128(st + KA + (r0 + 8) * 64 + t * 16);
+    const uint32_t xl[4] = {a_lo.x, a_lo.y, a_lo.z, a_lo.w};
+    const uint32_t xh[4] = {a_hi.x, a_hi.y, a_hi.z, a_hi.w};
+    if (!FULL) {
+#pragma unroll
+      for (int wd = 0; wd < 4; ++wd) {
+        uint32_t rl[4], rh[4];
+        nib4_to_h2(xl[wd], rl);  // pairs (e0,e4) (e1,e5) (e2,e6) (e3,e7) of row g
+        nib4_to_h2(xh[wd], rh);  // same of row g+8
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          mma16816(s[nt], rl[0], rh[0], rl[1], rh[1], w.qf[nt][2 * wd][0], w.qf[nt][2 * wd][1]);
+          mma16816(s[nt], rl[2], rh[2], rl[3], rh[3], w.qf[nt][2 * wd + 1][0], w.qf[nt][2 * wd + 1][1]);
+        }
+      }
+    } else {
+      const uint4 b_lo = lds128(st + KR + r0 * 64 + t * 16);
+      const uint4 b_hi = lds128(st + KR + (r0 + 8) * 64 + t * 16);
+      const uint32_t yl[4] = {b_lo.x, b_lo.y, b_lo.z, b_lo.w};
+      const uint32_t yh[4] = {b_hi.x, b_hi.y, b_hi.z, b_hi.w};
+#pragma unroll
+      for (int wd = 0; wd < 4; ++wd) {
+        uint32_t evl, odl, evh, odh;
+        merge_codes(xl[wd], yl[wd], evl, odl);
+        merge_codes(xh[wd], yh[wd], evh, odh);
+        // (e0,e2) (e4,e6) from ev; (e1,e3) (e5,e7) from od; value = code - 128
+        const uint32_t l0 = hadd2(prmt(evl, kMagic, 0x5140), kNeg1152), l1 = hadd2(prmt(evl, kMagic, 0x7362), kNeg1152);
+        const uint32_t l2 = hadd2(prmt(odl, kMagic, 0x5140), kNeg1152), l3 = hadd2(prmt(odl, kMagic, 0x7362), kNeg1152);
+        const uint32_t h0 = hadd2(prmt(evh, kMagic, 0x5140), kNeg1152), h1 = hadd2(prmt(evh, kMagic, 0x7362), kNeg1152);
+        const uint32_t h2 = hadd2(prmt(odh, kMagic, 0x5140), kNeg1152), h3 = hadd2(prmt(odh, kMagic, 0x7362), kNeg1152);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          mma16816(s[nt], l0, h0, l2, h2, w.qf[nt][2 * wd][0], w.qf[nt][2 * wd][1]);
+          mma16816(s[nt], l1, h1, l3, h3, w.qf[nt][2 * wd + 1][0], w.qf[nt][2 * wd + 1][1]);
+        }
+      }
+    }
+  }
+
+  // ---- per-token scalars, scores in log2 units -----------------------------------------
+  float2 km_lo = lds64f(st + KM + r0 * 8), km_hi = lds64f(st + KM + (r0 + 8) * 8);
+  float2 vm_lo = lds64f(st + VM + r0 * 8), vm_hi = lds64f(st + VM + (r0 + 8) * 8);
+  const int tok_lo = tile_t0 + pi_row(g), tok_hi = tok_lo + 8;
+  if (masked) {
+    // rows beyond every column's limit may hold arbitrary bits: neutralise their scalars
+    int maxlim = 0;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) maxlim = max(maxlim, max(w.lim[nt][0], w.lim[nt][1]));
+    maxlim = max(maxlim, __shfl_xor_sync(0xFFFFFFFFu, maxlim, 1));
+    maxlim = max(maxlim, __shfl_xor_sync(0xFFFFFFFFu, maxlim, 2));
+    if (tok_lo >= maxlim) { km_lo = make_float2(0.f, 0.f); vm_lo = make_float2(0.f, 0.f); }
+    if (tok_hi >= maxlim) { km_hi = make_float2(0.f, 0.f); vm_hi = make_float2(0.f, 0.f); }
+  }
+  const float al_lo = km_lo.x * ca, al_hi = km_hi.x * ca;
+  const float be_lo = fmaf(km_lo.x, kMidK, km_lo.y) * cb, be_hi = fmaf(km_hi.x, kMidK, km_hi.y) * cb;
+  bool grow = false;
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    s[nt][0] = fmaf(al_lo, s[nt][0], be_lo * w.qs[nt][0]);
+    s[nt][1] = fmaf(al_lo, s[nt][1], be_lo * w.qs[nt][1]);
+    s[nt][2] = fmaf(al_hi, s[nt][2], be_hi * w.qs[nt][0]);
+    s[nt][3] = fmaf(al_hi, s[nt][3], be_hi * w.qs[nt][1]);
+    if (masked) {
+      if (tok_lo >= w.lim[nt][0]) s[nt][0] = -INFINITY;
+      if (tok_lo >= w.lim[nt][1]) s[nt][1] = -INFINITY;
+      if (tok_hi >= w.lim[nt][0]) s[nt][2] = -INFINITY;
+      if (tok_hi >= w.lim[nt][1]) s[nt][3] = -INFINITY;
+    }
+    grow |= fmaxf(s[nt][0], s[nt][2]) > w.m[nt][0] + 4.0f;
+    grow |= fmaxf(s[nt][1], s[nt][3]) > w.m[nt][1] + 4.0f;
+  }
+  // ---- lazy maximum: raise it only when some score exceeds it by more than 4 (p <= 16) --
+  if (__any_sync(0xFFFFFFFFu, grow)) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        float mx = fmaxf(s[nt][c], s[nt][c + 2]);
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 4));
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 8));
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));
+        const float mn = fmaxf(w.m[nt][c], mx);
+        const float f = ex2(w.m[nt][c] - mn);
+        w.m[nt][c] = mn;
+        w.l[nt][c] *= f;
+        w.zs[nt][c] *= f;
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          w.o[nt][mt][c] *= f;
+          w.o[nt][mt][c + 2] *= f;
+        }
+      }
+    }
+  }
+  // ---- p, denominators, zero-point sums, P^T fragments ---------------------------------
+  const float sv_lo = vm_lo.x * kLevelScaleV, sv_hi = vm_hi.x * kLevelScaleV;
+  const float zv_lo = fmaf(vm_lo.x, kMidK, vm_lo.y), zv_hi = fmaf(vm_hi.x, kMidK, vm_hi.y);
+  uint32_t pb[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const float p0 = ex2(s[nt][0] - w.m[nt][0]), p1 = ex2(s[nt][1] - w.m[nt][1]);
+    const float p2 = ex2(s[nt][2] - w.m[nt][0]), p3 = ex2(s[nt][3] - w.m[nt][1]);
+    w.l[nt][0] += p0 + p2;
+    w.l[nt][1] += p1 + p3;
+    w.zs[nt][0] = fmaf(p0, zv_lo, fmaf(p2, zv_hi, w.zs[nt][0]));
+    w.zs[nt][1] = fmaf(p1, zv_lo, fmaf(p3, zv_hi, w.zs[nt][1]));
+    pb[nt][0] = movmatrix_trans(pack_f16x2(p0 * sv_lo, p1 * sv_lo));  // tokens (2t,2t+1) of rows 0..7
+    pb[nt][1] = movmatrix_trans(pack_f16x2(p2 * sv_hi, p3 * sv_hi));  // tokens of rows 8..15
+  }
+
+  // ---- O^T += level(V)^T . P^T ---------------------------------------------------------
+  // this thread feeds tokens pi(2t), pi(2t+1) (+8) and dims 16g .. 16g+15
+  const int ta = tw * 16 + pi_row(2 * t), tb = tw * 16 + pi_row(2 * t + 1);
+  const uint2 va = lds64(st + VA + ta * 64 + g * 8), vb = lds64(st + VA + tb * 64 + g * 8);
+  const uint2 vc = lds64(st + VA + (ta + 8) * 64 + g * 8), vd = lds64(st + VA + (tb + 8) * 64 + g * 8);
+  const uint32_t A[2] = {va.x, va.y}, Bw[2] = {vb.x, vb.y}, C[2] = {vc.x, vc.y}, Dw[2] = {vd.x, vd.y};
+  if (!FULL) {
+#pragma unroll
+    for (int wd = 0; wd < 2; ++wd) {
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const uint32_t sel = half ? 0x7632u : 0x5410u;
+        uint32_t ab[4], cd[4];
+        nib4_to_h2(prmt(A[wd], Bw[wd], sel), ab);  // dims e(4half+0..3), token pair (a, b)
+        nib4_to_h2(prmt(C[wd], Dw[wd], sel), cd);  // same dims, token pair (c, d)
+#pragma unroll
+        for (int qd = 0; qd < 2; ++qd) {
+          const int mt = wd * 4 + half * 2 + qd;
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+            mma16816(w.o[nt][mt], ab[2 * qd], ab[2 * qd + 1], cd[2 * qd], cd[2 * qd + 1], pb[nt][0], pb[nt][1]);
+        }
+      }
+    }
+  } else {
+    const uint2 ra = lds64(st + VR + ta * 64 + g * 8), rb = lds64(st + VR + tb * 64 + g * 8);
+    const uint2 rc = lds64(st + VR + (ta + 8) * 64 + g * 8), rd = lds64(st + VR + (tb + 8) * 64 + g * 8);
+    const uint32_t RA[2] = {ra.x, ra.y}, RB[2] = {rb.x, rb.y}, RC[2] = {rc.x, rc.y}, RD[2] = {rd.x, rd.y};
+#pragma unroll
+    for (int wd = 0; wd < 2; ++wd) {
+      uint32_t ea, oa, eb, ob, ec, oc, ed, od;
+      merge_codes(A[wd], RA[wd], ea, oa);
+      merge_codes(Bw[wd], RB[wd], eb, ob);
+      merge_codes(C[wd], RC[wd], ec, oc);
+      merge_codes(Dw[wd], RD[wd], ed, od);
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const uint32_t sel = half ? 0x7632u : 0x5410u;
+        // bytes: [x.e(4half), x.e(4half+2), y.e(4half), y.e(4half+2)] for ev; odd elements for od
+        const uint32_t uab = prmt(ea, eb, sel), vab = prmt(oa, ob, sel);
+        const uint32_t ucd = prmt(ec, ed, sel), vcd = prmt(oc, od, sel);
+        // m-tile qd=0: dims e(4half+0) [row g] and e(4half+1) [row g+8]; qd=1: e(4half+2), e(4half+3)
+        const uint32_t ab0 = hadd2((uab & 0x00FF00FFu) | kMagic, kNeg1152);
+        const uint32_t ab1 = hadd2((vab & 0x00FF00FFu) | kMagic, kNeg1152);
+        const uint32_t ab2 = hadd2(prmt(uab, kMagic, 0x5341), kNeg1152);
+        const uint32_t ab3 = hadd2(prmt(vab, kMagic, 0x5341), kNeg1152);
+        const uint32_t cd0 = hadd2((ucd & 0x00FF00FFu) | kMagic, kNeg1152);
+        const uint32_t cd1 = hadd2((vcd & 0x00FF00FFu) | kMagic, kNeg1152);
+        const uint32_t cd2 = hadd2(prmt(ucd, kMagic, 0x5341), kNeg1152);
+        const uint32_t cd3 = hadd2(prmt(vcd, kMagic, 0x5341), kNeg1152);
+        const int mt = wd * 4 + half * 2;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          mma16816(w.o[nt][mt], ab0, ab1, cd0, cd1, pb[nt][0], pb[nt][1]);
+          mma16816(w.o[nt][mt + 1], ab2, ab3, cd2, cd3, pb[nt][0], pb[nt][1]);
+        }
+      }
+    }
+  }
+}
+
+template <bool FULL, int NT, int TW, int CG, int NSTAGE>
+struct Cfg {
+  static constexpr int kST = TW * 16;                       // tokens per stage
+  static constexpr int kSubBytes = FULL ? 16 * 272 : 16 * 144;
+  static constexpr int kStageBytes = kST * (FULL ? 272 : 144);
+  static constexpr int kConsWarps = TW * CG;
+  static constexpr int kThreads = (kConsWarps + 1) * 32;
+  static constexpr int kColsPad = CG * NT * 8;
+  static constexpr int kRing = NSTAGE * kStageBytes;
+  static constexpr int kMergeBytes = kConsWarps * NT * 8 * kPartStride * 4;
+  static constexpr int kRingAlloc = kRing > kMergeBytes ? kRing : kMergeBytes;
+  static constexpr int kQBytes = kColsPad * LYNX_D * 2;
+  static constexpr int kBlkBytes = (kMaxChunkTokens / 16) * 4;
+  static constexpr int kBarBytes = 2 * NSTAGE * 8;
+  static constexpr int kMiscBytes = 64;
+  static constexpr int kSmem = kRingAlloc + kQBytes + kBlkBytes + kBarBytes + kMiscBytes;
+};
+
+template <bool FULL, int NT, int TW, int CG, int NSTAGE>
+__global__ void __launch_bounds__((TW * CG + 1) * 32)
+attn_kernel(const AttnParams p) {
+  using C = Cfg<FULL, NT, TW, CG, NSTAGE>;
+  constexpr int ST = C::kST;
+  extern __shared__ __align__(128) unsigned char smem[];
+  unsigned char* ring = smem;
+  __nv_bfloat16* q_s = reinterpret_cast<__nv_bfloat16*>(smem + C::kRingAlloc);
+  uint32_t* blk_s = reinterpret_cast<uint32_t*>(smem + C::kRingAlloc + C::kQBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kRingAlloc + C::kQBytes + C::kBlkBytes);
+  int* misc = reinterpret_cast<int*>(smem + C::kRingAlloc + C::kQBytes + C::kBlkBytes + C::kBarBytes);
+  // misc[0] = abort word, misc[1] = max |q| bits, misc[2] = "this CTA is last" flag, misc[4..] dev
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int chunk = blockIdx.x, hkv = blockIdx.y, b = blockIdx.z;
+  const int cap = p.max_blocks * p.bt;
+  int len = p.seq_lens[b];
+  len = len < 0 ? 0 : (len > cap ? cap : len);
+  const int nchunks = len > 0 ? (len + p.chunk_tokens - 1) / p.chunk_tokens : 1;
+  if (chunk >= nchunks) return;
+  const int t_begin = chunk * p.chunk_tokens;
+  const int t_end = min(len, t_begin + p.chunk_tokens);
+  const int n_sub = (t_end - t_begin + 15) >> 4;
+  const int n_stage = (n_sub + TW - 1) / TW;
+  const uint32_t ring_u32 = smem_u32(ring);
+  const uint32_t full0 = smem_u32(bars), empty0 = full0 + NSTAGE * 8;
+  volatile int* abort_word = misc;
+
+  if (tid == 0) {
+    for (int i = 0; i < NSTAGE; ++i) {
+      mbar_init(full0 + i * 8, 1);
+      mbar_init(empty0 + i * 8, C::kConsWarps);
+    }
+    misc[0] = 0; misc[1] = 0; misc[2] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  WarpState<FULL, NT> w;
+  const int g = lane >> 2, t = lane & 3;
+  const int tw = warp % TW, cg = warp / TW;
+
+  if (warp == C::kConsWarps) {
+    // =============================== producer warp ===============================
+    for (int i = lane; i < n_sub; i += 32) {
+      const int t0 = t_begin + i * 16;
+      int blk = __ldg(p.block_table + (size_t)b * p.max_blocks + t0 / p.bt);
+      if (blk < 0 || blk >= p.num_blocks) {
+        atomicOr(p.ws_flags, kFlagBadBlock);
+        blk = blk < 0 ? 0 : p.num_blocks - 1;
+      }
+      blk_s[i] = (uint32_t)(((size_t)blk * p.Hkv + hkv) * p.bt + (t0 % p.bt));
+    }
+    __syncwarp();
+    constexpr int NARR = FULL ? 6 : 4;
+    int issued = 0;
+    for (int s = 0; s < n_stage; ++s) {
+      const int slot = s % NSTAGE;
+      if (s >= NSTAGE && !mbar_wait(empty0 + slot * 8, ((s / NSTAGE) - 1) & 1, abort_word)) break;
+      if (*abort_word) break;
+      const int nsub = min(TW, n_sub - s * TW);
+      const uint32_t bar = full0 + slot * 8;
+      if (lane == 0) mbar_expect_tx(bar, nsub * C::kSubBytes);
+      __syncwarp();
+      const uint32_t stage = ring_u32 + slot * C::kStageBytes;
+      for (int idx = lane; idx < nsub * NARR; idx += 32) {
+        const int sub = idx / NARR, arr = idx - sub * NARR;
+        const size_t row = blk_s[s * TW + sub];
+        switch (arr) {
+          case 0: bulk_g2s(stage + sub * 1024, p.ka + row * 64, 1024, bar); break;
+          case 1: bulk_g2s(stage + ST * 64 + sub * 1024, p.va + row * 64, 1024, bar); break;
+          case 2: bulk_g2s(stage + (FULL ? ST * 256 : ST * 128) + sub * 128, p.km + row * 2, 128, bar); break;
+          case 3: bulk_g2s(stage + (FULL ? ST * 264 : ST * 136) + sub * 128, p.vm + row * 2, 128, bar); break;
+          case 4: bulk_g2s(stage + ST * 128 + sub * 1024, p.kr + row * 64, 1024, bar); break;
+          default: bulk_g2s(stage + ST * 192 + sub * 1024, p.vr + row * 64, 1024, bar); break;
+        }
+      }
+      issued = s + 1;
+    }
+    if (*abort_word && lane == 0) {
+      // gave up: let the copies already issued land before the CTA's memory is reused
+      atomicOr(p.ws_flags, kFlagTimeout);
+      const uint64_t t0 = globaltimer_ns();
+      for (int s = max(0, issued - NSTAGE); s < issued; ++s)
+        while (!mbar_try_wait(full0 + (s % NSTAGE) * 8, (s / NSTAGE) & 1) &&
+               globaltimer_ns() - t0 < 1000000000ull) {}
+    }
+  } else {
+    // =============================== consumer warps ==============================
+    // stage Q of this (sequence, KV head): columns c = j*G + hh
+    constexpr int kConsThreads = C::kConsWarps * 32;
+    {
+      float amax = 0.0f;
+      for (int i = tid; i < C::kColsPad * (LYNX_D / 8); i += kConsThreads) {
+        const int c = i / (LYNX_D / 8), part = i % (LYNX_D / 8);
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (c < p.ncols) {
+          const int j = c / p.G, hh = c % p.G;
+          const size_t qrow = ((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh;
+          v = __ldg(reinterpret_cast<const uint4*>(p.q + qrow * LYNX_D) + part);
+        }
+        reinterpret_cast<uint4*>(q_s)[i] = v;
+        const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          amax = fmaxf(amax, fabsf(__uint_as_float(ww[k] << 16)));
+          amax = fmaxf(amax, fabsf(__uint_as_float(ww[k] & 0xFFFF0000u)));
+        }
+      }
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, off));
+      if (lane == 0) atomicMax(misc + 1, __float_as_int(amax));
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsThreads) : "memory");
+    // power-of-two prescale so that max|q| lands in [2^14, 2^15): FP16 then holds every BF16
+    // query value that is within 2^-29 of the largest one exactly
+    const float qmax = __int_as_float(misc[1]);
+    int e = 0;
+    if (qmax > 0.0f && qmax < INFINITY) e = 14 - (((__float_as_int(qmax) >> 23) & 0xFF) - 127);
+    e = max(-100, min(100, e));
+    const float up = __int_as_float((127 + e) << 23), down = __int_as_float((127 - e) << 23);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const int c = (cg * NT + nt) * 8 + g;  // column of this thread's B-fragment rows
+      const __nv_bfloat16* qc = q_s + c * LYNX_D;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const int base = 32 * t + 8 * (ks >> 1), h = ks & 1;
+        int d0, d1, d2, d3;
+        if (!FULL) { d0 = base + 2 * h; d1 = d0 + 4; d2 = d0 + 1; d3 = d0 + 5; }
+        else       { d0 = base + 4 * h; d1 = d0 + 2; d2 = d0 + 1; d3 = d0 + 3; }
+        w.qf[nt][ks][0] = pack_f16x2(__bfloat162float(qc[d0]) * up, __bfloat162float(qc[d1]) * up);
+        w.qf[nt][ks][1] = pack_f16x2(__bfloat162float(qc[d2]) * up, __bfloat162float(qc[d3]) * up);
+      }
+#pragma unroll
+      for (int cc = 0; cc < 2; ++cc) {
+        const int col = (cg * NT + nt) * 8 + 2 * t + cc;  // column of this thread's C-fragment
+        const __nv_bfloat16* qq = q_s + col * LYNX_D;
+        float sum = 0.0f;
+        for (int d = 0; d < LYNX_D; ++d) sum += __bfloat162float(qq[d]);
+        w.qs[nt][cc] = sum;
+        const int j = col / p.G;
+        w.lim[nt][cc] = col < p.ncols ? (p.causal ? len - p.nq + j + 1 : len) : 0;
+        w.m[nt][cc] = -1.0e30f;
+        w.l[nt][cc] = 0.0f;
+        w.zs[nt][cc] = 0.0f;
+      }
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) w.o[nt][mt][i] = 0.0f;
+    }
+    const float ca = p.sm_log2 * down * (FULL ? 1.0f : 16.0f);  // per level unit of the K dot
+    const float cb = p.sm_log2;
+    const int full_lim = p.causal ? len - p.nq + 1 : len;  // tokens below this are visible to all
+
+    for (int s = 0; s < n_stage; ++s) {
+      const int slot = s % NSTAGE;
+      if (!mbar_wait(full0 + slot * 8, (s / NSTAGE) & 1, abort_word)) break;
+      const int tile_t0 = t_begin + (s * TW + tw) * 16;
+      if (tile_t0 < t_end)
+        process_tile<FULL, NT, ST>(w, ring_u32 + slot * C::kStageBytes, tw, tile_t0,
+                                   tile_t0 + 16 > full_lim, ca, cb, g, t);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + slot * 8);
+    }
+  }
+
+  __syncthreads();  // ring is free from here on: reuse it for the CTA-level merge
+  if (tid == 0 && misc[0]) atomicOr(p.ws_flags, kFlagTimeout);
+  float* mbuf = reinterpret_cast<float*>(ring);
+  if (warp < C::kConsWarps) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+      for (int cc = 0; cc < 2; ++cc) {
+        float l = w.l[nt][cc], z = w.zs[nt][cc];
+#pragma unroll
+        for (int off = 4; off <= 16; off <<= 1) {
+          l += __shfl_xor_sync(0xFFFFFFFFu, l, off);
+          z += __shfl_xor_sync(0xFFFFFFFFu, z, off);
+        }
+        float* dst = mbuf + ((size_t)warp * NT * 8 + nt * 8 + 2 * t + cc) * kPartStride;
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          const int d = 16 * g + 8 * (mt >> 2) + 2 * (mt & 3);
+          dst[d] = w.o[nt][mt][cc] + z;
+          dst[d + 1] = w.o[nt][mt][cc + 2] + z;
+        }
+        if (g == 0) { dst[128] = w.m[nt][cc]; dst[129] = l; }
+      }
+    }
+  }
+  __syncthreads();
+
+  // merge the TW token warps of each column; write the result or a chunk partial
+  const size_t bh = (size_t)b * p.Hkv + hkv;
+  float* part = p.ws_part + (bh * p.max_chunks + chunk) * (size_t)C::kColsPad * kPartStride;
+  for (int idx = tid; idx < C::kColsPad * LYNX_D; idx += C::kThreads) {
+    const int c = idx >> 7, d = idx & 127;
+    if (c >= p.ncols) continue;
+    const int cgi = c / (NT * 8), cl = c % (NT * 8);
+    float M = -INFINITY;
+#pragma unroll
+    for (int x = 0; x < TW; ++x)
+      M = fmaxf(M, mbuf[((size_t)(cgi * TW + x) * NT * 8 + cl) * kPartStride + 128]);
+    float acc = 0.0f, L = 0.0f;
+#pragma unroll
+    for (int x = 0; x < TW; ++x) {
+      const float* src = mbuf + ((size_t)(cgi * TW + x) * NT * 8 + cl) * kPartStride;
+      const float f = ex2(src[128] - M);
+      acc = fmaf(src[d], f, acc);
+      L = fmaf(src[129], f, L);
+    }
+    if (nchunks == 1) {
+      const int j = c / p.G, hh = c % p.G;
+      p.out[(((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
+    } else {
+      part[(size_t)c * kPartStride + d] = acc;
+      if (d == 0) { part[(size_t)c * kPartStride + 128] = M; part[(size_t)c * kPartStride + 129] = L; }
+    }
+  }
+
+  // split-K: the last CTA of this (sequence, KV head) to finish merges the chunk partials
+  if (nchunks > 1) {
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) misc[2] = (atomicInc(p.ws_chunk_ctr + bh, (uint32_t)nchunks - 1) == (uint32_t)nchunks - 1);
+    __syncthreads();
+    if (!misc[2]) return;
+    __threadfence();
+    const float* base = p.ws_part + bh * p.max_chunks * (size_t)C::kColsPad * kPartStride;
+    for (int idx = tid; idx < C::kColsPad * LYNX_D; idx += C::kThreads) {
+      const int c = idx >> 7, d = idx & 127;
+      if (c >= p.ncols) continue;
+      const float* col = base + (size_t)c * kPartStride;
+      const size_t cstride = (size_t)C::kColsPad * kPartStride;
+      float M = -INFINITY;
+      for (int i = 0; i < nchunks; ++i) M = fmaxf(M, __ldcg(col + i * cstride + 128));
+      float acc = 0.0f, L = 0.0f;
+      for (int i = 0; i < nchunks; ++i) {
+        const float f = ex2(__ldcg(col + i * cstride + 128) - M);
+        acc = fmaf(__ldcg(col + i * cstride + d), f, acc);
+        L = fmaf(__ldcg(col + i * cstride + 129), f, L);
+      }
+      const int j = c / p.G, hh = c % p.G;
+      p.out[(((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
+    }
+  }
+
+  // accept / reject (Section 4.3): only the CTA that wrote the final outputs gets here
+  if (FULL && p.draft != nullptr) {
+    __syncthreads();  // this CTA's out values are visible to all its threads
+    int* devs = misc + 4;
+    if (tid < kMaxQ) devs[tid] = 0;
+    __syncthreads();
+    for (int idx = tid; idx < p.ncols * LYNX_D; idx += C::kThreads) {
+      const int c = idx >> 7, d = idx & 127;
+      const int j = c / p.G, hh = c % p.G;
+      const size_t o = (((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh) * LYNX_D + d;
+      const float f = p.out[o], dr = __ldg(p.draft + o);
+      const float r = fabsf(f - dr) / (p.atol + p.rtol * fabsf(f));
+      atomicMax(devs + j, __float_as_int(r));  // r >= 0: integer order = float order
+    }
+    __syncthreads();
+    if (tid < p.nq) p.ws_dev[bh * kMaxQ + tid] = __int_as_float(devs[tid]);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) misc[2] = (atomicInc(p.ws_seq_ctr + b, (uint32_t)p.Hkv - 1) == (uint32_t)p.Hkv - 1);
+    __syncthreads();
+    if (!misc[2]) return;
+    __threadfence();
+    if (tid == 0) {
+      int fr = p.nq;
+      for (int j = p.nq - 1; j >= 0; --j) {
+        float worst = 0.0f;
+        for (int h = 0; h < p.Hkv; ++h)
+          worst = fmaxf(worst, __ldcg(p.ws_dev + ((size_t)b * p.Hkv + h) * kMaxQ + j));
+        p.dev[(size_t)b * p.nq + j] = worst;
+        if (worst > 1.0f) fr = j;
+      }
+      p.first_reject[b] = fr;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ host side
+struct Plan {
+  int ncols, variant;  // variant: 0: NT1 TW4 CG1; 1: NT2 TW4 CG1; 2: NT2 TW4 CG2; 3: NT2 TW2 CG4
+  int cols_pad, chunk_tokens, max_chunks;
+  size_t off_chunk_ctr, off_seq_ctr, off_dev, off_part, bytes;
+};
+
+bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
+  if (!s || s->head_dim != LYNX_D || s->num_kv_heads <= 0 || s->num_q_heads <= 0 ||
+      s->num_q_heads % s->num_kv_heads != 0 || s->block_tokens <= 0 || s->block_tokens % 16 != 0 ||
+      s->num_blocks <= 0 || s->max_blocks_per_seq <= 0 || B <= 0 || nq <= 0 || nq > kMaxQ)
+    return false;
+  if (B > 65535 || s->num_kv_heads > 65535) return false;
+  const int G = s->num_q_heads / s->num_kv_heads;
+  const int ncols = nq * G;
+  if (ncols > kMaxCols) return false;
+  const int64_t cap = (int64_t)s->max_blocks_per_seq * s->block_tokens;
+  if (cap >= (1ll << 31)) return false;
+  if ((int64_t)s->num_blocks * s->num_kv_heads * s->block_tokens >= (1ll << 32)) return false;
+  pl->ncols = ncols;
+  pl->variant = ncols <= 8 ? 0 : ncols <= 16 ? 1 : ncols <= 32 ? 2 : 3;
+  pl->cols_pad = ncols <= 8 ? 8 : ncols <= 16 ? 16 : ncols <= 32 ? 32 : 64;
+  // chunk: the largest of {4096 .. 256} that still leaves >= 6 CTAs per resident slot
+  const int64_t slots = (int64_t)sm_count() * 2;
+  int chunk = 256;
+  for (int c = 4096; c >= 256; c >>= 1) {
+    const int64_t items = (int64_t)B * s->num_kv_heads * ((cap + c - 1) / c);
+    if (items >= slots * 6) { chunk = c; break; }
+  }
+  pl->chunk_tokens = chunk;
+  pl->max_chunks = (int)((cap + chunk - 1) / chunk);
+  size_t off = kWsHeaderBytes;
+  pl->off_chunk_ctr = off; off += (size_t)B * s->num_kv_heads * 4;
+  pl->off_seq_ctr = off;   off += (size_t)B * 4;
+  off = (off + 255) & ~(size_t)255;
+  pl->off_dev = off;       off += (size_t)B * s->num_kv_heads * kMaxQ * 4;
+  off = (off + 255) & ~(size_t)255;
+  pl->off_part = off;
+  off += (size_t)B * s->num_kv_heads * pl->max_chunks * pl->cols_pad * kPartStride * 4;
+  pl->bytes = off;
+  return true;
+}
+
+template <bool FULL, int NT, int TW, int CG, int NSTAGE>
+lynx_status launch(const AttnParams& p, cudaStream_t st) {
+  using C = Cfg<FULL, NT, TW, CG, NSTAGE>;
+  static_assert(C::kSmem <= 227 * 1024, "shared memory budget");
+  auto kern = attn_kernel<FULL, NT, TW, CG, NSTAGE>;
+  static bool configured[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmem) != cudaSuccess)
+      return LYNX_ERR_CUDA;
+    configured[dev] = true;
+  }
+  dim3 grid(p.max_chunks, p.Hkv, p.B);
+  kern<<<grid, C::kThreads, C::kSmem, st>>>(p);
+  return launch_status();
+}
+
+lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int B, int nq, int causal,
+                          lynx_plane K, lynx_plane V, const int32_t* block_table,
+                          const int32_t* seq_lens, float softmax_scale, const float* draft,
+                          float atol, float rtol, float* out, int32_t* first_reject, float* dev,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+  if (B == 0) return LYNX_OK;
+  if (!shape) return LYNX_ERR_NULL;
+  if (B < 0 || nq <= 0) return LYNX_ERR_SHAPE;
+  if (shape->head_dim != LYNX_D || shape->block_tokens <= 0 || shape->block_tokens % 16 != 0)
+    return LYNX_ERR_UNSUPPORTED;
+  Plan pl;
+  if (!make_plan(shape, B, nq, &pl)) return LYNX_ERR_UNSUPPORTED;
+  if (!q || !K.anchor || !K.meta || !V.anchor || !V.meta || !block_table || !seq_lens || !out || !workspace)
+    return LYNX_ERR_NULL;
+  if (full && (!K.residual || !V.residual)) return LYNX_ERR_NULL;
+  if (full && draft && (!first_reject || !dev)) return LYNX_ERR_NULL;
+  if (!aligned16(q) || !aligned16(K.anchor) || !aligned16(V.anchor) || !aligned16(K.meta) ||
+      !aligned16(V.meta) || !aligned16(workspace) || (full && (!aligned16(K.residual) || !aligned16(V.residual))))
+    return LYNX_ERR_ALIGN;
+  if (workspace_bytes < pl.bytes) return LYNX_ERR_WORKSPACE;
+  if (full && draft && !(atol >= 0.0f && rtol >= 0.0f && atol + rtol > 0.0f)) return LYNX_ERR_SHAPE;
+
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  AttnParams p;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.ka = K.anchor; p.kr = K.residual; p.km = K.meta;
+  p.va = V.anchor; p.vr = V.residual; p.vm = V.meta;
+  p.block_table = block_table; p.seq_lens = seq_lens;
+  p.out = out; p.draft = full ? draft : nullptr; p.first_reject = first_reject; p.dev = dev;
+  p.ws_flags = reinterpret_cast<uint32_t*>(ws);
+  p.ws_chunk_ctr = reinterpret_cast<uint32_t*>(ws + pl.off_chunk_ctr);
+  p.ws_seq_ctr = reinterpret_cast<uint32_t*>(ws + pl.off_seq_ctr);
+  p.ws_dev = reinterpret_cast<float*>(ws + pl.off_dev);
+  p.ws_part = reinterpret_cast<float*>(ws + pl.off_part);
+  p.atol = atol; p.rtol = rtol;
+  const float sc = softmax_scale == 0.0f ? 0.08838834764831845f : softmax_scale;
+  p.sm_log2 = sc * 1.4426950408889634f;
+  p.B = B; p.nq = nq; p.causal = causal ? 1 : 0;
+  p.Hq = shape->num_q_heads; p.Hkv = shape->num_kv_heads; p.G = p.Hq / p.Hkv;
+  p.bt = shape->block_tokens; p.num_blocks = shape->num_blocks; p.max_blocks = shape->max_blocks_per_seq;
+  p.chunk_tokens = pl.chunk_tokens; p.max_chunks = pl.max_chunks; p.ncols = pl.ncols;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!full) {
+    switch (pl.variant) {
+      case 0: return launch<false, 1, 4, 1, 8>(p, st);
+      case 1: return launch<false, 2, 4, 1, 8>(p, st);
+      case 2: return launch<false, 2, 4, 2, 8>(p, st);
+      default: return launch<false, 2, 2, 4, 16>(p, st);
+    }
+  }
+  switch (pl.variant) {
+    case 0: return launch<true, 1, 4, 1, 5>(p, st);
+    case 1: return launch<true, 2, 4, 1, 5>(p, st);
+    case 2: return launch<true, 2, 4, 2, 5>(p, st);
+    default: return launch<true, 2, 2, 4, 8>(p, st);
+  }
+}
+
+}  // namespace
+}  // namespace lynx
+
+extern "C" size_t lynx_workspace_bytes(const lynx_shape* shape, int32_t batch, int32_t n_cols_q) {
+  lynx::Plan pl;
+  if (!lynx::make_plan(shape, batch, n_cols_q, &pl)) return 0;
+  return pl.bytes;
+}
+
+extern "C" lynx_status lynx_anchor_attention(const lynx_shape* shape, const void* q_bf16, int32_t batch,
+                                             int32_t n_q, int32_t causal, lynx_plane K, lynx_plane V,
+                                             const int32_t* block_table, const int32_t* seq_lens,
+                                             float softmax_scale, float* out, void* workspace,
+                                             size_t workspace_bytes, void* stream) {
+  return lynx::run_attention(false, shape, q_bf16, batch, n_q, causal, K, V, block_table, seq_lens,
+                             softmax_scale, nullptr, 0.f, 0.f, out, nullptr, nullptr, workspace,
+                             workspace_bytes, stream);
+}
+
+extern "C" lynx_status lynx_merge_verify_attention(const lynx_shape* shape, const void* q_bf16,
+                                                   int32_t batch, int32_t k, int32_t causal,
+                                                   lynx_plane K, lynx_plane V,
+                                                   const int32_t* block_table, const int32_t* seq_lens,
+                                                   float softmax_scale, const float* draft_out,
+                                                   float atol, float rtol, float* out_full,
+                                                   int32_t* first_reject, float* dev, void* workspace,
+                                                   size_t workspace_bytes, void* stream) {
+  return lynx::run_attention(true, shape, q_bf16, batch, k, causal, K, V, block_table, seq_lens,
+                             softmax_scale, draft_out, atol, rtol, out_full, first_reject, dev,
+                             workspace, workspace_bytes, stream);
+}

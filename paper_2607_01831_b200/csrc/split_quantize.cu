@@ -1,0 +1,201 @@
+// lynx_split_quantize and lynx_recombine: streaming codec kernels (HBM-bound).
+//
+// Split-quantise follows the linear grouped quantiser of Section 2.3 (one group = one token's
+// 128-element head vector), the MSB/LSB split of Section 4.1 stage 4 and the two-nibbles-per-
+// byte, one-contiguous-buffer-per-stream packing of the Compression Kernel paragraph.
+// Recombine is the Residual-phase refinement to Q_full of Section 4.2.
+//
+// Mapping: a row is 256 B of BF16 = 16 lanes x 16 B, so a half-warp owns a row: one 128-bit
+// streaming load per lane, min/max by 4 xor-shuffles, 8 codes per lane, 4 B of each plane per
+// lane (a warp writes 128 contiguous bytes per plane).  Several rows are in flight per lane.
+#include <cuda_bf16.h>
+
+#include "lynx_common.cuh"
+
+namespace lynx {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kRowsInFlight = 4;  // rows per half-warp per loop trip
+
+// Round-half-even of the exact product u*inv, as the low byte of an FP32 whose ulp is 1:
+// fma(u, inv, 1.5 * 2^23) rounds the exact sum once, to an integer, ties to even.
+__device__ __forceinline__ uint32_t code_bits(float x, float mn, float inv) {
+  return __float_as_uint(__fmaf_rn(__fsub_rn(x, mn), inv, 12582912.0f));
+}
+
+template <bool kIds>
+__global__ void __launch_bounds__(kThreads)
+split_quantize_kernel(const uint4* __restrict__ src, int64_t n_logical_rows,
+                      const int32_t* __restrict__ block_ids, uint32_t rows_per_block,
+                      int64_t n_blocks_total, uint32_t* __restrict__ anchor,
+                      uint32_t* __restrict__ residual, float2* __restrict__ meta) {
+  const int lane16 = threadIdx.x & 15;
+  const int64_t hw = (int64_t)blockIdx.x * (kThreads / 16) + (threadIdx.x >> 4);
+  const int64_t hw_total = (int64_t)gridDim.x * (kThreads / 16);
+
+  for (int64_t r0 = hw * kRowsInFlight; r0 < n_logical_rows; r0 += hw_total * kRowsInFlight) {
+    uint4 raw[kRowsInFlight];
+    int64_t row[kRowsInFlight];
+#pragma unroll
+    for (int u = 0; u < kRowsInFlight; ++u) {
+      int64_t lr = r0 + u;
+      row[u] = -1;
+      if (lr < n_logical_rows) {
+        if (kIds) {
+          uint32_t lb = (uint32_t)lr / rows_per_block;
+          uint32_t in = (uint32_t)lr - lb * rows_per_block;
+          int32_t blk = __ldg(block_ids + lb);
+          if (blk >= 0 && blk < n_blocks_total) row[u] = (int64_t)blk * rows_per_block + in;
+        } else {
+          row[u] = lr;
+        }
+      }
+      raw[u] = make_uint4(0, 0, 0, 0);
+      if (row[u] >= 0) raw[u] = __ldcs(src + row[u] * 16 + lane16);
+    }
+#pragma unroll
+    for (int u = 0; u < kRowsInFlight; ++u) {
+      // the shuffles below are executed by every lane of the warp, valid row or not
+      float f[8];
+      const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        f[2 * i] = __uint_as_float(w[i] << 16);
+        f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+      }
+      float mn = fminf(fminf(fminf(f[0], f[1]), fminf(f[2], f[3])),
+                       fminf(fminf(f[4], f[5]), fminf(f[6], f[7])));
+      float mx = fmaxf(fmaxf(fmaxf(f[0], f[1]), fmaxf(f[2], f[3])),
+                       fmaxf(fmaxf(f[4], f[5]), fmaxf(f[6], f[7])));
+#pragma unroll
+      for (int off = 8; off >= 1; off >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+      }
+      const float range = __fsub_rn(mx, mn);
+      const bool live = range >= 0x1p-100f;
+      const float scale = live ? __fdiv_rn(range, 255.0f) : 0.0f;
+      const float inv = live ? __fdiv_rn(255.0f, range) : 0.0f;
+      const float zero = __fadd_rn(mn, 0.0f);  // -0 -> +0
+
+      uint32_t c[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) c[i] = code_bits(f[i], mn, inv);
+      // gather the low bytes: w0 = codes 0..3, w1 = codes 4..7
+      const uint32_t w0 = __byte_perm(__byte_perm(c[0], c[1], 0x0040), __byte_perm(c[2], c[3], 0x0040), 0x5410);
+      const uint32_t w1 = __byte_perm(__byte_perm(c[4], c[5], 0x0040), __byte_perm(c[6], c[7], 0x0040), 0x5410);
+      // nibble planes: bytes 0 and 2 of (x | x >> 4) hold two packed nibbles each
+      const uint32_t h0 = (w0 >> 4) & 0x0F0F0F0Fu, h1 = (w1 >> 4) & 0x0F0F0F0Fu;
+      const uint32_t l0 = w0 & 0x0F0F0F0Fu, l1 = w1 & 0x0F0F0F0Fu;
+      const uint32_t a = __byte_perm(h0 | (h0 >> 4), h1 | (h1 >> 4), 0x6420);
+      const uint32_t r = __byte_perm(l0 | (l0 >> 4), l1 | (l1 >> 4), 0x6420);
+      if (row[u] >= 0) {
+        __stcs(anchor + row[u] * 16 + lane16, a);
+        __stcs(residual + row[u] * 16 + lane16, r);
+        if (lane16 == 0) __stcs(meta + row[u], make_float2(scale, zero));
+      }
+    }
+  }
+}
+
+template <bool kCodes, bool kBf16>
+__global__ void __launch_bounds__(kThreads)
+recombine_kernel(const uint32_t* __restrict__ anchor, const uint32_t* __restrict__ residual,
+                 const float2* __restrict__ meta, int64_t n_rows, uint2* __restrict__ codes,
+                 uint4* __restrict__ deq) {
+  const int64_t n_items = n_rows * 16;  // 16 lanes per row, 8 elements per lane
+  const int64_t stride = (int64_t)gridDim.x * kThreads;
+  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n_items; i += stride) {
+    const uint32_t xa = __ldcs(anchor + i), xr = __ldcs(residual + i);
+    // even elements: (a << 4) | r from the low nibbles; odd elements from the high nibbles
+    const uint32_t ev = ((xa << 4) & 0xF0F0F0F0u) | (xr & 0x0F0F0F0Fu);
+    const uint32_t od = (xa & 0xF0F0F0F0u) | ((xr >> 4) & 0x0F0F0F0Fu);
+    const uint32_t c0 = __byte_perm(ev, od, 0x5140);  // elements 0..3
+    const uint32_t c1 = __byte_perm(ev, od, 0x7362);  // elements 4..7
+    if (kCodes) __stcs(codes + i, make_uint2(c0, c1));
+    if (kBf16) {
+      const float2 m = __ldg(meta + (i >> 4));
+      uint32_t o[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t cw = j < 2 ? c0 : c1;
+        const float lo = __fmaf_rn((float)((cw >> ((j & 1) * 16)) & 0xFFu), m.x, m.y);
+        const float hi = __fmaf_rn((float)((cw >> ((j & 1) * 16 + 8)) & 0xFFu), m.x, m.y);
+        const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+        o[j] = *reinterpret_cast<const uint32_t*>(&p);
+      }
+      __stcs(deq + i, make_uint4(o[0], o[1], o[2], o[3]));
+    }
+  }
+}
+
+int grid_for(int64_t items_per_block_unit, int blocks_per_sm) {
+  int64_t cap = (int64_t)sm_count() * blocks_per_sm;
+  int64_t g = items_per_block_unit < cap ? items_per_block_unit : cap;
+  return (int)(g < 1 ? 1 : g);
+}
+
+}  // namespace
+}  // namespace lynx
+
+extern "C" lynx_status lynx_split_quantize(const void* src_bf16, int64_t n_rows,
+                                           const int32_t* block_ids, int32_t n_block_ids,
+                                           int32_t rows_per_block, uint8_t* anchor,
+                                           uint8_t* residual, float* meta, void* stream) {
+  using namespace lynx;
+  if (n_rows < 0) return LYNX_ERR_SHAPE;
+  if (n_rows == 0) return LYNX_OK;
+  if (!src_bf16 || !anchor || !residual || !meta) return LYNX_ERR_NULL;
+  if (!aligned16(src_bf16) || !aligned16(anchor) || !aligned16(residual) ||
+      (reinterpret_cast<uintptr_t>(meta) & 7u))
+    return LYNX_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int rows_per_cta_trip = (kThreads / 16) * kRowsInFlight;
+  if (block_ids) {
+    if (n_block_ids < 0 || rows_per_block <= 0 || n_rows % rows_per_block != 0) return LYNX_ERR_SHAPE;
+    if (n_block_ids == 0) return LYNX_OK;
+    const int64_t logical = (int64_t)n_block_ids * rows_per_block;
+    if (logical >= (1ll << 31)) return LYNX_ERR_UNSUPPORTED;
+    const int grid = grid_for((logical + rows_per_cta_trip - 1) / rows_per_cta_trip, 8);
+    split_quantize_kernel<true><<<grid, kThreads, 0, st>>>(
+        static_cast<const uint4*>(src_bf16), logical, block_ids, (uint32_t)rows_per_block,
+        n_rows / rows_per_block, reinterpret_cast<uint32_t*>(anchor),
+        reinterpret_cast<uint32_t*>(residual), reinterpret_cast<float2*>(meta));
+  } else {
+    const int grid = grid_for((n_rows + rows_per_cta_trip - 1) / rows_per_cta_trip, 8);
+    split_quantize_kernel<false><<<grid, kThreads, 0, st>>>(
+        static_cast<const uint4*>(src_bf16), n_rows, nullptr, 1u, n_rows,
+        reinterpret_cast<uint32_t*>(anchor), reinterpret_cast<uint32_t*>(residual),
+        reinterpret_cast<float2*>(meta));
+  }
+  return launch_status();
+}
+
+extern "C" lynx_status lynx_recombine(const uint8_t* anchor, const uint8_t* residual,
+                                      const float* meta, int64_t n_rows, uint8_t* codes_u8,
+                                      void* dequant_bf16, void* stream) {
+  using namespace lynx;
+  if (n_rows < 0) return LYNX_ERR_SHAPE;
+  if (n_rows == 0) return LYNX_OK;
+  if (!anchor || !residual || (!codes_u8 && !dequant_bf16)) return LYNX_ERR_NULL;
+  if (dequant_bf16 && !meta) return LYNX_ERR_NULL;
+  if (!aligned16(anchor) || !aligned16(residual) || !aligned16(codes_u8) ||
+      !aligned16(dequant_bf16) || (reinterpret_cast<uintptr_t>(meta) & 7u))
+    return LYNX_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int grid = grid_for((n_rows * 16 + kThreads - 1) / kThreads, 8);
+  const uint32_t* a = reinterpret_cast<const uint32_t*>(anchor);
+  const uint32_t* r = reinterpret_cast<const uint32_t*>(residual);
+  const float2* m = reinterpret_cast<const float2*>(meta);
+  uint2* c = reinterpret_cast<uint2*>(codes_u8);
+  uint4* d = static_cast<uint4*>(dequant_bf16);
+  if (codes_u8 && dequant_bf16)
+    recombine_kernel<true, true><<<grid, kThreads, 0, st>>>(a, r, m, n_rows, c, d);
+  else if (codes_u8)
+    recombine_kernel<true, false><<<grid, kThreads, 0, st>>>(a, r, m, n_rows, c, d);
+  else
+    recombine_kernel<false, true><<<grid, kThreads, 0, st>>>(a, r, m, n_rows, c, d);
+  return launch_status();
+}

@@ -1,0 +1,284 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element.
+
+Codes, planes, metadata bits and accept/reject indices must match bit-exactly; attention
+outputs within |gpu - ref| <= 2e-3 + 1e-2 |ref| against the float64 oracle.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from util import bf16_bits, f32_to_bf16_tensor
+
+pytestmark = pytest.mark.gpu
+
+ATOL, RTOL = 2e-3, 1e-2
+
+
+@pytest.fixture(scope="module")
+def lynx():
+    import paper_2607_01831_b200 as m
+    m.load()
+    return m
+
+
+def _planes_np(p):
+    return (p.anchor.cpu().numpy(), None if p.residual is None else p.residual.cpu().numpy(),
+            p.meta.cpu().numpy())
+
+
+def _assert_planes_equal(got, want):
+    ga, gr, gm = got
+    wa, wr, wm = want
+    assert np.array_equal(ga, wa), "anchor plane differs"
+    assert np.array_equal(gr, wr), "residual plane differs"
+    assert np.array_equal(gm.view(np.uint32), wm.view(np.uint32)), "meta bits differ"
+
+
+# ------------------------------------------------------------------------- split-quantise
+@pytest.mark.parametrize("recipe", ["normal_outlier4x8", "lognormal_channels", "student_t4",
+                                    "normal_outlier2pct_x10"])
+@pytest.mark.parametrize("n_blocks", [1, 37, 300])
+def test_split_quantize_bit_exact(lynx, recipe, n_blocks):
+    x = synth.kv_block_values(recipe, n_blocks, 8, 16, "cpu", "sq", n_blocks)
+    x = x.reshape(-1, 128)[: x.numel() // 128 - 3]          # ragged tail: not a multiple of 64 rows
+    got = lynx.split_quantize(x.cuda())
+    torch.cuda.synchronize()
+    _assert_planes_equal(_planes_np(got), oracle.split_quantize(bf16_bits(x)))
+
+
+def test_split_quantize_special_rows(lynx):
+    rows = [
+        [0.0, 255.0] + [float(v) for v in range(1, 127)],
+        [0.0, 255.0] + [k + 0.5 for k in range(126)],          # ties -> even
+        [1.5] * 128,                                           # constant row
+        [-0.0] * 128,                                          # minus zero
+        [0.0] * 127 + [2.0 ** -120],                           # sub-threshold range
+        [-3.0 + 0.5 * i for i in range(128)],
+        [1.0e38] * 64 + [-1.0e38] * 64,                        # huge but finite range
+    ]
+    x = f32_to_bf16_tensor(np.array(rows, np.float32))
+    got = lynx.split_quantize(x.cuda())
+    torch.cuda.synchronize()
+    _assert_planes_equal(_planes_np(got), oracle.split_quantize(bf16_bits(x)))
+
+
+def test_split_quantize_block_ids_only_touch_listed_blocks(lynx):
+    nb, hkv, bt = 20, 4, 16
+    x = synth.kv_block_values("student_t4", nb, hkv, bt, "cpu", "ids", 1)
+    ids = torch.tensor([3, 17, 0, 9, 25, -1], dtype=torch.int32)     # 25 and -1 are skipped
+    out = lynx.alloc_planes((nb, hkv, bt), "cuda")
+    out.anchor.fill_(0xAB); out.residual.fill_(0xCD); out.meta.fill_(-7.0)
+    lynx.split_quantize(x.cuda(), out=out, block_ids=ids.cuda(), rows_per_block=hkv * bt)
+    torch.cuda.synchronize()
+    wa, wr, wm = oracle.split_quantize(bf16_bits(x))
+    ga, gr, gm = _planes_np(out)
+    listed = [3, 17, 0, 9]
+    for b in range(nb):
+        if b in listed:
+            assert np.array_equal(ga[b], wa[b]) and np.array_equal(gr[b], wr[b])
+            assert np.array_equal(gm[b].view(np.uint32), wm[b].view(np.uint32))
+        else:
+            assert np.all(ga[b] == 0xAB) and np.all(gr[b] == 0xCD) and np.all(gm[b] == -7.0)
+
+
+def test_split_quantize_empty_and_errors(lynx):
+    L = lynx.load()
+    assert L.lynx_split_quantize(None, 0, None, 0, 0, None, None, None, None) == 0
+    x = torch.zeros(4, 128, dtype=torch.bfloat16, device="cuda")
+    p = lynx.alloc_planes((4,), "cuda")
+    assert L.lynx_split_quantize(x.data_ptr(), 4, None, 0, 0, None, p.residual.data_ptr(),
+                                 p.meta.data_ptr(), None) == 1                      # NULL
+    assert L.lynx_split_quantize(x.data_ptr() + 2, 3, None, 0, 0, p.anchor.data_ptr(),
+                                 p.residual.data_ptr(), p.meta.data_ptr(), None) == 3  # alignment
+    assert L.lynx_split_quantize(x.data_ptr(), -1, None, 0, 0, p.anchor.data_ptr(),
+                                 p.residual.data_ptr(), p.meta.data_ptr(), None) == 2  # shape
+    assert L.lynx_status_string(3).decode().startswith("pointer")
+
+
+# ------------------------------------------------------------------------------ recombine
+def test_recombine_bit_exact(lynx):
+    x = synth.kv_block_values("lognormal_channels", 61, 8, 16, "cpu", "rc", 1).reshape(-1, 128)[:-5]
+    p = lynx.split_quantize(x.cuda())
+    codes, deq = lynx.recombine(p, want_codes=True, want_bf16=True)
+    codes_only, _ = lynx.recombine(p, want_codes=True, want_bf16=False)
+    _, deq_only = lynx.recombine(p, want_codes=False, want_bf16=True)
+    torch.cuda.synchronize()
+    wa, wr, wm, wcodes = oracle.split_quantize(bf16_bits(x), want_codes=True)
+    ocodes, odeq = oracle.recombine(wa, wr, wm)
+    assert np.array_equal(ocodes, wcodes)
+    assert np.array_equal(codes.cpu().numpy(), ocodes)
+    assert np.array_equal(codes_only.cpu().numpy(), ocodes)
+    assert np.array_equal(bf16_bits(deq), odeq)
+    assert np.array_equal(bf16_bits(deq_only), odeq)
+    # the identity the split is defined by
+    a = p.anchor.cpu().numpy(); r = p.residual.cpu().numpy()
+    lo = ((a & 15).astype(np.uint16) << 4) | (r & 15)
+    hi = ((a >> 4).astype(np.uint16) << 4) | (r >> 4)
+    assert np.array_equal(np.stack([lo, hi], -1).reshape(-1, 128), ocodes)
+
+
+# ------------------------------------------------------------------------------ attention
+def _case(lynx, seed, B, Hkv, G, n_q, lens, bt=16, shuffled=True, recipe="normal_outlier4x8"):
+    lens_t = torch.tensor(lens, dtype=torch.int32)
+    cap = [max(int(l), 1) for l in lens]
+    table, nb = synth.block_table(torch.tensor(cap, dtype=torch.int32), bt, shuffled, "gp", seed)
+    k = synth.kv_block_values(recipe, nb, Hkv, bt, "cpu", "gpK", seed)
+    v = synth.kv_block_values(recipe, nb, Hkv, bt, "cpu", "gpV", seed)
+    q = synth.queries(B, n_q, Hkv * G, "cpu", "gpQ", seed)
+    K = lynx.split_quantize(k.cuda())
+    V = lynx.split_quantize(v.cuda())
+    torch.cuda.synchronize()
+    kp, vp = oracle.split_quantize(bf16_bits(k)), oracle.split_quantize(bf16_bits(v))
+    _assert_planes_equal(_planes_np(K), kp)
+    geo = lynx.Geometry(Hkv * G, Hkv, bt, nb, table.shape[1])
+    ws = lynx.make_workspace(geo, B, n_q, "cuda")
+    return dict(geo=geo, ws=ws, q=q, K=K, V=V, kp=kp, vp=vp, table=table, lens=lens_t, Hkv=Hkv, bt=bt)
+
+
+def _close(got, ref, what):
+    err = np.abs(got - ref)
+    bound = ATOL + RTOL * np.abs(ref)
+    assert np.all(np.isfinite(got)), what + ": non-finite output"
+    worst = float(np.max(err / bound))
+    assert worst <= 1.0, f"{what}: worst error/bound {worst:.3f}, max abs err {err.max():.3e}"
+    return float(err.max())
+
+
+ATTN_CASES = [
+    # B, Hkv, G, n_q, lens, bt, shuffled, recipe
+    (1, 8, 4, 1, (4096,), 16, False, "normal_outlier4x8"),         # config-1 shape, several chunks
+    (2, 2, 4, 1, (1000, 37), 16, True, "lognormal_channels"),      # ragged, not multiples of 16
+    (3, 2, 8, 1, (1, 15, 17), 16, True, "student_t4"),             # tiny lengths, G = 8
+    (2, 1, 1, 1, (300, 0), 16, True, "normal"),                    # G = 1 and an empty sequence
+    (1, 2, 2, 3, (777,), 32, True, "normal_outlier2pct_x10"),      # 32-token blocks, n_q = 3
+    (1, 2, 4, 4, (2500,), 16, True, "student_t4"),                 # 16 columns
+    (1, 1, 4, 8, (1300,), 16, True, "lognormal_channels"),         # 32 columns
+    (1, 1, 8, 8, (900,), 64, True, "normal_outlier4x8"),           # 64 columns, 64-token blocks
+    (1, 1, 16, 1, (500,), 16, False, "normal"),                    # G = 16
+]
+
+
+@pytest.mark.parametrize("case", ATTN_CASES, ids=[str(i) for i in range(len(ATTN_CASES))])
+@pytest.mark.parametrize("causal", [False, True])
+def test_anchor_attention_matches_oracle(lynx, case, causal):
+    B, Hkv, G, n_q, lens, bt, shuffled, recipe = case
+    c = _case(lynx, 100 + len(lens) + n_q, B, Hkv, G, n_q, lens, bt, shuffled, recipe)
+    out = lynx.anchor_attention(c["geo"], c["q"].cuda(), c["K"], c["V"], c["table"].cuda(),
+                                c["lens"].cuda(), c["ws"], causal=causal)
+    lynx.check(c["ws"])
+    ref = oracle.attention(False, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                           c["lens"].numpy(), Hkv, bt, causal=causal)
+    _close(out.cpu().numpy().astype(np.float64), ref, "anchor attention")
+    # a second call on the same workspace gives the same bits (counters reset themselves)
+    out2 = lynx.anchor_attention(c["geo"], c["q"].cuda(), c["K"], c["V"], c["table"].cuda(),
+                                 c["lens"].cuda(), c["ws"], causal=causal)
+    lynx.check(c["ws"])
+    assert torch.equal(out, out2)
+
+
+@pytest.mark.parametrize("case", ATTN_CASES, ids=[str(i) for i in range(len(ATTN_CASES))])
+@pytest.mark.parametrize("causal", [True, False])
+def test_merge_verify_matches_oracle_and_decides_identically(lynx, case, causal):
+    B, Hkv, G, k, lens, bt, shuffled, recipe = case
+    c = _case(lynx, 200 + len(lens) + k, B, Hkv, G, k, lens, bt, shuffled, recipe)
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    draft = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=causal)
+    draft_np = draft.cpu().numpy()
+    ref = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                           c["lens"].numpy(), Hkv, bt, causal=causal)
+    # thresholds: pick (atol, rtol) so that every oracle dev is outside the guard band around 1
+    for atol, rtol in [(2e-2, 2e-2), (5e-2, 5e-2), (1e-1, 1e-1), (3e-1, 1e-1), (1.0, 0.0), (3e-3, 0.0)]:
+        want_fr, want_dev = oracle.verify_decision(ref, draft_np, atol, rtol)
+        if np.all(np.abs(want_dev - 1.0) > 0.05):
+            out, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"],
+                                                       draft_out=draft, atol=atol, rtol=rtol,
+                                                       causal=causal)
+            lynx.check(c["ws"])
+            _close(out.cpu().numpy().astype(np.float64), ref, "merge-verify attention")
+            assert np.array_equal(fr.cpu().numpy(), want_fr), (atol, rtol, want_dev)
+            assert np.allclose(dev.cpu().numpy(), want_dev, rtol=0.05, atol=1e-3)
+    # the full result fed back as its own draft is accepted everywhere
+    out, _, _ = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=causal)
+    _close(out.cpu().numpy().astype(np.float64), ref, "merge-verify attention (no draft)")
+    out2, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"],
+                                                draft_out=out, atol=1e-3, rtol=1e-2, causal=causal)
+    lynx.check(c["ws"])
+    assert torch.equal(out, out2)
+    assert fr.cpu().tolist() == [k] * B and float(dev.max()) == 0.0
+    # perturbing position j of sequence 0 makes it the first rejection
+    for j in range(k):
+        bad = out.clone()
+        bad[0, j, 1 % (Hkv * G), 5] += 1.0
+        _, fr, _ = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"],
+                                               draft_out=bad, atol=1e-3, rtol=1e-2, causal=causal)
+        assert int(fr[0]) == j
+
+
+def test_anchor_then_verify_window_like_the_decoder(lynx):
+    # k draft steps on the Anchor state with growing context, then one verify pass on Q_full
+    B, Hkv, G, k, L = 1, 2, 4, 4, 1203
+    c = _case(lynx, 301, B, Hkv, G, k, (L,), 16, True, "lognormal_channels")
+    qd, td = c["q"].cuda(), c["table"].cuda()
+    ws1 = lynx.make_workspace(c["geo"], B, 1, "cuda")
+    draft = torch.empty(B, k, Hkv * G, 128, dtype=torch.float32, device="cuda")
+    for j in range(k):
+        lens_j = torch.tensor([L - k + j + 1], dtype=torch.int32).cuda()
+        draft[:, j:j + 1] = lynx.anchor_attention(c["geo"], qd[:, j:j + 1].contiguous(), c["K"], c["V"],
+                                                  td, lens_j, ws1)
+    ref_draft = oracle.attention(False, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                                 c["lens"].numpy(), Hkv, 16, causal=True)
+    _close(draft.cpu().numpy().astype(np.float64), ref_draft, "stepwise drafts vs causal anchor")
+    ref = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                           c["lens"].numpy(), Hkv, 16, causal=True)
+    want_fr, want_dev = oracle.verify_decision(ref, draft.cpu().numpy(), 0.5, 0.0)
+    assert np.all(np.abs(want_dev - 1.0) > 0.05)
+    out, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, c["lens"].cuda(),
+                                               c["ws"], draft_out=draft, atol=0.5, rtol=0.0)
+    lynx.check(c["ws"])
+    _close(out.cpu().numpy().astype(np.float64), ref, "verify")
+    assert np.array_equal(fr.cpu().numpy(), want_fr)
+
+
+def test_attention_argument_errors_and_bad_block_table(lynx):
+    c = _case(lynx, 302, 1, 2, 4, 1, (100,), 16, True, "normal")
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    with pytest.raises(lynx.LynxError):                      # workspace too small
+        lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"][:128])
+    bad_geo = lynx.Geometry(8, 2, 24, c["geo"].num_blocks, c["geo"].max_blocks_per_seq)
+    with pytest.raises(lynx.LynxError):                      # block_tokens not a multiple of 16
+        lynx.anchor_attention(bad_geo, qd, c["K"], c["V"], td, ld, c["ws"])
+    assert lynx.workspace_bytes(bad_geo, 1, 1) == 0
+    q17 = torch.zeros(1, 17, 8, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lynx.LynxError):                      # too many query positions
+        lynx.anchor_attention(c["geo"], q17, c["K"], c["V"], td, ld, c["ws"])
+    # an out-of-range block id is clamped on the device and reported by lynx_check
+    bad_table = td.clone()
+    bad_table[0, 1] = 10_000
+    lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], bad_table, ld, c["ws"])
+    with pytest.raises(lynx.LynxError, match="block id"):
+        lynx.check(c["ws"])
+    lynx.check(c["ws"])                                      # the status word was cleared
+    out = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"])
+    lynx.check(c["ws"])
+    ref = oracle.attention(False, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                           c["lens"].numpy(), 2, 16)
+    _close(out.cpu().numpy().astype(np.float64), ref, "after a bad table")
+
+
+def test_long_context_multi_chunk_sampled(lynx):
+    # one KV head pair at 40k tokens: many chunks per (sequence, head), ragged end
+    B, Hkv, G, k, L = 1, 2, 4, 4, 40_003
+    c = _case(lynx, 303, B, Hkv, G, k, (L,), 16, True, "lognormal_channels")
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    out_a = lynx.anchor_attention(c["geo"], qd[:, :1].contiguous(), c["K"], c["V"], td, ld,
+                                  lynx.make_workspace(c["geo"], B, 1, "cuda"))
+    out_v, _, _ = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"])
+    lynx.check(c["ws"])
+    ref_a = oracle.attention(False, bf16_bits(c["q"][:, :1]), c["kp"], c["vp"], c["table"].numpy(),
+                             c["lens"].numpy(), Hkv, 16)
+    ref_v = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                             c["lens"].numpy(), Hkv, 16, causal=True)
+    _close(out_a.cpu().numpy().astype(np.float64), ref_a, "anchor 40k")
+    _close(out_v.cpu().numpy().astype(np.float64), ref_v, "verify 40k")
