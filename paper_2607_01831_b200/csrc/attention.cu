@@ -247,10 +247,10 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
         merge_codes(xl[wd], yl[wd], evl, odl);
         merge_codes(xh[wd], yh[wd], evh, odh);
         // (e0,e2) (e4,e6) from ev; (e1,e3) (e5,e7) from od; value = code - 128
-        const uint32_t l0 = hadd2(prmt(evl, kMagic, 0x5140), kNeg1152), l1 = hadd2(prmt(evl, kMagic, 0x7362), kNeg1152);
-        const uint32_t l2 = hadd2(prmt(odl, kMagic, 0x5140), kNeg1152), l3 = hadd2(prmt(odl, kMagic, 0x7362), kNeg1152);
-        const uint32_t h0 = hadd2(prmt(evh, kMagic, 0x5140), kNeg1152), h1 = hadd2(prmt(evh, kMagic, 0x7362), kNeg1152);
-        const uint32_t h2 = hadd2(prmt(odh, kMagic, 0x5140), kNeg1152), h3 = hadd2(prmt(odh, kMagic, 0x7362), kNeg1152);
+        const uint32_t l0 = hadd2(prmt(evl, kMagic, 0x7150), kNeg1152), l1 = hadd2(prmt(evl, kMagic, 0x7352), kNeg1152);
+        const uint32_t l2 = hadd2(prmt(odl, kMagic, 0x7150), kNeg1152), l3 = hadd2(prmt(odl, kMagic, 0x7352), kNeg1152);
+        const uint32_t h0 = hadd2(prmt(evh, kMagic, 0x7150), kNeg1152), h1 = hadd2(prmt(evh, kMagic, 0x7352), kNeg1152);
+        const uint32_t h2 = hadd2(prmt(odh, kMagic, 0x7150), kNeg1152), h3 = hadd2(prmt(odh, kMagic, 0x7352), kNeg1152);
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           mma16816(s[nt], l0, h0, l2, h2, w.qf[nt][2 * wd][0], w.qf[nt][2 * wd][1]);
@@ -375,12 +375,12 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
         // m-tile qd=0: dims e(4half+0) [row g] and e(4half+1) [row g+8]; qd=1: e(4half+2), e(4half+3)
         const uint32_t ab0 = hadd2((uab & 0x00FF00FFu) | kMagic, kNeg1152);
         const uint32_t ab1 = hadd2((vab & 0x00FF00FFu) | kMagic, kNeg1152);
-        const uint32_t ab2 = hadd2(prmt(uab, kMagic, 0x5341), kNeg1152);
-        const uint32_t ab3 = hadd2(prmt(vab, kMagic, 0x5341), kNeg1152);
+        const uint32_t ab2 = hadd2(prmt(uab, kMagic, 0x7351), kNeg1152);
+        const uint32_t ab3 = hadd2(prmt(vab, kMagic, 0x7351), kNeg1152);
         const uint32_t cd0 = hadd2((ucd & 0x00FF00FFu) | kMagic, kNeg1152);
         const uint32_t cd1 = hadd2((vcd & 0x00FF00FFu) | kMagic, kNeg1152);
-        const uint32_t cd2 = hadd2(prmt(ucd, kMagic, 0x5341), kNeg1152);
-        const uint32_t cd3 = hadd2(prmt(vcd, kMagic, 0x5341), kNeg1152);
+        const uint32_t cd2 = hadd2(prmt(ucd, kMagic, 0x7351), kNeg1152);
+        const uint32_t cd3 = hadd2(prmt(vcd, kMagic, 0x7351), kNeg1152);
         const int mt = wd * 4 + half * 2;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
