@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the Lynx hot path on B200: split-quantise, anchor decode attention, merge-verify.
+
+One "step" is one pass of the whole hot path over one synthetic batch of the chosen workload:
+split-quantise the whole BF16 KV cache (K and V, all layers), then for every speculation depth
+k of the workload: k anchor decode steps on the Anchor planes (growing context) followed by
+one merge-verify pass over the k drafted positions with its accept/reject index.
+
+Prints ONE JSON line (see README for the fields).  `--impl reference` times the CPU
+oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import synth  # noqa: E402
+
+METRIC = "split-quant & anchor/verify decode-attn HBM GB/s (% of B200 peak); tokens/s"
+BYTES_PER_ROW = {"split_quantize": 392, "anchor_attention": 72, "merge_verify_attention": 136}
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------- workload set-up
+class Workload:
+    """All device state of one configuration, layers flattened into the batch dimension."""
+
+    def __init__(self, cfg_id: int, device, rank: int = 0, layers: int = 0):
+        import dataclasses
+
+        import paper_2607_01831_b200 as lynx
+        self.lynx = lynx
+        wl = synth.WORKLOADS[cfg_id]
+        if layers:   # a reduced copy of the workload (profiling captures), never the bench default
+            wl = dataclasses.replace(wl, layers=layers, name=f"{wl.name}[layers={layers}]")
+        self.wl, self.cfg_id, self.device = wl, cfg_id, device
+        bt, Hkv = wl.block_tokens, wl.num_kv_heads
+        if wl.ragged:
+            lens = synth.seq_lens(wl.batch, wl.min_context, wl.context, wl.name, rank)
+        else:
+            lens = torch.full((wl.batch,), wl.context, dtype=torch.int32)
+        table, nb_layer = synth.block_table(lens, bt, wl.shuffled_blocks, wl.name, rank)
+        self.lens_cpu, self.nb_layer = lens, nb_layer
+        L = wl.layers
+        self.B = L * wl.batch
+        offs = (torch.arange(L, dtype=torch.int32) * nb_layer).view(L, 1, 1)
+        self.table = (table.unsqueeze(0) + offs).reshape(self.B, -1).contiguous().to(device)
+        self.lens_flat_cpu = lens.repeat(L)
+        self.geo = lynx.Geometry(wl.num_q_heads, Hkv, bt, L * nb_layer, table.shape[1])
+        # BF16 source cache, generated per layer into one flat allocation per tensor
+        self.src = {}
+        for which in "KV":
+            buf = torch.empty(L * nb_layer, Hkv, bt, 128, dtype=torch.bfloat16, device=device)
+            for l in range(L):
+                synth.kv_block_values(wl.recipe, nb_layer, Hkv, bt, device, wl.name, which, l, rank,
+                                      out=buf[l * nb_layer:(l + 1) * nb_layer])
+            self.src[which] = buf
+        self.planes = {w: lynx.alloc_planes((L * nb_layer, Hkv, bt), device) for w in "KV"}
+        self.block_ids = None
+        if wl.shuffled_blocks:   # newly arrived blocks, in arrival (table) order, every layer
+            ids = [table[b, :(int(lens[b]) + bt - 1) // bt] for b in range(wl.batch)]
+            ids = torch.cat(ids).to(torch.int32)
+            self.block_ids = (ids.unsqueeze(0) + offs.view(L, 1)).reshape(-1).contiguous().to(device)
+        # windows: (k, [lens tensor per draft step], q [B][k][Hq][128], draft, ws)
+        reps = max(1, wl.anchor_steps // max(wl.k_list)) if wl.anchor_steps else 1
+        self.windows = []
+        for k in wl.k_list:
+            q = synth.queries(self.B, k, wl.num_q_heads, device, wl.name, "q", k, rank)
+            step_lens = [(self.lens_flat_cpu - k + j + 1).clamp(min=0).to(torch.int32).to(device)
+                         for j in range(k)]
+            qs = [q[:, j:j + 1].contiguous() for j in range(k)]
+            self.windows.append(dict(
+                k=k, q=q, qs=qs, step_lens=step_lens, reps=reps,
+                step_out=[torch.empty(self.B, 1, wl.num_q_heads, 128, dtype=torch.float32, device=device)
+                          for _ in range(k)],
+                draft=torch.empty(self.B, k, wl.num_q_heads, 128, dtype=torch.float32, device=device),
+                out_full=torch.empty(self.B, k, wl.num_q_heads, 128, dtype=torch.float32, device=device),
+                first_reject=torch.empty(self.B, dtype=torch.int32, device=device),
+                dev=torch.empty(self.B, k, dtype=torch.float32, device=device),
+                ws=lynx.make_workspace(self.geo, self.B, k, device)))
+        self.lens_flat = self.lens_flat_cpu.to(device)
+        self.ws1 = lynx.make_workspace(self.geo, self.B, 1, device)
+        # algorithmic bytes per launch kind
+        rows_kv = 2 * L * Hkv * int(lens.sum())          # K rows + V rows over all layers
+        self.rows_kv = rows_kv
+        self.tokens_ctx = L * int(lens.sum())
+        self.launch_rows = {"split_quantize": L * nb_layer * Hkv * bt, "anchor_attention": rows_kv,
+                            "merge_verify_attention": rows_kv}
+        torch.cuda.synchronize()
+
+    # one pass of the hot path; `rec` (optional) receives (kind, start_event, end_event)
+    def step(self, rec=None):
+        lynx = self.lynx
+
+        def timed(kind, fn):
+            if rec is None:
+                return fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            r = fn()
+            b.record()
+            rec.append((kind, a, b))
+            return r
+
+        for w in "KV":
+            timed("split_quantize", lambda w=w: lynx.split_quantize(
+                self.src[w], out=self.planes[w], block_ids=self.block_ids,
+                rows_per_block=self.wl.num_kv_heads * self.wl.block_tokens if self.block_ids is not None else 0))
+        K, V = self.planes["K"], self.planes["V"]
+        n = 2
+        for win in self.windows:
+            for _ in range(win["reps"]):
+                for j in range(win["k"]):
+                    timed("anchor_attention", lambda j=j: lynx.anchor_attention(
+                        self.geo, win["qs"][j], K, V, self.table, win["step_lens"][j], self.ws1,
+                        out=win["step_out"][j]))
+                    win["draft"][:, j:j + 1].copy_(win["step_out"][j])
+                timed("merge_verify_attention", lambda: lynx.merge_verify_attention(
+                    self.geo, win["q"], K, V, self.table, self.lens_flat, win["ws"], draft_out=win["draft"],
+                    atol=0.5, rtol=0.1, causal=True, out_full=win["out_full"],
+                    first_reject=win["first_reject"], dev=win["dev"]))
+                n += win["k"] + 1
+        return n
+
+    def launches_per_step(self):
+        return 2 + sum(w["reps"] * (w["k"] + 1) for w in self.windows)
+
+    def bytes_per_step(self):
+        b = 2 * self.launch_rows["split_quantize"] * BYTES_PER_ROW["split_quantize"]
+        for w in self.windows:
+            b += w["reps"] * (w["k"] * self.rows_kv * BYTES_PER_ROW["anchor_attention"]
+                              + self.rows_kv * BYTES_PER_ROW["merge_verify_attention"])
+        return b
+
+
+# ------------------------------------------------------------------------------ clock sampling
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                 c[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# --------------------------------------------------------------------------------- CPU oracle
+def oracle_sample(cfg_id: int, budget_note: bool = True):
+    """Times the oracle, as it stands, on a bounded sample of the workload (one layer's K rows
+    for split-quantise; one layer, one decode step, a subset of KV heads for the two attention
+    kernels).  Returns (GB/s over the sample, description, threads, seconds)."""
+    import numpy as np
+
+    import oracle
+    wl = synth.WORKLOADS[cfg_id]
+    bt = wl.block_tokens
+    ctx = min(wl.context, 32768)                       # bounded context for the sample
+    heads = 2                                          # KV heads in the attention sample
+    G = wl.num_q_heads // wl.num_kv_heads
+    k = wl.k_list[-1] if len(wl.k_list) == 1 else 4
+    lens = torch.tensor([ctx], dtype=torch.int32)
+    table, nb = synth.block_table(lens, bt, wl.shuffled_blocks, "cpu_sample")
+    bits = lambda t: t.contiguous().view(torch.int16).numpy().view(np.uint16)
+    kk = synth.kv_block_values(wl.recipe, nb, heads, bt, "cpu", "cpu_sample", "K")
+    vv = synth.kv_block_values(wl.recipe, nb, heads, bt, "cpu", "cpu_sample", "V")
+    q = synth.queries(1, k, heads * G, "cpu", "cpu_sample")
+    kb, vb = bits(kk), bits(vv)
+    t0 = time.perf_counter()
+    kp = oracle.split_quantize(kb)
+    vp = oracle.split_quantize(vb)
+    t1 = time.perf_counter()
+    oracle.attention(False, bits(q[:, :1]), kp, vp, table.numpy(), lens.numpy(), heads, bt)
+    t2 = time.perf_counter()
+    of = oracle.attention(True, bits(q), kp, vp, table.numpy(), lens.numpy(), heads, bt, causal=True)
+    oracle.verify_decision(of, of.astype(np.float32), 0.5, 0.1)
+    t3 = time.perf_counter()
+    rows = 2 * heads * ctx
+    nbytes = rows * (BYTES_PER_ROW["split_quantize"] + BYTES_PER_ROW["anchor_attention"]
+                     + BYTES_PER_ROW["merge_verify_attention"])
+    secs = t3 - t0
+    desc = (f"{wl.name}: one layer, {heads} of {wl.num_kv_heads} KV heads, {ctx} of {wl.context} tokens: "
+            f"split-quantise K+V ({t1 - t0:.2f} s), 1 anchor step ({t2 - t1:.2f} s), 1 verify k={k} "
+            f"({t3 - t2:.2f} s); same algorithmic bytes per row as the GPU arm")
+    return nbytes / secs / 1e9, desc, oracle.threads(), secs
+
+
+# --------------------------------------------------------------------------------------- main
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    desc, threads = "", 0
+    for i in range(args.warmup + args.steps):
+        v, desc, threads, _ = oracle_sample(args.config)
+        if i >= args.warmup:
+            vals.append(v)
+    wl = synth.WORKLOADS[args.config]
+    value = len(vals) / sum(1.0 / v for v in vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "note": "CPU oracle on host cores, bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="lynx", choices=["lynx", "reference"])
+    ap.add_argument("--config", type=int, default=3, choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--layers", type=int, default=0,
+                    help="run a reduced copy of the workload with this many layers (for ncu captures)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "lynx" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    wlk = Workload(args.config, device, rank, args.layers)
+    wl = wlk.wl
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        wlk.step()
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    rec = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    n_launch = 0
+    for _ in range(args.steps):
+        n_launch += wlk.step(rec)
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+    if dist is not None:
+        t = torch.tensor([ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    lynx = wlk.lynx
+    for w in wlk.windows:
+        lynx.check(w["ws"])
+    lynx.check(wlk.ws1)
+
+    ms_per_step = ms / args.steps
+    step_bytes = wlk.bytes_per_step()
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+
+    per = {}
+    for kind, a, b in rec:
+        per.setdefault(kind, []).append(a.elapsed_time(b))
+    kernels = {}
+    for kind, ts in per.items():
+        avg = sum(ts) / len(ts)
+        nbytes = wlk.launch_rows[kind] * BYTES_PER_ROW[kind]
+        gbs = nbytes / (avg * 1e-3) / 1e9
+        kernels[kind] = {"launches": len(ts), "avg_ms": avg, "min_ms": min(ts), "GBps": gbs,
+                         "frac_of_measured": gbs / peak, "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
+                         "share_of_step": sum(ts) / args.steps / ms_per_step}
+    kernels["split_quantize"]["tokens_per_s"] = wlk.tokens_ctx / (2 * kernels["split_quantize"]["avg_ms"] * 1e-3)
+    kernels["anchor_attention"]["tokens_per_s"] = wl.batch / (kernels["anchor_attention"]["avg_ms"] * 1e-3)
+    mv = [t for k_, a, b in rec if k_ == "merge_verify_attention" for t in [a.elapsed_time(b)]]
+    ks = [w["k"] for w in wlk.windows for _ in range(w["reps"])] * args.steps
+    kernels["merge_verify_attention"]["tokens_per_s"] = wl.batch * sum(ks) / (sum(mv) * 1e-3)
+    dom = max(kernels, key=lambda k_: kernels[k_]["share_of_step"])
+    roof = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["GBps"], "peak": peak, "unit": "GB/s",
+            "frac": kernels[dom]["GBps"] / peak, "peak_source": peak_kind + " (MEASURED_PEAKS.json hbm_gbs)"
+            if peak_kind == "measured" else "fallback 6.65 TB/s",
+            "traffic": None, "algorithmic_bytes_per_launch": wlk.launch_rows[dom] * BYTES_PER_ROW[dom]}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16 levels x f16 q/p, f32 accumulate (quantiser f32)",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "layers": wl.layers, "batch": wl.batch, "context": wl.context,
+                   "num_kv_heads": wl.num_kv_heads, "num_q_heads": wl.num_q_heads, "k": list(wl.k_list),
+                   "block_tokens": wl.block_tokens, "layers_flattened_into_batch": True,
+                   "l2": "inputs larger than L2 (no flush)" if step_bytes > 1e9 else "inputs fit in L2",
+                   "step": "split-quantise K,V; per k: k anchor steps then 1 merge-verify"},
+        "gpu_launches": n_launch, "frac_of_measured_peak": value / world / peak,
+        "frac_of_nominal_8TBps": value / world / NOMINAL_HBM_GBS,
+        "kernels": kernels, "roofline": roof, "clocks": clocks,
+    }
+
+    if rank == 0 and world == 1 and not args.no_e2e:
+        line["e2e"] = run_e2e(wlk, args.e2e_steps, step_bytes)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, desc, threads, secs = oracle_sample(args.config)
+        line["cpu_baseline"] = {"value": v, "unit": "GB/s", "cores": threads, "kind": "oracle",
+                                "sample": desc, "seconds": secs}
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+def run_e2e(wlk: "Workload", steps: int, step_bytes: int):
+    """The same step driven from HOST buffers: every step copies the BF16 KV cache and the queries
+    from pinned host memory to the device, runs the path, and reads the verified outputs and the
+    accept/reject indices back."""
+    host_src = {w: torch.empty(wlk.src[w].shape, dtype=torch.bfloat16, pin_memory=True) for w in "KV"}
+    for w in "KV":
+        host_src[w].copy_(wlk.src[w])
+    host_q = [win["q"].cpu().pin_memory() for win in wlk.windows]
+    host_out = [torch.empty(win["out_full"].shape, dtype=torch.float32, pin_memory=True) for win in wlk.windows]
+    host_fr = [torch.empty(win["first_reject"].shape, dtype=torch.int32, pin_memory=True) for win in wlk.windows]
+    h2d = sum(t.numel() * t.element_size() for t in host_src.values()) + sum(t.numel() * 2 for t in host_q)
+    d2h = sum(t.numel() * 4 for t in host_out) + sum(t.numel() * 4 for t in host_fr)
+
+    def one():
+        for w in "KV":
+            wlk.src[w].copy_(host_src[w], non_blocking=True)
+        for win, hq in zip(wlk.windows, host_q):
+            win["q"].copy_(hq, non_blocking=True)
+            for j in range(win["k"]):
+                win["qs"][j].copy_(win["q"][:, j:j + 1])
+        wlk.step()
+        for win, ho, hf in zip(wlk.windows, host_out, host_fr):
+            ho.copy_(win["out_full"], non_blocking=True)
+            hf.copy_(win["first_reject"], non_blocking=True)
+
+    one()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return {"value": step_bytes / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+
+if __name__ == "__main__":
+    main()

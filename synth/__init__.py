@@ -80,7 +80,7 @@ def channel_scale(recipe: str, num_kv_heads: int, device, *key) -> torch.Tensor:
 
 
 def kv_block_values(recipe: str, num_blocks: int, num_kv_heads: int, block_tokens: int, device,
-                    *key) -> torch.Tensor:
+                    *key, out: torch.Tensor | None = None) -> torch.Tensor:
     """BF16 [num_blocks][Hkv][block_tokens][128] drawn per the recipe.
 
     normal_outlier4x8       N(0,1), 4 fixed channels per head scaled x8
@@ -88,11 +88,14 @@ def kv_block_values(recipe: str, num_blocks: int, num_kv_heads: int, block_token
     lognormal_channels      N(0, sigma_c^2), sigma_c ~ LogNormal(0, 0.5) per (head, channel)
     student_t4              Student-t with 4 degrees of freedom
     normal                  N(0,1)
+    `out` (optional) is a preallocated BF16 tensor of that shape to fill.
     """
     dev = torch.device(device)
     g = _gen(dev, "kv", recipe, *key)
     cs = channel_scale(recipe, num_kv_heads, dev, *key)
-    out = torch.empty(num_blocks, num_kv_heads, block_tokens, D, dtype=torch.bfloat16, device=dev)
+    if out is None:
+        out = torch.empty(num_blocks, num_kv_heads, block_tokens, D, dtype=torch.bfloat16, device=dev)
+    assert tuple(out.shape) == (num_blocks, num_kv_heads, block_tokens, D) and out.dtype == torch.bfloat16
     step = max(1, (1 << 24) // (num_kv_heads * block_tokens * D))   # ~16 M elements at a time
     for b0 in range(0, num_blocks, step):
         nb = min(step, num_blocks - b0)
