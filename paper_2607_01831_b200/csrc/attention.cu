@@ -35,7 +35,7 @@ namespace {
 
 constexpr int kMaxQ = 16;          // query positions per call
 constexpr int kMaxCols = 64;       // n_q * G
-constexpr int kMaxChunkTokens = 8192;
+constexpr int kMaxChunkTokens = 4096;
 constexpr int kPartStride = 132;   // floats per (chunk, column) partial: O[128], m, l, pad
 
 struct AttnParams {
@@ -406,12 +406,12 @@ struct Cfg {
   static constexpr int kQBytes = kColsPad * LYNX_D * 2;
   static constexpr int kBlkBytes = (kMaxChunkTokens / 16) * 4;
   static constexpr int kBarBytes = 2 * NSTAGE * 8;
-  static constexpr int kMiscBytes = 64;
+  static constexpr int kMiscBytes = 128;   // 8 control words + kMaxQ deviation words
   static constexpr int kSmem = kRingAlloc + kQBytes + kBlkBytes + kBarBytes + kMiscBytes;
 };
 
-template <bool FULL, int NT, int TW, int CG, int NSTAGE>
-__global__ void __launch_bounds__((TW * CG + 1) * 32)
+template <bool FULL, int NT, int TW, int CG, int NSTAGE, int MINB>
+__global__ void __launch_bounds__((TW * CG + 1) * 32, MINB)
 attn_kernel(const AttnParams p) {
   using C = Cfg<FULL, NT, TW, CG, NSTAGE>;
   constexpr int ST = C::kST;
@@ -421,7 +421,7 @@ attn_kernel(const AttnParams p) {
   uint32_t* blk_s = reinterpret_cast<uint32_t*>(smem + C::kRingAlloc + C::kQBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kRingAlloc + C::kQBytes + C::kBlkBytes);
   int* misc = reinterpret_cast<int*>(smem + C::kRingAlloc + C::kQBytes + C::kBlkBytes + C::kBarBytes);
-  // misc[0] = abort word, misc[1] = max |q| bits, misc[2] = "this CTA is last" flag, misc[4..] dev
+  // misc[0] = abort word, misc[1] = max |q| bits, misc[2] = "this CTA is last" flag, misc[8..] dev
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int chunk = blockIdx.x, hkv = blockIdx.y, b = blockIdx.z;
@@ -663,7 +663,8 @@ attn_kernel(const AttnParams p) {
   // accept / reject (Section 4.3): only the CTA that wrote the final outputs gets here
   if (FULL && p.draft != nullptr) {
     __syncthreads();  // this CTA's out values are visible to all its threads
-    int* devs = misc + 4;
+    int* devs = misc + 8;
+    static_assert((8 + kMaxQ) * 4 <= C::kMiscBytes, "misc area too small");
     if (tid < kMaxQ) devs[tid] = 0;
     __syncthreads();
     for (int idx = tid; idx < p.ncols * LYNX_D; idx += C::kThreads) {
@@ -719,7 +720,7 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   pl->variant = ncols <= 8 ? 0 : ncols <= 16 ? 1 : ncols <= 32 ? 2 : 3;
   pl->cols_pad = ncols <= 8 ? 8 : ncols <= 16 ? 16 : ncols <= 32 ? 32 : 64;
   // chunk: the largest of {4096 .. 256} that still leaves >= 6 CTAs per resident slot
-  const int64_t slots = (int64_t)sm_count() * 2;
+  const int64_t slots = (int64_t)sm_count() * 4;
   int chunk = 256;
   for (int c = 4096; c >= 256; c >>= 1) {
     const int64_t items = (int64_t)B * s->num_kv_heads * ((cap + c - 1) / c);
@@ -739,11 +740,11 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   return true;
 }
 
-template <bool FULL, int NT, int TW, int CG, int NSTAGE>
+template <bool FULL, int NT, int TW, int CG, int NSTAGE, int MINB>
 lynx_status launch(const AttnParams& p, cudaStream_t st) {
   using C = Cfg<FULL, NT, TW, CG, NSTAGE>;
-  static_assert(C::kSmem <= 227 * 1024, "shared memory budget");
-  auto kern = attn_kernel<FULL, NT, TW, CG, NSTAGE>;
+  static_assert(MINB * (C::kSmem + 1024) <= 228 * 1024, "shared memory budget for MINB CTAs per SM");
+  auto kern = attn_kernel<FULL, NT, TW, CG, NSTAGE, MINB>;
   static bool configured[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -801,17 +802,17 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (!full) {
     switch (pl.variant) {
-      case 0: return launch<false, 1, 4, 1, 8>(p, st);
-      case 1: return launch<false, 2, 4, 1, 8>(p, st);
-      case 2: return launch<false, 2, 4, 2, 8>(p, st);
-      default: return launch<false, 2, 2, 4, 16>(p, st);
+      case 0: return launch<false, 1, 4, 1, 4, 4>(p, st);
+      case 1: return launch<false, 2, 4, 1, 5, 3>(p, st);
+      case 2: return launch<false, 2, 4, 2, 8, 1>(p, st);
+      default: return launch<false, 2, 2, 4, 16, 1>(p, st);
     }
   }
   switch (pl.variant) {
-    case 0: return launch<true, 1, 4, 1, 5>(p, st);
-    case 1: return launch<true, 2, 4, 1, 5>(p, st);
-    case 2: return launch<true, 2, 4, 2, 5>(p, st);
-    default: return launch<true, 2, 2, 4, 8>(p, st);
+    case 0: return launch<true, 1, 4, 1, 3, 4>(p, st);
+    case 1: return launch<true, 2, 4, 1, 4, 3>(p, st);
+    case 2: return launch<true, 2, 4, 2, 5, 1>(p, st);
+    default: return launch<true, 2, 2, 4, 8, 1>(p, st);
   }
 }
 

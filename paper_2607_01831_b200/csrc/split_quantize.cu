@@ -5,9 +5,10 @@
 // byte, one-contiguous-buffer-per-stream packing of the Compression Kernel paragraph.
 // Recombine is the Residual-phase refinement to Q_full of Section 4.2.
 //
-// Mapping: a row is 256 B of BF16 = 16 lanes x 16 B, so a half-warp owns a row: one 128-bit
-// streaming load per lane, min/max by 4 xor-shuffles, 8 codes per lane, 4 B of each plane per
-// lane (a warp writes 128 contiguous bytes per plane).  Several rows are in flight per lane.
+// Mapping: a row is 256 B of BF16; a quarter-warp (8 lanes) owns a row: two 128-bit streaming
+// loads per lane (each instruction covers 128 contiguous bytes of the row), min/max on packed
+// BF16 pairs and three xor-shuffles, 16 codes per lane, 2 x 4 B of each plane per lane.
+// Two rows are in flight per quarter-warp.
 #include <cuda_bf16.h>
 
 #include "lynx_common.cuh"
@@ -17,12 +18,45 @@ namespace lynx {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kRowsInFlight = 4;  // rows per half-warp per loop trip
+constexpr int kLanesPerRow = 8;   // a quarter-warp owns a row: 2 x 16 B per lane
+constexpr int kRowsInFlight = 2;  // rows per quarter-warp per loop trip
 
 // Round-half-even of the exact product u*inv, as the low byte of an FP32 whose ulp is 1:
 // fma(u, inv, 1.5 * 2^23) rounds the exact sum once, to an integer, ties to even.
 __device__ __forceinline__ uint32_t code_bits(float x, float mn, float inv) {
   return __float_as_uint(__fmaf_rn(__fsub_rn(x, mn), inv, 12582912.0f));
+}
+__device__ __forceinline__ uint32_t bf2min(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("min.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf2max(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+
+// Codes of 8 consecutive elements (4 BF16 pairs in w) -> 4 bytes of each nibble plane.
+__device__ __forceinline__ void codes8(const uint32_t (&w)[4], float mn, float inv, uint32_t& a,
+                                       uint32_t& r) {
+  uint32_t c[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    c[2 * i] = code_bits(__uint_as_float(w[i] << 16), mn, inv);
+    c[2 * i + 1] = code_bits(__uint_as_float(w[i] & 0xFFFF0000u), mn, inv);
+  }
+  // low bytes gathered: w0 = codes 0..3, w1 = codes 4..7
+  const uint32_t w0 = __byte_perm(__byte_perm(c[0], c[1], 0x0040), __byte_perm(c[2], c[3], 0x0040), 0x5410);
+  const uint32_t w1 = __byte_perm(__byte_perm(c[4], c[5], 0x0040), __byte_perm(c[6], c[7], 0x0040), 0x5410);
+  // bytes 0 and 2 of each combination hold two packed nibbles (the other bytes are unused)
+  const uint32_t s0 = w0 >> 4, s1 = w1 >> 4;
+  const uint32_t a0 = (s0 & 0x0F0F0F0Fu) | ((w0 >> 8) & 0xF0F0F0F0u);
+  const uint32_t a1 = (s1 & 0x0F0F0F0Fu) | ((w1 >> 8) & 0xF0F0F0F0u);
+  const uint32_t r0 = (w0 & 0x0F0F0F0Fu) | (s0 & 0xF0F0F0F0u);
+  const uint32_t r1 = (w1 & 0x0F0F0F0Fu) | (s1 & 0xF0F0F0F0u);
+  a = __byte_perm(a0, a1, 0x6420);
+  r = __byte_perm(r0, r1, 0x6420);
 }
 
 template <bool kIds>
@@ -31,12 +65,12 @@ split_quantize_kernel(const uint4* __restrict__ src, int64_t n_logical_rows,
                       const int32_t* __restrict__ block_ids, uint32_t rows_per_block,
                       int64_t n_blocks_total, uint32_t* __restrict__ anchor,
                       uint32_t* __restrict__ residual, float2* __restrict__ meta) {
-  const int lane16 = threadIdx.x & 15;
-  const int64_t hw = (int64_t)blockIdx.x * (kThreads / 16) + (threadIdx.x >> 4);
-  const int64_t hw_total = (int64_t)gridDim.x * (kThreads / 16);
+  const int ln = threadIdx.x & (kLanesPerRow - 1);
+  const int64_t grp = (int64_t)blockIdx.x * (kThreads / kLanesPerRow) + (threadIdx.x / kLanesPerRow);
+  const int64_t grp_total = (int64_t)gridDim.x * (kThreads / kLanesPerRow);
 
-  for (int64_t r0 = hw * kRowsInFlight; r0 < n_logical_rows; r0 += hw_total * kRowsInFlight) {
-    uint4 raw[kRowsInFlight];
+  for (int64_t r0 = grp * kRowsInFlight; r0 < n_logical_rows; r0 += grp_total * kRowsInFlight) {
+    uint4 lo[kRowsInFlight], hi[kRowsInFlight];
     int64_t row[kRowsInFlight];
 #pragma unroll
     for (int u = 0; u < kRowsInFlight; ++u) {
@@ -52,49 +86,44 @@ split_quantize_kernel(const uint4* __restrict__ src, int64_t n_logical_rows,
           row[u] = lr;
         }
       }
-      raw[u] = make_uint4(0, 0, 0, 0);
-      if (row[u] >= 0) raw[u] = __ldcs(src + row[u] * 16 + lane16);
+      lo[u] = hi[u] = make_uint4(0, 0, 0, 0);
+      if (row[u] >= 0) {
+        lo[u] = __ldcs(src + row[u] * 16 + ln);      // elements 8*ln .. 8*ln+7
+        hi[u] = __ldcs(src + row[u] * 16 + 8 + ln);  // elements 64+8*ln .. 64+8*ln+7
+      }
     }
 #pragma unroll
     for (int u = 0; u < kRowsInFlight; ++u) {
       // the shuffles below are executed by every lane of the warp, valid row or not
-      float f[8];
-      const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+      const uint32_t wl[4] = {lo[u].x, lo[u].y, lo[u].z, lo[u].w};
+      const uint32_t wh[4] = {hi[u].x, hi[u].y, hi[u].z, hi[u].w};
+      // packed BF16 min / max over the lane's 16 values, then one register (min, -max) through
+      // three xor-shuffles of the 8 lanes that own the row
+      const uint32_t mn2 = bf2min(bf2min(bf2min(wl[0], wl[1]), bf2min(wl[2], wl[3])),
+                                  bf2min(bf2min(wh[0], wh[1]), bf2min(wh[2], wh[3])));
+      const uint32_t mx2 = bf2max(bf2max(bf2max(wl[0], wl[1]), bf2max(wl[2], wl[3])),
+                                  bf2max(bf2max(wh[0], wh[1]), bf2max(wh[2], wh[3])));
+      uint32_t v = bf2min(__byte_perm(mn2, mx2, 0x5410) ^ 0x80000000u,
+                          __byte_perm(mn2, mx2, 0x7632) ^ 0x80000000u);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        f[2 * i] = __uint_as_float(w[i] << 16);
-        f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-      }
-      float mn = fminf(fminf(fminf(f[0], f[1]), fminf(f[2], f[3])),
-                       fminf(fminf(f[4], f[5]), fminf(f[6], f[7])));
-      float mx = fmaxf(fmaxf(fmaxf(f[0], f[1]), fmaxf(f[2], f[3])),
-                       fmaxf(fmaxf(f[4], f[5]), fmaxf(f[6], f[7])));
-#pragma unroll
-      for (int off = 8; off >= 1; off >>= 1) {
-        mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
-        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
-      }
+      for (int off = 4; off >= 1; off >>= 1) v = bf2min(v, __shfl_xor_sync(0xFFFFFFFFu, v, off));
+      const float mn = __uint_as_float(v << 16);
+      const float mx = __uint_as_float((v & 0xFFFF0000u) ^ 0x80000000u);
       const float range = __fsub_rn(mx, mn);
       const bool live = range >= 0x1p-100f;
       const float scale = live ? __fdiv_rn(range, 255.0f) : 0.0f;
       const float inv = live ? __fdiv_rn(255.0f, range) : 0.0f;
       const float zero = __fadd_rn(mn, 0.0f);  // -0 -> +0
 
-      uint32_t c[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) c[i] = code_bits(f[i], mn, inv);
-      // gather the low bytes: w0 = codes 0..3, w1 = codes 4..7
-      const uint32_t w0 = __byte_perm(__byte_perm(c[0], c[1], 0x0040), __byte_perm(c[2], c[3], 0x0040), 0x5410);
-      const uint32_t w1 = __byte_perm(__byte_perm(c[4], c[5], 0x0040), __byte_perm(c[6], c[7], 0x0040), 0x5410);
-      // nibble planes: bytes 0 and 2 of (x | x >> 4) hold two packed nibbles each
-      const uint32_t h0 = (w0 >> 4) & 0x0F0F0F0Fu, h1 = (w1 >> 4) & 0x0F0F0F0Fu;
-      const uint32_t l0 = w0 & 0x0F0F0F0Fu, l1 = w1 & 0x0F0F0F0Fu;
-      const uint32_t a = __byte_perm(h0 | (h0 >> 4), h1 | (h1 >> 4), 0x6420);
-      const uint32_t r = __byte_perm(l0 | (l0 >> 4), l1 | (l1 >> 4), 0x6420);
+      uint32_t a_lo, r_lo, a_hi, r_hi;
+      codes8(wl, mn, inv, a_lo, r_lo);
+      codes8(wh, mn, inv, a_hi, r_hi);
       if (row[u] >= 0) {
-        __stcs(anchor + row[u] * 16 + lane16, a);
-        __stcs(residual + row[u] * 16 + lane16, r);
-        if (lane16 == 0) __stcs(meta + row[u], make_float2(scale, zero));
+        __stcs(anchor + row[u] * 16 + ln, a_lo);
+        __stcs(anchor + row[u] * 16 + 8 + ln, a_hi);
+        __stcs(residual + row[u] * 16 + ln, r_lo);
+        __stcs(residual + row[u] * 16 + 8 + ln, r_hi);
+        if (ln == 0) __stcs(meta + row[u], make_float2(scale, zero));
       }
     }
   }
@@ -152,7 +181,7 @@ extern "C" lynx_status lynx_split_quantize(const void* src_bf16, int64_t n_rows,
       (reinterpret_cast<uintptr_t>(meta) & 7u))
     return LYNX_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int rows_per_cta_trip = (kThreads / 16) * kRowsInFlight;
+  const int rows_per_cta_trip = (kThreads / kLanesPerRow) * kRowsInFlight;
   if (block_ids) {
     if (n_block_ids < 0 || rows_per_block <= 0 || n_rows % rows_per_block != 0) return LYNX_ERR_SHAPE;
     if (n_block_ids == 0) return LYNX_OK;
