@@ -8,20 +8,22 @@
 // Per-token groups make dequantisation almost free: with x^ = zero_t + scale_t * level,
 //     q . K^_t        = scale_t * (q . level_t) + zero_t * sum_d q_d
 //     sum_t p_t V^_t  = sum_t (p_t scale_t) level_t + (sum_t p_t zero_t) * 1
-// so the two contractions run on the integer levels, which are exact in FP16, and the scalars
-// are applied per token outside.  Levels are centred (a-8 for the Anchor state, code-128 for
-// the full state) so that no large bias enters the FP32 accumulation.
+// so the two contractions run on the integer levels and the scalars are applied per token
+// outside.  Q.K^T is exact integer arithmetic on the int8 tensor-core path (u8 levels times two
+// s8 digit planes of the query); P.V runs in FP16 with centred levels (a-8 for the Anchor
+// state, code-128 for the full state) so that no large bias enters the FP32 accumulation.
 //
 // Kernel shape.  Grid = (chunk, KV head, sequence): flash-decoding split-K over the context.
 // A CTA has TW*CG consumer warps and one producer warp.  The producer streams 16-token
 // sub-blocks (1 KiB per plane + 128 B of meta, each contiguous in the paged layout) into a
 // shared-memory ring with cp.async.bulk (TMA, 1-D) completing on mbarriers.  Consumer warp
 // (tw, cg) takes 16-token tile tw of every stage for columns [cg*NT*8, (cg+1)*NT*8):
-//   S^T[16 tok x 8 col] = level(K)[16 x 128] . Q^T        mma.m16n8k16, tokens are M
+//   S^T[16 tok x 8 col] = level(K)[16 x 128] . Q^T        mma.m16n8k32 u8 x s8, tokens are M
 //   online softmax with a lazily updated maximum (one warp vote per tile, no shuffles)
 //   P^T -> B operand by movmatrix (8x8 b16 transpose)
-//   O^T[128 dim x 8 col] += level(V)^T[128 x 16 tok] . P^T  mma.m16n8k16, dims are M
-// Operands are built straight from the nibbles with LOP3/PRMT and one FP16 add/fma per pair.
+//   O^T[128 dim x 8 col] += level(V)^T[128 x 16 tok] . P^T  mma.m16n8k16 f16, dims are M
+// K operands are the nibbles / merged codes themselves (one or two logic ops per 4 levels);
+// V operands are built from the nibbles with LOP3/PRMT and one FP16 add/fma per pair.
 // Partials (m, l, O) are merged across the CTA's token warps in shared memory, written to the
 // workspace, and the last CTA of a (sequence, KV head) (atomic ticket, no waiting) merges the
 // chunks; for verification the last CTA of a sequence also takes the accept/reject decision.
@@ -120,6 +122,14 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                         uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
   uint32_t d;
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
@@ -192,8 +202,8 @@ __device__ __forceinline__ int pi_row(int r) { return r ^ ((r >> 1) & 1); }
 
 template <bool FULL, int NT>
 struct WarpState {
-  uint32_t qf[NT][8][2];  // Q^T B-fragments: [n-tile][k-step][reg]
-  float qs[NT][2];        // sum_d q_d of the thread's two columns (times 2^-e already folded)
+  uint32_t qf[NT][2][4][2];  // Q^T B-fragments (s8): [n-tile][digit plane hi/lo][k32 step][reg]
+  float qs[NT][2];        // sum_d q_d of the thread's two columns
   float m[NT][2];         // running (lazy) maximum, log2 units
   float l[NT][2];         // partial softmax denominators (this thread's rows only)
   float zs[NT][2];        // partial sum p * (zero + mid*scale) of V
@@ -209,55 +219,51 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
                                              bool masked, float ca, float cb, int g, int t) {
   constexpr uint32_t KA = 0, VA = ST * 64, KR = ST * 128, VR = ST * 192;
   constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
-  constexpr float kMidK = FULL ? 128.0f : 136.0f;
+  constexpr float kMidK = FULL ? 0.0f : 8.0f;      // K levels are the unsigned codes / nibbles
+  constexpr float kMidV = FULL ? 128.0f : 136.0f;  // V levels are centred (code-128, 16(a-8))
   constexpr float kLevelScaleV = FULL ? 1.0f : 16.0f;
   const int r0 = tw * 16 + pi_row(g);  // stage row of S row g; S row g+8 is r0 + 8
 
-  // ---- S^T = level(K) . Q^T ------------------------------------------------------------
+  // ---- S^T = level(K) . Q^T, exact in integers (u8 levels x two s8 digit planes of q) -----
   float s[NT][4];
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) s[nt][i] = 0.0f;
   {
+    int shi[NT][4], slo[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) shi[nt][i] = slo[nt][i] = 0;
     const uint4 a_lo = lds128(st + KA + r0 * 64 + t * 16);
     const uint4 a_hi = lds128(st + KA + (r0 + 8) * 64 + t * 16);
     const uint32_t xl[4] = {a_lo.x, a_lo.y, a_lo.z, a_lo.w};
     const uint32_t xh[4] = {a_hi.x, a_hi.y, a_hi.z, a_hi.w};
-    if (!FULL) {
-#pragma unroll
-      for (int wd = 0; wd < 4; ++wd) {
-        uint32_t rl[4], rh[4];
-        nib4_to_h2(xl[wd], rl);  // pairs (e0,e4) (e1,e5) (e2,e6) (e3,e7) of row g
-        nib4_to_h2(xh[wd], rh);  // same of row g+8
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          mma16816(s[nt], rl[0], rh[0], rl[1], rh[1], w.qf[nt][2 * wd][0], w.qf[nt][2 * wd][1]);
-          mma16816(s[nt], rl[2], rh[2], rl[3], rh[3], w.qf[nt][2 * wd + 1][0], w.qf[nt][2 * wd + 1][1]);
-        }
-      }
-    } else {
+    uint32_t yl[4] = {0, 0, 0, 0}, yh[4] = {0, 0, 0, 0};
+    if (FULL) {
       const uint4 b_lo = lds128(st + KR + r0 * 64 + t * 16);
       const uint4 b_hi = lds128(st + KR + (r0 + 8) * 64 + t * 16);
-      const uint32_t yl[4] = {b_lo.x, b_lo.y, b_lo.z, b_lo.w};
-      const uint32_t yh[4] = {b_hi.x, b_hi.y, b_hi.z, b_hi.w};
+      yl[0] = b_lo.x; yl[1] = b_lo.y; yl[2] = b_lo.z; yl[3] = b_lo.w;
+      yh[0] = b_hi.x; yh[1] = b_hi.y; yh[2] = b_hi.z; yh[3] = b_hi.w;
+    }
 #pragma unroll
-      for (int wd = 0; wd < 4; ++wd) {
-        uint32_t evl, odl, evh, odh;
+    for (int wd = 0; wd < 4; ++wd) {
+      // bytes of ev*: levels of elements 0,2,4,6 of the word; od*: elements 1,3,5,7
+      uint32_t evl, odl, evh, odh;
+      if (FULL) {
         merge_codes(xl[wd], yl[wd], evl, odl);
         merge_codes(xh[wd], yh[wd], evh, odh);
-        // (e0,e2) (e4,e6) from ev; (e1,e3) (e5,e7) from od; value = code - 128
-        const uint32_t l0 = hadd2(prmt(evl, kMagic, 0x7150), kNeg1152), l1 = hadd2(prmt(evl, kMagic, 0x7352), kNeg1152);
-        const uint32_t l2 = hadd2(prmt(odl, kMagic, 0x7150), kNeg1152), l3 = hadd2(prmt(odl, kMagic, 0x7352), kNeg1152);
-        const uint32_t h0 = hadd2(prmt(evh, kMagic, 0x7150), kNeg1152), h1 = hadd2(prmt(evh, kMagic, 0x7352), kNeg1152);
-        const uint32_t h2 = hadd2(prmt(odh, kMagic, 0x7150), kNeg1152), h3 = hadd2(prmt(odh, kMagic, 0x7352), kNeg1152);
+      } else {
+        evl = xl[wd] & 0x0F0F0F0Fu; odl = (xl[wd] >> 4) & 0x0F0F0F0Fu;
+        evh = xh[wd] & 0x0F0F0F0Fu; odh = (xh[wd] >> 4) & 0x0F0F0F0Fu;
+      }
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          mma16816(s[nt], l0, h0, l2, h2, w.qf[nt][2 * wd][0], w.qf[nt][2 * wd][1]);
-          mma16816(s[nt], l1, h1, l3, h3, w.qf[nt][2 * wd + 1][0], w.qf[nt][2 * wd + 1][1]);
-        }
+      for (int nt = 0; nt < NT; ++nt) {
+        mma_u8s8(shi[nt], evl, evh, odl, odh, w.qf[nt][0][wd][0], w.qf[nt][0][wd][1]);
+        mma_u8s8(slo[nt], evl, evh, odl, odh, w.qf[nt][1][wd][0], w.qf[nt][1][wd][1]);
       }
     }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) s[nt][i] = (float)(shi[nt][i] * 128 + slo[nt][i]);
   }
 
   // ---- per-token scalars, scores in log2 units -----------------------------------------
@@ -317,7 +323,7 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
   }
   // ---- p, denominators, zero-point sums, P^T fragments ---------------------------------
   const float sv_lo = vm_lo.x * kLevelScaleV, sv_hi = vm_hi.x * kLevelScaleV;
-  const float zv_lo = fmaf(vm_lo.x, kMidK, vm_lo.y), zv_hi = fmaf(vm_hi.x, kMidK, vm_hi.y);
+  const float zv_lo = fmaf(vm_lo.x, kMidV, vm_lo.y), zv_hi = fmaf(vm_hi.x, kMidV, vm_hi.y);
   uint32_t pb[NT][2];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
@@ -524,32 +530,55 @@ attn_kernel(const AttnParams p) {
       if (lane == 0) atomicMax(misc + 1, __float_as_int(amax));
     }
     asm volatile("bar.sync 1, %0;" ::"n"(kConsThreads) : "memory");
-    // power-of-two prescale so that max|q| lands in [2^14, 2^15): FP16 then holds every BF16
-    // query value that is within 2^-29 of the largest one exactly
+    // Two s8 digit planes of q: q_int = rint(q * 2^e) with max|q| * 2^e in [2^13, 2^14), so
+    // q_int = 128 * hi + lo with hi in [-128, 127], lo in [0, 127].  BF16 values within 2^-6 of
+    // the largest are exact; smaller ones are rounded to max|q| * 2^-14 absolute.
     const float qmax = __int_as_float(misc[1]);
     int e = 0;
-    if (qmax > 0.0f && qmax < INFINITY) e = 14 - (((__float_as_int(qmax) >> 23) & 0xFF) - 127);
+    if (qmax > 0.0f && qmax < INFINITY) e = 13 - (((__float_as_int(qmax) >> 23) & 0xFF) - 127);
     e = max(-100, min(100, e));
     const float up = __int_as_float((127 + e) << 23), down = __int_as_float((127 - e) << 23);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       const int c = (cg * NT + nt) * 8 + g;  // column of this thread's B-fragment rows
-      const __nv_bfloat16* qc = q_s + c * LYNX_D;
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        const int base = 32 * t + 8 * (ks >> 1), h = ks & 1;
-        int d0, d1, d2, d3;
-        if (!FULL) { d0 = base + 2 * h; d1 = d0 + 4; d2 = d0 + 1; d3 = d0 + 5; }
-        else       { d0 = base + 4 * h; d1 = d0 + 2; d2 = d0 + 1; d3 = d0 + 3; }
-        w.qf[nt][ks][0] = pack_f16x2(__bfloat162float(qc[d0]) * up, __bfloat162float(qc[d1]) * up);
-        w.qf[nt][ks][1] = pack_f16x2(__bfloat162float(qc[d2]) * up, __bfloat162float(qc[d3]) * up);
+      for (int wd = 0; wd < 4; ++wd) {
+        const uint4 v = *reinterpret_cast<const uint4*>(q_s + c * LYNX_D + 32 * t + 8 * wd);
+        const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+        int qi[8];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          qi[2 * k] = __float2int_rn(__uint_as_float(ww[k] << 16) * up);
+          qi[2 * k + 1] = __float2int_rn(__uint_as_float(ww[k] & 0xFFFF0000u) * up);
+        }
+        uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;  // bytes for dims {0,2,4,6} / {1,3,5,7}
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          hi_e |= (uint32_t)((qi[2 * k] >> 7) & 0xFF) << (8 * k);
+          lo_e |= (uint32_t)(qi[2 * k] & 127) << (8 * k);
+          hi_o |= (uint32_t)((qi[2 * k + 1] >> 7) & 0xFF) << (8 * k);
+          lo_o |= (uint32_t)(qi[2 * k + 1] & 127) << (8 * k);
+        }
+        w.qf[nt][0][wd][0] = hi_e; w.qf[nt][0][wd][1] = hi_o;
+        w.qf[nt][1][wd][0] = lo_e; w.qf[nt][1][wd][1] = lo_o;
       }
 #pragma unroll
       for (int cc = 0; cc < 2; ++cc) {
         const int col = (cg * NT + nt) * 8 + 2 * t + cc;  // column of this thread's C-fragment
-        const __nv_bfloat16* qq = q_s + col * LYNX_D;
+        // sum over d of q_d: this lane adds dims [16g, 16g+16), the 8 lanes sharing t add up
+        const uint4* qq = reinterpret_cast<const uint4*>(q_s + col * LYNX_D + 16 * g);
         float sum = 0.0f;
-        for (int d = 0; d < LYNX_D; ++d) sum += __bfloat162float(qq[d]);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint4 v = qq[h];
+          const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            sum += __uint_as_float(ww[k] << 16) + __uint_as_float(ww[k] & 0xFFFF0000u);
+        }
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 4);
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 8);
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 16);
         w.qs[nt][cc] = sum;
         const int j = col / p.G;
         w.lim[nt][cc] = col < p.ncols ? (p.causal ? len - p.nq + j + 1 : len) : 0;
