@@ -13,7 +13,8 @@
 // s8 digit planes of the query); P.V runs in FP16 with centred levels (a-8 for the Anchor
 // state, code-128 for the full state) so that no large bias enters the FP32 accumulation.
 //
-// Kernel shape.  Grid = (chunk, KV head, sequence): flash-decoding split-K over the context.
+// Kernel shape.  Persistent grid (a few CTAs per SM), flash-decoding split-K in stream-K form:
+// the (sequence, KV head, 64-token unit) list is cut into equal contiguous ranges, one per CTA.
 // A CTA has TW*CG consumer warps and one producer warp.  The producer streams 16-token
 // sub-blocks (1 KiB per plane + 128 B of meta, each contiguous in the paged layout) into a
 // shared-memory ring with cp.async.bulk (TMA, 1-D) completing on mbarriers.  Consumer warp
@@ -24,9 +25,10 @@
 //   O^T[128 dim x 8 col] += level(V)^T[128 x 16 tok] . P^T  mma.m16n8k16 f16, dims are M
 // K operands are the nibbles / merged codes themselves (one or two logic ops per 4 levels);
 // V operands are built from the nibbles with LOP3/PRMT and one FP16 add/fma per pair.
-// Partials (m, l, O) are merged across the CTA's token warps in shared memory, written to the
-// workspace, and the last CTA of a (sequence, KV head) (atomic ticket, no waiting) merges the
-// chunks; for verification the last CTA of a sequence also takes the accept/reject decision.
+// Partials (m, l, O) are merged across the CTA's token warps register-wise through shared
+// memory; a range that covers a whole (sequence, KV head) writes the output directly, otherwise
+// the partial goes to the workspace and the last contributor (atomic ticket, no waiting) merges
+// them; for verification the last CTA of a sequence also takes the accept/reject decision.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -37,7 +39,6 @@ namespace {
 
 constexpr int kMaxQ = 16;          // query positions per call
 constexpr int kMaxCols = 64;       // n_q * G
-constexpr int kMaxChunkTokens = 4096;
 constexpr int kPartStride = 132;   // floats per (chunk, column) partial: O[128], m, l, pad
 
 struct AttnParams {
@@ -54,10 +55,10 @@ struct AttnParams {
   uint32_t* ws_chunk_ctr;  // [B*Hkv]
   uint32_t* ws_seq_ctr;    // [B]
   float* ws_dev;           // [B*Hkv][kMaxQ]
-  float* ws_part;          // [B*Hkv][max_chunks][ncols_pad][kPartStride]
+  float* ws_part;          // [B*Hkv + CTAs][ncols_pad][kPartStride], slot = segment + CTA index
   float atol, rtol;
   float sm_log2;           // softmax_scale * log2(e)
-  int B, nq, causal, Hq, Hkv, G, bt, num_blocks, max_blocks, chunk_tokens, max_chunks, ncols;
+  int B, nq, causal, Hq, Hkv, G, bt, num_blocks, max_blocks, ncols;
 };
 
 // ------------------------------------------------------------------ PTX helpers
@@ -90,9 +91,12 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait: gives up after ~2 s (or as soon as another thread of the CTA gave up), records
-// it in the CTA's abort word and returns false.  Nothing in this kernel waits on another CTA.
+// Bounded wait: gives up after ~2 s (at once if another thread of the CTA already gave up),
+// records it in the CTA's abort word and returns false.  Callers carry on without the data (every
+// loop has a fixed trip count, so the kernel still ends) and the host is told through the
+// workspace status word.  Nothing in this kernel waits on another CTA.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_word) {
+  if (*abort_word) return false;
   const uint64_t t0 = globaltimer_ns();
   for (;;) {
     for (int i = 0; i < 256; ++i)
@@ -398,24 +402,41 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
   }
 }
 
+constexpr int kPieceUnits = 64;  // stage-units whose block ids are looked up at a time
+
 template <bool FULL, int NT, int TW, int CG, int NSTAGE>
 struct Cfg {
-  static constexpr int kST = TW * 16;                       // tokens per stage
+  static constexpr int kST = TW * 16;                       // tokens per stage-unit
   static constexpr int kSubBytes = FULL ? 16 * 272 : 16 * 144;
   static constexpr int kStageBytes = kST * (FULL ? 272 : 144);
   static constexpr int kConsWarps = TW * CG;
+  static constexpr int kConsThreads = kConsWarps * 32;
   static constexpr int kThreads = (kConsWarps + 1) * 32;
   static constexpr int kColsPad = CG * NT * 8;
   static constexpr int kRing = NSTAGE * kStageBytes;
-  static constexpr int kMergeBytes = kConsWarps * NT * 8 * kPartStride * 4;
-  static constexpr int kRingAlloc = kRing > kMergeBytes ? kRing : kMergeBytes;
-  static constexpr int kQBytes = kColsPad * LYNX_D * 2;
-  static constexpr int kBlkBytes = (kMaxChunkTokens / 16) * 4;
-  static constexpr int kBarBytes = 2 * NSTAGE * 8;
-  static constexpr int kMiscBytes = 128;   // 8 control words + kMaxQ deviation words
-  static constexpr int kSmem = kRingAlloc + kQBytes + kBlkBytes + kBarBytes + kMiscBytes;
+  static constexpr int kMailRegs = 38 * NT;                 // o[NT][8][4] + m, l, zs [NT][2]
+  static constexpr int kMailBytes = CG * kMailRegs * 32 * 4;  // one mailbox per column group
+  static constexpr int kQBytes = 2 * kColsPad * LYNX_D * 2; // two item slots
+  static constexpr int kBlkBytes = kPieceUnits * TW * 4;
+  static constexpr int kInfoBytes = NSTAGE * 16 + 2 * 32;   // int4 per stage + two item records
+  static constexpr int kBarBytes = (2 * NSTAGE + 4) * 8;
+  static constexpr int kMiscBytes = 256;
+  static constexpr int kSmem = kRing + kMailBytes + kQBytes + kBlkBytes + kInfoBytes + kBarBytes + kMiscBytes;
 };
 
+struct Item {  // one piece: a run of stage-units of one (sequence, KV head) given to one CTA
+  int b, hkv, len, first_cta, n_contrib, pad0, pad1, pad2;
+};
+
+__device__ __forceinline__ void named_bar(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// Persistent, stream-K style kernel.  The work is the list of stage-units (ST tokens of one
+// (sequence, KV head)) in (sequence, head, position) order; CTA i owns the contiguous range
+// [i*q, (i+1)*q) of it, q = ceil(total / gridDim.x).  A range is cut into pieces at segment
+// boundaries; each piece is one online-softmax pass whose result goes to the output directly
+// (the segment lies inside the range) or to a partial slot that the last contributor merges.
 template <bool FULL, int NT, int TW, int CG, int NSTAGE, int MINB>
 __global__ void __launch_bounds__((TW * CG + 1) * 32, MINB)
 attn_kernel(const AttnParams p) {
@@ -423,25 +444,24 @@ attn_kernel(const AttnParams p) {
   constexpr int ST = C::kST;
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* ring = smem;
-  __nv_bfloat16* q_s = reinterpret_cast<__nv_bfloat16*>(smem + C::kRingAlloc);
-  uint32_t* blk_s = reinterpret_cast<uint32_t*>(smem + C::kRingAlloc + C::kQBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kRingAlloc + C::kQBytes + C::kBlkBytes);
-  int* misc = reinterpret_cast<int*>(smem + C::kRingAlloc + C::kQBytes + C::kBlkBytes + C::kBarBytes);
-  // misc[0] = abort word, misc[1] = max |q| bits, misc[2] = "this CTA is last" flag, misc[8..] dev
-
+  float* mail = reinterpret_cast<float*>(smem + C::kRing);
+  __nv_bfloat16* q_s = reinterpret_cast<__nv_bfloat16*>(smem + C::kRing + C::kMailBytes);
+  uint32_t* blk_s = reinterpret_cast<uint32_t*>(smem + C::kRing + C::kMailBytes + C::kQBytes);
+  int4* info_s = reinterpret_cast<int4*>(smem + C::kRing + C::kMailBytes + C::kQBytes + C::kBlkBytes);
+  Item* items = reinterpret_cast<Item*>(info_s + NSTAGE);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kRing + C::kMailBytes + C::kQBytes +
+                                               C::kBlkBytes + C::kInfoBytes);
+  int* misc = reinterpret_cast<int*>(smem + C::kRing + C::kMailBytes + C::kQBytes + C::kBlkBytes +
+                                     C::kInfoBytes + C::kBarBytes);
+  // misc[0] abort word, [1] "last contributor" flag, [2..3] total units (int64), [4] units per
+  // CTA, [5] first sequence of this CTA's range, [6] unit offset inside that sequence,
+  // [7] number of units of this CTA, [16..31] per-position deviations
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int chunk = blockIdx.x, hkv = blockIdx.y, b = blockIdx.z;
+  const int n_cta = gridDim.x, cta = blockIdx.x;
   const int cap = p.max_blocks * p.bt;
-  int len = p.seq_lens[b];
-  len = len < 0 ? 0 : (len > cap ? cap : len);
-  const int nchunks = len > 0 ? (len + p.chunk_tokens - 1) / p.chunk_tokens : 1;
-  if (chunk >= nchunks) return;
-  const int t_begin = chunk * p.chunk_tokens;
-  const int t_end = min(len, t_begin + p.chunk_tokens);
-  const int n_sub = (t_end - t_begin + 15) >> 4;
-  const int n_stage = (n_sub + TW - 1) / TW;
   const uint32_t ring_u32 = smem_u32(ring);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + NSTAGE * 8;
+  const uint32_t qfull0 = empty0 + NSTAGE * 8, qempty0 = qfull0 + 16;
   volatile int* abort_word = misc;
 
   if (tid == 0) {
@@ -449,75 +469,201 @@ attn_kernel(const AttnParams p) {
       mbar_init(full0 + i * 8, 1);
       mbar_init(empty0 + i * 8, C::kConsWarps);
     }
-    misc[0] = 0; misc[1] = 0; misc[2] = 0;
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(qfull0 + i * 8, 1);
+      mbar_init(qempty0 + i * 8, C::kConsWarps);
+    }
+    misc[0] = 0; misc[1] = 0; misc[7] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // padded query columns must read as zero: clear both item slots once
+  for (int i = tid; i < C::kQBytes / 16; i += C::kThreads) reinterpret_cast<uint4*>(q_s)[i] = make_uint4(0, 0, 0, 0);
+  // make the generic-proxy zeros visible to later async-proxy (TMA) writes of the same bytes
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
 
+  auto clamp_len = [&](int b) {
+    int len = __ldg(p.seq_lens + b);
+    return len < 0 ? 0 : (len > cap ? cap : len);
+  };
+
+  if (warp == C::kConsWarps) {
+    // ---- prologue (producer warp): total work, this CTA's range, empty sequences ----------
+    long long tot = 0;
+    for (int b = lane; b < p.B; b += 32) tot += (clamp_len(b) + ST - 1) / ST;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) tot += __shfl_xor_sync(0xFFFFFFFFu, tot, off);
+    const long long T = tot * p.Hkv;
+    const long long q = (T + n_cta - 1) / n_cta;
+    const long long lo = (long long)cta * q, hi = (lo + q < T) ? lo + q : T;
+    int b_lo = 0;
+    long long off_lo = 0;
+    if (lo < hi) {
+      long long running = 0;
+      for (int b0 = 0; b0 < p.B; b0 += 32) {
+        const int b = b0 + lane;
+        const long long u = b < p.B ? (long long)p.Hkv * ((clamp_len(b) + ST - 1) / ST) : 0;
+        long long incl = u;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const long long v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+          if (lane >= o) incl += v;
+        }
+        const long long excl = running + incl - u;
+        const bool hit = u > 0 && lo >= excl && lo < excl + u;
+        const unsigned m = __ballot_sync(0xFFFFFFFFu, hit);
+        if (m) {
+          const int src = __ffs(m) - 1;
+          b_lo = b0 + src;
+          off_lo = lo - __shfl_sync(0xFFFFFFFFu, excl, src);
+          break;
+        }
+        running += __shfl_sync(0xFFFFFFFFu, incl, 31);
+      }
+    }
+    if (lane == 0) {
+      misc[4] = (int)(q > 0x7FFFFFFF ? 0x7FFFFFFF : q);
+      misc[7] = lo < hi ? (int)(hi - lo) : 0;
+    }
+    // sequences with no token: outputs are zero, nothing is rejected unless the draft is not zero
+    for (int b = cta; b < p.B; b += n_cta) {
+      if (clamp_len(b) != 0) continue;
+      const size_t n = (size_t)p.nq * p.Hq * LYNX_D;
+      for (size_t i = lane; i < n; i += 32) p.out[(size_t)b * n + i] = 0.0f;
+      if (FULL && p.draft != nullptr) {
+        int fr = p.nq;
+        for (int j = p.nq - 1; j >= 0; --j) {
+          float worst = 0.0f;
+          for (int i = lane; i < p.Hq * LYNX_D; i += 32)
+            worst = fmaxf(worst, fabsf(__ldg(p.draft + ((size_t)b * p.nq + j) * p.Hq * LYNX_D + i)) / p.atol);
+#pragma unroll
+          for (int off = 16; off >= 1; off >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xFFFFFFFFu, worst, off));
+          if (lane == 0) p.dev[(size_t)b * p.nq + j] = worst;
+          if (worst > 1.0f) fr = j;
+        }
+        if (lane == 0) p.first_reject[b] = fr;
+      }
+    }
+    __syncthreads();  // (A) the range is published
+    const int n_units = (int)(lo < hi ? hi - lo : 0);
+    if (n_units == 0) return;
+
+    // =============================== producer loop ===============================
+    constexpr int NARR = FULL ? 6 : 4;
+    int b = b_lo, len = clamp_len(b), U = (len + ST - 1) / ST;
+    int hkv = (int)(off_lo / U), u = (int)(off_lo % U);
+    int remaining = n_units, gs = 0, ic = 0;
+    while (remaining > 0) {
+      const int n = min(remaining, U - u);
+      const int qi = ic & 1;
+      if (ic >= 2) mbar_wait(qempty0 + qi * 8, ((ic >> 1) - 1) & 1, abort_word);
+      const long long seg0 = lo + (n_units - remaining) - u;  // first unit of this segment
+      if (lane == 0) {
+        Item it;
+        it.b = b; it.hkv = hkv; it.len = len;
+        it.first_cta = (int)(seg0 / q);
+        it.n_contrib = (int)((seg0 + U - 1) / q) - it.first_cta + 1;
+        it.pad0 = it.pad1 = it.pad2 = 0;
+        items[qi] = it;
+        mbar_expect_tx(qfull0 + qi * 8, (uint32_t)(p.nq * p.G * LYNX_D * 2));
+      }
+      __syncwarp();
+      for (int j = lane; j < p.nq; j += 32)
+        bulk_g2s(smem_u32(q_s + ((size_t)qi * C::kColsPad + j * p.G) * LYNX_D),
+                 p.q + (((size_t)b * p.nq + j) * p.Hq + (size_t)hkv * p.G) * LYNX_D,
+                 (uint32_t)(p.G * LYNX_D * 2), qfull0 + qi * 8);
+      for (int c0 = 0; c0 < n; c0 += kPieceUnits) {
+        const int cn = min(kPieceUnits, n - c0);
+        for (int i = lane; i < cn * TW; i += 32) {
+          const int t0 = (u + c0) * ST + i * 16;
+          uint32_t row = 0;
+          if (t0 < len) {
+            int blk = __ldg(p.block_table + (size_t)b * p.max_blocks + t0 / p.bt);
+            if (blk < 0 || blk >= p.num_blocks) {
+              atomicOr(p.ws_flags, kFlagBadBlock);
+              blk = blk < 0 ? 0 : p.num_blocks - 1;
+            }
+            row = (uint32_t)(((size_t)blk * p.Hkv + hkv) * p.bt + (t0 % p.bt));
+          }
+          blk_s[i] = row;
+        }
+        __syncwarp();
+        for (int k = 0; k < cn; ++k, ++gs) {
+          const int slot = gs % NSTAGE;
+          if (gs >= NSTAGE) mbar_wait(empty0 + slot * 8, ((gs / NSTAGE) - 1) & 1, abort_word);
+          const int uu = u + c0 + k;
+          const int nsub = min(TW, (len - uu * ST + 15) >> 4);
+          const uint32_t bar = full0 + slot * 8;
+          if (lane == 0) {
+            info_s[slot] = make_int4(qi, uu, (c0 + k == 0 ? 1 : 0) | (c0 + k == n - 1 ? 2 : 0), 0);
+            mbar_expect_tx(bar, nsub * C::kSubBytes);
+          }
+          __syncwarp();
+          const uint32_t stage = ring_u32 + slot * C::kStageBytes;
+          for (int idx = lane; idx < nsub * NARR; idx += 32) {
+            const int sub = idx / NARR, arr = idx - sub * NARR;
+            const size_t row = blk_s[k * TW + sub];
+            switch (arr) {
+              case 0: bulk_g2s(stage + sub * 1024, p.ka + row * 64, 1024, bar); break;
+              case 1: bulk_g2s(stage + ST * 64 + sub * 1024, p.va + row * 64, 1024, bar); break;
+              case 2: bulk_g2s(stage + (FULL ? ST * 256 : ST * 128) + sub * 128, p.km + row * 2, 128, bar); break;
+              case 3: bulk_g2s(stage + (FULL ? ST * 264 : ST * 136) + sub * 128, p.vm + row * 2, 128, bar); break;
+              case 4: bulk_g2s(stage + ST * 128 + sub * 1024, p.kr + row * 64, 1024, bar); break;
+              default: bulk_g2s(stage + ST * 192 + sub * 1024, p.vr + row * 64, 1024, bar); break;
+            }
+          }
+        }
+        __syncwarp();  // blk_s is rewritten by the next round
+      }
+      remaining -= n;
+      u += n;
+      ++ic;
+      if (u == U && remaining > 0) {
+        u = 0;
+        if (++hkv == p.Hkv) {
+          hkv = 0;
+          do {
+            ++b;
+            len = b < p.B ? clamp_len(b) : 0;
+            U = (len + ST - 1) / ST;
+          } while (b < p.B && U == 0);
+          if (b >= p.B) break;  // cannot happen: the range ends inside the list
+        }
+      }
+    }
+    return;
+  }
+
+  // =============================== consumer warps ==============================
+  __syncthreads();  // (A)
+  const int n_units = misc[7];
+  if (n_units == 0) return;
+  const long long q_units = misc[4];
+  (void)q_units;
   WarpState<FULL, NT> w;
   const int g = lane >> 2, t = lane & 3;
   const int tw = warp % TW, cg = warp / TW;
+  const float cb = p.sm_log2;
+  float ca = 0.0f;
+  int len = 0, full_lim = 0, ic = 0;
+  Item item;
+  item.b = 0; item.hkv = 0; item.len = 0; item.first_cta = 0; item.n_contrib = 1;
 
-  if (warp == C::kConsWarps) {
-    // =============================== producer warp ===============================
-    for (int i = lane; i < n_sub; i += 32) {
-      const int t0 = t_begin + i * 16;
-      int blk = __ldg(p.block_table + (size_t)b * p.max_blocks + t0 / p.bt);
-      if (blk < 0 || blk >= p.num_blocks) {
-        atomicOr(p.ws_flags, kFlagBadBlock);
-        blk = blk < 0 ? 0 : p.num_blocks - 1;
-      }
-      blk_s[i] = (uint32_t)(((size_t)blk * p.Hkv + hkv) * p.bt + (t0 % p.bt));
-    }
-    __syncwarp();
-    constexpr int NARR = FULL ? 6 : 4;
-    int issued = 0;
-    for (int s = 0; s < n_stage; ++s) {
-      const int slot = s % NSTAGE;
-      if (s >= NSTAGE && !mbar_wait(empty0 + slot * 8, ((s / NSTAGE) - 1) & 1, abort_word)) break;
-      if (*abort_word) break;
-      const int nsub = min(TW, n_sub - s * TW);
-      const uint32_t bar = full0 + slot * 8;
-      if (lane == 0) mbar_expect_tx(bar, nsub * C::kSubBytes);
-      __syncwarp();
-      const uint32_t stage = ring_u32 + slot * C::kStageBytes;
-      for (int idx = lane; idx < nsub * NARR; idx += 32) {
-        const int sub = idx / NARR, arr = idx - sub * NARR;
-        const size_t row = blk_s[s * TW + sub];
-        switch (arr) {
-          case 0: bulk_g2s(stage + sub * 1024, p.ka + row * 64, 1024, bar); break;
-          case 1: bulk_g2s(stage + ST * 64 + sub * 1024, p.va + row * 64, 1024, bar); break;
-          case 2: bulk_g2s(stage + (FULL ? ST * 256 : ST * 128) + sub * 128, p.km + row * 2, 128, bar); break;
-          case 3: bulk_g2s(stage + (FULL ? ST * 264 : ST * 136) + sub * 128, p.vm + row * 2, 128, bar); break;
-          case 4: bulk_g2s(stage + ST * 128 + sub * 1024, p.kr + row * 64, 1024, bar); break;
-          default: bulk_g2s(stage + ST * 192 + sub * 1024, p.vr + row * 64, 1024, bar); break;
-        }
-      }
-      issued = s + 1;
-    }
-    if (*abort_word && lane == 0) {
-      // gave up: let the copies already issued land before the CTA's memory is reused
-      atomicOr(p.ws_flags, kFlagTimeout);
-      const uint64_t t0 = globaltimer_ns();
-      for (int s = max(0, issued - NSTAGE); s < issued; ++s)
-        while (!mbar_try_wait(full0 + (s % NSTAGE) * 8, (s / NSTAGE) & 1) &&
-               globaltimer_ns() - t0 < 1000000000ull) {}
-    }
-  } else {
-    // =============================== consumer warps ==============================
-    // stage Q of this (sequence, KV head): columns c = j*G + hh
-    constexpr int kConsThreads = C::kConsWarps * 32;
-    {
+  for (int gs = 0; gs < n_units; ++gs) {
+    const int slot = gs % NSTAGE;
+    mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
+    const int4 info = info_s[slot];
+    if (info.z & 1) {
+      // ---- a new piece: queries, digit planes, fresh softmax state -----------------------
+      const int qi = info.x & 1;
+      mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
+      item = items[qi];
+      len = item.len;
+      full_lim = p.causal ? len - p.nq + 1 : len;
+      const __nv_bfloat16* qb = q_s + (size_t)qi * C::kColsPad * LYNX_D;
       float amax = 0.0f;
-      for (int i = tid; i < C::kColsPad * (LYNX_D / 8); i += kConsThreads) {
-        const int c = i / (LYNX_D / 8), part = i % (LYNX_D / 8);
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (c < p.ncols) {
-          const int j = c / p.G, hh = c % p.G;
-          const size_t qrow = ((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh;
-          v = __ldg(reinterpret_cast<const uint4*>(p.q + qrow * LYNX_D) + part);
-        }
-        reinterpret_cast<uint4*>(q_s)[i] = v;
+      for (int i = lane; i < C::kColsPad * (LYNX_D / 8); i += 32) {
+        const uint4 v = reinterpret_cast<const uint4*>(qb)[i];
         const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -527,209 +673,248 @@ attn_kernel(const AttnParams p) {
       }
 #pragma unroll
       for (int off = 16; off >= 1; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, off));
-      if (lane == 0) atomicMax(misc + 1, __float_as_int(amax));
-    }
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsThreads) : "memory");
-    // Two s8 digit planes of q: q_int = rint(q * 2^e) with max|q| * 2^e in [2^13, 2^14), so
-    // q_int = 128 * hi + lo with hi in [-128, 127], lo in [0, 127].  BF16 values within 2^-6 of
-    // the largest are exact; smaller ones are rounded to max|q| * 2^-14 absolute.
-    const float qmax = __int_as_float(misc[1]);
-    int e = 0;
-    if (qmax > 0.0f && qmax < INFINITY) e = 13 - (((__float_as_int(qmax) >> 23) & 0xFF) - 127);
-    e = max(-100, min(100, e));
-    const float up = __int_as_float((127 + e) << 23), down = __int_as_float((127 - e) << 23);
+      // Two s8 digit planes of q: q_int = rint(q * 2^e) with max|q| * 2^e in [2^13, 2^14), so
+      // q_int = 128 * hi + lo with hi in [-128, 127], lo in [0, 127].  BF16 values within 2^-6
+      // of the largest are exact; smaller ones are rounded to max|q| * 2^-14 absolute.
+      int e = 0;
+      if (amax > 0.0f && amax < INFINITY) e = 13 - (((__float_as_int(amax) >> 23) & 0xFF) - 127);
+      e = max(-100, min(100, e));
+      const float up = __int_as_float((127 + e) << 23), down = __int_as_float((127 - e) << 23);
+      ca = p.sm_log2 * down * (FULL ? 1.0f : 16.0f);  // per level unit of the K dot product
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const int c = (cg * NT + nt) * 8 + g;  // column of this thread's B-fragment rows
+      for (int nt = 0; nt < NT; ++nt) {
+        const int c = (cg * NT + nt) * 8 + g;  // column of this thread's B-fragment rows
 #pragma unroll
-      for (int wd = 0; wd < 4; ++wd) {
-        const uint4 v = *reinterpret_cast<const uint4*>(q_s + c * LYNX_D + 32 * t + 8 * wd);
-        const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
-        int qi[8];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          qi[2 * k] = __float2int_rn(__uint_as_float(ww[k] << 16) * up);
-          qi[2 * k + 1] = __float2int_rn(__uint_as_float(ww[k] & 0xFFFF0000u) * up);
-        }
-        uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;  // bytes for dims {0,2,4,6} / {1,3,5,7}
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          hi_e |= (uint32_t)((qi[2 * k] >> 7) & 0xFF) << (8 * k);
-          lo_e |= (uint32_t)(qi[2 * k] & 127) << (8 * k);
-          hi_o |= (uint32_t)((qi[2 * k + 1] >> 7) & 0xFF) << (8 * k);
-          lo_o |= (uint32_t)(qi[2 * k + 1] & 127) << (8 * k);
-        }
-        w.qf[nt][0][wd][0] = hi_e; w.qf[nt][0][wd][1] = hi_o;
-        w.qf[nt][1][wd][0] = lo_e; w.qf[nt][1][wd][1] = lo_o;
-      }
-#pragma unroll
-      for (int cc = 0; cc < 2; ++cc) {
-        const int col = (cg * NT + nt) * 8 + 2 * t + cc;  // column of this thread's C-fragment
-        // sum over d of q_d: this lane adds dims [16g, 16g+16), the 8 lanes sharing t add up
-        const uint4* qq = reinterpret_cast<const uint4*>(q_s + col * LYNX_D + 16 * g);
-        float sum = 0.0f;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const uint4 v = qq[h];
+        for (int wd = 0; wd < 4; ++wd) {
+          const uint4 v = *reinterpret_cast<const uint4*>(qb + c * LYNX_D + 32 * t + 8 * wd);
           const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+          int qv[8];
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            sum += __uint_as_float(ww[k] << 16) + __uint_as_float(ww[k] & 0xFFFF0000u);
+          for (int k = 0; k < 4; ++k) {
+            qv[2 * k] = __float2int_rn(__uint_as_float(ww[k] << 16) * up);
+            qv[2 * k + 1] = __float2int_rn(__uint_as_float(ww[k] & 0xFFFF0000u) * up);
+          }
+          uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;  // bytes for dims {0,2,4,6} / {1,3,5,7}
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            hi_e |= (uint32_t)((qv[2 * k] >> 7) & 0xFF) << (8 * k);
+            lo_e |= (uint32_t)(qv[2 * k] & 127) << (8 * k);
+            hi_o |= (uint32_t)((qv[2 * k + 1] >> 7) & 0xFF) << (8 * k);
+            lo_o |= (uint32_t)(qv[2 * k + 1] & 127) << (8 * k);
+          }
+          w.qf[nt][0][wd][0] = hi_e; w.qf[nt][0][wd][1] = hi_o;
+          w.qf[nt][1][wd][0] = lo_e; w.qf[nt][1][wd][1] = lo_o;
         }
-        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 4);
-        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 8);
-        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 16);
-        w.qs[nt][cc] = sum;
-        const int j = col / p.G;
-        w.lim[nt][cc] = col < p.ncols ? (p.causal ? len - p.nq + j + 1 : len) : 0;
-        w.m[nt][cc] = -1.0e30f;
-        w.l[nt][cc] = 0.0f;
-        w.zs[nt][cc] = 0.0f;
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+          const int col = (cg * NT + nt) * 8 + 2 * t + cc;  // column of this thread's C-fragment
+          // sum over d of q_d: this lane adds dims [16g, 16g+16), the 8 lanes sharing t add up
+          const uint4* qq = reinterpret_cast<const uint4*>(qb + col * LYNX_D + 16 * g);
+          float sum = 0.0f;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const uint4 v = qq[h];
+            const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              sum += __uint_as_float(ww[k] << 16) + __uint_as_float(ww[k] & 0xFFFF0000u);
+          }
+          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 4);
+          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 8);
+          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 16);
+          w.qs[nt][cc] = sum;
+          const int j = col / p.G;
+          w.lim[nt][cc] = col < p.ncols ? (p.causal ? len - p.nq + j + 1 : len) : 0;
+          w.m[nt][cc] = -1.0e30f;
+          w.l[nt][cc] = 0.0f;
+          w.zs[nt][cc] = 0.0f;
+        }
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) w.o[nt][mt][i] = 0.0f;
       }
-#pragma unroll
-      for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) w.o[nt][mt][i] = 0.0f;
     }
-    const float ca = p.sm_log2 * down * (FULL ? 1.0f : 16.0f);  // per level unit of the K dot
-    const float cb = p.sm_log2;
-    const int full_lim = p.causal ? len - p.nq + 1 : len;  // tokens below this are visible to all
+    const int tile_t0 = info.y * ST + tw * 16;
+    if (tile_t0 < len)
+      process_tile<FULL, NT, ST>(w, ring_u32 + slot * C::kStageBytes, tw, tile_t0,
+                                 tile_t0 + 16 > full_lim, ca, cb, g, t);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty0 + slot * 8);
+    if (!(info.z & 2)) continue;
 
-    for (int s = 0; s < n_stage; ++s) {
-      const int slot = s % NSTAGE;
-      if (!mbar_wait(full0 + slot * 8, (s / NSTAGE) & 1, abort_word)) break;
-      const int tile_t0 = t_begin + (s * TW + tw) * 16;
-      if (tile_t0 < t_end)
-        process_tile<FULL, NT, ST>(w, ring_u32 + slot * C::kStageBytes, tw, tile_t0,
-                                   tile_t0 + 16 > full_lim, ca, cb, g, t);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty0 + slot * 8);
+    // ---- end of the piece: warp 0 of the column group absorbs the other token warps one by
+    //      one (register-wise, through a lane-private mailbox), then writes the result --------
+    for (int src = 1; src < TW; ++src) {
+      float* box = mail + (size_t)cg * C::kMailRegs * 32 + lane;
+      if (tw == src) {
+        int r = 0;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+          for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) box[(r++) * 32] = w.o[nt][mt][i];
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            box[(r++) * 32] = w.m[nt][cc];
+            box[(r++) * 32] = w.l[nt][cc];
+            box[(r++) * 32] = w.zs[nt][cc];
+          }
+        }
+      }
+      named_bar(2 + cg, TW * 32);
+      if (tw == 0) {
+        int r = 0;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          float f1[2], f2[2];
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            const float m2 = box[(38 * nt + 32 + 3 * cc) * 32];
+            const float M = fmaxf(w.m[nt][cc], m2);
+            f1[cc] = ex2(w.m[nt][cc] - M);
+            f2[cc] = ex2(m2 - M);
+            w.m[nt][cc] = M;
+          }
+#pragma unroll
+          for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float o2 = box[(r++) * 32];
+              w.o[nt][mt][i] = w.o[nt][mt][i] * f1[i & 1] + o2 * f2[i & 1];
+            }
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            r++;  // m (already used)
+            const float l2 = box[(r++) * 32];
+            const float z2 = box[(r++) * 32];
+            w.l[nt][cc] = w.l[nt][cc] * f1[cc] + l2 * f2[cc];
+            w.zs[nt][cc] = w.zs[nt][cc] * f1[cc] + z2 * f2[cc];
+          }
+        }
+      }
+      named_bar(2 + cg, TW * 32);
     }
+
+    const size_t bh = (size_t)item.b * p.Hkv + item.hkv;
+    const bool direct = item.n_contrib == 1;
+    if (tw == 0) {
+      float* part = p.ws_part + (bh + (size_t)cta) * (size_t)C::kColsPad * kPartStride;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+          float l = w.l[nt][cc], z = w.zs[nt][cc];
+#pragma unroll
+          for (int off = 4; off <= 16; off <<= 1) {
+            l += __shfl_xor_sync(0xFFFFFFFFu, l, off);
+            z += __shfl_xor_sync(0xFFFFFFFFu, z, off);
+          }
+          const int c = (cg * NT + nt) * 8 + 2 * t + cc;
+          if (c >= p.ncols) continue;
+          if (direct) {
+            const int j = c / p.G, hh = c % p.G;
+            float* dst = p.out + (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D;
+            const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+              const int d = 16 * g + 8 * (mt >> 2) + 2 * (mt & 3);
+              *reinterpret_cast<float2*>(dst + d) =
+                  make_float2((w.o[nt][mt][cc] + z) * inv, (w.o[nt][mt][cc + 2] + z) * inv);
+            }
+          } else {
+            float* dst = part + (size_t)c * kPartStride;
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+              const int d = 16 * g + 8 * (mt >> 2) + 2 * (mt & 3);
+              *reinterpret_cast<float2*>(dst + d) = make_float2(w.o[nt][mt][cc] + z, w.o[nt][mt][cc + 2] + z);
+            }
+            if (g == 0) { dst[128] = w.m[nt][cc]; dst[129] = l; }
+          }
+        }
+      }
+      __threadfence();
+    }
+    bool final_here = direct;
+    if (!direct) {
+      // the last contributor of this (sequence, KV head) merges the partial slots
+      named_bar(1, C::kConsThreads);
+      if (tid == 0)
+        misc[1] = (atomicInc(p.ws_chunk_ctr + bh, (uint32_t)item.n_contrib - 1) == (uint32_t)item.n_contrib - 1);
+      named_bar(1, C::kConsThreads);
+      final_here = misc[1] != 0;
+      if (final_here) {
+        __threadfence();
+        const float* base = p.ws_part + (bh + (size_t)item.first_cta) * (size_t)C::kColsPad * kPartStride;
+        const size_t cstride = (size_t)C::kColsPad * kPartStride;
+        for (int idx = tid; idx < C::kColsPad * LYNX_D; idx += C::kConsThreads) {
+          const int c = idx >> 7, d = idx & 127;
+          if (c >= p.ncols) continue;
+          const float* col = base + (size_t)c * kPartStride;
+          float M = -INFINITY;
+          for (int i = 0; i < item.n_contrib; ++i) M = fmaxf(M, __ldcg(col + i * cstride + 128));
+          float acc = 0.0f, L = 0.0f;
+          for (int i = 0; i < item.n_contrib; ++i) {
+            const float f = ex2(__ldcg(col + i * cstride + 128) - M);
+            acc = fmaf(__ldcg(col + i * cstride + d), f, acc);
+            L = fmaf(__ldcg(col + i * cstride + 129), f, L);
+          }
+          const int j = c / p.G, hh = c % p.G;
+          p.out[(((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
+        }
+      }
+    }
+    // accept / reject (Section 4.3): by the CTA that wrote the final outputs of this head
+    if (FULL && p.draft != nullptr) {
+      int* devs = misc + 16;
+      named_bar(1, C::kConsThreads);  // final outputs written; devs free
+      if (final_here) {
+        if (tid < kMaxQ) devs[tid] = 0;
+        named_bar(1, C::kConsThreads);
+        for (int idx = tid; idx < p.ncols * LYNX_D; idx += C::kConsThreads) {
+          const int c = idx >> 7, d = idx & 127;
+          const int j = c / p.G, hh = c % p.G;
+          const size_t o = (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + d;
+          const float f = p.out[o], dr = __ldg(p.draft + o);
+          const float r = fabsf(f - dr) / (p.atol + p.rtol * fabsf(f));
+          atomicMax(devs + j, __float_as_int(r));  // r >= 0: integer order = float order
+        }
+        named_bar(1, C::kConsThreads);
+        if (tid < p.nq) p.ws_dev[bh * kMaxQ + tid] = __int_as_float(devs[tid]);
+        __threadfence();
+        named_bar(1, C::kConsThreads);
+        if (tid == 0)
+          misc[1] = (atomicInc(p.ws_seq_ctr + item.b, (uint32_t)p.Hkv - 1) == (uint32_t)p.Hkv - 1);
+        named_bar(1, C::kConsThreads);
+        if (misc[1] && tid == 0) {
+          __threadfence();
+          int fr = p.nq;
+          for (int j = p.nq - 1; j >= 0; --j) {
+            float worst = 0.0f;
+            for (int h = 0; h < p.Hkv; ++h)
+              worst = fmaxf(worst, __ldcg(p.ws_dev + ((size_t)item.b * p.Hkv + h) * kMaxQ + j));
+            p.dev[(size_t)item.b * p.nq + j] = worst;
+            if (worst > 1.0f) fr = j;
+          }
+          p.first_reject[item.b] = fr;
+        }
+      }
+      named_bar(1, C::kConsThreads);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(qempty0 + (info.x & 1) * 8);
+    ++ic;
   }
-
-  __syncthreads();  // ring is free from here on: reuse it for the CTA-level merge
   if (tid == 0 && misc[0]) atomicOr(p.ws_flags, kFlagTimeout);
-  float* mbuf = reinterpret_cast<float*>(ring);
-  if (warp < C::kConsWarps) {
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-      for (int cc = 0; cc < 2; ++cc) {
-        float l = w.l[nt][cc], z = w.zs[nt][cc];
-#pragma unroll
-        for (int off = 4; off <= 16; off <<= 1) {
-          l += __shfl_xor_sync(0xFFFFFFFFu, l, off);
-          z += __shfl_xor_sync(0xFFFFFFFFu, z, off);
-        }
-        float* dst = mbuf + ((size_t)warp * NT * 8 + nt * 8 + 2 * t + cc) * kPartStride;
-#pragma unroll
-        for (int mt = 0; mt < 8; ++mt) {
-          const int d = 16 * g + 8 * (mt >> 2) + 2 * (mt & 3);
-          dst[d] = w.o[nt][mt][cc] + z;
-          dst[d + 1] = w.o[nt][mt][cc + 2] + z;
-        }
-        if (g == 0) { dst[128] = w.m[nt][cc]; dst[129] = l; }
-      }
-    }
-  }
-  __syncthreads();
-
-  // merge the TW token warps of each column; write the result or a chunk partial
-  const size_t bh = (size_t)b * p.Hkv + hkv;
-  float* part = p.ws_part + (bh * p.max_chunks + chunk) * (size_t)C::kColsPad * kPartStride;
-  for (int idx = tid; idx < C::kColsPad * LYNX_D; idx += C::kThreads) {
-    const int c = idx >> 7, d = idx & 127;
-    if (c >= p.ncols) continue;
-    const int cgi = c / (NT * 8), cl = c % (NT * 8);
-    float M = -INFINITY;
-#pragma unroll
-    for (int x = 0; x < TW; ++x)
-      M = fmaxf(M, mbuf[((size_t)(cgi * TW + x) * NT * 8 + cl) * kPartStride + 128]);
-    float acc = 0.0f, L = 0.0f;
-#pragma unroll
-    for (int x = 0; x < TW; ++x) {
-      const float* src = mbuf + ((size_t)(cgi * TW + x) * NT * 8 + cl) * kPartStride;
-      const float f = ex2(src[128] - M);
-      acc = fmaf(src[d], f, acc);
-      L = fmaf(src[129], f, L);
-    }
-    if (nchunks == 1) {
-      const int j = c / p.G, hh = c % p.G;
-      p.out[(((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
-    } else {
-      part[(size_t)c * kPartStride + d] = acc;
-      if (d == 0) { part[(size_t)c * kPartStride + 128] = M; part[(size_t)c * kPartStride + 129] = L; }
-    }
-  }
-
-  // split-K: the last CTA of this (sequence, KV head) to finish merges the chunk partials
-  if (nchunks > 1) {
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) misc[2] = (atomicInc(p.ws_chunk_ctr + bh, (uint32_t)nchunks - 1) == (uint32_t)nchunks - 1);
-    __syncthreads();
-    if (!misc[2]) return;
-    __threadfence();
-    const float* base = p.ws_part + bh * p.max_chunks * (size_t)C::kColsPad * kPartStride;
-    for (int idx = tid; idx < C::kColsPad * LYNX_D; idx += C::kThreads) {
-      const int c = idx >> 7, d = idx & 127;
-      if (c >= p.ncols) continue;
-      const float* col = base + (size_t)c * kPartStride;
-      const size_t cstride = (size_t)C::kColsPad * kPartStride;
-      float M = -INFINITY;
-      for (int i = 0; i < nchunks; ++i) M = fmaxf(M, __ldcg(col + i * cstride + 128));
-      float acc = 0.0f, L = 0.0f;
-      for (int i = 0; i < nchunks; ++i) {
-        const float f = ex2(__ldcg(col + i * cstride + 128) - M);
-        acc = fmaf(__ldcg(col + i * cstride + d), f, acc);
-        L = fmaf(__ldcg(col + i * cstride + 129), f, L);
-      }
-      const int j = c / p.G, hh = c % p.G;
-      p.out[(((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
-    }
-  }
-
-  // accept / reject (Section 4.3): only the CTA that wrote the final outputs gets here
-  if (FULL && p.draft != nullptr) {
-    __syncthreads();  // this CTA's out values are visible to all its threads
-    int* devs = misc + 8;
-    static_assert((8 + kMaxQ) * 4 <= C::kMiscBytes, "misc area too small");
-    if (tid < kMaxQ) devs[tid] = 0;
-    __syncthreads();
-    for (int idx = tid; idx < p.ncols * LYNX_D; idx += C::kThreads) {
-      const int c = idx >> 7, d = idx & 127;
-      const int j = c / p.G, hh = c % p.G;
-      const size_t o = (((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh) * LYNX_D + d;
-      const float f = p.out[o], dr = __ldg(p.draft + o);
-      const float r = fabsf(f - dr) / (p.atol + p.rtol * fabsf(f));
-      atomicMax(devs + j, __float_as_int(r));  // r >= 0: integer order = float order
-    }
-    __syncthreads();
-    if (tid < p.nq) p.ws_dev[bh * kMaxQ + tid] = __int_as_float(devs[tid]);
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) misc[2] = (atomicInc(p.ws_seq_ctr + b, (uint32_t)p.Hkv - 1) == (uint32_t)p.Hkv - 1);
-    __syncthreads();
-    if (!misc[2]) return;
-    __threadfence();
-    if (tid == 0) {
-      int fr = p.nq;
-      for (int j = p.nq - 1; j >= 0; --j) {
-        float worst = 0.0f;
-        for (int h = 0; h < p.Hkv; ++h)
-          worst = fmaxf(worst, __ldcg(p.ws_dev + ((size_t)b * p.Hkv + h) * kMaxQ + j));
-        p.dev[(size_t)b * p.nq + j] = worst;
-        if (worst > 1.0f) fr = j;
-      }
-      p.first_reject[b] = fr;
-    }
-  }
 }
 
 // ------------------------------------------------------------------ host side
+constexpr int kMaxCtasPerSm = 4;
+
 struct Plan {
   int ncols, variant;  // variant: 0: NT1 TW4 CG1; 1: NT2 TW4 CG1; 2: NT2 TW4 CG2; 3: NT2 TW2 CG4
-  int cols_pad, chunk_tokens, max_chunks;
+  int cols_pad;
   size_t off_chunk_ctr, off_seq_ctr, off_dev, off_part, bytes;
 };
 
@@ -738,7 +923,6 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
       s->num_q_heads % s->num_kv_heads != 0 || s->block_tokens <= 0 || s->block_tokens % 16 != 0 ||
       s->num_blocks <= 0 || s->max_blocks_per_seq <= 0 || B <= 0 || nq <= 0 || nq > kMaxQ)
     return false;
-  if (B > 65535 || s->num_kv_heads > 65535) return false;
   const int G = s->num_q_heads / s->num_kv_heads;
   const int ncols = nq * G;
   if (ncols > kMaxCols) return false;
@@ -748,15 +932,6 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   pl->ncols = ncols;
   pl->variant = ncols <= 8 ? 0 : ncols <= 16 ? 1 : ncols <= 32 ? 2 : 3;
   pl->cols_pad = ncols <= 8 ? 8 : ncols <= 16 ? 16 : ncols <= 32 ? 32 : 64;
-  // chunk: the largest of {4096 .. 256} that still leaves >= 6 CTAs per resident slot
-  const int64_t slots = (int64_t)sm_count() * 4;
-  int chunk = 256;
-  for (int c = 4096; c >= 256; c >>= 1) {
-    const int64_t items = (int64_t)B * s->num_kv_heads * ((cap + c - 1) / c);
-    if (items >= slots * 6) { chunk = c; break; }
-  }
-  pl->chunk_tokens = chunk;
-  pl->max_chunks = (int)((cap + chunk - 1) / chunk);
   size_t off = kWsHeaderBytes;
   pl->off_chunk_ctr = off; off += (size_t)B * s->num_kv_heads * 4;
   pl->off_seq_ctr = off;   off += (size_t)B * 4;
@@ -764,7 +939,7 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   pl->off_dev = off;       off += (size_t)B * s->num_kv_heads * kMaxQ * 4;
   off = (off + 255) & ~(size_t)255;
   pl->off_part = off;
-  off += (size_t)B * s->num_kv_heads * pl->max_chunks * pl->cols_pad * kPartStride * 4;
+  off += ((size_t)B * s->num_kv_heads + (size_t)sm_count() * kMaxCtasPerSm) * pl->cols_pad * kPartStride * 4;
   pl->bytes = off;
   return true;
 }
@@ -772,6 +947,7 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
 template <bool FULL, int NT, int TW, int CG, int NSTAGE, int MINB>
 lynx_status launch(const AttnParams& p, cudaStream_t st) {
   using C = Cfg<FULL, NT, TW, CG, NSTAGE>;
+  static_assert(MINB <= kMaxCtasPerSm, "partial slots are sized for kMaxCtasPerSm CTAs per SM");
   static_assert(MINB * (C::kSmem + 1024) <= 228 * 1024, "shared memory budget for MINB CTAs per SM");
   auto kern = attn_kernel<FULL, NT, TW, CG, NSTAGE, MINB>;
   static bool configured[64] = {false};
@@ -782,8 +958,7 @@ lynx_status launch(const AttnParams& p, cudaStream_t st) {
       return LYNX_ERR_CUDA;
     configured[dev] = true;
   }
-  dim3 grid(p.max_chunks, p.Hkv, p.B);
-  kern<<<grid, C::kThreads, C::kSmem, st>>>(p);
+  kern<<<sm_count() * MINB, C::kThreads, C::kSmem, st>>>(p);
   return launch_status();
 }
 
@@ -804,10 +979,11 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   if (full && (!K.residual || !V.residual)) return LYNX_ERR_NULL;
   if (full && draft && (!first_reject || !dev)) return LYNX_ERR_NULL;
   if (!aligned16(q) || !aligned16(K.anchor) || !aligned16(V.anchor) || !aligned16(K.meta) ||
-      !aligned16(V.meta) || !aligned16(workspace) || (full && (!aligned16(K.residual) || !aligned16(V.residual))))
+      !aligned16(V.meta) || !aligned16(workspace) || !aligned16(out) ||
+      (full && (!aligned16(K.residual) || !aligned16(V.residual))))
     return LYNX_ERR_ALIGN;
   if (workspace_bytes < pl.bytes) return LYNX_ERR_WORKSPACE;
-  if (full && draft && !(atol >= 0.0f && rtol >= 0.0f && atol + rtol > 0.0f)) return LYNX_ERR_SHAPE;
+  if (full && draft && !(atol > 0.0f && rtol >= 0.0f)) return LYNX_ERR_SHAPE;
 
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   AttnParams p;
@@ -827,19 +1003,19 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   p.B = B; p.nq = nq; p.causal = causal ? 1 : 0;
   p.Hq = shape->num_q_heads; p.Hkv = shape->num_kv_heads; p.G = p.Hq / p.Hkv;
   p.bt = shape->block_tokens; p.num_blocks = shape->num_blocks; p.max_blocks = shape->max_blocks_per_seq;
-  p.chunk_tokens = pl.chunk_tokens; p.max_chunks = pl.max_chunks; p.ncols = pl.ncols;
+  p.ncols = pl.ncols;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (!full) {
     switch (pl.variant) {
       case 0: return launch<false, 1, 4, 1, 4, 4>(p, st);
-      case 1: return launch<false, 2, 4, 1, 5, 3>(p, st);
-      case 2: return launch<false, 2, 4, 2, 8, 1>(p, st);
-      default: return launch<false, 2, 2, 4, 16, 1>(p, st);
+      case 1: return launch<false, 2, 4, 1, 4, 3>(p, st);
+      case 2: return launch<false, 2, 4, 2, 6, 1>(p, st);
+      default: return launch<false, 2, 2, 4, 12, 1>(p, st);
     }
   }
   switch (pl.variant) {
-    case 0: return launch<true, 1, 4, 1, 3, 4>(p, st);
-    case 1: return launch<true, 2, 4, 1, 4, 3>(p, st);
+    case 0: return launch<true, 1, 4, 1, 3, 3>(p, st);
+    case 1: return launch<true, 2, 4, 1, 3, 3>(p, st);
     case 2: return launch<true, 2, 4, 2, 5, 1>(p, st);
     default: return launch<true, 2, 2, 4, 8, 1>(p, st);
   }
