@@ -185,14 +185,27 @@ constexpr uint32_t kSixteenth = 0x2C002C00u;  // 1/16
 constexpr uint32_t kNeg72 = 0xD480D480u;      // -72
 constexpr uint32_t kNeg1152 = 0xE480E480u;    // -1152
 
+// (a & mask) | c in one LOP3: the mask is an immediate, c must sit in a register
+template <uint32_t kMask>
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "n"(kMask), "r"(c));
+  return d;
+}
 // Four FP16 pairs (value - 8) from the low 16 bits of each half of u: nibbles 0..3 of the low
-// half go to the low lanes, nibbles 0..3 of the high half to the high lanes.
-__device__ __forceinline__ void nib4_to_h2(uint32_t u, uint32_t (&r)[4]) {
+// half go to the low lanes, nibbles 0..3 of the high half to the high lanes.  `magic` holds
+// kMagic in a register the compiler cannot fold away (see opaque_magic).
+__device__ __forceinline__ void nib4_to_h2(uint32_t u, uint32_t magic, uint32_t (&r)[4]) {
   const uint32_t s = u >> 8;
-  r[0] = hadd2((u & 0x000F000Fu) | kMagic, kNeg1032);
-  r[1] = hfma2((u & 0x00F000F0u) | kMagic, kSixteenth, kNeg72);
-  r[2] = hadd2((s & 0x000F000Fu) | kMagic, kNeg1032);
-  r[3] = hfma2((s & 0x00F000F0u) | kMagic, kSixteenth, kNeg72);
+  r[0] = hadd2(and_or<0x000F000Fu>(u, magic), kNeg1032);
+  r[1] = hfma2(and_or<0x00F000F0u>(u, magic), kSixteenth, kNeg72);
+  r[2] = hadd2(and_or<0x000F000Fu>(s, magic), kNeg1032);
+  r[3] = hfma2(and_or<0x00F000F0u>(s, magic), kSixteenth, kNeg72);
+}
+__device__ __forceinline__ uint32_t opaque_magic() {
+  uint32_t m;
+  asm volatile("mov.u32 %0, 0x64006400;" : "=r"(m));
+  return m;
 }
 // Full codes of 8 elements from an anchor word and a residual word: ev = codes of elements
 // 0,2,4,6 (one per byte), od = codes of elements 1,3,5,7.
@@ -213,6 +226,7 @@ struct WarpState {
   float zs[NT][2];        // partial sum p * (zero + mid*scale) of V
   float o[NT][8][4];      // O^T accumulators: [n-tile][m-tile (16 dims)][c-reg]
   int lim[NT][2];         // exclusive token limit of the thread's two columns
+  bool fresh;             // no tile processed yet: the first one sets the maximum outright
 };
 
 // One 16-token tile.  st = shared address of the stage, tw = tile index within the stage,
@@ -220,7 +234,7 @@ struct WarpState {
 // tile is not visible.
 template <bool FULL, int NT, int ST>
 __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st, int tw, int tile_t0,
-                                             bool masked, float ca, float cb, int g, int t) {
+                                             bool masked, float ca, float cb, int g, int t, uint32_t magic) {
   constexpr uint32_t KA = 0, VA = ST * 64, KR = ST * 128, VR = ST * 192;
   constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
   constexpr float kMidK = FULL ? 0.0f : 8.0f;      // K levels are the unsigned codes / nibbles
@@ -286,22 +300,23 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
   }
   const float al_lo = km_lo.x * ca, al_hi = km_hi.x * ca;
   const float be_lo = fmaf(km_lo.x, kMidK, km_lo.y) * cb, be_hi = fmaf(km_hi.x, kMidK, km_hi.y) * cb;
+  // s holds score - m (log2 units) from here on
   bool grow = false;
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
-    s[nt][0] = fmaf(al_lo, s[nt][0], be_lo * w.qs[nt][0]);
-    s[nt][1] = fmaf(al_lo, s[nt][1], be_lo * w.qs[nt][1]);
-    s[nt][2] = fmaf(al_hi, s[nt][2], be_hi * w.qs[nt][0]);
-    s[nt][3] = fmaf(al_hi, s[nt][3], be_hi * w.qs[nt][1]);
+    s[nt][0] = fmaf(al_lo, s[nt][0], fmaf(be_lo, w.qs[nt][0], -w.m[nt][0]));
+    s[nt][1] = fmaf(al_lo, s[nt][1], fmaf(be_lo, w.qs[nt][1], -w.m[nt][1]));
+    s[nt][2] = fmaf(al_hi, s[nt][2], fmaf(be_hi, w.qs[nt][0], -w.m[nt][0]));
+    s[nt][3] = fmaf(al_hi, s[nt][3], fmaf(be_hi, w.qs[nt][1], -w.m[nt][1]));
     if (masked) {
       if (tok_lo >= w.lim[nt][0]) s[nt][0] = -INFINITY;
       if (tok_lo >= w.lim[nt][1]) s[nt][1] = -INFINITY;
       if (tok_hi >= w.lim[nt][0]) s[nt][2] = -INFINITY;
       if (tok_hi >= w.lim[nt][1]) s[nt][3] = -INFINITY;
     }
-    grow |= fmaxf(s[nt][0], s[nt][2]) > w.m[nt][0] + 4.0f;
-    grow |= fmaxf(s[nt][1], s[nt][3]) > w.m[nt][1] + 4.0f;
+    grow |= fmaxf(fmaxf(s[nt][0], s[nt][2]), fmaxf(s[nt][1], s[nt][3])) > 4.0f;
   }
+  grow |= w.fresh;
   // ---- lazy maximum: raise it only when some score exceeds it by more than 4 (p <= 16) --
   if (__any_sync(0xFFFFFFFFu, grow)) {
 #pragma unroll
@@ -312,9 +327,13 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
         mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 4));
         mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 8));
         mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));
-        const float mn = fmaxf(w.m[nt][c], mx);
-        const float f = ex2(w.m[nt][c] - mn);
-        w.m[nt][c] = mn;
+        // how far the maximum moves: up only, except for the first tile, which sets it outright
+        // (a column that sees none of the first tile's tokens sees none of the later ones either)
+        const float up = w.fresh ? fmaxf(mx, -1.0e4f) : fmaxf(mx, 0.0f);
+        const float f = w.fresh ? 0.0f : ex2(-up);  // nothing accumulated yet when fresh
+        w.m[nt][c] += up;
+        s[nt][c] -= up;
+        s[nt][c + 2] -= up;
         w.l[nt][c] *= f;
         w.zs[nt][c] *= f;
 #pragma unroll
@@ -331,8 +350,8 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
   uint32_t pb[NT][2];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
-    const float p0 = ex2(s[nt][0] - w.m[nt][0]), p1 = ex2(s[nt][1] - w.m[nt][1]);
-    const float p2 = ex2(s[nt][2] - w.m[nt][0]), p3 = ex2(s[nt][3] - w.m[nt][1]);
+    const float p0 = ex2(s[nt][0]), p1 = ex2(s[nt][1]);
+    const float p2 = ex2(s[nt][2]), p3 = ex2(s[nt][3]);
     w.l[nt][0] += p0 + p2;
     w.l[nt][1] += p1 + p3;
     w.zs[nt][0] = fmaf(p0, zv_lo, fmaf(p2, zv_hi, w.zs[nt][0]));
@@ -340,6 +359,7 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
     pb[nt][0] = movmatrix_trans(pack_f16x2(p0 * sv_lo, p1 * sv_lo));  // tokens (2t,2t+1) of rows 0..7
     pb[nt][1] = movmatrix_trans(pack_f16x2(p2 * sv_hi, p3 * sv_hi));  // tokens of rows 8..15
   }
+  w.fresh = false;
 
   // ---- O^T += level(V)^T . P^T ---------------------------------------------------------
   // this thread feeds tokens pi(2t), pi(2t+1) (+8) and dims 16g .. 16g+15
@@ -354,8 +374,8 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
       for (int half = 0; half < 2; ++half) {
         const uint32_t sel = half ? 0x7632u : 0x5410u;
         uint32_t ab[4], cd[4];
-        nib4_to_h2(prmt(A[wd], Bw[wd], sel), ab);  // dims e(4half+0..3), token pair (a, b)
-        nib4_to_h2(prmt(C[wd], Dw[wd], sel), cd);  // same dims, token pair (c, d)
+        nib4_to_h2(prmt(A[wd], Bw[wd], sel), magic, ab);  // dims e(4half+0..3), token pair (a, b)
+        nib4_to_h2(prmt(C[wd], Dw[wd], sel), magic, cd);  // same dims, token pair (c, d)
 #pragma unroll
         for (int qd = 0; qd < 2; ++qd) {
           const int mt = wd * 4 + half * 2 + qd;
@@ -383,14 +403,14 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
         const uint32_t uab = prmt(ea, eb, sel), vab = prmt(oa, ob, sel);
         const uint32_t ucd = prmt(ec, ed, sel), vcd = prmt(oc, od, sel);
         // m-tile qd=0: dims e(4half+0) [row g] and e(4half+1) [row g+8]; qd=1: e(4half+2), e(4half+3)
-        const uint32_t ab0 = hadd2((uab & 0x00FF00FFu) | kMagic, kNeg1152);
-        const uint32_t ab1 = hadd2((vab & 0x00FF00FFu) | kMagic, kNeg1152);
-        const uint32_t ab2 = hadd2(prmt(uab, kMagic, 0x7351), kNeg1152);
-        const uint32_t ab3 = hadd2(prmt(vab, kMagic, 0x7351), kNeg1152);
-        const uint32_t cd0 = hadd2((ucd & 0x00FF00FFu) | kMagic, kNeg1152);
-        const uint32_t cd1 = hadd2((vcd & 0x00FF00FFu) | kMagic, kNeg1152);
-        const uint32_t cd2 = hadd2(prmt(ucd, kMagic, 0x7351), kNeg1152);
-        const uint32_t cd3 = hadd2(prmt(vcd, kMagic, 0x7351), kNeg1152);
+        const uint32_t ab0 = hadd2(and_or<0x00FF00FFu>(uab, magic), kNeg1152);
+        const uint32_t ab1 = hadd2(and_or<0x00FF00FFu>(vab, magic), kNeg1152);
+        const uint32_t ab2 = hadd2(prmt(uab, magic, 0x7351), kNeg1152);
+        const uint32_t ab3 = hadd2(prmt(vab, magic, 0x7351), kNeg1152);
+        const uint32_t cd0 = hadd2(and_or<0x00FF00FFu>(ucd, magic), kNeg1152);
+        const uint32_t cd1 = hadd2(and_or<0x00FF00FFu>(vcd, magic), kNeg1152);
+        const uint32_t cd2 = hadd2(prmt(ucd, magic, 0x7351), kNeg1152);
+        const uint32_t cd3 = hadd2(prmt(vcd, magic, 0x7351), kNeg1152);
         const int mt = wd * 4 + half * 2;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
@@ -549,7 +569,27 @@ attn_kernel(const AttnParams p) {
     if (n_units == 0) return;
 
     // =============================== producer loop ===============================
+    // every lane below TW*NARR has a fixed role: one array of one 16-token sub-block per stage
     constexpr int NARR = FULL ? 6 : 4;
+    static_assert(TW * NARR <= 32, "one copy per producer lane");
+    const int my_sub = lane < TW * NARR ? lane / NARR : TW;  // TW = no role
+    const int my_arr = lane % NARR;
+    const unsigned char* my_src;
+    uint32_t my_mul, my_dst, my_bytes;
+    {
+      const bool is_meta = my_arr == 2 || my_arr == 3;
+      my_src = my_arr == 0 ? p.ka : my_arr == 1 ? p.va
+             : my_arr == 2 ? reinterpret_cast<const unsigned char*>(p.km)
+             : my_arr == 3 ? reinterpret_cast<const unsigned char*>(p.vm)
+             : my_arr == 4 ? p.kr : p.vr;
+      const uint32_t dst0 = my_arr == 0 ? 0u : my_arr == 1 ? ST * 64u
+                          : my_arr == 2 ? (FULL ? ST * 256u : ST * 128u)
+                          : my_arr == 3 ? (FULL ? ST * 264u : ST * 136u)
+                          : my_arr == 4 ? ST * 128u : ST * 192u;
+      my_mul = is_meta ? 8u : 64u;
+      my_bytes = is_meta ? 128u : 1024u;
+      my_dst = dst0 + (uint32_t)(my_sub < TW ? my_sub : 0) * my_bytes;
+    }
     int b = b_lo, len = clamp_len(b), U = (len + ST - 1) / ST;
     int hkv = (int)(off_lo / U), u = (int)(off_lo % U);
     int remaining = n_units, gs = 0, ic = 0;
@@ -599,19 +639,9 @@ attn_kernel(const AttnParams p) {
             mbar_expect_tx(bar, nsub * C::kSubBytes);
           }
           __syncwarp();
-          const uint32_t stage = ring_u32 + slot * C::kStageBytes;
-          for (int idx = lane; idx < nsub * NARR; idx += 32) {
-            const int sub = idx / NARR, arr = idx - sub * NARR;
-            const size_t row = blk_s[k * TW + sub];
-            switch (arr) {
-              case 0: bulk_g2s(stage + sub * 1024, p.ka + row * 64, 1024, bar); break;
-              case 1: bulk_g2s(stage + ST * 64 + sub * 1024, p.va + row * 64, 1024, bar); break;
-              case 2: bulk_g2s(stage + (FULL ? ST * 256 : ST * 128) + sub * 128, p.km + row * 2, 128, bar); break;
-              case 3: bulk_g2s(stage + (FULL ? ST * 264 : ST * 136) + sub * 128, p.vm + row * 2, 128, bar); break;
-              case 4: bulk_g2s(stage + ST * 128 + sub * 1024, p.kr + row * 64, 1024, bar); break;
-              default: bulk_g2s(stage + ST * 192 + sub * 1024, p.vr + row * 64, 1024, bar); break;
-            }
-          }
+          if (my_sub < nsub)
+            bulk_g2s(ring_u32 + slot * C::kStageBytes + my_dst, my_src + (size_t)blk_s[k * TW + my_sub] * my_mul,
+                     my_bytes, bar);
         }
         __syncwarp();  // blk_s is rewritten by the next round
       }
@@ -644,6 +674,7 @@ attn_kernel(const AttnParams p) {
   const int g = lane >> 2, t = lane & 3;
   const int tw = warp % TW, cg = warp / TW;
   const float cb = p.sm_log2;
+  const uint32_t magic = opaque_magic();
   float ca = 0.0f;
   int len = 0, full_lim = 0, ic = 0;
   Item item;
@@ -725,7 +756,7 @@ attn_kernel(const AttnParams p) {
           w.qs[nt][cc] = sum;
           const int j = col / p.G;
           w.lim[nt][cc] = col < p.ncols ? (p.causal ? len - p.nq + j + 1 : len) : 0;
-          w.m[nt][cc] = -1.0e30f;
+          w.m[nt][cc] = 0.0f;
           w.l[nt][cc] = 0.0f;
           w.zs[nt][cc] = 0.0f;
         }
@@ -734,14 +765,19 @@ attn_kernel(const AttnParams p) {
 #pragma unroll
           for (int i = 0; i < 4; ++i) w.o[nt][mt][i] = 0.0f;
       }
+      w.fresh = true;
     }
     const int tile_t0 = info.y * ST + tw * 16;
     if (tile_t0 < len)
       process_tile<FULL, NT, ST>(w, ring_u32 + slot * C::kStageBytes, tw, tile_t0,
-                                 tile_t0 + 16 > full_lim, ca, cb, g, t);
+                                 tile_t0 + 16 > full_lim, ca, cb, g, t, magic);
     __syncwarp();
     if (lane == 0) mbar_arrive(empty0 + slot * 8);
     if (!(info.z & 2)) continue;
+    if (w.fresh) {  // this warp saw no token of the piece: it must not weigh in the merge
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) w.m[nt][0] = w.m[nt][1] = -1.0e30f;
+    }
 
     // ---- end of the piece: warp 0 of the column group absorbs the other token warps one by
     //      one (register-wise, through a lane-private mailbox), then writes the result --------
