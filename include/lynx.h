@@ -134,6 +134,27 @@ lynx_status lynx_merge_verify_attention(const lynx_shape* shape, const void* q_b
                                         float* out_full, int32_t* first_reject, float* dev,
                                         void* workspace, size_t workspace_bytes, void* stream);
 
+/* Anchor attention without a caller workspace (the paper has no counterpart; this exists for
+ * deployments where the calling code may not allocate device memory: a plug-in running inside
+ * another framework's memory plan, a latency-critical serving loop that has frozen its
+ * allocations, or a host that must not touch the allocator while other streams are being
+ * captured).  Same computation, arguments and result as lynx_anchor_attention, but the scratch
+ * memory is a fixed 8 MiB array inside the library image (every GPU that loads the library
+ * holds it until the process exits); the call itself allocates nothing.
+ *  - Problems whose scratch need (lynx_workspace_bytes) exceeds 8 MiB are rejected with
+ *    LYNX_ERR_WORKSPACE and nothing is launched.
+ *  - The first call on each device looks up the array's device address (a one-time set-up,
+ *    done with that device current); make that first call before any stream capture begins.
+ *  - All calls share the one array.  Each call clears the words that must start at zero, on
+ *    `stream`; two calls that overlap on the GPU (different streams, or different host threads
+ *    without ordering) race on it and produce wrong results.  Order them on one stream.
+ *  - Out-of-range block ids are clamped as usual but cannot be reported (there is no workspace
+ *    for lynx_check to read). */
+lynx_status lynx_anchor_attention_static(const lynx_shape* shape, const void* q_bf16, int32_t batch,
+                                         int32_t n_q, int32_t causal, lynx_plane K, lynx_plane V,
+                                         const int32_t* block_table, const int32_t* seq_lens,
+                                         float softmax_scale, float* out, void* stream);
+
 /* Synchronises `stream`, reads and clears the workspace's status word.  Test / debug use. */
 lynx_status lynx_check(void* workspace, void* stream);
 

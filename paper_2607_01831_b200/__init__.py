@@ -37,7 +37,8 @@ class _Shape(ctypes.Structure):
 
 
 EXPORTS = ["lynx_split_quantize", "lynx_recombine", "lynx_workspace_bytes", "lynx_workspace_init",
-           "lynx_anchor_attention", "lynx_merge_verify_attention", "lynx_check",
+           "lynx_anchor_attention", "lynx_merge_verify_attention", "lynx_anchor_attention_static",
+           "lynx_check",
            "lynx_status_string", "lynx_version"]
 
 
@@ -70,6 +71,9 @@ def load():
                                                 _Plane, vp, vp, f32, vp, f32, f32, vp, vp, vp, vp,
                                                 ctypes.c_size_t, vp]
     lib.lynx_merge_verify_attention.restype = ctypes.c_int
+    lib.lynx_anchor_attention_static.argtypes = [ctypes.POINTER(_Shape), vp, i32, i32, i32, _Plane,
+                                                 _Plane, vp, vp, f32, vp, vp]
+    lib.lynx_anchor_attention_static.restype = ctypes.c_int
     lib.lynx_check.argtypes = [vp, vp]
     lib.lynx_check.restype = ctypes.c_int
     lib.lynx_status_string.argtypes = [ctypes.c_int]
@@ -190,6 +194,25 @@ def anchor_attention(geo: Geometry, q: torch.Tensor, K: Planes, V: Planes, block
                                      V._c(), _ptr(block_table), _ptr(seq_lens), softmax_scale,
                                      _ptr(out), _ptr(workspace), workspace.numel(), _stream()),
         "lynx_anchor_attention")
+    return out
+
+
+def anchor_attention_static(geo: Geometry, q: torch.Tensor, K: Planes, V: Planes,
+                            block_table: torch.Tensor, seq_lens: torch.Tensor, causal: bool = False,
+                            softmax_scale: float = 0.0, out: torch.Tensor | None = None) -> torch.Tensor:
+    """lynx_anchor_attention_static: anchor attention whose scratch memory is a fixed 8 MiB array
+    inside the library, for callers that may not allocate a workspace.  Only `out` is allocated
+    here when the caller does not pass it; the library call allocates nothing.  Calls share the
+    array: keep them ordered on one stream.  Raises LynxError if the problem needs more scratch."""
+    B, n_q, Hq, d = q.shape
+    if q.dtype != torch.bfloat16 or d != D or Hq != geo.num_q_heads:
+        raise LynxError("q must be BF16 [B][n_q][Hq][128]")
+    if out is None:
+        out = torch.empty(B, n_q, Hq, D, dtype=torch.float32, device=q.device)
+    _ok(load().lynx_anchor_attention_static(ctypes.byref(geo._c()), _ptr(q), B, n_q, int(causal),
+                                            K._c(), V._c(), _ptr(block_table), _ptr(seq_lens),
+                                            softmax_scale, _ptr(out), _stream()),
+        "lynx_anchor_attention_static")
     return out
 
 

@@ -1088,3 +1088,56 @@ extern "C" lynx_status lynx_merge_verify_attention(const lynx_shape* shape, cons
                              softmax_scale, draft_out, atol, rtol, out_full, first_reject, dev,
                              workspace, workspace_bytes, stream);
 }
+
+// ---------------------------------------------------------------------------------------------
+// Anchor attention for callers that cannot hand over a workspace (no paper counterpart).
+//
+// The split-K partials, tickets and status word live in one fixed array in device memory that
+// is part of the loaded library image: nothing is allocated, by this call or by any routine it
+// uses.  Host code cannot use the array's name as an address (on the host the name is only a
+// handle for the runtime), so the device address is looked up once per device with
+// cudaGetSymbolAddress, while that device is current, and the kernels are given that address.
+namespace lynx {
+namespace {
+
+constexpr size_t kStaticScratchBytes = 8u << 20;  // 8 MiB held by every GPU that loads the library
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+lynx_status static_scratch_address(void** out) {
+  static void* resolved[64] = {nullptr};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LYNX_ERR_CUDA;
+  if (resolved[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return LYNX_ERR_CUDA;
+    resolved[dev] = ptr;
+  }
+  *out = resolved[dev];
+  return LYNX_OK;
+}
+
+}  // namespace
+}  // namespace lynx
+
+extern "C" lynx_status lynx_anchor_attention_static(const lynx_shape* shape, const void* q_bf16,
+                                                    int32_t batch, int32_t n_q, int32_t causal,
+                                                    lynx_plane K, lynx_plane V,
+                                                    const int32_t* block_table, const int32_t* seq_lens,
+                                                    float softmax_scale, float* out, void* stream) {
+  using namespace lynx;
+  if (batch == 0) return LYNX_OK;
+  if (!shape) return LYNX_ERR_NULL;
+  if (batch < 0 || n_q <= 0) return LYNX_ERR_SHAPE;
+  Plan pl;
+  if (!make_plan(shape, batch, n_q, &pl)) return LYNX_ERR_UNSUPPORTED;
+  if (pl.bytes > kStaticScratchBytes) return LYNX_ERR_WORKSPACE;  // problem too large for the fixed array
+  void* scratch = nullptr;
+  const lynx_status st = static_scratch_address(&scratch);
+  if (st != LYNX_OK) return st;
+  // the array keeps what the previous call left: the status word and the tickets must be zero
+  if (cudaMemsetAsync(scratch, 0, pl.off_dev, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return LYNX_ERR_CUDA;
+  return run_attention(false, shape, q_bf16, batch, n_q, causal, K, V, block_table, seq_lens,
+                       softmax_scale, nullptr, 0.f, 0.f, out, nullptr, nullptr, scratch,
+                       kStaticScratchBytes, stream);
+}
