@@ -452,6 +452,177 @@ __device__ __forceinline__ void named_bar(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// The producer warp: works out this CTA's range of stage-units (and handles sequences with no
+// token), then streams the pieces of the range: queries of each piece into one of two slots,
+// 16-token sub-blocks of the planes into the ring.  `C` supplies the shared-memory geometry.
+template <class C, bool FULL, int TW, int NSTAGE>
+__device__ __forceinline__ void producer_warp(const AttnParams& p, int lane, uint32_t ring_u32,
+                                              uint32_t full0, uint32_t empty0, uint32_t qfull0,
+                                              uint32_t qempty0, __nv_bfloat16* q_s, uint32_t* blk_s,
+                                              int4* info_s, Item* items, int* misc,
+                                              volatile int* abort_word) {
+  constexpr int ST = C::kST;
+  const int n_cta = gridDim.x, cta = blockIdx.x;
+  const int cap = p.max_blocks * p.bt;
+  auto clamp_len = [&](int b) {
+    int len = __ldg(p.seq_lens + b);
+    return len < 0 ? 0 : (len > cap ? cap : len);
+  };
+  // ---- prologue (producer warp): total work, this CTA's range, empty sequences ----------
+  long long tot = 0;
+  for (int b = lane; b < p.B; b += 32) tot += (clamp_len(b) + ST - 1) / ST;
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) tot += __shfl_xor_sync(0xFFFFFFFFu, tot, off);
+  const long long T = tot * p.Hkv;
+  const long long q = (T + n_cta - 1) / n_cta;
+  const long long lo = (long long)cta * q, hi = (lo + q < T) ? lo + q : T;
+  int b_lo = 0;
+  long long off_lo = 0;
+  if (lo < hi) {
+    long long running = 0;
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+      const int b = b0 + lane;
+      const long long u = b < p.B ? (long long)p.Hkv * ((clamp_len(b) + ST - 1) / ST) : 0;
+      long long incl = u;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const long long v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      const long long excl = running + incl - u;
+      const bool hit = u > 0 && lo >= excl && lo < excl + u;
+      const unsigned m = __ballot_sync(0xFFFFFFFFu, hit);
+      if (m) {
+        const int src = __ffs(m) - 1;
+        b_lo = b0 + src;
+        off_lo = lo - __shfl_sync(0xFFFFFFFFu, excl, src);
+        break;
+      }
+      running += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+  }
+  if (lane == 0) {
+    misc[4] = (int)(q > 0x7FFFFFFF ? 0x7FFFFFFF : q);
+    misc[7] = lo < hi ? (int)(hi - lo) : 0;
+  }
+  // sequences with no token: outputs are zero, nothing is rejected unless the draft is not zero
+  for (int b = cta; b < p.B; b += n_cta) {
+    if (clamp_len(b) != 0) continue;
+    const size_t n = (size_t)p.nq * p.Hq * LYNX_D;
+    for (size_t i = lane; i < n; i += 32) p.out[(size_t)b * n + i] = 0.0f;
+    if (FULL && p.draft != nullptr) {
+      int fr = p.nq;
+      for (int j = p.nq - 1; j >= 0; --j) {
+        float worst = 0.0f;
+        for (int i = lane; i < p.Hq * LYNX_D; i += 32)
+          worst = fmaxf(worst, fabsf(__ldg(p.draft + ((size_t)b * p.nq + j) * p.Hq * LYNX_D + i)) / p.atol);
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xFFFFFFFFu, worst, off));
+        if (lane == 0) p.dev[(size_t)b * p.nq + j] = worst;
+        if (worst > 1.0f) fr = j;
+      }
+      if (lane == 0) p.first_reject[b] = fr;
+    }
+  }
+  __syncthreads();  // (A) the range is published
+  const int n_units = (int)(lo < hi ? hi - lo : 0);
+  if (n_units == 0) return;
+
+  // =============================== producer loop ===============================
+  // every lane below TW*NARR has a fixed role: one array of one 16-token sub-block per stage
+  constexpr int NARR = FULL ? 6 : 4;
+  static_assert(TW * NARR <= 32, "one copy per producer lane");
+  const int my_sub = lane < TW * NARR ? lane / NARR : TW;  // TW = no role
+  const int my_arr = lane % NARR;
+  const unsigned char* my_src;
+  uint32_t my_mul, my_dst, my_bytes;
+  {
+    const bool is_meta = my_arr == 2 || my_arr == 3;
+    my_src = my_arr == 0 ? p.ka : my_arr == 1 ? p.va
+           : my_arr == 2 ? reinterpret_cast<const unsigned char*>(p.km)
+           : my_arr == 3 ? reinterpret_cast<const unsigned char*>(p.vm)
+           : my_arr == 4 ? p.kr : p.vr;
+    const uint32_t dst0 = my_arr == 0 ? 0u : my_arr == 1 ? ST * 64u
+                        : my_arr == 2 ? (FULL ? ST * 256u : ST * 128u)
+                        : my_arr == 3 ? (FULL ? ST * 264u : ST * 136u)
+                        : my_arr == 4 ? ST * 128u : ST * 192u;
+    my_mul = is_meta ? 8u : 64u;
+    my_bytes = is_meta ? 128u : 1024u;
+    my_dst = dst0 + (uint32_t)(my_sub < TW ? my_sub : 0) * my_bytes;
+  }
+  int b = b_lo, len = clamp_len(b), U = (len + ST - 1) / ST;
+  int hkv = (int)(off_lo / U), u = (int)(off_lo % U);
+  int remaining = n_units, gs = 0, ic = 0;
+  while (remaining > 0) {
+    const int n = min(remaining, U - u);
+    const int qi = ic & 1;
+    if (ic >= 2) mbar_wait(qempty0 + qi * 8, ((ic >> 1) - 1) & 1, abort_word);
+    const long long seg0 = lo + (n_units - remaining) - u;  // first unit of this segment
+    if (lane == 0) {
+      Item it;
+      it.b = b; it.hkv = hkv; it.len = len;
+      it.first_cta = (int)(seg0 / q);
+      it.n_contrib = (int)((seg0 + U - 1) / q) - it.first_cta + 1;
+      it.pad0 = it.pad1 = it.pad2 = 0;
+      items[qi] = it;
+      mbar_expect_tx(qfull0 + qi * 8, (uint32_t)(p.nq * p.G * LYNX_D * 2));
+    }
+    __syncwarp();
+    for (int j = lane; j < p.nq; j += 32)
+      bulk_g2s(smem_u32(q_s + ((size_t)qi * C::kColsPad + j * p.G) * LYNX_D),
+               p.q + (((size_t)b * p.nq + j) * p.Hq + (size_t)hkv * p.G) * LYNX_D,
+               (uint32_t)(p.G * LYNX_D * 2), qfull0 + qi * 8);
+    for (int c0 = 0; c0 < n; c0 += kPieceUnits) {
+      const int cn = min(kPieceUnits, n - c0);
+      for (int i = lane; i < cn * TW; i += 32) {
+        const int t0 = (u + c0) * ST + i * 16;
+        uint32_t row = 0;
+        if (t0 < len) {
+          int blk = __ldg(p.block_table + (size_t)b * p.max_blocks + t0 / p.bt);
+          if (blk < 0 || blk >= p.num_blocks) {
+            atomicOr(p.ws_flags, kFlagBadBlock);
+            blk = blk < 0 ? 0 : p.num_blocks - 1;
+          }
+          row = (uint32_t)(((size_t)blk * p.Hkv + hkv) * p.bt + (t0 % p.bt));
+        }
+        blk_s[i] = row;
+      }
+      __syncwarp();
+      for (int k = 0; k < cn; ++k, ++gs) {
+        const int slot = gs % NSTAGE;
+        if (gs >= NSTAGE) mbar_wait(empty0 + slot * 8, ((gs / NSTAGE) - 1) & 1, abort_word);
+        const int uu = u + c0 + k;
+        const int nsub = min(TW, (len - uu * ST + 15) >> 4);
+        const uint32_t bar = full0 + slot * 8;
+        if (lane == 0) {
+          info_s[slot] = make_int4(qi, uu, (c0 + k == 0 ? 1 : 0) | (c0 + k == n - 1 ? 2 : 0), 0);
+          mbar_expect_tx(bar, nsub * C::kSubBytes);
+        }
+        __syncwarp();
+        if (my_sub < nsub)
+          bulk_g2s(ring_u32 + slot * C::kStageBytes + my_dst, my_src + (size_t)blk_s[k * TW + my_sub] * my_mul,
+                   my_bytes, bar);
+      }
+      __syncwarp();  // blk_s is rewritten by the next round
+    }
+    remaining -= n;
+    u += n;
+    ++ic;
+    if (u == U && remaining > 0) {
+      u = 0;
+      if (++hkv == p.Hkv) {
+        hkv = 0;
+        do {
+          ++b;
+          len = b < p.B ? clamp_len(b) : 0;
+          U = (len + ST - 1) / ST;
+        } while (b < p.B && U == 0);
+        if (b >= p.B) break;  // cannot happen: the range ends inside the list
+      }
+    }
+  }
+}
+
 // Persistent, stream-K style kernel.  The work is the list of stage-units (ST tokens of one
 // (sequence, KV head)) in (sequence, head, position) order; CTA i owns the contiguous range
 // [i*q, (i+1)*q) of it, q = ceil(total / gridDim.x).  A range is cut into pieces at segment
@@ -502,165 +673,9 @@ attn_kernel(const AttnParams p) {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
 
-  auto clamp_len = [&](int b) {
-    int len = __ldg(p.seq_lens + b);
-    return len < 0 ? 0 : (len > cap ? cap : len);
-  };
-
   if (warp == C::kConsWarps) {
-    // ---- prologue (producer warp): total work, this CTA's range, empty sequences ----------
-    long long tot = 0;
-    for (int b = lane; b < p.B; b += 32) tot += (clamp_len(b) + ST - 1) / ST;
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) tot += __shfl_xor_sync(0xFFFFFFFFu, tot, off);
-    const long long T = tot * p.Hkv;
-    const long long q = (T + n_cta - 1) / n_cta;
-    const long long lo = (long long)cta * q, hi = (lo + q < T) ? lo + q : T;
-    int b_lo = 0;
-    long long off_lo = 0;
-    if (lo < hi) {
-      long long running = 0;
-      for (int b0 = 0; b0 < p.B; b0 += 32) {
-        const int b = b0 + lane;
-        const long long u = b < p.B ? (long long)p.Hkv * ((clamp_len(b) + ST - 1) / ST) : 0;
-        long long incl = u;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const long long v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-          if (lane >= o) incl += v;
-        }
-        const long long excl = running + incl - u;
-        const bool hit = u > 0 && lo >= excl && lo < excl + u;
-        const unsigned m = __ballot_sync(0xFFFFFFFFu, hit);
-        if (m) {
-          const int src = __ffs(m) - 1;
-          b_lo = b0 + src;
-          off_lo = lo - __shfl_sync(0xFFFFFFFFu, excl, src);
-          break;
-        }
-        running += __shfl_sync(0xFFFFFFFFu, incl, 31);
-      }
-    }
-    if (lane == 0) {
-      misc[4] = (int)(q > 0x7FFFFFFF ? 0x7FFFFFFF : q);
-      misc[7] = lo < hi ? (int)(hi - lo) : 0;
-    }
-    // sequences with no token: outputs are zero, nothing is rejected unless the draft is not zero
-    for (int b = cta; b < p.B; b += n_cta) {
-      if (clamp_len(b) != 0) continue;
-      const size_t n = (size_t)p.nq * p.Hq * LYNX_D;
-      for (size_t i = lane; i < n; i += 32) p.out[(size_t)b * n + i] = 0.0f;
-      if (FULL && p.draft != nullptr) {
-        int fr = p.nq;
-        for (int j = p.nq - 1; j >= 0; --j) {
-          float worst = 0.0f;
-          for (int i = lane; i < p.Hq * LYNX_D; i += 32)
-            worst = fmaxf(worst, fabsf(__ldg(p.draft + ((size_t)b * p.nq + j) * p.Hq * LYNX_D + i)) / p.atol);
-#pragma unroll
-          for (int off = 16; off >= 1; off >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xFFFFFFFFu, worst, off));
-          if (lane == 0) p.dev[(size_t)b * p.nq + j] = worst;
-          if (worst > 1.0f) fr = j;
-        }
-        if (lane == 0) p.first_reject[b] = fr;
-      }
-    }
-    __syncthreads();  // (A) the range is published
-    const int n_units = (int)(lo < hi ? hi - lo : 0);
-    if (n_units == 0) return;
-
-    // =============================== producer loop ===============================
-    // every lane below TW*NARR has a fixed role: one array of one 16-token sub-block per stage
-    constexpr int NARR = FULL ? 6 : 4;
-    static_assert(TW * NARR <= 32, "one copy per producer lane");
-    const int my_sub = lane < TW * NARR ? lane / NARR : TW;  // TW = no role
-    const int my_arr = lane % NARR;
-    const unsigned char* my_src;
-    uint32_t my_mul, my_dst, my_bytes;
-    {
-      const bool is_meta = my_arr == 2 || my_arr == 3;
-      my_src = my_arr == 0 ? p.ka : my_arr == 1 ? p.va
-             : my_arr == 2 ? reinterpret_cast<const unsigned char*>(p.km)
-             : my_arr == 3 ? reinterpret_cast<const unsigned char*>(p.vm)
-             : my_arr == 4 ? p.kr : p.vr;
-      const uint32_t dst0 = my_arr == 0 ? 0u : my_arr == 1 ? ST * 64u
-                          : my_arr == 2 ? (FULL ? ST * 256u : ST * 128u)
-                          : my_arr == 3 ? (FULL ? ST * 264u : ST * 136u)
-                          : my_arr == 4 ? ST * 128u : ST * 192u;
-      my_mul = is_meta ? 8u : 64u;
-      my_bytes = is_meta ? 128u : 1024u;
-      my_dst = dst0 + (uint32_t)(my_sub < TW ? my_sub : 0) * my_bytes;
-    }
-    int b = b_lo, len = clamp_len(b), U = (len + ST - 1) / ST;
-    int hkv = (int)(off_lo / U), u = (int)(off_lo % U);
-    int remaining = n_units, gs = 0, ic = 0;
-    while (remaining > 0) {
-      const int n = min(remaining, U - u);
-      const int qi = ic & 1;
-      if (ic >= 2) mbar_wait(qempty0 + qi * 8, ((ic >> 1) - 1) & 1, abort_word);
-      const long long seg0 = lo + (n_units - remaining) - u;  // first unit of this segment
-      if (lane == 0) {
-        Item it;
-        it.b = b; it.hkv = hkv; it.len = len;
-        it.first_cta = (int)(seg0 / q);
-        it.n_contrib = (int)((seg0 + U - 1) / q) - it.first_cta + 1;
-        it.pad0 = it.pad1 = it.pad2 = 0;
-        items[qi] = it;
-        mbar_expect_tx(qfull0 + qi * 8, (uint32_t)(p.nq * p.G * LYNX_D * 2));
-      }
-      __syncwarp();
-      for (int j = lane; j < p.nq; j += 32)
-        bulk_g2s(smem_u32(q_s + ((size_t)qi * C::kColsPad + j * p.G) * LYNX_D),
-                 p.q + (((size_t)b * p.nq + j) * p.Hq + (size_t)hkv * p.G) * LYNX_D,
-                 (uint32_t)(p.G * LYNX_D * 2), qfull0 + qi * 8);
-      for (int c0 = 0; c0 < n; c0 += kPieceUnits) {
-        const int cn = min(kPieceUnits, n - c0);
-        for (int i = lane; i < cn * TW; i += 32) {
-          const int t0 = (u + c0) * ST + i * 16;
-          uint32_t row = 0;
-          if (t0 < len) {
-            int blk = __ldg(p.block_table + (size_t)b * p.max_blocks + t0 / p.bt);
-            if (blk < 0 || blk >= p.num_blocks) {
-              atomicOr(p.ws_flags, kFlagBadBlock);
-              blk = blk < 0 ? 0 : p.num_blocks - 1;
-            }
-            row = (uint32_t)(((size_t)blk * p.Hkv + hkv) * p.bt + (t0 % p.bt));
-          }
-          blk_s[i] = row;
-        }
-        __syncwarp();
-        for (int k = 0; k < cn; ++k, ++gs) {
-          const int slot = gs % NSTAGE;
-          if (gs >= NSTAGE) mbar_wait(empty0 + slot * 8, ((gs / NSTAGE) - 1) & 1, abort_word);
-          const int uu = u + c0 + k;
-          const int nsub = min(TW, (len - uu * ST + 15) >> 4);
-          const uint32_t bar = full0 + slot * 8;
-          if (lane == 0) {
-            info_s[slot] = make_int4(qi, uu, (c0 + k == 0 ? 1 : 0) | (c0 + k == n - 1 ? 2 : 0), 0);
-            mbar_expect_tx(bar, nsub * C::kSubBytes);
-          }
-          __syncwarp();
-          if (my_sub < nsub)
-            bulk_g2s(ring_u32 + slot * C::kStageBytes + my_dst, my_src + (size_t)blk_s[k * TW + my_sub] * my_mul,
-                     my_bytes, bar);
-        }
-        __syncwarp();  // blk_s is rewritten by the next round
-      }
-      remaining -= n;
-      u += n;
-      ++ic;
-      if (u == U && remaining > 0) {
-        u = 0;
-        if (++hkv == p.Hkv) {
-          hkv = 0;
-          do {
-            ++b;
-            len = b < p.B ? clamp_len(b) : 0;
-            U = (len + ST - 1) / ST;
-          } while (b < p.B && U == 0);
-          if (b >= p.B) break;  // cannot happen: the range ends inside the list
-        }
-      }
-    }
+    producer_warp<C, FULL, TW, NSTAGE>(p, lane, ring_u32, full0, empty0, qfull0, qempty0, q_s, blk_s,
+                                       info_s, items, misc, abort_word);
     return;
   }
 
