@@ -217,33 +217,14 @@ __device__ __forceinline__ void merge_codes(uint32_t xa, uint32_t xr, uint32_t& 
 // K fragments and the V fragments at <= 2-way bank conflicts)
 __device__ __forceinline__ int pi_row(int r) { return r ^ ((r >> 1) & 1); }
 
-template <bool FULL, int NT>
-struct WarpState {
-  uint32_t qf[NT][2][4][2];  // Q^T B-fragments (s8): [n-tile][digit plane hi/lo][k32 step][reg]
-  float qs[NT][2];        // sum_d q_d of the thread's two columns
-  float m[NT][2];         // running (lazy) maximum, log2 units
-  float l[NT][2];         // partial softmax denominators (this thread's rows only)
-  float zs[NT][2];        // partial sum p * (zero + mid*scale) of V
-  float o[NT][8][4];      // O^T accumulators: [n-tile][m-tile (16 dims)][c-reg]
-  int lim[NT][2];         // exclusive token limit of the thread's two columns
-  bool fresh;             // no tile processed yet: the first one sets the maximum outright
-};
-
-// One 16-token tile.  st = shared address of the stage, tw = tile index within the stage,
-// tile_t0 = absolute index of the tile's first token, masked = some (token, column) of this
-// tile is not visible.
+// S^T[16 tokens x NT*8 columns] = level(K) . Q^T for the tile whose S rows g / g+8 are stage
+// rows r0 / r0+8: exact integer arithmetic (u8 levels x two s8 digit planes of q), returned
+// as floats (units: level x q_int).
 template <bool FULL, int NT, int ST>
-__device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st, int tw, int tile_t0,
-                                             bool masked, float ca, float cb, int g, int t, uint32_t magic) {
-  constexpr uint32_t KA = 0, VA = ST * 64, KR = ST * 128, VR = ST * 192;
-  constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
-  constexpr float kMidK = FULL ? 0.0f : 8.0f;      // K levels are the unsigned codes / nibbles
-  constexpr float kMidV = FULL ? 128.0f : 136.0f;  // V levels are centred (code-128, 16(a-8))
-  constexpr float kLevelScaleV = FULL ? 1.0f : 16.0f;
-  const int r0 = tw * 16 + pi_row(g);  // stage row of S row g; S row g+8 is r0 + 8
-
+__device__ __forceinline__ void qk_int8(const uint32_t (&qf)[NT][2][4][2], uint32_t st, int r0, int t,
+                                        float (&s)[NT][4]) {
+  constexpr uint32_t KA = 0, KR = ST * 128;
   // ---- S^T = level(K) . Q^T, exact in integers (u8 levels x two s8 digit planes of q) -----
-  float s[NT][4];
   {
     int shi[NT][4], slo[NT][4];
 #pragma unroll
@@ -274,8 +255,8 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
       }
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        mma_u8s8(shi[nt], evl, evh, odl, odh, w.qf[nt][0][wd][0], w.qf[nt][0][wd][1]);
-        mma_u8s8(slo[nt], evl, evh, odl, odh, w.qf[nt][1][wd][0], w.qf[nt][1][wd][1]);
+        mma_u8s8(shi[nt], evl, evh, odl, odh, qf[nt][0][wd][0], qf[nt][0][wd][1]);
+        mma_u8s8(slo[nt], evl, evh, odl, odh, qf[nt][1][wd][0], qf[nt][1][wd][1]);
       }
     }
 #pragma unroll
@@ -283,6 +264,36 @@ __device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st
 #pragma unroll
       for (int i = 0; i < 4; ++i) s[nt][i] = (float)(shi[nt][i] * 128 + slo[nt][i]);
   }
+
+}
+
+template <bool FULL, int NT>
+struct WarpState {
+  uint32_t qf[NT][2][4][2];  // Q^T B-fragments (s8): [n-tile][digit plane hi/lo][k32 step][reg]
+  float qs[NT][2];        // sum_d q_d of the thread's two columns
+  float m[NT][2];         // running (lazy) maximum, log2 units
+  float l[NT][2];         // partial softmax denominators (this thread's rows only)
+  float zs[NT][2];        // partial sum p * (zero + mid*scale) of V
+  float o[NT][8][4];      // O^T accumulators: [n-tile][m-tile (16 dims)][c-reg]
+  int lim[NT][2];         // exclusive token limit of the thread's two columns
+  bool fresh;             // no tile processed yet: the first one sets the maximum outright
+};
+
+// One 16-token tile.  st = shared address of the stage, tw = tile index within the stage,
+// tile_t0 = absolute index of the tile's first token, masked = some (token, column) of this
+// tile is not visible.
+template <bool FULL, int NT, int ST>
+__device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st, int tw, int tile_t0,
+                                             bool masked, float ca, float cb, int g, int t, uint32_t magic) {
+  constexpr uint32_t KA = 0, VA = ST * 64, KR = ST * 128, VR = ST * 192;
+  constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
+  constexpr float kMidK = FULL ? 0.0f : 8.0f;      // K levels are the unsigned codes / nibbles
+  constexpr float kMidV = FULL ? 128.0f : 136.0f;  // V levels are centred (code-128, 16(a-8))
+  constexpr float kLevelScaleV = FULL ? 1.0f : 16.0f;
+  const int r0 = tw * 16 + pi_row(g);  // stage row of S row g; S row g+8 is r0 + 8
+
+  float s[NT][4];
+  qk_int8<FULL, NT, ST>(w.qf, st, r0, t, s);
 
   // ---- per-token scalars, scores in log2 units -----------------------------------------
   float2 km_lo = lds64f(st + KM + r0 * 8), km_hi = lds64f(st + KM + (r0 + 8) * 8);
@@ -450,6 +461,82 @@ struct Item {  // one piece: a run of stage-units of one (sequence, KV head) giv
 
 __device__ __forceinline__ void named_bar(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// After a piece's result is in the output (direct) or in its partial slot: the last
+// contributor of the (sequence, KV head) merges the slots, and for verification the CTA holding
+// the final outputs of a head takes part in the accept / reject decision (Section 4.3).
+// Called by all consumer threads of the CTA (named barrier 1).
+template <bool FULL, int kColsPad, int kConsThreads>
+__device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& item, bool direct, int tid,
+                                             int* misc) {
+  const size_t bh = (size_t)item.b * p.Hkv + item.hkv;
+  bool final_here = direct;
+  if (!direct) {
+    // the last contributor of this (sequence, KV head) merges the partial slots
+    named_bar(1, kConsThreads);
+    if (tid == 0)
+      misc[1] = (atomicInc(p.ws_chunk_ctr + bh, (uint32_t)item.n_contrib - 1) == (uint32_t)item.n_contrib - 1);
+    named_bar(1, kConsThreads);
+    final_here = misc[1] != 0;
+    if (final_here) {
+      __threadfence();
+      const float* base = p.ws_part + (bh + (size_t)item.first_cta) * (size_t)kColsPad * kPartStride;
+      const size_t cstride = (size_t)kColsPad * kPartStride;
+      for (int idx = tid; idx < kColsPad * LYNX_D; idx += kConsThreads) {
+        const int c = idx >> 7, d = idx & 127;
+        if (c >= p.ncols) continue;
+        const float* col = base + (size_t)c * kPartStride;
+        float M = -INFINITY;
+        for (int i = 0; i < item.n_contrib; ++i) M = fmaxf(M, __ldcg(col + i * cstride + 128));
+        float acc = 0.0f, L = 0.0f;
+        for (int i = 0; i < item.n_contrib; ++i) {
+          const float f = ex2(__ldcg(col + i * cstride + 128) - M);
+          acc = fmaf(__ldcg(col + i * cstride + d), f, acc);
+          L = fmaf(__ldcg(col + i * cstride + 129), f, L);
+        }
+        const int j = c / p.G, hh = c % p.G;
+        p.out[(((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
+      }
+    }
+  }
+  // accept / reject (Section 4.3): by the CTA that wrote the final outputs of this head
+  if (FULL && p.draft != nullptr) {
+    int* devs = misc + 16;
+    named_bar(1, kConsThreads);  // final outputs written; devs free
+    if (final_here) {
+      if (tid < kMaxQ) devs[tid] = 0;
+      named_bar(1, kConsThreads);
+      for (int idx = tid; idx < p.ncols * LYNX_D; idx += kConsThreads) {
+        const int c = idx >> 7, d = idx & 127;
+        const int j = c / p.G, hh = c % p.G;
+        const size_t o = (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + d;
+        const float f = p.out[o], dr = __ldg(p.draft + o);
+        const float r = fabsf(f - dr) / (p.atol + p.rtol * fabsf(f));
+        atomicMax(devs + j, __float_as_int(r));  // r >= 0: integer order = float order
+      }
+      named_bar(1, kConsThreads);
+      if (tid < p.nq) p.ws_dev[bh * kMaxQ + tid] = __int_as_float(devs[tid]);
+      __threadfence();
+      named_bar(1, kConsThreads);
+      if (tid == 0)
+        misc[1] = (atomicInc(p.ws_seq_ctr + item.b, (uint32_t)p.Hkv - 1) == (uint32_t)p.Hkv - 1);
+      named_bar(1, kConsThreads);
+      if (misc[1] && tid == 0) {
+        __threadfence();
+        int fr = p.nq;
+        for (int j = p.nq - 1; j >= 0; --j) {
+          float worst = 0.0f;
+          for (int h = 0; h < p.Hkv; ++h)
+            worst = fmaxf(worst, __ldcg(p.ws_dev + ((size_t)item.b * p.Hkv + h) * kMaxQ + j));
+          p.dev[(size_t)item.b * p.nq + j] = worst;
+          if (worst > 1.0f) fr = j;
+        }
+        p.first_reject[item.b] = fr;
+      }
+    }
+    named_bar(1, kConsThreads);
+  }
 }
 
 // The producer warp: works out this CTA's range of stage-units (and handles sequences with no
@@ -887,72 +974,499 @@ attn_kernel(const AttnParams p) {
       }
       __threadfence();
     }
-    bool final_here = direct;
-    if (!direct) {
-      // the last contributor of this (sequence, KV head) merges the partial slots
+    finish_piece<FULL, C::kColsPad, C::kConsThreads>(p, item, direct, tid, misc);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(qempty0 + (info.x & 1) * 8);
+    ++ic;
+  }
+  if (tid == 0 && misc[0]) atomicOr(p.ws_flags, kFlagTimeout);
+}
+
+// =============================================================================================
+// Team variant for more than 8 columns.  DS consumer warps form a team that takes DS tiles of a
+// stage: warp d computes Q.K^T and the softmax weights of tile d for ALL columns and publishes
+// its P^T fragments in shared memory; every warp then accumulates P.V of all DS tiles for its
+// own slice of 128/DS output dims.  The K/V nibbles are dequantised once per tile (no column
+// groups repeating the work) and the accumulators shrink with DS.  The team keeps one running
+// maximum per column (two named barriers per step; growth is agreed through shared memory).
+// =============================================================================================
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE>
+struct TeamCfg {
+  static constexpr int kTW = DS * TEAMS;                    // consumer warps = tiles per stage
+  static constexpr int kST = kTW * 16;
+  static constexpr int kSubBytes = FULL ? 16 * 272 : 16 * 144;
+  static constexpr int kStageBytes = kST * (FULL ? 272 : 144);
+  static constexpr int kConsWarps = kTW;
+  static constexpr int kConsThreads = kConsWarps * 32;
+  static constexpr int kThreads = (kConsWarps + 1) * 32;
+  static constexpr int kColsPad = NT * 8;
+  static constexpr int kMT = 8 / DS;                        // m-tiles (16 dims) per warp
+  static constexpr int kRing = NSTAGE * kStageBytes;
+  static constexpr int kMailRegs = NT * kMT * 4 + NT * 6;   // o slice + m, l, zs
+  static constexpr int kMailBytes = DS * kMailRegs * 32 * 4;
+  static constexpr int kXchgBytes = kTW * (16 + kColsPad * 4 + NT * 2 * 32 * 4);  // flag, colmax, P^T
+  static constexpr int kLzBytes = DS * kColsPad * 2 * 4;
+  static constexpr int kQBytes = 2 * kColsPad * LYNX_D * 2;
+  static constexpr int kBlkBytes = kPieceUnits * kTW * 4;
+  static constexpr int kInfoBytes = NSTAGE * 16 + 2 * 32;
+  static constexpr int kBarBytes = (2 * NSTAGE + 4) * 8;
+  static constexpr int kMiscBytes = 256;
+  static constexpr int kSmem = kRing + kMailBytes + kXchgBytes + kLzBytes + kQBytes + kBlkBytes +
+                               kInfoBytes + kBarBytes + kMiscBytes;
+};
+
+// O^T slice += level(V)^T[slice dims x 16 tokens] . P^T for one tile (stage rows row0..row0+15).
+// Slice d of DS covers the m-tiles (word, half) of every lane's 16 dims: DS=1 all eight, DS=2
+// word d, DS=4 word d>>1 / half d&1.
+template <bool FULL, int NT, int ST, int DS>
+__device__ __forceinline__ void pv_slice(float (&o)[NT][8 / DS][4], uint32_t st, int row0, int g, int t,
+                                         int d, const uint32_t (&pb)[NT][2], uint32_t magic) {
+  constexpr uint32_t VA = ST * 64, VR = ST * 192;
+  constexpr int NW = DS == 1 ? 2 : 1;  // words of the lane's 8 V bytes this warp touches
+  constexpr int NH = DS == 4 ? 1 : 2;  // halves of each word
+  const int ta = row0 + pi_row(2 * t), tb = row0 + pi_row(2 * t + 1);
+  uint32_t A[NW], Bw[NW], C[NW], Dw[NW], RA[NW], RB[NW], RC[NW], RD[NW];
+  const uint32_t wofs = DS == 1 ? 0u : (DS == 2 ? (uint32_t)d * 4u : (uint32_t)(d >> 1) * 4u);
+#pragma unroll
+  for (int i = 0; i < NW; ++i) {
+    const uint32_t off = g * 8 + wofs + i * 4;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(A[i]) : "r"(st + VA + ta * 64 + off));
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(Bw[i]) : "r"(st + VA + tb * 64 + off));
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(C[i]) : "r"(st + VA + (ta + 8) * 64 + off));
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(Dw[i]) : "r"(st + VA + (tb + 8) * 64 + off));
+    if (FULL) {
+      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RA[i]) : "r"(st + VR + ta * 64 + off));
+      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RB[i]) : "r"(st + VR + tb * 64 + off));
+      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RC[i]) : "r"(st + VR + (ta + 8) * 64 + off));
+      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RD[i]) : "r"(st + VR + (tb + 8) * 64 + off));
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < NW; ++i) {
+    uint32_t ea = 0, oa = 0, eb = 0, ob = 0, ec = 0, oc = 0, ed = 0, od = 0;
+    if (FULL) {
+      merge_codes(A[i], RA[i], ea, oa);
+      merge_codes(Bw[i], RB[i], eb, ob);
+      merge_codes(C[i], RC[i], ec, oc);
+      merge_codes(Dw[i], RD[i], ed, od);
+    }
+#pragma unroll
+    for (int hh = 0; hh < NH; ++hh) {
+      const int half = DS == 4 ? (d & 1) : hh;
+      const uint32_t sel = half ? 0x7632u : 0x5410u;
+      uint32_t ab[4], cd[4];
+      if (!FULL) {
+        nib4_to_h2(prmt(A[i], Bw[i], sel), magic, ab);  // dims e(4half+0..3), token pair (a, b)
+        nib4_to_h2(prmt(C[i], Dw[i], sel), magic, cd);  // same dims, token pair (c, d)
+      } else {
+        const uint32_t uab = prmt(ea, eb, sel), vab = prmt(oa, ob, sel);
+        const uint32_t ucd = prmt(ec, ed, sel), vcd = prmt(oc, od, sel);
+        ab[0] = hadd2(and_or<0x00FF00FFu>(uab, magic), kNeg1152);
+        ab[1] = hadd2(and_or<0x00FF00FFu>(vab, magic), kNeg1152);
+        ab[2] = hadd2(prmt(uab, magic, 0x7351), kNeg1152);
+        ab[3] = hadd2(prmt(vab, magic, 0x7351), kNeg1152);
+        cd[0] = hadd2(and_or<0x00FF00FFu>(ucd, magic), kNeg1152);
+        cd[1] = hadd2(and_or<0x00FF00FFu>(vcd, magic), kNeg1152);
+        cd[2] = hadd2(prmt(ucd, magic, 0x7351), kNeg1152);
+        cd[3] = hadd2(prmt(vcd, magic, 0x7351), kNeg1152);
+      }
+#pragma unroll
+      for (int qd = 0; qd < 2; ++qd) {
+        const int lm = (DS == 1 ? i * 4 : 0) + (DS == 4 ? 0 : hh * 2) + qd;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+          mma16816(o[nt][lm], ab[2 * qd], ab[2 * qd + 1], cd[2 * qd], cd[2 * qd + 1], pb[nt][0], pb[nt][1]);
+      }
+    }
+  }
+}
+
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB>
+__global__ void __launch_bounds__((DS * TEAMS + 1) * 32, MINB)
+attn_team_kernel(const AttnParams p) {
+  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE>;
+  constexpr int ST = C::kST, TW = C::kTW, MT = C::kMT;
+  constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
+  constexpr float kMidK = FULL ? 0.0f : 8.0f;
+  constexpr float kMidV = FULL ? 128.0f : 136.0f;
+  constexpr float kLevelScaleV = FULL ? 1.0f : 16.0f;
+  extern __shared__ __align__(128) unsigned char smem[];
+  unsigned char* ring = smem;
+  float* mail = reinterpret_cast<float*>(smem + C::kRing);
+  unsigned char* xchg = smem + C::kRing + C::kMailBytes;
+  float* lz = reinterpret_cast<float*>(xchg + C::kXchgBytes);
+  __nv_bfloat16* q_s = reinterpret_cast<__nv_bfloat16*>(xchg + C::kXchgBytes + C::kLzBytes);
+  uint32_t* blk_s = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(q_s) + C::kQBytes);
+  int4* info_s = reinterpret_cast<int4*>(reinterpret_cast<unsigned char*>(blk_s) + C::kBlkBytes);
+  Item* items = reinterpret_cast<Item*>(info_s + NSTAGE);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(info_s) + C::kInfoBytes);
+  int* misc = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(bars) + C::kBarBytes);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int cta = blockIdx.x;
+  const uint32_t ring_u32 = smem_u32(ring);
+  const uint32_t full0 = smem_u32(bars), empty0 = full0 + NSTAGE * 8;
+  const uint32_t qfull0 = empty0 + NSTAGE * 8, qempty0 = qfull0 + 16;
+  volatile int* abort_word = misc;
+
+  if (tid == 0) {
+    for (int i = 0; i < NSTAGE; ++i) {
+      mbar_init(full0 + i * 8, 1);
+      mbar_init(empty0 + i * 8, C::kConsWarps);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(qfull0 + i * 8, 1);
+      mbar_init(qempty0 + i * 8, C::kConsWarps);
+    }
+    misc[0] = 0; misc[1] = 0; misc[7] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = tid; i < C::kQBytes / 16; i += C::kThreads) reinterpret_cast<uint4*>(q_s)[i] = make_uint4(0, 0, 0, 0);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+
+  if (warp == C::kConsWarps) {
+    producer_warp<C, FULL, TW, NSTAGE>(p, lane, ring_u32, full0, empty0, qfull0, qempty0, q_s, blk_s,
+                                       info_s, items, misc, abort_word);
+    return;
+  }
+  __syncthreads();  // (A)
+  const int n_units = misc[7];
+  if (n_units == 0) return;
+
+  // per-warp exchange area: [flag (16 B)] [column maxima: kColsPad floats] [P^T: NT x 2 x 32 words]
+  constexpr int kXW = 16 + C::kColsPad * 4 + NT * 2 * 32 * 4;
+  const int g = lane >> 2, t = lane & 3;
+  const int team = warp / DS, d = warp % DS;
+  const float cb = p.sm_log2;
+  const uint32_t magic = opaque_magic();
+  uint32_t qf[NT][2][4][2];
+  float qs[NT][2], m[NT][2], l[NT][2], zs[NT][2], o[NT][MT][4];
+  int lim[NT][2];
+  bool fresh = true;
+  float ca = 0.0f;
+  int len = 0, full_lim = 0, ic = 0;
+  Item item;
+  item.b = 0; item.hkv = 0; item.len = 0; item.first_cta = 0; item.n_contrib = 1;
+
+  for (int gs = 0; gs < n_units; ++gs) {
+    const int slot = gs % NSTAGE;
+    mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
+    const int4 info = info_s[slot];
+    if (info.z & 1) {
+      const int qi = info.x & 1;
+      mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
+      item = items[qi];
+      len = item.len;
+      full_lim = p.causal ? len - p.nq + 1 : len;
+      const __nv_bfloat16* qb = q_s + (size_t)qi * C::kColsPad * LYNX_D;
+      float amax = 0.0f;
+      for (int i = lane; i < C::kColsPad * (LYNX_D / 8); i += 32) {
+        const uint4 v = reinterpret_cast<const uint4*>(qb)[i];
+        const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          amax = fmaxf(amax, fabsf(__uint_as_float(ww[k] << 16)));
+          amax = fmaxf(amax, fabsf(__uint_as_float(ww[k] & 0xFFFF0000u)));
+        }
+      }
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, off));
+      int e = 0;  // two s8 digit planes of q, see attn_kernel
+      if (amax > 0.0f && amax < INFINITY) e = 13 - (((__float_as_int(amax) >> 23) & 0xFF) - 127);
+      e = max(-100, min(100, e));
+      const float up = __int_as_float((127 + e) << 23), down = __int_as_float((127 - e) << 23);
+      ca = p.sm_log2 * down * (FULL ? 1.0f : 16.0f);
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const int c = nt * 8 + g;
+#pragma unroll
+        for (int wd = 0; wd < 4; ++wd) {
+          const uint4 v = *reinterpret_cast<const uint4*>(qb + c * LYNX_D + 32 * t + 8 * wd);
+          const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+          int qv[8];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            qv[2 * k] = __float2int_rn(__uint_as_float(ww[k] << 16) * up);
+            qv[2 * k + 1] = __float2int_rn(__uint_as_float(ww[k] & 0xFFFF0000u) * up);
+          }
+          uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            hi_e |= (uint32_t)((qv[2 * k] >> 7) & 0xFF) << (8 * k);
+            lo_e |= (uint32_t)(qv[2 * k] & 127) << (8 * k);
+            hi_o |= (uint32_t)((qv[2 * k + 1] >> 7) & 0xFF) << (8 * k);
+            lo_o |= (uint32_t)(qv[2 * k + 1] & 127) << (8 * k);
+          }
+          qf[nt][0][wd][0] = hi_e; qf[nt][0][wd][1] = hi_o;
+          qf[nt][1][wd][0] = lo_e; qf[nt][1][wd][1] = lo_o;
+        }
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+          const int col = nt * 8 + 2 * t + cc;
+          const uint4* qq = reinterpret_cast<const uint4*>(qb + col * LYNX_D + 16 * g);
+          float sum = 0.0f;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const uint4 v = qq[h];
+            const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              sum += __uint_as_float(ww[k] << 16) + __uint_as_float(ww[k] & 0xFFFF0000u);
+          }
+          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 4);
+          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 8);
+          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 16);
+          qs[nt][cc] = sum;
+          const int j = col / p.G;
+          lim[nt][cc] = col < p.ncols ? (p.causal ? len - p.nq + j + 1 : len) : 0;
+          m[nt][cc] = 0.0f; l[nt][cc] = 0.0f; zs[nt][cc] = 0.0f;
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) o[nt][mt][i] = 0.0f;
+      }
+      fresh = true;
+    }
+
+    const uint32_t st = ring_u32 + slot * C::kStageBytes;
+    const int unit_t0 = info.y * ST;
+    const int tile_t0 = unit_t0 + warp * 16;
+    const bool valid = tile_t0 < len;                             // this warp's own tile
+    const bool team_valid = unit_t0 + team * DS * 16 < len;       // the team's first tile
+    unsigned char* my_x = xchg + (size_t)warp * kXW;
+    float s[NT][4];
+    float2 vm_lo = make_float2(0.f, 0.f), vm_hi = make_float2(0.f, 0.f);
+    const int r0 = warp * 16 + pi_row(g);
+    const int tok_lo = tile_t0 + pi_row(g), tok_hi = tok_lo + 8;
+    const bool masked = tile_t0 + 16 > full_lim;
+    // ---- phase A: scores of this warp's tile, growth vote -------------------------------
+    bool gw = false;
+    if (valid) {
+      qk_int8<FULL, NT, ST>(qf, st, r0, t, s);
+      float2 km_lo = lds64f(st + KM + r0 * 8), km_hi = lds64f(st + KM + (r0 + 8) * 8);
+      vm_lo = lds64f(st + VM + r0 * 8); vm_hi = lds64f(st + VM + (r0 + 8) * 8);
+      if (masked) {
+        int maxlim = 0;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) maxlim = max(maxlim, max(lim[nt][0], lim[nt][1]));
+        maxlim = max(maxlim, __shfl_xor_sync(0xFFFFFFFFu, maxlim, 1));
+        maxlim = max(maxlim, __shfl_xor_sync(0xFFFFFFFFu, maxlim, 2));
+        if (tok_lo >= maxlim) { km_lo = make_float2(0.f, 0.f); vm_lo = make_float2(0.f, 0.f); }
+        if (tok_hi >= maxlim) { km_hi = make_float2(0.f, 0.f); vm_hi = make_float2(0.f, 0.f); }
+      }
+      const float al_lo = km_lo.x * ca, al_hi = km_hi.x * ca;
+      const float be_lo = fmaf(km_lo.x, kMidK, km_lo.y) * cb, be_hi = fmaf(km_hi.x, kMidK, km_hi.y) * cb;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        s[nt][0] = fmaf(al_lo, s[nt][0], fmaf(be_lo, qs[nt][0], -m[nt][0]));
+        s[nt][1] = fmaf(al_lo, s[nt][1], fmaf(be_lo, qs[nt][1], -m[nt][1]));
+        s[nt][2] = fmaf(al_hi, s[nt][2], fmaf(be_hi, qs[nt][0], -m[nt][0]));
+        s[nt][3] = fmaf(al_hi, s[nt][3], fmaf(be_hi, qs[nt][1], -m[nt][1]));
+        if (masked) {
+          if (tok_lo >= lim[nt][0]) s[nt][0] = -INFINITY;
+          if (tok_lo >= lim[nt][1]) s[nt][1] = -INFINITY;
+          if (tok_hi >= lim[nt][0]) s[nt][2] = -INFINITY;
+          if (tok_hi >= lim[nt][1]) s[nt][3] = -INFINITY;
+        }
+        gw |= fmaxf(fmaxf(s[nt][0], s[nt][2]), fmaxf(s[nt][1], s[nt][3])) > 4.0f;
+      }
+      gw = __any_sync(0xFFFFFFFFu, gw) || fresh;
+      if (gw) {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            float mx = fmaxf(s[nt][cc], s[nt][cc + 2]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));
+            if (g == 0) reinterpret_cast<float*>(my_x + 16)[nt * 8 + 2 * t + cc] = mx;
+          }
+      }
+    }
+    if (lane == 0) *reinterpret_cast<int*>(my_x) = gw ? 1 : 0;
+    named_bar(2 + team, DS * 32);
+    // ---- agree on the running maxima ----------------------------------------------------
+    {
+      bool any = false;
+      int flags[DS];
+#pragma unroll
+      for (int dd = 0; dd < DS; ++dd) {
+        flags[dd] = *reinterpret_cast<const volatile int*>(xchg + (size_t)(team * DS + dd) * kXW);
+        any |= flags[dd] != 0;
+      }
+      if (any) {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            float mx = -INFINITY;
+#pragma unroll
+            for (int dd = 0; dd < DS; ++dd)
+              if (flags[dd])
+                mx = fmaxf(mx, reinterpret_cast<const volatile float*>(xchg + (size_t)(team * DS + dd) * kXW + 16)[nt * 8 + 2 * t + cc]);
+            const float up = fresh ? fmaxf(mx, -1.0e4f) : fmaxf(mx, 0.0f);
+            const float f = fresh ? 0.0f : ex2(-up);
+            m[nt][cc] += up;
+            s[nt][cc] -= up;
+            s[nt][cc + 2] -= up;
+            l[nt][cc] *= f;
+            zs[nt][cc] *= f;
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+              o[nt][mt][cc] *= f;
+              o[nt][mt][cc + 2] *= f;
+            }
+          }
+      }
+      if (team_valid) fresh = false;
+    }
+    // ---- weights of this warp's tile, P^T fragments to shared memory ---------------------
+    if (valid) {
+      const float sv_lo = vm_lo.x * kLevelScaleV, sv_hi = vm_hi.x * kLevelScaleV;
+      const float zv_lo = fmaf(vm_lo.x, kMidV, vm_lo.y), zv_hi = fmaf(vm_hi.x, kMidV, vm_hi.y);
+      uint32_t* pf = reinterpret_cast<uint32_t*>(my_x + 16 + C::kColsPad * 4) + lane;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const float p0 = ex2(s[nt][0]), p1 = ex2(s[nt][1]);
+        const float p2 = ex2(s[nt][2]), p3 = ex2(s[nt][3]);
+        l[nt][0] += p0 + p2;
+        l[nt][1] += p1 + p3;
+        zs[nt][0] = fmaf(p0, zv_lo, fmaf(p2, zv_hi, zs[nt][0]));
+        zs[nt][1] = fmaf(p1, zv_lo, fmaf(p3, zv_hi, zs[nt][1]));
+        pf[(nt * 2 + 0) * 32] = movmatrix_trans(pack_f16x2(p0 * sv_lo, p1 * sv_lo));
+        pf[(nt * 2 + 1) * 32] = movmatrix_trans(pack_f16x2(p2 * sv_hi, p3 * sv_hi));
+      }
+    }
+    named_bar(2 + team, DS * 32);
+    // ---- phase C: P.V of the team's tiles for this warp's slice of the output dims --------
+#pragma unroll
+    for (int tau = 0; tau < DS; ++tau) {
+      const int src = team * DS + tau;
+      if (unit_t0 + src * 16 >= len) break;  // uniform: later tiles of the unit are beyond len too
+      uint32_t pb[NT][2];
+      const uint32_t* pf = reinterpret_cast<const uint32_t*>(xchg + (size_t)src * kXW + 16 + C::kColsPad * 4) + lane;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        pb[nt][0] = *reinterpret_cast<const volatile uint32_t*>(pf + (nt * 2 + 0) * 32);
+        pb[nt][1] = *reinterpret_cast<const volatile uint32_t*>(pf + (nt * 2 + 1) * 32);
+      }
+      pv_slice<FULL, NT, ST, DS>(o, st, src * 16, g, t, d, pb, magic);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty0 + slot * 8);
+    if (!(info.z & 2)) continue;
+
+    // ---- end of the piece -----------------------------------------------------------------
+    if (fresh) {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) m[nt][0] = m[nt][1] = -1.0e30f;
+    }
+    // teams 1.. are absorbed into team 0, slice by slice, through lane-private mailboxes
+    for (int src = 1; src < TEAMS; ++src) {
+      float* box = mail + (size_t)d * C::kMailRegs * 32 + lane;
+      if (team == src) {
+        int r = 0;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) box[(r++) * 32] = o[nt][mt][i];
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            box[(r++) * 32] = m[nt][cc];
+            box[(r++) * 32] = l[nt][cc];
+            box[(r++) * 32] = zs[nt][cc];
+          }
+        }
+      }
       named_bar(1, C::kConsThreads);
-      if (tid == 0)
-        misc[1] = (atomicInc(p.ws_chunk_ctr + bh, (uint32_t)item.n_contrib - 1) == (uint32_t)item.n_contrib - 1);
+      if (team == 0) {
+        int r = 0;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          float f1[2], f2[2];
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            const float m2 = box[((MT * 4 + 6) * nt + MT * 4 + 3 * cc) * 32];
+            const float M = fmaxf(m[nt][cc], m2);
+            f1[cc] = ex2(m[nt][cc] - M);
+            f2[cc] = ex2(m2 - M);
+            m[nt][cc] = M;
+          }
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float o2 = box[(r++) * 32];
+              o[nt][mt][i] = o[nt][mt][i] * f1[i & 1] + o2 * f2[i & 1];
+            }
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            r++;
+            const float l2 = box[(r++) * 32];
+            const float z2 = box[(r++) * 32];
+            l[nt][cc] = l[nt][cc] * f1[cc] + l2 * f2[cc];
+            zs[nt][cc] = zs[nt][cc] * f1[cc] + z2 * f2[cc];
+          }
+        }
+      }
       named_bar(1, C::kConsThreads);
-      final_here = misc[1] != 0;
-      if (final_here) {
-        __threadfence();
-        const float* base = p.ws_part + (bh + (size_t)item.first_cta) * (size_t)C::kColsPad * kPartStride;
-        const size_t cstride = (size_t)C::kColsPad * kPartStride;
-        for (int idx = tid; idx < C::kColsPad * LYNX_D; idx += C::kConsThreads) {
-          const int c = idx >> 7, d = idx & 127;
+    }
+    // team 0: totals of l and zs over its DS warps (each saw different tokens)
+    if (team == 0) {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+          float lv = l[nt][cc], z = zs[nt][cc];
+#pragma unroll
+          for (int off = 4; off <= 16; off <<= 1) {
+            lv += __shfl_xor_sync(0xFFFFFFFFu, lv, off);
+            z += __shfl_xor_sync(0xFFFFFFFFu, z, off);
+          }
+          if (g == 0) {
+            lz[((size_t)d * C::kColsPad + nt * 8 + 2 * t + cc) * 2 + 0] = lv;
+            lz[((size_t)d * C::kColsPad + nt * 8 + 2 * t + cc) * 2 + 1] = z;
+          }
+        }
+    }
+    named_bar(1, C::kConsThreads);
+    const bool direct = item.n_contrib == 1;
+    if (team == 0) {
+      const size_t bh = (size_t)item.b * p.Hkv + item.hkv;
+      float* part = p.ws_part + (bh + (size_t)cta) * (size_t)C::kColsPad * kPartStride;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+          const int c = nt * 8 + 2 * t + cc;
+          float lt = 0.0f, z = 0.0f;
+#pragma unroll
+          for (int dd = 0; dd < DS; ++dd) {
+            lt += lz[((size_t)dd * C::kColsPad + c) * 2 + 0];
+            z += lz[((size_t)dd * C::kColsPad + c) * 2 + 1];
+          }
           if (c >= p.ncols) continue;
-          const float* col = base + (size_t)c * kPartStride;
-          float M = -INFINITY;
-          for (int i = 0; i < item.n_contrib; ++i) M = fmaxf(M, __ldcg(col + i * cstride + 128));
-          float acc = 0.0f, L = 0.0f;
-          for (int i = 0; i < item.n_contrib; ++i) {
-            const float f = ex2(__ldcg(col + i * cstride + 128) - M);
-            acc = fmaf(__ldcg(col + i * cstride + d), f, acc);
-            L = fmaf(__ldcg(col + i * cstride + 129), f, L);
-          }
           const int j = c / p.G, hh = c % p.G;
-          p.out[(((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
+          float* dst = direct ? p.out + (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D
+                              : part + (size_t)c * kPartStride;
+          const float inv = direct ? (lt > 0.0f ? 1.0f / lt : 0.0f) : 1.0f;
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            const int gmt = d * MT + mt;  // m-tile index among the eight of a lane's 16 dims
+            const int dim = 16 * g + 8 * (gmt >> 2) + 2 * (gmt & 3);
+            *reinterpret_cast<float2*>(dst + dim) =
+                make_float2((o[nt][mt][cc] + z) * inv, (o[nt][mt][cc + 2] + z) * inv);
+          }
+          if (!direct && d == 0 && g == 0) { dst[128] = m[nt][cc]; dst[129] = lt; }
         }
       }
+      __threadfence();
     }
-    // accept / reject (Section 4.3): by the CTA that wrote the final outputs of this head
-    if (FULL && p.draft != nullptr) {
-      int* devs = misc + 16;
-      named_bar(1, C::kConsThreads);  // final outputs written; devs free
-      if (final_here) {
-        if (tid < kMaxQ) devs[tid] = 0;
-        named_bar(1, C::kConsThreads);
-        for (int idx = tid; idx < p.ncols * LYNX_D; idx += C::kConsThreads) {
-          const int c = idx >> 7, d = idx & 127;
-          const int j = c / p.G, hh = c % p.G;
-          const size_t o = (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + d;
-          const float f = p.out[o], dr = __ldg(p.draft + o);
-          const float r = fabsf(f - dr) / (p.atol + p.rtol * fabsf(f));
-          atomicMax(devs + j, __float_as_int(r));  // r >= 0: integer order = float order
-        }
-        named_bar(1, C::kConsThreads);
-        if (tid < p.nq) p.ws_dev[bh * kMaxQ + tid] = __int_as_float(devs[tid]);
-        __threadfence();
-        named_bar(1, C::kConsThreads);
-        if (tid == 0)
-          misc[1] = (atomicInc(p.ws_seq_ctr + item.b, (uint32_t)p.Hkv - 1) == (uint32_t)p.Hkv - 1);
-        named_bar(1, C::kConsThreads);
-        if (misc[1] && tid == 0) {
-          __threadfence();
-          int fr = p.nq;
-          for (int j = p.nq - 1; j >= 0; --j) {
-            float worst = 0.0f;
-            for (int h = 0; h < p.Hkv; ++h)
-              worst = fmaxf(worst, __ldcg(p.ws_dev + ((size_t)item.b * p.Hkv + h) * kMaxQ + j));
-            p.dev[(size_t)item.b * p.nq + j] = worst;
-            if (worst > 1.0f) fr = j;
-          }
-          p.first_reject[item.b] = fr;
-        }
-      }
-      named_bar(1, C::kConsThreads);
-    }
+    finish_piece<FULL, C::kColsPad, C::kConsThreads>(p, item, direct, tid, misc);
     __syncwarp();
     if (lane == 0) mbar_arrive(qempty0 + (info.x & 1) * 8);
     ++ic;
@@ -1013,6 +1527,25 @@ lynx_status launch(const AttnParams& p, cudaStream_t st) {
   return launch_status();
 }
 
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB>
+lynx_status launch_team(const AttnParams& p, cudaStream_t st) {
+  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE>;
+  static_assert(MINB <= kMaxCtasPerSm, "partial slots are sized for kMaxCtasPerSm CTAs per SM");
+  static_assert(MINB * (C::kSmem + 1024) <= 228 * 1024, "shared memory budget for MINB CTAs per SM");
+  static_assert(2 + TEAMS <= 16, "named barriers");
+  auto kern = attn_team_kernel<FULL, NT, DS, TEAMS, NSTAGE, MINB>;
+  static bool configured[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmem) != cudaSuccess)
+      return LYNX_ERR_CUDA;
+    configured[dev] = true;
+  }
+  kern<<<sm_count() * MINB, C::kThreads, C::kSmem, st>>>(p);
+  return launch_status();
+}
+
 lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int B, int nq, int causal,
                           lynx_plane K, lynx_plane V, const int32_t* block_table,
                           const int32_t* seq_lens, float softmax_scale, const float* draft,
@@ -1059,14 +1592,14 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   if (!full) {
     switch (pl.variant) {
       case 0: return launch<false, 1, 4, 1, 4, 4>(p, st);
-      case 1: return launch<false, 2, 4, 1, 4, 3>(p, st);
+      case 1: return launch_team<false, 2, 2, 2, 4, 3>(p, st);
       case 2: return launch<false, 2, 4, 2, 6, 1>(p, st);
       default: return launch<false, 2, 2, 4, 12, 1>(p, st);
     }
   }
   switch (pl.variant) {
     case 0: return launch<true, 1, 4, 1, 3, 3>(p, st);
-    case 1: return launch<true, 2, 4, 1, 3, 3>(p, st);
+    case 1: return launch_team<true, 2, 2, 2, 3, 3>(p, st);
     case 2: return launch<true, 2, 4, 2, 5, 1>(p, st);
     default: return launch<true, 2, 2, 4, 8, 1>(p, st);
   }
