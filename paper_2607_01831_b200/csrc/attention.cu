@@ -616,26 +616,29 @@ __device__ __forceinline__ void producer_warp(const AttnParams& p, int lane, uin
   if (n_units == 0) return;
 
   // =============================== producer loop ===============================
-  // every lane below TW*NARR has a fixed role: one array of one 16-token sub-block per stage
+  // every lane has fixed roles: role r = lane + 32 i copies one array of one 16-token sub-block
   constexpr int NARR = FULL ? 6 : 4;
-  static_assert(TW * NARR <= 32, "one copy per producer lane");
-  const int my_sub = lane < TW * NARR ? lane / NARR : TW;  // TW = no role
-  const int my_arr = lane % NARR;
-  const unsigned char* my_src;
-  uint32_t my_mul, my_dst, my_bytes;
-  {
-    const bool is_meta = my_arr == 2 || my_arr == 3;
-    my_src = my_arr == 0 ? p.ka : my_arr == 1 ? p.va
-           : my_arr == 2 ? reinterpret_cast<const unsigned char*>(p.km)
-           : my_arr == 3 ? reinterpret_cast<const unsigned char*>(p.vm)
-           : my_arr == 4 ? p.kr : p.vr;
-    const uint32_t dst0 = my_arr == 0 ? 0u : my_arr == 1 ? ST * 64u
-                        : my_arr == 2 ? (FULL ? ST * 256u : ST * 128u)
-                        : my_arr == 3 ? (FULL ? ST * 264u : ST * 136u)
-                        : my_arr == 4 ? ST * 128u : ST * 192u;
-    my_mul = is_meta ? 8u : 64u;
-    my_bytes = is_meta ? 128u : 1024u;
-    my_dst = dst0 + (uint32_t)(my_sub < TW ? my_sub : 0) * my_bytes;
+  constexpr int NROLE = (TW * NARR + 31) / 32;
+  int my_sub[NROLE];
+  const unsigned char* my_src[NROLE];
+  uint32_t my_mul[NROLE], my_dst[NROLE], my_bytes[NROLE];
+#pragma unroll
+  for (int i = 0; i < NROLE; ++i) {
+    const int r = lane + 32 * i;
+    my_sub[i] = r < TW * NARR ? r / NARR : TW;  // TW = no role
+    const int arr = r % NARR;
+    const bool is_meta = arr == 2 || arr == 3;
+    my_src[i] = arr == 0 ? p.ka : arr == 1 ? p.va
+              : arr == 2 ? reinterpret_cast<const unsigned char*>(p.km)
+              : arr == 3 ? reinterpret_cast<const unsigned char*>(p.vm)
+              : arr == 4 ? p.kr : p.vr;
+    const uint32_t dst0 = arr == 0 ? 0u : arr == 1 ? ST * 64u
+                        : arr == 2 ? (FULL ? ST * 256u : ST * 128u)
+                        : arr == 3 ? (FULL ? ST * 264u : ST * 136u)
+                        : arr == 4 ? ST * 128u : ST * 192u;
+    my_mul[i] = is_meta ? 8u : 64u;
+    my_bytes[i] = is_meta ? 128u : 1024u;
+    my_dst[i] = dst0 + (uint32_t)(my_sub[i] < TW ? my_sub[i] : 0) * my_bytes[i];
   }
   int b = b_lo, len = clamp_len(b), U = (len + ST - 1) / ST;
   int hkv = (int)(off_lo / U), u = (int)(off_lo % U);
@@ -686,9 +689,11 @@ __device__ __forceinline__ void producer_warp(const AttnParams& p, int lane, uin
           mbar_expect_tx(bar, nsub * C::kSubBytes);
         }
         __syncwarp();
-        if (my_sub < nsub)
-          bulk_g2s(ring_u32 + slot * C::kStageBytes + my_dst, my_src + (size_t)blk_s[k * TW + my_sub] * my_mul,
-                   my_bytes, bar);
+#pragma unroll
+        for (int i = 0; i < NROLE; ++i)
+          if (my_sub[i] < nsub)
+            bulk_g2s(ring_u32 + slot * C::kStageBytes + my_dst[i],
+                     my_src[i] + (size_t)blk_s[k * TW + my_sub[i]] * my_mul[i], my_bytes[i], bar);
       }
       __syncwarp();  // blk_s is rewritten by the next round
     }
@@ -1003,17 +1008,47 @@ struct TeamCfg {
   static constexpr int kMT = 8 / DS;                        // m-tiles (16 dims) per warp
   static constexpr int kRing = NSTAGE * kStageBytes;
   static constexpr int kMailRegs = NT * kMT * 4 + NT * 6;   // o slice + m, l, zs
-  static constexpr int kMailBytes = DS * kMailRegs * 32 * 4;
+  static constexpr int kMailBytes = TEAMS > 1 ? kMailRegs * 32 * 4 : 0;  // one box, used slice by slice
   static constexpr int kXchgBytes = kTW * (16 + kColsPad * 4 + NT * 2 * 32 * 4);  // flag, colmax, P^T
   static constexpr int kLzBytes = DS * kColsPad * 2 * 4;
+  static constexpr bool kQfShared = NT > 2;                 // query fragments in shared memory
+  static constexpr int kQfBytes = kQfShared ? NT * 2 * 4 * 32 * 8 + kColsPad * 4 : 0;
   static constexpr int kQBytes = 2 * kColsPad * LYNX_D * 2;
   static constexpr int kBlkBytes = kPieceUnits * kTW * 4;
   static constexpr int kInfoBytes = NSTAGE * 16 + 2 * 32;
   static constexpr int kBarBytes = (2 * NSTAGE + 4) * 8;
   static constexpr int kMiscBytes = 256;
-  static constexpr int kSmem = kRing + kMailBytes + kXchgBytes + kLzBytes + kQBytes + kBlkBytes +
-                               kInfoBytes + kBarBytes + kMiscBytes;
+  static constexpr int kSmem = kRing + kMailBytes + kXchgBytes + kLzBytes + kQfBytes + kQBytes +
+                               kBlkBytes + kInfoBytes + kBarBytes + kMiscBytes;
 };
+
+// K operand fragments of one tile for all four k32 steps: a[wd] = {ev(row g), ev(row g+8),
+// od(row g), od(row g+8)} (ev/od: levels of the even / odd elements of word wd).
+template <bool FULL, int ST>
+__device__ __forceinline__ void k_fragments(uint32_t st, int r0, int t, uint32_t (&a)[4][4]) {
+  constexpr uint32_t KA = 0, KR = ST * 128;
+  const uint4 a_lo = lds128(st + KA + r0 * 64 + t * 16);
+  const uint4 a_hi = lds128(st + KA + (r0 + 8) * 64 + t * 16);
+  const uint32_t xl[4] = {a_lo.x, a_lo.y, a_lo.z, a_lo.w};
+  const uint32_t xh[4] = {a_hi.x, a_hi.y, a_hi.z, a_hi.w};
+  if (FULL) {
+    const uint4 b_lo = lds128(st + KR + r0 * 64 + t * 16);
+    const uint4 b_hi = lds128(st + KR + (r0 + 8) * 64 + t * 16);
+    const uint32_t yl[4] = {b_lo.x, b_lo.y, b_lo.z, b_lo.w};
+    const uint32_t yh[4] = {b_hi.x, b_hi.y, b_hi.z, b_hi.w};
+#pragma unroll
+    for (int wd = 0; wd < 4; ++wd) {
+      merge_codes(xl[wd], yl[wd], a[wd][0], a[wd][2]);
+      merge_codes(xh[wd], yh[wd], a[wd][1], a[wd][3]);
+    }
+  } else {
+#pragma unroll
+    for (int wd = 0; wd < 4; ++wd) {
+      a[wd][0] = xl[wd] & 0x0F0F0F0Fu; a[wd][2] = (xl[wd] >> 4) & 0x0F0F0F0Fu;
+      a[wd][1] = xh[wd] & 0x0F0F0F0Fu; a[wd][3] = (xh[wd] >> 4) & 0x0F0F0F0Fu;
+    }
+  }
+}
 
 // O^T slice += level(V)^T[slice dims x 16 tokens] . P^T for one tile (stage rows row0..row0+15).
 // Slice d of DS covers the m-tiles (word, half) of every lane's 16 dims: DS=1 all eight, DS=2
@@ -1095,7 +1130,9 @@ attn_team_kernel(const AttnParams p) {
   float* mail = reinterpret_cast<float*>(smem + C::kRing);
   unsigned char* xchg = smem + C::kRing + C::kMailBytes;
   float* lz = reinterpret_cast<float*>(xchg + C::kXchgBytes);
-  __nv_bfloat16* q_s = reinterpret_cast<__nv_bfloat16*>(xchg + C::kXchgBytes + C::kLzBytes);
+  unsigned char* qf_s = xchg + C::kXchgBytes + C::kLzBytes;   // [nt][plane][wd][lane] uint2, then qs[col]
+  float* qs_s = reinterpret_cast<float*>(qf_s + NT * 2 * 4 * 32 * 8);
+  __nv_bfloat16* q_s = reinterpret_cast<__nv_bfloat16*>(xchg + C::kXchgBytes + C::kLzBytes + C::kQfBytes);
   uint32_t* blk_s = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(q_s) + C::kQBytes);
   int4* info_s = reinterpret_cast<int4*>(reinterpret_cast<unsigned char*>(blk_s) + C::kBlkBytes);
   Item* items = reinterpret_cast<Item*>(info_s + NSTAGE);
@@ -1139,9 +1176,15 @@ attn_team_kernel(const AttnParams p) {
   const int team = warp / DS, d = warp % DS;
   const float cb = p.sm_log2;
   const uint32_t magic = opaque_magic();
-  uint32_t qf[NT][2][4][2];
-  float qs[NT][2], m[NT][2], l[NT][2], zs[NT][2], o[NT][MT][4];
-  int lim[NT][2];
+  constexpr bool QFS = C::kQfShared;
+  constexpr int NTR = QFS ? 1 : NT;  // register copies exist only when the fragments are not shared
+  uint32_t qf[NTR][2][4][2];
+  float qs[NTR][2], m[NT][2], l[NT][2], zs[NT][2], o[NT][MT][4];
+  int lim[NTR][2];
+  const uint32_t qf_u32 = smem_u32(qf_s), qs_u32 = smem_u32(qs_s);
+  auto col_limit = [&](int col, int len_) {
+    return col < p.ncols ? (p.causal ? len_ - p.nq + col / p.G + 1 : len_) : 0;
+  };
   bool fresh = true;
   float ca = 0.0f;
   int len = 0, full_lim = 0, ic = 0;
@@ -1178,54 +1221,68 @@ attn_team_kernel(const AttnParams p) {
       ca = p.sm_log2 * down * (FULL ? 1.0f : 16.0f);
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        const int c = nt * 8 + g;
+        // with shared fragments, warp w builds the n-tiles nt = w, w + TW, ... for everybody
+        const bool mine = !QFS || (nt % TW) == warp;
+        if (mine) {
+          const int c = nt * 8 + g;
 #pragma unroll
-        for (int wd = 0; wd < 4; ++wd) {
-          const uint4 v = *reinterpret_cast<const uint4*>(qb + c * LYNX_D + 32 * t + 8 * wd);
-          const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
-          int qv[8];
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            qv[2 * k] = __float2int_rn(__uint_as_float(ww[k] << 16) * up);
-            qv[2 * k + 1] = __float2int_rn(__uint_as_float(ww[k] & 0xFFFF0000u) * up);
-          }
-          uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            hi_e |= (uint32_t)((qv[2 * k] >> 7) & 0xFF) << (8 * k);
-            lo_e |= (uint32_t)(qv[2 * k] & 127) << (8 * k);
-            hi_o |= (uint32_t)((qv[2 * k + 1] >> 7) & 0xFF) << (8 * k);
-            lo_o |= (uint32_t)(qv[2 * k + 1] & 127) << (8 * k);
-          }
-          qf[nt][0][wd][0] = hi_e; qf[nt][0][wd][1] = hi_o;
-          qf[nt][1][wd][0] = lo_e; qf[nt][1][wd][1] = lo_o;
-        }
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          const int col = nt * 8 + 2 * t + cc;
-          const uint4* qq = reinterpret_cast<const uint4*>(qb + col * LYNX_D + 16 * g);
-          float sum = 0.0f;
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const uint4 v = qq[h];
+          for (int wd = 0; wd < 4; ++wd) {
+            const uint4 v = *reinterpret_cast<const uint4*>(qb + c * LYNX_D + 32 * t + 8 * wd);
             const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+            int qv[8];
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              sum += __uint_as_float(ww[k] << 16) + __uint_as_float(ww[k] & 0xFFFF0000u);
+            for (int k = 0; k < 4; ++k) {
+              qv[2 * k] = __float2int_rn(__uint_as_float(ww[k] << 16) * up);
+              qv[2 * k + 1] = __float2int_rn(__uint_as_float(ww[k] & 0xFFFF0000u) * up);
+            }
+            uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              hi_e |= (uint32_t)((qv[2 * k] >> 7) & 0xFF) << (8 * k);
+              lo_e |= (uint32_t)(qv[2 * k] & 127) << (8 * k);
+              hi_o |= (uint32_t)((qv[2 * k + 1] >> 7) & 0xFF) << (8 * k);
+              lo_o |= (uint32_t)(qv[2 * k + 1] & 127) << (8 * k);
+            }
+            if constexpr (QFS) {
+              reinterpret_cast<uint2*>(qf_s)[((nt * 2 + 0) * 4 + wd) * 32 + lane] = make_uint2(hi_e, hi_o);
+              reinterpret_cast<uint2*>(qf_s)[((nt * 2 + 1) * 4 + wd) * 32 + lane] = make_uint2(lo_e, lo_o);
+            } else {
+              qf[nt][0][wd][0] = hi_e; qf[nt][0][wd][1] = hi_o;
+              qf[nt][1][wd][0] = lo_e; qf[nt][1][wd][1] = lo_o;
+            }
           }
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 4);
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 8);
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 16);
-          qs[nt][cc] = sum;
-          const int j = col / p.G;
-          lim[nt][cc] = col < p.ncols ? (p.causal ? len - p.nq + j + 1 : len) : 0;
-          m[nt][cc] = 0.0f; l[nt][cc] = 0.0f; zs[nt][cc] = 0.0f;
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            const int col = nt * 8 + 2 * t + cc;
+            const uint4* qq = reinterpret_cast<const uint4*>(qb + col * LYNX_D + 16 * g);
+            float sum = 0.0f;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const uint4 v = qq[h];
+              const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                sum += __uint_as_float(ww[k] << 16) + __uint_as_float(ww[k] & 0xFFFF0000u);
+            }
+            sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 4);
+            sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 8);
+            sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 16);
+            if constexpr (QFS) {
+              if (g == 0) qs_s[col] = sum;
+            } else {
+              qs[nt][cc] = sum;
+              lim[nt][cc] = col_limit(col, len);
+            }
+          }
         }
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) { m[nt][cc] = 0.0f; l[nt][cc] = 0.0f; zs[nt][cc] = 0.0f; }
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
           for (int i = 0; i < 4; ++i) o[nt][mt][i] = 0.0f;
       }
+      if constexpr (QFS) named_bar(1, C::kConsThreads);  // the shared fragments are complete
       fresh = true;
     }
 
@@ -1243,13 +1300,32 @@ attn_team_kernel(const AttnParams p) {
     // ---- phase A: scores of this warp's tile, growth vote -------------------------------
     bool gw = false;
     if (valid) {
-      qk_int8<FULL, NT, ST>(qf, st, r0, t, s);
+      if constexpr (QFS) {
+        uint32_t a[4][4];
+        k_fragments<FULL, ST>(st, r0, t, a);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          int shi[4] = {0, 0, 0, 0}, slo[4] = {0, 0, 0, 0};
+#pragma unroll
+          for (int wd = 0; wd < 4; ++wd) {
+            const uint2 bh = lds64(qf_u32 + (((nt * 2 + 0) * 4 + wd) * 32 + lane) * 8);
+            const uint2 bl = lds64(qf_u32 + (((nt * 2 + 1) * 4 + wd) * 32 + lane) * 8);
+            mma_u8s8(shi, a[wd][0], a[wd][1], a[wd][2], a[wd][3], bh.x, bh.y);
+            mma_u8s8(slo, a[wd][0], a[wd][1], a[wd][2], a[wd][3], bl.x, bl.y);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) s[nt][i] = (float)(shi[i] * 128 + slo[i]);
+        }
+      } else {
+        qk_int8<FULL, NT, ST>(qf, st, r0, t, s);
+      }
       float2 km_lo = lds64f(st + KM + r0 * 8), km_hi = lds64f(st + KM + (r0 + 8) * 8);
       vm_lo = lds64f(st + VM + r0 * 8); vm_hi = lds64f(st + VM + (r0 + 8) * 8);
       if (masked) {
         int maxlim = 0;
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) maxlim = max(maxlim, max(lim[nt][0], lim[nt][1]));
+        for (int nt = 0; nt < NT; ++nt)
+          maxlim = max(maxlim, max(col_limit(nt * 8 + 2 * t, len), col_limit(nt * 8 + 2 * t + 1, len)));
         maxlim = max(maxlim, __shfl_xor_sync(0xFFFFFFFFu, maxlim, 1));
         maxlim = max(maxlim, __shfl_xor_sync(0xFFFFFFFFu, maxlim, 2));
         if (tok_lo >= maxlim) { km_lo = make_float2(0.f, 0.f); vm_lo = make_float2(0.f, 0.f); }
@@ -1259,15 +1335,24 @@ attn_team_kernel(const AttnParams p) {
       const float be_lo = fmaf(km_lo.x, kMidK, km_lo.y) * cb, be_hi = fmaf(km_hi.x, kMidK, km_hi.y) * cb;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        s[nt][0] = fmaf(al_lo, s[nt][0], fmaf(be_lo, qs[nt][0], -m[nt][0]));
-        s[nt][1] = fmaf(al_lo, s[nt][1], fmaf(be_lo, qs[nt][1], -m[nt][1]));
-        s[nt][2] = fmaf(al_hi, s[nt][2], fmaf(be_hi, qs[nt][0], -m[nt][0]));
-        s[nt][3] = fmaf(al_hi, s[nt][3], fmaf(be_hi, qs[nt][1], -m[nt][1]));
+        float q0, q1;
+        if constexpr (QFS) {
+          const float2 qq = lds64f(qs_u32 + (nt * 8 + 2 * t) * 4);
+          q0 = qq.x; q1 = qq.y;
+        } else {
+          q0 = qs[nt][0]; q1 = qs[nt][1];
+        }
+        s[nt][0] = fmaf(al_lo, s[nt][0], fmaf(be_lo, q0, -m[nt][0]));
+        s[nt][1] = fmaf(al_lo, s[nt][1], fmaf(be_lo, q1, -m[nt][1]));
+        s[nt][2] = fmaf(al_hi, s[nt][2], fmaf(be_hi, q0, -m[nt][0]));
+        s[nt][3] = fmaf(al_hi, s[nt][3], fmaf(be_hi, q1, -m[nt][1]));
         if (masked) {
-          if (tok_lo >= lim[nt][0]) s[nt][0] = -INFINITY;
-          if (tok_lo >= lim[nt][1]) s[nt][1] = -INFINITY;
-          if (tok_hi >= lim[nt][0]) s[nt][2] = -INFINITY;
-          if (tok_hi >= lim[nt][1]) s[nt][3] = -INFINITY;
+          const int l0 = QFS ? col_limit(nt * 8 + 2 * t, len) : lim[QFS ? 0 : nt][0];
+          const int l1 = QFS ? col_limit(nt * 8 + 2 * t + 1, len) : lim[QFS ? 0 : nt][1];
+          if (tok_lo >= l0) s[nt][0] = -INFINITY;
+          if (tok_lo >= l1) s[nt][1] = -INFINITY;
+          if (tok_hi >= l0) s[nt][2] = -INFINITY;
+          if (tok_hi >= l1) s[nt][3] = -INFINITY;
         }
         gw |= fmaxf(fmaxf(s[nt][0], s[nt][2]), fmaxf(s[nt][1], s[nt][3])) > 4.0f;
       }
@@ -1365,55 +1450,57 @@ attn_team_kernel(const AttnParams p) {
     }
     // teams 1.. are absorbed into team 0, slice by slice, through lane-private mailboxes
     for (int src = 1; src < TEAMS; ++src) {
-      float* box = mail + (size_t)d * C::kMailRegs * 32 + lane;
-      if (team == src) {
-        int r = 0;
+      for (int dd = 0; dd < DS; ++dd) {
+        float* box = mail + lane;
+        if (team == src && d == dd) {
+          int r = 0;
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
+          for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
-          for (int mt = 0; mt < MT; ++mt)
+            for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) box[(r++) * 32] = o[nt][mt][i];
+              for (int i = 0; i < 4; ++i) box[(r++) * 32] = o[nt][mt][i];
 #pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            box[(r++) * 32] = m[nt][cc];
-            box[(r++) * 32] = l[nt][cc];
-            box[(r++) * 32] = zs[nt][cc];
+            for (int cc = 0; cc < 2; ++cc) {
+              box[(r++) * 32] = m[nt][cc];
+              box[(r++) * 32] = l[nt][cc];
+              box[(r++) * 32] = zs[nt][cc];
+            }
           }
         }
-      }
-      named_bar(1, C::kConsThreads);
-      if (team == 0) {
-        int r = 0;
+        named_bar(1, C::kConsThreads);
+        if (team == 0 && d == dd) {
+          int r = 0;
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          float f1[2], f2[2];
+          for (int nt = 0; nt < NT; ++nt) {
+            float f1[2], f2[2];
 #pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            const float m2 = box[((MT * 4 + 6) * nt + MT * 4 + 3 * cc) * 32];
-            const float M = fmaxf(m[nt][cc], m2);
-            f1[cc] = ex2(m[nt][cc] - M);
-            f2[cc] = ex2(m2 - M);
-            m[nt][cc] = M;
-          }
-#pragma unroll
-          for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const float o2 = box[(r++) * 32];
-              o[nt][mt][i] = o[nt][mt][i] * f1[i & 1] + o2 * f2[i & 1];
+            for (int cc = 0; cc < 2; ++cc) {
+              const float m2 = box[((MT * 4 + 6) * nt + MT * 4 + 3 * cc) * 32];
+              const float M = fmaxf(m[nt][cc], m2);
+              f1[cc] = ex2(m[nt][cc] - M);
+              f2[cc] = ex2(m2 - M);
+              m[nt][cc] = M;
             }
 #pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            r++;
-            const float l2 = box[(r++) * 32];
-            const float z2 = box[(r++) * 32];
-            l[nt][cc] = l[nt][cc] * f1[cc] + l2 * f2[cc];
-            zs[nt][cc] = zs[nt][cc] * f1[cc] + z2 * f2[cc];
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float o2 = box[(r++) * 32];
+                o[nt][mt][i] = o[nt][mt][i] * f1[i & 1] + o2 * f2[i & 1];
+              }
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc) {
+              r++;
+              const float l2 = box[(r++) * 32];
+              const float z2 = box[(r++) * 32];
+              l[nt][cc] = l[nt][cc] * f1[cc] + l2 * f2[cc];
+              zs[nt][cc] = zs[nt][cc] * f1[cc] + z2 * f2[cc];
+            }
           }
         }
+        named_bar(1, C::kConsThreads);
       }
-      named_bar(1, C::kConsThreads);
     }
     // team 0: totals of l and zs over its DS warps (each saw different tokens)
     if (team == 0) {
@@ -1593,15 +1680,15 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
     switch (pl.variant) {
       case 0: return launch<false, 1, 4, 1, 4, 4>(p, st);
       case 1: return launch_team<false, 2, 2, 2, 4, 3>(p, st);
-      case 2: return launch<false, 2, 4, 2, 6, 1>(p, st);
-      default: return launch<false, 2, 2, 4, 12, 1>(p, st);
+      case 2: return launch_team<false, 4, 4, 2, 3, 1>(p, st);
+      default: return launch_team<false, 8, 4, 2, 3, 1>(p, st);
     }
   }
   switch (pl.variant) {
     case 0: return launch<true, 1, 4, 1, 3, 3>(p, st);
     case 1: return launch_team<true, 2, 2, 2, 3, 3>(p, st);
-    case 2: return launch<true, 2, 4, 2, 5, 1>(p, st);
-    default: return launch<true, 2, 2, 4, 8, 1>(p, st);
+    case 2: return launch_team<true, 4, 4, 2, 3, 1>(p, st);
+    default: return launch_team<true, 8, 4, 2, 3, 1>(p, st);
   }
 }
 
