@@ -14,21 +14,25 @@
 // state, code-128 for the full state) so that no large bias enters the FP32 accumulation.
 //
 // Kernel shape.  Persistent grid (a few CTAs per SM), flash-decoding split-K in stream-K form:
-// the (sequence, KV head, 64-token unit) list is cut into equal contiguous ranges, one per CTA.
-// A CTA has TW*CG consumer warps and one producer warp.  The producer streams 16-token
+// the (sequence, KV head, stage-unit) list is cut into equal contiguous ranges, one per CTA.
+// A CTA has DS*TEAMS consumer warps and one producer warp.  The producer streams 16-token
 // sub-blocks (1 KiB per plane + 128 B of meta, each contiguous in the paged layout) into a
-// shared-memory ring with cp.async.bulk (TMA, 1-D) completing on mbarriers.  Consumer warp
-// (tw, cg) takes 16-token tile tw of every stage for columns [cg*NT*8, (cg+1)*NT*8):
+// shared-memory ring with cp.async.bulk (TMA, 1-D) completing on mbarriers, and the queries of
+// each piece into one of two slots.  A team of DS consumer warps takes DS 16-token tiles of
+// every stage; warp d of the team does, for ALL columns,
 //   S^T[16 tok x 8 col] = level(K)[16 x 128] . Q^T        mma.m16n8k32 u8 x s8, tokens are M
-//   online softmax with a lazily updated maximum (one warp vote per tile, no shuffles)
-//   P^T -> B operand by movmatrix (8x8 b16 transpose)
-//   O^T[128 dim x 8 col] += level(V)^T[128 x 16 tok] . P^T  mma.m16n8k16 f16, dims are M
+//   online softmax with a lazily updated maximum shared by the team
+//   P^T -> B operand by movmatrix (8x8 b16 transpose), published in shared memory (DS > 1)
+// for tile d, and then, for every tile of the team,
+//   O^T[slice x 8 col] += level(V)^T[slice x 16 tok] . P^T  mma.m16n8k16 f16, dims are M
+// for its own slice of 128/DS output dims: the nibbles of a tile are dequantised once however
+// many columns there are, and the accumulators shrink with DS.
 // K operands are the nibbles / merged codes themselves (one or two logic ops per 4 levels);
 // V operands are built from the nibbles with LOP3/PRMT and one FP16 add/fma per pair.
-// Partials (m, l, O) are merged across the CTA's token warps register-wise through shared
-// memory; a range that covers a whole (sequence, KV head) writes the output directly, otherwise
-// the partial goes to the workspace and the last contributor (atomic ticket, no waiting) merges
-// them; for verification the last CTA of a sequence also takes the accept/reject decision.
+// A range that covers a whole (sequence, KV head) writes the output directly, otherwise the
+// partial (m, l, O) goes to the workspace and the last contributor (atomic ticket, no waiting)
+// merges them; for verification the last CTA of a sequence also takes the accept/reject
+// decision.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -75,14 +79,17 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                : "memory");
 }
+// One probe of the barrier.  The hint lets the hardware park the thread (up to ~20 us here)
+// until the phase completes instead of returning at once, so a waiting warp does not burn
+// issue slots on polling; completion wakes it early.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(20000u)
       : "memory");
   return ok != 0;
 }
@@ -267,193 +274,7 @@ __device__ __forceinline__ void qk_int8(const uint32_t (&qf)[NT][2][4][2], uint3
 
 }
 
-template <bool FULL, int NT>
-struct WarpState {
-  uint32_t qf[NT][2][4][2];  // Q^T B-fragments (s8): [n-tile][digit plane hi/lo][k32 step][reg]
-  float qs[NT][2];        // sum_d q_d of the thread's two columns
-  float m[NT][2];         // running (lazy) maximum, log2 units
-  float l[NT][2];         // partial softmax denominators (this thread's rows only)
-  float zs[NT][2];        // partial sum p * (zero + mid*scale) of V
-  float o[NT][8][4];      // O^T accumulators: [n-tile][m-tile (16 dims)][c-reg]
-  int lim[NT][2];         // exclusive token limit of the thread's two columns
-  bool fresh;             // no tile processed yet: the first one sets the maximum outright
-};
-
-// One 16-token tile.  st = shared address of the stage, tw = tile index within the stage,
-// tile_t0 = absolute index of the tile's first token, masked = some (token, column) of this
-// tile is not visible.
-template <bool FULL, int NT, int ST>
-__device__ __forceinline__ void process_tile(WarpState<FULL, NT>& w, uint32_t st, int tw, int tile_t0,
-                                             bool masked, float ca, float cb, int g, int t, uint32_t magic) {
-  constexpr uint32_t KA = 0, VA = ST * 64, KR = ST * 128, VR = ST * 192;
-  constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
-  constexpr float kMidK = FULL ? 0.0f : 8.0f;      // K levels are the unsigned codes / nibbles
-  constexpr float kMidV = FULL ? 128.0f : 136.0f;  // V levels are centred (code-128, 16(a-8))
-  constexpr float kLevelScaleV = FULL ? 1.0f : 16.0f;
-  const int r0 = tw * 16 + pi_row(g);  // stage row of S row g; S row g+8 is r0 + 8
-
-  float s[NT][4];
-  qk_int8<FULL, NT, ST>(w.qf, st, r0, t, s);
-
-  // ---- per-token scalars, scores in log2 units -----------------------------------------
-  float2 km_lo = lds64f(st + KM + r0 * 8), km_hi = lds64f(st + KM + (r0 + 8) * 8);
-  float2 vm_lo = lds64f(st + VM + r0 * 8), vm_hi = lds64f(st + VM + (r0 + 8) * 8);
-  const int tok_lo = tile_t0 + pi_row(g), tok_hi = tok_lo + 8;
-  if (masked) {
-    // rows beyond every column's limit may hold arbitrary bits: neutralise their scalars
-    int maxlim = 0;
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) maxlim = max(maxlim, max(w.lim[nt][0], w.lim[nt][1]));
-    maxlim = max(maxlim, __shfl_xor_sync(0xFFFFFFFFu, maxlim, 1));
-    maxlim = max(maxlim, __shfl_xor_sync(0xFFFFFFFFu, maxlim, 2));
-    if (tok_lo >= maxlim) { km_lo = make_float2(0.f, 0.f); vm_lo = make_float2(0.f, 0.f); }
-    if (tok_hi >= maxlim) { km_hi = make_float2(0.f, 0.f); vm_hi = make_float2(0.f, 0.f); }
-  }
-  const float al_lo = km_lo.x * ca, al_hi = km_hi.x * ca;
-  const float be_lo = fmaf(km_lo.x, kMidK, km_lo.y) * cb, be_hi = fmaf(km_hi.x, kMidK, km_hi.y) * cb;
-  // s holds score - m (log2 units) from here on
-  bool grow = false;
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    s[nt][0] = fmaf(al_lo, s[nt][0], fmaf(be_lo, w.qs[nt][0], -w.m[nt][0]));
-    s[nt][1] = fmaf(al_lo, s[nt][1], fmaf(be_lo, w.qs[nt][1], -w.m[nt][1]));
-    s[nt][2] = fmaf(al_hi, s[nt][2], fmaf(be_hi, w.qs[nt][0], -w.m[nt][0]));
-    s[nt][3] = fmaf(al_hi, s[nt][3], fmaf(be_hi, w.qs[nt][1], -w.m[nt][1]));
-    if (masked) {
-      if (tok_lo >= w.lim[nt][0]) s[nt][0] = -INFINITY;
-      if (tok_lo >= w.lim[nt][1]) s[nt][1] = -INFINITY;
-      if (tok_hi >= w.lim[nt][0]) s[nt][2] = -INFINITY;
-      if (tok_hi >= w.lim[nt][1]) s[nt][3] = -INFINITY;
-    }
-    grow |= fmaxf(fmaxf(s[nt][0], s[nt][2]), fmaxf(s[nt][1], s[nt][3])) > 4.0f;
-  }
-  grow |= w.fresh;
-  // ---- lazy maximum: raise it only when some score exceeds it by more than 4 (p <= 16) --
-  if (__any_sync(0xFFFFFFFFu, grow)) {
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        float mx = fmaxf(s[nt][c], s[nt][c + 2]);
-        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 4));
-        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 8));
-        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));
-        // how far the maximum moves: up only, except for the first tile, which sets it outright
-        // (a column that sees none of the first tile's tokens sees none of the later ones either)
-        const float up = w.fresh ? fmaxf(mx, -1.0e4f) : fmaxf(mx, 0.0f);
-        const float f = w.fresh ? 0.0f : ex2(-up);  // nothing accumulated yet when fresh
-        w.m[nt][c] += up;
-        s[nt][c] -= up;
-        s[nt][c + 2] -= up;
-        w.l[nt][c] *= f;
-        w.zs[nt][c] *= f;
-#pragma unroll
-        for (int mt = 0; mt < 8; ++mt) {
-          w.o[nt][mt][c] *= f;
-          w.o[nt][mt][c + 2] *= f;
-        }
-      }
-    }
-  }
-  // ---- p, denominators, zero-point sums, P^T fragments ---------------------------------
-  const float sv_lo = vm_lo.x * kLevelScaleV, sv_hi = vm_hi.x * kLevelScaleV;
-  const float zv_lo = fmaf(vm_lo.x, kMidV, vm_lo.y), zv_hi = fmaf(vm_hi.x, kMidV, vm_hi.y);
-  uint32_t pb[NT][2];
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    const float p0 = ex2(s[nt][0]), p1 = ex2(s[nt][1]);
-    const float p2 = ex2(s[nt][2]), p3 = ex2(s[nt][3]);
-    w.l[nt][0] += p0 + p2;
-    w.l[nt][1] += p1 + p3;
-    w.zs[nt][0] = fmaf(p0, zv_lo, fmaf(p2, zv_hi, w.zs[nt][0]));
-    w.zs[nt][1] = fmaf(p1, zv_lo, fmaf(p3, zv_hi, w.zs[nt][1]));
-    pb[nt][0] = movmatrix_trans(pack_f16x2(p0 * sv_lo, p1 * sv_lo));  // tokens (2t,2t+1) of rows 0..7
-    pb[nt][1] = movmatrix_trans(pack_f16x2(p2 * sv_hi, p3 * sv_hi));  // tokens of rows 8..15
-  }
-  w.fresh = false;
-
-  // ---- O^T += level(V)^T . P^T ---------------------------------------------------------
-  // this thread feeds tokens pi(2t), pi(2t+1) (+8) and dims 16g .. 16g+15
-  const int ta = tw * 16 + pi_row(2 * t), tb = tw * 16 + pi_row(2 * t + 1);
-  const uint2 va = lds64(st + VA + ta * 64 + g * 8), vb = lds64(st + VA + tb * 64 + g * 8);
-  const uint2 vc = lds64(st + VA + (ta + 8) * 64 + g * 8), vd = lds64(st + VA + (tb + 8) * 64 + g * 8);
-  const uint32_t A[2] = {va.x, va.y}, Bw[2] = {vb.x, vb.y}, C[2] = {vc.x, vc.y}, Dw[2] = {vd.x, vd.y};
-  if (!FULL) {
-#pragma unroll
-    for (int wd = 0; wd < 2; ++wd) {
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const uint32_t sel = half ? 0x7632u : 0x5410u;
-        uint32_t ab[4], cd[4];
-        nib4_to_h2(prmt(A[wd], Bw[wd], sel), magic, ab);  // dims e(4half+0..3), token pair (a, b)
-        nib4_to_h2(prmt(C[wd], Dw[wd], sel), magic, cd);  // same dims, token pair (c, d)
-#pragma unroll
-        for (int qd = 0; qd < 2; ++qd) {
-          const int mt = wd * 4 + half * 2 + qd;
-#pragma unroll
-          for (int nt = 0; nt < NT; ++nt)
-            mma16816(w.o[nt][mt], ab[2 * qd], ab[2 * qd + 1], cd[2 * qd], cd[2 * qd + 1], pb[nt][0], pb[nt][1]);
-        }
-      }
-    }
-  } else {
-    const uint2 ra = lds64(st + VR + ta * 64 + g * 8), rb = lds64(st + VR + tb * 64 + g * 8);
-    const uint2 rc = lds64(st + VR + (ta + 8) * 64 + g * 8), rd = lds64(st + VR + (tb + 8) * 64 + g * 8);
-    const uint32_t RA[2] = {ra.x, ra.y}, RB[2] = {rb.x, rb.y}, RC[2] = {rc.x, rc.y}, RD[2] = {rd.x, rd.y};
-#pragma unroll
-    for (int wd = 0; wd < 2; ++wd) {
-      uint32_t ea, oa, eb, ob, ec, oc, ed, od;
-      merge_codes(A[wd], RA[wd], ea, oa);
-      merge_codes(Bw[wd], RB[wd], eb, ob);
-      merge_codes(C[wd], RC[wd], ec, oc);
-      merge_codes(Dw[wd], RD[wd], ed, od);
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const uint32_t sel = half ? 0x7632u : 0x5410u;
-        // bytes: [x.e(4half), x.e(4half+2), y.e(4half), y.e(4half+2)] for ev; odd elements for od
-        const uint32_t uab = prmt(ea, eb, sel), vab = prmt(oa, ob, sel);
-        const uint32_t ucd = prmt(ec, ed, sel), vcd = prmt(oc, od, sel);
-        // m-tile qd=0: dims e(4half+0) [row g] and e(4half+1) [row g+8]; qd=1: e(4half+2), e(4half+3)
-        const uint32_t ab0 = hadd2(and_or<0x00FF00FFu>(uab, magic), kNeg1152);
-        const uint32_t ab1 = hadd2(and_or<0x00FF00FFu>(vab, magic), kNeg1152);
-        const uint32_t ab2 = hadd2(prmt(uab, magic, 0x7351), kNeg1152);
-        const uint32_t ab3 = hadd2(prmt(vab, magic, 0x7351), kNeg1152);
-        const uint32_t cd0 = hadd2(and_or<0x00FF00FFu>(ucd, magic), kNeg1152);
-        const uint32_t cd1 = hadd2(and_or<0x00FF00FFu>(vcd, magic), kNeg1152);
-        const uint32_t cd2 = hadd2(prmt(ucd, magic, 0x7351), kNeg1152);
-        const uint32_t cd3 = hadd2(prmt(vcd, magic, 0x7351), kNeg1152);
-        const int mt = wd * 4 + half * 2;
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          mma16816(w.o[nt][mt], ab0, ab1, cd0, cd1, pb[nt][0], pb[nt][1]);
-          mma16816(w.o[nt][mt + 1], ab2, ab3, cd2, cd3, pb[nt][0], pb[nt][1]);
-        }
-      }
-    }
-  }
-}
-
 constexpr int kPieceUnits = 64;  // stage-units whose block ids are looked up at a time
-
-template <bool FULL, int NT, int TW, int CG, int NSTAGE>
-struct Cfg {
-  static constexpr int kST = TW * 16;                       // tokens per stage-unit
-  static constexpr int kSubBytes = FULL ? 16 * 272 : 16 * 144;
-  static constexpr int kStageBytes = kST * (FULL ? 272 : 144);
-  static constexpr int kConsWarps = TW * CG;
-  static constexpr int kConsThreads = kConsWarps * 32;
-  static constexpr int kThreads = (kConsWarps + 1) * 32;
-  static constexpr int kColsPad = CG * NT * 8;
-  static constexpr int kRing = NSTAGE * kStageBytes;
-  static constexpr int kMailRegs = 38 * NT;                 // o[NT][8][4] + m, l, zs [NT][2]
-  static constexpr int kMailBytes = CG * kMailRegs * 32 * 4;  // one mailbox per column group
-  static constexpr int kQBytes = 2 * kColsPad * LYNX_D * 2; // two item slots
-  static constexpr int kBlkBytes = kPieceUnits * TW * 4;
-  static constexpr int kInfoBytes = NSTAGE * 16 + 2 * 32;   // int4 per stage + two item records
-  static constexpr int kBarBytes = (2 * NSTAGE + 4) * 8;
-  static constexpr int kMiscBytes = 256;
-  static constexpr int kSmem = kRing + kMailBytes + kQBytes + kBlkBytes + kInfoBytes + kBarBytes + kMiscBytes;
-};
 
 struct Item {  // one piece: a run of stage-units of one (sequence, KV head) given to one CTA
   int b, hkv, len, first_cta, n_contrib, pad0, pad1, pad2;
@@ -715,287 +536,14 @@ __device__ __forceinline__ void producer_warp(const AttnParams& p, int lane, uin
   }
 }
 
-// Persistent, stream-K style kernel.  The work is the list of stage-units (ST tokens of one
-// (sequence, KV head)) in (sequence, head, position) order; CTA i owns the contiguous range
-// [i*q, (i+1)*q) of it, q = ceil(total / gridDim.x).  A range is cut into pieces at segment
-// boundaries; each piece is one online-softmax pass whose result goes to the output directly
-// (the segment lies inside the range) or to a partial slot that the last contributor merges.
-template <bool FULL, int NT, int TW, int CG, int NSTAGE, int MINB>
-__global__ void __launch_bounds__((TW * CG + 1) * 32, MINB)
-attn_kernel(const AttnParams p) {
-  using C = Cfg<FULL, NT, TW, CG, NSTAGE>;
-  constexpr int ST = C::kST;
-  extern __shared__ __align__(128) unsigned char smem[];
-  unsigned char* ring = smem;
-  float* mail = reinterpret_cast<float*>(smem + C::kRing);
-  __nv_bfloat16* q_s = reinterpret_cast<__nv_bfloat16*>(smem + C::kRing + C::kMailBytes);
-  uint32_t* blk_s = reinterpret_cast<uint32_t*>(smem + C::kRing + C::kMailBytes + C::kQBytes);
-  int4* info_s = reinterpret_cast<int4*>(smem + C::kRing + C::kMailBytes + C::kQBytes + C::kBlkBytes);
-  Item* items = reinterpret_cast<Item*>(info_s + NSTAGE);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kRing + C::kMailBytes + C::kQBytes +
-                                               C::kBlkBytes + C::kInfoBytes);
-  int* misc = reinterpret_cast<int*>(smem + C::kRing + C::kMailBytes + C::kQBytes + C::kBlkBytes +
-                                     C::kInfoBytes + C::kBarBytes);
-  // misc[0] abort word, [1] "last contributor" flag, [2..3] total units (int64), [4] units per
-  // CTA, [5] first sequence of this CTA's range, [6] unit offset inside that sequence,
-  // [7] number of units of this CTA, [16..31] per-position deviations
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n_cta = gridDim.x, cta = blockIdx.x;
-  const int cap = p.max_blocks * p.bt;
-  const uint32_t ring_u32 = smem_u32(ring);
-  const uint32_t full0 = smem_u32(bars), empty0 = full0 + NSTAGE * 8;
-  const uint32_t qfull0 = empty0 + NSTAGE * 8, qempty0 = qfull0 + 16;
-  volatile int* abort_word = misc;
-
-  if (tid == 0) {
-    for (int i = 0; i < NSTAGE; ++i) {
-      mbar_init(full0 + i * 8, 1);
-      mbar_init(empty0 + i * 8, C::kConsWarps);
-    }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(qfull0 + i * 8, 1);
-      mbar_init(qempty0 + i * 8, C::kConsWarps);
-    }
-    misc[0] = 0; misc[1] = 0; misc[7] = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  // padded query columns must read as zero: clear both item slots once
-  for (int i = tid; i < C::kQBytes / 16; i += C::kThreads) reinterpret_cast<uint4*>(q_s)[i] = make_uint4(0, 0, 0, 0);
-  // make the generic-proxy zeros visible to later async-proxy (TMA) writes of the same bytes
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  __syncthreads();
-
-  if (warp == C::kConsWarps) {
-    producer_warp<C, FULL, TW, NSTAGE>(p, lane, ring_u32, full0, empty0, qfull0, qempty0, q_s, blk_s,
-                                       info_s, items, misc, abort_word);
-    return;
-  }
-
-  // =============================== consumer warps ==============================
-  __syncthreads();  // (A)
-  const int n_units = misc[7];
-  if (n_units == 0) return;
-  const long long q_units = misc[4];
-  (void)q_units;
-  WarpState<FULL, NT> w;
-  const int g = lane >> 2, t = lane & 3;
-  const int tw = warp % TW, cg = warp / TW;
-  const float cb = p.sm_log2;
-  const uint32_t magic = opaque_magic();
-  float ca = 0.0f;
-  int len = 0, full_lim = 0, ic = 0;
-  Item item;
-  item.b = 0; item.hkv = 0; item.len = 0; item.first_cta = 0; item.n_contrib = 1;
-
-  for (int gs = 0; gs < n_units; ++gs) {
-    const int slot = gs % NSTAGE;
-    mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
-    const int4 info = info_s[slot];
-    if (info.z & 1) {
-      // ---- a new piece: queries, digit planes, fresh softmax state -----------------------
-      const int qi = info.x & 1;
-      mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
-      item = items[qi];
-      len = item.len;
-      full_lim = p.causal ? len - p.nq + 1 : len;
-      const __nv_bfloat16* qb = q_s + (size_t)qi * C::kColsPad * LYNX_D;
-      float amax = 0.0f;
-      for (int i = lane; i < C::kColsPad * (LYNX_D / 8); i += 32) {
-        const uint4 v = reinterpret_cast<const uint4*>(qb)[i];
-        const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          amax = fmaxf(amax, fabsf(__uint_as_float(ww[k] << 16)));
-          amax = fmaxf(amax, fabsf(__uint_as_float(ww[k] & 0xFFFF0000u)));
-        }
-      }
-#pragma unroll
-      for (int off = 16; off >= 1; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, off));
-      // Two s8 digit planes of q: q_int = rint(q * 2^e) with max|q| * 2^e in [2^13, 2^14), so
-      // q_int = 128 * hi + lo with hi in [-128, 127], lo in [0, 127].  BF16 values within 2^-6
-      // of the largest are exact; smaller ones are rounded to max|q| * 2^-14 absolute.
-      int e = 0;
-      if (amax > 0.0f && amax < INFINITY) e = 13 - (((__float_as_int(amax) >> 23) & 0xFF) - 127);
-      e = max(-100, min(100, e));
-      const float up = __int_as_float((127 + e) << 23), down = __int_as_float((127 - e) << 23);
-      ca = p.sm_log2 * down * (FULL ? 1.0f : 16.0f);  // per level unit of the K dot product
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        const int c = (cg * NT + nt) * 8 + g;  // column of this thread's B-fragment rows
-#pragma unroll
-        for (int wd = 0; wd < 4; ++wd) {
-          const uint4 v = *reinterpret_cast<const uint4*>(qb + c * LYNX_D + 32 * t + 8 * wd);
-          const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
-          int qv[8];
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            qv[2 * k] = __float2int_rn(__uint_as_float(ww[k] << 16) * up);
-            qv[2 * k + 1] = __float2int_rn(__uint_as_float(ww[k] & 0xFFFF0000u) * up);
-          }
-          uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;  // bytes for dims {0,2,4,6} / {1,3,5,7}
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            hi_e |= (uint32_t)((qv[2 * k] >> 7) & 0xFF) << (8 * k);
-            lo_e |= (uint32_t)(qv[2 * k] & 127) << (8 * k);
-            hi_o |= (uint32_t)((qv[2 * k + 1] >> 7) & 0xFF) << (8 * k);
-            lo_o |= (uint32_t)(qv[2 * k + 1] & 127) << (8 * k);
-          }
-          w.qf[nt][0][wd][0] = hi_e; w.qf[nt][0][wd][1] = hi_o;
-          w.qf[nt][1][wd][0] = lo_e; w.qf[nt][1][wd][1] = lo_o;
-        }
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          const int col = (cg * NT + nt) * 8 + 2 * t + cc;  // column of this thread's C-fragment
-          // sum over d of q_d: this lane adds dims [16g, 16g+16), the 8 lanes sharing t add up
-          const uint4* qq = reinterpret_cast<const uint4*>(qb + col * LYNX_D + 16 * g);
-          float sum = 0.0f;
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const uint4 v = qq[h];
-            const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              sum += __uint_as_float(ww[k] << 16) + __uint_as_float(ww[k] & 0xFFFF0000u);
-          }
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 4);
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 8);
-          sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 16);
-          w.qs[nt][cc] = sum;
-          const int j = col / p.G;
-          w.lim[nt][cc] = col < p.ncols ? (p.causal ? len - p.nq + j + 1 : len) : 0;
-          w.m[nt][cc] = 0.0f;
-          w.l[nt][cc] = 0.0f;
-          w.zs[nt][cc] = 0.0f;
-        }
-#pragma unroll
-        for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-          for (int i = 0; i < 4; ++i) w.o[nt][mt][i] = 0.0f;
-      }
-      w.fresh = true;
-    }
-    const int tile_t0 = info.y * ST + tw * 16;
-    if (tile_t0 < len)
-      process_tile<FULL, NT, ST>(w, ring_u32 + slot * C::kStageBytes, tw, tile_t0,
-                                 tile_t0 + 16 > full_lim, ca, cb, g, t, magic);
-    __syncwarp();
-    if (lane == 0) mbar_arrive(empty0 + slot * 8);
-    if (!(info.z & 2)) continue;
-    if (w.fresh) {  // this warp saw no token of the piece: it must not weigh in the merge
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) w.m[nt][0] = w.m[nt][1] = -1.0e30f;
-    }
-
-    // ---- end of the piece: warp 0 of the column group absorbs the other token warps one by
-    //      one (register-wise, through a lane-private mailbox), then writes the result --------
-    for (int src = 1; src < TW; ++src) {
-      float* box = mail + (size_t)cg * C::kMailRegs * 32 + lane;
-      if (tw == src) {
-        int r = 0;
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-          for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) box[(r++) * 32] = w.o[nt][mt][i];
-#pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            box[(r++) * 32] = w.m[nt][cc];
-            box[(r++) * 32] = w.l[nt][cc];
-            box[(r++) * 32] = w.zs[nt][cc];
-          }
-        }
-      }
-      named_bar(2 + cg, TW * 32);
-      if (tw == 0) {
-        int r = 0;
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          float f1[2], f2[2];
-#pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            const float m2 = box[(38 * nt + 32 + 3 * cc) * 32];
-            const float M = fmaxf(w.m[nt][cc], m2);
-            f1[cc] = ex2(w.m[nt][cc] - M);
-            f2[cc] = ex2(m2 - M);
-            w.m[nt][cc] = M;
-          }
-#pragma unroll
-          for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const float o2 = box[(r++) * 32];
-              w.o[nt][mt][i] = w.o[nt][mt][i] * f1[i & 1] + o2 * f2[i & 1];
-            }
-#pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            r++;  // m (already used)
-            const float l2 = box[(r++) * 32];
-            const float z2 = box[(r++) * 32];
-            w.l[nt][cc] = w.l[nt][cc] * f1[cc] + l2 * f2[cc];
-            w.zs[nt][cc] = w.zs[nt][cc] * f1[cc] + z2 * f2[cc];
-          }
-        }
-      }
-      named_bar(2 + cg, TW * 32);
-    }
-
-    const size_t bh = (size_t)item.b * p.Hkv + item.hkv;
-    const bool direct = item.n_contrib == 1;
-    if (tw == 0) {
-      float* part = p.ws_part + (bh + (size_t)cta) * (size_t)C::kColsPad * kPartStride;
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          float l = w.l[nt][cc], z = w.zs[nt][cc];
-#pragma unroll
-          for (int off = 4; off <= 16; off <<= 1) {
-            l += __shfl_xor_sync(0xFFFFFFFFu, l, off);
-            z += __shfl_xor_sync(0xFFFFFFFFu, z, off);
-          }
-          const int c = (cg * NT + nt) * 8 + 2 * t + cc;
-          if (c >= p.ncols) continue;
-          if (direct) {
-            const int j = c / p.G, hh = c % p.G;
-            float* dst = p.out + (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D;
-            const float inv = l > 0.0f ? 1.0f / l : 0.0f;
-#pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-              const int d = 16 * g + 8 * (mt >> 2) + 2 * (mt & 3);
-              *reinterpret_cast<float2*>(dst + d) =
-                  make_float2((w.o[nt][mt][cc] + z) * inv, (w.o[nt][mt][cc + 2] + z) * inv);
-            }
-          } else {
-            float* dst = part + (size_t)c * kPartStride;
-#pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-              const int d = 16 * g + 8 * (mt >> 2) + 2 * (mt & 3);
-              *reinterpret_cast<float2*>(dst + d) = make_float2(w.o[nt][mt][cc] + z, w.o[nt][mt][cc + 2] + z);
-            }
-            if (g == 0) { dst[128] = w.m[nt][cc]; dst[129] = l; }
-          }
-        }
-      }
-      __threadfence();
-    }
-    finish_piece<FULL, C::kColsPad, C::kConsThreads>(p, item, direct, tid, misc);
-    __syncwarp();
-    if (lane == 0) mbar_arrive(qempty0 + (info.x & 1) * 8);
-    ++ic;
-  }
-  if (tid == 0 && misc[0]) atomicOr(p.ws_flags, kFlagTimeout);
-}
-
 // =============================================================================================
-// Team variant for more than 8 columns.  DS consumer warps form a team that takes DS tiles of a
-// stage: warp d computes Q.K^T and the softmax weights of tile d for ALL columns and publishes
-// its P^T fragments in shared memory; every warp then accumulates P.V of all DS tiles for its
-// own slice of 128/DS output dims.  The K/V nibbles are dequantised once per tile (no column
-// groups repeating the work) and the accumulators shrink with DS.  The team keeps one running
-// maximum per column (two named barriers per step; growth is agreed through shared memory).
+// Shared-memory geometry of one kernel variant.  NT = 8-column tiles (all of them in every
+// warp), DS = warps per team = tiles per team and step = slices of the output dims,
+// TEAMS = teams per CTA, QFS = query fragments kept in shared memory instead of registers.
+// With DS > 1 a team keeps one running maximum per column: two named barriers per step, growth
+// agreed through shared memory.  With DS == 1 a warp is its own team and nothing is exchanged.
 // =============================================================================================
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, bool QFS>
 struct TeamCfg {
   static constexpr int kTW = DS * TEAMS;                    // consumer warps = tiles per stage
   static constexpr int kST = kTW * 16;
@@ -1009,9 +557,9 @@ struct TeamCfg {
   static constexpr int kRing = NSTAGE * kStageBytes;
   static constexpr int kMailRegs = NT * kMT * 4 + NT * 6;   // o slice + m, l, zs
   static constexpr int kMailBytes = TEAMS > 1 ? kMailRegs * 32 * 4 : 0;  // one box, used slice by slice
-  static constexpr int kXchgBytes = kTW * (16 + kColsPad * 4 + NT * 2 * 32 * 4);  // flag, colmax, P^T
-  static constexpr int kLzBytes = DS * kColsPad * 2 * 4;
-  static constexpr bool kQfShared = NT > 2;                 // query fragments in shared memory
+  static constexpr int kXchgBytes = DS > 1 ? kTW * (16 + kColsPad * 4 + NT * 2 * 32 * 4) : 0;  // flag, colmax, P^T
+  static constexpr int kLzBytes = DS * kColsPad * 2 * 4 + 16;
+  static constexpr bool kQfShared = QFS;                    // query fragments in shared memory
   static constexpr int kQfBytes = kQfShared ? NT * 2 * 4 * 32 * 8 + kColsPad * 4 : 0;
   static constexpr int kQBytes = 2 * kColsPad * LYNX_D * 2;
   static constexpr int kBlkBytes = kPieceUnits * kTW * 4;
@@ -1116,10 +664,9 @@ __device__ __forceinline__ void pv_slice(float (&o)[NT][8 / DS][4], uint32_t st,
   }
 }
 
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB>
-__global__ void __launch_bounds__((DS * TEAMS + 1) * 32, MINB)
-attn_team_kernel(const AttnParams p) {
-  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE>;
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, bool QFS>
+__device__ __forceinline__ void attn_team_body(const AttnParams& p) {
+  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE, QFS>;
   constexpr int ST = C::kST, TW = C::kTW, MT = C::kMT;
   constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
   constexpr float kMidK = FULL ? 0.0f : 8.0f;
@@ -1176,7 +723,6 @@ attn_team_kernel(const AttnParams p) {
   const int team = warp / DS, d = warp % DS;
   const float cb = p.sm_log2;
   const uint32_t magic = opaque_magic();
-  constexpr bool QFS = C::kQfShared;
   constexpr int NTR = QFS ? 1 : NT;  // register copies exist only when the fragments are not shared
   uint32_t qf[NTR][2][4][2];
   float qs[NTR][2], m[NT][2], l[NT][2], zs[NT][2], o[NT][MT][4];
@@ -1293,6 +839,7 @@ attn_team_kernel(const AttnParams p) {
     const bool team_valid = unit_t0 + team * DS * 16 < len;       // the team's first tile
     unsigned char* my_x = xchg + (size_t)warp * kXW;
     float s[NT][4];
+    float cmx[DS > 1 ? 1 : NT][2];  // column maxima of this tile (kept in registers when DS == 1)
     float2 vm_lo = make_float2(0.f, 0.f), vm_hi = make_float2(0.f, 0.f);
     const int r0 = warp * 16 + pi_row(g);
     const int tok_lo = tile_t0 + pi_row(g), tok_hi = tok_lo + 8;
@@ -1366,20 +913,29 @@ attn_team_kernel(const AttnParams p) {
             mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 4));
             mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 8));
             mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));
-            if (g == 0) reinterpret_cast<float*>(my_x + 16)[nt * 8 + 2 * t + cc] = mx;
+            if constexpr (DS > 1) {
+              if (g == 0) reinterpret_cast<float*>(my_x + 16)[nt * 8 + 2 * t + cc] = mx;
+            } else {
+              cmx[nt][cc] = mx;
+            }
           }
       }
     }
-    if (lane == 0) *reinterpret_cast<int*>(my_x) = gw ? 1 : 0;
-    named_bar(2 + team, DS * 32);
+    if constexpr (DS > 1) {
+      if (lane == 0) *reinterpret_cast<int*>(my_x) = gw ? 1 : 0;
+      named_bar(2 + team, DS * 32);
+    }
     // ---- agree on the running maxima ----------------------------------------------------
     {
-      bool any = false;
+      bool any = gw;
       int flags[DS];
+      if constexpr (DS > 1) {
+        any = false;
 #pragma unroll
-      for (int dd = 0; dd < DS; ++dd) {
-        flags[dd] = *reinterpret_cast<const volatile int*>(xchg + (size_t)(team * DS + dd) * kXW);
-        any |= flags[dd] != 0;
+        for (int dd = 0; dd < DS; ++dd) {
+          flags[dd] = *reinterpret_cast<const volatile int*>(xchg + (size_t)(team * DS + dd) * kXW);
+          any |= flags[dd] != 0;
+        }
       }
       if (any) {
 #pragma unroll
@@ -1387,10 +943,14 @@ attn_team_kernel(const AttnParams p) {
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
             float mx = -INFINITY;
+            if constexpr (DS > 1) {
 #pragma unroll
-            for (int dd = 0; dd < DS; ++dd)
-              if (flags[dd])
-                mx = fmaxf(mx, reinterpret_cast<const volatile float*>(xchg + (size_t)(team * DS + dd) * kXW + 16)[nt * 8 + 2 * t + cc]);
+              for (int dd = 0; dd < DS; ++dd)
+                if (flags[dd])
+                  mx = fmaxf(mx, reinterpret_cast<const volatile float*>(xchg + (size_t)(team * DS + dd) * kXW + 16)[nt * 8 + 2 * t + cc]);
+            } else {
+              mx = cmx[nt][cc];
+            }
             const float up = fresh ? fmaxf(mx, -1.0e4f) : fmaxf(mx, 0.0f);
             const float f = fresh ? 0.0f : ex2(-up);
             m[nt][cc] += up;
@@ -1408,6 +968,7 @@ attn_team_kernel(const AttnParams p) {
       if (team_valid) fresh = false;
     }
     // ---- weights of this warp's tile, P^T fragments to shared memory ---------------------
+    uint32_t pown[DS > 1 ? 1 : NT][2];  // P^T fragments of the own tile (DS == 1)
     if (valid) {
       const float sv_lo = vm_lo.x * kLevelScaleV, sv_hi = vm_hi.x * kLevelScaleV;
       const float zv_lo = fmaf(vm_lo.x, kMidV, vm_lo.y), zv_hi = fmaf(vm_hi.x, kMidV, vm_hi.y);
@@ -1420,14 +981,24 @@ attn_team_kernel(const AttnParams p) {
         l[nt][1] += p1 + p3;
         zs[nt][0] = fmaf(p0, zv_lo, fmaf(p2, zv_hi, zs[nt][0]));
         zs[nt][1] = fmaf(p1, zv_lo, fmaf(p3, zv_hi, zs[nt][1]));
-        pf[(nt * 2 + 0) * 32] = movmatrix_trans(pack_f16x2(p0 * sv_lo, p1 * sv_lo));
-        pf[(nt * 2 + 1) * 32] = movmatrix_trans(pack_f16x2(p2 * sv_hi, p3 * sv_hi));
+        const uint32_t f0 = movmatrix_trans(pack_f16x2(p0 * sv_lo, p1 * sv_lo));
+        const uint32_t f1 = movmatrix_trans(pack_f16x2(p2 * sv_hi, p3 * sv_hi));
+        if constexpr (DS > 1) {
+          pf[(nt * 2 + 0) * 32] = f0;
+          pf[(nt * 2 + 1) * 32] = f1;
+        } else {
+          pown[nt][0] = f0;
+          pown[nt][1] = f1;
+        }
       }
     }
-    named_bar(2 + team, DS * 32);
+    if constexpr (DS > 1) named_bar(2 + team, DS * 32);
     // ---- phase C: P.V of the team's tiles for this warp's slice of the output dims --------
+    if constexpr (DS == 1) {
+      if (valid) pv_slice<FULL, NT, ST, 1>(o, st, warp * 16, g, t, 0, pown, magic);
+    }
 #pragma unroll
-    for (int tau = 0; tau < DS; ++tau) {
+    for (int tau = 0; tau < (DS > 1 ? DS : 0); ++tau) {
       const int src = team * DS + tau;
       if (unit_t0 + src * 16 >= len) break;  // uniform: later tiles of the unit are beyond len too
       uint32_t pb[NT][2];
@@ -1561,6 +1132,13 @@ attn_team_kernel(const AttnParams p) {
   if (tid == 0 && misc[0]) atomicOr(p.ws_flags, kFlagTimeout);
 }
 
+// At least MINB CTAs per SM (the compiler caps registers accordingly).  Nine warps cannot
+// have more than 168 registers each: three of them share one SM sub-partition's 16 K registers.
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB, bool QFS>
+__global__ void __launch_bounds__((DS * TEAMS + 1) * 32, MINB)
+attn_team_kernel(const AttnParams p) {
+  attn_team_body<FULL, NT, DS, TEAMS, NSTAGE, QFS>(p);
+}
 // ------------------------------------------------------------------ host side
 constexpr int kMaxCtasPerSm = 4;
 
@@ -1596,31 +1174,14 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   return true;
 }
 
-template <bool FULL, int NT, int TW, int CG, int NSTAGE, int MINB>
-lynx_status launch(const AttnParams& p, cudaStream_t st) {
-  using C = Cfg<FULL, NT, TW, CG, NSTAGE>;
-  static_assert(MINB <= kMaxCtasPerSm, "partial slots are sized for kMaxCtasPerSm CTAs per SM");
-  static_assert(MINB * (C::kSmem + 1024) <= 228 * 1024, "shared memory budget for MINB CTAs per SM");
-  auto kern = attn_kernel<FULL, NT, TW, CG, NSTAGE, MINB>;
-  static bool configured[64] = {false};
-  int dev = 0;
-  cudaGetDevice(&dev);
-  if (dev >= 0 && dev < 64 && !configured[dev]) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmem) != cudaSuccess)
-      return LYNX_ERR_CUDA;
-    configured[dev] = true;
-  }
-  kern<<<sm_count() * MINB, C::kThreads, C::kSmem, st>>>(p);
-  return launch_status();
-}
-
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB, bool QFS>
 lynx_status launch_team(const AttnParams& p, cudaStream_t st) {
-  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE>;
+  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE, QFS>;
   static_assert(MINB <= kMaxCtasPerSm, "partial slots are sized for kMaxCtasPerSm CTAs per SM");
-  static_assert(MINB * (C::kSmem + 1024) <= 228 * 1024, "shared memory budget for MINB CTAs per SM");
+  constexpr int kCtasPerSm = MINB;
+  static_assert(kCtasPerSm * (C::kSmem + 1024) <= 228 * 1024, "shared memory budget per SM");
   static_assert(2 + TEAMS <= 16, "named barriers");
-  auto kern = attn_team_kernel<FULL, NT, DS, TEAMS, NSTAGE, MINB>;
+  auto kern = attn_team_kernel<FULL, NT, DS, TEAMS, NSTAGE, MINB, QFS>;
   static bool configured[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -1629,7 +1190,13 @@ lynx_status launch_team(const AttnParams& p, cudaStream_t st) {
       return LYNX_ERR_CUDA;
     configured[dev] = true;
   }
-  kern<<<sm_count() * MINB, C::kThreads, C::kSmem, st>>>(p);
+  // small problems: no more CTAs than ranges of at least 8 stage-units (an upper bound from the
+  // table capacity: the lengths live on the device)
+  const long long cap_units = (long long)p.B * p.Hkv * (((long long)p.max_blocks * p.bt + C::kST - 1) / C::kST);
+  long long grid = (cap_units + 7) / 8;
+  const long long full = (long long)sm_count() * kCtasPerSm;
+  grid = grid < 1 ? 1 : (grid > full ? full : grid);
+  kern<<<(unsigned)grid, C::kThreads, C::kSmem, st>>>(p);
   return launch_status();
 }
 
@@ -1676,19 +1243,20 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   p.bt = shape->block_tokens; p.num_blocks = shape->num_blocks; p.max_blocks = shape->max_blocks_per_seq;
   p.ncols = pl.ncols;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // <FULL, NT, DS, TEAMS, stages, CTAs/SM, shared query fragments>
   if (!full) {
     switch (pl.variant) {
-      case 0: return launch<false, 1, 4, 1, 4, 4>(p, st);
-      case 1: return launch_team<false, 2, 2, 2, 4, 3>(p, st);
-      case 2: return launch_team<false, 4, 4, 2, 3, 1>(p, st);
-      default: return launch_team<false, 8, 4, 2, 3, 1>(p, st);
+      case 0: return launch_team<false, 1, 1, 4, 4, 4, true>(p, st);
+      case 1: return launch_team<false, 2, 2, 2, 4, 3, false>(p, st);
+      case 2: return launch_team<false, 4, 4, 1, 3, 3, true>(p, st);
+      default: return launch_team<false, 8, 4, 2, 3, 1, true>(p, st);
     }
   }
   switch (pl.variant) {
-    case 0: return launch<true, 1, 4, 1, 3, 3>(p, st);
-    case 1: return launch_team<true, 2, 2, 2, 3, 3>(p, st);
-    case 2: return launch_team<true, 4, 4, 2, 3, 1>(p, st);
-    default: return launch_team<true, 8, 4, 2, 3, 1>(p, st);
+    case 0: return launch_team<true, 1, 1, 4, 3, 3, true>(p, st);
+    case 1: return launch_team<true, 2, 2, 2, 3, 3, false>(p, st);
+    case 2: return launch_team<true, 4, 4, 1, 2, 3, true>(p, st);
+    default: return launch_team<true, 8, 4, 2, 3, 1, true>(p, st);
   }
 }
 

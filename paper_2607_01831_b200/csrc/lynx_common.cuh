@@ -2,6 +2,8 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
 
 #include "lynx.h"
 
@@ -11,8 +13,13 @@ namespace lynx {
 
 __host__ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Status of the launch just made.  With LYNX_DEBUG set in the environment the CUDA error text
+// goes to stderr.
 __host__ inline lynx_status launch_status() {
-  return cudaGetLastError() == cudaSuccess ? LYNX_OK : LYNX_ERR_CUDA;
+  const cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) return LYNX_OK;
+  if (getenv("LYNX_DEBUG")) fprintf(stderr, "lynx: CUDA error at launch: %s\n", cudaGetErrorString(e));
+  return LYNX_ERR_CUDA;
 }
 
 // Number of SMs of the current device (cached per device id).
