@@ -304,20 +304,43 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
       __threadfence();
       const float* base = p.ws_part + (bh + (size_t)item.first_cta) * (size_t)kColsPad * kPartStride;
       const size_t cstride = (size_t)kColsPad * kPartStride;
-      for (int idx = tid; idx < kColsPad * LYNX_D; idx += kConsThreads) {
-        const int c = idx >> 7, d = idx & 127;
-        if (c >= p.ncols) continue;
+      // a warp per column, a lane per 4 dims; the slots are merged online, four loads ahead
+      const int lane = tid & 31;
+      for (int c = tid >> 5; c < p.ncols; c += kConsThreads / 32) {
         const float* col = base + (size_t)c * kPartStride;
-        float M = -INFINITY;
-        for (int i = 0; i < item.n_contrib; ++i) M = fmaxf(M, __ldcg(col + i * cstride + 128));
-        float acc = 0.0f, L = 0.0f;
-        for (int i = 0; i < item.n_contrib; ++i) {
-          const float f = ex2(__ldcg(col + i * cstride + 128) - M);
-          acc = fmaf(__ldcg(col + i * cstride + d), f, acc);
-          L = fmaf(__ldcg(col + i * cstride + 129), f, L);
+        float M = -INFINITY, L = 0.0f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i0 = 0; i0 < item.n_contrib; i0 += 4) {
+          float mi[4], li[4];
+          float4 oi[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const bool in = i0 + u < item.n_contrib;
+            const float* src = col + (size_t)(in ? i0 + u : i0) * cstride;
+            mi[u] = in ? __ldcg(src + 128) : -INFINITY;
+            li[u] = __ldcg(src + 129);
+            oi[u] = __ldcg(reinterpret_cast<const float4*>(src) + lane);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float Mn = fmaxf(M, mi[u]);
+            // an absent slot (mi = -inf) keeps fa = 1, fb = 0 once M is finite; while M is still
+            // -inf both factors are forced to 0 / taken from the slot without forming inf - inf
+            const float fa = M == -INFINITY ? 0.0f : ex2(M - Mn);
+            const float fb = mi[u] == -INFINITY ? 0.0f : ex2(mi[u] - Mn);
+            acc.x = acc.x * fa + oi[u].x * fb;
+            acc.y = acc.y * fa + oi[u].y * fb;
+            acc.z = acc.z * fa + oi[u].z * fb;
+            acc.w = acc.w * fa + oi[u].w * fb;
+            L = L * fa + li[u] * fb;
+            M = Mn;
+          }
         }
+        const float inv = L > 0.0f ? 1.0f / L : 0.0f;
         const int j = c / p.G, hh = c % p.G;
-        p.out[(((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
+        float4* dst = reinterpret_cast<float4*>(
+            p.out + (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D);
+        dst[lane] = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
       }
     }
   }
@@ -610,18 +633,32 @@ __device__ __forceinline__ void pv_slice(float (&o)[NT][8 / DS][4], uint32_t st,
   const int ta = row0 + pi_row(2 * t), tb = row0 + pi_row(2 * t + 1);
   uint32_t A[NW], Bw[NW], C[NW], Dw[NW], RA[NW], RB[NW], RC[NW], RD[NW];
   const uint32_t wofs = DS == 1 ? 0u : (DS == 2 ? (uint32_t)d * 4u : (uint32_t)(d >> 1) * 4u);
-#pragma unroll
-  for (int i = 0; i < NW; ++i) {
-    const uint32_t off = g * 8 + wofs + i * 4;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(A[i]) : "r"(st + VA + ta * 64 + off));
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(Bw[i]) : "r"(st + VA + tb * 64 + off));
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(C[i]) : "r"(st + VA + (ta + 8) * 64 + off));
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(Dw[i]) : "r"(st + VA + (tb + 8) * 64 + off));
+  if constexpr (DS == 1) {  // both words of the lane's 8 bytes: one 64-bit load per token row
+    const uint32_t off = g * 8;
+    const uint2 va = lds64(st + VA + ta * 64 + off), vb = lds64(st + VA + tb * 64 + off);
+    const uint2 vc = lds64(st + VA + (ta + 8) * 64 + off), vd = lds64(st + VA + (tb + 8) * 64 + off);
+    A[0] = va.x; A[NW - 1] = va.y; Bw[0] = vb.x; Bw[NW - 1] = vb.y;
+    C[0] = vc.x; C[NW - 1] = vc.y; Dw[0] = vd.x; Dw[NW - 1] = vd.y;
     if (FULL) {
-      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RA[i]) : "r"(st + VR + ta * 64 + off));
-      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RB[i]) : "r"(st + VR + tb * 64 + off));
-      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RC[i]) : "r"(st + VR + (ta + 8) * 64 + off));
-      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RD[i]) : "r"(st + VR + (tb + 8) * 64 + off));
+      const uint2 ra = lds64(st + VR + ta * 64 + off), rb = lds64(st + VR + tb * 64 + off);
+      const uint2 rc = lds64(st + VR + (ta + 8) * 64 + off), rd = lds64(st + VR + (tb + 8) * 64 + off);
+      RA[0] = ra.x; RA[NW - 1] = ra.y; RB[0] = rb.x; RB[NW - 1] = rb.y;
+      RC[0] = rc.x; RC[NW - 1] = rc.y; RD[0] = rd.x; RD[NW - 1] = rd.y;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < NW; ++i) {
+      const uint32_t off = g * 8 + wofs + i * 4;
+      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(A[i]) : "r"(st + VA + ta * 64 + off));
+      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(Bw[i]) : "r"(st + VA + tb * 64 + off));
+      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(C[i]) : "r"(st + VA + (ta + 8) * 64 + off));
+      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(Dw[i]) : "r"(st + VA + (tb + 8) * 64 + off));
+      if (FULL) {
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RA[i]) : "r"(st + VR + ta * 64 + off));
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RB[i]) : "r"(st + VR + tb * 64 + off));
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RC[i]) : "r"(st + VR + (ta + 8) * 64 + off));
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(RD[i]) : "r"(st + VR + (tb + 8) * 64 + off));
+      }
     }
   }
 #pragma unroll
