@@ -441,6 +441,8 @@ def main():
         "kernels": kernels, "roofline": roof, "clocks": clocks,
     }
 
+    if rank == 0 and world == 1:
+        line["per_layer_launches"] = run_per_layer(wlk, peak)
     if rank == 0 and world == 1 and not args.no_e2e:
         line["e2e"] = run_e2e(wlk, args.e2e_steps, step_bytes)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -452,6 +454,55 @@ def main():
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(line))
+
+
+def run_per_layer(wlk: "Workload", peak: float):
+    """Context for the flattened numbers: one anchor decode step and one verify pass issued the
+    way a decoder has to, one launch per layer (batch = the workload's sequences), back to back
+    on one stream.  Not part of `value`."""
+    lynx, wl = wlk.lynx, wlk.wl
+    L, Bs = wl.layers, wl.batch
+    win = wlk.windows[0]
+    k = win["k"]
+    geo = wlk.geo
+    ws1 = lynx.make_workspace(geo, Bs, 1, wlk.device)
+    wsk = lynx.make_workspace(geo, Bs, k, wlk.device)
+    K, V = wlk.planes["K"], wlk.planes["V"]
+    views = []
+    for l in range(L):
+        sl = slice(l * Bs, (l + 1) * Bs)
+        views.append((win["qs"][k - 1][sl], win["q"][sl], wlk.table[sl], wlk.lens_flat[sl], win["step_out"][k - 1][sl],
+                      win["draft"][sl], win["out_full"][sl], win["first_reject"][sl], win["dev"][sl]))
+
+    def anchor_all():
+        for q1, qk, tb, ln, o1, dr, of, fr, dv in views:
+            lynx.anchor_attention(geo, q1, K, V, tb, ln, ws1, out=o1)
+
+    def verify_all():
+        for q1, qk, tb, ln, o1, dr, of, fr, dv in views:
+            lynx.merge_verify_attention(geo, qk, K, V, tb, ln, wsk, draft_out=dr, atol=0.5, rtol=0.1,
+                                        causal=True, out_full=of, first_reject=fr, dev=dv)
+
+    out = {}
+    for name, fn, bpr in (("anchor_attention", anchor_all, BYTES_PER_ROW["anchor_attention"]),
+                          (f"merge_verify_attention[k={k}]", verify_all, BYTES_PER_ROW["merge_verify_attention"])):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 5
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        gbs = wlk.rows_kv * bpr / (ms * 1e-3) / 1e9
+        out[name] = {"launches": L, "ms_all_layers": ms, "us_per_layer": ms * 1e3 / L, "GBps": gbs,
+                     "frac_of_measured": gbs / peak}
+    lynx.check(ws1)
+    lynx.check(wsk)
+    return out
 
 
 def run_e2e(wlk: "Workload", steps: int, step_bytes: int):
