@@ -185,6 +185,31 @@ __device__ __forceinline__ float2 lds64f(uint32_t addr) {
   return v;
 }
 
+// Packed FP32 pairs (Blackwell fma/add/mul .f32x2: two lanes per instruction).
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // FP16x2 constants
 constexpr uint32_t kMagic = 0x64006400u;      // 1024, 1024
 constexpr uint32_t kNeg1032 = 0xE408E408u;    // -1032
@@ -762,6 +787,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
   const uint32_t magic = opaque_magic();
   constexpr int NTR = QFS ? 1 : NT;  // register copies exist only when the fragments are not shared
   uint32_t qf[NTR][2][4][2];
+  // m holds MINUS the running maximum inside the stage loop (it enters the score FMA directly)
   float qs[NTR][2], m[NT][2], l[NT][2], zs[NT][2], o[NT][MT][4];
   int lim[NTR][2];
   const uint32_t qf_u32 = smem_u32(qf_s), qs_u32 = smem_u32(qs_s);
@@ -872,8 +898,10 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
     const uint32_t st = ring_u32 + slot * C::kStageBytes;
     const int unit_t0 = info.y * ST;
     const int tile_t0 = unit_t0 + warp * 16;
-    const bool valid = tile_t0 < len;                             // this warp's own tile
+    const bool in_range = tile_t0 < len;                          // this warp's own tile
     const bool team_valid = unit_t0 + team * DS * 16 < len;       // the team's first tile
+    if (DS > 1 || in_range) {  // a lone warp (DS == 1) has nothing to do for a tile beyond the end
+    const bool valid = DS == 1 ? true : in_range;
     unsigned char* my_x = xchg + (size_t)warp * kXW;
     float s[NT][4];
     float cmx[DS > 1 ? 1 : NT][2];  // column maxima of this tile (kept in registers when DS == 1)
@@ -926,10 +954,13 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
         } else {
           q0 = qs[nt][0]; q1 = qs[nt][1];
         }
-        s[nt][0] = fmaf(al_lo, s[nt][0], fmaf(be_lo, q0, -m[nt][0]));
-        s[nt][1] = fmaf(al_lo, s[nt][1], fmaf(be_lo, q1, -m[nt][1]));
-        s[nt][2] = fmaf(al_hi, s[nt][2], fmaf(be_hi, q0, -m[nt][0]));
-        s[nt][3] = fmaf(al_hi, s[nt][3], fmaf(be_hi, q1, -m[nt][1]));
+        {  // score - max for the lane's 2 rows x 2 columns, two lanes of FP32 per instruction
+          const uint64_t qq2 = pk2(q0, q1), nm2 = pk2(m[nt][0], m[nt][1]);  // m = minus the maximum
+          const uint64_t lo2 = ffma2(pk2(al_lo, al_lo), pk2(s[nt][0], s[nt][1]), ffma2(pk2(be_lo, be_lo), qq2, nm2));
+          const uint64_t hi2 = ffma2(pk2(al_hi, al_hi), pk2(s[nt][2], s[nt][3]), ffma2(pk2(be_hi, be_hi), qq2, nm2));
+          upk2(lo2, s[nt][0], s[nt][1]);
+          upk2(hi2, s[nt][2], s[nt][3]);
+        }
         if (masked) {
           const int l0 = QFS ? col_limit(nt * 8 + 2 * t, len) : lim[QFS ? 0 : nt][0];
           const int l1 = QFS ? col_limit(nt * 8 + 2 * t + 1, len) : lim[QFS ? 0 : nt][1];
@@ -990,7 +1021,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
             }
             const float up = fresh ? fmaxf(mx, -1.0e4f) : fmaxf(mx, 0.0f);
             const float f = fresh ? 0.0f : ex2(-up);
-            m[nt][cc] += up;
+            m[nt][cc] -= up;  // minus the maximum
             s[nt][cc] -= up;
             s[nt][cc + 2] -= up;
             l[nt][cc] *= f;
@@ -1014,12 +1045,15 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       for (int nt = 0; nt < NT; ++nt) {
         const float p0 = ex2(s[nt][0]), p1 = ex2(s[nt][1]);
         const float p2 = ex2(s[nt][2]), p3 = ex2(s[nt][3]);
-        l[nt][0] += p0 + p2;
-        l[nt][1] += p1 + p3;
-        zs[nt][0] = fmaf(p0, zv_lo, fmaf(p2, zv_hi, zs[nt][0]));
-        zs[nt][1] = fmaf(p1, zv_lo, fmaf(p3, zv_hi, zs[nt][1]));
-        const uint32_t f0 = movmatrix_trans(pack_f16x2(p0 * sv_lo, p1 * sv_lo));
-        const uint32_t f1 = movmatrix_trans(pack_f16x2(p2 * sv_hi, p3 * sv_hi));
+        const uint64_t plo = pk2(p0, p1), phi = pk2(p2, p3);
+        upk2(fadd2(pk2(l[nt][0], l[nt][1]), fadd2(plo, phi)), l[nt][0], l[nt][1]);
+        upk2(ffma2(plo, pk2(zv_lo, zv_lo), ffma2(phi, pk2(zv_hi, zv_hi), pk2(zs[nt][0], zs[nt][1]))),
+             zs[nt][0], zs[nt][1]);
+        float w0, w1, w2, w3;
+        upk2(fmul2(plo, pk2(sv_lo, sv_lo)), w0, w1);
+        upk2(fmul2(phi, pk2(sv_hi, sv_hi)), w2, w3);
+        const uint32_t f0 = movmatrix_trans(pack_f16x2(w0, w1));
+        const uint32_t f1 = movmatrix_trans(pack_f16x2(w2, w3));
         if constexpr (DS > 1) {
           pf[(nt * 2 + 0) * 32] = f0;
           pf[(nt * 2 + 1) * 32] = f1;
@@ -1047,11 +1081,14 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       }
       pv_slice<FULL, NT, ST, DS>(o, st, src * 16, g, t, d, pb, magic);
     }
+    }  // if (DS > 1 || in_range)
     __syncwarp();
     if (lane == 0) mbar_arrive(empty0 + slot * 8);
     if (!(info.z & 2)) continue;
 
     // ---- end of the piece -----------------------------------------------------------------
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) { m[nt][0] = -m[nt][0]; m[nt][1] = -m[nt][1]; }  // back to the maximum
     if (fresh) {
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) m[nt][0] = m[nt][1] = -1.0e30f;
@@ -1284,14 +1321,14 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   if (!full) {
     switch (pl.variant) {
       case 0: return launch_team<false, 1, 1, 4, 4, 4, true>(p, st);
-      case 1: return launch_team<false, 2, 2, 2, 4, 3, false>(p, st);
+      case 1: return launch_team<false, 2, 2, 2, 4, 3, true>(p, st);
       case 2: return launch_team<false, 4, 4, 1, 3, 3, true>(p, st);
       default: return launch_team<false, 8, 4, 2, 3, 1, true>(p, st);
     }
   }
   switch (pl.variant) {
     case 0: return launch_team<true, 1, 1, 4, 3, 3, true>(p, st);
-    case 1: return launch_team<true, 2, 2, 2, 3, 3, false>(p, st);
+    case 1: return launch_team<true, 2, 2, 2, 3, 3, true>(p, st);
     case 2: return launch_team<true, 4, 4, 1, 2, 3, true>(p, st);
     default: return launch_team<true, 8, 4, 2, 3, 1, true>(p, st);
   }
