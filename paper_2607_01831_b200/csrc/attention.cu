@@ -249,56 +249,6 @@ __device__ __forceinline__ void merge_codes(uint32_t xa, uint32_t xr, uint32_t& 
 // K fragments and the V fragments at <= 2-way bank conflicts)
 __device__ __forceinline__ int pi_row(int r) { return r ^ ((r >> 1) & 1); }
 
-// S^T[16 tokens x NT*8 columns] = level(K) . Q^T for the tile whose S rows g / g+8 are stage
-// rows r0 / r0+8: exact integer arithmetic (u8 levels x two s8 digit planes of q), returned
-// as floats (units: level x q_int).
-template <bool FULL, int NT, int ST>
-__device__ __forceinline__ void qk_int8(const uint32_t (&qf)[NT][2][4][2], uint32_t st, int r0, int t,
-                                        float (&s)[NT][4]) {
-  constexpr uint32_t KA = 0, KR = ST * 128;
-  // ---- S^T = level(K) . Q^T, exact in integers (u8 levels x two s8 digit planes of q) -----
-  {
-    int shi[NT][4], slo[NT][4];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) shi[nt][i] = slo[nt][i] = 0;
-    const uint4 a_lo = lds128(st + KA + r0 * 64 + t * 16);
-    const uint4 a_hi = lds128(st + KA + (r0 + 8) * 64 + t * 16);
-    const uint32_t xl[4] = {a_lo.x, a_lo.y, a_lo.z, a_lo.w};
-    const uint32_t xh[4] = {a_hi.x, a_hi.y, a_hi.z, a_hi.w};
-    uint32_t yl[4] = {0, 0, 0, 0}, yh[4] = {0, 0, 0, 0};
-    if (FULL) {
-      const uint4 b_lo = lds128(st + KR + r0 * 64 + t * 16);
-      const uint4 b_hi = lds128(st + KR + (r0 + 8) * 64 + t * 16);
-      yl[0] = b_lo.x; yl[1] = b_lo.y; yl[2] = b_lo.z; yl[3] = b_lo.w;
-      yh[0] = b_hi.x; yh[1] = b_hi.y; yh[2] = b_hi.z; yh[3] = b_hi.w;
-    }
-#pragma unroll
-    for (int wd = 0; wd < 4; ++wd) {
-      // bytes of ev*: levels of elements 0,2,4,6 of the word; od*: elements 1,3,5,7
-      uint32_t evl, odl, evh, odh;
-      if (FULL) {
-        merge_codes(xl[wd], yl[wd], evl, odl);
-        merge_codes(xh[wd], yh[wd], evh, odh);
-      } else {
-        evl = xl[wd] & 0x0F0F0F0Fu; odl = (xl[wd] >> 4) & 0x0F0F0F0Fu;
-        evh = xh[wd] & 0x0F0F0F0Fu; odh = (xh[wd] >> 4) & 0x0F0F0F0Fu;
-      }
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        mma_u8s8(shi[nt], evl, evh, odl, odh, qf[nt][0][wd][0], qf[nt][0][wd][1]);
-        mma_u8s8(slo[nt], evl, evh, odl, odh, qf[nt][1][wd][0], qf[nt][1][wd][1]);
-      }
-    }
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) s[nt][i] = (float)(shi[nt][i] * 128 + slo[nt][i]);
-  }
-
-}
-
 constexpr int kPieceUnits = 64;  // stage-units whose block ids are looked up at a time
 
 struct Item {  // one piece: a run of stage-units of one (sequence, KV head) given to one CTA
@@ -587,11 +537,12 @@ __device__ __forceinline__ void producer_warp(const AttnParams& p, int lane, uin
 // =============================================================================================
 // Shared-memory geometry of one kernel variant.  NT = 8-column tiles (all of them in every
 // warp), DS = warps per team = tiles per team and step = slices of the output dims,
-// TEAMS = teams per CTA, QFS = query fragments kept in shared memory instead of registers.
+// TEAMS = teams per CTA.  The query fragments (two s8 digit planes) and sum-of-q live in shared
+// memory, built once per piece.
 // With DS > 1 a team keeps one running maximum per column: two named barriers per step, growth
 // agreed through shared memory.  With DS == 1 a warp is its own team and nothing is exchanged.
 // =============================================================================================
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, bool QFS>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE>
 struct TeamCfg {
   static constexpr int kTW = DS * TEAMS;                    // consumer warps = tiles per stage
   static constexpr int kST = kTW * 16;
@@ -607,8 +558,7 @@ struct TeamCfg {
   static constexpr int kMailBytes = TEAMS > 1 ? kMailRegs * 32 * 4 : 0;  // one box, used slice by slice
   static constexpr int kXchgBytes = DS > 1 ? kTW * (16 + kColsPad * 4 + NT * 2 * 32 * 4) : 0;  // flag, colmax, P^T
   static constexpr int kLzBytes = DS * kColsPad * 2 * 4 + 16;
-  static constexpr bool kQfShared = QFS;                    // query fragments in shared memory
-  static constexpr int kQfBytes = kQfShared ? NT * 2 * 4 * 32 * 8 + kColsPad * 4 : 0;
+  static constexpr int kQfBytes = NT * 2 * 4 * 32 * 8 + kColsPad * 4;  // query fragments, sum of q
   static constexpr int kQBytes = 2 * kColsPad * LYNX_D * 2;
   static constexpr int kBlkBytes = kPieceUnits * kTW * 4;
   static constexpr int kInfoBytes = NSTAGE * 16 + 2 * 32;
@@ -726,9 +676,9 @@ __device__ __forceinline__ void pv_slice(float (&o)[NT][8 / DS][4], uint32_t st,
   }
 }
 
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, bool QFS>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE>
 __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
-  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE, QFS>;
+  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE>;
   constexpr int ST = C::kST, TW = C::kTW, MT = C::kMT;
   constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
   constexpr float kMidK = FULL ? 0.0f : 8.0f;
@@ -785,11 +735,8 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
   const int team = warp / DS, d = warp % DS;
   const float cb = p.sm_log2;
   const uint32_t magic = opaque_magic();
-  constexpr int NTR = QFS ? 1 : NT;  // register copies exist only when the fragments are not shared
-  uint32_t qf[NTR][2][4][2];
   // m holds MINUS the running maximum inside the stage loop (it enters the score FMA directly)
-  float qs[NTR][2], m[NT][2], l[NT][2], zs[NT][2], o[NT][MT][4];
-  int lim[NTR][2];
+  float m[NT][2], l[NT][2], zs[NT][2], o[NT][MT][4];
   const uint32_t qf_u32 = smem_u32(qf_s), qs_u32 = smem_u32(qs_s);
   auto col_limit = [&](int col, int len_) {
     return col < p.ncols ? (p.causal ? len_ - p.nq + col / p.G + 1 : len_) : 0;
@@ -830,8 +777,8 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       ca = p.sm_log2 * down * (FULL ? 1.0f : 16.0f);
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        // with shared fragments, warp w builds the n-tiles nt = w, w + TW, ... for everybody
-        const bool mine = !QFS || (nt % TW) == warp;
+        // warp w builds the shared fragments of the n-tiles nt = w, w + TW, ... for everybody
+        const bool mine = (nt % TW) == warp;
         if (mine) {
           const int c = nt * 8 + g;
 #pragma unroll
@@ -852,13 +799,8 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
               hi_o |= (uint32_t)((qv[2 * k + 1] >> 7) & 0xFF) << (8 * k);
               lo_o |= (uint32_t)(qv[2 * k + 1] & 127) << (8 * k);
             }
-            if constexpr (QFS) {
-              reinterpret_cast<uint2*>(qf_s)[((nt * 2 + 0) * 4 + wd) * 32 + lane] = make_uint2(hi_e, hi_o);
-              reinterpret_cast<uint2*>(qf_s)[((nt * 2 + 1) * 4 + wd) * 32 + lane] = make_uint2(lo_e, lo_o);
-            } else {
-              qf[nt][0][wd][0] = hi_e; qf[nt][0][wd][1] = hi_o;
-              qf[nt][1][wd][0] = lo_e; qf[nt][1][wd][1] = lo_o;
-            }
+            reinterpret_cast<uint2*>(qf_s)[((nt * 2 + 0) * 4 + wd) * 32 + lane] = make_uint2(hi_e, hi_o);
+            reinterpret_cast<uint2*>(qf_s)[((nt * 2 + 1) * 4 + wd) * 32 + lane] = make_uint2(lo_e, lo_o);
           }
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
@@ -876,12 +818,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
             sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 4);
             sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 8);
             sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 16);
-            if constexpr (QFS) {
-              if (g == 0) qs_s[col] = sum;
-            } else {
-              qs[nt][cc] = sum;
-              lim[nt][cc] = col_limit(col, len);
-            }
+            if (g == 0) qs_s[col] = sum;
           }
         }
 #pragma unroll
@@ -891,7 +828,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 #pragma unroll
           for (int i = 0; i < 4; ++i) o[nt][mt][i] = 0.0f;
       }
-      if constexpr (QFS) named_bar(1, C::kConsThreads);  // the shared fragments are complete
+      named_bar(1, C::kConsThreads);  // the shared fragments are complete
       fresh = true;
     }
 
@@ -912,7 +849,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
     // ---- phase A: scores of this warp's tile, growth vote -------------------------------
     bool gw = false;
     if (valid) {
-      if constexpr (QFS) {
+      {
         uint32_t a[4][4];
         k_fragments<FULL, ST>(st, r0, t, a);
 #pragma unroll
@@ -928,8 +865,6 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 #pragma unroll
           for (int i = 0; i < 4; ++i) s[nt][i] = (float)(shi[i] * 128 + slo[i]);
         }
-      } else {
-        qk_int8<FULL, NT, ST>(qf, st, r0, t, s);
       }
       float2 km_lo = lds64f(st + KM + r0 * 8), km_hi = lds64f(st + KM + (r0 + 8) * 8);
       vm_lo = lds64f(st + VM + r0 * 8); vm_hi = lds64f(st + VM + (r0 + 8) * 8);
@@ -947,13 +882,8 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       const float be_lo = fmaf(km_lo.x, kMidK, km_lo.y) * cb, be_hi = fmaf(km_hi.x, kMidK, km_hi.y) * cb;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        float q0, q1;
-        if constexpr (QFS) {
-          const float2 qq = lds64f(qs_u32 + (nt * 8 + 2 * t) * 4);
-          q0 = qq.x; q1 = qq.y;
-        } else {
-          q0 = qs[nt][0]; q1 = qs[nt][1];
-        }
+        const float2 qq = lds64f(qs_u32 + (nt * 8 + 2 * t) * 4);
+        const float q0 = qq.x, q1 = qq.y;
         {  // score - max for the lane's 2 rows x 2 columns, two lanes of FP32 per instruction
           const uint64_t qq2 = pk2(q0, q1), nm2 = pk2(m[nt][0], m[nt][1]);  // m = minus the maximum
           const uint64_t lo2 = ffma2(pk2(al_lo, al_lo), pk2(s[nt][0], s[nt][1]), ffma2(pk2(be_lo, be_lo), qq2, nm2));
@@ -962,8 +892,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
           upk2(hi2, s[nt][2], s[nt][3]);
         }
         if (masked) {
-          const int l0 = QFS ? col_limit(nt * 8 + 2 * t, len) : lim[QFS ? 0 : nt][0];
-          const int l1 = QFS ? col_limit(nt * 8 + 2 * t + 1, len) : lim[QFS ? 0 : nt][1];
+          const int l0 = col_limit(nt * 8 + 2 * t, len), l1 = col_limit(nt * 8 + 2 * t + 1, len);
           if (tok_lo >= l0) s[nt][0] = -INFINITY;
           if (tok_lo >= l1) s[nt][1] = -INFINITY;
           if (tok_hi >= l0) s[nt][2] = -INFINITY;
@@ -1208,10 +1137,10 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 
 // At least MINB CTAs per SM (the compiler caps registers accordingly).  Nine warps cannot
 // have more than 168 registers each: three of them share one SM sub-partition's 16 K registers.
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB, bool QFS>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB>
 __global__ void __launch_bounds__((DS * TEAMS + 1) * 32, MINB)
 attn_team_kernel(const AttnParams p) {
-  attn_team_body<FULL, NT, DS, TEAMS, NSTAGE, QFS>(p);
+  attn_team_body<FULL, NT, DS, TEAMS, NSTAGE>(p);
 }
 // ------------------------------------------------------------------ host side
 constexpr int kMaxCtasPerSm = 4;
@@ -1248,14 +1177,14 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   return true;
 }
 
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB, bool QFS>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB>
 lynx_status launch_team(const AttnParams& p, cudaStream_t st) {
-  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE, QFS>;
+  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE>;
   static_assert(MINB <= kMaxCtasPerSm, "partial slots are sized for kMaxCtasPerSm CTAs per SM");
   constexpr int kCtasPerSm = MINB;
   static_assert(kCtasPerSm * (C::kSmem + 1024) <= 228 * 1024, "shared memory budget per SM");
   static_assert(2 + TEAMS <= 16, "named barriers");
-  auto kern = attn_team_kernel<FULL, NT, DS, TEAMS, NSTAGE, MINB, QFS>;
+  auto kern = attn_team_kernel<FULL, NT, DS, TEAMS, NSTAGE, MINB>;
   static bool configured[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -1317,20 +1246,20 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   p.bt = shape->block_tokens; p.num_blocks = shape->num_blocks; p.max_blocks = shape->max_blocks_per_seq;
   p.ncols = pl.ncols;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // <FULL, NT, DS, TEAMS, stages, CTAs/SM, shared query fragments>
+  // <FULL, NT, DS, TEAMS, stages, CTAs/SM>
   if (!full) {
     switch (pl.variant) {
-      case 0: return launch_team<false, 1, 1, 4, 4, 4, true>(p, st);
-      case 1: return launch_team<false, 2, 2, 2, 4, 3, true>(p, st);
-      case 2: return launch_team<false, 4, 4, 1, 3, 3, true>(p, st);
-      default: return launch_team<false, 8, 4, 2, 3, 1, true>(p, st);
+      case 0: return launch_team<false, 1, 1, 4, 4, 4>(p, st);
+      case 1: return launch_team<false, 2, 2, 2, 4, 3>(p, st);
+      case 2: return launch_team<false, 4, 4, 1, 3, 3>(p, st);
+      default: return launch_team<false, 8, 4, 2, 3, 1>(p, st);
     }
   }
   switch (pl.variant) {
-    case 0: return launch_team<true, 1, 1, 4, 3, 3, true>(p, st);
-    case 1: return launch_team<true, 2, 2, 2, 3, 3, true>(p, st);
-    case 2: return launch_team<true, 4, 4, 1, 2, 3, true>(p, st);
-    default: return launch_team<true, 8, 4, 2, 3, 1, true>(p, st);
+    case 0: return launch_team<true, 1, 1, 4, 3, 3>(p, st);
+    case 1: return launch_team<true, 2, 2, 2, 3, 3>(p, st);
+    case 2: return launch_team<true, 4, 4, 1, 2, 3>(p, st);
+    default: return launch_team<true, 8, 4, 2, 3, 1>(p, st);
   }
 }
 
