@@ -151,16 +151,6 @@ __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
   asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
   return d;
 }
-__device__ __forceinline__ uint32_t hadd2(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("add.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-__device__ __forceinline__ uint32_t hfma2(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t d;
-  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -210,34 +200,18 @@ __device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
   return d;
 }
 
-// FP16x2 constants
-constexpr uint32_t kMagic = 0x64006400u;      // 1024, 1024
-constexpr uint32_t kNeg1032 = 0xE408E408u;    // -1032
-constexpr uint32_t kSixteenth = 0x2C002C00u;  // 1/16
-constexpr uint32_t kNeg72 = 0xD480D480u;      // -72
-constexpr uint32_t kNeg1152 = 0xE480E480u;    // -1152
-
-// (a & mask) | c in one LOP3: the mask is an immediate, c must sit in a register
-template <uint32_t kMask>
-__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t c) {
-  uint32_t d;
-  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "n"(kMask), "r"(c));
-  return d;
-}
-// Four FP16 pairs (value - 8) from the low 16 bits of each half of u: nibbles 0..3 of the low
-// half go to the low lanes, nibbles 0..3 of the high half to the high lanes.  `magic` holds
-// kMagic in a register the compiler cannot fold away (see opaque_magic).
-__device__ __forceinline__ void nib4_to_h2(uint32_t u, uint32_t magic, uint32_t (&r)[4]) {
+// Four FP16 pairs from the low 16 bits of each half of u, with no arithmetic at all: a 16-bit
+// pattern 0x000n is the FP16 subnormal n * 2^-24 and 0x00n0 is 16 n * 2^-24, both exact, and the
+// tensor core takes subnormal FP16 operands as they are.  r[0], r[2] hold nibbles 0 and 2 of
+// each half (scale 2^-24), r[1], r[3] nibbles 1 and 3 (scale 2^-20); the scales are undone
+// when the accumulators are written out.  (Full codes use the same idea with one byte per
+// 16-bit lane: 0x00cc = code * 2^-24.)
+__device__ __forceinline__ void nib4_to_h2(uint32_t u, uint32_t (&r)[4]) {
   const uint32_t s = u >> 8;
-  r[0] = hadd2(and_or<0x000F000Fu>(u, magic), kNeg1032);
-  r[1] = hfma2(and_or<0x00F000F0u>(u, magic), kSixteenth, kNeg72);
-  r[2] = hadd2(and_or<0x000F000Fu>(s, magic), kNeg1032);
-  r[3] = hfma2(and_or<0x00F000F0u>(s, magic), kSixteenth, kNeg72);
-}
-__device__ __forceinline__ uint32_t opaque_magic() {
-  uint32_t m;
-  asm volatile("mov.u32 %0, 0x64006400;" : "=r"(m));
-  return m;
+  r[0] = u & 0x000F000Fu;
+  r[1] = u & 0x00F000F0u;
+  r[2] = s & 0x000F000Fu;
+  r[3] = s & 0x00F000F0u;
 }
 // Full codes of 8 elements from an anchor word and a residual word: ev = codes of elements
 // 0,2,4,6 (one per byte), od = codes of elements 1,3,5,7.
@@ -554,10 +528,10 @@ struct TeamCfg {
   static constexpr int kColsPad = NT * 8;
   static constexpr int kMT = 8 / DS;                        // m-tiles (16 dims) per warp
   static constexpr int kRing = NSTAGE * kStageBytes;
-  static constexpr int kMailRegs = NT * kMT * 4 + NT * 6;   // o slice + m, l, zs
+  static constexpr int kMailRegs = NT * kMT * 4 + NT * 10;  // o slice + m, l, zs, sw, hw
   static constexpr int kMailBytes = TEAMS > 1 ? kMailRegs * 32 * 4 : 0;  // one box, used slice by slice
   static constexpr int kXchgBytes = DS > 1 ? kTW * (16 + kColsPad * 4 + NT * 2 * 32 * 4) : 0;  // flag, colmax, P^T
-  static constexpr int kLzBytes = DS * kColsPad * 2 * 4 + 16;
+  static constexpr int kLzBytes = DS * kColsPad * 4 * 4 + 16;
   static constexpr int kQfBytes = NT * 2 * 4 * 32 * 8 + kColsPad * 4;  // query fragments, sum of q
   static constexpr int kQBytes = 2 * kColsPad * LYNX_D * 2;
   static constexpr int kBlkBytes = kPieceUnits * kTW * 4;
@@ -601,7 +575,7 @@ __device__ __forceinline__ void k_fragments(uint32_t st, int r0, int t, uint32_t
 // word d, DS=4 word d>>1 / half d&1.
 template <bool FULL, int NT, int ST, int DS>
 __device__ __forceinline__ void pv_slice(float (&o)[NT][8 / DS][4], uint32_t st, int row0, int g, int t,
-                                         int d, const uint32_t (&pb)[NT][2], uint32_t magic) {
+                                         int d, const uint32_t (&pb)[NT][2]) {
   constexpr uint32_t VA = ST * 64, VR = ST * 192;
   constexpr int NW = DS == 1 ? 2 : 1;  // words of the lane's 8 V bytes this warp touches
   constexpr int NH = DS == 4 ? 1 : 2;  // halves of each word
@@ -651,19 +625,16 @@ __device__ __forceinline__ void pv_slice(float (&o)[NT][8 / DS][4], uint32_t st,
       const uint32_t sel = half ? 0x7632u : 0x5410u;
       uint32_t ab[4], cd[4];
       if (!FULL) {
-        nib4_to_h2(prmt(A[i], Bw[i], sel), magic, ab);  // dims e(4half+0..3), token pair (a, b)
-        nib4_to_h2(prmt(C[i], Dw[i], sel), magic, cd);  // same dims, token pair (c, d)
+        nib4_to_h2(prmt(A[i], Bw[i], sel), ab);  // dims e(4half+0..3), token pair (a, b)
+        nib4_to_h2(prmt(C[i], Dw[i], sel), cd);  // same dims, token pair (c, d)
       } else {
         const uint32_t uab = prmt(ea, eb, sel), vab = prmt(oa, ob, sel);
         const uint32_t ucd = prmt(ec, ed, sel), vcd = prmt(oc, od, sel);
-        ab[0] = hadd2(and_or<0x00FF00FFu>(uab, magic), kNeg1152);
-        ab[1] = hadd2(and_or<0x00FF00FFu>(vab, magic), kNeg1152);
-        ab[2] = hadd2(prmt(uab, magic, 0x7351), kNeg1152);
-        ab[3] = hadd2(prmt(vab, magic, 0x7351), kNeg1152);
-        cd[0] = hadd2(and_or<0x00FF00FFu>(ucd, magic), kNeg1152);
-        cd[1] = hadd2(and_or<0x00FF00FFu>(vcd, magic), kNeg1152);
-        cd[2] = hadd2(prmt(ucd, magic, 0x7351), kNeg1152);
-        cd[3] = hadd2(prmt(vcd, magic, 0x7351), kNeg1152);
+        // a 16-bit pattern 0x00cc is the FP16 subnormal code * 2^-24: one byte per 16-bit lane
+        ab[0] = uab & 0x00FF00FFu; ab[1] = vab & 0x00FF00FFu;
+        ab[2] = prmt(uab, 0u, 0x4341); ab[3] = prmt(vab, 0u, 0x4341);
+        cd[0] = ucd & 0x00FF00FFu; cd[1] = vcd & 0x00FF00FFu;
+        cd[2] = prmt(ucd, 0u, 0x4341); cd[3] = prmt(vcd, 0u, 0x4341);
       }
 #pragma unroll
       for (int qd = 0; qd < 2; ++qd) {
@@ -682,8 +653,9 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
   constexpr int ST = C::kST, TW = C::kTW, MT = C::kMT;
   constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
   constexpr float kMidK = FULL ? 0.0f : 8.0f;
-  constexpr float kMidV = FULL ? 128.0f : 136.0f;
+  constexpr float kMidV = FULL ? 0.0f : 8.0f;      // V levels: plain codes (full) / plain nibbles (anchor)
   constexpr float kLevelScaleV = FULL ? 1.0f : 16.0f;
+  constexpr uint32_t kOnesH2 = 0x3C003C00u;        // FP16 pair (1, 1)
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* ring = smem;
   float* mail = reinterpret_cast<float*>(smem + C::kRing);
@@ -734,9 +706,13 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
   const int g = lane >> 2, t = lane & 3;
   const int team = warp / DS, d = warp % DS;
   const float cb = p.sm_log2;
-  const uint32_t magic = opaque_magic();
   // m holds MINUS the running maximum inside the stage loop (it enters the score FMA directly)
-  float m[NT][2], l[NT][2], zs[NT][2], o[NT][MT][4];
+  // sw, hw: sums of the V weights p * scale before and after their rounding to FP16; the ratio
+  // sw / hw scales the accumulators at the end, which removes the rounding's first-order effect
+  // (the residue is the rounding error times a level's distance from the weighted mean level)
+  // (hw comes from one extra MMA per n-tile with an all-ones A operand, which gives every lane
+  // the complete sums of the warp's own tile for its columns 2t, 2t+1)
+  float m[NT][2], l[NT][2], zs[NT][2], sw[NT][2], hw[NT][2], o[NT][MT][4];
   const uint32_t qf_u32 = smem_u32(qf_s), qs_u32 = smem_u32(qs_s);
   auto col_limit = [&](int col, int len_) {
     return col < p.ncols ? (p.causal ? len_ - p.nq + col / p.G + 1 : len_) : 0;
@@ -822,7 +798,10 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
           }
         }
 #pragma unroll
-        for (int cc = 0; cc < 2; ++cc) { m[nt][cc] = 0.0f; l[nt][cc] = 0.0f; zs[nt][cc] = 0.0f; }
+        for (int cc = 0; cc < 2; ++cc) {
+          m[nt][cc] = 0.0f; l[nt][cc] = 0.0f; zs[nt][cc] = 0.0f; sw[nt][cc] = 0.0f;
+          hw[nt][cc] = 0.0f;
+        }
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -955,6 +934,8 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
             s[nt][cc + 2] -= up;
             l[nt][cc] *= f;
             zs[nt][cc] *= f;
+            sw[nt][cc] *= f;
+            hw[nt][cc] *= f;
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
               o[nt][mt][cc] *= f;
@@ -981,8 +962,13 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
         float w0, w1, w2, w3;
         upk2(fmul2(plo, pk2(sv_lo, sv_lo)), w0, w1);
         upk2(fmul2(phi, pk2(sv_hi, sv_hi)), w2, w3);
-        const uint32_t f0 = movmatrix_trans(pack_f16x2(w0, w1));
-        const uint32_t f1 = movmatrix_trans(pack_f16x2(w2, w3));
+        const uint32_t h01 = pack_f16x2(w0, w1), h23 = pack_f16x2(w2, w3);
+        upk2(fadd2(pk2(sw[nt][0], sw[nt][1]), fadd2(pk2(w0, w1), pk2(w2, w3))), sw[nt][0], sw[nt][1]);
+        const uint32_t f0 = movmatrix_trans(h01);
+        const uint32_t f1 = movmatrix_trans(h23);
+        float hsum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        mma16816(hsum, kOnesH2, kOnesH2, kOnesH2, kOnesH2, f0, f1);
+        upk2(fadd2(pk2(hw[nt][0], hw[nt][1]), pk2(hsum[0], hsum[1])), hw[nt][0], hw[nt][1]);
         if constexpr (DS > 1) {
           pf[(nt * 2 + 0) * 32] = f0;
           pf[(nt * 2 + 1) * 32] = f1;
@@ -995,7 +981,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
     if constexpr (DS > 1) named_bar(2 + team, DS * 32);
     // ---- phase C: P.V of the team's tiles for this warp's slice of the output dims --------
     if constexpr (DS == 1) {
-      if (valid) pv_slice<FULL, NT, ST, 1>(o, st, warp * 16, g, t, 0, pown, magic);
+      if (valid) pv_slice<FULL, NT, ST, 1>(o, st, warp * 16, g, t, 0, pown);
     }
 #pragma unroll
     for (int tau = 0; tau < (DS > 1 ? DS : 0); ++tau) {
@@ -1008,7 +994,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
         pb[nt][0] = *reinterpret_cast<const volatile uint32_t*>(pf + (nt * 2 + 0) * 32);
         pb[nt][1] = *reinterpret_cast<const volatile uint32_t*>(pf + (nt * 2 + 1) * 32);
       }
-      pv_slice<FULL, NT, ST, DS>(o, st, src * 16, g, t, d, pb, magic);
+      pv_slice<FULL, NT, ST, DS>(o, st, src * 16, g, t, d, pb);
     }
     }  // if (DS > 1 || in_range)
     __syncwarp();
@@ -1039,6 +1025,8 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
               box[(r++) * 32] = m[nt][cc];
               box[(r++) * 32] = l[nt][cc];
               box[(r++) * 32] = zs[nt][cc];
+              box[(r++) * 32] = sw[nt][cc];
+              box[(r++) * 32] = hw[nt][cc];
             }
           }
         }
@@ -1050,7 +1038,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
             float f1[2], f2[2];
 #pragma unroll
             for (int cc = 0; cc < 2; ++cc) {
-              const float m2 = box[((MT * 4 + 6) * nt + MT * 4 + 3 * cc) * 32];
+              const float m2 = box[((MT * 4 + 10) * nt + MT * 4 + 5 * cc) * 32];
               const float M = fmaxf(m[nt][cc], m2);
               f1[cc] = ex2(m[nt][cc] - M);
               f2[cc] = ex2(m2 - M);
@@ -1068,8 +1056,12 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
               r++;
               const float l2 = box[(r++) * 32];
               const float z2 = box[(r++) * 32];
+              const float s2 = box[(r++) * 32];
+              const float h2 = box[(r++) * 32];
               l[nt][cc] = l[nt][cc] * f1[cc] + l2 * f2[cc];
               zs[nt][cc] = zs[nt][cc] * f1[cc] + z2 * f2[cc];
+              sw[nt][cc] = sw[nt][cc] * f1[cc] + s2 * f2[cc];
+              hw[nt][cc] = hw[nt][cc] * f1[cc] + h2 * f2[cc];
             }
           }
         }
@@ -1082,16 +1074,17 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int cc = 0; cc < 2; ++cc) {
-          float lv = l[nt][cc], z = zs[nt][cc];
+          float lv = l[nt][cc], z = zs[nt][cc], sv = sw[nt][cc];
+          const float hv = hw[nt][cc];  // already complete over the tile's rows
 #pragma unroll
           for (int off = 4; off <= 16; off <<= 1) {
             lv += __shfl_xor_sync(0xFFFFFFFFu, lv, off);
             z += __shfl_xor_sync(0xFFFFFFFFu, z, off);
+            sv += __shfl_xor_sync(0xFFFFFFFFu, sv, off);
           }
-          if (g == 0) {
-            lz[((size_t)d * C::kColsPad + nt * 8 + 2 * t + cc) * 2 + 0] = lv;
-            lz[((size_t)d * C::kColsPad + nt * 8 + 2 * t + cc) * 2 + 1] = z;
-          }
+          if (g == 0)
+            *reinterpret_cast<float4*>(lz + ((size_t)d * C::kColsPad + nt * 8 + 2 * t + cc) * 4) =
+                make_float4(lv, z, sv, hv);
         }
     }
     named_bar(1, C::kConsThreads);
@@ -1104,23 +1097,27 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 #pragma unroll
         for (int cc = 0; cc < 2; ++cc) {
           const int c = nt * 8 + 2 * t + cc;
-          float lt = 0.0f, z = 0.0f;
+          float lt = 0.0f, z = 0.0f, st_ = 0.0f, ht = 0.0f;
 #pragma unroll
           for (int dd = 0; dd < DS; ++dd) {
-            lt += lz[((size_t)dd * C::kColsPad + c) * 2 + 0];
-            z += lz[((size_t)dd * C::kColsPad + c) * 2 + 1];
+            const float4 v = *reinterpret_cast<const float4*>(lz + ((size_t)dd * C::kColsPad + c) * 4);
+            lt += v.x; z += v.y; st_ += v.z; ht += v.w;
           }
           if (c >= p.ncols) continue;
           const int j = c / p.G, hh = c % p.G;
           float* dst = direct ? p.out + (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D
                               : part + (size_t)c * kPartStride;
           const float inv = direct ? (lt > 0.0f ? 1.0f / lt : 0.0f) : 1.0f;
+          // undo the subnormal scales of the V operands (2^-24; odd dims of the anchor 2^-20) and
+          // apply the exact-to-rounded weight ratio
+          const float ratio = ht > 0.0f ? st_ / ht : 1.0f;
+          const float fix_even = 16777216.0f * ratio, fix_odd = (FULL ? 16777216.0f : 1048576.0f) * ratio;
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
             const int gmt = d * MT + mt;  // m-tile index among the eight of a lane's 16 dims
             const int dim = 16 * g + 8 * (gmt >> 2) + 2 * (gmt & 3);
             *reinterpret_cast<float2*>(dst + dim) =
-                make_float2((o[nt][mt][cc] + z) * inv, (o[nt][mt][cc + 2] + z) * inv);
+                make_float2(fmaf(o[nt][mt][cc], fix_even, z) * inv, fmaf(o[nt][mt][cc + 2], fix_odd, z) * inv);
           }
           if (!direct && d == 0 && g == 0) { dst[128] = m[nt][cc]; dst[129] = lt; }
         }

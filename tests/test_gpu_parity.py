@@ -216,6 +216,49 @@ def test_merge_verify_matches_oracle_and_decides_identically(lynx, case, causal)
         assert int(fr[0]) == j
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_short_heavy_tailed_contexts_keep_a_margin(lynx, seed):
+    # a few tokens with heavy-tailed values: one token dominates, so the rounding of its weight to
+    # FP16 is not averaged away; the weight-ratio correction must keep the error well inside the bound
+    c = _case(lynx, 400 + seed, 4, 2, 8, 1, (1, 15, 17, 3), 16, True, "student_t4")
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    for full in (False, True):
+        if full:
+            got = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"])[0]
+        else:
+            got = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"])
+        lynx.check(c["ws"])
+        ref = oracle.attention(full, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                               c["lens"].numpy(), 2, 16, causal=full)
+        got = got.cpu().numpy().astype(np.float64)
+        worst = float(np.max(np.abs(got - ref) / (ATOL + RTOL * np.abs(ref))))
+        assert worst <= 0.5, f"full={full}: worst error/bound {worst:.3f}"
+
+
+@pytest.mark.parametrize("recipe", ["student_t4", "normal_outlier2pct_x10"])
+def test_single_token_context_returns_its_value_row(lynx, recipe):
+    # softmax over one token is 1, so the output is that token's dequantised V row: FP32 rounding
+    # only, whatever the magnitude of the row (the FP16 rounding of the weight cancels exactly)
+    B, Hkv, G = 6, 2, 4
+    c = _case(lynx, 500, B, Hkv, G, 1, (1,) * B, 16, True, recipe)
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    from util import dequant
+    for full in (False, True):
+        if full:
+            got = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"])[0]
+        else:
+            got = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"])
+        lynx.check(c["ws"])
+        got = got.cpu().numpy().astype(np.float64)
+        va, vr, vm = c["vp"]
+        for b in range(B):
+            blk = int(c["table"][b, 0])
+            for h in range(Hkv * G):
+                row = dequant(va[blk, h // G, 0], vr[blk, h // G, 0], vm[blk, h // G, 0], full)
+                size = abs(float(vm[blk, h // G, 0, 1])) + 255.0 * float(vm[blk, h // G, 0, 0])
+                assert np.max(np.abs(got[b, 0, h] - row)) <= 4e-6 * size + 1e-30
+
+
 def test_anchor_then_verify_window_like_the_decoder(lynx):
     # k draft steps on the Anchor state with growing context, then one verify pass on Q_full
     B, Hkv, G, k, L = 1, 2, 4, 4, 1203
