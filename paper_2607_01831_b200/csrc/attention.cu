@@ -215,9 +215,15 @@ __device__ __forceinline__ void nib4_to_h2(uint32_t u, uint32_t (&r)[4]) {
 }
 // Full codes of 8 elements from an anchor word and a residual word: ev = codes of elements
 // 0,2,4,6 (one per byte), od = codes of elements 1,3,5,7.
+// Each is one shift and one bitwise select, (a & mask) | (b & ~mask), in a single LOP3.
+__device__ __forceinline__ uint32_t bit_select(uint32_t a, uint32_t b, uint32_t mask) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xE4;" : "=r"(d) : "r"(a), "r"(b), "r"(mask));
+  return d;
+}
 __device__ __forceinline__ void merge_codes(uint32_t xa, uint32_t xr, uint32_t& ev, uint32_t& od) {
-  ev = ((xa << 4) & 0xF0F0F0F0u) | (xr & 0x0F0F0F0Fu);
-  od = (xa & 0xF0F0F0F0u) | ((xr >> 4) & 0x0F0F0F0Fu);
+  ev = bit_select(xa << 4, xr, 0xF0F0F0F0u);
+  od = bit_select(xa, xr >> 4, 0xF0F0F0F0u);
 }
 // token row permutation inside a 16-token tile (keeps the shared-memory reads of both the
 // K fragments and the V fragments at <= 2-way bank conflicts)
