@@ -232,7 +232,7 @@ __device__ __forceinline__ int pi_row(int r) { return r ^ ((r >> 1) & 1); }
 constexpr int kPieceUnits = 64;  // stage-units whose block ids are looked up at a time
 
 struct Item {  // one piece: a run of stage-units of one (sequence, KV head) given to one CTA
-  int b, hkv, len, first_cta, n_contrib, pad0, pad1, pad2;
+  int b, hkv, len, first_cta, n_contrib, pad0, pad1, pad2;  // pad0 = units, pad1 = first unit
 };
 
 __device__ __forceinline__ void named_bar(int id, int nthreads) {
@@ -452,7 +452,9 @@ __device__ __forceinline__ void producer_warp(const AttnParams& p, int lane, uin
       it.b = b; it.hkv = hkv; it.len = len;
       it.first_cta = (int)(seg0 / q);
       it.n_contrib = (int)((seg0 + U - 1) / q) - it.first_cta + 1;
-      it.pad0 = it.pad1 = it.pad2 = 0;
+      it.pad0 = n;   // units of this piece
+      it.pad1 = u;   // index of its first unit within the sequence
+      it.pad2 = 0;
       items[qi] = it;
       mbar_expect_tx(qfull0 + qi * 8, (uint32_t)(p.nq * p.G * LYNX_D * 2));
     }
@@ -1145,6 +1147,11 @@ __global__ void __launch_bounds__((DS * TEAMS + 1) * 32, MINB)
 attn_team_kernel(const AttnParams p) {
   attn_team_body<FULL, NT, DS, TEAMS, NSTAGE>(p);
 }
+#ifndef LYNX_WIDE_VERIFY
+#define LYNX_WIDE_VERIFY 1   // 0: keep the mma.sync kernels for 17..64 verify columns (comparison builds)
+#endif
+#include "attention_wide.cuh"
+
 // ------------------------------------------------------------------ host side
 constexpr int kMaxCtasPerSm = 4;
 
@@ -1258,6 +1265,12 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
       default: return launch_team<false, 8, 4, 2, 3, 1>(p, st);
     }
   }
+#if LYNX_WIDE_VERIFY
+  if (pl.variant == 3) return launch_wide<2>(p, st);
+#if LYNX_WIDE_VERIFY > 1
+  if (pl.variant == 2) return launch_wide<4>(p, st);
+#endif
+#endif
   switch (pl.variant) {
     case 0: return launch_team<true, 1, 1, 4, 3, 3>(p, st);
     case 1: return launch_team<true, 2, 2, 2, 3, 3>(p, st);

@@ -1,0 +1,594 @@
+// Merge-verify attention for 17..64 columns on the fifth-generation tensor cores (tcgen05, TMEM).
+// Included by attention.cu inside its namespace: shares the stream-K producer warp, the piece
+// bookkeeping and finish_piece with the mma.sync kernels.
+//
+// With k*G >= 17 query rows per KV head the verify pass of Section 4.3 is a dense contraction
+// (about 60 / 120 flop per plane byte at 32 / 64 columns), which the mma.sync kernels cannot
+// feed: their tensor pipe would have to be busier than 100 % at the HBM roofline.  Here the two
+// contractions of a 64-token stage-unit are two tcgen05.mma groups with M = 128:
+//   S[128 rows x 64 tokens]  = Q[128 x 128 dims] . codes(K)^T      A, B in shared memory (FP16)
+//   O[128 rows x 128 dims]  += P[128 x 64 tokens] . codes(V)       A = P in TMEM, B in shared memory
+// Row r of the M = 128 is (copy, column): the k*G columns (padded to 32 or 64) are replicated
+// NCOPY = 4 or 2 times and copy i owns tokens [i*64/NCOPY, (i+1)*64/NCOPY) of the unit: its P
+// entries for the other tokens stay zero, so every row is an independent flash-decoding split
+// with its own running maximum and all 128 TMEM lanes (threads) have softmax work.  Rows are
+// merged at the end of a piece.
+//
+// Two warpgroups (4 warps each) alternate over the units of a piece; each has its own S, P, O
+// regions in TMEM (64 + 32 + 128 columns) and its own FP16 operand tiles, so one group's
+// conversion and softmax overlap the other's MMAs.  Per unit a group
+//   1. expands the nibble planes of the raw stage to FP16 code tiles (subnormal patterns
+//      0x00cc = code * 2^-24, one PRMT/LOP3 per word) in the canonical 128-byte-swizzled layout,
+//      the same bytes serving as K-major B operand (K) and MN-major B operand (V);
+//   2. one thread issues S = Q.K^T (8 k-steps) and commits to an mbarrier;
+//   3. every thread reads its row's scores from TMEM, applies the per-token scale / zero point,
+//      the causal limit and the lazily raised running maximum, writes FP16 weights p*scale_v
+//      to its part of P;
+//   4. one thread issues O += P.V (4 k-steps) and commits.
+// Element order along head_dim inside each group of 8 is {0,4,2,6,1,5,3,7} in all operand
+// tiles (what the nibble expansion produces for free); it is undone when O is written out.
+
+// position -> element within a group of 8: {0,4,2,6,1,5,3,7}, the 3-bit reversal
+__host__ __device__ constexpr int wide_perm(int pos) { return ((pos & 1) << 2) | (pos & 2) | ((pos >> 2) & 1); }
+
+template <int NCOPY>
+struct WideCfg {
+  static constexpr int kST = 64;                 // tokens per stage-unit
+  static constexpr int kTW = 4;                  // 16-token sub-blocks per stage
+  static constexpr int kNStage = 7;
+  static constexpr int kSubBytes = 16 * 272;
+  static constexpr int kStageBytes = kST * 272;  // KA, VA, KR, VR (4 KiB each), KM, VM (512 B each)
+  static constexpr int kColsPad = 128 / NCOPY;
+  static constexpr int kTok = kST / NCOPY;       // tokens of a unit that one row owns
+  static constexpr int kConsWarps = 8;
+  static constexpr int kConsThreads = 256;
+  static constexpr int kThreads = 288;
+  // shared memory map (offsets from a 1024-byte aligned base)
+  static constexpr int kTileBytes = 2 * 64 * 128;              // [2 dim blocks][64 tokens][128 B]
+  static constexpr int kOffCanon = 0;                          // [wg][K tile, V tile]
+  static constexpr int kOffRing = 4 * kTileBytes;
+  static constexpr int kOffScal = kOffRing + kNStage * kStageBytes;  // [wg][set][alpha, beta, zz, sv][64]
+  static constexpr int kOffQs = kOffScal + 2 * 2 * 4 * 64 * 4;       // sum of q per column
+  static constexpr int kOffQ = kOffQs + kColsPad * 4;                // raw BF16 queries, 2 slots
+  static constexpr int kOffBlk = kOffQ + 2 * kColsPad * LYNX_D * 2;
+  static constexpr int kOffInfo = kOffBlk + kPieceUnits * kTW * 4;
+  static constexpr int kOffBars = kOffInfo + kNStage * 16 + 2 * 32;
+  static constexpr int kOffMisc = kOffBars + (2 * kNStage + 8) * 8;  // full, empty, qfull/qempty, sready, odone
+  static constexpr int kSmem = kOffMisc + 256 + 1024;                // + alignment slack
+  // TMEM columns of a warpgroup
+  static constexpr int kTmemQ = 0, kTmemWg0 = 64, kTmemS = 0, kTmemP = 64, kTmemO = 96, kTmemWg = 224, kTmemCols = 512;
+  static_assert(kOffRing % 16 == 0 && kTileBytes % 1024 == 0, "operand tiles are 1024-byte aligned");
+  static_assert(kOffQ % 16 == 0 && kOffBars % 8 == 0, "alignment");
+  static_assert(kSmem <= 227 * 1024, "shared memory");
+  // scratch of the end-of-piece merge lives in the operand tiles (idle by then)
+  static constexpr int kMergeStride = 129;                     // floats per column (odd: no bank conflicts)
+  static_assert(kColsPad * kMergeStride * 4 + 3 * 256 * 4 <= 4 * kTileBytes, "merge scratch");
+};
+
+// ---- tcgen05 wrappers -------------------------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] . B[smem]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+// D[tmem] (+)= A[tmem] . B[smem]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+// Shared-memory matrix descriptor, 128-byte swizzle: start address, leading / stride byte
+// offsets (16-byte units), descriptor version 1, layout type 2 (SWIZZLE_128B).
+__device__ __forceinline__ uint64_t tc_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: FP32 accumulate, FP16 A and B, A K-major, M = 128.
+__host__ __device__ constexpr uint32_t tc_idesc(int n, bool b_mn_major) {
+  return (1u << 4) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+template <int N>
+struct TmemRegs;  // loads / stores of N consecutive 32-bit columns of the thread's own lane
+template <>
+struct TmemRegs<8> {
+  static __device__ __forceinline__ void ld(uint32_t a, uint32_t* r) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(a) : "memory");
+  }
+  static __device__ __forceinline__ void st(uint32_t a, const uint32_t* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"r"(a), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+  }
+};
+template <>
+struct TmemRegs<16> {
+  static __device__ __forceinline__ void ld(uint32_t a, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(a) : "memory");
+  }
+  static __device__ __forceinline__ void st(uint32_t a, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(a), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+  }
+};
+template <>
+struct TmemRegs<32> {
+  static __device__ __forceinline__ void ld(uint32_t a, uint32_t* r) {
+    TmemRegs<16>::ld(a, r);
+    TmemRegs<16>::ld(a + 16, r + 16);
+  }
+  static __device__ __forceinline__ void st(uint32_t a, const uint32_t* r) {
+    TmemRegs<16>::st(a, r);
+    TmemRegs<16>::st(a + 16, r + 16);
+  }
+};
+
+// Expand the nibble planes of one tensor of a 64-token raw stage into the FP16 code tile.
+// Thread i of the warpgroup converts the 16-byte chunk i & 3 (32 elements) of rows i >> 2 and
+// (i >> 2) + 32: two 128-bit loads, per word two merges and four expansions, four 128-bit
+// stores at the swizzled chunk positions.
+__device__ __forceinline__ void wide_expand(uint32_t raw_a, uint32_t raw_r, uint32_t tile, int i) {
+  const int cc = i & 3;
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int row = (i >> 2) + 32 * j;
+    const uint4 xa = lds128(raw_a + row * 64 + cc * 16);
+    const uint4 xr = lds128(raw_r + row * 64 + cc * 16);
+    const uint32_t wa[4] = {xa.x, xa.y, xa.z, xa.w}, wr[4] = {xr.x, xr.y, xr.z, xr.w};
+    const uint32_t base = tile + (uint32_t)(cc >> 1) * 8192u + (uint32_t)row * 128u;
+#pragma unroll
+    for (int wd = 0; wd < 4; ++wd) {
+      uint32_t ev, od;
+      merge_codes(wa[wd], wr[wd], ev, od);
+      const uint32_t chunk = (uint32_t)(((cc & 1) * 4 + wd) ^ (row & 7));
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + chunk * 16u),
+                   "r"(ev & 0x00FF00FFu), "r"(prmt(ev, 0u, 0x4341)), "r"(od & 0x00FF00FFu),
+                   "r"(prmt(od, 0u, 0x4341)) : "memory");
+    }
+  }
+}
+
+template <int NCOPY>
+__global__ void __launch_bounds__(288, 1) attn_wide_kernel(const AttnParams p) {
+  using C = WideCfg<NCOPY>;
+  constexpr int NSTAGE = C::kNStage, KT = C::kTok, CP = C::kColsPad;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  const uint32_t sbase = smem_u32(smem);
+  float* scal = reinterpret_cast<float*>(smem + C::kOffScal);
+  float* qs_s = reinterpret_cast<float*>(smem + C::kOffQs);
+  __nv_bfloat16* q_s = reinterpret_cast<__nv_bfloat16*>(smem + C::kOffQ);
+  uint32_t* blk_s = reinterpret_cast<uint32_t*>(smem + C::kOffBlk);
+  int4* info_s = reinterpret_cast<int4*>(smem + C::kOffInfo);
+  Item* items = reinterpret_cast<Item*>(info_s + NSTAGE);
+  int* misc = reinterpret_cast<int*>(smem + C::kOffMisc);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int cta = blockIdx.x;
+  const uint32_t ring_u32 = sbase + C::kOffRing;
+  const uint32_t full0 = sbase + C::kOffBars, empty0 = full0 + NSTAGE * 8;
+  const uint32_t qfull0 = empty0 + NSTAGE * 8, qempty0 = qfull0 + 16;
+  const uint32_t sready0 = qempty0 + 16, odone0 = sready0 + 16;
+  volatile int* abort_word = misc;
+
+  if (tid == 0) {
+    for (int i = 0; i < NSTAGE; ++i) {
+      mbar_init(full0 + i * 8, 1);
+      mbar_init(empty0 + i * 8, 4);  // the four warps of the group that owns the unit
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(qfull0 + i * 8, 1);
+      mbar_init(qempty0 + i * 8, C::kConsWarps);
+      mbar_init(sready0 + i * 8, 1);
+      mbar_init(odone0 + i * 8, 1);
+    }
+    misc[0] = 0; misc[1] = 0; misc[7] = 0; misc[8] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = tid; i < 2 * CP * LYNX_D * 2 / 16; i += C::kThreads)
+    reinterpret_cast<uint4*>(q_s)[i] = make_uint4(0, 0, 0, 0);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+
+  if (warp == C::kConsWarps) {
+    producer_warp<C, true, C::kTW, NSTAGE>(p, lane, ring_u32, full0, empty0, qfull0, qempty0, q_s, blk_s,
+                                           info_s, items, misc, abort_word);
+    return;
+  }
+  __syncthreads();  // (A)
+  const int n_units = misc[7];
+  if (n_units == 0) return;
+
+  // ---- tensor memory: all 512 columns of the SM (one CTA per SM) -------------------------------
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(misc + 8)),
+                 "r"((uint32_t)C::kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  named_bar(1, C::kConsThreads);
+  tc_fence_after();
+  const uint32_t tmem0 = *reinterpret_cast<volatile uint32_t*>(misc + 8);
+  const int wg = warp >> 2, w4 = warp & 3;
+  const int r = tid & 127;                       // row of the M = 128 = TMEM lane
+  const int copy = r / CP, c = r % CP;           // warp-uniform copy
+  const uint32_t lane_sel = (uint32_t)(w4 * 32) << 16;
+  const uint32_t tm_q = tmem0 + C::kTmemQ;
+  const uint32_t tm_s = tmem0 + C::kTmemWg0 + wg * C::kTmemWg + C::kTmemS;
+  const uint32_t tm_p = tmem0 + C::kTmemWg0 + wg * C::kTmemWg + C::kTmemP;
+  const uint32_t tm_o = tmem0 + C::kTmemWg0 + wg * C::kTmemWg + C::kTmemO;
+  {  // P starts as zero: a row only ever writes its own tokens
+    uint32_t z[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) z[i] = 0u;
+    TmemRegs<32>::st(tm_p + lane_sel, z);
+    tc_wait_st();
+  }
+  const uint32_t tile_k = sbase + C::kOffCanon + wg * 2 * C::kTileBytes, tile_v = tile_k + C::kTileBytes;
+  float* my_scal = scal + wg * 512;
+  const float cb = p.sm_log2;
+  constexpr uint32_t kIdescS = tc_idesc(64, false), kIdescO = tc_idesc(128, true);
+
+  int gs_base = 0, ic = 0;
+  uint32_t n_s = 0, n_o = 0;   // commits so far on this group's two MMA barriers
+  bool o_pending = false;      // the last O commit has not been waited for yet
+
+  while (gs_base < n_units) {
+    const int qi = ic & 1;
+    mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
+    const Item item = items[qi];
+    const int len = item.len, n_piece = item.pad0;
+    const int full_lim = p.causal ? len - p.nq + 1 : len;
+    const int lim_c = c < p.ncols ? (p.causal ? len - p.nq + c / p.G + 1 : len) : 0;
+    const __nv_bfloat16* qb = q_s + (size_t)qi * CP * LYNX_D;
+    // ---- the piece's queries: common power-of-two scale, FP16 A operand, sum of q ------------
+    float amax = 0.0f;
+    for (int i = lane; i < CP * (LYNX_D / 8); i += 32) {
+      const uint4 v = reinterpret_cast<const uint4*>(qb)[i];
+      const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        amax = fmaxf(amax, fabsf(__uint_as_float(ww[k] << 16)));
+        amax = fmaxf(amax, fabsf(__uint_as_float(ww[k] & 0xFFFF0000u)));
+      }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, off));
+    int e = 0;  // |q * 2^e| < 2^14: exact in FP16 down to 2^-24 of the largest entry
+    if (amax > 0.0f && amax < INFINITY) e = 13 - (((__float_as_int(amax) >> 23) & 0xFF) - 127);
+    e = max(-100, min(100, e));
+    const float up = __int_as_float((127 + e) << 23), down = __int_as_float((127 - e) << 23);
+    const float ca = p.sm_log2 * down * 16777216.0f;  // undoes 2^e of q and 2^-24 of the K codes
+    {
+      // A operand of Q.K^T in TMEM: lane = row, column j = K positions 2j, 2j+1 (FP16 pairs); this
+      // group writes the half of head_dim it is numbered after (32 columns)
+      const int half = wg;
+      uint32_t h[32];
+#pragma unroll
+      for (int g8 = 0; g8 < 8; ++g8) {
+        h[4 * g8] = h[4 * g8 + 1] = h[4 * g8 + 2] = h[4 * g8 + 3] = 0u;
+        if (c < p.ncols) {
+          const uint4 v = *reinterpret_cast<const uint4*>(qb + c * LYNX_D + 64 * half + 8 * g8);
+          const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+          float f[8];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            f[2 * k] = __uint_as_float(ww[k] << 16) * up;
+            f[2 * k + 1] = __uint_as_float(ww[k] & 0xFFFF0000u) * up;
+          }
+          h[4 * g8] = pack_f16x2(f[0], f[4]); h[4 * g8 + 1] = pack_f16x2(f[2], f[6]);
+          h[4 * g8 + 2] = pack_f16x2(f[1], f[5]); h[4 * g8 + 3] = pack_f16x2(f[3], f[7]);
+        }
+      }
+      TmemRegs<32>::st(tm_q + lane_sel + (uint32_t)half * 32u, h);
+      tc_wait_st();
+      if (tid < CP) {
+        float sum = 0.0f;
+        if (tid < p.ncols) {
+          const uint4* qq = reinterpret_cast<const uint4*>(qb + tid * LYNX_D);
+          for (int i = 0; i < 16; ++i) {
+            const uint4 v = qq[i];
+            const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) sum += __uint_as_float(ww[k] << 16) + __uint_as_float(ww[k] & 0xFFFF0000u);
+          }
+        }
+        qs_s[tid] = sum;
+      }
+    }
+    tc_fence_before();
+    named_bar(1, C::kConsThreads);
+    const float qsum = qs_s[c];
+
+    float m = 0.0f, l = 0.0f, zs = 0.0f, sw = 0.0f, hw = 0.0f;  // m: the running maximum (log2 units)
+    bool fresh = true;
+    int my_units = 0;
+
+    // K side of unit k of this piece: code tile, per-token scalars (set `set`), S = Q . K^T.  The K
+    // tile is free: the previous Q.K^T of this group has been waited for.
+    auto prefetch = [&](int k, int set) {
+      const int gs = gs_base + k;
+      const int slot = gs % NSTAGE;
+      mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
+      const uint32_t st = ring_u32 + slot * C::kStageBytes;
+      wide_expand(st, st + 8192u, tile_k, r);            // KA, KR
+      if (r < 64) {
+        const int unit_t0 = (item.pad1 + k) * C::kST;
+        const float2 km = lds64f(st + 16384u + r * 8), vm = lds64f(st + 16896u + r * 8);
+        const bool in = unit_t0 + r < len;
+        float* sc = my_scal + set * 256;
+        sc[r] = in ? km.x * ca : 0.0f;        // alpha: score per unit of the raw dot product
+        sc[64 + r] = in ? km.y * cb : 0.0f;   // beta: score per unit of sum(q)
+        sc[128 + r] = in ? vm.y : 0.0f;       // zero point of the V row
+        sc[192 + r] = in ? vm.x : 0.0f;       // scale of the V row
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tc_fence_before();
+      named_bar(2 + wg, 128);   // every row has its previous scores in registers: S may be overwritten
+      if (r == 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          tc_mma_ts(tm_s, tm_q + (uint32_t)ks * 8u,
+                    tc_desc(tile_k + (uint32_t)(ks >> 2) * 8192u + (uint32_t)(ks & 3) * 32u, 16u, 1024u), kIdescS,
+                    ks > 0 ? 1u : 0u);
+        tc_commit(sready0 + wg * 8);
+      }
+      ++n_s;
+    };
+    if (wg < n_piece) prefetch(wg, 0);
+
+    for (int k = wg; k < n_piece; k += 2, ++my_units) {
+      const int set = my_units & 1;
+      const int gs = gs_base + k;
+      const int slot = gs % NSTAGE;
+      const int unit_t0 = (item.pad1 + k) * C::kST;
+      const uint32_t scal_u32 = smem_u32(my_scal + set * 256);
+      // the scores of this unit (the only outstanding Q.K^T commit of the group)
+      mbar_wait(sready0 + wg * 8, (n_s - 1) & 1, abort_word);
+      tc_fence_after();
+      float x[KT];
+      {
+        uint32_t raw[KT];
+        TmemRegs<KT>::ld(tm_s + lane_sel + (uint32_t)(copy * KT), raw);
+        tc_wait_ld();
+        const uint64_t qs2 = pk2(qsum, qsum), nm2 = pk2(-m, -m);
+#pragma unroll
+        for (int i = 0; i < KT; i += 2) {
+          const int t = copy * KT + i;
+          uint64_t al2, be2;
+          asm volatile("ld.shared.b64 %0, [%1];" : "=l"(al2) : "r"(scal_u32 + t * 4));
+          asm volatile("ld.shared.b64 %0, [%1];" : "=l"(be2) : "r"(scal_u32 + 256 + t * 4));
+          const uint64_t s2 = pk2(__uint_as_float(raw[i]), __uint_as_float(raw[i + 1]));
+          upk2(ffma2(al2, s2, ffma2(be2, qs2, nm2)), x[i], x[i + 1]);
+        }
+      }
+      // the next unit's K side runs on the tensor core while this unit's softmax is computed
+      if (k + 2 < n_piece) prefetch(k + 2, set ^ 1);
+      // ---- softmax of this row's tokens ----------------------------------------------------------
+      const int tok0 = unit_t0 + copy * KT;
+      if (unit_t0 + C::kST > full_lim) {
+#pragma unroll
+        for (int i = 0; i < KT; ++i)
+          if (tok0 + i >= lim_c) x[i] = -INFINITY;
+      }
+      float mx = x[0];
+#pragma unroll
+      for (int i = 1; i < KT; ++i) mx = fmaxf(mx, x[i]);
+      const bool grow = fresh || mx > 4.0f;
+      if (__any_sync(0xFFFFFFFFu, grow)) {
+        float up = 0.0f, f = 1.0f;
+        if (grow) {
+          up = fresh ? fmaxf(mx, -1.0e4f) : fmaxf(mx, 0.0f);
+          f = fresh ? 0.0f : ex2(-up);
+          m += up;
+          l *= f; zs *= f; sw *= f; hw *= f;
+#pragma unroll
+          for (int i = 0; i < KT; ++i) x[i] -= up;
+        }
+        if (my_units > 0) {  // O holds earlier units of this piece: rescale the row in TMEM
+          if (o_pending) {
+            mbar_wait(odone0 + wg * 8, (n_o - 1) & 1, abort_word);
+            o_pending = false;
+          }
+          tc_fence_after();
+#pragma unroll
+          for (int cch = 0; cch < 4; ++cch) {
+            uint32_t o[32];
+            TmemRegs<32>::ld(tm_o + lane_sel + cch * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+            TmemRegs<32>::st(tm_o + lane_sel + cch * 32, o);
+          }
+        }
+      }
+      fresh = false;
+      {
+        uint32_t ph[KT / 2];
+        uint64_t l2 = pk2(l, 0.0f), z2 = pk2(zs, 0.0f), s2 = pk2(sw, 0.0f), h2 = pk2(hw, 0.0f);
+#pragma unroll
+        for (int i = 0; i < KT; i += 2) {
+          const int t = copy * KT + i;
+          uint64_t zz2, sv2;
+          asm volatile("ld.shared.b64 %0, [%1];" : "=l"(zz2) : "r"(scal_u32 + 512 + t * 4));
+          asm volatile("ld.shared.b64 %0, [%1];" : "=l"(sv2) : "r"(scal_u32 + 768 + t * 4));
+          const uint64_t p2 = pk2(ex2(x[i]), ex2(x[i + 1]));
+          l2 = fadd2(l2, p2);
+          z2 = ffma2(p2, zz2, z2);
+          const uint64_t w2 = fmul2(p2, sv2);
+          s2 = fadd2(s2, w2);
+          float w0, w1, b0, b1;
+          upk2(w2, w0, w1);
+          const uint32_t hh = pack_f16x2(w0, w1);
+          ph[i / 2] = hh;
+          b0 = __half2float(__ushort_as_half((unsigned short)(hh & 0xFFFFu)));
+          b1 = __half2float(__ushort_as_half((unsigned short)(hh >> 16)));
+          h2 = fadd2(h2, pk2(b0, b1));
+        }
+        float a0, a1;
+        upk2(l2, a0, a1); l = a0 + a1;
+        upk2(z2, a0, a1); zs = a0 + a1;
+        upk2(s2, a0, a1); sw = a0 + a1;
+        upk2(h2, a0, a1); hw = a0 + a1;
+        // P and the V tile are free once the previous P.V of this group is complete
+        if (o_pending) {
+          mbar_wait(odone0 + wg * 8, (n_o - 1) & 1, abort_word);
+          o_pending = false;
+        }
+        tc_fence_after();
+        TmemRegs<KT / 2>::st(tm_p + lane_sel + (uint32_t)(copy * (KT / 2)), ph);
+      }
+      // ---- V side: code tile, then O += P . V ------------------------------------------------------
+      {
+        const uint32_t st = ring_u32 + slot * C::kStageBytes;
+        wide_expand(st + 4096u, st + 12288u, tile_v, r);   // VA, VR
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + slot * 8);
+      tc_wait_st();
+      tc_fence_before();
+      named_bar(2 + wg, 128);
+      if (r == 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          tc_mma_ts(tm_o, tm_p + (uint32_t)ks * 8u, tc_desc(tile_v + (uint32_t)ks * 2048u, 8192u, 1024u), kIdescO,
+                    (my_units > 0 || ks > 0) ? 1u : 0u);
+        tc_commit(odone0 + wg * 8);
+      }
+      ++n_o;
+      o_pending = true;
+    }
+
+    // ---- end of the piece: merge the 2 * NCOPY partial rows of every column ----------------------
+    if (o_pending) {
+      mbar_wait(odone0 + wg * 8, (n_o - 1) & 1, abort_word);
+      o_pending = false;
+    }
+    tc_fence_after();
+    float* msc = reinterpret_cast<float*>(smem + C::kOffCanon);        // [CP][kMergeStride]
+    float* sc_m = msc + CP * C::kMergeStride;                          // [256] maxima, then [256] l, [256] zs
+    float* sc_l = sc_m + 256;
+    float* sc_z = sc_l + 256;
+    const bool have = my_units > 0;
+    named_bar(1, C::kConsThreads);  // both groups are done with the operand tiles the scratch overlays
+    sc_m[tid] = have ? m : -INFINITY;
+    named_bar(1, C::kConsThreads);
+    float M = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 2 * NCOPY; ++i) M = fmaxf(M, sc_m[(i / NCOPY) * 128 + (i % NCOPY) * CP + c]);
+    const float f = (have && m > -INFINITY && M > -INFINITY) ? ex2(m - M) : 0.0f;
+    sc_l[tid] = l * f;
+    sc_z[tid] = zs * f;
+    // undo the 2^-24 of the V codes and apply the exact-to-rounded weight ratio of this row
+    const float coef = f * 16777216.0f * (hw > 0.0f ? sw / hw : 1.0f);
+    const int part = wg * NCOPY + copy;
+    for (int round = 0; round < 2 * NCOPY; ++round) {
+      if (part == round && have) {   // warp-uniform
+#pragma unroll
+        for (int cch = 0; cch < 4; ++cch) {
+          uint32_t o[32];
+          TmemRegs<32>::ld(tm_o + lane_sel + cch * 32, o);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int d = cch * 32 + (i & ~7) + wide_perm(i & 7);   // logical head dim of column i
+            float* dst = msc + c * C::kMergeStride + d;
+            const float v = coef * __uint_as_float(o[i]);
+            *dst = round == 0 ? v : *dst + v;
+          }
+        }
+      } else if (round == 0 && part == 0) {  // group 0 had no unit: cannot happen (k starts at wg = 0)
+#pragma unroll 4
+        for (int d = 0; d < LYNX_D; ++d) msc[c * C::kMergeStride + d] = 0.0f;
+      }
+      named_bar(1, C::kConsThreads);
+    }
+    const bool direct = item.n_contrib == 1;
+    {
+      const size_t bh = (size_t)item.b * p.Hkv + item.hkv;
+      float* part_dst = p.ws_part + (bh + (size_t)cta) * (size_t)CP * kPartStride;
+      for (int idx = tid; idx < p.ncols * LYNX_D; idx += C::kConsThreads) {
+        const int cc = idx >> 7, d = idx & 127;
+        float lt = 0.0f, z = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 2 * NCOPY; ++i) {
+          lt += sc_l[(i / NCOPY) * 128 + (i % NCOPY) * CP + cc];
+          z += sc_z[(i / NCOPY) * 128 + (i % NCOPY) * CP + cc];
+        }
+        const float v = msc[cc * C::kMergeStride + d] + z;
+        if (direct) {
+          const int j = cc / p.G, hh = cc % p.G;
+          p.out[(((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + d] =
+              lt > 0.0f ? v / lt : 0.0f;
+        } else {
+          part_dst[(size_t)cc * kPartStride + d] = v;
+          if (d == 0) {
+            float Mc = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 2 * NCOPY; ++i) Mc = fmaxf(Mc, sc_m[(i / NCOPY) * 128 + (i % NCOPY) * CP + cc]);
+            part_dst[(size_t)cc * kPartStride + 128] = Mc > -INFINITY ? Mc : -1.0e30f;
+            part_dst[(size_t)cc * kPartStride + 129] = lt;
+          }
+        }
+      }
+      __threadfence();
+    }
+    finish_piece<true, CP, C::kConsThreads>(p, item, direct, tid, misc);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(qempty0 + qi * 8);
+    gs_base += n_piece;
+    ++ic;
+  }
+  // ---- release the tensor memory ---------------------------------------------------------------
+  tc_fence_before();
+  named_bar(1, C::kConsThreads);
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem0), "r"((uint32_t)C::kTmemCols)
+                 : "memory");
+  }
+  if (tid == 0 && misc[0]) atomicOr(p.ws_flags, kFlagTimeout);
+}
+
+template <int NCOPY>
+lynx_status launch_wide(const AttnParams& p, cudaStream_t st) {
+  using C = WideCfg<NCOPY>;
+  auto kern = attn_wide_kernel<NCOPY>;
+  static bool configured[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmem) != cudaSuccess)
+      return LYNX_ERR_CUDA;
+    configured[dev] = true;
+  }
+  const long long cap_units = (long long)p.B * p.Hkv * (((long long)p.max_blocks * p.bt + C::kST - 1) / C::kST);
+  long long grid = (cap_units + 7) / 8;
+  const long long full = sm_count();   // one CTA per SM: it owns all of the SM's tensor memory
+  grid = grid < 1 ? 1 : (grid > full ? full : grid);
+  kern<<<(unsigned)grid, C::kThreads, C::kSmem, st>>>(p);
+  return launch_status();
+}
