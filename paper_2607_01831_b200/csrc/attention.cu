@@ -82,6 +82,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 // One probe of the barrier.  The hint lets the hardware park the thread (up to ~20 us here)
 // until the phase completes instead of returning at once, so a waiting warp does not burn
 // issue slots on polling; completion wakes it early.
+#ifndef LYNX_MBAR_HINT_NS
+#define LYNX_MBAR_HINT_NS 20000
+#endif
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -89,7 +92,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(20000u)
+      : "r"(bar), "r"(parity), "r"((uint32_t)LYNX_MBAR_HINT_NS)
       : "memory");
   return ok != 0;
 }
@@ -1148,7 +1151,7 @@ attn_team_kernel(const AttnParams p) {
   attn_team_body<FULL, NT, DS, TEAMS, NSTAGE>(p);
 }
 #ifndef LYNX_WIDE_VERIFY
-#define LYNX_WIDE_VERIFY 1   // 0: keep the mma.sync kernels for 17..64 verify columns (comparison builds)
+#define LYNX_WIDE_VERIFY 2   // 0: keep the mma.sync kernels for 17..64 verify columns (comparison builds)
 #endif
 #include "attention_wide.cuh"
 

@@ -42,7 +42,8 @@ struct WideCfg {
   static constexpr int kTok = kST / NCOPY;       // tokens of a unit that one row owns
   static constexpr int kConsWarps = 8;
   static constexpr int kConsThreads = 256;
-  static constexpr int kThreads = 288;
+  static constexpr int kProdWarps = 4;           // producer warp i streams 16-token sub-block i of every unit
+  static constexpr int kThreads = (kConsWarps + kProdWarps) * 32;
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int kTileBytes = 2 * 64 * 128;              // [2 dim blocks][64 tokens][128 B]
   static constexpr int kOffCanon = 0;                          // [wg][K tile, V tile]
@@ -51,7 +52,7 @@ struct WideCfg {
   static constexpr int kOffQs = kOffScal + 2 * 2 * 4 * 64 * 4;       // sum of q per column
   static constexpr int kOffQ = kOffQs + kColsPad * 4;                // raw BF16 queries, 2 slots
   static constexpr int kOffBlk = kOffQ + 2 * kColsPad * LYNX_D * 2;
-  static constexpr int kOffInfo = kOffBlk + kPieceUnits * kTW * 4;
+  static constexpr int kOffInfo = kOffBlk + kProdWarps * kPieceUnits * 4;
   static constexpr int kOffBars = kOffInfo + kNStage * 16 + 2 * 32;
   static constexpr int kOffMisc = kOffBars + (2 * kNStage + 8) * 8;  // full, empty, qfull/qempty, sready, odone
   static constexpr int kSmem = kOffMisc + 256 + 1024;                // + alignment slack
@@ -169,8 +170,166 @@ __device__ __forceinline__ void wide_expand(uint32_t raw_a, uint32_t raw_r, uint
   }
 }
 
+// One of the four producer warps of the wide kernel: the stream-K bookkeeping of producer_warp
+// (every warp derives the same range and pieces; warp 0 alone publishes them, loads the queries
+// and handles empty sequences), and per unit the six plane arrays of 16-token sub-block `pw`.
+// One warp issuing all 24 copies of a unit sustains only about 2.7 TB/s over the GPU; four warps
+// with six copies each lift that limit.
+template <class C>
+__device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int lane, uint32_t ring_u32,
+                                              uint32_t full0, uint32_t empty0, uint32_t qfull0, uint32_t qempty0,
+                                              __nv_bfloat16* q_s, uint32_t* blk_s, Item* items, int* misc,
+                                              volatile int* abort_word) {
+  constexpr int ST = C::kST, NSTAGE = C::kNStage;
+  const int n_cta = gridDim.x, cta = blockIdx.x;
+  const int cap = p.max_blocks * p.bt;
+  auto clamp_len = [&](int b) {
+    int len = __ldg(p.seq_lens + b);
+    return len < 0 ? 0 : (len > cap ? cap : len);
+  };
+  long long tot = 0;
+  for (int b = lane; b < p.B; b += 32) tot += (clamp_len(b) + ST - 1) / ST;
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) tot += __shfl_xor_sync(0xFFFFFFFFu, tot, off);
+  const long long T = tot * p.Hkv;
+  const long long q = (T + n_cta - 1) / n_cta;
+  const long long lo = (long long)cta * q, hi = (lo + q < T) ? lo + q : T;
+  int b_lo = 0;
+  long long off_lo = 0;
+  if (lo < hi) {
+    long long running = 0;
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+      const int b = b0 + lane;
+      const long long u = b < p.B ? (long long)p.Hkv * ((clamp_len(b) + ST - 1) / ST) : 0;
+      long long incl = u;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const long long v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      const long long excl = running + incl - u;
+      const bool hit = u > 0 && lo >= excl && lo < excl + u;
+      const unsigned mk = __ballot_sync(0xFFFFFFFFu, hit);
+      if (mk) {
+        const int src = __ffs(mk) - 1;
+        b_lo = b0 + src;
+        off_lo = lo - __shfl_sync(0xFFFFFFFFu, excl, src);
+        break;
+      }
+      running += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+  }
+  if (pw == 0) {
+    if (lane == 0) misc[7] = lo < hi ? (int)(hi - lo) : 0;
+    // sequences with no token: outputs are zero, nothing is rejected unless the draft is not zero
+    for (int b = cta; b < p.B; b += n_cta) {
+      if (clamp_len(b) != 0) continue;
+      const size_t n = (size_t)p.nq * p.Hq * LYNX_D;
+      for (size_t i = lane; i < n; i += 32) p.out[(size_t)b * n + i] = 0.0f;
+      if (p.draft != nullptr) {
+        int fr = p.nq;
+        for (int j = p.nq - 1; j >= 0; --j) {
+          float worst = 0.0f;
+          for (int i = lane; i < p.Hq * LYNX_D; i += 32)
+            worst = fmaxf(worst, fabsf(__ldg(p.draft + ((size_t)b * p.nq + j) * p.Hq * LYNX_D + i)) / p.atol);
+#pragma unroll
+          for (int off = 16; off >= 1; off >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xFFFFFFFFu, worst, off));
+          if (lane == 0) p.dev[(size_t)b * p.nq + j] = worst;
+          if (worst > 1.0f) fr = j;
+        }
+        if (lane == 0) p.first_reject[b] = fr;
+      }
+    }
+  }
+  __syncthreads();  // (A) the range is published
+  const int n_units = (int)(lo < hi ? hi - lo : 0);
+  if (n_units == 0) return;
+
+  // lane a < 6 copies array a of the warp's sub-block: K anchor, V anchor, K meta, V meta, K residual, V residual
+  const bool is_meta = lane == 2 || lane == 3;
+  const unsigned char* my_src = lane == 0 ? p.ka : lane == 1 ? p.va
+                              : lane == 2 ? reinterpret_cast<const unsigned char*>(p.km)
+                              : lane == 3 ? reinterpret_cast<const unsigned char*>(p.vm)
+                              : lane == 4 ? p.kr : p.vr;
+  const uint32_t my_bytes = is_meta ? 128u : 1024u, my_mul = is_meta ? 8u : 64u;
+  const uint32_t my_dst = (lane == 0 ? 0u : lane == 1 ? ST * 64u : lane == 2 ? ST * 256u : lane == 3 ? ST * 264u
+                           : lane == 4 ? ST * 128u : ST * 192u) + (uint32_t)pw * my_bytes;
+  uint32_t* my_blk = blk_s + pw * kPieceUnits;
+  int b = b_lo, len = clamp_len(b), U = (len + ST - 1) / ST;
+  int hkv = (int)(off_lo / U), u = (int)(off_lo % U);
+  int remaining = n_units, gs = 0, ic = 0;
+  while (remaining > 0) {
+    const int n = min(remaining, U - u);
+    const int qi = ic & 1;
+    if (pw == 0) {
+      if (ic >= 2) mbar_wait(qempty0 + qi * 8, ((ic >> 1) - 1) & 1, abort_word);
+      const long long seg0 = lo + (n_units - remaining) - u;  // first unit of this segment
+      if (lane == 0) {
+        Item it;
+        it.b = b; it.hkv = hkv; it.len = len;
+        it.first_cta = (int)(seg0 / q);
+        it.n_contrib = (int)((seg0 + U - 1) / q) - it.first_cta + 1;
+        it.pad0 = n; it.pad1 = u; it.pad2 = 0;
+        items[qi] = it;
+        mbar_expect_tx(qfull0 + qi * 8, (uint32_t)(p.nq * p.G * LYNX_D * 2));
+      }
+      __syncwarp();
+      for (int j = lane; j < p.nq; j += 32)
+        bulk_g2s(smem_u32(q_s + ((size_t)qi * C::kColsPad + j * p.G) * LYNX_D),
+                 p.q + (((size_t)b * p.nq + j) * p.Hq + (size_t)hkv * p.G) * LYNX_D,
+                 (uint32_t)(p.G * LYNX_D * 2), qfull0 + qi * 8);
+    }
+    for (int c0 = 0; c0 < n; c0 += kPieceUnits) {
+      const int cn = min(kPieceUnits, n - c0);
+      for (int i = lane; i < cn; i += 32) {
+        const int t0 = (u + c0 + i) * ST + pw * 16;
+        uint32_t row = 0xFFFFFFFFu;  // sub-block beyond the end of the sequence: nothing to copy
+        if (t0 < len) {
+          int blk = __ldg(p.block_table + (size_t)b * p.max_blocks + t0 / p.bt);
+          if (blk < 0 || blk >= p.num_blocks) {
+            atomicOr(p.ws_flags, kFlagBadBlock);
+            blk = blk < 0 ? 0 : p.num_blocks - 1;
+          }
+          row = (uint32_t)(((size_t)blk * p.Hkv + hkv) * p.bt + (t0 % p.bt));
+        }
+        my_blk[i] = row;
+      }
+      __syncwarp();
+      for (int k = 0; k < cn; ++k, ++gs) {
+        const int slot = gs % NSTAGE;
+        if (gs >= NSTAGE) mbar_wait(empty0 + slot * 8, ((gs / NSTAGE) - 1) & 1, abort_word);
+        const uint32_t row = my_blk[k];
+        const uint32_t bar = full0 + slot * 8;
+        if (lane == 0) {
+          if (row != 0xFFFFFFFFu) mbar_expect_tx(bar, (uint32_t)C::kSubBytes);
+          else mbar_arrive(bar);
+        }
+        __syncwarp();
+        if (lane < 6 && row != 0xFFFFFFFFu)
+          bulk_g2s(ring_u32 + slot * C::kStageBytes + my_dst, my_src + (size_t)row * my_mul, my_bytes, bar);
+      }
+      __syncwarp();  // my_blk is rewritten by the next round
+    }
+    remaining -= n;
+    u += n;
+    ++ic;
+    if (u == U && remaining > 0) {
+      u = 0;
+      if (++hkv == p.Hkv) {
+        hkv = 0;
+        do {
+          ++b;
+          len = b < p.B ? clamp_len(b) : 0;
+          U = (len + ST - 1) / ST;
+        } while (b < p.B && U == 0);
+        if (b >= p.B) break;  // cannot happen: the range ends inside the list
+      }
+    }
+  }
+}
+
 template <int NCOPY>
-__global__ void __launch_bounds__(288, 1) attn_wide_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(const AttnParams p) {
   using C = WideCfg<NCOPY>;
   constexpr int NSTAGE = C::kNStage, KT = C::kTok, CP = C::kColsPad;
   extern __shared__ unsigned char smem_raw[];
@@ -193,7 +352,7 @@ __global__ void __launch_bounds__(288, 1) attn_wide_kernel(const AttnParams p) {
 
   if (tid == 0) {
     for (int i = 0; i < NSTAGE; ++i) {
-      mbar_init(full0 + i * 8, 1);
+      mbar_init(full0 + i * 8, C::kProdWarps);
       mbar_init(empty0 + i * 8, 4);  // the four warps of the group that owns the unit
     }
     for (int i = 0; i < 2; ++i) {
@@ -210,9 +369,9 @@ __global__ void __launch_bounds__(288, 1) attn_wide_kernel(const AttnParams p) {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
 
-  if (warp == C::kConsWarps) {
-    producer_warp<C, true, C::kTW, NSTAGE>(p, lane, ring_u32, full0, empty0, qfull0, qempty0, q_s, blk_s,
-                                           info_s, items, misc, abort_word);
+  if (warp >= C::kConsWarps) {
+    wide_producer<C>(p, warp - C::kConsWarps, lane, ring_u32, full0, empty0, qfull0, qempty0, q_s, blk_s, items,
+                     misc, abort_word);
     return;
   }
   __syncthreads();  // (A)
@@ -336,11 +495,12 @@ __global__ void __launch_bounds__(288, 1) attn_wide_kernel(const AttnParams p) {
         const int unit_t0 = (item.pad1 + k) * C::kST;
         const float2 km = lds64f(st + 16384u + r * 8), vm = lds64f(st + 16896u + r * 8);
         const bool in = unit_t0 + r < len;
-        float* sc = my_scal + set * 256;
-        sc[r] = in ? km.x * ca : 0.0f;        // alpha: score per unit of the raw dot product
-        sc[64 + r] = in ? km.y * cb : 0.0f;   // beta: score per unit of sum(q)
-        sc[128 + r] = in ? vm.y : 0.0f;       // zero point of the V row
-        sc[192 + r] = in ? vm.x : 0.0f;       // scale of the V row
+        // [pair][alpha0, alpha1, beta0, beta1] and [pair][zero0, zero1, scale0, scale1]
+        float* sc = my_scal + set * 256 + (r >> 1) * 4 + (r & 1);
+        sc[0] = in ? km.x * ca : 0.0f;     // alpha: score per unit of the raw dot product
+        sc[2] = in ? km.y * cb : 0.0f;     // beta: score per unit of sum(q)
+        sc[128] = in ? vm.y : 0.0f;        // zero point of the V row
+        sc[130] = in ? vm.x : 0.0f;        // scale of the V row
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
@@ -375,12 +535,10 @@ __global__ void __launch_bounds__(288, 1) attn_wide_kernel(const AttnParams p) {
         const uint64_t qs2 = pk2(qsum, qsum), nm2 = pk2(-m, -m);
 #pragma unroll
         for (int i = 0; i < KT; i += 2) {
-          const int t = copy * KT + i;
-          uint64_t al2, be2;
-          asm volatile("ld.shared.b64 %0, [%1];" : "=l"(al2) : "r"(scal_u32 + t * 4));
-          asm volatile("ld.shared.b64 %0, [%1];" : "=l"(be2) : "r"(scal_u32 + 256 + t * 4));
+          const uint4 ab = lds128(scal_u32 + (uint32_t)(copy * KT + i) * 8u);  // alpha0, alpha1, beta0, beta1
           const uint64_t s2 = pk2(__uint_as_float(raw[i]), __uint_as_float(raw[i + 1]));
-          upk2(ffma2(al2, s2, ffma2(be2, qs2, nm2)), x[i], x[i + 1]);
+          upk2(ffma2(pk2(__uint_as_float(ab.x), __uint_as_float(ab.y)), s2,
+                     ffma2(pk2(__uint_as_float(ab.z), __uint_as_float(ab.w)), qs2, nm2)), x[i], x[i + 1]);
         }
       }
       // the next unit's K side runs on the tensor core while this unit's softmax is computed
@@ -392,20 +550,50 @@ __global__ void __launch_bounds__(288, 1) attn_wide_kernel(const AttnParams p) {
         for (int i = 0; i < KT; ++i)
           if (tok0 + i >= lim_c) x[i] = -INFINITY;
       }
-      float mx = x[0];
+      // ---- weights: fast path without the maximum; redone when a weight may have grown too large -----
+      uint32_t ph[KT / 2];
+      float l_n, zs_n, sw_n, hw_n;
+      auto weights = [&]() {
+        uint64_t l2 = pk2(l, 0.0f), z2 = pk2(zs, 0.0f), s2 = pk2(sw, 0.0f), h2 = pk2(hw, 0.0f);
 #pragma unroll
-      for (int i = 1; i < KT; ++i) mx = fmaxf(mx, x[i]);
-      const bool grow = fresh || mx > 4.0f;
+        for (int i = 0; i < KT; i += 2) {
+          const uint4 zv = lds128(scal_u32 + 512u + (uint32_t)(copy * KT + i) * 8u);  // zero0, zero1, scale0, scale1
+          const uint64_t p2 = pk2(ex2(x[i]), ex2(x[i + 1]));
+          l2 = fadd2(l2, p2);
+          z2 = ffma2(p2, pk2(__uint_as_float(zv.x), __uint_as_float(zv.y)), z2);
+          const uint64_t w2 = fmul2(p2, pk2(__uint_as_float(zv.z), __uint_as_float(zv.w)));
+          s2 = fadd2(s2, w2);
+          float w0, w1, b0, b1;
+          upk2(w2, w0, w1);
+          const uint32_t hh = pack_f16x2(w0, w1);
+          ph[i / 2] = hh;
+          asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tcvt.f32.f16 %0, lo;\n\tcvt.f32.f16 %1, hi;\n\t}"
+              : "=f"(b0), "=f"(b1) : "r"(hh));
+          h2 = fadd2(h2, pk2(b0, b1));
+        }
+        float a0, a1;
+        upk2(l2, a0, a1); l_n = a0 + a1;
+        upk2(z2, a0, a1); zs_n = a0 + a1;
+        upk2(s2, a0, a1); sw_n = a0 + a1;
+        upk2(h2, a0, a1); hw_n = a0 + a1;
+      };
+      weights();
+      // every weight of the unit is below 64 unless the unit's sum says otherwise
+      const bool grow = fresh || !(l_n - l <= 64.0f);
       if (__any_sync(0xFFFFFFFFu, grow)) {
-        float up = 0.0f, f = 1.0f;
+        float f = 1.0f;
         if (grow) {
-          up = fresh ? fmaxf(mx, -1.0e4f) : fmaxf(mx, 0.0f);
-          f = fresh ? 0.0f : ex2(-up);
-          m += up;
+          float mx = x[0];
+#pragma unroll
+          for (int i = 1; i < KT; ++i) mx = fmaxf(mx, x[i]);
+          const float upm = fresh ? fmaxf(mx, -1.0e4f) : fmaxf(mx, 0.0f);
+          f = fresh ? 0.0f : ex2(-upm);
+          m += upm;
           l *= f; zs *= f; sw *= f; hw *= f;
 #pragma unroll
-          for (int i = 0; i < KT; ++i) x[i] -= up;
+          for (int i = 0; i < KT; ++i) x[i] -= upm;
         }
+        weights();
         if (my_units > 0) {  // O holds earlier units of this piece: rescale the row in TMEM
           if (o_pending) {
             mbar_wait(odone0 + wg * 8, (n_o - 1) & 1, abort_word);
@@ -424,33 +612,8 @@ __global__ void __launch_bounds__(288, 1) attn_wide_kernel(const AttnParams p) {
         }
       }
       fresh = false;
+      l = l_n; zs = zs_n; sw = sw_n; hw = hw_n;
       {
-        uint32_t ph[KT / 2];
-        uint64_t l2 = pk2(l, 0.0f), z2 = pk2(zs, 0.0f), s2 = pk2(sw, 0.0f), h2 = pk2(hw, 0.0f);
-#pragma unroll
-        for (int i = 0; i < KT; i += 2) {
-          const int t = copy * KT + i;
-          uint64_t zz2, sv2;
-          asm volatile("ld.shared.b64 %0, [%1];" : "=l"(zz2) : "r"(scal_u32 + 512 + t * 4));
-          asm volatile("ld.shared.b64 %0, [%1];" : "=l"(sv2) : "r"(scal_u32 + 768 + t * 4));
-          const uint64_t p2 = pk2(ex2(x[i]), ex2(x[i + 1]));
-          l2 = fadd2(l2, p2);
-          z2 = ffma2(p2, zz2, z2);
-          const uint64_t w2 = fmul2(p2, sv2);
-          s2 = fadd2(s2, w2);
-          float w0, w1, b0, b1;
-          upk2(w2, w0, w1);
-          const uint32_t hh = pack_f16x2(w0, w1);
-          ph[i / 2] = hh;
-          b0 = __half2float(__ushort_as_half((unsigned short)(hh & 0xFFFFu)));
-          b1 = __half2float(__ushort_as_half((unsigned short)(hh >> 16)));
-          h2 = fadd2(h2, pk2(b0, b1));
-        }
-        float a0, a1;
-        upk2(l2, a0, a1); l = a0 + a1;
-        upk2(z2, a0, a1); zs = a0 + a1;
-        upk2(s2, a0, a1); sw = a0 + a1;
-        upk2(h2, a0, a1); hw = a0 + a1;
         // P and the V tile are free once the previous P.V of this group is complete
         if (o_pending) {
           mbar_wait(odone0 + wg * 8, (n_o - 1) & 1, abort_word);
