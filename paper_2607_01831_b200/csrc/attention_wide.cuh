@@ -42,19 +42,20 @@ struct WideCfg {
   static constexpr int kTok = kST / NCOPY;       // tokens of a unit that one row owns
   static constexpr int kConsWarps = 8;
   static constexpr int kConsThreads = 256;
-  static constexpr int kProdWarps = 4;           // producer warp i streams 16-token sub-block i of every unit
-  static constexpr int kThreads = (kConsWarps + kProdWarps) * 32;
+  static constexpr int kProdWarps = 3;           // each issues 8 of the 24 plane copies of a unit
+  static constexpr int kMmaWarp = kConsWarps + kProdWarps;   // one thread of it issues every tcgen05.mma
+  static constexpr int kThreads = (kConsWarps + kProdWarps + 1) * 32;
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int kTileBytes = 2 * 64 * 128;              // [2 dim blocks][64 tokens][128 B]
   static constexpr int kOffCanon = 0;                          // [wg][K tile, V tile]
   static constexpr int kOffRing = 4 * kTileBytes;
-  static constexpr int kOffScal = kOffRing + kNStage * kStageBytes;  // [wg][set][alpha, beta, zz, sv][64]
-  static constexpr int kOffQs = kOffScal + 2 * 2 * 4 * 64 * 4;       // sum of q per column
+  static constexpr int kOffScal = kOffRing + kNStage * kStageBytes;  // [group][3 sets][256 floats]
+  static constexpr int kOffQs = kOffScal + 2 * 3 * 4 * 64 * 4;       // sum of q per column
   static constexpr int kOffQ = kOffQs + kColsPad * 4;                // raw BF16 queries, 2 slots
   static constexpr int kOffBlk = kOffQ + 2 * kColsPad * LYNX_D * 2;
-  static constexpr int kOffInfo = kOffBlk + kProdWarps * kPieceUnits * 4;
+  static constexpr int kOffInfo = kOffBlk + kProdWarps * 2 * kPieceUnits * 4;
   static constexpr int kOffBars = kOffInfo + kNStage * 16 + 2 * 32;
-  static constexpr int kOffMisc = kOffBars + (2 * kNStage + 8) * 8;  // full, empty, qfull/qempty, sready, odone
+  static constexpr int kOffMisc = kOffBars + (2 * kNStage + 12) * 8;  // full, empty, q full/empty, sready, odone, kready, pready
   static constexpr int kSmem = kOffMisc + 256 + 1024;                // + alignment slack
   // TMEM columns of a warpgroup
   static constexpr int kTmemQ = 0, kTmemWg0 = 64, kTmemS = 0, kTmemP = 64, kTmemO = 96, kTmemWg = 224, kTmemCols = 512;
@@ -65,6 +66,17 @@ struct WideCfg {
   static constexpr int kMergeStride = 129;                     // floats per column (odd: no bank conflicts)
   static_assert(kColsPad * kMergeStride * 4 + 3 * 256 * 4 <= 4 * kTileBytes, "merge scratch");
 };
+
+// One non-blocking probe of an mbarrier phase.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
 
 // ---- tcgen05 wrappers -------------------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -245,16 +257,28 @@ __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int l
   const int n_units = (int)(lo < hi ? hi - lo : 0);
   if (n_units == 0) return;
 
-  // lane a < 6 copies array a of the warp's sub-block: K anchor, V anchor, K meta, V meta, K residual, V residual
-  const bool is_meta = lane == 2 || lane == 3;
-  const unsigned char* my_src = lane == 0 ? p.ka : lane == 1 ? p.va
-                              : lane == 2 ? reinterpret_cast<const unsigned char*>(p.km)
-                              : lane == 3 ? reinterpret_cast<const unsigned char*>(p.vm)
-                              : lane == 4 ? p.kr : p.vr;
+  // role = (sub-block, array) of a unit's 24 copies; arrays: K anchor, V anchor, K meta, V meta, K residual,
+  // V residual.  Warp pw has the roles 8 pw .. 8 pw + 7 (lanes 0..7), which lie in two sub-blocks.
+  constexpr int RP = 24 / C::kProdWarps;
+  const int role = pw * RP + (lane < RP ? lane : 0);
+  const int sub = role / 6, arr = role % 6, sub_first = (pw * RP) / 6;
+  const bool is_meta = arr == 2 || arr == 3;
+  const unsigned char* my_src = arr == 0 ? p.ka : arr == 1 ? p.va
+                              : arr == 2 ? reinterpret_cast<const unsigned char*>(p.km)
+                              : arr == 3 ? reinterpret_cast<const unsigned char*>(p.vm)
+                              : arr == 4 ? p.kr : p.vr;
   const uint32_t my_bytes = is_meta ? 128u : 1024u, my_mul = is_meta ? 8u : 64u;
-  const uint32_t my_dst = (lane == 0 ? 0u : lane == 1 ? ST * 64u : lane == 2 ? ST * 256u : lane == 3 ? ST * 264u
-                           : lane == 4 ? ST * 128u : ST * 192u) + (uint32_t)pw * my_bytes;
-  uint32_t* my_blk = blk_s + pw * kPieceUnits;
+  const uint32_t my_dst = (arr == 0 ? 0u : arr == 1 ? ST * 64u : arr == 2 ? ST * 256u : arr == 3 ? ST * 264u
+                           : arr == 4 ? ST * 128u : ST * 192u) + (uint32_t)sub * my_bytes;
+  uint32_t bytes_sub[2];   // bytes this warp copies of its first / second sub-block
+#pragma unroll
+  for (int s2 = 0; s2 < 2; ++s2) {
+    uint32_t v = (lane < RP && sub == sub_first + s2) ? my_bytes : 0u;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+    bytes_sub[s2] = v;
+  }
+  uint32_t* my_blk = blk_s + pw * 2 * kPieceUnits;   // [2 sub-blocks][kPieceUnits]
   int b = b_lo, len = clamp_len(b), U = (len + ST - 1) / ST;
   int hkv = (int)(off_lo / U), u = (int)(off_lo % U);
   int remaining = n_units, gs = 0, ic = 0;
@@ -281,8 +305,9 @@ __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int l
     }
     for (int c0 = 0; c0 < n; c0 += kPieceUnits) {
       const int cn = min(kPieceUnits, n - c0);
-      for (int i = lane; i < cn; i += 32) {
-        const int t0 = (u + c0 + i) * ST + pw * 16;
+      for (int i2 = lane; i2 < 2 * cn; i2 += 32) {
+        const int i = i2 >> 1;
+        const int t0 = (u + c0 + i) * ST + (sub_first + (i2 & 1)) * 16;
         uint32_t row = 0xFFFFFFFFu;  // sub-block beyond the end of the sequence: nothing to copy
         if (t0 < len) {
           int blk = __ldg(p.block_table + (size_t)b * p.max_blocks + t0 / p.bt);
@@ -292,20 +317,22 @@ __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int l
           }
           row = (uint32_t)(((size_t)blk * p.Hkv + hkv) * p.bt + (t0 % p.bt));
         }
-        my_blk[i] = row;
+        my_blk[(i2 & 1) * kPieceUnits + i] = row;
       }
       __syncwarp();
       for (int k = 0; k < cn; ++k, ++gs) {
         const int slot = gs % NSTAGE;
         if (gs >= NSTAGE) mbar_wait(empty0 + slot * 8, ((gs / NSTAGE) - 1) & 1, abort_word);
-        const uint32_t row = my_blk[k];
+        const uint32_t row0 = my_blk[k], row1 = my_blk[kPieceUnits + k];
+        const uint32_t row = sub == sub_first ? row0 : row1;
         const uint32_t bar = full0 + slot * 8;
         if (lane == 0) {
-          if (row != 0xFFFFFFFFu) mbar_expect_tx(bar, (uint32_t)C::kSubBytes);
+          const uint32_t bytes = (row0 != 0xFFFFFFFFu ? bytes_sub[0] : 0u) + (row1 != 0xFFFFFFFFu ? bytes_sub[1] : 0u);
+          if (bytes) mbar_expect_tx(bar, bytes);
           else mbar_arrive(bar);
         }
         __syncwarp();
-        if (lane < 6 && row != 0xFFFFFFFFu)
+        if (lane < RP && row != 0xFFFFFFFFu)
           bulk_g2s(ring_u32 + slot * C::kStageBytes + my_dst, my_src + (size_t)row * my_mul, my_bytes, bar);
       }
       __syncwarp();  // my_blk is rewritten by the next round
@@ -347,7 +374,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
   const uint32_t ring_u32 = sbase + C::kOffRing;
   const uint32_t full0 = sbase + C::kOffBars, empty0 = full0 + NSTAGE * 8;
   const uint32_t qfull0 = empty0 + NSTAGE * 8, qempty0 = qfull0 + 16;
-  const uint32_t sready0 = qempty0 + 16, odone0 = sready0 + 16;
+  const uint32_t sready0 = qempty0 + 16, odone0 = sready0 + 16, kready0 = odone0 + 16, pready0 = kready0 + 16;
   volatile int* abort_word = misc;
 
   if (tid == 0) {
@@ -360,6 +387,8 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       mbar_init(qempty0 + i * 8, C::kConsWarps);
       mbar_init(sready0 + i * 8, 1);
       mbar_init(odone0 + i * 8, 1);
+      mbar_init(kready0 + i * 8, 4);   // K tile and scalars of group i written, its previous scores in registers
+      mbar_init(pready0 + i * 8, 4);   // P and V tile of group i written
     }
     misc[0] = 0; misc[1] = 0; misc[7] = 0; misc[8] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -369,7 +398,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
 
-  if (warp >= C::kConsWarps) {
+  if (warp >= C::kConsWarps && warp < C::kMmaWarp) {
     wide_producer<C>(p, warp - C::kConsWarps, lane, ring_u32, full0, empty0, qfull0, qempty0, q_s, blk_s, items,
                      misc, abort_word);
     return;
@@ -385,9 +414,67 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
-  named_bar(1, C::kConsThreads);
+  named_bar(5, C::kConsThreads + 32);
   tc_fence_after();
   const uint32_t tmem0 = *reinterpret_cast<volatile uint32_t*>(misc + 8);
+  constexpr uint32_t kIdescS = tc_idesc(64, false), kIdescO = tc_idesc(128, true);
+  // =============================================================================================
+  // The MMA warp: one thread issues every tcgen05.mma, so that no softmax warp stalls on the
+  // tensor pipe's queue.  It polls the four "operands ready" barriers and issues what is ready.
+  // =============================================================================================
+  if (warp == C::kMmaWarp) {
+    if (lane == 0) {
+      const uint32_t tm_q = tmem0 + C::kTmemQ;
+      uint32_t gk[2] = {0, 0}, gp[2] = {0, 0};   // Q.K^T / P.V issued so far, per group (barrier phases)
+      int gs_base = 0, ic = 0;
+      while (gs_base < n_units) {
+        const int qi = ic & 1;
+        mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
+        const int n_piece = items[qi].pad0;
+        int todo_k[2] = {(n_piece + 1) >> 1, n_piece >> 1}, todo_p[2] = {(n_piece + 1) >> 1, n_piece >> 1};
+        int first_p[2] = {1, 1};
+        uint64_t t0 = globaltimer_ns();
+        while (todo_k[0] + todo_k[1] + todo_p[0] + todo_p[1] > 0) {
+          bool progress = false;
+#pragma unroll
+          for (int w = 0; w < 2; ++w) {
+            const uint32_t tile_k = sbase + C::kOffCanon + w * 2 * C::kTileBytes, tile_v = tile_k + C::kTileBytes;
+            const uint32_t tm_w = tmem0 + C::kTmemWg0 + w * C::kTmemWg;
+            if (todo_k[w] > 0 && mbar_test(kready0 + w * 8, gk[w] & 1)) {
+              tc_fence_after();
+#pragma unroll
+              for (int ks = 0; ks < 8; ++ks)
+                tc_mma_ts(tm_w + C::kTmemS, tm_q + (uint32_t)ks * 8u,
+                          tc_desc(tile_k + (uint32_t)(ks >> 2) * 8192u + (uint32_t)(ks & 3) * 32u, 16u, 1024u),
+                          kIdescS, ks > 0 ? 1u : 0u);
+              tc_commit(sready0 + w * 8);
+              ++gk[w]; --todo_k[w]; progress = true;
+            }
+            if (todo_p[w] > 0 && mbar_test(pready0 + w * 8, gp[w] & 1)) {
+              tc_fence_after();
+#pragma unroll
+              for (int ks = 0; ks < 4; ++ks)
+                tc_mma_ts(tm_w + C::kTmemO, tm_w + C::kTmemP + (uint32_t)ks * 8u,
+                          tc_desc(tile_v + (uint32_t)ks * 2048u, 8192u, 1024u), kIdescO,
+                          (!first_p[w] || ks > 0) ? 1u : 0u);
+              tc_commit(odone0 + w * 8);
+              first_p[w] = 0;
+              ++gp[w]; --todo_p[w]; progress = true;
+            }
+          }
+          if (progress) {
+            t0 = globaltimer_ns();
+          } else if (*abort_word || globaltimer_ns() - t0 > 2000000000ull) {
+            *abort_word = 1;   // give up: the waiting groups see the abort word and run out their loops
+            break;
+          }
+        }
+        gs_base += n_piece;
+        ++ic;
+      }
+    }
+    return;
+  }
   const int wg = warp >> 2, w4 = warp & 3;
   const int r = tid & 127;                       // row of the M = 128 = TMEM lane
   const int copy = r / CP, c = r % CP;           // warp-uniform copy
@@ -404,11 +491,11 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
     tc_wait_st();
   }
   const uint32_t tile_k = sbase + C::kOffCanon + wg * 2 * C::kTileBytes, tile_v = tile_k + C::kTileBytes;
-  float* my_scal = scal + wg * 512;
+  float* my_scal = scal + wg * 768;
   const float cb = p.sm_log2;
-  constexpr uint32_t kIdescS = tc_idesc(64, false), kIdescO = tc_idesc(128, true);
 
   int gs_base = 0, ic = 0;
+  uint32_t n_u = 0;            // units of this group so far (selects the scalar set)
   uint32_t n_s = 0, n_o = 0;   // commits so far on this group's two MMA barriers
   bool o_pending = false;      // the last O commit has not been waited for yet
 
@@ -504,22 +591,14 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
-      named_bar(2 + wg, 128);   // every row has its previous scores in registers: S may be overwritten
-      if (r == 0) {
-        tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          tc_mma_ts(tm_s, tm_q + (uint32_t)ks * 8u,
-                    tc_desc(tile_k + (uint32_t)(ks >> 2) * 8192u + (uint32_t)(ks & 3) * 32u, 16u, 1024u), kIdescS,
-                    ks > 0 ? 1u : 0u);
-        tc_commit(sready0 + wg * 8);
-      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(kready0 + wg * 8);   // this warp's part of the K side is ready and its S is in registers
       ++n_s;
     };
-    if (wg < n_piece) prefetch(wg, 0);
+    if (wg < n_piece) prefetch(wg, (int)(n_u % 3u));
 
     for (int k = wg; k < n_piece; k += 2, ++my_units) {
-      const int set = my_units & 1;
+      const int set = (int)(n_u % 3u);
       const int gs = gs_base + k;
       const int slot = gs % NSTAGE;
       const int unit_t0 = (item.pad1 + k) * C::kST;
@@ -542,7 +621,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
         }
       }
       // the next unit's K side runs on the tensor core while this unit's softmax is computed
-      if (k + 2 < n_piece) prefetch(k + 2, set ^ 1);
+      if (k + 2 < n_piece) prefetch(k + 2, (set + 1) % 3);
       // ---- softmax of this row's tokens ----------------------------------------------------------
       const int tok0 = unit_t0 + copy * KT;
       if (unit_t0 + C::kST > full_lim) {
@@ -632,15 +711,9 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       if (lane == 0) mbar_arrive(empty0 + slot * 8);
       tc_wait_st();
       tc_fence_before();
-      named_bar(2 + wg, 128);
-      if (r == 0) {
-        tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          tc_mma_ts(tm_o, tm_p + (uint32_t)ks * 8u, tc_desc(tile_v + (uint32_t)ks * 2048u, 8192u, 1024u), kIdescO,
-                    (my_units > 0 || ks > 0) ? 1u : 0u);
-        tc_commit(odone0 + wg * 8);
-      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pready0 + wg * 8);   // this warp's rows of P and part of the V tile are ready
+      ++n_u;
       ++n_o;
       o_pending = true;
     }
