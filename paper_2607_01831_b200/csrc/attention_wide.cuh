@@ -44,7 +44,9 @@ struct WideCfg {
   static constexpr int kConsThreads = 256;
   static constexpr int kProdWarps = 3;           // each issues 8 of the 24 plane copies of a unit
   static constexpr int kMmaWarp = kConsWarps + kProdWarps;   // one thread of it issues every tcgen05.mma
-  static constexpr int kThreads = (kConsWarps + kProdWarps + 1) * 32;
+  static constexpr int kVWarp0 = kMmaWarp + 1;    // warps that expand the V tiles; without them the softmax groups do it
+  static constexpr int kVWarps = NCOPY == 4 ? 4 : 0;   // (16 warps leave 128 registers per thread: too few for 32 tokens per row)
+  static constexpr int kThreads = (kConsWarps + kProdWarps + 1 + kVWarps) * 32;
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int kTileBytes = 2 * 64 * 128;              // [2 dim blocks][64 tokens][128 B]
   static constexpr int kOffCanon = 0;                          // [wg][K tile, V tile]
@@ -162,20 +164,31 @@ struct TmemRegs<32> {
 // (i >> 2) + 32: two 128-bit loads, per word two merges and four expansions, four 128-bit
 // stores at the swizzled chunk positions.
 __device__ __forceinline__ void wide_expand(uint32_t raw_a, uint32_t raw_r, uint32_t tile, int i) {
-  const int cc = i & 3;
+  const int cc = i & 3, row0 = i >> 2;
+  // Threads with cc >= 2 take the two halves of their 16 bytes in the other order (sw = 2): the
+  // four threads of a row then store to four different chunk positions in every store
+  // instruction, which makes the 128-bit stores free of bank conflicts.
+  const uint32_t sw = (uint32_t)(cc & 2);
+  // all loads first: the shared-memory accesses are volatile asm and keep their order
+  uint2 xa[2][2], xr[2][2];
 #pragma unroll
   for (int j = 0; j < 2; ++j) {
-    const int row = (i >> 2) + 32 * j;
-    const uint4 xa = lds128(raw_a + row * 64 + cc * 16);
-    const uint4 xr = lds128(raw_r + row * 64 + cc * 16);
-    const uint32_t wa[4] = {xa.x, xa.y, xa.z, xa.w}, wr[4] = {xr.x, xr.y, xr.z, xr.w};
-    const uint32_t base = tile + (uint32_t)(cc >> 1) * 8192u + (uint32_t)row * 128u;
+    const uint32_t off = (uint32_t)((row0 + 32 * j) * 64 + cc * 16);
+    xa[j][0] = lds64(raw_a + off + sw * 4u); xa[j][1] = lds64(raw_a + off + (sw ^ 2u) * 4u);
+    xr[j][0] = lds64(raw_r + off + sw * 4u); xr[j][1] = lds64(raw_r + off + (sw ^ 2u) * 4u);
+  }
+  // rows row0 and row0 + 32 have the same row & 7: one set of swizzled chunk offsets
+  const uint32_t base = tile + (uint32_t)(cc >> 1) * 8192u + (uint32_t)row0 * 128u;
+  const uint32_t swz = (uint32_t)(((cc & 1) * 4) ^ (row0 & 7) ^ (int)sw) * 16u;
 #pragma unroll
-    for (int wd = 0; wd < 4; ++wd) {
+  for (int j = 0; j < 2; ++j) {
+    const uint32_t wa[4] = {xa[j][0].x, xa[j][0].y, xa[j][1].x, xa[j][1].y};
+    const uint32_t wr[4] = {xr[j][0].x, xr[j][0].y, xr[j][1].x, xr[j][1].y};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {   // register k holds word k ^ sw of the chunk
       uint32_t ev, od;
-      merge_codes(wa[wd], wr[wd], ev, od);
-      const uint32_t chunk = (uint32_t)(((cc & 1) * 4 + wd) ^ (row & 7));
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + chunk * 16u),
+      merge_codes(wa[k], wr[k], ev, od);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + (uint32_t)j * 4096u + (swz ^ (uint32_t)(k * 16))),
                    "r"(ev & 0x00FF00FFu), "r"(prmt(ev, 0u, 0x4341)), "r"(od & 0x00FF00FFu),
                    "r"(prmt(od, 0u, 0x4341)) : "memory");
     }
@@ -380,7 +393,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
   if (tid == 0) {
     for (int i = 0; i < NSTAGE; ++i) {
       mbar_init(full0 + i * 8, C::kProdWarps);
-      mbar_init(empty0 + i * 8, 4);  // the four warps of the group that owns the unit
+      mbar_init(empty0 + i * 8, 4 + C::kVWarps);  // the owning group (K side) and the V converters
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(qfull0 + i * 8, 1);
@@ -388,7 +401,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       mbar_init(sready0 + i * 8, 1);
       mbar_init(odone0 + i * 8, 1);
       mbar_init(kready0 + i * 8, 4);   // K tile and scalars of group i written, its previous scores in registers
-      mbar_init(pready0 + i * 8, 4);   // P and V tile of group i written
+      mbar_init(pready0 + i * 8, 4 + C::kVWarps);   // P (the group) and V tile (the V converters) of group i written
     }
     misc[0] = 0; misc[1] = 0; misc[7] = 0; misc[8] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -413,10 +426,48 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
                  "r"((uint32_t)C::kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  tc_fence_before();
-  named_bar(5, C::kConsThreads + 32);
-  tc_fence_after();
-  const uint32_t tmem0 = *reinterpret_cast<volatile uint32_t*>(misc + 8);
+  uint32_t tmem0 = 0;
+  if (warp < C::kVWarp0) {
+    tc_fence_before();
+    named_bar(5, C::kConsThreads + 32);
+    tc_fence_after();
+    tmem0 = *reinterpret_cast<volatile uint32_t*>(misc + 8);
+  }
+  // =============================================================================================
+  // V converters (4 warps): expand the V planes of every unit into the V tile of the group that
+  // owns the unit, as soon as that group's previous P.V has released the tile
+  // =============================================================================================
+  if (C::kVWarps > 0 && warp >= C::kVWarp0) {
+    const int vt = tid - C::kVWarp0 * 32;  // 0..127
+    uint32_t nv[2] = {0, 0};               // V tiles so far, per group
+    int gs_base = 0, ic = 0;
+    while (gs_base < n_units) {
+      const int qi = ic & 1;
+      mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
+      const int n_piece = items[qi].pad0;
+      named_bar(6, C::kConsThreads + C::kVWarps * 32);   // the end-of-piece merge no longer uses the tiles
+      for (int u = 0; u < n_piece; ++u) {
+        const int w = u & 1;
+        const int gs = gs_base + u, slot = gs % NSTAGE;
+        const uint32_t tile_v = sbase + C::kOffCanon + w * 2 * C::kTileBytes + C::kTileBytes;
+        mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
+        const uint32_t nvw = w ? nv[1] : nv[0];
+        if (nvw > 0) mbar_wait(odone0 + w * 8, (nvw - 1) & 1, abort_word);   // V tile free
+        const uint32_t st = ring_u32 + slot * C::kStageBytes;
+        wide_expand(st + 4096u, st + 12288u, tile_v, vt);   // VA, VR
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(empty0 + slot * 8);
+          mbar_arrive(pready0 + w * 8);
+        }
+        if (w) ++nv[1]; else ++nv[0];
+      }
+      gs_base += n_piece;
+      ++ic;
+    }
+    return;
+  }
   constexpr uint32_t kIdescS = tc_idesc(64, false), kIdescO = tc_idesc(128, true);
   // =============================================================================================
   // The MMA warp: one thread issues every tcgen05.mma, so that no softmax warp stalls on the
@@ -563,7 +614,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       }
     }
     tc_fence_before();
-    named_bar(1, C::kConsThreads);
+    named_bar(6, C::kConsThreads + C::kVWarps * 32);
     const float qsum = qs_s[c];
 
     float m = 0.0f, l = 0.0f, zs = 0.0f, sw = 0.0f, hw = 0.0f;  // m: the running maximum (log2 units)
@@ -577,10 +628,11 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       const int slot = gs % NSTAGE;
       mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
       const uint32_t st = ring_u32 + slot * C::kStageBytes;
+      float2 km = make_float2(0.f, 0.f), vm = km;
+      if (r < 64) { km = lds64f(st + 16384u + r * 8); vm = lds64f(st + 16896u + r * 8); }
       wide_expand(st, st + 8192u, tile_k, r);            // KA, KR
       if (r < 64) {
         const int unit_t0 = (item.pad1 + k) * C::kST;
-        const float2 km = lds64f(st + 16384u + r * 8), vm = lds64f(st + 16896u + r * 8);
         const bool in = unit_t0 + r < len;
         // [pair][alpha0, alpha1, beta0, beta1] and [pair][zero0, zero1, scale0, scale1]
         float* sc = my_scal + set * 256 + (r >> 1) * 4 + (r & 1);
@@ -592,15 +644,17 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(kready0 + wg * 8);   // this warp's part of the K side is ready and its S is in registers
+      if (lane == 0) {
+        if (C::kVWarps > 0) mbar_arrive(empty0 + slot * 8);   // the V converters release the slot too
+        mbar_arrive(kready0 + wg * 8);    // this warp's part of the K side is ready and its S is in registers
+      }
       ++n_s;
     };
     if (wg < n_piece) prefetch(wg, (int)(n_u % 3u));
 
     for (int k = wg; k < n_piece; k += 2, ++my_units) {
       const int set = (int)(n_u % 3u);
-      const int gs = gs_base + k;
-      const int slot = gs % NSTAGE;
+      const int slot = (gs_base + k) % NSTAGE;
       const int unit_t0 = (item.pad1 + k) * C::kST;
       const uint32_t scal_u32 = smem_u32(my_scal + set * 256);
       // the scores of this unit (the only outstanding Q.K^T commit of the group)
@@ -701,14 +755,13 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
         tc_fence_after();
         TmemRegs<KT / 2>::st(tm_p + lane_sel + (uint32_t)(copy * (KT / 2)), ph);
       }
-      // ---- V side: code tile, then O += P . V ------------------------------------------------------
-      {
+      if constexpr (C::kVWarps == 0) {  // this group expands its own V tile (free: the odone wait above)
         const uint32_t st = ring_u32 + slot * C::kStageBytes;
         wide_expand(st + 4096u, st + 12288u, tile_v, r);   // VA, VR
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + slot * 8);
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty0 + slot * 8);
       tc_wait_st();
       tc_fence_before();
       __syncwarp();
