@@ -165,10 +165,11 @@ struct TmemRegs<32> {
 // stores at the swizzled chunk positions.
 __device__ __forceinline__ void wide_expand(uint32_t raw_a, uint32_t raw_r, uint32_t tile, int i) {
   const int cc = i & 3, row0 = i >> 2;
-  // Threads with cc >= 2 take the two halves of their 16 bytes in the other order (sw = 2): the
-  // four threads of a row then store to four different chunk positions in every store
-  // instruction, which makes the 128-bit stores free of bank conflicts.
-  const uint32_t sw = (uint32_t)(cc & 2);
+  // Half of the threads take the two 8-byte halves of their 16 bytes in the other order (sw = 2):
+  // cc >= 2 xor an odd row pair.  The four threads of a row then store to four different chunk
+  // positions in every store instruction (conflict-free 128-bit stores), and rows r and r + 2, which
+  // share their banks in the raw stage, read different halves (conflict-free 64-bit loads).
+  const uint32_t sw = (uint32_t)(((cc >> 1) ^ (row0 >> 1)) & 1) * 2u;
   // all loads first: the shared-memory accesses are volatile asm and keep their order
   uint2 xa[2][2], xr[2][2];
 #pragma unroll
