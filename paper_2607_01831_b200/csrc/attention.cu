@@ -10,8 +10,10 @@
 //     sum_t p_t V^_t  = sum_t (p_t scale_t) level_t + (sum_t p_t zero_t) * 1
 // so the two contractions run on the integer levels and the scalars are applied per token
 // outside.  Q.K^T is exact integer arithmetic on the int8 tensor-core path (u8 levels times two
-// s8 digit planes of the query); P.V runs in FP16 with centred levels (a-8 for the Anchor
-// state, code-128 for the full state) so that no large bias enters the FP32 accumulation.
+// s8 digit planes of the query).  P.V runs in FP16 with the levels as FP16 subnormals (the bit
+// pattern 0x00cc is code * 2^-24: no conversion arithmetic), the weights p * scale rounded to
+// FP16 and the rounding corrected to first order by the ratio of the exact to the rounded weight
+// sums.  From 17 columns on the verify pass runs on tcgen05 (attention_wide.cuh).
 //
 // Kernel shape.  Persistent grid (a few CTAs per SM), flash-decoding split-K in stream-K form:
 // the (sequence, KV head, stage-unit) list is cut into equal contiguous ranges, one per CTA.
@@ -28,7 +30,7 @@
 // for its own slice of 128/DS output dims: the nibbles of a tile are dequantised once however
 // many columns there are, and the accumulators shrink with DS.
 // K operands are the nibbles / merged codes themselves (one or two logic ops per 4 levels);
-// V operands are built from the nibbles with LOP3/PRMT and one FP16 add/fma per pair.
+// V operands are built from the nibbles with LOP3/PRMT alone.
 // A range that covers a whole (sequence, KV head) writes the output directly, otherwise the
 // partial (m, l, O) goes to the workspace and the last contributor (atomic ticket, no waiting)
 // merges them; for verification the last CTA of a sequence also takes the accept/reject

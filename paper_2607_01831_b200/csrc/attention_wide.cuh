@@ -1,12 +1,12 @@
 // Merge-verify attention for 17..64 columns on the fifth-generation tensor cores (tcgen05, TMEM).
-// Included by attention.cu inside its namespace: shares the stream-K producer warp, the piece
+// Included by attention.cu inside its namespace: shares the stream-K cut of the work, the piece
 // bookkeeping and finish_piece with the mma.sync kernels.
 //
 // With k*G >= 17 query rows per KV head the verify pass of Section 4.3 is a dense contraction
 // (about 60 / 120 flop per plane byte at 32 / 64 columns), which the mma.sync kernels cannot
 // feed: their tensor pipe would have to be busier than 100 % at the HBM roofline.  Here the two
 // contractions of a 64-token stage-unit are two tcgen05.mma groups with M = 128:
-//   S[128 rows x 64 tokens]  = Q[128 x 128 dims] . codes(K)^T      A, B in shared memory (FP16)
+//   S[128 rows x 64 tokens]  = Q[128 x 128 dims] . codes(K)^T      A = Q in TMEM, B in shared memory
 //   O[128 rows x 128 dims]  += P[128 x 64 tokens] . codes(V)       A = P in TMEM, B in shared memory
 // Row r of the M = 128 is (copy, column): the k*G columns (padded to 32 or 64) are replicated
 // NCOPY = 4 or 2 times and copy i owns tokens [i*64/NCOPY, (i+1)*64/NCOPY) of the unit: its P
@@ -14,19 +14,25 @@
 // with its own running maximum and all 128 TMEM lanes (threads) have softmax work.  Rows are
 // merged at the end of a piece.
 //
-// Two warpgroups (4 warps each) alternate over the units of a piece; each has its own S, P, O
-// regions in TMEM (64 + 32 + 128 columns) and its own FP16 operand tiles, so one group's
-// conversion and softmax overlap the other's MMAs.  Per unit a group
-//   1. expands the nibble planes of the raw stage to FP16 code tiles (subnormal patterns
-//      0x00cc = code * 2^-24, one PRMT/LOP3 per word) in the canonical 128-byte-swizzled layout,
-//      the same bytes serving as K-major B operand (K) and MN-major B operand (V);
-//   2. one thread issues S = Q.K^T (8 k-steps) and commits to an mbarrier;
-//   3. every thread reads its row's scores from TMEM, applies the per-token scale / zero point,
-//      the causal limit and the lazily raised running maximum, writes FP16 weights p*scale_v
-//      to its part of P;
-//   4. one thread issues O += P.V (4 k-steps) and commits.
-// Element order along head_dim inside each group of 8 is {0,4,2,6,1,5,3,7} in all operand
-// tiles (what the nibble expansion produces for free); it is undone when O is written out.
+// Warp roles of a CTA (one CTA per SM: it owns all 512 TMEM columns):
+//   2 softmax warpgroups (4 warps each) alternate over the units of a piece; each has its own
+//     S, P, O regions in TMEM (64 + 32 + 128 columns; Q takes the other 64) and its own K and V
+//     operand tiles.  Per unit a group reads its rows' scores from TMEM, applies the per-token
+//     scale / zero point, the causal limit and the lazily raised running maximum, and writes FP16
+//     weights p * scale_v to its part of P.  It also expands the NEXT unit's K planes into the
+//     K tile (so that S of the next unit is computed under this unit's softmax) and, in the
+//     64-column variant, its own V tile.
+//   4 V converter warps (32-column variant) expand the V planes.
+//   3 producer warps stream the raw planes into a shared-memory ring (cp.async.bulk, 8 of the
+//     24 copies of a unit each: one warp issuing all of them caps at about 2.7 TB/s).
+//   1 MMA warp: one thread polls the "operands ready" mbarriers and issues every tcgen05.mma
+//     and its commit, so that no softmax warp stalls on the tensor pipe's queue.
+// The expansion writes FP16 code tiles as subnormal patterns (0x00cc = code * 2^-24, one
+// PRMT/LOP3 per word) in the canonical 128-byte-swizzled layout; the same bytes serve as K-major
+// B operand (K) and as MN-major B operand (V).  All hand-offs are mbarriers (tcgen05.commit for
+// the MMAs); every wait is bounded.  Element order along head_dim inside each group of 8 is
+// {0,4,2,6,1,5,3,7} in all operand tiles (what the nibble expansion produces for free); it is
+// undone when O is written out.
 
 // position -> element within a group of 8: {0,4,2,6,1,5,3,7}, the 3-bit reversal
 __host__ __device__ constexpr int wide_perm(int pos) { return ((pos & 1) << 2) | (pos & 2) | ((pos >> 2) & 1); }
@@ -196,11 +202,11 @@ __device__ __forceinline__ void wide_expand(uint32_t raw_a, uint32_t raw_r, uint
   }
 }
 
-// One of the four producer warps of the wide kernel: the stream-K bookkeeping of producer_warp
-// (every warp derives the same range and pieces; warp 0 alone publishes them, loads the queries
-// and handles empty sequences), and per unit the six plane arrays of 16-token sub-block `pw`.
-// One warp issuing all 24 copies of a unit sustains only about 2.7 TB/s over the GPU; four warps
-// with six copies each lift that limit.
+// One of the producer warps of the wide kernel: the stream-K bookkeeping of producer_warp (every
+// warp derives the same range and pieces; warp 0 alone publishes them, loads the queries and
+// handles empty sequences), and per unit its share of the 24 plane copies (4 sub-blocks of 16
+// tokens x 6 arrays).  One warp issuing all 24 copies of a unit sustains only about 2.7 TB/s
+// over the GPU; three warps with eight copies each lift that limit.
 template <class C>
 __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int lane, uint32_t ring_u32,
                                               uint32_t full0, uint32_t empty0, uint32_t qfull0, uint32_t qempty0,

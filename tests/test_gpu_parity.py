@@ -325,3 +325,78 @@ def test_long_context_multi_chunk_sampled(lynx):
                              c["lens"].numpy(), Hkv, 16, causal=True)
     _close(out_a.cpu().numpy().astype(np.float64), ref_a, "anchor 40k")
     _close(out_v.cpu().numpy().astype(np.float64), ref_v, "verify 40k")
+
+
+# ------------------------------------------------------ verify with 17..64 columns (tcgen05 path)
+WIDE_CASES = [
+    # B, Hkv, G, k, lens, bt, recipe
+    (4, 2, 4, 8, (1, 15, 17, 0), 16, "student_t4"),              # 32 columns: tiny, ragged and empty sequences
+    (2, 2, 8, 8, (63, 130), 16, "normal_outlier2pct_x10"),       # 64 columns around one and two 64-token units
+    (1, 2, 4, 5, (700,), 32, "lognormal_channels"),              # 20 columns, padded to 32
+    (1, 2, 8, 5, (333,), 16, "normal_outlier4x8"),               # 40 columns, padded to 64
+    (1, 1, 3, 11, (513,), 16, "normal"),                         # 33 columns, group of 3, 11 positions
+    (3, 1, 16, 4, (64, 128, 65), 64, "student_t4"),              # 64 columns from G = 16, exact unit multiples
+]
+
+
+@pytest.mark.parametrize("case", WIDE_CASES, ids=[str(i) for i in range(len(WIDE_CASES))])
+@pytest.mark.parametrize("causal", [True, False])
+def test_wide_verify_matches_oracle_and_decides_identically(lynx, case, causal):
+    B, Hkv, G, k, lens, bt, recipe = case
+    c = _case(lynx, 600 + k + G, B, Hkv, G, k, lens, bt, True, recipe)
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    ref = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                           c["lens"].numpy(), Hkv, bt, causal=causal)
+    out, _, _ = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=causal)
+    lynx.check(c["ws"])
+    _close(out.cpu().numpy().astype(np.float64), ref, "wide verify")
+    out2, _, _ = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=causal)
+    assert torch.equal(out, out2)                 # same bits on a second call (deterministic merges)
+    # a draft that differs from the full result at known positions: identical decisions
+    rng = np.random.default_rng(7)
+    draft = torch.from_numpy((ref + rng.normal(0.0, 0.02, ref.shape)).astype(np.float32))
+    draft[0, k // 2] += 0.5
+    for atol, rtol in [(0.2, 0.0), (0.1, 0.1), (0.3, 0.1), (1.0, 0.0)]:
+        want_fr, want_dev = oracle.verify_decision(ref, draft.numpy(), atol, rtol)
+        if np.all(np.abs(want_dev - 1.0) > 0.05):
+            _, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"],
+                                                     draft_out=draft.cuda(), atol=atol, rtol=rtol,
+                                                     causal=causal)
+            lynx.check(c["ws"])
+            assert np.array_equal(fr.cpu().numpy(), want_fr), (atol, rtol, want_dev)
+            assert np.allclose(dev.cpu().numpy(), want_dev, rtol=0.05, atol=2e-3)
+
+
+def test_wide_verify_long_context_many_pieces(lynx):
+    # 32 and 64 columns at 40k tokens: every (sequence, head) is split over several CTAs, so the
+    # partial slots, the last-contributor merge and the decision tickets are exercised
+    for G, k in ((4, 8), (8, 8)):
+        B, Hkv, L = 2, 2, 40_003
+        c = _case(lynx, 700 + G, B, Hkv, G, k, (L, 9_000), 16, True, "lognormal_channels")
+        qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+        ref = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                               c["lens"].numpy(), Hkv, 16, causal=True)
+        out, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"],
+                                                   draft_out=torch.from_numpy(ref.astype(np.float32)).cuda(),
+                                                   atol=0.05, rtol=0.0)
+        lynx.check(c["ws"])
+        _close(out.cpu().numpy().astype(np.float64), ref, f"wide verify 40k, {k * G} columns")
+        assert fr.cpu().tolist() == [k] * B      # the oracle's own result as draft is accepted
+        assert float(dev.max()) < 0.1
+
+
+def test_wide_verify_single_token_returns_its_value_row(lynx):
+    # the weight-ratio correction on the tcgen05 path: one attended token gives its V row exactly
+    B, Hkv, G, k = 3, 1, 8, 8
+    c = _case(lynx, 800, B, Hkv, G, k, (1,) * B, 16, True, "student_t4")
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    out, _, _ = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=False)
+    lynx.check(c["ws"])
+    from util import dequant
+    va, vr, vm = c["vp"]
+    got = out.cpu().numpy().astype(np.float64)
+    for b in range(B):
+        blk = int(c["table"][b, 0])
+        row = dequant(va[blk, 0, 0], vr[blk, 0, 0], vm[blk, 0, 0], True)
+        size = abs(float(vm[blk, 0, 0, 1])) + 255.0 * float(vm[blk, 0, 0, 0])
+        assert np.max(np.abs(got[b] - row[None, None, :])) <= 4e-6 * size + 1e-30
