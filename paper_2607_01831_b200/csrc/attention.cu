@@ -529,13 +529,14 @@ __device__ __forceinline__ void producer_warp(const AttnParams& p, int lane, uin
 // With DS > 1 a team keeps one running maximum per column: two named barriers per step, growth
 // agreed through shared memory.  With DS == 1 a warp is its own team and nothing is exchanged.
 // =============================================================================================
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int TPW = 1>
 struct TeamCfg {
-  static constexpr int kTW = DS * TEAMS;                    // consumer warps = tiles per stage
+  static_assert(TPW == 1 || DS == 1, "several tiles per warp and stage only without teams");
+  static constexpr int kTW = DS * TEAMS * TPW;              // tiles per stage (TPW per consumer warp)
   static constexpr int kST = kTW * 16;
   static constexpr int kSubBytes = FULL ? 16 * 272 : 16 * 144;
   static constexpr int kStageBytes = kST * (FULL ? 272 : 144);
-  static constexpr int kConsWarps = kTW;
+  static constexpr int kConsWarps = DS * TEAMS;
   static constexpr int kConsThreads = kConsWarps * 32;
   static constexpr int kThreads = (kConsWarps + 1) * 32;
   static constexpr int kColsPad = NT * 8;
@@ -543,7 +544,7 @@ struct TeamCfg {
   static constexpr int kRing = NSTAGE * kStageBytes;
   static constexpr int kMailRegs = NT * kMT * 4 + NT * 10;  // o slice + m, l, zs, sw, hw
   static constexpr int kMailBytes = TEAMS > 1 ? kMailRegs * 32 * 4 : 0;  // one box, used slice by slice
-  static constexpr int kXchgBytes = DS > 1 ? kTW * (16 + kColsPad * 4 + NT * 2 * 32 * 4) : 0;  // flag, colmax, P^T
+  static constexpr int kXchgBytes = DS > 1 ? kConsWarps * (16 + kColsPad * 4 + NT * 2 * 32 * 4) : 0;  // flag, colmax, P^T
   static constexpr int kLzBytes = DS * kColsPad * 4 * 4 + 16;
   static constexpr int kQfBytes = NT * 2 * 4 * 32 * 8 + kColsPad * 4;  // query fragments, sum of q
   static constexpr int kQBytes = 2 * kColsPad * LYNX_D * 2;
@@ -660,9 +661,9 @@ __device__ __forceinline__ void pv_slice(float (&o)[NT][8 / DS][4], uint32_t st,
   }
 }
 
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int TPW>
 __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
-  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE>;
+  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE, TPW>;
   constexpr int ST = C::kST, TW = C::kTW, MT = C::kMT;
   constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
   constexpr float kMidK = FULL ? 0.0f : 8.0f;
@@ -766,8 +767,8 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       ca = p.sm_log2 * down * (FULL ? 1.0f : 16.0f);
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        // warp w builds the shared fragments of the n-tiles nt = w, w + TW, ... for everybody
-        const bool mine = (nt % TW) == warp;
+        // warp w builds the shared fragments of the n-tiles nt = w, w + (consumer warps), ... for everybody
+        const bool mine = (nt % C::kConsWarps) == warp;
         if (mine) {
           const int c = nt * 8 + g;
 #pragma unroll
@@ -826,16 +827,19 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 
     const uint32_t st = ring_u32 + slot * C::kStageBytes;
     const int unit_t0 = info.y * ST;
-    const int tile_t0 = unit_t0 + warp * 16;
+#pragma unroll
+    for (int tp = 0; tp < TPW; ++tp) {   // the tiles of this warp in the stage
+    const int wt = warp + tp * C::kConsWarps;
+    const int tile_t0 = unit_t0 + wt * 16;
     const bool in_range = tile_t0 < len;                          // this warp's own tile
-    const bool team_valid = unit_t0 + team * DS * 16 < len;       // the team's first tile
+    const bool team_valid = unit_t0 + (DS == 1 ? wt : team * DS) * 16 < len;   // the team's first tile
     if (DS > 1 || in_range) {  // a lone warp (DS == 1) has nothing to do for a tile beyond the end
     const bool valid = DS == 1 ? true : in_range;
     unsigned char* my_x = xchg + (size_t)warp * kXW;
     float s[NT][4];
     float cmx[DS > 1 ? 1 : NT][2];  // column maxima of this tile (kept in registers when DS == 1)
     float2 vm_lo = make_float2(0.f, 0.f), vm_hi = make_float2(0.f, 0.f);
-    const int r0 = warp * 16 + pi_row(g);
+    const int r0 = wt * 16 + pi_row(g);
     const int tok_lo = tile_t0 + pi_row(g), tok_hi = tok_lo + 8;
     const bool masked = tile_t0 + 16 > full_lim;
     // ---- phase A: scores of this warp's tile, growth vote -------------------------------
@@ -994,7 +998,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
     if constexpr (DS > 1) named_bar(2 + team, DS * 32);
     // ---- phase C: P.V of the team's tiles for this warp's slice of the output dims --------
     if constexpr (DS == 1) {
-      if (valid) pv_slice<FULL, NT, ST, 1>(o, st, warp * 16, g, t, 0, pown);
+      if (valid) pv_slice<FULL, NT, ST, 1>(o, st, wt * 16, g, t, 0, pown);
     }
 #pragma unroll
     for (int tau = 0; tau < (DS > 1 ? DS : 0); ++tau) {
@@ -1010,6 +1014,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       pv_slice<FULL, NT, ST, DS>(o, st, src * 16, g, t, d, pb);
     }
     }  // if (DS > 1 || in_range)
+    }  // tiles of this warp
     __syncwarp();
     if (lane == 0) mbar_arrive(empty0 + slot * 8);
     if (!(info.z & 2)) continue;
@@ -1147,10 +1152,10 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 
 // At least MINB CTAs per SM (the compiler caps registers accordingly).  Nine warps cannot
 // have more than 168 registers each: three of them share one SM sub-partition's 16 K registers.
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB, int TPW>
 __global__ void __launch_bounds__((DS * TEAMS + 1) * 32, MINB)
 attn_team_kernel(const AttnParams p) {
-  attn_team_body<FULL, NT, DS, TEAMS, NSTAGE>(p);
+  attn_team_body<FULL, NT, DS, TEAMS, NSTAGE, TPW>(p);
 }
 #ifndef LYNX_WIDE_VERIFY
 #define LYNX_WIDE_VERIFY 2   // 0: keep the mma.sync kernels for 17..64 verify columns (comparison builds)
@@ -1192,14 +1197,14 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   return true;
 }
 
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB, int TPW = 1>
 lynx_status launch_team(const AttnParams& p, cudaStream_t st) {
-  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE>;
+  using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE, TPW>;
   static_assert(MINB <= kMaxCtasPerSm, "partial slots are sized for kMaxCtasPerSm CTAs per SM");
   constexpr int kCtasPerSm = MINB;
   static_assert(kCtasPerSm * (C::kSmem + 1024) <= 228 * 1024, "shared memory budget per SM");
   static_assert(2 + TEAMS <= 16, "named barriers");
-  auto kern = attn_team_kernel<FULL, NT, DS, TEAMS, NSTAGE, MINB>;
+  auto kern = attn_team_kernel<FULL, NT, DS, TEAMS, NSTAGE, MINB, TPW>;
   static bool configured[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -1264,7 +1269,7 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   // <FULL, NT, DS, TEAMS, stages, CTAs/SM>
   if (!full) {
     switch (pl.variant) {
-      case 0: return launch_team<false, 1, 1, 4, 4, 4>(p, st);
+      case 0: return launch_team<false, 1, 1, 4, 2, 4, 2>(p, st);   // two tiles per warp and stage
       case 1: return launch_team<false, 2, 2, 2, 4, 3>(p, st);
       case 2: return launch_team<false, 4, 4, 1, 3, 3>(p, st);
       default: return launch_team<false, 8, 4, 2, 3, 1>(p, st);
