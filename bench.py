@@ -443,6 +443,7 @@ def main():
 
     if rank == 0 and world == 1:
         line["per_layer_launches"] = run_per_layer(wlk, peak)
+        line["recombine"] = run_recombine(wlk, peak)
     if rank == 0 and world == 1 and not args.no_e2e:
         line["e2e"] = run_e2e(wlk, args.e2e_steps, step_bytes)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -454,6 +455,43 @@ def main():
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(line))
+
+
+def run_recombine(wlk: "Workload", peak: float, max_rows: int = 4 << 20):
+    """Context: the stand-alone refinement `lynx_recombine` (Anchor + Residual -> 8-bit codes and/or
+    dequantised BF16 rows, the layout a stock BF16 attention would read) on the first rows of the
+    K planes, at most 4 Mi rows (1 GiB of BF16 output).  Not part of `value`."""
+    lynx = wlk.lynx
+    K = wlk.planes["K"]
+    rows = min(K.anchor.numel() // 64, max_rows)
+    a, r, m = K.anchor.view(-1, 64)[:rows], K.residual.view(-1, 64)[:rows], K.meta.view(-1, 2)[:rows]
+    codes = torch.empty(rows, 128, dtype=torch.uint8, device=wlk.device)
+    deq = torch.empty(rows, 128, dtype=torch.bfloat16, device=wlk.device)
+    lib = lynx.load()
+    stream = torch.cuda.current_stream().cuda_stream
+    out = {"rows": rows}
+    for name, c, d, bpr in (("bf16", None, deq, 136 + 256), ("codes", codes, None, 136 + 128),
+                            ("codes+bf16", codes, deq, 136 + 128 + 256)):
+        def call():
+            st = lib.lynx_recombine(a.data_ptr(), r.data_ptr(), m.data_ptr(), rows,
+                                    c.data_ptr() if c is not None else None,
+                                    d.data_ptr() if d is not None else None, stream)
+            if st != 0:
+                raise RuntimeError(f"lynx_recombine: status {st}")
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 10
+        e0.record()
+        for _ in range(reps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        gbs = rows * bpr / (ms * 1e-3) / 1e9
+        out[name] = {"ms": ms, "bytes_per_row": bpr, "GBps": gbs, "frac_of_measured": gbs / peak}
+    return out
 
 
 def run_per_layer(wlk: "Workload", peak: float):
