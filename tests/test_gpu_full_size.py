@@ -35,8 +35,6 @@ def test_config3_full_size_sampled_layers():
     nbl, Hkv, bt = wlk.nb_layer, wl.num_kv_heads, wl.block_tokens
     table = torch.arange(nbl, dtype=torch.int32).view(1, nbl).numpy()
     lens = np.array([wl.context], np.int32)
-    win = wlk.windows[0]                       # k = 2
-    k = win["k"]
     for layer in (0, wl.layers - 1):
         sl = slice(layer * nbl, (layer + 1) * nbl)
         planes = {}
@@ -47,15 +45,52 @@ def test_config3_full_size_sampled_layers():
             assert np.array_equal(got.residual[sl].cpu().numpy(), want[1])
             assert np.array_equal(got.meta[sl].cpu().numpy().view(np.uint32), want[2].view(np.uint32))
             planes[which] = want
-        q = _bits(win["q"][layer:layer + 1])
-        ref_a = oracle.attention(False, q, planes["K"], planes["V"], table, lens, Hkv, bt, causal=True)
-        ref_f = oracle.attention(True, q, planes["K"], planes["V"], table, lens, Hkv, bt, causal=True)
-        draft = win["draft"][layer:layer + 1].cpu().numpy()
-        full = win["out_full"][layer:layer + 1].cpu().numpy()
-        for got, ref in ((draft, ref_a), (full, ref_f)):
-            g = got.astype(np.float64)
-            assert np.all(np.abs(g - ref) <= ATOL + RTOL * np.abs(ref)), float(np.abs(g - ref).max())
-        want_fr, want_dev = oracle.verify_decision(ref_f, draft, 0.5, 0.1)
-        if np.all(np.abs(want_dev - 1.0) > 0.05):
-            assert int(win["first_reject"][layer]) == int(want_fr[0])
-        assert np.allclose(win["dev"][layer].cpu().numpy(), want_dev[0], rtol=0.05, atol=1e-3)
+        for win in wlk.windows:                # k = 2, 4, 8: 8, 16 and 32 columns
+            _check_window(oracle, win, layer, planes, table, lens, Hkv, bt)
+
+
+def _check_window(oracle, win, b, planes, table, lens, Hkv, bt):
+    q = _bits(win["q"][b:b + 1])
+    ref_a = oracle.attention(False, q, planes["K"], planes["V"], table, lens, Hkv, bt, causal=True)
+    ref_f = oracle.attention(True, q, planes["K"], planes["V"], table, lens, Hkv, bt, causal=True)
+    draft = win["draft"][b:b + 1].cpu().numpy()
+    full = win["out_full"][b:b + 1].cpu().numpy()
+    for got, ref in ((draft, ref_a), (full, ref_f)):
+        g = got.astype(np.float64)
+        assert np.all(np.abs(g - ref) <= ATOL + RTOL * np.abs(ref)), (win["k"], float(np.abs(g - ref).max()))
+    want_fr, want_dev = oracle.verify_decision(ref_f, draft, 0.5, 0.1)
+    if np.all(np.abs(want_dev - 1.0) > 0.05):
+        assert int(win["first_reject"][b]) == int(want_fr[0])
+    assert np.allclose(win["dev"][b].cpu().numpy(), want_dev[0], rtol=0.05, atol=1e-3)
+
+
+def test_config5_shape_two_layers_sampled():
+    """The 70B-class shape (GQA group 8, batch 2, k = 8: 64 verify columns) at two of its 80 layers,
+    through the same Workload class and launches as bench.py: sampled (layer, sequence) pairs."""
+    import bench
+    import oracle
+    free, _ = torch.cuda.mem_get_info()
+    if free < 12 * 2 ** 30:
+        pytest.skip("needs ~8 GB of device memory")
+    wlk = bench.Workload(5, torch.device("cuda", 0), layers=2)
+    wl = wlk.wl
+    wlk.step()
+    torch.cuda.synchronize()
+    for w in wlk.windows:
+        wlk.lynx.check(w["ws"])
+    nbl, Hkv, bt = wlk.nb_layer, wl.num_kv_heads, wl.block_tokens
+    table_all = wlk.table.cpu().numpy()
+    for b in (0, wlk.B - 1):                   # flattened (layer, sequence) index
+        layer, seq = divmod(b, wl.batch)
+        sl = slice(layer * nbl, (layer + 1) * nbl)
+        planes = {}
+        for which in "KV":
+            want = oracle.split_quantize(_bits(wlk.src[which][sl]))
+            got = wlk.planes[which]
+            assert np.array_equal(got.anchor[sl].cpu().numpy(), want[0])
+            assert np.array_equal(got.residual[sl].cpu().numpy(), want[1])
+            planes[which] = want
+        table = (table_all[b:b + 1] - layer * nbl).astype(np.int32)
+        lens = np.array([int(wlk.lens_flat_cpu[b])], np.int32)
+        for win in wlk.windows:
+            _check_window(oracle, win, b, planes, table, lens, Hkv, bt)
