@@ -760,8 +760,9 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       }
 #pragma unroll
       for (int off = 16; off >= 1; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, off));
-      int e = 0;  // two s8 digit planes of q, see attn_kernel
-      if (amax > 0.0f && amax < INFINITY) e = 13 - (((__float_as_int(amax) >> 23) & 0xFF) - 127);
+      // two balanced s8 digit planes of q: q_int = rint(q * 2^e) = 256 * hi + lo, |q_int| < 2^15
+      int e = 0;
+      if (amax > 0.0f && amax < INFINITY) e = 14 - (((__float_as_int(amax) >> 23) & 0xFF) - 127);
       e = max(-100, min(100, e));
       const float up = __int_as_float((127 + e) << 23), down = __int_as_float((127 - e) << 23);
       ca = p.sm_log2 * down * (FULL ? 1.0f : 16.0f);
@@ -778,16 +779,18 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
             int qv[8];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              qv[2 * k] = __float2int_rn(__uint_as_float(ww[k] << 16) * up);
-              qv[2 * k + 1] = __float2int_rn(__uint_as_float(ww[k] & 0xFFFF0000u) * up);
+              // (32640, the largest BF16 mantissa at the top exponent, would need hi = 128)
+              qv[2 * k] = min(__float2int_rn(__uint_as_float(ww[k] << 16) * up), 32639);
+              qv[2 * k + 1] = min(__float2int_rn(__uint_as_float(ww[k] & 0xFFFF0000u) * up), 32639);
             }
             uint32_t hi_e = 0, hi_o = 0, lo_e = 0, lo_o = 0;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              hi_e |= (uint32_t)((qv[2 * k] >> 7) & 0xFF) << (8 * k);
-              lo_e |= (uint32_t)(qv[2 * k] & 127) << (8 * k);
-              hi_o |= (uint32_t)((qv[2 * k + 1] >> 7) & 0xFF) << (8 * k);
-              lo_o |= (uint32_t)(qv[2 * k + 1] & 127) << (8 * k);
+              const int he = (qv[2 * k] + 128) >> 8, ho = (qv[2 * k + 1] + 128) >> 8;   // lo in [-128, 127]
+              hi_e |= (uint32_t)(he & 0xFF) << (8 * k);
+              lo_e |= (uint32_t)((qv[2 * k] - (he << 8)) & 0xFF) << (8 * k);
+              hi_o |= (uint32_t)(ho & 0xFF) << (8 * k);
+              lo_o |= (uint32_t)((qv[2 * k + 1] - (ho << 8)) & 0xFF) << (8 * k);
             }
             reinterpret_cast<uint2*>(qf_s)[((nt * 2 + 0) * 4 + wd) * 32 + lane] = make_uint2(hi_e, hi_o);
             reinterpret_cast<uint2*>(qf_s)[((nt * 2 + 1) * 4 + wd) * 32 + lane] = make_uint2(lo_e, lo_o);
@@ -859,7 +862,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
             mma_u8s8(slo, a[wd][0], a[wd][1], a[wd][2], a[wd][3], bl.x, bl.y);
           }
 #pragma unroll
-          for (int i = 0; i < 4; ++i) s[nt][i] = (float)(shi[i] * 128 + slo[i]);
+          for (int i = 0; i < 4; ++i) s[nt][i] = (float)(shi[i] * 256 + slo[i]);
         }
       }
       float2 km_lo = lds64f(st + KM + r0 * 8), km_hi = lds64f(st + KM + (r0 + 8) * 8);

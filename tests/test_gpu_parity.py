@@ -400,3 +400,39 @@ def test_wide_verify_single_token_returns_its_value_row(lynx):
         row = dequant(va[blk, 0, 0], vr[blk, 0, 0], vm[blk, 0, 0], True)
         size = abs(float(vm[blk, 0, 0, 1])) + 255.0 * float(vm[blk, 0, 0, 0])
         assert np.max(np.abs(got[b] - row[None, None, :])) <= 4e-6 * size + 1e-30
+
+
+def test_seeded_random_shapes_all_variants(lynx):
+    # a seeded sweep over shapes (KV heads, GQA group, positions, block size, ragged lengths) that
+    # reaches every kernel variant: 1..64 columns, anchor and verify, causal or not
+    rng = np.random.default_rng(20250607)
+    recipes = ["normal_outlier4x8", "lognormal_channels", "student_t4", "normal_outlier2pct_x10", "normal"]
+    done = 0
+    while done < 14:
+        Hkv = int(rng.choice([1, 2, 3]))
+        G = int(rng.choice([1, 2, 3, 4, 6, 8, 16]))
+        k = int(rng.integers(1, 17))
+        if k * G > 64:
+            continue
+        B = int(rng.integers(1, 4))
+        bt = int(rng.choice([16, 32, 64]))
+        lens = tuple(int(x) for x in rng.choice([0, 1, 5, 16, 63, 64, 65, 200, 777, 1500, 3100], size=B))
+        causal = bool(rng.integers(0, 2))
+        c = _case(lynx, 900 + done, B, Hkv, G, k, lens, bt, True, recipes[done % len(recipes)])
+        qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+        what = f"B={B} Hkv={Hkv} G={G} k={k} bt={bt} lens={lens} causal={causal}"
+        ref_a = oracle.attention(False, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                                 c["lens"].numpy(), Hkv, bt, causal=causal)
+        out_a = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=causal)
+        lynx.check(c["ws"])
+        _close(out_a.cpu().numpy().astype(np.float64), ref_a, "anchor " + what)
+        ref_f = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                                 c["lens"].numpy(), Hkv, bt, causal=causal)
+        out_f, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"],
+                                                     draft_out=out_a, atol=0.25, rtol=0.05, causal=causal)
+        lynx.check(c["ws"])
+        _close(out_f.cpu().numpy().astype(np.float64), ref_f, "verify " + what)
+        want_fr, want_dev = oracle.verify_decision(ref_f, out_a.cpu().numpy(), 0.25, 0.05)
+        if np.all(np.abs(want_dev - 1.0) > 0.05):
+            assert np.array_equal(fr.cpu().numpy(), want_fr), what
+        done += 1
