@@ -11,9 +11,10 @@
 // so the two contractions run on the integer levels and the scalars are applied per token
 // outside.  Q.K^T is exact integer arithmetic on the int8 tensor-core path (u8 levels times two
 // s8 digit planes of the query).  P.V runs in FP16 with the levels as FP16 subnormals (the bit
-// pattern 0x00cc is code * 2^-24: no conversion arithmetic), the weights p * scale rounded to
-// FP16 and the rounding corrected to first order by the ratio of the exact to the rounded weight
-// sums.  From 17 columns on the verify pass runs on tcgen05 (attention_wide.cuh).
+// pattern 0x00cc is code * 2^-24: no conversion arithmetic) and the weights p * scale as the sum
+// of two FP16 numbers (the rounded weight and the rounding's remainder, each with its own MMA), so
+// the weights carry about 22 bits.  From 17 columns on the verify pass runs on tcgen05
+// (attention_wide.cuh).
 //
 // Kernel shape.  Persistent grid (a few CTAs per SM), flash-decoding split-K in stream-K form:
 // the (sequence, KV head, stage-unit) list is cut into equal contiguous ranges, one per CTA.
@@ -155,6 +156,11 @@ __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
   uint32_t d;
   asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
   return d;
+}
+// the two FP16 halves of h as FP32 (exact)
+__device__ __forceinline__ void unpack_f16x2(uint32_t h, float& lo, float& hi) {
+  asm("{\n\t.reg .b16 l, u;\n\tmov.b32 {l, u}, %2;\n\tcvt.f32.f16 %0, l;\n\tcvt.f32.f16 %1, u;\n\t}"
+      : "=f"(lo), "=f"(hi) : "r"(h));
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -542,10 +548,10 @@ struct TeamCfg {
   static constexpr int kColsPad = NT * 8;
   static constexpr int kMT = 8 / DS;                        // m-tiles (16 dims) per warp
   static constexpr int kRing = NSTAGE * kStageBytes;
-  static constexpr int kMailRegs = NT * kMT * 4 + NT * 10;  // o slice + m, l, zs, sw, hw
+  static constexpr int kMailRegs = NT * kMT * 4 + NT * 6;   // o slice + m, l, zs
   static constexpr int kMailBytes = TEAMS > 1 ? kMailRegs * 32 * 4 : 0;  // one box, used slice by slice
-  static constexpr int kXchgBytes = DS > 1 ? kConsWarps * (16 + kColsPad * 4 + NT * 2 * 32 * 4) : 0;  // flag, colmax, P^T
-  static constexpr int kLzBytes = DS * kColsPad * 4 * 4 + 16;
+  static constexpr int kXchgBytes = DS > 1 ? kConsWarps * (16 + kColsPad * 4 + NT * 4 * 32 * 4) : 0;  // flag, colmax, P^T (two terms)
+  static constexpr int kLzBytes = DS * kColsPad * 2 * 4 + 16;
   static constexpr int kQfBytes = NT * 2 * 4 * 32 * 8 + kColsPad * 4;  // query fragments, sum of q
   static constexpr int kQBytes = 2 * kColsPad * LYNX_D * 2;
   static constexpr int kBlkBytes = kPieceUnits * kTW * 4;
@@ -589,7 +595,7 @@ __device__ __forceinline__ void k_fragments(uint32_t st, int r0, int t, uint32_t
 // word d, DS=4 word d>>1 / half d&1.
 template <bool FULL, int NT, int ST, int DS>
 __device__ __forceinline__ void pv_slice(float (&o)[NT][8 / DS][4], uint32_t st, int row0, int g, int t,
-                                         int d, const uint32_t (&pb)[NT][2]) {
+                                         int d, const uint32_t (&pb)[NT][4]) {
   constexpr uint32_t VA = ST * 64, VR = ST * 192;
   constexpr int NW = DS == 1 ? 2 : 1;  // words of the lane's 8 V bytes this warp touches
   constexpr int NH = DS == 4 ? 1 : 2;  // halves of each word
@@ -655,7 +661,10 @@ __device__ __forceinline__ void pv_slice(float (&o)[NT][8 / DS][4], uint32_t st,
         const int lm = (DS == 1 ? i * 4 : 0) + (DS == 4 ? 0 : hh * 2) + qd;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
+        {  // the rounded weights, then the remainders of their rounding
           mma16816(o[nt][lm], ab[2 * qd], ab[2 * qd + 1], cd[2 * qd], cd[2 * qd + 1], pb[nt][0], pb[nt][1]);
+          mma16816(o[nt][lm], ab[2 * qd], ab[2 * qd + 1], cd[2 * qd], cd[2 * qd + 1], pb[nt][2], pb[nt][3]);
+        }
       }
     }
   }
@@ -669,7 +678,6 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
   constexpr float kMidK = FULL ? 0.0f : 8.0f;
   constexpr float kMidV = FULL ? 0.0f : 8.0f;      // V levels: plain codes (full) / plain nibbles (anchor)
   constexpr float kLevelScaleV = FULL ? 1.0f : 16.0f;
-  constexpr uint32_t kOnesH2 = 0x3C003C00u;        // FP16 pair (1, 1)
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* ring = smem;
   float* mail = reinterpret_cast<float*>(smem + C::kRing);
@@ -716,17 +724,19 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
   if (n_units == 0) return;
 
   // per-warp exchange area: [flag (16 B)] [column maxima: kColsPad floats] [P^T: NT x 2 x 32 words]
-  constexpr int kXW = 16 + C::kColsPad * 4 + NT * 2 * 32 * 4;
+  constexpr int kXW = 16 + C::kColsPad * 4 + NT * 4 * 32 * 4;
   const int g = lane >> 2, t = lane & 3;
   const int team = warp / DS, d = warp % DS;
   const float cb = p.sm_log2;
   // m holds MINUS the running maximum inside the stage loop (it enters the score FMA directly)
-  // sw, hw: sums of the V weights p * scale before and after their rounding to FP16; the ratio
-  // sw / hw scales the accumulators at the end, which removes the rounding's first-order effect
-  // (the residue is the rounding error times a level's distance from the weighted mean level)
-  // (hw comes from one extra MMA per n-tile with an all-ones A operand, which gives every lane
-  // the complete sums of the warp's own tile for its columns 2t, 2t+1)
-  float m[NT][2], l[NT][2], zs[NT][2], sw[NT][2], hw[NT][2], o[NT][MT][4];
+  // The tensor core truncates when it adds into its FP32 accumulators: every MMA loses half a unit
+  // in the last place of the accumulator on average, about 0.4 * 2^-23 of its value (measured; mantissas spread
+  // log-uniformly).  Over the thousands of MMAs of a long piece that is a relative bias of some
+  // 1e-4 on the uncentred level sums, which are large against the outputs they cancel into.  The
+  // MMAs into each accumulator are counted and the expected loss is put back at the end of a piece.
+  constexpr float kTruncPerMma = 0.40f * 1.1920929e-7f;
+  int n_mma = 0;
+  float m[NT][2], l[NT][2], zs[NT][2], o[NT][MT][4];
   const uint32_t qf_u32 = smem_u32(qf_s), qs_u32 = smem_u32(qs_s);
   auto col_limit = [&](int col, int len_) {
     return col < p.ncols ? (p.causal ? len_ - p.nq + col / p.G + 1 : len_) : 0;
@@ -816,8 +826,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
         }
 #pragma unroll
         for (int cc = 0; cc < 2; ++cc) {
-          m[nt][cc] = 0.0f; l[nt][cc] = 0.0f; zs[nt][cc] = 0.0f; sw[nt][cc] = 0.0f;
-          hw[nt][cc] = 0.0f;
+          m[nt][cc] = 0.0f; l[nt][cc] = 0.0f; zs[nt][cc] = 0.0f;
         }
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
@@ -826,6 +835,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       }
       named_bar(1, C::kConsThreads);  // the shared fragments are complete
       fresh = true;
+      n_mma = 0;
     }
 
     const uint32_t st = ring_u32 + slot * C::kStageBytes;
@@ -954,8 +964,6 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
             s[nt][cc + 2] -= up;
             l[nt][cc] *= f;
             zs[nt][cc] *= f;
-            sw[nt][cc] *= f;
-            hw[nt][cc] *= f;
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
               o[nt][mt][cc] *= f;
@@ -966,7 +974,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       if (team_valid) fresh = false;
     }
     // ---- weights of this warp's tile, P^T fragments to shared memory ---------------------
-    uint32_t pown[DS > 1 ? 1 : NT][2];  // P^T fragments of the own tile (DS == 1)
+    uint32_t pown[DS > 1 ? 1 : NT][4];  // P^T fragments of the own tile (DS == 1): rounded weights, remainders
     if (valid) {
       const float sv_lo = vm_lo.x * kLevelScaleV, sv_hi = vm_hi.x * kLevelScaleV;
       const float zv_lo = fmaf(vm_lo.x, kMidV, vm_lo.y), zv_hi = fmaf(vm_hi.x, kMidV, vm_hi.y);
@@ -982,39 +990,45 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
         float w0, w1, w2, w3;
         upk2(fmul2(plo, pk2(sv_lo, sv_lo)), w0, w1);
         upk2(fmul2(phi, pk2(sv_hi, sv_hi)), w2, w3);
+        // w = h + r: h the FP16 rounding of w, r its remainder (exact in FP32, rounded to FP16)
         const uint32_t h01 = pack_f16x2(w0, w1), h23 = pack_f16x2(w2, w3);
-        upk2(fadd2(pk2(sw[nt][0], sw[nt][1]), fadd2(pk2(w0, w1), pk2(w2, w3))), sw[nt][0], sw[nt][1]);
-        const uint32_t f0 = movmatrix_trans(h01);
-        const uint32_t f1 = movmatrix_trans(h23);
-        float hsum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        mma16816(hsum, kOnesH2, kOnesH2, kOnesH2, kOnesH2, f0, f1);
-        upk2(fadd2(pk2(hw[nt][0], hw[nt][1]), pk2(hsum[0], hsum[1])), hw[nt][0], hw[nt][1]);
+        float b0, b1, b2, b3;
+        unpack_f16x2(h01, b0, b1);
+        unpack_f16x2(h23, b2, b3);
+        const uint32_t r01 = pack_f16x2(w0 - b0, w1 - b1), r23 = pack_f16x2(w2 - b2, w3 - b3);
+        const uint32_t f0 = movmatrix_trans(h01), f1 = movmatrix_trans(h23);
+        const uint32_t f2 = movmatrix_trans(r01), f3 = movmatrix_trans(r23);
         if constexpr (DS > 1) {
-          pf[(nt * 2 + 0) * 32] = f0;
-          pf[(nt * 2 + 1) * 32] = f1;
+          pf[(nt * 4 + 0) * 32] = f0;
+          pf[(nt * 4 + 1) * 32] = f1;
+          pf[(nt * 4 + 2) * 32] = f2;
+          pf[(nt * 4 + 3) * 32] = f3;
         } else {
-          pown[nt][0] = f0;
-          pown[nt][1] = f1;
+          pown[nt][0] = f0; pown[nt][1] = f1; pown[nt][2] = f2; pown[nt][3] = f3;
         }
       }
     }
     if constexpr (DS > 1) named_bar(2 + team, DS * 32);
     // ---- phase C: P.V of the team's tiles for this warp's slice of the output dims --------
     if constexpr (DS == 1) {
-      if (valid) pv_slice<FULL, NT, ST, 1>(o, st, wt * 16, g, t, 0, pown);
+      if (valid) {
+        pv_slice<FULL, NT, ST, 1>(o, st, wt * 16, g, t, 0, pown);
+        n_mma += 2;   // into every accumulator: the rounded weights and their remainders
+      }
     }
 #pragma unroll
     for (int tau = 0; tau < (DS > 1 ? DS : 0); ++tau) {
       const int src = team * DS + tau;
       if (unit_t0 + src * 16 >= len) break;  // uniform: later tiles of the unit are beyond len too
-      uint32_t pb[NT][2];
+      uint32_t pb[NT][4];
       const uint32_t* pf = reinterpret_cast<const uint32_t*>(xchg + (size_t)src * kXW + 16 + C::kColsPad * 4) + lane;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        pb[nt][0] = *reinterpret_cast<const volatile uint32_t*>(pf + (nt * 2 + 0) * 32);
-        pb[nt][1] = *reinterpret_cast<const volatile uint32_t*>(pf + (nt * 2 + 1) * 32);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) pb[nt][i] = *reinterpret_cast<const volatile uint32_t*>(pf + (nt * 4 + i) * 32);
       }
       pv_slice<FULL, NT, ST, DS>(o, st, src * 16, g, t, d, pb);
+      n_mma += 2;
     }
     }  // if (DS > 1 || in_range)
     }  // tiles of this warp
@@ -1023,6 +1037,15 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
     if (!(info.z & 2)) continue;
 
     // ---- end of the piece -----------------------------------------------------------------
+    {
+      const float back = 1.0f + (float)n_mma * kTruncPerMma;   // the expected truncation loss, put back
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) o[nt][mt][i] *= back;
+    }
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) { m[nt][0] = -m[nt][0]; m[nt][1] = -m[nt][1]; }  // back to the maximum
     if (fresh) {
@@ -1046,8 +1069,6 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
               box[(r++) * 32] = m[nt][cc];
               box[(r++) * 32] = l[nt][cc];
               box[(r++) * 32] = zs[nt][cc];
-              box[(r++) * 32] = sw[nt][cc];
-              box[(r++) * 32] = hw[nt][cc];
             }
           }
         }
@@ -1059,7 +1080,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
             float f1[2], f2[2];
 #pragma unroll
             for (int cc = 0; cc < 2; ++cc) {
-              const float m2 = box[((MT * 4 + 10) * nt + MT * 4 + 5 * cc) * 32];
+              const float m2 = box[((MT * 4 + 6) * nt + MT * 4 + 3 * cc) * 32];
               const float M = fmaxf(m[nt][cc], m2);
               f1[cc] = ex2(m[nt][cc] - M);
               f2[cc] = ex2(m2 - M);
@@ -1077,12 +1098,8 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
               r++;
               const float l2 = box[(r++) * 32];
               const float z2 = box[(r++) * 32];
-              const float s2 = box[(r++) * 32];
-              const float h2 = box[(r++) * 32];
               l[nt][cc] = l[nt][cc] * f1[cc] + l2 * f2[cc];
               zs[nt][cc] = zs[nt][cc] * f1[cc] + z2 * f2[cc];
-              sw[nt][cc] = sw[nt][cc] * f1[cc] + s2 * f2[cc];
-              hw[nt][cc] = hw[nt][cc] * f1[cc] + h2 * f2[cc];
             }
           }
         }
@@ -1095,17 +1112,14 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int cc = 0; cc < 2; ++cc) {
-          float lv = l[nt][cc], z = zs[nt][cc], sv = sw[nt][cc];
-          const float hv = hw[nt][cc];  // already complete over the tile's rows
+          float lv = l[nt][cc], z = zs[nt][cc];
 #pragma unroll
           for (int off = 4; off <= 16; off <<= 1) {
             lv += __shfl_xor_sync(0xFFFFFFFFu, lv, off);
             z += __shfl_xor_sync(0xFFFFFFFFu, z, off);
-            sv += __shfl_xor_sync(0xFFFFFFFFu, sv, off);
           }
           if (g == 0)
-            *reinterpret_cast<float4*>(lz + ((size_t)d * C::kColsPad + nt * 8 + 2 * t + cc) * 4) =
-                make_float4(lv, z, sv, hv);
+            *reinterpret_cast<float2*>(lz + ((size_t)d * C::kColsPad + nt * 8 + 2 * t + cc) * 2) = make_float2(lv, z);
         }
     }
     named_bar(1, C::kConsThreads);
@@ -1118,21 +1132,19 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 #pragma unroll
         for (int cc = 0; cc < 2; ++cc) {
           const int c = nt * 8 + 2 * t + cc;
-          float lt = 0.0f, z = 0.0f, st_ = 0.0f, ht = 0.0f;
+          float lt = 0.0f, z = 0.0f;
 #pragma unroll
           for (int dd = 0; dd < DS; ++dd) {
-            const float4 v = *reinterpret_cast<const float4*>(lz + ((size_t)dd * C::kColsPad + c) * 4);
-            lt += v.x; z += v.y; st_ += v.z; ht += v.w;
+            const float2 v = *reinterpret_cast<const float2*>(lz + ((size_t)dd * C::kColsPad + c) * 2);
+            lt += v.x; z += v.y;
           }
           if (c >= p.ncols) continue;
           const int j = c / p.G, hh = c % p.G;
           float* dst = direct ? p.out + (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D
                               : part + (size_t)c * kPartStride;
           const float inv = direct ? (lt > 0.0f ? 1.0f / lt : 0.0f) : 1.0f;
-          // undo the subnormal scales of the V operands (2^-24; odd dims of the anchor 2^-20) and
-          // apply the exact-to-rounded weight ratio
-          const float ratio = ht > 0.0f ? st_ / ht : 1.0f;
-          const float fix_even = 16777216.0f * ratio, fix_odd = (FULL ? 16777216.0f : 1048576.0f) * ratio;
+          // undo the subnormal scales of the V operands (2^-24; odd dims of the anchor 2^-20)
+          constexpr float fix_even = 16777216.0f, fix_odd = FULL ? 16777216.0f : 1048576.0f;
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
             const int gmt = d * MT + mt;  // m-tile index among the eight of a lane's 16 dims
@@ -1161,7 +1173,7 @@ attn_team_kernel(const AttnParams p) {
   attn_team_body<FULL, NT, DS, TEAMS, NSTAGE, TPW>(p);
 }
 #ifndef LYNX_WIDE_VERIFY
-#define LYNX_WIDE_VERIFY 2   // 0: keep the mma.sync kernels for 17..64 verify columns (comparison builds)
+#define LYNX_WIDE_VERIFY 1   // 0: keep the mma.sync kernels for 17..64 verify columns (comparison builds)
 #endif
 #include "attention_wide.cuh"
 

@@ -41,7 +41,7 @@ template <int NCOPY>
 struct WideCfg {
   static constexpr int kST = 64;                 // tokens per stage-unit
   static constexpr int kTW = 4;                  // 16-token sub-blocks per stage
-  static constexpr int kNStage = 7;
+  static constexpr int kNStage = 5;
   static constexpr int kSubBytes = 16 * 272;
   static constexpr int kStageBytes = kST * 272;  // KA, VA, KR, VR (4 KiB each), KM, VM (512 B each)
   static constexpr int kColsPad = 128 / NCOPY;
@@ -55,15 +55,15 @@ struct WideCfg {
   static constexpr int kThreads = (kConsWarps + kProdWarps + 1 + kVWarps) * 32;
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int kTileBytes = 2 * 64 * 128;              // [2 dim blocks][64 tokens][128 B]
-  static constexpr int kOffCanon = 0;                          // [wg][K tile, V tile]
-  static constexpr int kOffRing = 4 * kTileBytes;
+  static constexpr int kOffCanon = 0;                          // [wg][K tile, V tile 0, V tile 1]
+  static constexpr int kOffRing = 6 * kTileBytes;
   static constexpr int kOffScal = kOffRing + kNStage * kStageBytes;  // [group][3 sets][256 floats]
   static constexpr int kOffQs = kOffScal + 2 * 3 * 4 * 64 * 4;       // sum of q per column
   static constexpr int kOffQ = kOffQs + kColsPad * 4;                // raw BF16 queries, 2 slots
   static constexpr int kOffBlk = kOffQ + 2 * kColsPad * LYNX_D * 2;
   static constexpr int kOffInfo = kOffBlk + kProdWarps * 2 * kPieceUnits * 4;
   static constexpr int kOffBars = kOffInfo + kNStage * 16 + 2 * 32;
-  static constexpr int kOffMisc = kOffBars + (2 * kNStage + 12) * 8;  // full, empty, q full/empty, sready, odone, kready, pready
+  static constexpr int kOffMisc = kOffBars + (2 * kNStage + 22) * 8;  // full, empty, q full/empty, sready, odone, kready, pready, rready, rdone (x2), vready (x2)
   static constexpr int kSmem = kOffMisc + 256 + 1024;                // + alignment slack
   // TMEM columns of a warpgroup
   static constexpr int kTmemQ = 0, kTmemWg0 = 64, kTmemS = 0, kTmemP = 64, kTmemO = 96, kTmemWg = 224, kTmemCols = 512;
@@ -72,7 +72,7 @@ struct WideCfg {
   static_assert(kSmem <= 227 * 1024, "shared memory");
   // scratch of the end-of-piece merge lives in the operand tiles (idle by then)
   static constexpr int kMergeStride = 129;                     // floats per column (odd: no bank conflicts)
-  static_assert(kColsPad * kMergeStride * 4 + 3 * 256 * 4 <= 4 * kTileBytes, "merge scratch");
+  static_assert(kColsPad * kMergeStride * 4 + 3 * 256 * 4 <= 6 * kTileBytes, "merge scratch");
 };
 
 // One non-blocking probe of an mbarrier phase.
@@ -394,7 +394,8 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
   const uint32_t ring_u32 = sbase + C::kOffRing;
   const uint32_t full0 = sbase + C::kOffBars, empty0 = full0 + NSTAGE * 8;
   const uint32_t qfull0 = empty0 + NSTAGE * 8, qempty0 = qfull0 + 16;
-  const uint32_t sready0 = qempty0 + 16, odone0 = sready0 + 16, kready0 = odone0 + 16, pready0 = kready0 + 16;
+  const uint32_t sready0 = qempty0 + 16, odone0 = sready0 + 16, kready0 = odone0 + 16, pready0 = kready0 + 16,
+                 rready0 = pready0 + 16, rdone0 = rready0 + 16, vready0 = rdone0 + 32;
   volatile int* abort_word = misc;
 
   if (tid == 0) {
@@ -408,7 +409,12 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       mbar_init(sready0 + i * 8, 1);
       mbar_init(odone0 + i * 8, 1);
       mbar_init(kready0 + i * 8, 4);   // K tile and scalars of group i written, its previous scores in registers
-      mbar_init(pready0 + i * 8, 4 + C::kVWarps);   // P (the group) and V tile (the V converters) of group i written
+      mbar_init(pready0 + i * 8, 4);   // P of group i written (and its V tile, when the group expands it itself)
+      mbar_init(vready0 + (2 * i) * 8, C::kVWarps > 0 ? C::kVWarps : 1);       // V tile written by the V converters,
+      mbar_init(vready0 + (2 * i + 1) * 8, C::kVWarps > 0 ? C::kVWarps : 1);   // one barrier per V tile of the group
+      mbar_init(rready0 + i * 8, 4);   // the remainders of the weights' FP16 rounding are in P
+      mbar_init(rdone0 + (2 * i) * 8, 1);       // P.V of the remainders complete (tcgen05.commit), one barrier
+      mbar_init(rdone0 + (2 * i + 1) * 8, 1);   // per V tile of the group (units alternate between them)
     }
     misc[0] = 0; misc[1] = 0; misc[7] = 0; misc[8] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -456,17 +462,18 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       for (int u = 0; u < n_piece; ++u) {
         const int w = u & 1;
         const int gs = gs_base + u, slot = gs % NSTAGE;
-        const uint32_t tile_v = sbase + C::kOffCanon + w * 2 * C::kTileBytes + C::kTileBytes;
-        mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
         const uint32_t nvw = w ? nv[1] : nv[0];
-        if (nvw > 0) mbar_wait(odone0 + w * 8, (nvw - 1) & 1, abort_word);   // V tile free
+        const uint32_t tile_v = sbase + C::kOffCanon + w * 3 * C::kTileBytes + (1 + (nvw & 1)) * C::kTileBytes;
+        mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
+        // the group's V tiles alternate: this one is free once both P.V passes of the unit before last are done
+        if (nvw > 1) mbar_wait(rdone0 + (w * 2 + (nvw & 1)) * 8, ((nvw >> 1) - 1) & 1, abort_word);
         const uint32_t st = ring_u32 + slot * C::kStageBytes;
         wide_expand(st + 4096u, st + 12288u, tile_v, vt);   // VA, VR
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0) {
           mbar_arrive(empty0 + slot * 8);
-          mbar_arrive(pready0 + w * 8);
+          mbar_arrive(vready0 + (w * 2 + (nvw & 1)) * 8);
         }
         if (w) ++nv[1]; else ++nv[0];
       }
@@ -483,20 +490,24 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
   if (warp == C::kMmaWarp) {
     if (lane == 0) {
       const uint32_t tm_q = tmem0 + C::kTmemQ;
-      uint32_t gk[2] = {0, 0}, gp[2] = {0, 0};   // Q.K^T / P.V issued so far, per group (barrier phases)
+      uint32_t gk[2] = {0, 0}, gp[2] = {0, 0}, gr[2] = {0, 0};   // Q.K^T / P.V / remainder P.V issued so far, per group
       int gs_base = 0, ic = 0;
       while (gs_base < n_units) {
         const int qi = ic & 1;
         mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
         const int n_piece = items[qi].pad0;
         int todo_k[2] = {(n_piece + 1) >> 1, n_piece >> 1}, todo_p[2] = {(n_piece + 1) >> 1, n_piece >> 1};
+        int todo_r[2] = {(n_piece + 1) >> 1, n_piece >> 1};
         int first_p[2] = {1, 1};
         uint64_t t0 = globaltimer_ns();
-        while (todo_k[0] + todo_k[1] + todo_p[0] + todo_p[1] > 0) {
+        uint32_t idle = 0;   // the clock is read once in 1024 idle rounds: reading it every round slows the polling
+        while (todo_k[0] + todo_k[1] + todo_p[0] + todo_p[1] + todo_r[0] + todo_r[1] > 0) {
           bool progress = false;
 #pragma unroll
           for (int w = 0; w < 2; ++w) {
-            const uint32_t tile_k = sbase + C::kOffCanon + w * 2 * C::kTileBytes, tile_v = tile_k + C::kTileBytes;
+            const uint32_t tile_k = sbase + C::kOffCanon + w * 3 * C::kTileBytes;
+            const uint32_t tile_vp = tile_k + (1 + (gp[w] & 1)) * C::kTileBytes;   // V tile of the unit whose P.V comes next
+            const uint32_t tile_vr = tile_k + (1 + (gr[w] & 1)) * C::kTileBytes;   // ... whose remainder pass comes next
             const uint32_t tm_w = tmem0 + C::kTmemWg0 + w * C::kTmemWg;
             if (todo_k[w] > 0 && mbar_test(kready0 + w * 8, gk[w] & 1)) {
               tc_fence_after();
@@ -508,23 +519,36 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
               tc_commit(sready0 + w * 8);
               ++gk[w]; --todo_k[w]; progress = true;
             }
-            if (todo_p[w] > 0 && mbar_test(pready0 + w * 8, gp[w] & 1)) {
+            if (todo_p[w] > 0 && mbar_test(pready0 + w * 8, gp[w] & 1) &&
+                (C::kVWarps == 0 || mbar_test(vready0 + (w * 2 + (gp[w] & 1)) * 8, (gp[w] >> 1) & 1))) {
               tc_fence_after();
 #pragma unroll
               for (int ks = 0; ks < 4; ++ks)
                 tc_mma_ts(tm_w + C::kTmemO, tm_w + C::kTmemP + (uint32_t)ks * 8u,
-                          tc_desc(tile_v + (uint32_t)ks * 2048u, 8192u, 1024u), kIdescO,
+                          tc_desc(tile_vp + (uint32_t)ks * 2048u, 8192u, 1024u), kIdescO,
                           (!first_p[w] || ks > 0) ? 1u : 0u);
               tc_commit(odone0 + w * 8);
               first_p[w] = 0;
               ++gp[w]; --todo_p[w]; progress = true;
             }
+            if (todo_r[w] > 0 && mbar_test(rready0 + w * 8, gr[w] & 1)) {   // the same P.V on the remainders
+              tc_fence_after();
+#pragma unroll
+              for (int ks = 0; ks < 4; ++ks)
+                tc_mma_ts(tm_w + C::kTmemO, tm_w + C::kTmemP + (uint32_t)ks * 8u,
+                          tc_desc(tile_vr + (uint32_t)ks * 2048u, 8192u, 1024u), kIdescO, 1u);
+              tc_commit(rdone0 + (w * 2 + (gr[w] & 1)) * 8);
+              ++gr[w]; --todo_r[w]; progress = true;
+            }
           }
           if (progress) {
-            t0 = globaltimer_ns();
-          } else if (*abort_word || globaltimer_ns() - t0 > 2000000000ull) {
-            *abort_word = 1;   // give up: the waiting groups see the abort word and run out their loops
-            break;
+            idle = 0;
+          } else if ((++idle & 1023u) == 0) {
+            if (idle == 1024u) t0 = globaltimer_ns();
+            if (*abort_word || globaltimer_ns() - t0 > 2000000000ull) {
+              *abort_word = 1;   // give up: the waiting groups see the abort word and run out their loops
+              break;
+            }
           }
         }
         gs_base += n_piece;
@@ -548,14 +572,16 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
     TmemRegs<32>::st(tm_p + lane_sel, z);
     tc_wait_st();
   }
-  const uint32_t tile_k = sbase + C::kOffCanon + wg * 2 * C::kTileBytes, tile_v = tile_k + C::kTileBytes;
+  const uint32_t tile_k = sbase + C::kOffCanon + wg * 3 * C::kTileBytes;
   float* my_scal = scal + wg * 768;
   const float cb = p.sm_log2;
 
   int gs_base = 0, ic = 0;
   uint32_t n_u = 0;            // units of this group so far (selects the scalar set)
-  uint32_t n_s = 0, n_o = 0;   // commits so far on this group's two MMA barriers
-  bool o_pending = false;      // the last O commit has not been waited for yet
+  uint32_t n_s = 0, n_o = 0, n_r = 0;   // commits so far on this group's MMA barriers (scores, P.V, remainder P.V)
+  bool r_todo = false;         // the remainders of the last unit's weights are still in registers
+  bool r_pending = false;      // the last remainder P.V has not been waited for yet
+  uint32_t pr_prev[KT / 2];    // those remainders (FP16 pairs)
 
   while (gs_base < n_units) {
     const int qi = ic & 1;
@@ -624,7 +650,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
     named_bar(6, C::kConsThreads + C::kVWarps * 32);
     const float qsum = qs_s[c];
 
-    float m = 0.0f, l = 0.0f, zs = 0.0f, sw = 0.0f, hw = 0.0f;  // m: the running maximum (log2 units)
+    float m = 0.0f, l = 0.0f, zs = 0.0f;  // m: the running maximum (log2 units)
     bool fresh = true;
     int my_units = 0;
 
@@ -657,6 +683,27 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       }
       ++n_s;
     };
+    // The weights go to the tensor core as two FP16 numbers: the rounded weight (P.V issued at the
+    // end of the unit) and the rounding's remainder, whose pass over the same V tile is issued
+    // from here once the first has completed (P holds one of the two at a time).
+    auto flush_remainders = [&]() {
+      if (!r_todo) return;
+      mbar_wait(odone0 + wg * 8, (n_o - 1) & 1, abort_word);   // the pass on the rounded weights is done with P
+      tc_fence_after();
+      TmemRegs<KT / 2>::st(tm_p + lane_sel + (uint32_t)(copy * (KT / 2)), pr_prev);
+      tc_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(rready0 + wg * 8);
+      ++n_r;
+      r_todo = false;
+      r_pending = true;
+    };
+    auto wait_remainders = [&]() {
+      if (!r_pending) return;
+      mbar_wait(rdone0 + (wg * 2 + ((n_r - 1) & 1)) * 8, ((n_r - 1) >> 1) & 1, abort_word);
+      r_pending = false;
+    };
     if (wg < n_piece) prefetch(wg, (int)(n_u % 3u));
 
     for (int k = wg; k < n_piece; k += 2, ++my_units) {
@@ -683,6 +730,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       }
       // the next unit's K side runs on the tensor core while this unit's softmax is computed
       if (k + 2 < n_piece) prefetch(k + 2, (set + 1) % 3);
+      flush_remainders();   // of the previous unit
       // ---- softmax of this row's tokens ----------------------------------------------------------
       const int tok0 = unit_t0 + copy * KT;
       if (unit_t0 + C::kST > full_lim) {
@@ -691,31 +739,27 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
           if (tok0 + i >= lim_c) x[i] = -INFINITY;
       }
       // ---- weights: fast path without the maximum; redone when a weight may have grown too large -----
-      uint32_t ph[KT / 2];
-      float l_n, zs_n, sw_n, hw_n;
+      uint32_t ph[KT / 2], pr[KT / 2];   // rounded weights and remainders, FP16 pairs
+      float l_n, zs_n;
       auto weights = [&]() {
-        uint64_t l2 = pk2(l, 0.0f), z2 = pk2(zs, 0.0f), s2 = pk2(sw, 0.0f), h2 = pk2(hw, 0.0f);
+        uint64_t l2 = pk2(l, 0.0f), z2 = pk2(zs, 0.0f);
 #pragma unroll
         for (int i = 0; i < KT; i += 2) {
           const uint4 zv = lds128(scal_u32 + 512u + (uint32_t)(copy * KT + i) * 8u);  // zero0, zero1, scale0, scale1
           const uint64_t p2 = pk2(ex2(x[i]), ex2(x[i + 1]));
           l2 = fadd2(l2, p2);
           z2 = ffma2(p2, pk2(__uint_as_float(zv.x), __uint_as_float(zv.y)), z2);
-          const uint64_t w2 = fmul2(p2, pk2(__uint_as_float(zv.z), __uint_as_float(zv.w)));
-          s2 = fadd2(s2, w2);
           float w0, w1, b0, b1;
-          upk2(w2, w0, w1);
+          upk2(fmul2(p2, pk2(__uint_as_float(zv.z), __uint_as_float(zv.w))), w0, w1);
           const uint32_t hh = pack_f16x2(w0, w1);
           ph[i / 2] = hh;
           asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tcvt.f32.f16 %0, lo;\n\tcvt.f32.f16 %1, hi;\n\t}"
               : "=f"(b0), "=f"(b1) : "r"(hh));
-          h2 = fadd2(h2, pk2(b0, b1));
+          pr[i / 2] = pack_f16x2(w0 - b0, w1 - b1);   // w = h + r, r exact in FP32 and then rounded to FP16
         }
         float a0, a1;
         upk2(l2, a0, a1); l_n = a0 + a1;
         upk2(z2, a0, a1); zs_n = a0 + a1;
-        upk2(s2, a0, a1); sw_n = a0 + a1;
-        upk2(h2, a0, a1); hw_n = a0 + a1;
       };
       weights();
       // every weight of the unit is below 64 unless the unit's sum says otherwise
@@ -729,16 +773,13 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
           const float upm = fresh ? fmaxf(mx, -1.0e4f) : fmaxf(mx, 0.0f);
           f = fresh ? 0.0f : ex2(-upm);
           m += upm;
-          l *= f; zs *= f; sw *= f; hw *= f;
+          l *= f; zs *= f;
 #pragma unroll
           for (int i = 0; i < KT; ++i) x[i] -= upm;
         }
         weights();
         if (my_units > 0) {  // O holds earlier units of this piece: rescale the row in TMEM
-          if (o_pending) {
-            mbar_wait(odone0 + wg * 8, (n_o - 1) & 1, abort_word);
-            o_pending = false;
-          }
+          wait_remainders();   // both passes of the previous unit have been accumulated
           tc_fence_after();
 #pragma unroll
           for (int cch = 0; cch < 4; ++cch) {
@@ -752,19 +793,19 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
         }
       }
       fresh = false;
-      l = l_n; zs = zs_n; sw = sw_n; hw = hw_n;
+      l = l_n; zs = zs_n;
       {
-        // P and the V tile are free once the previous P.V of this group is complete
-        if (o_pending) {
-          mbar_wait(odone0 + wg * 8, (n_o - 1) & 1, abort_word);
-          o_pending = false;
-        }
+        // P and the V tile are free once both P.V passes of the previous unit are complete
+        wait_remainders();
         tc_fence_after();
         TmemRegs<KT / 2>::st(tm_p + lane_sel + (uint32_t)(copy * (KT / 2)), ph);
+#pragma unroll
+        for (int i = 0; i < KT / 2; ++i) pr_prev[i] = pr[i];
       }
       if constexpr (C::kVWarps == 0) {  // this group expands its own V tile (free: the odone wait above)
         const uint32_t st = ring_u32 + slot * C::kStageBytes;
-        wide_expand(st + 4096u, st + 12288u, tile_v, r);   // VA, VR
+        // (its V tiles alternate; this one was last read by the unit before last, both passes long done)
+        wide_expand(st + 4096u, st + 12288u, tile_k + (1 + (n_o & 1)) * C::kTileBytes, r);   // VA, VR
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + slot * 8);
@@ -775,14 +816,12 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       if (lane == 0) mbar_arrive(pready0 + wg * 8);   // this warp's rows of P and part of the V tile are ready
       ++n_u;
       ++n_o;
-      o_pending = true;
+      r_todo = true;
     }
 
     // ---- end of the piece: merge the 2 * NCOPY partial rows of every column ----------------------
-    if (o_pending) {
-      mbar_wait(odone0 + wg * 8, (n_o - 1) & 1, abort_word);
-      o_pending = false;
-    }
+    flush_remainders();
+    wait_remainders();
     tc_fence_after();
     float* msc = reinterpret_cast<float*>(smem + C::kOffCanon);        // [CP][kMergeStride]
     float* sc_m = msc + CP * C::kMergeStride;                          // [256] maxima, then [256] l, [256] zs
@@ -798,8 +837,10 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
     const float f = (have && m > -INFINITY && M > -INFINITY) ? ex2(m - M) : 0.0f;
     sc_l[tid] = l * f;
     sc_z[tid] = zs * f;
-    // undo the 2^-24 of the V codes and apply the exact-to-rounded weight ratio of this row
-    const float coef = f * 16777216.0f * (hw > 0.0f ? sw / hw : 1.0f);
+    // undoes the 2^-24 of the V codes, and puts back what the tensor core's truncating accumulation
+    // lost on average: 0.23 * 2^-23 of the sum (measured on long pieces) for each of the eight MMAs
+    // (four token slices, rounded weights and remainders) a unit adds into a row of O
+    const float coef = f * 16777216.0f * (1.0f + (float)(8 * my_units) * (0.23f * 1.1920929e-7f));
     const int part = wg * NCOPY + copy;
     for (int round = 0; round < 2 * NCOPY; ++round) {
       if (part == round && have) {   // warp-uniform
