@@ -593,7 +593,7 @@ __device__ __forceinline__ void k_fragments(uint32_t st, int r0, int t, uint32_t
 // O^T slice += level(V)^T[slice dims x 16 tokens] . P^T for one tile (stage rows row0..row0+15).
 // Slice d of DS covers the m-tiles (word, half) of every lane's 16 dims: DS=1 all eight, DS=2
 // word d, DS=4 word d>>1 / half d&1.
-template <bool FULL, int NT, int ST, int DS>
+template <bool FULL, int NT, int ST, int DS, bool TWO>
 __device__ __forceinline__ void pv_slice(float (&o)[NT][8 / DS][4], uint32_t st, int row0, int g, int t,
                                          int d, const uint32_t (&pb)[NT][4]) {
   constexpr uint32_t VA = ST * 64, VR = ST * 192;
@@ -663,15 +663,18 @@ __device__ __forceinline__ void pv_slice(float (&o)[NT][8 / DS][4], uint32_t st,
         for (int nt = 0; nt < NT; ++nt)
         {  // the rounded weights, then the remainders of their rounding
           mma16816(o[nt][lm], ab[2 * qd], ab[2 * qd + 1], cd[2 * qd], cd[2 * qd + 1], pb[nt][0], pb[nt][1]);
-          mma16816(o[nt][lm], ab[2 * qd], ab[2 * qd + 1], cd[2 * qd], cd[2 * qd + 1], pb[nt][2], pb[nt][3]);
+          if (TWO) mma16816(o[nt][lm], ab[2 * qd], ab[2 * qd + 1], cd[2 * qd], cd[2 * qd + 1], pb[nt][2], pb[nt][3]);
         }
       }
     }
   }
 }
 
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int TPW>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int TPW, bool PACK>
 __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
+  // PACK (at most four query columns): columns 4..7 of the n-tile repeat columns 0..3 and carry the
+  // remainders of the weights' rounding, so one MMA per operand does the work of two
+  static_assert(!PACK || (NT == 1 && DS == 1), "column packing is for the single n-tile kernels");
   using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE, TPW>;
   constexpr int ST = C::kST, TW = C::kTW, MT = C::kMT;
   constexpr uint32_t KM = FULL ? ST * 256 : ST * 128, VM = KM + ST * 8;
@@ -739,6 +742,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
   float m[NT][2], l[NT][2], zs[NT][2], o[NT][MT][4];
   const uint32_t qf_u32 = smem_u32(qf_s), qs_u32 = smem_u32(qs_s);
   auto col_limit = [&](int col, int len_) {
+    if (PACK) col &= 3;
     return col < p.ncols ? (p.causal ? len_ - p.nq + col / p.G + 1 : len_) : 0;
   };
   bool fresh = true;
@@ -781,7 +785,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
         // warp w builds the shared fragments of the n-tiles nt = w, w + (consumer warps), ... for everybody
         const bool mine = (nt % C::kConsWarps) == warp;
         if (mine) {
-          const int c = nt * 8 + g;
+          const int c = PACK ? (g & 3) : nt * 8 + g;
 #pragma unroll
           for (int wd = 0; wd < 4; ++wd) {
             const uint4 v = *reinterpret_cast<const uint4*>(qb + c * LYNX_D + 32 * t + 8 * wd);
@@ -808,7 +812,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
             const int col = nt * 8 + 2 * t + cc;
-            const uint4* qq = reinterpret_cast<const uint4*>(qb + col * LYNX_D + 16 * g);
+            const uint4* qq = reinterpret_cast<const uint4*>(qb + (PACK ? (col & 3) : col) * LYNX_D + 16 * g);
             float sum = 0.0f;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
@@ -996,6 +1000,12 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
         unpack_f16x2(h01, b0, b1);
         unpack_f16x2(h23, b2, b3);
         const uint32_t r01 = pack_f16x2(w0 - b0, w1 - b1), r23 = pack_f16x2(w2 - b2, w3 - b3);
+        if constexpr (PACK) {   // columns 0..3: the rounded weights; their repeats 4..7: the remainders
+          pown[nt][0] = movmatrix_trans(t >= 2 ? r01 : h01);
+          pown[nt][1] = movmatrix_trans(t >= 2 ? r23 : h23);
+          pown[nt][2] = 0u; pown[nt][3] = 0u;
+          continue;
+        }
         const uint32_t f0 = movmatrix_trans(h01), f1 = movmatrix_trans(h23);
         const uint32_t f2 = movmatrix_trans(r01), f3 = movmatrix_trans(r23);
         if constexpr (DS > 1) {
@@ -1012,8 +1022,8 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
     // ---- phase C: P.V of the team's tiles for this warp's slice of the output dims --------
     if constexpr (DS == 1) {
       if (valid) {
-        pv_slice<FULL, NT, ST, 1>(o, st, wt * 16, g, t, 0, pown);
-        n_mma += 2;   // into every accumulator: the rounded weights and their remainders
+        pv_slice<FULL, NT, ST, 1, !PACK>(o, st, wt * 16, g, t, 0, pown);
+        n_mma += PACK ? 1 : 2;   // into every accumulator: the rounded weights and their remainders
       }
     }
 #pragma unroll
@@ -1027,7 +1037,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) pb[nt][i] = *reinterpret_cast<const volatile uint32_t*>(pf + (nt * 4 + i) * 32);
       }
-      pv_slice<FULL, NT, ST, DS>(o, st, src * 16, g, t, d, pb);
+      pv_slice<FULL, NT, ST, DS, true>(o, st, src * 16, g, t, d, pb);
       n_mma += 2;
     }
     }  // if (DS > 1 || in_range)
@@ -1044,7 +1054,11 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-          for (int i = 0; i < 4; ++i) o[nt][mt][i] *= back;
+          for (int i = 0; i < 4; ++i) {
+            o[nt][mt][i] *= back;
+            // the remainders' part, accumulated under the repeated columns, joins its column
+            if (PACK) o[nt][mt][i] += __shfl_xor_sync(0xFFFFFFFFu, o[nt][mt][i], 2);
+          }
     }
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) { m[nt][0] = -m[nt][0]; m[nt][1] = -m[nt][1]; }  // back to the maximum
@@ -1167,10 +1181,10 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 
 // At least MINB CTAs per SM (the compiler caps registers accordingly).  Nine warps cannot
 // have more than 168 registers each: three of them share one SM sub-partition's 16 K registers.
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB, int TPW>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB, int TPW, bool PACK>
 __global__ void __launch_bounds__((DS * TEAMS + 1) * 32, MINB)
 attn_team_kernel(const AttnParams p) {
-  attn_team_body<FULL, NT, DS, TEAMS, NSTAGE, TPW>(p);
+  attn_team_body<FULL, NT, DS, TEAMS, NSTAGE, TPW, PACK>(p);
 }
 #ifndef LYNX_WIDE_VERIFY
 #define LYNX_WIDE_VERIFY 1   // 0: keep the mma.sync kernels for 17..64 verify columns (comparison builds)
@@ -1212,14 +1226,14 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   return true;
 }
 
-template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB, int TPW = 1>
+template <bool FULL, int NT, int DS, int TEAMS, int NSTAGE, int MINB, int TPW = 1, bool PACK = false>
 lynx_status launch_team(const AttnParams& p, cudaStream_t st) {
   using C = TeamCfg<FULL, NT, DS, TEAMS, NSTAGE, TPW>;
   static_assert(MINB <= kMaxCtasPerSm, "partial slots are sized for kMaxCtasPerSm CTAs per SM");
   constexpr int kCtasPerSm = MINB;
   static_assert(kCtasPerSm * (C::kSmem + 1024) <= 228 * 1024, "shared memory budget per SM");
   static_assert(2 + TEAMS <= 16, "named barriers");
-  auto kern = attn_team_kernel<FULL, NT, DS, TEAMS, NSTAGE, MINB, TPW>;
+  auto kern = attn_team_kernel<FULL, NT, DS, TEAMS, NSTAGE, MINB, TPW, PACK>;
   static bool configured[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -1284,7 +1298,9 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   // <FULL, NT, DS, TEAMS, stages, CTAs/SM>
   if (!full) {
     switch (pl.variant) {
-      case 0: return launch_team<false, 1, 1, 4, 2, 4, 2>(p, st);   // two tiles per warp and stage
+      case 0:   // two tiles per warp and stage
+        if (pl.ncols <= 4) return launch_team<false, 1, 1, 4, 2, 4, 2, true>(p, st);
+        return launch_team<false, 1, 1, 4, 2, 4, 2>(p, st);
       case 1: return launch_team<false, 2, 2, 2, 4, 3>(p, st);
       case 2: return launch_team<false, 4, 4, 1, 3, 3>(p, st);
       default: return launch_team<false, 8, 4, 2, 3, 1>(p, st);
@@ -1297,7 +1313,9 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
 #endif
 #endif
   switch (pl.variant) {
-    case 0: return launch_team<true, 1, 1, 4, 3, 3>(p, st);
+    case 0:
+      if (pl.ncols <= 4) return launch_team<true, 1, 1, 4, 3, 3, 1, true>(p, st);
+      return launch_team<true, 1, 1, 4, 3, 3>(p, st);
     case 1: return launch_team<true, 2, 2, 2, 3, 3>(p, st);
     case 2: return launch_team<true, 4, 4, 1, 2, 3>(p, st);
     default: return launch_team<true, 8, 4, 2, 3, 1>(p, st);
