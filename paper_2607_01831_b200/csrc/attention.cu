@@ -13,7 +13,7 @@
 // s8 digit planes of the query).  P.V runs in FP16 with the levels as FP16 subnormals (the bit
 // pattern 0x00cc is code * 2^-24: no conversion arithmetic) and the weights p * scale as the sum
 // of two FP16 numbers (the rounded weight and the rounding's remainder, each with its own MMA), so
-// the weights carry about 22 bits.  From 17 columns on the verify pass runs on tcgen05
+// the weights carry about 22 bits.  From 33 columns on the verify pass runs on tcgen05
 // (attention_wide.cuh).
 //
 // Kernel shape.  Persistent grid (a few CTAs per SM), flash-decoding split-K in stream-K form:

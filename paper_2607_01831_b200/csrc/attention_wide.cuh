@@ -1,13 +1,16 @@
-// Merge-verify attention for 17..64 columns on the fifth-generation tensor cores (tcgen05, TMEM).
+// Merge-verify attention for 33..64 columns on the fifth-generation tensor cores (tcgen05, TMEM;
+// the 32-column instantiation is kept for comparison builds).
 // Included by attention.cu inside its namespace: shares the stream-K cut of the work, the piece
 // bookkeeping and finish_piece with the mma.sync kernels.
 //
-// With k*G >= 17 query rows per KV head the verify pass of Section 4.3 is a dense contraction
-// (about 60 / 120 flop per plane byte at 32 / 64 columns), which the mma.sync kernels cannot
-// feed: their tensor pipe would have to be busier than 100 % at the HBM roofline.  Here the two
+// With this many query rows per KV head the verify pass of Section 4.3 is a dense contraction
+// (about 120 flop per plane byte at 64 columns), which the mma.sync kernels cannot feed: their
+// tensor pipe would have to be busier than 100 % at the HBM roofline.  Here the two
 // contractions of a 64-token stage-unit are two tcgen05.mma groups with M = 128:
 //   S[128 rows x 64 tokens]  = Q[128 x 128 dims] . codes(K)^T      A = Q in TMEM, B in shared memory
 //   O[128 rows x 128 dims]  += P[128 x 64 tokens] . codes(V)       A = P in TMEM, B in shared memory
+// The weights go in as two FP16 terms, p * scale_v = h + r (the rounded weight and the rounding's
+// remainder): P holds h for a first pass and r for a second pass over the same V tile.
 // Row r of the M = 128 is (copy, column): the k*G columns (padded to 32 or 64) are replicated
 // NCOPY = 4 or 2 times and copy i owns tokens [i*64/NCOPY, (i+1)*64/NCOPY) of the unit: its P
 // entries for the other tokens stay zero, so every row is an independent flash-decoding split
