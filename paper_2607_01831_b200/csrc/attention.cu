@@ -13,7 +13,7 @@
 // s8 digit planes of the query).  P.V runs in FP16 with the levels as FP16 subnormals (the bit
 // pattern 0x00cc is code * 2^-24: no conversion arithmetic) and the weights p * scale as the sum
 // of two FP16 numbers (the rounded weight and the rounding's remainder, each with its own MMA), so
-// the weights carry about 22 bits.  From 33 columns on the verify pass runs on tcgen05
+// the weights carry about 22 bits.  From 17 columns on the verify pass runs on tcgen05
 // (attention_wide.cuh).
 //
 // Kernel shape.  Persistent grid (a few CTAs per SM), flash-decoding split-K in stream-K form:
@@ -1187,7 +1187,7 @@ attn_team_kernel(const AttnParams p) {
   attn_team_body<FULL, NT, DS, TEAMS, NSTAGE, TPW, PACK>(p);
 }
 #ifndef LYNX_WIDE_VERIFY
-#define LYNX_WIDE_VERIFY 1   // 0: keep the mma.sync kernels for 17..64 verify columns (comparison builds)
+#define LYNX_WIDE_VERIFY 2   // 0: keep the mma.sync kernels for 17..64 verify columns (comparison builds)
 #endif
 #include "attention_wide.cuh"
 
@@ -1307,9 +1307,9 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
     }
   }
 #if LYNX_WIDE_VERIFY
-  if (pl.variant == 3) return launch_wide<2>(p, st);
+  if (pl.variant == 3) return launch_wide<2, 1>(p, st);
 #if LYNX_WIDE_VERIFY > 1
-  if (pl.variant == 2) return launch_wide<4>(p, st);
+  if (pl.variant == 2) return launch_wide<2, 2>(p, st);
 #endif
 #endif
   switch (pl.variant) {

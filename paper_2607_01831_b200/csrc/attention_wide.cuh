@@ -1,5 +1,4 @@
-// Merge-verify attention for 33..64 columns on the fifth-generation tensor cores (tcgen05, TMEM;
-// the 32-column instantiation is kept for comparison builds).
+// Merge-verify attention for 17..64 columns on the fifth-generation tensor cores (tcgen05, TMEM).
 // Included by attention.cu inside its namespace: shares the stream-K cut of the work, the piece
 // bookkeeping and finish_piece with the mma.sync kernels.
 //
@@ -10,9 +9,11 @@
 //   S[128 rows x 64 tokens]  = Q[128 x 128 dims] . codes(K)^T      A = Q in TMEM, B in shared memory
 //   O[128 rows x 128 dims]  += P[128 x 64 tokens] . codes(V)       A = P in TMEM, B in shared memory
 // The weights go in as two FP16 terms, p * scale_v = h + r (the rounded weight and the rounding's
-// remainder): P holds h for a first pass and r for a second pass over the same V tile.
-// Row r of the M = 128 is (copy, column): the k*G columns (padded to 32 or 64) are replicated
-// NCOPY = 4 or 2 times and copy i owns tokens [i*64/NCOPY, (i+1)*64/NCOPY) of the unit: its P
+// remainder).  With up to 32 columns the two terms have rows of their own in the M = 128 and one
+// pass does both; with 64 columns P holds h for a first pass and r for a second pass over the
+// same V tile.
+// Row r of the M = 128 is (term, copy, column): the k*G columns (padded to 32 or 64) are replicated
+// NCOPY times and copy i owns tokens [i*64/NCOPY, (i+1)*64/NCOPY) of the unit: its P
 // entries for the other tokens stay zero, so every row is an independent flash-decoding split
 // with its own running maximum and all 128 TMEM lanes (threads) have softmax work.  Rows are
 // merged at the end of a piece.
@@ -25,7 +26,7 @@
 //     weights p * scale_v to its part of P.  It also expands the NEXT unit's K planes into the
 //     K tile (so that S of the next unit is computed under this unit's softmax) and, in the
 //     64-column variant, its own V tile.
-//   4 V converter warps (32-column variant) expand the V planes.
+//   (4 V converter warps expand the V planes in instantiations with four token copies.)
 //   3 producer warps stream the raw planes into a shared-memory ring (cp.async.bulk, 8 of the
 //     24 copies of a unit each: one warp issuing all of them caps at about 2.7 TB/s).
 //   1 MMA warp: one thread polls the "operands ready" mbarriers and issues every tcgen05.mma
@@ -40,14 +41,18 @@
 // position -> element within a group of 8: {0,4,2,6,1,5,3,7}, the 3-bit reversal
 __host__ __device__ constexpr int wide_perm(int pos) { return ((pos & 1) << 2) | (pos & 2) | ((pos >> 2) & 1); }
 
-template <int NCOPY>
+// NCOPY: token slices of a unit, each with its own rows.  TERMS = 1: a row's weights go in as two
+// P.V passes (rounded weights, then remainders); TERMS = 2: the rounded weights and the remainders
+// have rows of their own and one pass does both (half as many columns fit).
+template <int NCOPY, int TERMS>
 struct WideCfg {
+  static constexpr int kRows = NCOPY * TERMS;    // rows of the M = 128 per column
   static constexpr int kST = 64;                 // tokens per stage-unit
   static constexpr int kTW = 4;                  // 16-token sub-blocks per stage
-  static constexpr int kNStage = 5;
+  static constexpr int kNStage = TERMS == 2 ? 6 : 5;   // what fits beside the operand tiles and the query slots
   static constexpr int kSubBytes = 16 * 272;
   static constexpr int kStageBytes = kST * 272;  // KA, VA, KR, VR (4 KiB each), KM, VM (512 B each)
-  static constexpr int kColsPad = 128 / NCOPY;
+  static constexpr int kColsPad = 128 / kRows;
   static constexpr int kTok = kST / NCOPY;       // tokens of a unit that one row owns
   static constexpr int kConsWarps = 8;
   static constexpr int kConsThreads = 256;
@@ -378,9 +383,10 @@ __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int l
   }
 }
 
-template <int NCOPY>
-__global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(const AttnParams p) {
-  using C = WideCfg<NCOPY>;
+template <int NCOPY, int TERMS>
+__global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_kernel(const AttnParams p) {
+  using C = WideCfg<NCOPY, TERMS>;
+  constexpr int NR = C::kRows;
   constexpr int NSTAGE = C::kNStage, KT = C::kTok, CP = C::kColsPad;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -500,7 +506,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
         mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
         const int n_piece = items[qi].pad0;
         int todo_k[2] = {(n_piece + 1) >> 1, n_piece >> 1}, todo_p[2] = {(n_piece + 1) >> 1, n_piece >> 1};
-        int todo_r[2] = {(n_piece + 1) >> 1, n_piece >> 1};
+        int todo_r[2] = {TERMS == 1 ? (n_piece + 1) >> 1 : 0, TERMS == 1 ? n_piece >> 1 : 0};
         int first_p[2] = {1, 1};
         uint64_t t0 = globaltimer_ns();
         uint32_t idle = 0;   // the clock is read once in 1024 idle rounds: reading it every round slows the polling
@@ -531,6 +537,10 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
                           tc_desc(tile_vp + (uint32_t)ks * 2048u, 8192u, 1024u), kIdescO,
                           (!first_p[w] || ks > 0) ? 1u : 0u);
               tc_commit(odone0 + w * 8);
+              if (TERMS == 2) {   // no second pass: the V tile is free with this one
+                tc_commit(rdone0 + (w * 2 + (gr[w] & 1)) * 8);
+                ++gr[w];
+              }
               first_p[w] = 0;
               ++gp[w]; --todo_p[w]; progress = true;
             }
@@ -562,7 +572,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
   }
   const int wg = warp >> 2, w4 = warp & 3;
   const int r = tid & 127;                       // row of the M = 128 = TMEM lane
-  const int copy = r / CP, c = r % CP;           // warp-uniform copy
+  const int copy = (r / CP) % NCOPY, term = r / (CP * NCOPY), c = r % CP;   // warp-uniform copy and term
   const uint32_t lane_sel = (uint32_t)(w4 * 32) << 16;
   const uint32_t tm_q = tmem0 + C::kTmemQ;
   const uint32_t tm_s = tmem0 + C::kTmemWg0 + wg * C::kTmemWg + C::kTmemS;
@@ -691,6 +701,12 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
     // from here once the first has completed (P holds one of the two at a time).
     auto flush_remainders = [&]() {
       if (!r_todo) return;
+      r_todo = false;
+      if (TERMS == 2) {   // one pass: only its completion is still to be waited for
+        ++n_r;
+        r_pending = true;
+        return;
+      }
       mbar_wait(odone0 + wg * 8, (n_o - 1) & 1, abort_word);   // the pass on the rounded weights is done with P
       tc_fence_after();
       TmemRegs<KT / 2>::st(tm_p + lane_sel + (uint32_t)(copy * (KT / 2)), pr_prev);
@@ -755,10 +771,15 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
           float w0, w1, b0, b1;
           upk2(fmul2(p2, pk2(__uint_as_float(zv.z), __uint_as_float(zv.w))), w0, w1);
           const uint32_t hh = pack_f16x2(w0, w1);
-          ph[i / 2] = hh;
           asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tcvt.f32.f16 %0, lo;\n\tcvt.f32.f16 %1, hi;\n\t}"
               : "=f"(b0), "=f"(b1) : "r"(hh));
-          pr[i / 2] = pack_f16x2(w0 - b0, w1 - b1);   // w = h + r, r exact in FP32 and then rounded to FP16
+          const uint32_t rr = pack_f16x2(w0 - b0, w1 - b1);   // w = h + r, r exact in FP32 and then rounded to FP16
+          if (TERMS == 2) {
+            ph[i / 2] = term ? rr : hh;   // the rows of the second term carry the remainders
+          } else {
+            ph[i / 2] = hh;
+            pr[i / 2] = rr;
+          }
         }
         float a0, a1;
         upk2(l2, a0, a1); l_n = a0 + a1;
@@ -803,7 +824,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
         tc_fence_after();
         TmemRegs<KT / 2>::st(tm_p + lane_sel + (uint32_t)(copy * (KT / 2)), ph);
 #pragma unroll
-        for (int i = 0; i < KT / 2; ++i) pr_prev[i] = pr[i];
+        for (int i = 0; i < KT / 2; ++i) pr_prev[i] = TERMS == 1 ? pr[i] : 0u;
       }
       if constexpr (C::kVWarps == 0) {  // this group expands its own V tile (free: the odone wait above)
         const uint32_t st = ring_u32 + slot * C::kStageBytes;
@@ -822,7 +843,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
       r_todo = true;
     }
 
-    // ---- end of the piece: merge the 2 * NCOPY partial rows of every column ----------------------
+    // ---- end of the piece: merge the 2 * NR partial rows of every column ----------------------------
     flush_remainders();
     wait_remainders();
     tc_fence_after();
@@ -836,16 +857,16 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
     named_bar(1, C::kConsThreads);
     float M = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < 2 * NCOPY; ++i) M = fmaxf(M, sc_m[(i / NCOPY) * 128 + (i % NCOPY) * CP + c]);
+    for (int i = 0; i < 2 * NR; ++i) M = fmaxf(M, sc_m[(i / NR) * 128 + (i % NR) * CP + c]);
     const float f = (have && m > -INFINITY && M > -INFINITY) ? ex2(m - M) : 0.0f;
-    sc_l[tid] = l * f;
-    sc_z[tid] = zs * f;
+    sc_l[tid] = term == 0 ? l * f : 0.0f;   // the rows of the second term repeat the first term's sums
+    sc_z[tid] = term == 0 ? zs * f : 0.0f;
     // undoes the 2^-24 of the V codes, and puts back what the tensor core's truncating accumulation
-    // lost on average: 0.23 * 2^-23 of the sum (measured on long pieces) for each of the eight MMAs
-    // (four token slices, rounded weights and remainders) a unit adds into a row of O
-    const float coef = f * 16777216.0f * (1.0f + (float)(8 * my_units) * (0.23f * 1.1920929e-7f));
-    const int part = wg * NCOPY + copy;
-    for (int round = 0; round < 2 * NCOPY; ++round) {
+    // lost on average: 0.23 * 2^-23 of the sum (measured on long pieces) for each of the MMAs a unit
+    // adds into a row of O (four token slices a pass)
+    const float coef = f * 16777216.0f * (1.0f + (float)((TERMS == 1 ? 8 : 4) * my_units) * (0.23f * 1.1920929e-7f));
+    const int part = wg * NR + r / CP;
+    for (int round = 0; round < 2 * NR; ++round) {
       if (part == round && have) {   // warp-uniform
 #pragma unroll
         for (int cch = 0; cch < 4; ++cch) {
@@ -874,9 +895,9 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
         const int cc = idx >> 7, d = idx & 127;
         float lt = 0.0f, z = 0.0f;
 #pragma unroll
-        for (int i = 0; i < 2 * NCOPY; ++i) {
-          lt += sc_l[(i / NCOPY) * 128 + (i % NCOPY) * CP + cc];
-          z += sc_z[(i / NCOPY) * 128 + (i % NCOPY) * CP + cc];
+        for (int i = 0; i < 2 * NR; ++i) {
+          lt += sc_l[(i / NR) * 128 + (i % NR) * CP + cc];
+          z += sc_z[(i / NR) * 128 + (i % NR) * CP + cc];
         }
         const float v = msc[cc * C::kMergeStride + d] + z;
         if (direct) {
@@ -888,7 +909,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
           if (d == 0) {
             float Mc = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 2 * NCOPY; ++i) Mc = fmaxf(Mc, sc_m[(i / NCOPY) * 128 + (i % NCOPY) * CP + cc]);
+            for (int i = 0; i < 2 * NR; ++i) Mc = fmaxf(Mc, sc_m[(i / NR) * 128 + (i % NR) * CP + cc]);
             part_dst[(size_t)cc * kPartStride + 128] = Mc > -INFINITY ? Mc : -1.0e30f;
             part_dst[(size_t)cc * kPartStride + 129] = lt;
           }
@@ -913,10 +934,10 @@ __global__ void __launch_bounds__(WideCfg<NCOPY>::kThreads, 1) attn_wide_kernel(
   if (tid == 0 && misc[0]) atomicOr(p.ws_flags, kFlagTimeout);
 }
 
-template <int NCOPY>
+template <int NCOPY, int TERMS>
 lynx_status launch_wide(const AttnParams& p, cudaStream_t st) {
-  using C = WideCfg<NCOPY>;
-  auto kern = attn_wide_kernel<NCOPY>;
+  using C = WideCfg<NCOPY, TERMS>;
+  auto kern = attn_wide_kernel<NCOPY, TERMS>;
   static bool configured[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
