@@ -61,6 +61,7 @@ struct AttnParams {
   uint32_t* ws_flags;
   uint32_t* ws_chunk_ctr;  // [B*Hkv]
   uint32_t* ws_seq_ctr;    // [B]
+  uint32_t* ws_group_ctr;  // [2 * CTAs of the largest grid]: tickets of the groups of partial slots
   float* ws_dev;           // [B*Hkv][kMaxQ]
   float* ws_part;          // [B*Hkv + CTAs][ncols_pad][kPartStride], slot = segment + CTA index
   float atol, rtol;
@@ -260,29 +261,54 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
   const size_t bh = (size_t)item.b * p.Hkv + item.hkv;
   bool final_here = direct;
   if (!direct) {
-    // the last contributor of this (sequence, KV head) merges the partial slots
+    // The partial slots of this (sequence, KV head) are merged in two levels, so that no CTA walks
+    // through all of them one L2 round trip after the other (74 slots for a 131072-token head on
+    // 592 CTAs: 20 us at the tail of the launch).  The last CTA to arrive of each group of kGroup
+    // neighbouring contributors merges the group into its first slot; the last group to finish
+    // merges the group results into the output.  Every ticket resets itself; nobody waits.
+    constexpr int kGroup = 8, kOneLevel = 16;   // up to kOneLevel slots are merged in one go
+    const int n = item.n_contrib;
+    const int ng = (n + kGroup - 1) / kGroup;
+    const int g = ((int)blockIdx.x - item.first_cta) / kGroup;
+    const int gsize = min(kGroup, n - g * kGroup);
+    float* seg = p.ws_part + (bh + (size_t)item.first_cta) * (size_t)kColsPad * kPartStride;
+    const size_t cstride = (size_t)kColsPad * kPartStride;
+    const int lane = tid & 31;
     named_bar(1, kConsThreads);
-    if (tid == 0)
-      misc[1] = (atomicInc(p.ws_chunk_ctr + bh, (uint32_t)item.n_contrib - 1) == (uint32_t)item.n_contrib - 1);
+    if (tid == 0) {
+      bool last = true;   // of this CTA's group (n <= kOneLevel: of the whole segment)
+      if (n <= kOneLevel) {
+        last = atomicInc(p.ws_chunk_ctr + bh, (uint32_t)n - 1) == (uint32_t)n - 1;
+      } else if (gsize > 1) {
+        // the group's ticket lives with its first CTA; a CTA can lead two groups at most: the first
+        // group of the segment that starts in its range, and a later group of the one that ends there
+        uint32_t* ctr = p.ws_group_ctr + 2 * (item.first_cta + g * kGroup) + (g == 0 ? 1 : 0);
+        last = atomicInc(ctr, (uint32_t)gsize - 1) == (uint32_t)gsize - 1;
+      }
+      misc[1] = last ? 1 : 0;
+    }
     named_bar(1, kConsThreads);
-    final_here = misc[1] != 0;
-    if (final_here) {
+    final_here = false;
+    bool top = n <= kOneLevel;   // this pass writes the output
+    // (one copy of the merge code, run once or twice: uniform over the CTA)
+    for (bool go = misc[1] != 0; go;) {
       __threadfence();
-      const float* base = p.ws_part + (bh + (size_t)item.first_cta) * (size_t)kColsPad * kPartStride;
-      const size_t cstride = (size_t)kColsPad * kPartStride;
-      // a warp per column, a lane per 4 dims; the slots are merged online, four loads ahead
-      const int lane = tid & 31;
+      const int first = top ? 0 : g * kGroup;
+      const int count = top ? (n <= kOneLevel ? n : ng) : gsize;
+      const size_t sstride = (top && n > kOneLevel ? (size_t)kGroup : (size_t)1) * cstride;
+      // a warp per column, a lane per 4 dims; `count` slots from `first` on, merged online, four
+      // loads ahead; the result goes to the output (normalised) or back to slot `first`
       for (int c = tid >> 5; c < p.ncols; c += kConsThreads / 32) {
-        const float* col = base + (size_t)c * kPartStride;
+        float* col = seg + (size_t)first * cstride + (size_t)c * kPartStride;
         float M = -INFINITY, L = 0.0f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int i0 = 0; i0 < item.n_contrib; i0 += 4) {
+        for (int i0 = 0; i0 < count; i0 += 4) {
           float mi[4], li[4];
           float4 oi[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
-            const bool in = i0 + u < item.n_contrib;
-            const float* src = col + (size_t)(in ? i0 + u : i0) * cstride;
+            const bool in = i0 + u < count;
+            const float* src = col + (size_t)(in ? i0 + u : i0) * sstride;
             mi[u] = in ? __ldcg(src + 128) : -INFINITY;
             li[u] = __ldcg(src + 129);
             oi[u] = __ldcg(reinterpret_cast<const float4*>(src) + lane);
@@ -302,12 +328,28 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
             M = Mn;
           }
         }
-        const float inv = L > 0.0f ? 1.0f / L : 0.0f;
-        const int j = c / p.G, hh = c % p.G;
-        float4* dst = reinterpret_cast<float4*>(
-            p.out + (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D);
-        dst[lane] = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+        if (top) {
+          const float inv = L > 0.0f ? 1.0f / L : 0.0f;
+          const int j = c / p.G, hh = c % p.G;
+          float4* dst = reinterpret_cast<float4*>(
+              p.out + (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D);
+          dst[lane] = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+        } else {
+          reinterpret_cast<float4*>(col)[lane] = acc;
+          if (lane == 0) { col[128] = M; col[129] = L; }
+        }
       }
+      if (top) {
+        final_here = true;
+        break;
+      }
+      // the group's result is in its first slot: one more ticket, among the groups
+      __threadfence();
+      named_bar(1, kConsThreads);
+      if (tid == 0) misc[1] = (atomicInc(p.ws_chunk_ctr + bh, (uint32_t)ng - 1) == (uint32_t)ng - 1);
+      named_bar(1, kConsThreads);
+      go = misc[1] != 0;
+      top = true;
     }
   }
   // accept / reject (Section 4.3): by the CTA that wrote the final outputs of this head
@@ -1197,7 +1239,7 @@ constexpr int kMaxCtasPerSm = 4;
 struct Plan {
   int ncols, variant;  // variant: 0: NT1 TW4 CG1; 1: NT2 TW4 CG1; 2: NT2 TW4 CG2; 3: NT2 TW2 CG4
   int cols_pad;
-  size_t off_chunk_ctr, off_seq_ctr, off_dev, off_part, bytes;
+  size_t off_chunk_ctr, off_seq_ctr, off_group_ctr, off_dev, off_part, bytes;
 };
 
 bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
@@ -1217,6 +1259,7 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   size_t off = kWsHeaderBytes;
   pl->off_chunk_ctr = off; off += (size_t)B * s->num_kv_heads * 4;
   pl->off_seq_ctr = off;   off += (size_t)B * 4;
+  pl->off_group_ctr = off; off += (size_t)2 * sm_count() * kMaxCtasPerSm * 4;
   off = (off + 255) & ~(size_t)255;
   pl->off_dev = off;       off += (size_t)B * s->num_kv_heads * kMaxQ * 4;
   off = (off + 255) & ~(size_t)255;
@@ -1285,6 +1328,7 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   p.ws_flags = reinterpret_cast<uint32_t*>(ws);
   p.ws_chunk_ctr = reinterpret_cast<uint32_t*>(ws + pl.off_chunk_ctr);
   p.ws_seq_ctr = reinterpret_cast<uint32_t*>(ws + pl.off_seq_ctr);
+  p.ws_group_ctr = reinterpret_cast<uint32_t*>(ws + pl.off_group_ctr);
   p.ws_dev = reinterpret_cast<float*>(ws + pl.off_dev);
   p.ws_part = reinterpret_cast<float*>(ws + pl.off_part);
   p.atol = atol; p.rtol = rtol;

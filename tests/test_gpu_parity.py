@@ -385,6 +385,30 @@ def test_wide_verify_long_context_many_pieces(lynx):
         assert float(dev.max()) < 0.1
 
 
+def test_long_context_partial_slots_merge_in_two_levels(lynx):
+    # 40k tokens on two KV heads: every head is split over some 40 CTAs, more than one group of
+    # partial slots, so the group tickets and the merge of the group results are exercised (anchor
+    # and merge-verify at 4, 8 and 16 columns on the mma.sync kernels)
+    B, Hkv, G, L = 2, 2, 4, 40_003
+    for k in (1, 2, 4):
+        c = _case(lynx, 740 + k, B, Hkv, G, k, (L, 9_000), 16, True, "lognormal_channels")
+        qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+        for rep in range(2):   # the tickets reset themselves: a second call on the same workspace
+            ra = oracle.attention(False, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                                  c["lens"].numpy(), Hkv, 16, causal=True)
+            a = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True)
+            lynx.check(c["ws"])
+            _close(a.cpu().numpy().astype(np.float64), ra, f"anchor 40k, {k * G} columns, call {rep}")
+            rf = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                                  c["lens"].numpy(), Hkv, 16, causal=True)
+            out, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"],
+                                                       draft_out=torch.from_numpy(rf.astype(np.float32)).cuda(),
+                                                       atol=0.05, rtol=0.0)
+            lynx.check(c["ws"])
+            _close(out.cpu().numpy().astype(np.float64), rf, f"verify 40k, {k * G} columns, call {rep}")
+            assert fr.cpu().tolist() == [k] * B
+
+
 def test_wide_verify_single_token_returns_its_value_row(lynx):
     # the weight-ratio correction on the tcgen05 path: one attended token gives its V row exactly
     B, Hkv, G, k = 3, 1, 8, 8
