@@ -723,6 +723,11 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
   constexpr float kMidK = FULL ? 0.0f : 8.0f;
   constexpr float kMidV = FULL ? 0.0f : 8.0f;      // V levels: plain codes (full) / plain nibbles (anchor)
   constexpr float kLevelScaleV = FULL ? 1.0f : 16.0f;
+  // The FP16 weights are p * scale_v * 256 (p <= 16 against the lazily raised maximum): FP16 has no
+  // room below 2^-24, and weights that vanish there would still count in the softmax sum and in the
+  // zero-point term.  With the factor a weight vanishes only below 2^-27 of the running maximum
+  // (typical scale 2^-5); weights overflow from scale_v = 16 on, a value row with a range above 4080.
+  constexpr float kWeightUp = FULL ? 256.0f : 16.0f;
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* ring = smem;
   float* mail = reinterpret_cast<float*>(smem + C::kRing);
@@ -1022,7 +1027,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
     // ---- weights of this warp's tile, P^T fragments to shared memory ---------------------
     uint32_t pown[DS > 1 ? 1 : NT][4];  // P^T fragments of the own tile (DS == 1): rounded weights, remainders
     if (valid) {
-      const float sv_lo = vm_lo.x * kLevelScaleV, sv_hi = vm_hi.x * kLevelScaleV;
+      const float sv_lo = vm_lo.x * (kLevelScaleV * kWeightUp), sv_hi = vm_hi.x * (kLevelScaleV * kWeightUp);
       const float zv_lo = fmaf(vm_lo.x, kMidV, vm_lo.y), zv_hi = fmaf(vm_hi.x, kMidV, vm_hi.y);
       uint32_t* pf = reinterpret_cast<uint32_t*>(my_x + 16 + C::kColsPad * 4) + lane;
 #pragma unroll
@@ -1199,8 +1204,8 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
           float* dst = direct ? p.out + (((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D
                               : part + (size_t)c * kPartStride;
           const float inv = direct ? (lt > 0.0f ? 1.0f / lt : 0.0f) : 1.0f;
-          // undo the subnormal scales of the V operands (2^-24; odd dims of the anchor 2^-20)
-          constexpr float fix_even = 16777216.0f, fix_odd = FULL ? 16777216.0f : 1048576.0f;
+          // undo the subnormal scales of the V operands (2^-24; odd dims of the anchor 2^-20) and kWeightUp
+          constexpr float fix_even = 16777216.0f / kWeightUp, fix_odd = (FULL ? 16777216.0f : 1048576.0f) / kWeightUp;
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
             const int gmt = d * MT + mt;  // m-tile index among the eight of a lane's 16 dims

@@ -383,6 +383,11 @@ __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int l
   }
 }
 
+// The FP16 weights are p * scale_v * 64 (p <= 64 against the lazily raised maximum): FP16 has no
+// room below 2^-24, and weights that vanish there would still count in the softmax sum and the
+// zero-point term.  Weights overflow from scale_v = 16 on (a value row with a range above 4080).
+constexpr float kWideWeightUp = 64.0f;
+
 template <int NCOPY, int TERMS>
 __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_kernel(const AttnParams p) {
   using C = WideCfg<NCOPY, TERMS>;
@@ -685,7 +690,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
         sc[0] = in ? km.x * ca : 0.0f;     // alpha: score per unit of the raw dot product
         sc[2] = in ? km.y * cb : 0.0f;     // beta: score per unit of sum(q)
         sc[128] = in ? vm.y : 0.0f;        // zero point of the V row
-        sc[130] = in ? vm.x : 0.0f;        // scale of the V row
+        sc[130] = in ? vm.x * kWideWeightUp : 0.0f;   // scale of the V row, times the weights' factor
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
@@ -861,10 +866,11 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
     const float f = (have && m > -INFINITY && M > -INFINITY) ? ex2(m - M) : 0.0f;
     sc_l[tid] = term == 0 ? l * f : 0.0f;   // the rows of the second term repeat the first term's sums
     sc_z[tid] = term == 0 ? zs * f : 0.0f;
-    // undoes the 2^-24 of the V codes, and puts back what the tensor core's truncating accumulation
-    // lost on average: 0.23 * 2^-23 of the sum (measured on long pieces) for each of the MMAs a unit
-    // adds into a row of O (four token slices a pass)
-    const float coef = f * 16777216.0f * (1.0f + (float)((TERMS == 1 ? 8 : 4) * my_units) * (0.23f * 1.1920929e-7f));
+    // undoes the 2^-24 of the V codes and the weights' factor, and puts back what the tensor core's
+    // truncating accumulation lost on average: 0.46 * 2^-23 of the sum (measured on long pieces) for
+    // each of the four MMAs (token slices) with which a unit adds rounded weights into a row of O
+    // (the remainders of a second pass are too small to lose more than themselves)
+    const float coef = f * (16777216.0f / kWideWeightUp) * (1.0f + (float)(4 * my_units) * (0.46f * 1.1920929e-7f));
     const int part = wg * NR + r / CP;
     for (int round = 0; round < 2 * NR; ++round) {
       if (part == round && have) {   // warp-uniform

@@ -64,15 +64,18 @@ def _check_window(oracle, win, b, planes, table, lens, Hkv, bt):
     assert np.allclose(win["dev"][b].cpu().numpy(), want_dev[0], rtol=0.05, atol=1e-3)
 
 
-def test_config5_shape_two_layers_sampled():
-    """The 70B-class shape (GQA group 8, batch 2, k = 8: 64 verify columns) at two of its 80 layers,
-    through the same Workload class and launches as bench.py: sampled (layer, sequence) pairs."""
+@pytest.mark.parametrize("cfg", [5, 4])
+def test_config_shape_two_layers_sampled(cfg):
+    """Two layers of the 70B-class shape (config 5: GQA group 8, batch 2, k = 8: 64 verify columns)
+    and of the ragged serving mix (config 4: 16 sequences of 8192..65536 tokens, lengths that are no
+    multiples of 16, shuffled 16-token blocks, quantisation of listed blocks, k = 4), through the
+    same Workload class and launches as bench.py: sampled (layer, sequence) pairs."""
     import bench
     import oracle
     free, _ = torch.cuda.mem_get_info()
-    if free < 12 * 2 ** 30:
-        pytest.skip("needs ~8 GB of device memory")
-    wlk = bench.Workload(5, torch.device("cuda", 0), layers=2)
+    if free < 16 * 2 ** 30:
+        pytest.skip("needs ~10 GB of device memory")
+    wlk = bench.Workload(cfg, torch.device("cuda", 0), layers=2)
     wl = wlk.wl
     wlk.step()
     torch.cuda.synchronize()
@@ -80,18 +83,20 @@ def test_config5_shape_two_layers_sampled():
         wlk.lynx.check(w["ws"])
     nbl, Hkv, bt = wlk.nb_layer, wl.num_kv_heads, wl.block_tokens
     table_all = wlk.table.cpu().numpy()
-    for b in (0, wlk.B - 1):                   # flattened (layer, sequence) index
+    for b in (0, wlk.B // 2 + 1, wlk.B - 1)[::(1 if cfg == 4 else 2)]:   # flattened (layer, sequence) index
         layer, seq = divmod(b, wl.batch)
         sl = slice(layer * nbl, (layer + 1) * nbl)
         planes = {}
+        table = (table_all[b:b + 1] - layer * nbl).astype(np.int32)
+        lens = np.array([int(wlk.lens_flat_cpu[b])], np.int32)
+        used = table[0, :(int(lens[0]) + bt - 1) // bt]       # the sequence's blocks (the listed ones)
         for which in "KV":
             want = oracle.split_quantize(_bits(wlk.src[which][sl]))
             got = wlk.planes[which]
-            assert np.array_equal(got.anchor[sl].cpu().numpy(), want[0])
-            assert np.array_equal(got.residual[sl].cpu().numpy(), want[1])
+            assert np.array_equal(got.anchor[sl].cpu().numpy()[used], want[0][used])
+            assert np.array_equal(got.residual[sl].cpu().numpy()[used], want[1][used])
+            assert np.array_equal(got.meta[sl].cpu().numpy().view(np.uint32)[used], want[2].view(np.uint32)[used])
             planes[which] = want
-        table = (table_all[b:b + 1] - layer * nbl).astype(np.int32)
-        lens = np.array([int(wlk.lens_flat_cpu[b])], np.int32)
         for win in wlk.windows:
             _check_window(oracle, win, b, planes, table, lens, Hkv, bt)
 
