@@ -1,5 +1,5 @@
-"""Parity at a full-size workload, in the launch configuration bench.py times: config 3
-(32 layers x 8 KV heads x 131072 tokens, layers flattened into the batch), checked on sampled
+"""Parity at full-size workloads, in the launch configuration bench.py times: configs 3 and 2
+(32 layers x 8 KV heads x 131072 / 32768 tokens, layers flattened into the batch), checked on sampled
 layers the oracle can compute one by one: planes bit-exact, drafts and verified outputs within
 tolerance, accept/reject indices identical when outside the guard band."""
 import os
@@ -20,13 +20,14 @@ def _bits(t):
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
-def test_config3_full_size_sampled_layers():
+@pytest.mark.parametrize("cfg", [3, 2])
+def test_config_full_size_sampled_layers(cfg):
     import bench
     import oracle
     free, _ = torch.cuda.mem_get_info()
     if free < 40 * 2 ** 30:
         pytest.skip("needs ~30 GB of device memory")
-    wlk = bench.Workload(3, torch.device("cuda", 0))
+    wlk = bench.Workload(cfg, torch.device("cuda", 0))
     wl = wlk.wl
     wlk.step()
     torch.cuda.synchronize()
@@ -64,18 +65,21 @@ def _check_window(oracle, win, b, planes, table, lens, Hkv, bt):
     assert np.allclose(win["dev"][b].cpu().numpy(), want_dev[0], rtol=0.05, atol=1e-3)
 
 
-@pytest.mark.parametrize("cfg", [5, 4])
-def test_config_shape_two_layers_sampled(cfg):
-    """Two layers of the 70B-class shape (config 5: GQA group 8, batch 2, k = 8: 64 verify columns)
-    and of the ragged serving mix (config 4: 16 sequences of 8192..65536 tokens, lengths that are no
-    multiples of 16, shuffled 16-token blocks, quantisation of listed blocks, k = 4), through the
-    same Workload class and launches as bench.py: sampled (layer, sequence) pairs."""
+@pytest.mark.parametrize("cfg,layers", [(5, 2), (4, 2), (5, 0)])
+def test_config_shape_sampled(cfg, layers):
+    """The 70B-class shape (config 5: GQA group 8, batch 2, k = 8: 64 verify columns) at two layers
+    and at its full 80 (a CTA then works through whole 131072-token heads: the longest accumulation
+    chains of any configuration), and two layers of the ragged serving mix (config 4: 16 sequences
+    of 8192..65536 tokens, lengths that are no multiples of 16, shuffled 16-token blocks,
+    quantisation of listed blocks, k = 4), through the same Workload class and launches as bench.py:
+    sampled (layer, sequence) pairs."""
     import bench
     import oracle
     free, _ = torch.cuda.mem_get_info()
-    if free < 16 * 2 ** 30:
-        pytest.skip("needs ~10 GB of device memory")
-    wlk = bench.Workload(cfg, torch.device("cuda", 0), layers=2)
+    need = 150 if layers == 0 else 16
+    if free < need * 2 ** 30:
+        pytest.skip(f"needs ~{need} GB of device memory")
+    wlk = bench.Workload(cfg, torch.device("cuda", 0), layers=layers)
     wl = wlk.wl
     wlk.step()
     torch.cuda.synchronize()
