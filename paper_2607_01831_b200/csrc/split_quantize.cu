@@ -8,7 +8,7 @@
 // Mapping: a row is 256 B of BF16; a quarter-warp (8 lanes) owns a row: two 128-bit streaming
 // loads per lane (each instruction covers 128 contiguous bytes of the row), min/max on packed
 // BF16 pairs and three xor-shuffles, 16 codes per lane, 2 x 4 B of each plane per lane.
-// Two rows are in flight per quarter-warp.
+// Eight rows are in flight per quarter-warp.
 #include <cuda_bf16.h>
 
 #include "lynx_common.cuh"
@@ -19,7 +19,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kLanesPerRow = 8;   // a quarter-warp owns a row: 2 x 16 B per lane
-constexpr int kRowsInFlight = 2;  // rows per quarter-warp per loop trip
+constexpr int kRowsInFlight = 8;  // rows per quarter-warp per loop trip (2: 0.84, 4: 0.87, 8: 0.90 of the copy rate; 12: spills)
 
 // Round-half-even of the exact product u*inv, as the low byte of an FP32 whose ulp is 1:
 // fma(u, inv, 1.5 * 2^23) rounds the exact sum once, to an integer, ties to even.
@@ -136,8 +136,20 @@ recombine_kernel(const uint32_t* __restrict__ anchor, const uint32_t* __restrict
                  uint4* __restrict__ deq) {
   const int64_t n_items = n_rows * 16;  // 16 lanes per row, 8 elements per lane
   const int64_t stride = (int64_t)gridDim.x * kThreads;
-  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n_items; i += stride) {
-    const uint32_t xa = __ldcs(anchor + i), xr = __ldcs(residual + i);
+  constexpr int kAhead = 4;             // items per thread and trip: their loads are issued together
+  for (int64_t i0 = (int64_t)blockIdx.x * kThreads + threadIdx.x; i0 < n_items; i0 += stride * kAhead) {
+    uint32_t xas[kAhead], xrs[kAhead];
+#pragma unroll
+    for (int u = 0; u < kAhead; ++u) {
+      const int64_t i = i0 + u * stride;
+      xas[u] = i < n_items ? __ldcs(anchor + i) : 0u;
+      xrs[u] = i < n_items ? __ldcs(residual + i) : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < kAhead; ++u) {
+    const int64_t i = i0 + u * stride;
+    if (i >= n_items) break;
+    const uint32_t xa = xas[u], xr = xrs[u];
     // even elements: (a << 4) | r from the low nibbles; odd elements from the high nibbles
     const uint32_t ev = ((xa << 4) & 0xF0F0F0F0u) | (xr & 0x0F0F0F0Fu);
     const uint32_t od = (xa & 0xF0F0F0F0u) | ((xr >> 4) & 0x0F0F0F0Fu);
@@ -156,6 +168,7 @@ recombine_kernel(const uint32_t* __restrict__ anchor, const uint32_t* __restrict
         o[j] = *reinterpret_cast<const uint32_t*>(&p);
       }
       __stcs(deq + i, make_uint4(o[0], o[1], o[2], o[3]));
+    }
     }
   }
 }
