@@ -219,7 +219,7 @@ def test_merge_verify_matches_oracle_and_decides_identically(lynx, case, causal)
 @pytest.mark.parametrize("seed", range(6))
 def test_short_heavy_tailed_contexts_keep_a_margin(lynx, seed):
     # a few tokens with heavy-tailed values: one token dominates, so the rounding of its weight to
-    # FP16 is not averaged away; the weight-ratio correction must keep the error well inside the bound
+    # FP16 is not averaged away; the two FP16 weight terms must keep the error well inside the bound
     c = _case(lynx, 400 + seed, 4, 2, 8, 1, (1, 15, 17, 3), 16, True, "student_t4")
     qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
     for full in (False, True):
@@ -410,7 +410,7 @@ def test_long_context_partial_slots_merge_in_two_levels(lynx):
 
 
 def test_wide_verify_single_token_returns_its_value_row(lynx):
-    # the weight-ratio correction on the tcgen05 path: one attended token gives its V row exactly
+    # the two weight terms on the tcgen05 path: one attended token gives its V row to FP32 rounding
     B, Hkv, G, k = 3, 1, 8, 8
     c = _case(lynx, 800, B, Hkv, G, k, (1,) * B, 16, True, "student_t4")
     qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
