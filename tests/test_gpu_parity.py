@@ -426,21 +426,26 @@ def test_wide_verify_single_token_returns_its_value_row(lynx):
         assert np.max(np.abs(got[b] - row[None, None, :])) <= 4e-6 * size + 1e-30
 
 
-def test_seeded_random_shapes_all_variants(lynx):
+@pytest.mark.parametrize("long_batches", [False, True])
+def test_seeded_random_shapes_all_variants(lynx, long_batches):
     # a seeded sweep over shapes (KV heads, GQA group, positions, block size, ragged lengths) that
-    # reaches every kernel variant: 1..64 columns, anchor and verify, causal or not
-    rng = np.random.default_rng(20250607)
+    # reaches every kernel variant: 1..64 columns, anchor and verify, causal or not; once with short
+    # contexts and once with ragged batches of up to 47001 tokens (pieces of hundreds of units,
+    # partial slots, empty and one-token sequences next to long ones)
+    rng = np.random.default_rng(20250607 + int(long_batches))
     recipes = ["normal_outlier4x8", "lognormal_channels", "student_t4", "normal_outlier2pct_x10", "normal"]
+    pool = [0, 1, 17, 300, 5000, 12345, 20000, 33333, 47001] if long_batches else \
+        [0, 1, 5, 16, 63, 64, 65, 200, 777, 1500, 3100]
     done = 0
-    while done < 14:
+    while done < (8 if long_batches else 14):
         Hkv = int(rng.choice([1, 2, 3]))
         G = int(rng.choice([1, 2, 3, 4, 6, 8, 16]))
         k = int(rng.integers(1, 17))
         if k * G > 64:
             continue
-        B = int(rng.integers(1, 4))
+        B = int(rng.integers(2, 6)) if long_batches else int(rng.integers(1, 4))
         bt = int(rng.choice([16, 32, 64]))
-        lens = tuple(int(x) for x in rng.choice([0, 1, 5, 16, 63, 64, 65, 200, 777, 1500, 3100], size=B))
+        lens = tuple(int(x) for x in rng.choice(pool, size=B))
         causal = bool(rng.integers(0, 2))
         c = _case(lynx, 900 + done, B, Hkv, G, k, lens, bt, True, recipes[done % len(recipes)])
         qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
