@@ -429,7 +429,7 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f16 levels x f16 q/p, f32 accumulate (quantiser f32)",
+        "vs_baseline": None, "dtype": "u8 x s8 -> s32 (Q.K^T; f16 on tcgen05), f16 x f16 -> f32 (P.V), f32 softmax and quantiser",
         "data": "synthetic",
         "config": {"workload": wl.name, "layers": wl.layers, "batch": wl.batch, "context": wl.context,
                    "num_kv_heads": wl.num_kv_heads, "num_q_heads": wl.num_q_heads, "k": list(wl.k_list),
