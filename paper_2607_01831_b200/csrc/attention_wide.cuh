@@ -499,7 +499,8 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
   constexpr uint32_t kIdescS = tc_idesc(64, false), kIdescO = tc_idesc(128, true);
   // =============================================================================================
   // The MMA warp: one thread issues every tcgen05.mma, so that no softmax warp stalls on the
-  // tensor pipe's queue.  It polls the four "operands ready" barriers and issues what is ready.
+  // tensor pipe's queue.  It polls the "operands ready" barriers and issues what is ready, the P.V
+  // passes (which a group waits for soonest) before the next unit's Q.K^T.
   // =============================================================================================
   if (warp == C::kMmaWarp) {
     if (lane == 0) {
@@ -523,15 +524,14 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
             const uint32_t tile_vp = tile_k + (1 + (gp[w] & 1)) * C::kTileBytes;   // V tile of the unit whose P.V comes next
             const uint32_t tile_vr = tile_k + (1 + (gr[w] & 1)) * C::kTileBytes;   // ... whose remainder pass comes next
             const uint32_t tm_w = tmem0 + C::kTmemWg0 + w * C::kTmemWg;
-            if (todo_k[w] > 0 && mbar_test(kready0 + w * 8, gk[w] & 1)) {
+            if (todo_r[w] > 0 && mbar_test(rready0 + w * 8, gr[w] & 1)) {   // the same P.V on the remainders
               tc_fence_after();
 #pragma unroll
-              for (int ks = 0; ks < 8; ++ks)
-                tc_mma_ts(tm_w + C::kTmemS, tm_q + (uint32_t)ks * 8u,
-                          tc_desc(tile_k + (uint32_t)(ks >> 2) * 8192u + (uint32_t)(ks & 3) * 32u, 16u, 1024u),
-                          kIdescS, ks > 0 ? 1u : 0u);
-              tc_commit(sready0 + w * 8);
-              ++gk[w]; --todo_k[w]; progress = true;
+              for (int ks = 0; ks < 4; ++ks)
+                tc_mma_ts(tm_w + C::kTmemO, tm_w + C::kTmemP + (uint32_t)ks * 8u,
+                          tc_desc(tile_vr + (uint32_t)ks * 2048u, 8192u, 1024u), kIdescO, 1u);
+              tc_commit(rdone0 + (w * 2 + (gr[w] & 1)) * 8);
+              ++gr[w]; --todo_r[w]; progress = true;
             }
             if (todo_p[w] > 0 && mbar_test(pready0 + w * 8, gp[w] & 1) &&
                 (C::kVWarps == 0 || mbar_test(vready0 + (w * 2 + (gp[w] & 1)) * 8, (gp[w] >> 1) & 1))) {
@@ -549,14 +549,15 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
               first_p[w] = 0;
               ++gp[w]; --todo_p[w]; progress = true;
             }
-            if (todo_r[w] > 0 && mbar_test(rready0 + w * 8, gr[w] & 1)) {   // the same P.V on the remainders
+            if (todo_k[w] > 0 && mbar_test(kready0 + w * 8, gk[w] & 1)) {
               tc_fence_after();
 #pragma unroll
-              for (int ks = 0; ks < 4; ++ks)
-                tc_mma_ts(tm_w + C::kTmemO, tm_w + C::kTmemP + (uint32_t)ks * 8u,
-                          tc_desc(tile_vr + (uint32_t)ks * 2048u, 8192u, 1024u), kIdescO, 1u);
-              tc_commit(rdone0 + (w * 2 + (gr[w] & 1)) * 8);
-              ++gr[w]; --todo_r[w]; progress = true;
+              for (int ks = 0; ks < 8; ++ks)
+                tc_mma_ts(tm_w + C::kTmemS, tm_q + (uint32_t)ks * 8u,
+                          tc_desc(tile_k + (uint32_t)(ks >> 2) * 8192u + (uint32_t)(ks & 3) * 32u, 16u, 1024u),
+                          kIdescS, ks > 0 ? 1u : 0u);
+              tc_commit(sready0 + w * 8);
+              ++gk[w]; --todo_k[w]; progress = true;
             }
           }
           if (progress) {
