@@ -465,3 +465,23 @@ def test_seeded_random_shapes_all_variants(lynx, long_batches):
         if np.all(np.abs(want_dev - 1.0) > 0.05):
             assert np.array_equal(fr.cpu().numpy(), want_fr), what
         done += 1
+
+
+@pytest.mark.parametrize("bt,G,k,lens", [(48, 4, 4, (1000, 5, 48, 49)), (112, 2, 16, (4000,)),
+                                         (256, 4, 2, (513, 255))])
+def test_block_sizes_that_are_no_power_of_two_or_large(lynx, bt, G, k, lens):
+    # any multiple of 16 tokens per block is accepted: three 16-token sub-blocks per block, seven,
+    # sixteen; sequences that end inside a block, in its first and in its last sub-block
+    Hkv = 2
+    c = _case(lynx, 7100 + bt, len(lens), Hkv, G, k, lens, bt, True, "student_t4")
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    for causal in (False, True):
+        ref_a = oracle.attention(False, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                                 c["lens"].numpy(), Hkv, bt, causal=causal)
+        out_a = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=causal)
+        ref_f = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                                 c["lens"].numpy(), Hkv, bt, causal=causal)
+        out_f = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=causal)[0]
+        lynx.check(c["ws"])
+        _close(out_a.cpu().numpy().astype(np.float64), ref_a, f"anchor bt={bt} causal={causal}")
+        _close(out_f.cpu().numpy().astype(np.float64), ref_f, f"verify bt={bt} causal={causal}")
