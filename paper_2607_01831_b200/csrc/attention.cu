@@ -1234,7 +1234,7 @@ attn_team_kernel(const AttnParams p) {
   attn_team_body<FULL, NT, DS, TEAMS, NSTAGE, TPW, PACK>(p);
 }
 #ifndef LYNX_WIDE_VERIFY
-#define LYNX_WIDE_VERIFY 2   // 0: keep the mma.sync kernels for 17..64 verify columns (comparison builds)
+#define LYNX_WIDE_VERIFY 2   // comparison builds: 1 = mma.sync kernel for 17..32 verify columns, 0 = for 33..64 too
 #endif
 #include "attention_wide.cuh"
 
@@ -1355,19 +1355,22 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
       default: return launch_team<false, 8, 4, 2, 3, 1>(p, st);
     }
   }
-#if LYNX_WIDE_VERIFY
-  if (pl.variant == 3) return launch_wide<2, 1>(p, st);
-#if LYNX_WIDE_VERIFY > 1
-  if (pl.variant == 2) return launch_wide<2, 2>(p, st);
-#endif
-#endif
   switch (pl.variant) {
     case 0:
       if (pl.ncols <= 4) return launch_team<true, 1, 1, 4, 3, 3, 1, true>(p, st);
       return launch_team<true, 1, 1, 4, 3, 3>(p, st);
     case 1: return launch_team<true, 2, 2, 2, 3, 3>(p, st);
+    // 17..64 columns: tcgen05.  (The mma.sync kernels for them are built in comparison builds only.)
+#if LYNX_WIDE_VERIFY > 1
+    case 2: return launch_wide<2, 2>(p, st);
+#else
     case 2: return launch_team<true, 4, 4, 1, 2, 3>(p, st);
+#endif
+#if LYNX_WIDE_VERIFY
+    default: return launch_wide<2, 1>(p, st);
+#else
     default: return launch_team<true, 8, 4, 2, 3, 1>(p, st);
+#endif
   }
 }
 
