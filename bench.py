@@ -538,6 +538,26 @@ def run_per_layer(wlk: "Workload", peak: float):
         gbs = wlk.rows_kv * bpr / (ms * 1e-3) / 1e9
         out[name] = {"launches": L, "ms_all_layers": ms, "us_per_layer": ms * 1e3 / L, "GBps": gbs,
                      "frac_of_measured": gbs / peak}
+        # the same launches replayed from one CUDA graph (no host work between them)
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                fn()
+            for _ in range(2):
+                graph.replay()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(reps):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            gms = e0.elapsed_time(e1) / reps
+            out[name]["cuda_graph_us_per_layer"] = gms * 1e3 / L
+            del graph
+        except Exception as exc:   # capture is an extra: the eager figure above stands on its own
+            out[name]["cuda_graph_us_per_layer"] = None
+            out[name]["cuda_graph_error"] = str(exc)[:200]
+            torch.cuda.synchronize()
     lynx.check(ws1)
     lynx.check(wsk)
     return out
