@@ -103,7 +103,12 @@ lynx_status lynx_recombine(const uint8_t* anchor, const uint8_t* residual, const
  * positions (n_q or k) and sequences of at most max_blocks_per_seq * block_tokens tokens.
  * Returns 0 for an unsupported shape.  The workspace must be zero-filled once before its first
  * use (lynx_workspace_init, or cudaMemsetAsync of the whole buffer); each call leaves it ready
- * for the next.  Calls sharing a workspace must be ordered on one stream. */
+ * for the next.  Calls sharing a workspace must be ordered on one stream.
+ * The figure includes 10 to 20 MB for FP32 copies of the kernels' accumulators, into which long
+ * accumulation chains are cut (what the tensor cores lose by truncating when they accumulate is
+ * then bounded whatever the context length).  A call given less than the full figure, but enough
+ * for the rest, runs without that cut: fine for value rows with a modest range, up to a few 1e-3
+ * of absolute error for rows whose range is in the hundreds and contexts of 100k tokens. */
 size_t lynx_workspace_bytes(const lynx_shape* shape, int32_t batch, int32_t n_cols_q);
 lynx_status lynx_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
@@ -141,8 +146,8 @@ lynx_status lynx_merge_verify_attention(const lynx_shape* shape, const void* q_b
  * captured).  Same computation, arguments and result as lynx_anchor_attention, but the scratch
  * memory is a fixed 8 MiB array inside the library image (every GPU that loads the library
  * holds it until the process exits); the call itself allocates nothing.
- *  - Problems whose scratch need (lynx_workspace_bytes) exceeds 8 MiB are rejected with
- *    LYNX_ERR_WORKSPACE and nothing is launched.
+ *  - Problems whose scratch need (lynx_workspace_bytes less the accumulator copies, which this
+ *    call does without) exceeds 8 MiB are rejected with LYNX_ERR_WORKSPACE and nothing is launched.
  *  - The first call on each device looks up the array's device address (a one-time set-up,
  *    done with that device current); make that first call before any stream capture begins.
  *  - All calls share the one array.  Each call clears the words that must start at zero, on

@@ -62,6 +62,7 @@ struct AttnParams {
   uint32_t* ws_chunk_ctr;  // [B*Hkv]
   uint32_t* ws_seq_ctr;    // [B]
   uint32_t* ws_group_ctr;  // [2 * CTAs of the largest grid]: tickets of the groups of partial slots
+  float* ws_shadow;        // FP32 copies of the O accumulators (see kFlushMmas), or null
   float* ws_dev;           // [B*Hkv][kMaxQ]
   float* ws_part;          // [B*Hkv + CTAs][ncols_pad][kPartStride], slot = segment + CTA index
   float atol, rtol;
@@ -784,8 +785,18 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
   // log-uniformly).  Over the thousands of MMAs of a long piece that is a relative bias of some
   // 1e-4 on the uncentred level sums, which are large against the outputs they cancel into.  The
   // MMAs into each accumulator are counted and the expected loss is put back at the end of a piece.
+  // The estimate is good to some 30 %, which is not enough for the longest chains (a CTA that
+  // works through a whole 131072-token head adds 16 000 MMAs into an accumulator) on rows whose
+  // level sums are a hundred times their outputs.  So the chains are cut: every kFlushMmas MMAs the
+  // accumulators are added in FP32 (round to nearest, by the L2's reduction unit: no load, nothing
+  // to wait for) into a copy of the O slice in the workspace and start again from zero.  Without
+  // that part of the workspace (see lynx_workspace_bytes) the chains are not cut.
   constexpr float kTruncPerMma = 0.40f * 1.1920929e-7f;
-  int n_mma = 0;
+  constexpr int kFlushMmas = 1024;
+  int n_mma = 0;          // MMAs into each accumulator since the last flush
+  bool flushed = false;   // the copy holds earlier parts of this piece
+  float* shadow = p.ws_shadow == nullptr ? nullptr
+      : p.ws_shadow + ((size_t)cta * C::kConsWarps + warp) * (NT * MT * 4 * 32) + lane;
   float m[NT][2], l[NT][2], zs[NT][2], o[NT][MT][4];
   const uint32_t qf_u32 = smem_u32(qf_s), qs_u32 = smem_u32(qs_s);
   auto col_limit = [&](int col, int len_) {
@@ -887,6 +898,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
       named_bar(1, C::kConsThreads);  // the shared fragments are complete
       fresh = true;
       n_mma = 0;
+      flushed = false;
     }
 
     const uint32_t st = ring_u32 + slot * C::kStageBytes;
@@ -1019,6 +1031,11 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
             for (int mt = 0; mt < MT; ++mt) {
               o[nt][mt][cc] *= f;
               o[nt][mt][cc + 2] *= f;
+              if (flushed) {   // rare: the copy follows the new maximum
+                float* s0 = shadow + ((nt * MT + mt) * 4 + cc) * 32;
+                __stcg(s0, __ldcg(s0) * f);
+                __stcg(s0 + 64, __ldcg(s0 + 64) * f);
+              }
             }
           }
       }
@@ -1089,6 +1106,22 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
     }
     }  // if (DS > 1 || in_range)
     }  // tiles of this warp
+    if (shadow != nullptr && n_mma >= kFlushMmas) {   // uniform over the warp
+      const float back = 1.0f + (float)n_mma * kTruncPerMma;   // the expected truncation loss, put back
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            float* sh = shadow + ((nt * MT + mt) * 4 + i) * 32;
+            const float v = o[nt][mt][i] * back;
+            if (flushed) atomicAdd(sh, v); else __stcg(sh, v);
+            o[nt][mt][i] = 0.0f;
+          }
+      flushed = true;
+      n_mma = 0;
+    }
     __syncwarp();
     if (lane == 0) mbar_arrive(empty0 + slot * 8);
     if (!(info.z & 2)) continue;
@@ -1103,6 +1136,7 @@ __device__ __forceinline__ void attn_team_body(const AttnParams& p) {
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             o[nt][mt][i] *= back;
+            if (flushed) o[nt][mt][i] += __ldcg(shadow + ((nt * MT + mt) * 4 + i) * 32);
             // the remainders' part, accumulated under the repeated columns, joins its column
             if (PACK) o[nt][mt][i] += __shfl_xor_sync(0xFFFFFFFFu, o[nt][mt][i], 2);
           }
@@ -1245,6 +1279,7 @@ struct Plan {
   int ncols, variant;  // variant: 0: NT1 TW4 CG1; 1: NT2 TW4 CG1; 2: NT2 TW4 CG2; 3: NT2 TW2 CG4
   int cols_pad;
   size_t off_chunk_ctr, off_seq_ctr, off_group_ctr, off_dev, off_part, bytes;
+  size_t shadow_bytes;   // optional tail of the workspace: FP32 copies of the accumulators (see kFlushMmas)
 };
 
 bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
@@ -1270,7 +1305,11 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   off = (off + 255) & ~(size_t)255;
   pl->off_part = off;
   off += ((size_t)B * s->num_kv_heads + (size_t)sm_count() * kMaxCtasPerSm) * pl->cols_pad * kPartStride * 4;
-  pl->bytes = off;
+  pl->bytes = (off + 255) & ~(size_t)255;
+  // mma.sync kernels: one O slice per consumer warp, 16 KB per CTA (64 KB with 64 columns, one CTA per
+  // SM); tcgen05 kernels: 2 groups x 128 rows x 128 dims per CTA
+  pl->shadow_bytes = (size_t)sm_count() * (ncols > 16 && ncols <= 64 ? 131072 : kMaxCtasPerSm * 16384);
+  if (pl->shadow_bytes < (size_t)sm_count() * kMaxCtasPerSm * 16384) pl->shadow_bytes = (size_t)sm_count() * kMaxCtasPerSm * 16384;
   return true;
 }
 
@@ -1334,6 +1373,7 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   p.ws_chunk_ctr = reinterpret_cast<uint32_t*>(ws + pl.off_chunk_ctr);
   p.ws_seq_ctr = reinterpret_cast<uint32_t*>(ws + pl.off_seq_ctr);
   p.ws_group_ctr = reinterpret_cast<uint32_t*>(ws + pl.off_group_ctr);
+  p.ws_shadow = workspace_bytes >= pl.bytes + pl.shadow_bytes ? reinterpret_cast<float*>(ws + pl.bytes) : nullptr;
   p.ws_dev = reinterpret_cast<float*>(ws + pl.off_dev);
   p.ws_part = reinterpret_cast<float*>(ws + pl.off_part);
   p.atol = atol; p.rtol = rtol;
@@ -1380,7 +1420,7 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
 extern "C" size_t lynx_workspace_bytes(const lynx_shape* shape, int32_t batch, int32_t n_cols_q) {
   lynx::Plan pl;
   if (!lynx::make_plan(shape, batch, n_cols_q, &pl)) return 0;
-  return pl.bytes;
+  return pl.bytes + pl.shadow_bytes;
 }
 
 extern "C" lynx_status lynx_anchor_attention(const lynx_shape* shape, const void* q_bf16, int32_t batch,

@@ -387,6 +387,11 @@ __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int l
 // room below 2^-24, and weights that vanish there would still count in the softmax sum and the
 // zero-point term.  Weights overflow from scale_v = 16 on (a value row with a range above 4080).
 constexpr float kWideWeightUp = 64.0f;
+// Truncation loss per MMA that adds rounded weights into a row of O: 0.46 * 2^-23 of the sum
+// (measured on long pieces).  The estimate is good to some 30 %; so that this is enough for the
+// longest pieces, a row of O is moved to an FP32 copy in the workspace every kWideFlushUnits units.
+constexpr float kWideTruncPerMma = 0.46f * 1.1920929e-7f;
+constexpr int kWideFlushUnits = 256;
 
 template <int NCOPY, int TERMS>
 __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_kernel(const AttnParams p) {
@@ -584,6 +589,9 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
   const uint32_t tm_s = tmem0 + C::kTmemWg0 + wg * C::kTmemWg + C::kTmemS;
   const uint32_t tm_p = tmem0 + C::kTmemWg0 + wg * C::kTmemWg + C::kTmemP;
   const uint32_t tm_o = tmem0 + C::kTmemWg0 + wg * C::kTmemWg + C::kTmemO;
+  // FP32 copy of this row of O in the workspace: [CTA][group][dim][row] (worked out where it is
+  // used: the address is not worth two registers in the unit loop)
+  auto shadow_row = [&]() { return p.ws_shadow + (((size_t)cta * 2 + wg) * 128) * 128 + r; };
   {  // P starts as zero: a row only ever writes its own tokens
     uint32_t z[32];
 #pragma unroll
@@ -672,6 +680,9 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
     float m = 0.0f, l = 0.0f, zs = 0.0f;  // m: the running maximum (log2 units)
     bool fresh = true;
     int my_units = 0;
+    int units_since = 0;      // units added into this row of O since it was last moved to the copy
+    bool w_flushed = false;   // the copy in the workspace holds earlier units of this piece ...
+    float m_sh = 0.0f;        // ... relative to this running maximum
 
     // K side of unit k of this piece: code tile, per-token scalars (set `set`), S = Q . K^T.  The K
     // tile is free: the previous Q.K^T of this group has been waited for.
@@ -731,7 +742,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
     };
     if (wg < n_piece) prefetch(wg, (int)(n_u % 3u));
 
-    for (int k = wg; k < n_piece; k += 2, ++my_units) {
+    for (int k = wg; k < n_piece; k += 2, ++my_units, ++units_since) {
       const int set = (int)(n_u % 3u);
       const int slot = (gs_base + k) % NSTAGE;
       const int unit_t0 = (item.pad1 + k) * C::kST;
@@ -828,6 +839,40 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
         // P and the V tile are free once both P.V passes of the previous unit are complete
         wait_remainders();
         tc_fence_after();
+        if (units_since >= kWideFlushUnits && p.ws_shadow != nullptr) {
+          float* wsh = shadow_row();
+          // cut the accumulation chain: this row of O is added in FP32 (reductions in L2, round to
+          // nearest: no load, nothing to wait for), with the expected truncation loss put back, to
+          // its copy and starts again from zero.  The copy stays relative to the running maximum
+          // m_sh of the row's first flush, so a later rise of the maximum does not touch it; what is
+          // added is scaled up by 2^(m - m_sh) (a rise of more than 60 moves the copy instead).
+          float up = w_flushed ? m - m_sh : 0.0f;
+          if (!w_flushed) m_sh = m;
+          if (up > 60.0f) {   // rare, per row
+            const float down = ex2(-up);
+#pragma unroll 8
+            for (int col = 0; col < 128; ++col) __stcg(wsh + col * 128, __ldcg(wsh + col * 128) * down);
+            m_sh = m;
+            up = 0.0f;
+          }
+          const float corr = (1.0f + (float)(4 * units_since) * kWideTruncPerMma) * ex2(up);
+#pragma unroll
+          for (int cch = 0; cch < 4; ++cch) {
+            uint32_t o[32];
+            TmemRegs<32>::ld(tm_o + lane_sel + cch * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              float* sh = wsh + (cch * 32 + i) * 128;
+              const float v = __uint_as_float(o[i]) * corr;
+              if (w_flushed) atomicAdd(sh, v); else __stcg(sh, v);
+              o[i] = 0u;
+            }
+            TmemRegs<32>::st(tm_o + lane_sel + cch * 32, o);
+          }
+          w_flushed = true;
+          units_since = 0;
+        }
         TmemRegs<KT / 2>::st(tm_p + lane_sel + (uint32_t)(copy * (KT / 2)), ph);
 #pragma unroll
         for (int i = 0; i < KT / 2; ++i) pr_prev[i] = TERMS == 1 ? pr[i] : 0u;
@@ -868,10 +913,13 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
     sc_l[tid] = term == 0 ? l * f : 0.0f;   // the rows of the second term repeat the first term's sums
     sc_z[tid] = term == 0 ? zs * f : 0.0f;
     // undoes the 2^-24 of the V codes and the weights' factor, and puts back what the tensor core's
-    // truncating accumulation lost on average: 0.46 * 2^-23 of the sum (measured on long pieces) for
-    // each of the four MMAs (token slices) with which a unit adds rounded weights into a row of O
-    // (the remainders of a second pass are too small to lose more than themselves)
-    const float coef = f * (16777216.0f / kWideWeightUp) * (1.0f + (float)(4 * my_units) * (0.46f * 1.1920929e-7f));
+    // truncating accumulation lost on average: kWideTruncPerMma of the sum for each of the four
+    // MMAs (token slices) with which a unit adds rounded weights into a row of O (the remainders of
+    // a second pass are too small to lose more than themselves)
+    const float coef = f * (16777216.0f / kWideWeightUp);
+    const float corr = 1.0f + (float)(4 * units_since) * kWideTruncPerMma;
+    const float keep_sh = w_flushed ? ex2(m_sh - m) : 0.0f;   // the copy, brought to the row's final maximum
+    const float* wsh = shadow_row();
     const int part = wg * NR + r / CP;
     for (int round = 0; round < 2 * NR; ++round) {
       if (part == round && have) {   // warp-uniform
@@ -884,7 +932,9 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
           for (int i = 0; i < 32; ++i) {
             const int d = cch * 32 + (i & ~7) + wide_perm(i & 7);   // logical head dim of column i
             float* dst = msc + c * C::kMergeStride + d;
-            const float v = coef * __uint_as_float(o[i]);
+            float part_o = __uint_as_float(o[i]) * corr;
+            if (w_flushed) part_o = fmaf(__ldcg(wsh + (cch * 32 + i) * 128), keep_sh, part_o);   // earlier units of the piece
+            const float v = coef * part_o;
             *dst = round == 0 ? v : *dst + v;
           }
         }

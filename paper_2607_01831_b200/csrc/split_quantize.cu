@@ -19,7 +19,13 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kLanesPerRow = 8;   // a quarter-warp owns a row: 2 x 16 B per lane
-constexpr int kRowsInFlight = 8;  // rows per quarter-warp per loop trip (2: 0.84, 4: 0.87, 8: 0.90 of the copy rate; 12: spills)
+// rows per quarter-warp per loop trip: dense rows 8 (2: 0.84, 4: 0.87, 8: 0.90 of the copy rate; 12:
+// spills); rows of listed blocks 4 (2: 0.81, 4: 0.87, 8: 0.77: the block lookups cost registers)
+constexpr int kRowsInFlight = 8;
+#ifndef LYNX_SQ_IDS_ROWS
+#define LYNX_SQ_IDS_ROWS 4
+#endif
+constexpr int kRowsInFlightIds = LYNX_SQ_IDS_ROWS;
 
 // Round-half-even of the exact product u*inv, as the low byte of an FP32 whose ulp is 1:
 // fma(u, inv, 1.5 * 2^23) rounds the exact sum once, to an integer, ties to even.
@@ -69,11 +75,12 @@ split_quantize_kernel(const uint4* __restrict__ src, int64_t n_logical_rows,
   const int64_t grp = (int64_t)blockIdx.x * (kThreads / kLanesPerRow) + (threadIdx.x / kLanesPerRow);
   const int64_t grp_total = (int64_t)gridDim.x * (kThreads / kLanesPerRow);
 
-  for (int64_t r0 = grp * kRowsInFlight; r0 < n_logical_rows; r0 += grp_total * kRowsInFlight) {
-    uint4 lo[kRowsInFlight], hi[kRowsInFlight];
-    int64_t row[kRowsInFlight];
+  constexpr int kRows = kIds ? kRowsInFlightIds : kRowsInFlight;
+  for (int64_t r0 = grp * kRows; r0 < n_logical_rows; r0 += grp_total * kRows) {
+    uint4 lo[kRows], hi[kRows];
+    int64_t row[kRows];
 #pragma unroll
-    for (int u = 0; u < kRowsInFlight; ++u) {
+    for (int u = 0; u < kRows; ++u) {
       int64_t lr = r0 + u;
       row[u] = -1;
       if (lr < n_logical_rows) {
@@ -93,7 +100,7 @@ split_quantize_kernel(const uint4* __restrict__ src, int64_t n_logical_rows,
       }
     }
 #pragma unroll
-    for (int u = 0; u < kRowsInFlight; ++u) {
+    for (int u = 0; u < kRows; ++u) {
       // the shuffles below are executed by every lane of the warp, valid row or not
       const uint32_t wl[4] = {lo[u].x, lo[u].y, lo[u].z, lo[u].w};
       const uint32_t wh[4] = {hi[u].x, hi[u].y, hi[u].z, hi[u].w};
@@ -194,7 +201,7 @@ extern "C" lynx_status lynx_split_quantize(const void* src_bf16, int64_t n_rows,
       (reinterpret_cast<uintptr_t>(meta) & 7u))
     return LYNX_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int rows_per_cta_trip = (kThreads / kLanesPerRow) * kRowsInFlight;
+  const int rows_per_cta_trip = (kThreads / kLanesPerRow) * (block_ids ? kRowsInFlightIds : kRowsInFlight);
   if (block_ids) {
     if (n_block_ids < 0 || rows_per_block <= 0 || n_rows % rows_per_block != 0) return LYNX_ERR_SHAPE;
     if (n_block_ids == 0) return LYNX_OK;
