@@ -24,6 +24,7 @@ def _bits(t):
 def test_config_full_size_sampled_layers(cfg):
     import bench
     import oracle
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < 40 * 2 ** 30:
         pytest.skip("needs ~30 GB of device memory")
@@ -75,6 +76,7 @@ def test_config_shape_sampled(cfg, layers):
     sampled (layer, sequence) pairs."""
     import bench
     import oracle
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     need = 150 if layers == 0 else 16
     if free < need * 2 ** 30:
@@ -115,6 +117,7 @@ def test_long_accumulation_chains_carry_no_bias(G, k):
     import oracle
     import synth
     import paper_2607_01831_b200 as lynx
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < 12 * 2 ** 30:
         pytest.skip("needs ~8 GB of device memory")
@@ -145,3 +148,46 @@ def test_long_accumulation_chains_carry_no_bias(G, k):
         g = got[:1].cpu().numpy().astype(np.float64)
         assert np.all(np.abs(g - ref) <= ATOL + RTOL * np.abs(ref)), float(np.abs(g - ref).max())
         assert abs(float((g - ref).mean())) <= 0.25 * ATOL, float((g - ref).mean())
+
+
+def test_long_heavy_tailed_batches_stay_inside_the_tolerance():
+    """24 Student-t sequences of 131072 tokens: every CTA works through whole heads (the longest
+    accumulation chains there are) on value rows whose level sums are up to a hundred times their
+    outputs.  Needs the chains cut into FP32 copies (an estimate of the tensor cores' truncation
+    loss alone left such rows up to 2x outside the tolerance) and the FP16 weights scaled so that
+    small weights next to a dominant token do not vanish."""
+    import oracle
+    import synth
+    import paper_2607_01831_b200 as lynx
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * 2 ** 30:
+        pytest.skip("needs ~30 GB of device memory")
+    L, B, Hkv, bt = 131072, 24, 8, 16
+    lens = torch.full((B,), L, dtype=torch.int32)
+    table, nb = synth.block_table(lens, bt, True, "heavyT")
+    planes = {}
+    for which in "KV":
+        src = synth.kv_block_values("student_t4", nb, Hkv, bt, "cuda", "heavy" + which)
+        planes[which] = lynx.split_quantize(src)
+        del src
+    K, V = planes["K"], planes["V"]
+    td, ld = table.cuda(), lens.cuda()
+    # the oracle on sequence 0: its blocks, renumbered 0..n-1
+    blocks0 = torch.from_numpy(table[0].numpy().astype(np.int64)).cuda()
+    kp = tuple(x[blocks0].cpu().numpy() for x in (K.anchor, K.residual, K.meta))
+    vp = tuple(x[blocks0].cpu().numpy() for x in (V.anchor, V.residual, V.meta))
+    t1 = np.arange(table.shape[1], dtype=np.int32)[None]
+    l1 = lens[:1].numpy()
+    for G, k in ((4, 1), (4, 4), (4, 8), (8, 8)):      # 4, 16, 32 and 64 columns
+        q = synth.queries(B, k, Hkv * G, "cuda", "heavyQ", G, k)
+        geo = lynx.Geometry(Hkv * G, Hkv, bt, nb, table.shape[1])
+        ws = lynx.make_workspace(geo, B, k, "cuda")
+        full = lynx.merge_verify_attention(geo, q, K, V, td, ld, ws)[0]
+        draft = lynx.anchor_attention(geo, q, K, V, td, ld, ws, causal=True)
+        lynx.check(ws)
+        for got, is_full in ((full, True), (draft, False)):
+            ref = oracle.attention(is_full, _bits(q[:1]), kp, vp, t1, l1, Hkv, bt, causal=True)
+            g = got[:1].cpu().numpy().astype(np.float64)
+            worst = float((np.abs(g - ref) / (ATOL + RTOL * np.abs(ref))).max())
+            assert worst <= 1.0, (G, k, is_full, worst)
