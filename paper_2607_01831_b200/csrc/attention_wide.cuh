@@ -383,6 +383,25 @@ __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int l
   }
 }
 
+// Moves a row of O (128 FP32 columns of tensor memory, lane = row) to its FP32 copy in the
+// workspace and zeroes it; see the call.  Out of line: it runs once in hundreds of units.
+__device__ __noinline__ void wide_flush_row(uint32_t tm_row, float* wsh, float corr, bool add) {
+#pragma unroll
+  for (int cch = 0; cch < 4; ++cch) {
+    uint32_t o[32];
+    TmemRegs<32>::ld(tm_row + cch * 32, o);
+    tc_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      float* sh = wsh + (cch * 32 + i) * 128;
+      const float v = __uint_as_float(o[i]) * corr;
+      if (add) atomicAdd(sh, v); else __stcg(sh, v);
+      o[i] = 0u;
+    }
+    TmemRegs<32>::st(tm_row + cch * 32, o);
+  }
+}
+
 // The FP16 weights are p * scale_v * 64 (p <= 64 against the lazily raised maximum): FP16 has no
 // room below 2^-24, and weights that vanish there would still count in the softmax sum and the
 // zero-point term.  Weights overflow from scale_v = 16 on (a value row with a range above 4080).
@@ -856,20 +875,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
             up = 0.0f;
           }
           const float corr = (1.0f + (float)(4 * units_since) * kWideTruncPerMma) * ex2(up);
-#pragma unroll
-          for (int cch = 0; cch < 4; ++cch) {
-            uint32_t o[32];
-            TmemRegs<32>::ld(tm_o + lane_sel + cch * 32, o);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              float* sh = wsh + (cch * 32 + i) * 128;
-              const float v = __uint_as_float(o[i]) * corr;
-              if (w_flushed) atomicAdd(sh, v); else __stcg(sh, v);
-              o[i] = 0u;
-            }
-            TmemRegs<32>::st(tm_o + lane_sel + cch * 32, o);
-          }
+          wide_flush_row(tm_o + lane_sel, wsh, corr, w_flushed);
           w_flushed = true;
           units_since = 0;
         }
