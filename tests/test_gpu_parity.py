@@ -485,3 +485,25 @@ def test_block_sizes_that_are_no_power_of_two_or_large(lynx, bt, G, k, lens):
         lynx.check(c["ws"])
         _close(out_a.cpu().numpy().astype(np.float64), ref_a, f"anchor bt={bt} causal={causal}")
         _close(out_f.cpu().numpy().astype(np.float64), ref_f, f"verify bt={bt} causal={causal}")
+
+
+@pytest.mark.parametrize("scale", [0.3, 0.02])
+def test_custom_softmax_scale(lynx, scale):
+    # softmax_scale other than 1/sqrt(128): sharper and flatter attention than the default, on the
+    # mma.sync kernels (4 and 16 columns) and the tcgen05 kernel (32 columns)
+    Hkv, G = 2, 4
+    for k in (1, 4, 8):
+        c = _case(lynx, 7300 + k, 2, Hkv, G, k, (700, 65), 16, True, "lognormal_channels")
+        qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+        s32 = float(np.float32(scale))
+        ref_a = oracle.attention(False, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                                 c["lens"].numpy(), Hkv, 16, causal=True, softmax_scale=s32)
+        out_a = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True,
+                                      softmax_scale=s32)
+        ref_f = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
+                                 c["lens"].numpy(), Hkv, 16, causal=True, softmax_scale=s32)
+        out_f = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True,
+                                            softmax_scale=s32)[0]
+        lynx.check(c["ws"])
+        _close(out_a.cpu().numpy().astype(np.float64), ref_a, f"anchor scale={scale} k={k}")
+        _close(out_f.cpu().numpy().astype(np.float64), ref_f, f"verify scale={scale} k={k}")
