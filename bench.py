@@ -6,7 +6,7 @@ split-quantise the whole BF16 KV cache (K and V, all layers), then for every spe
 k of the workload: k anchor decode steps on the Anchor planes (growing context) followed by
 one merge-verify pass over the k drafted positions with its accept/reject index.
 
-Prints ONE JSON line (see README for the fields).  `--impl reference` times the CPU
+Prints ONE JSON line (the fields are described in the repository's design notes).  `--impl reference` times the CPU
 oracle on a bounded sample of the same workload instead.
 """
 from __future__ import annotations
