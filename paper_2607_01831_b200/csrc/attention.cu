@@ -258,7 +258,7 @@ __device__ __forceinline__ void named_bar(int id, int nthreads) {
 // Called by all consumer threads of the CTA (named barrier 1).
 template <bool FULL, int kColsPad, int kConsThreads>
 __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& item, bool direct, int tid,
-                                             int* misc) {
+                                             int* misc, int bar_id = 1) {
   const size_t bh = (size_t)item.b * p.Hkv + item.hkv;
   bool final_here = direct;
   if (!direct) {
@@ -275,7 +275,7 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
     float* seg = p.ws_part + (bh + (size_t)item.first_cta) * (size_t)kColsPad * kPartStride;
     const size_t cstride = (size_t)kColsPad * kPartStride;
     const int lane = tid & 31;
-    named_bar(1, kConsThreads);
+    named_bar(bar_id, kConsThreads);
     if (tid == 0) {
       bool last = true;   // of this CTA's group (n <= kOneLevel: of the whole segment)
       if (n <= kOneLevel) {
@@ -288,7 +288,7 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
       }
       misc[1] = last ? 1 : 0;
     }
-    named_bar(1, kConsThreads);
+    named_bar(bar_id, kConsThreads);
     final_here = false;
     bool top = n <= kOneLevel;   // this pass writes the output
     // (one copy of the merge code, run once or twice: uniform over the CTA)
@@ -346,9 +346,9 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
       }
       // the group's result is in its first slot: one more ticket, among the groups
       __threadfence();
-      named_bar(1, kConsThreads);
+      named_bar(bar_id, kConsThreads);
       if (tid == 0) misc[1] = (atomicInc(p.ws_chunk_ctr + bh, (uint32_t)ng - 1) == (uint32_t)ng - 1);
-      named_bar(1, kConsThreads);
+      named_bar(bar_id, kConsThreads);
       go = misc[1] != 0;
       top = true;
     }
@@ -356,10 +356,10 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
   // accept / reject (Section 4.3): by the CTA that wrote the final outputs of this head
   if (FULL && p.draft != nullptr) {
     int* devs = misc + 16;
-    named_bar(1, kConsThreads);  // final outputs written; devs free
+    named_bar(bar_id, kConsThreads);  // final outputs written; devs free
     if (final_here) {
       if (tid < kMaxQ) devs[tid] = 0;
-      named_bar(1, kConsThreads);
+      named_bar(bar_id, kConsThreads);
       for (int idx = tid; idx < p.ncols * LYNX_D; idx += kConsThreads) {
         const int c = idx >> 7, d = idx & 127;
         const int j = c / p.G, hh = c % p.G;
@@ -368,13 +368,13 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
         const float r = fabsf(f - dr) / (p.atol + p.rtol * fabsf(f));
         atomicMax(devs + j, __float_as_int(r));  // r >= 0: integer order = float order
       }
-      named_bar(1, kConsThreads);
+      named_bar(bar_id, kConsThreads);
       if (tid < p.nq) p.ws_dev[bh * kMaxQ + tid] = __int_as_float(devs[tid]);
       __threadfence();
-      named_bar(1, kConsThreads);
+      named_bar(bar_id, kConsThreads);
       if (tid == 0)
         misc[1] = (atomicInc(p.ws_seq_ctr + item.b, (uint32_t)p.Hkv - 1) == (uint32_t)p.Hkv - 1);
-      named_bar(1, kConsThreads);
+      named_bar(bar_id, kConsThreads);
       if (misc[1] && tid == 0) {
         __threadfence();
         int fr = p.nq;
@@ -388,7 +388,7 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
         p.first_reject[item.b] = fr;
       }
     }
-    named_bar(1, kConsThreads);
+    named_bar(bar_id, kConsThreads);
   }
 }
 
@@ -1271,6 +1271,7 @@ attn_team_kernel(const AttnParams p) {
 #define LYNX_WIDE_VERIFY 2   // comparison builds: 1 = mma.sync kernel for 17..32 verify columns, 0 = for 33..64 too
 #endif
 #include "attention_wide.cuh"
+#include "attention_i8.cuh"
 
 // ------------------------------------------------------------------ host side
 constexpr int kMaxCtasPerSm = 4;
@@ -1384,6 +1385,17 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   p.bt = shape->block_tokens; p.num_blocks = shape->num_blocks; p.max_blocks = shape->max_blocks_per_seq;
   p.ncols = pl.ncols;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // up to 16 columns: the integer tcgen05 kernels
+  if (pl.ncols <= 16) {
+    if (!full) {
+      if (pl.ncols <= 4) return launch_i8<false, 4>(p, st);
+      if (pl.ncols <= 8) return launch_i8<false, 8>(p, st);
+      return launch_i8<false, 16>(p, st);
+    }
+    if (pl.ncols <= 4) return launch_i8<true, 4>(p, st);
+    if (pl.ncols <= 8) return launch_i8<true, 8>(p, st);
+    return launch_i8<true, 16>(p, st);
+  }
   // <FULL, NT, DS, TEAMS, stages, CTAs/SM>
   if (!full) {
     switch (pl.variant) {

@@ -1,0 +1,927 @@
+// Anchor and merge-verify attention on the integer path of the fifth-generation tensor cores
+// (tcgen05.mma kind::i8, accumulators in tensor memory).  Included by attention.cu inside its
+// namespace: shares AttnParams, the stream-K cut of the work and finish_piece with the other
+// kernels.
+//
+// With one (scale, zero) per token row the two contractions of Section 2's attention run on the
+// integer levels themselves (see attention.cu).  Here both are exact integer tensor-core
+// products over a 128-token stage-unit:
+//   S^T[128 tokens x 3 CP]   = level(K)[128 x 128 dims] . Qd^T     A = K tile (u8, K-major),
+//                                                                   B = three balanced s8 digit planes
+//                                                                       of the fixed-point query
+//   O^T[128 dims x 4 CP]    += level(V)^T[128 x 128 tokens] . Wd    A = V tile (u8, MN-major),
+//                                                                   B = the four bytes of the u32
+//                                                                       fixed-point weights (MN-major)
+// CP = query columns (n_q * G) padded to 4, 8, 16 or 32.  The int32 accumulators are exact, so
+// there is no rounding in either product: the query is good to 2^-22 of its largest entry and a
+// weight to 2^-28 of the largest weight seen so far.
+//
+// Weights.  For token t and column c,  x = s * log2(e) + log2(scale_v(t))  and  W = 2^(x - ref[c])
+// rounded to a u32, with ref[c] chosen so that the largest W of the first unit is 2^28; a later x
+// that would push W beyond 2^31.5 raises ref[c] (rare), which ends the current accumulation: the
+// int32 accumulators are added, scaled, into an FP32 copy (also in tensor memory) and restart
+// from zero.  The same happens before they could overflow.  The softmax sums use the unrounded
+// W / scale_v, so a single attended token reproduces its value row to FP32 rounding.
+//
+// Warp roles of a CTA (one CTA per SM):
+//   2 softmax warpgroups take alternate units; each has its own S, O and FP32 copy in tensor
+//     memory, its own reference exponents and its own P tile.  A thread owns one token of the
+//     unit (TMEM lane = token for S) and, when accumulators are read back, one output dim.
+//   4 + 4 expander warps turn the nibble planes of a raw stage into the u8 level tiles of K and
+//     of V (128-byte-swizzled canonical layout, the same bytes K-major for K and MN-major for V);
+//     the K expanders also build the query digit planes of a piece.
+//   4 producer warps stream the raw planes into a shared-memory ring (cp.async.bulk).
+//   1 thread issues every tcgen05.mma and commit.
+// All hand-offs are mbarriers with bounded waits; nothing waits on another CTA.
+//
+// Element order along head_dim inside operand tiles: byte 16 (2 j + parity) + 4 w + i of a row
+// holds dim 32 j + 8 w + 2 i + parity (what the nibble expansion yields with two logic
+// operations per word); the query planes use the same order and O is un-permuted at write-out.
+
+template <bool FULL, int CP>
+struct I8Cfg {
+  static_assert(CP == 4 || CP == 8 || CP == 16, "padded column counts");
+  static constexpr int kST = 128;                   // tokens per stage-unit
+  static constexpr int kNArr = FULL ? 6 : 4;        // arrays copied per 16-token sub-block
+  static constexpr int kStageBytes = kST * (FULL ? 272 : 144);
+  static constexpr int kOffKA = 0, kOffVA = kST * 64, kOffKR = kST * 128, kOffVR = kST * 192;
+  static constexpr int kOffKM = FULL ? kST * 256 : kST * 128, kOffVM = kOffKM + kST * 8;
+  static constexpr int kNQK = (3 * CP + 15) / 16 * 16;   // N of the Q.K^T product
+  static constexpr int kNPV = 4 * CP;                    // N of the P.V product
+  static constexpr int kPartCols = CP < 8 ? 8 : CP;      // column stride of the partial slots
+  static constexpr int kColsPad = CP;
+  // warps: softmax 0..7, K expanders 8..11, V expanders 12..15, producers 16..19, MMA 20
+  static constexpr int kSoftWarps = 8, kKWarps = 4, kVWarps = 4, kProdWarps = 4;
+  static constexpr int kKWarp0 = kSoftWarps, kVWarp0 = kKWarp0 + kKWarps, kProdWarp0 = kVWarp0 + kVWarps;
+  static constexpr int kMmaWarp = kProdWarp0 + kProdWarps;
+  static constexpr int kThreads = (kMmaWarp + 1) * 32;
+  // shared memory map (offsets from a 1024-byte aligned base)
+  static constexpr int kTile = 16384;                    // [128 rows][128 B]
+  static constexpr int kOffKT = 0, kOffVT = 2 * kTile, kOffPT = 4 * kTile;
+  static constexpr int kOffQT = 6 * kTile;               // [2 slots][kNQK rows][128 B]
+  static constexpr int kQTile = kNQK * 128;
+  static constexpr int kOffRing = kOffQT + 2 * ((kQTile + 1023) / 1024 * 1024);
+  static constexpr int kFixedTail = 2 * CP * 256         // raw BF16 queries, 2 slots
+                                    + 2 * 8 * CP * 4     // per group: qs, ref, factor, limits, reduce scratch ...
+                                    + 2 * 4 * 2 * CP * 4 // ... [4 warps][2 CP]
+                                    + 2 * 2 * CP * 4     // ... totals of l and zs
+                                    + kProdWarps * 2 * kPieceUnits * 4 + 2 * 32 + 64 * 8 + 3 * 256 + 64;
+  static constexpr int kAvail = 227 * 1024 - 1024 - kOffRing - kFixedTail;
+  static constexpr int kNStage = kAvail / kStageBytes > 6 ? 6 : kAvail / kStageBytes;
+  static_assert(kNStage >= 2, "ring too small");
+  static constexpr int kOffQRaw = kOffRing + kNStage * kStageBytes;
+  static constexpr int kOffScal = kOffQRaw + 2 * CP * 256;       // per group [8][CP] floats
+  static constexpr int kOffRed = kOffScal + 2 * 8 * CP * 4;      // per group [4 warps][2 CP]
+  static constexpr int kOffLz = kOffRed + 2 * 4 * 2 * CP * 4;    // per group [2 CP]
+  static constexpr int kOffBlk = kOffLz + 2 * 2 * CP * 4;
+  static constexpr int kOffItems = kOffBlk + kProdWarps * 2 * kPieceUnits * 4;
+  static constexpr int kOffBars = kOffItems + 2 * 32;
+  static constexpr int kOffMisc = kOffBars + 64 * 8;             // [3][64] ints: common, group 0, group 1
+  static constexpr int kSmem = kOffMisc + 3 * 256 + 64 + 1024;   // + alignment slack
+  static_assert(kSmem <= 227 * 1024, "shared memory");
+  // tensor memory columns of a softmax group: S, O accumulators, FP32 copy of O
+  static constexpr int kTmS = 0, kTmO = kNQK, kTmOF = kNQK + kNPV;
+  static constexpr int kTmWg = CP == 4 ? 64 : 128;
+  static constexpr int kTmCols = 2 * kTmWg;
+  static_assert(kTmOF + CP <= kTmWg, "tensor memory");
+  static constexpr int kDrainUnits = FULL ? 256 : 4096;  // own units after which the int32 sums could overflow
+  static_assert(CP * 512 + 3 * CP * 4 <= kTile, "the end-of-piece mailbox lives in a P tile");
+};
+
+template <>
+struct TmemRegs<4> {
+  static __device__ __forceinline__ void ld(uint32_t a, uint32_t* r) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a) : "memory");
+  }
+  static __device__ __forceinline__ void st(uint32_t a, const uint32_t* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1,%2,%3,%4};"
+                 ::"r"(a), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
+  }
+};
+
+// Instruction descriptor of kind::i8: int32 accumulate, u8 A, u8 or s8 B, M = 128.
+__host__ __device__ constexpr uint32_t i8_idesc(int n, bool mn_major, bool b_signed) {
+  return (2u << 4) | ((b_signed ? 1u : 0u) << 10) | ((mn_major ? 1u : 0u) << 15) | ((mn_major ? 1u : 0u) << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void i8_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+// barrier among `n` threads that also ORs a predicate over them
+__device__ __forceinline__ bool bar_or(int id, int n, bool pred) {
+  uint32_t res;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\t"
+      "barrier.cta.red.or.pred q, %2, %3, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(res) : "r"(pred ? 1u : 0u), "r"(id), "r"(n) : "memory");
+  return res != 0;
+}
+__device__ __forceinline__ void bar_arrive(int id, int n) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory");
+}
+__device__ __forceinline__ float lg2_approx(float x) {
+  float y;
+  asm("lg2.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float ex2_full(float x) {   // no flush of small results
+  float y;
+  asm("ex2.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Expand the nibble planes of one tensor of a 128-token raw stage into its u8 level tile.  A warp
+// takes 8 token rows per step (512 contiguous raw bytes): lane = (row & 7) * 4 + 16-byte chunk.
+template <bool FULL>
+__device__ __forceinline__ void i8_expand(uint32_t raw_a, uint32_t raw_r, uint32_t tile, int w4, int lane) {
+  const int row8 = lane >> 2, j = lane & 3;
+  uint4 xa[4], xr[4];
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    const uint32_t off = (uint32_t)(((w4 + 4 * s) * 8 + row8) * 64 + j * 16);
+    xa[s] = lds128(raw_a + off);
+    if (FULL) xr[s] = lds128(raw_r + off);
+  }
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    const int row = (w4 + 4 * s) * 8 + row8;
+    const uint32_t a[4] = {xa[s].x, xa[s].y, xa[s].z, xa[s].w};
+    uint32_t ev[4], od[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (FULL) {
+        const uint32_t r[4] = {xr[s].x, xr[s].y, xr[s].z, xr[s].w};
+        merge_codes(a[k], r[k], ev[k], od[k]);
+      } else {
+        ev[k] = a[k] & 0x0F0F0F0Fu;
+        od[k] = (a[k] >> 4) & 0x0F0F0F0Fu;
+      }
+    }
+    const uint32_t base = tile + (uint32_t)row * 128u;
+    const uint32_t c0 = (uint32_t)((2 * j) ^ (row & 7)) << 4, c1 = (uint32_t)((2 * j + 1) ^ (row & 7)) << 4;
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + c0), "r"(ev[0]), "r"(ev[1]), "r"(ev[2]),
+                 "r"(ev[3]) : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + c1), "r"(od[0]), "r"(od[1]), "r"(od[2]),
+                 "r"(od[3]) : "memory");
+  }
+}
+
+// One of the producer warps: the stream-K bookkeeping (every warp derives the same range and
+// pieces; warp 0 alone publishes them, loads the queries and handles empty sequences) and, per
+// unit, its share of the plane copies: 8 sub-blocks of 16 tokens x kNArr arrays, two sub-blocks
+// per warp.
+template <class C, bool FULL>
+__device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lane, uint32_t ring_u32,
+                                            uint32_t full0, uint32_t empty0, uint32_t qfull0, uint32_t qempty0,
+                                            uint32_t qraw_u32, uint32_t* blk_s, Item* items, int* misc,
+                                            volatile int* abort_word) {
+  constexpr int ST = C::kST, NSTAGE = C::kNStage, NARR = C::kNArr;
+  const int n_cta = gridDim.x, cta = blockIdx.x;
+  const int cap = p.max_blocks * p.bt;
+  auto clamp_len = [&](int b) {
+    int len = __ldg(p.seq_lens + b);
+    return len < 0 ? 0 : (len > cap ? cap : len);
+  };
+  long long tot = 0;
+  for (int b = lane; b < p.B; b += 32) tot += (clamp_len(b) + ST - 1) / ST;
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) tot += __shfl_xor_sync(0xFFFFFFFFu, tot, off);
+  const long long T = tot * p.Hkv;
+  const long long q = (T + n_cta - 1) / n_cta;
+  const long long lo = (long long)cta * q, hi = (lo + q < T) ? lo + q : T;
+  int b_lo = 0;
+  long long off_lo = 0;
+  if (lo < hi) {
+    long long running = 0;
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+      const int b = b0 + lane;
+      const long long u = b < p.B ? (long long)p.Hkv * ((clamp_len(b) + ST - 1) / ST) : 0;
+      long long incl = u;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const long long v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      const long long excl = running + incl - u;
+      const bool hit = u > 0 && lo >= excl && lo < excl + u;
+      const unsigned mk = __ballot_sync(0xFFFFFFFFu, hit);
+      if (mk) {
+        const int src = __ffs(mk) - 1;
+        b_lo = b0 + src;
+        off_lo = lo - __shfl_sync(0xFFFFFFFFu, excl, src);
+        break;
+      }
+      running += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+  }
+  if (pw == 0) {
+    if (lane == 0) misc[7] = lo < hi ? (int)(hi - lo) : 0;
+    // sequences with no token: outputs are zero, nothing is rejected unless the draft is not zero
+    for (int b = cta; b < p.B; b += n_cta) {
+      if (clamp_len(b) != 0) continue;
+      const size_t n = (size_t)p.nq * p.Hq * LYNX_D;
+      for (size_t i = lane; i < n; i += 32) p.out[(size_t)b * n + i] = 0.0f;
+      if (FULL && p.draft != nullptr) {
+        int fr = p.nq;
+        for (int j = p.nq - 1; j >= 0; --j) {
+          float worst = 0.0f;
+          for (int i = lane; i < p.Hq * LYNX_D; i += 32)
+            worst = fmaxf(worst, fabsf(__ldg(p.draft + ((size_t)b * p.nq + j) * p.Hq * LYNX_D + i)) / p.atol);
+#pragma unroll
+          for (int off = 16; off >= 1; off >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xFFFFFFFFu, worst, off));
+          if (lane == 0) p.dev[(size_t)b * p.nq + j] = worst;
+          if (worst > 1.0f) fr = j;
+        }
+        if (lane == 0) p.first_reject[b] = fr;
+      }
+    }
+  }
+  __syncthreads();  // (A) the range is published
+  const int n_units = (int)(lo < hi ? hi - lo : 0);
+  if (n_units == 0) return;
+
+  constexpr int RP = 2 * NARR;                 // roles of this warp: (sub-block, array) of two sub-blocks
+  const int role = pw * RP + (lane < RP ? lane : 0);
+  const int sub = role / NARR, arr = role % NARR, sub_first = 2 * pw;
+  const bool is_meta = arr == 2 || arr == 3;
+  const unsigned char* my_src = arr == 0 ? p.ka : arr == 1 ? p.va
+                              : arr == 2 ? reinterpret_cast<const unsigned char*>(p.km)
+                              : arr == 3 ? reinterpret_cast<const unsigned char*>(p.vm)
+                              : arr == 4 ? p.kr : p.vr;
+  const uint32_t my_bytes = is_meta ? 128u : 1024u, my_mul = is_meta ? 8u : 64u;
+  const uint32_t my_dst = (uint32_t)(arr == 0 ? C::kOffKA : arr == 1 ? C::kOffVA : arr == 2 ? C::kOffKM
+                                     : arr == 3 ? C::kOffVM : arr == 4 ? C::kOffKR : C::kOffVR) +
+                          (uint32_t)sub * my_bytes;
+  constexpr uint32_t kBytesSub = (FULL ? 4u : 2u) * 1024u + 2u * 128u;   // bytes of one sub-block
+  uint32_t* my_blk = blk_s + pw * 2 * kPieceUnits;   // [2 sub-blocks][kPieceUnits]
+  int b = b_lo, len = clamp_len(b), U = (len + ST - 1) / ST;
+  int hkv = (int)(off_lo / U), u = (int)(off_lo % U);
+  int remaining = n_units, gs = 0, ic = 0;
+  while (remaining > 0) {
+    const int n = min(remaining, U - u);
+    const int qi = ic & 1;
+    if (pw == 0) {
+      if (ic >= 2) mbar_wait(qempty0 + qi * 8, ((ic >> 1) - 1) & 1, abort_word);
+      const long long seg0 = lo + (n_units - remaining) - u;  // first unit of this segment
+      if (lane == 0) {
+        Item it;
+        it.b = b; it.hkv = hkv; it.len = len;
+        it.first_cta = (int)(seg0 / q);
+        it.n_contrib = (int)((seg0 + U - 1) / q) - it.first_cta + 1;
+        it.pad0 = n; it.pad1 = u; it.pad2 = 0;
+        items[qi] = it;
+        mbar_expect_tx(qfull0 + qi * 8, (uint32_t)(p.nq * p.G * LYNX_D * 2));
+      }
+      __syncwarp();
+      for (int j = lane; j < p.nq; j += 32)
+        bulk_g2s(qraw_u32 + (uint32_t)((qi * C::kColsPad + j * p.G) * LYNX_D * 2),
+                 p.q + (((size_t)b * p.nq + j) * p.Hq + (size_t)hkv * p.G) * LYNX_D,
+                 (uint32_t)(p.G * LYNX_D * 2), qfull0 + qi * 8);
+    }
+    for (int c0 = 0; c0 < n; c0 += kPieceUnits) {
+      const int cn = min(kPieceUnits, n - c0);
+      for (int i2 = lane; i2 < 2 * cn; i2 += 32) {
+        const int i = i2 >> 1;
+        const int t0 = (u + c0 + i) * ST + (sub_first + (i2 & 1)) * 16;
+        uint32_t row = 0xFFFFFFFFu;  // sub-block beyond the end of the sequence: nothing to copy
+        if (t0 < len) {
+          int blk = __ldg(p.block_table + (size_t)b * p.max_blocks + t0 / p.bt);
+          if (blk < 0 || blk >= p.num_blocks) {
+            atomicOr(p.ws_flags, kFlagBadBlock);
+            blk = blk < 0 ? 0 : p.num_blocks - 1;
+          }
+          row = (uint32_t)(((size_t)blk * p.Hkv + hkv) * p.bt + (t0 % p.bt));
+        }
+        my_blk[(i2 & 1) * kPieceUnits + i] = row;
+      }
+      __syncwarp();
+      for (int k = 0; k < cn; ++k, ++gs) {
+        const int slot = gs % NSTAGE;
+        if (gs >= NSTAGE) mbar_wait(empty0 + slot * 8, ((gs / NSTAGE) - 1) & 1, abort_word);
+        const uint32_t row0 = my_blk[k], row1 = my_blk[kPieceUnits + k];
+        const uint32_t row = sub == sub_first ? row0 : row1;
+        const uint32_t bar = full0 + slot * 8;
+        if (lane == 0) {
+          const uint32_t bytes = (row0 != 0xFFFFFFFFu ? kBytesSub : 0u) + (row1 != 0xFFFFFFFFu ? kBytesSub : 0u);
+          if (bytes) mbar_expect_tx(bar, bytes);
+          else mbar_arrive(bar);
+        }
+        __syncwarp();
+        if (lane < RP && row != 0xFFFFFFFFu)
+          bulk_g2s(ring_u32 + slot * C::kStageBytes + my_dst, my_src + (size_t)row * my_mul, my_bytes, bar);
+      }
+      __syncwarp();  // my_blk is rewritten by the next round
+    }
+    remaining -= n;
+    u += n;
+    ++ic;
+    if (u == U && remaining > 0) {
+      u = 0;
+      if (++hkv == p.Hkv) {
+        hkv = 0;
+        do {
+          ++b;
+          len = b < p.B ? clamp_len(b) : 0;
+          U = (len + ST - 1) / ST;
+        } while (b < p.B && U == 0);
+        if (b >= p.B) break;  // cannot happen: the range ends inside the list
+      }
+    }
+  }
+}
+
+// Largest |q| of a piece's raw queries, by 128 threads (index i of 0..127), reduced over the
+// warp; the caller combines the warps.
+template <int CP>
+__device__ __forceinline__ float i8_q_absmax(const unsigned char* qraw, int i) {
+  float amax = 0.0f;
+  for (int k = i; k < CP * 16; k += 128) {
+    const uint4 v = reinterpret_cast<const uint4*>(qraw)[k];
+    const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      amax = fmaxf(amax, fabsf(__uint_as_float(ww[j] << 16)));
+      amax = fmaxf(amax, fabsf(__uint_as_float(ww[j] & 0xFFFF0000u)));
+    }
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, off));
+  return amax;
+}
+// Fixed-point exponent of a piece's queries: |q * 2^e| < 2^22.
+__device__ __forceinline__ int i8_q_exponent(float amax) {
+  int e = 0;
+  if (amax > 0.0f && amax < INFINITY) e = 21 - (((__float_as_int(amax) >> 23) & 0xFF) - 127);
+  return max(-100, min(100, e));
+}
+
+template <bool FULL, int CP>
+__global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(const AttnParams p) {
+  using C = I8Cfg<FULL, CP>;
+  constexpr int NSTAGE = C::kNStage;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  const uint32_t sbase = smem_u32(smem);
+  unsigned char* qraw = smem + C::kOffQRaw;
+  float* scal = reinterpret_cast<float*>(smem + C::kOffScal);
+  float* red = reinterpret_cast<float*>(smem + C::kOffRed);
+  float* lz = reinterpret_cast<float*>(smem + C::kOffLz);
+  uint32_t* blk_s = reinterpret_cast<uint32_t*>(smem + C::kOffBlk);
+  Item* items = reinterpret_cast<Item*>(smem + C::kOffItems);
+  int* misc = reinterpret_cast<int*>(smem + C::kOffMisc);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t ring_u32 = sbase + C::kOffRing;
+  const uint32_t full0 = sbase + C::kOffBars, empty0 = full0 + NSTAGE * 8;
+  const uint32_t qfull0 = empty0 + NSTAGE * 8, qempty0 = qfull0 + 16;
+  const uint32_t kready0 = qempty0 + 16, vready0 = kready0 + 16, sfull0 = vready0 + 16, sfree0 = sfull0 + 16,
+                 pready0 = sfree0 + 16, pvdone0 = pready0 + 16;
+  volatile int* abort_word = misc;
+  // misc[8] = tensor memory base, misc[10 + g] = "P.V of group g accumulates"; misc[12] = scratch of the K expanders
+
+  if (tid == 0) {
+    for (int i = 0; i < NSTAGE; ++i) {
+      mbar_init(full0 + i * 8, C::kProdWarps);
+      mbar_init(empty0 + i * 8, C::kKWarps + C::kVWarps + 4);   // both expander teams and the owning softmax group
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(qfull0 + i * 8, 1);
+      mbar_init(qempty0 + i * 8, C::kSoftWarps + C::kKWarps + C::kVWarps);
+      mbar_init(kready0 + i * 8, C::kKWarps);   // K tile (and, at the start of a piece, the query planes) written
+      mbar_init(vready0 + i * 8, C::kVWarps);   // V tile written
+      mbar_init(sfull0 + i * 8, 1);             // Q.K^T complete (tcgen05.commit): S valid, K tile free
+      mbar_init(sfree0 + i * 8, 4);             // the group holds its scores in registers
+      mbar_init(pready0 + i * 8, 4);            // the group's weights are in its P tile
+      mbar_init(pvdone0 + i * 8, 1);            // P.V complete (tcgen05.commit): P and V tiles free
+    }
+    for (int i = 0; i < 3 * 64 + 16; ++i) misc[i] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // raw query slots (their padding columns stay zero) and query digit planes (their padding rows too)
+  for (int i = tid; i < 2 * CP * 256 / 16; i += C::kThreads) reinterpret_cast<uint4*>(qraw)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < (C::kOffRing - C::kOffQT) / 16; i += C::kThreads)
+    reinterpret_cast<uint4*>(smem + C::kOffQT)[i] = make_uint4(0, 0, 0, 0);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+
+  if (warp >= C::kProdWarp0 && warp < C::kMmaWarp) {
+    i8_producer<C, FULL>(p, warp - C::kProdWarp0, lane, ring_u32, full0, empty0, qfull0, qempty0,
+                         sbase + C::kOffQRaw, blk_s, items, misc, abort_word);
+    return;
+  }
+  __syncthreads();  // (A)
+  const int n_units = misc[7];
+  if (n_units == 0) return;
+
+  constexpr uint32_t kIdescS = i8_idesc(C::kNQK, false, true), kIdescO = i8_idesc(C::kNPV, true, false);
+
+  // =============================================================================================
+  // K expanders: query digit planes at the start of a piece, K level tile of every unit
+  // =============================================================================================
+  if (warp >= C::kKWarp0 && warp < C::kVWarp0) {
+    const int w4 = warp - C::kKWarp0, kt = tid - C::kKWarp0 * 32;
+    float* amax_s = reinterpret_cast<float*>(misc + 12);
+    int gs_base = 0, ic = 0;
+    while (gs_base < n_units) {
+      const int qi = ic & 1;
+      mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
+      const int n_piece = items[qi].pad0;
+      for (int u = 0; u < n_piece; ++u) {
+        const int gs = gs_base + u, g = gs & 1, slot = gs % NSTAGE;
+        mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
+        // the K tile of this parity (and the query planes of the piece before last) were last read by
+        // the Q.K^T of unit gs - 2
+        if (gs >= 2) mbar_wait(sfull0 + g * 8, ((gs >> 1) - 1) & 1, abort_word);
+        if (u == 0) {
+          // three balanced s8 digit planes of q_int = rint(q 2^e), rows plane * CP + column
+          const unsigned char* qb = qraw + qi * CP * 256;
+          const float am = i8_q_absmax<CP>(qb, kt);
+          if (lane == 0) amax_s[w4] = am;
+          named_bar(7, C::kKWarps * 32);
+          const float amax = fmaxf(fmaxf(amax_s[0], amax_s[1]), fmaxf(amax_s[2], amax_s[3]));
+          const int e = i8_q_exponent(amax);
+          const float up = __int_as_float((127 + e) << 23);
+          const uint32_t qt = sbase + C::kOffQT + qi * ((C::kQTile + 1023) / 1024 * 1024);
+          if (kt < CP * 4) {
+            const int c = kt >> 2, j = kt & 3;
+            uint32_t pl[3][2][4];   // [plane][parity][word]
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+              const uint4 v = *reinterpret_cast<const uint4*>(qb + c * 256 + j * 64 + w * 16);
+              const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+              uint32_t acc[3][2] = {{0, 0}, {0, 0}, {0, 0}};
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+#pragma unroll
+                for (int par = 0; par < 2; ++par) {
+                  const float f = par ? __uint_as_float(ww[i] & 0xFFFF0000u) : __uint_as_float(ww[i] << 16);
+                  int qv = __float2int_rn(f * up);
+                  qv = max(-4194303, min(4194303, qv));
+#pragma unroll
+                  for (int pln = 0; pln < 3; ++pln) {
+                    const int dgt = (int)(signed char)(qv & 0xFF);
+                    acc[pln][par] |= (uint32_t)(dgt & 0xFF) << (8 * i);
+                    qv = (qv - dgt) >> 8;
+                  }
+                }
+              }
+#pragma unroll
+              for (int pln = 0; pln < 3; ++pln) { pl[pln][0][w] = acc[pln][0]; pl[pln][1][w] = acc[pln][1]; }
+            }
+#pragma unroll
+            for (int pln = 0; pln < 3; ++pln) {
+              const int n = pln * CP + c;
+#pragma unroll
+              for (int par = 0; par < 2; ++par) {
+                const uint32_t a = qt + (uint32_t)n * 128u + ((uint32_t)((2 * j + par) ^ (n & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pl[pln][par][0]),
+                             "r"(pl[pln][par][1]), "r"(pl[pln][par][2]), "r"(pl[pln][par][3]) : "memory");
+              }
+            }
+          }
+          named_bar(7, C::kKWarps * 32);   // amax_s may be rewritten
+        }
+        const uint32_t st = ring_u32 + slot * C::kStageBytes;
+        i8_expand<FULL>(st + C::kOffKA, st + C::kOffKR, sbase + C::kOffKT + g * C::kTile, w4, lane);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(kready0 + g * 8);
+          mbar_arrive(empty0 + slot * 8);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(qempty0 + qi * 8);
+      gs_base += n_piece;
+      ++ic;
+    }
+    return;
+  }
+  // =============================================================================================
+  // V expanders
+  // =============================================================================================
+  if (warp >= C::kVWarp0 && warp < C::kProdWarp0) {
+    const int w4 = warp - C::kVWarp0;
+    int gs_base = 0, ic = 0;
+    while (gs_base < n_units) {
+      const int qi = ic & 1;
+      mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
+      const int n_piece = items[qi].pad0;
+      for (int u = 0; u < n_piece; ++u) {
+        const int gs = gs_base + u, g = gs & 1, slot = gs % NSTAGE;
+        mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
+        if (gs >= 2) mbar_wait(pvdone0 + g * 8, ((gs >> 1) - 1) & 1, abort_word);   // the V tile was read by unit gs - 2
+        const uint32_t st = ring_u32 + slot * C::kStageBytes;
+        i8_expand<FULL>(st + C::kOffVA, st + C::kOffVR, sbase + C::kOffVT + g * C::kTile, w4, lane);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(vready0 + g * 8);
+          mbar_arrive(empty0 + slot * 8);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(qempty0 + qi * 8);
+      gs_base += n_piece;
+      ++ic;
+    }
+    return;
+  }
+
+  // ---- tensor memory ---------------------------------------------------------------------------
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(misc + 8)),
+                 "r"((uint32_t)C::kTmCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  named_bar(8, (C::kSoftWarps + 1) * 32);
+  tc_fence_after();
+  const uint32_t tmem0 = *reinterpret_cast<volatile uint32_t*>(misc + 8);
+
+  // =============================================================================================
+  // The MMA thread: issues what is ready, P.V before the next Q.K^T
+  // =============================================================================================
+  if (warp == C::kMmaWarp) {
+    if (lane == 0) {
+      int next_qk = 0, next_pv = 0, qk_end = 0, ic = 0, qk_qi = 0;
+      uint64_t t0 = globaltimer_ns();
+      uint32_t idle = 0;
+      while (next_pv < n_units) {
+        bool progress = false;
+        if (next_pv < next_qk) {
+          const int gs = next_pv, g = gs & 1;
+          const uint32_t par = (uint32_t)(gs >> 1) & 1u;
+          if (mbar_test(pready0 + g * 8, par) && mbar_test(vready0 + g * 8, par)) {
+            tc_fence_after();
+            const uint32_t acc = (uint32_t)*reinterpret_cast<volatile int*>(misc + 10 + g);
+            const uint32_t vt = sbase + C::kOffVT + g * C::kTile, pt = sbase + C::kOffPT + g * C::kTile;
+            const uint32_t d = tmem0 + g * C::kTmWg + C::kTmO;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              i8_mma_ss(d, tc_desc(vt + (uint32_t)ks * 4096u, 16384u, 1024u),
+                        tc_desc(pt + (uint32_t)ks * 4096u, 16384u, 1024u), kIdescO, (acc || ks > 0) ? 1u : 0u);
+            tc_commit(pvdone0 + g * 8);
+            ++next_pv;
+            progress = true;
+          }
+        }
+        if (next_qk < n_units) {
+          if (next_qk == qk_end) {   // the next piece: its length, its query slot
+            if (mbar_test(qfull0 + (ic & 1) * 8, (uint32_t)(ic >> 1) & 1u)) {
+              qk_qi = ic & 1;
+              qk_end += items[qk_qi].pad0;
+              ++ic;
+              progress = true;
+            }
+          } else {
+            const int gs = next_qk, g = gs & 1;
+            if (mbar_test(kready0 + g * 8, (uint32_t)(gs >> 1) & 1u) &&
+                (gs < 2 || mbar_test(sfree0 + g * 8, (uint32_t)((gs >> 1) - 1) & 1u))) {
+              tc_fence_after();
+              const uint32_t kt = sbase + C::kOffKT + g * C::kTile;
+              const uint32_t qt = sbase + C::kOffQT + qk_qi * ((C::kQTile + 1023) / 1024 * 1024);
+              const uint32_t d = tmem0 + g * C::kTmWg + C::kTmS;
+#pragma unroll
+              for (int ks = 0; ks < 4; ++ks)
+                i8_mma_ss(d, tc_desc(kt + (uint32_t)ks * 32u, 16u, 1024u), tc_desc(qt + (uint32_t)ks * 32u, 16u, 1024u),
+                          kIdescS, ks > 0 ? 1u : 0u);
+              tc_commit(sfull0 + g * 8);
+              ++next_qk;
+              progress = true;
+            }
+          }
+        }
+        if (progress) {
+          idle = 0;
+        } else if ((++idle & 1023u) == 0) {
+          if (idle == 1024u) t0 = globaltimer_ns();
+          if (*abort_word || globaltimer_ns() - t0 > 2000000000ull) {
+            *abort_word = 1;   // give up: the waiting groups see the abort word and run out their loops
+            break;
+          }
+        }
+      }
+    }
+    return;
+  }
+
+  // =============================================================================================
+  // Softmax groups
+  // =============================================================================================
+  const int wg = warp >> 2, w4 = warp & 3;
+  const int r = tid & 127;                        // token of the unit (S), output dim position (O): TMEM lane
+  const uint32_t lane_sel = (uint32_t)(w4 * 32) << 16;
+  const uint32_t tm_s = tmem0 + wg * C::kTmWg + C::kTmS + lane_sel;
+  const uint32_t tm_o = tmem0 + wg * C::kTmWg + C::kTmO + lane_sel;
+  const uint32_t tm_of = tmem0 + wg * C::kTmWg + C::kTmOF + lane_sel;
+  float* my_scal = scal + wg * 8 * CP;            // [0] qs, [1] ref, [2] factor, [3] limits (int), [4] column maxima
+  float* qs_s = my_scal, *ref_s = my_scal + CP, *fac_s = my_scal + 2 * CP;
+  int* lim_s = reinterpret_cast<int*>(my_scal + 3 * CP);
+  float* my_red = red + wg * 4 * 2 * CP;
+  float* my_lz = lz + wg * 2 * CP;
+  int* my_misc = misc + 64 * (1 + wg);
+  const int bar_wg = 1 + wg;                      // named barrier of this group
+  const uint32_t ptile = sbase + C::kOffPT + wg * C::kTile;
+  float* mail_mine = reinterpret_cast<float*>(smem + C::kOffPT + wg * C::kTile);          // this group deposits here
+  const float* mail_other = reinterpret_cast<const float*>(smem + C::kOffPT + (wg ^ 1) * C::kTile);
+  const int dim_out = 32 * (r >> 5) + 8 * ((r >> 2) & 3) + 2 * (r & 3) + ((r >> 4) & 1);   // head dim of lane r of O
+  const float cb = p.sm_log2;
+  bool deposit_pending = false;                   // the other group has not yet read this group's last deposit
+
+  int gs_base = 0, ic = 0;
+  while (gs_base < n_units) {
+    const int qi = ic & 1;
+    mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
+    const Item item = items[qi];
+    const int len = item.len, n_piece = item.pad0;
+    const int u_first = ((gs_base & 1) == wg) ? 0 : 1;   // this group's units of the piece: u_first, u_first + 2, ...
+    if (u_first < n_piece) {
+      const int u_last = u_first + ((n_piece - 1 - u_first) & ~1);
+      const bool finisher = u_last == n_piece - 1;
+      const int full_lim = p.causal ? len - p.nq + 1 : len;
+      // ---- the piece's queries: fixed-point exponent, sum of q per column, causal limits ----------
+      const unsigned char* qb = qraw + qi * CP * 256;
+      {
+        const float am = i8_q_absmax<CP>(qb, r);
+        if (lane == 0) my_red[w4] = am;
+        for (int c = w4; c < CP; c += 4) {
+          const uint2 v = *reinterpret_cast<const uint2*>(qb + c * 256 + lane * 8);
+          float sum = (__uint_as_float(v.x << 16) + __uint_as_float(v.x & 0xFFFF0000u)) +
+                      (__uint_as_float(v.y << 16) + __uint_as_float(v.y & 0xFFFF0000u));
+#pragma unroll
+          for (int off = 16; off >= 1; off >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, off);
+          if (lane == 0) qs_s[c] = sum;
+        }
+        if (r < CP) lim_s[r] = r < p.ncols ? (p.causal ? len - p.nq + r / p.G + 1 : len) : 0;
+        named_bar(bar_wg, 128);
+      }
+      const float amax = fmaxf(fmaxf(my_red[0], my_red[1]), fmaxf(my_red[2], my_red[3]));
+      const int e = i8_q_exponent(amax);
+      const float ca = p.sm_log2 * __int_as_float((127 - e) << 23) * (FULL ? 1.0f : 16.0f);
+      named_bar(bar_wg, 128);   // my_red is reused below
+
+      float l[CP], zs[CP];
+#pragma unroll
+      for (int c = 0; c < CP; ++c) { l[c] = 0.0f; zs[c] = 0.0f; }
+      bool fresh = true, have_of = false;
+      int units_in_acc = 0;
+      uint32_t n_own = (uint32_t)((gs_base + u_first) >> 1);   // index of the unit among this group's units
+
+      // Ends the current accumulation: O accumulators (int32, four byte planes per column) are added to
+      // the FP32 copy, and the sum is scaled by fac_s[] (the change of the reference exponents).
+      auto drain = [&](bool scale) {
+        if (units_in_acc > 0) {
+          mbar_wait(pvdone0 + wg * 8, (n_own - 1) & 1, abort_word);   // the group's previous P.V is complete
+          tc_fence_after();
+#pragma unroll
+          for (int c4 = 0; c4 < CP / 4; ++c4) {
+            uint32_t a[16], of[4];
+            TmemRegs<16>::ld(tm_o + c4 * 16, a);
+            if (have_of) TmemRegs<4>::ld(tm_of + c4 * 4, of);
+            tc_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float v = fmaf(fmaf(fmaf((float)(int)a[4 * k + 3], 256.0f, (float)(int)a[4 * k + 2]), 256.0f,
+                                        (float)(int)a[4 * k + 1]), 256.0f, (float)(int)a[4 * k]);
+              // both the copy and the accumulators are relative to the old reference exponent
+              const float old = have_of ? __uint_as_float(of[k]) : 0.0f;
+              of[k] = __float_as_uint((old + v) * (scale ? fac_s[c4 * 4 + k] : 1.0f));
+            }
+            TmemRegs<4>::st(tm_of + c4 * 4, of);
+          }
+          tc_wait_st();
+          have_of = true;
+          units_in_acc = 0;
+        } else if (have_of && scale) {
+#pragma unroll
+          for (int c4 = 0; c4 < CP / 4; ++c4) {
+            uint32_t of[4];
+            TmemRegs<4>::ld(tm_of + c4 * 4, of);
+            tc_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 4; ++k) of[k] = __float_as_uint(__uint_as_float(of[k]) * fac_s[c4 * 4 + k]);
+            TmemRegs<4>::st(tm_of + c4 * 4, of);
+          }
+          tc_wait_st();
+        }
+      };
+
+      for (int u = u_first; u < n_piece; u += 2, ++n_own) {
+        const int gs = gs_base + u, slot = gs % NSTAGE;
+        const int unit_t0 = (item.pad1 + u) * C::kST;
+        const int tok = unit_t0 + r;
+        const uint32_t st = ring_u32 + slot * C::kStageBytes;
+        mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
+        float2 km = lds64f(st + C::kOffKM + r * 8), vm = lds64f(st + C::kOffVM + r * 8);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + slot * 8);
+        const bool valid = tok < len;
+        if (!valid) { km = make_float2(0.f, 0.f); vm = make_float2(0.f, 0.f); }
+        const float sve = fmaxf(FULL ? vm.x : 16.0f * vm.x, 9.094947e-13f);   // floor 2^-40: see the header
+        const float al = km.x * ca;
+        const float be = (FULL ? km.y : fmaf(km.x, 8.0f, km.y)) * cb;
+        const float lsv = lg2_approx(sve);
+        const float ia = valid ? rcp_approx(sve) : 0.0f;
+        const float ib = (FULL ? vm.y : fmaf(vm.x, 8.0f, vm.y)) * ia;
+
+        // ---- scores of this thread's token -------------------------------------------------------
+        mbar_wait(sfull0 + wg * 8, n_own & 1, abort_word);
+        tc_fence_after();
+        float x[CP];
+        {
+          uint32_t s0[CP], s1[CP], s2[CP];
+          TmemRegs<CP>::ld(tm_s, s0);
+          TmemRegs<CP>::ld(tm_s + CP, s1);
+          TmemRegs<CP>::ld(tm_s + 2 * CP, s2);
+          tc_wait_ld();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(sfree0 + wg * 8);
+#pragma unroll
+          for (int c = 0; c < CP; ++c) {
+            const float sf = fmaf((float)((int)s2[c] * 256 + (int)s1[c]), 256.0f, (float)(int)s0[c]);
+            x[c] = fmaf(sf, al, fmaf(be, qs_s[c], lsv));
+          }
+        }
+        if (unit_t0 + C::kST > full_lim) {
+#pragma unroll
+          for (int c = 0; c < CP; ++c)
+            if (tok >= lim_s[c]) x[c] = -INFINITY;
+        }
+        // ---- reference exponents: raised when a weight would leave the u32 range -----------------------
+        bool need = fresh || units_in_acc >= C::kDrainUnits;
+#pragma unroll
+        for (int c = 0; c < CP; ++c) need |= x[c] - ref_s[c] > 31.5f;
+        if (bar_or(bar_wg, 128, need)) {
+#pragma unroll
+          for (int c = 0; c < CP; ++c) {
+            float mx = x[c];
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+            if (lane == 0) my_red[w4 * CP + c] = mx;
+          }
+          named_bar(bar_wg, 128);
+          if (r < CP) {
+            const float mx = fmaxf(fmaxf(my_red[r], my_red[CP + r]), fmaxf(my_red[2 * CP + r], my_red[3 * CP + r]));
+            const float old = ref_s[r];
+            float nw = old, f = 1.0f;
+            if (fresh) { nw = fmaxf(mx, -1.0e4f) - 28.0f; f = 0.0f; }
+            else if (mx - old > 31.5f) { nw = mx - 28.0f; f = ex2_full(old - nw); }
+            ref_s[r] = nw;
+            fac_s[r] = f;
+          }
+          named_bar(bar_wg, 128);
+#pragma unroll
+          for (int c = 0; c < CP; ++c) { l[c] *= fac_s[c]; zs[c] *= fac_s[c]; }
+          drain(true);
+          fresh = false;
+        }
+        // ---- weights ------------------------------------------------------------------------------
+        uint32_t wi[CP];
+#pragma unroll
+        for (int c = 0; c < CP; ++c) {
+          const float wf = ex2_full(x[c] - ref_s[c]);
+          asm("cvt.rni.u32.f32 %0, %1;" : "=r"(wi[c]) : "f"(wf));
+          l[c] = fmaf(wf, ia, l[c]);
+          zs[c] = fmaf(wf, ib, zs[c]);
+        }
+        // the P tile is free once the group's previous P.V is complete (and the other group has read
+        // what this group deposited there at the end of the last piece)
+        if (units_in_acc > 0) mbar_wait(pvdone0 + wg * 8, (n_own - 1) & 1, abort_word);
+        if (deposit_pending) {
+          named_bar(5 + wg, 256);
+          deposit_pending = false;
+        }
+#pragma unroll
+        for (int j = 0; j < CP / 4; ++j)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(ptile + (uint32_t)r * 128u + ((uint32_t)(j ^ (r & 7)) << 4)), "r"(wi[4 * j]),
+                         "r"(wi[4 * j + 1]), "r"(wi[4 * j + 2]), "r"(wi[4 * j + 3]) : "memory");
+        if (r == 0) *reinterpret_cast<volatile int*>(misc + 10 + wg) = units_in_acc > 0 ? 1 : 0;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pready0 + wg * 8);
+        ++units_in_acc;
+      }
+      // ---- end of the piece for this group -----------------------------------------------------------
+      drain(false);   // waits for the last P.V; the FP32 copy now holds this group's part of O
+      float of[CP];
+#pragma unroll
+      for (int c4 = 0; c4 < CP / 4; ++c4) {
+        uint32_t t[4];
+        TmemRegs<4>::ld(tm_of + c4 * 4, t);
+        tc_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 4; ++k) of[c4 * 4 + k] = __uint_as_float(t[k]);
+      }
+      tc_fence_before();
+      // totals of l and zs over the group's 128 token lanes
+#pragma unroll
+      for (int c = 0; c < CP; ++c) {
+        float a = l[c], b = zs[c];
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+          a += __shfl_xor_sync(0xFFFFFFFFu, a, off);
+          b += __shfl_xor_sync(0xFFFFFFFFu, b, off);
+        }
+        if (lane == 0) { my_red[w4 * 2 * CP + c] = a; my_red[w4 * 2 * CP + CP + c] = b; }
+      }
+      named_bar(bar_wg, 128);
+      if (r < 2 * CP) my_lz[r] = (my_red[r] + my_red[2 * CP + r]) + (my_red[4 * CP + r] + my_red[6 * CP + r]);
+      named_bar(bar_wg, 128);
+      if (!finisher) {
+        // deposit (O, l, zs, ref) in this group's idle P tile for the group that owns the piece's last unit
+#pragma unroll
+        for (int c = 0; c < CP; ++c) mail_mine[c * 128 + r] = of[c];
+        if (r < CP) {
+          mail_mine[CP * 128 + r] = my_lz[r];
+          mail_mine[CP * 128 + CP + r] = my_lz[CP + r];
+          mail_mine[CP * 128 + 2 * CP + r] = ref_s[r];
+        }
+        __threadfence_block();
+        bar_arrive(3 + wg, 256);
+        deposit_pending = true;
+      } else {
+        float lt[CP], zt[CP], mt[CP];
+#pragma unroll
+        for (int c = 0; c < CP; ++c) { lt[c] = my_lz[c]; zt[c] = my_lz[CP + c]; mt[c] = ref_s[c]; }
+        if (n_piece >= 2) {
+          named_bar(3 + (wg ^ 1), 256);   // the other group's deposit is complete
+#pragma unroll
+          for (int c = 0; c < CP; ++c) {
+            const float o2 = mail_other[c * 128 + r], l2 = mail_other[CP * 128 + c];
+            const float z2 = mail_other[CP * 128 + CP + c], m2 = mail_other[CP * 128 + 2 * CP + c];
+            const float M = fmaxf(mt[c], m2);
+            const float f1 = ex2_full(mt[c] - M), f2 = ex2_full(m2 - M);
+            of[c] = of[c] * f1 + o2 * f2;
+            lt[c] = lt[c] * f1 + l2 * f2;
+            zt[c] = zt[c] * f1 + z2 * f2;
+            mt[c] = M;
+          }
+          bar_arrive(5 + (wg ^ 1), 256);   // its P tile may be written again
+        }
+        const bool direct = item.n_contrib == 1;
+        const size_t bh = (size_t)item.b * p.Hkv + item.hkv;
+        float* part = p.ws_part + (bh + (size_t)blockIdx.x) * (size_t)C::kPartCols * kPartStride;
+#pragma unroll
+        for (int c = 0; c < CP; ++c) {
+          if (c >= p.ncols) break;
+          const float v = of[c] + zt[c];
+          if (direct) {
+            const int j = c / p.G, hh = c % p.G;
+            p.out[(((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + dim_out] =
+                lt[c] > 0.0f ? v / lt[c] : 0.0f;
+          } else {
+            part[(size_t)c * kPartStride + dim_out] = v;
+            if (r == 0) { part[(size_t)c * kPartStride + 128] = mt[c]; part[(size_t)c * kPartStride + 129] = lt[c]; }
+          }
+        }
+        __threadfence();
+        finish_piece<FULL, C::kPartCols, 128>(p, item, direct, r, my_misc, bar_wg);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(qempty0 + qi * 8);
+    gs_base += n_piece;
+    ++ic;
+  }
+  // ---- release the tensor memory ---------------------------------------------------------------
+  tc_fence_before();
+  named_bar(9, C::kSoftWarps * 32);
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem0), "r"((uint32_t)C::kTmCols)
+                 : "memory");
+  }
+  if (tid == 0 && misc[0]) atomicOr(p.ws_flags, kFlagTimeout);
+}
+
+template <bool FULL, int CP>
+lynx_status launch_i8(const AttnParams& p, cudaStream_t st) {
+  using C = I8Cfg<FULL, CP>;
+  auto kern = attn_i8_kernel<FULL, CP>;
+  static bool configured[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmem) != cudaSuccess)
+      return LYNX_ERR_CUDA;
+    configured[dev] = true;
+  }
+  const long long cap_units = (long long)p.B * p.Hkv * (((long long)p.max_blocks * p.bt + C::kST - 1) / C::kST);
+  long long grid = (cap_units + 3) / 4;
+  const long long full = sm_count();   // one CTA per SM
+  grid = grid < 1 ? 1 : (grid > full ? full : grid);
+  kern<<<(unsigned)grid, C::kThreads, C::kSmem, st>>>(p);
+  return launch_status();
+}
