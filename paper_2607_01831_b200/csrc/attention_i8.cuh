@@ -50,26 +50,33 @@ struct I8Cfg {
   static constexpr int kNPV = 4 * CP;                    // N of the P.V product
   static constexpr int kPartCols = CP < 8 ? 8 : CP;      // column stride of the partial slots
   static constexpr int kColsPad = CP;
-  // warps: softmax 0..7, K expanders 8..11, V expanders 12..15, producers 16..19, MMA 20
-  static constexpr int kSoftWarps = 8, kKWarps = 4, kVWarps = 4, kProdWarps = 4;
-  static constexpr int kKWarp0 = kSoftWarps, kVWarp0 = kKWarp0 + kKWarps, kProdWarp0 = kVWarp0 + kVWarps;
-  static constexpr int kMmaWarp = kProdWarp0 + kProdWarps;
-  static constexpr int kThreads = (kMmaWarp + 1) * 32;
+  // warps: softmax 0..7 (two groups), K expanders 8..11, producers 12..15
+  static constexpr int kSoftWarps = 8, kKWarps = 4, kProdWarps = 4;
+  static constexpr int kKWarp0 = kSoftWarps, kProdWarp0 = kKWarp0 + kKWarps;
+  static constexpr int kThreads = (kProdWarp0 + kProdWarps) * 32;
   // shared memory map (offsets from a 1024-byte aligned base)
-  static constexpr int kTile = 16384;                    // [128 rows][128 B]
-  static constexpr int kOffKT = 0, kOffVT = 2 * kTile, kOffPT = 4 * kTile;
-  static constexpr int kOffQT = 6 * kTile;               // [2 slots][kNQK rows][128 B]
-  static constexpr int kQTile = kNQK * 128;
-  static constexpr int kOffRing = kOffQT + 2 * ((kQTile + 1023) / 1024 * 1024);
-  static constexpr int kFixedTail = 2 * CP * 256         // raw BF16 queries, 2 slots
-                                    + 2 * 8 * CP * 4     // per group: qs, ref, factor, limits, reduce scratch ...
-                                    + 2 * 4 * 2 * CP * 4 // ... [4 warps][2 CP]
-                                    + 2 * 2 * CP * 4     // ... totals of l and zs
+  static constexpr int kTile = 16384;                    // K and V level tiles: [128 rows][128 B]
+  static constexpr int kKSlots = (FULL && CP == 16) ? 2 : 3;
+  static constexpr int kVS = FULL ? 1 : 2;               // V and P tiles per softmax group
+  static constexpr int kPRow = 4 * CP < 32 ? 32 : 4 * CP;   // bytes of a P tile row (one token)
+  static constexpr int kPTile = 128 * kPRow;
+  static constexpr int kPLayout = kPRow == 32 ? 6 : kPRow == 64 ? 4 : 2;   // descriptor swizzle mode of the P tile
+  static constexpr int kQTile = (kNQK * 128 + 1023) / 1024 * 1024;
+  static constexpr int kMail = (CP * 128 + 3 * CP) * 4;    // end-of-piece deposit of a group: O, l, zs, ref
+  static constexpr int kOffKT = 0, kOffVT = kKSlots * kTile, kOffPT = kOffVT + 2 * kVS * kTile;
+  static constexpr int kPTileA = (kPTile + 1023) / 1024 * 1024;
+  static constexpr int kOffQT = kOffPT + 2 * kVS * kPTileA;
+  static constexpr int kOffRing = kOffQT + 2 * kQTile;
+  static constexpr int kFixedTail = 2 * kMail + 2 * CP * 256   // deposits; raw BF16 queries, 2 slots
+                                    + 2 * 8 * CP * 4     // per group: qs, ref, factor, limits
+                                    + 2 * 4 * 2 * CP * 4 // per group: reduce scratch [4 warps][2 CP]
+                                    + 2 * 2 * CP * 4     // per group: totals of l and zs
                                     + kProdWarps * 2 * kPieceUnits * 4 + 2 * 32 + 64 * 8 + 3 * 256 + 64;
   static constexpr int kAvail = 227 * 1024 - 1024 - kOffRing - kFixedTail;
   static constexpr int kNStage = kAvail / kStageBytes > 6 ? 6 : kAvail / kStageBytes;
   static_assert(kNStage >= 2, "ring too small");
-  static constexpr int kOffQRaw = kOffRing + kNStage * kStageBytes;
+  static constexpr int kOffMail = kOffRing + kNStage * kStageBytes;
+  static constexpr int kOffQRaw = kOffMail + 2 * kMail;
   static constexpr int kOffScal = kOffQRaw + 2 * CP * 256;       // per group [8][CP] floats
   static constexpr int kOffRed = kOffScal + 2 * 8 * CP * 4;      // per group [4 warps][2 CP]
   static constexpr int kOffLz = kOffRed + 2 * 4 * 2 * CP * 4;    // per group [2 CP]
@@ -79,13 +86,13 @@ struct I8Cfg {
   static constexpr int kOffMisc = kOffBars + 64 * 8;             // [3][64] ints: common, group 0, group 1
   static constexpr int kSmem = kOffMisc + 3 * 256 + 64 + 1024;   // + alignment slack
   static_assert(kSmem <= 227 * 1024, "shared memory");
-  // tensor memory columns of a softmax group: S, O accumulators, FP32 copy of O
-  static constexpr int kTmS = 0, kTmO = kNQK, kTmOF = kNQK + kNPV;
-  static constexpr int kTmWg = CP == 4 ? 64 : 128;
+  static_assert(kOffMail % 16 == 0 && kMail % 16 == 0 && kOffBars % 8 == 0, "alignment");
+  // tensor memory columns of a softmax group: two S buffers, O accumulators, FP32 copy of O
+  static constexpr int kTmS = 0, kTmO = 2 * kNQK, kTmOF = 2 * kNQK + kNPV;
+  static constexpr int kTmWg = CP == 4 ? 64 : CP == 8 ? 128 : 256;
   static constexpr int kTmCols = 2 * kTmWg;
   static_assert(kTmOF + CP <= kTmWg, "tensor memory");
   static constexpr int kDrainUnits = FULL ? 256 : 4096;  // own units after which the int32 sums could overflow
-  static_assert(CP * 512 + 3 * CP * 4 <= kTile, "the end-of-piece mailbox lives in a P tile");
 };
 
 template <>
@@ -365,10 +372,16 @@ __device__ __forceinline__ int i8_q_exponent(float amax) {
   return max(-100, min(100, e));
 }
 
+// Shared-memory matrix descriptor with the swizzle mode given (2 = 128 B, 4 = 64 B, 6 = 32 B).
+__device__ __forceinline__ uint64_t i8_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout << 61);
+}
+
 template <bool FULL, int CP>
 __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(const AttnParams p) {
   using C = I8Cfg<FULL, CP>;
-  constexpr int NSTAGE = C::kNStage;
+  constexpr int NSTAGE = C::kNStage, KS = C::kKSlots;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
@@ -383,37 +396,39 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   const uint32_t ring_u32 = sbase + C::kOffRing;
   const uint32_t full0 = sbase + C::kOffBars, empty0 = full0 + NSTAGE * 8;
   const uint32_t qfull0 = empty0 + NSTAGE * 8, qempty0 = qfull0 + 16;
-  const uint32_t kready0 = qempty0 + 16, vready0 = kready0 + 16, sfull0 = vready0 + 16, sfree0 = sfull0 + 16,
-                 pready0 = sfree0 + 16, pvdone0 = pready0 + 16;
+  const uint32_t kfree0 = qempty0 + 16;           // [KS]   Q.K^T of the unit in this K tile complete
+  const uint32_t sfull0 = kfree0 + KS * 8;        // [group][S buffer]  Q.K^T complete: scores valid
+  const uint32_t sfree0 = sfull0 + 32;            // [group][S buffer]  the group holds the scores in registers
+  const uint32_t pvdone0 = sfree0 + 32;           // [group][tile]  P.V complete: P and V tiles free, accumulators current
   volatile int* abort_word = misc;
-  // misc[8] = tensor memory base, misc[10 + g] = "P.V of group g accumulates"; misc[12] = scratch of the K expanders
+  // misc[8] = tensor memory base; misc[12..15] = scratch of the K expanders
 
   if (tid == 0) {
     for (int i = 0; i < NSTAGE; ++i) {
       mbar_init(full0 + i * 8, C::kProdWarps);
-      mbar_init(empty0 + i * 8, C::kKWarps + C::kVWarps + 4);   // both expander teams and the owning softmax group
+      mbar_init(empty0 + i * 8, C::kKWarps + 4);   // the K expanders and the softmax group that owns the unit
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(qfull0 + i * 8, 1);
-      mbar_init(qempty0 + i * 8, C::kSoftWarps + C::kKWarps + C::kVWarps);
-      mbar_init(kready0 + i * 8, C::kKWarps);   // K tile (and, at the start of a piece, the query planes) written
-      mbar_init(vready0 + i * 8, C::kVWarps);   // V tile written
-      mbar_init(sfull0 + i * 8, 1);             // Q.K^T complete (tcgen05.commit): S valid, K tile free
-      mbar_init(sfree0 + i * 8, 4);             // the group holds its scores in registers
-      mbar_init(pready0 + i * 8, 4);            // the group's weights are in its P tile
-      mbar_init(pvdone0 + i * 8, 1);            // P.V complete (tcgen05.commit): P and V tiles free
+      mbar_init(qempty0 + i * 8, C::kSoftWarps + C::kKWarps);
+    }
+    for (int i = 0; i < KS; ++i) mbar_init(kfree0 + i * 8, 1);
+    for (int i = 0; i < 4; ++i) {
+      mbar_init(sfull0 + i * 8, 1);
+      mbar_init(sfree0 + i * 8, 4);
+      mbar_init(pvdone0 + i * 8, 1);
     }
     for (int i = 0; i < 3 * 64 + 16; ++i) misc[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // raw query slots (their padding columns stay zero) and query digit planes (their padding rows too)
   for (int i = tid; i < 2 * CP * 256 / 16; i += C::kThreads) reinterpret_cast<uint4*>(qraw)[i] = make_uint4(0, 0, 0, 0);
-  for (int i = tid; i < (C::kOffRing - C::kOffQT) / 16; i += C::kThreads)
+  for (int i = tid; i < 2 * C::kQTile / 16; i += C::kThreads)
     reinterpret_cast<uint4*>(smem + C::kOffQT)[i] = make_uint4(0, 0, 0, 0);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
 
-  if (warp >= C::kProdWarp0 && warp < C::kMmaWarp) {
+  if (warp >= C::kProdWarp0) {
     i8_producer<C, FULL>(p, warp - C::kProdWarp0, lane, ring_u32, full0, empty0, qfull0, qempty0,
                          sbase + C::kOffQRaw, blk_s, items, misc, abort_word);
     return;
@@ -422,12 +437,23 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   const int n_units = misc[7];
   if (n_units == 0) return;
 
+  // ---- tensor memory ---------------------------------------------------------------------------
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(misc + 8)),
+                 "r"((uint32_t)C::kTmCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  named_bar(8, (C::kSoftWarps + C::kKWarps) * 32);
+  tc_fence_after();
+  const uint32_t tmem0 = *reinterpret_cast<volatile uint32_t*>(misc + 8);
   constexpr uint32_t kIdescS = i8_idesc(C::kNQK, false, true), kIdescO = i8_idesc(C::kNPV, true, false);
 
   // =============================================================================================
-  // K expanders: query digit planes at the start of a piece, K level tile of every unit
+  // K expanders: query digit planes at the start of a piece, K level tile of every unit, and the
+  // Q.K^T of the unit, issued by one of their threads as soon as the tile is complete
   // =============================================================================================
-  if (warp >= C::kKWarp0 && warp < C::kVWarp0) {
+  if (warp >= C::kKWarp0) {
     const int w4 = warp - C::kKWarp0, kt = tid - C::kKWarp0 * 32;
     float* amax_s = reinterpret_cast<float*>(misc + 12);
     int gs_base = 0, ic = 0;
@@ -436,12 +462,13 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
       mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
       const int n_piece = items[qi].pad0;
       for (int u = 0; u < n_piece; ++u) {
-        const int gs = gs_base + u, g = gs & 1, slot = gs % NSTAGE;
+        const int gs = gs_base + u, slot = gs % NSTAGE, ks = gs % KS;
         mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
-        // the K tile of this parity (and the query planes of the piece before last) were last read by
-        // the Q.K^T of unit gs - 2
-        if (gs >= 2) mbar_wait(sfull0 + g * 8, ((gs >> 1) - 1) & 1, abort_word);
+        // the K tile was last read by the Q.K^T of unit gs - KS
+        if (gs >= KS) mbar_wait(kfree0 + ks * 8, ((gs / KS) - 1) & 1, abort_word);
         if (u == 0) {
+          // the query planes of the piece before last were last read by a unit up to gs - 2
+          if (gs >= 2) mbar_wait(kfree0 + ((gs - 2) % KS) * 8, ((gs - 2) / KS) & 1, abort_word);
           // three balanced s8 digit planes of q_int = rint(q 2^e), rows plane * CP + column
           const unsigned char* qb = qraw + qi * CP * 256;
           const float am = i8_q_absmax<CP>(qb, kt);
@@ -450,7 +477,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           const float amax = fmaxf(fmaxf(amax_s[0], amax_s[1]), fmaxf(amax_s[2], amax_s[3]));
           const int e = i8_q_exponent(amax);
           const float up = __int_as_float((127 + e) << 23);
-          const uint32_t qt = sbase + C::kOffQT + qi * ((C::kQTile + 1023) / 1024 * 1024);
+          const uint32_t qt = sbase + C::kOffQT + qi * C::kQTile;
           if (kt < CP * 4) {
             const int c = kt >> 2, j = kt & 3;
             uint32_t pl[3][2][4];   // [plane][parity][word]
@@ -488,46 +515,28 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
               }
             }
           }
-          named_bar(7, C::kKWarps * 32);   // amax_s may be rewritten
         }
         const uint32_t st = ring_u32 + slot * C::kStageBytes;
-        i8_expand<FULL>(st + C::kOffKA, st + C::kOffKR, sbase + C::kOffKT + g * C::kTile, w4, lane);
+        const uint32_t ktile = sbase + C::kOffKT + ks * C::kTile;
+        i8_expand<FULL>(st + C::kOffKA, st + C::kOffKR, ktile, w4, lane);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(kready0 + g * 8);
-          mbar_arrive(empty0 + slot * 8);
+        if (lane == 0) mbar_arrive(empty0 + slot * 8);
+        named_bar(7, C::kKWarps * 32);   // the tile (and the query planes) are complete; amax_s may be rewritten
+        if (kt == 0) {
+          const int g = gs & 1, n = gs >> 1, b = n & 1;   // softmax group, its unit index, its S buffer
+          if (n >= 2) mbar_wait(sfree0 + (g * 2 + b) * 8, ((n >> 1) - 1) & 1, abort_word);
+          tc_fence_after();
+          const uint32_t qt = sbase + C::kOffQT + qi * C::kQTile;
+          const uint32_t d = tmem0 + g * C::kTmWg + C::kTmS + b * C::kNQK;
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            i8_mma_ss(d, i8_desc(ktile + (uint32_t)k4 * 32u, 16u, 1024u, 2u), i8_desc(qt + (uint32_t)k4 * 32u, 16u, 1024u, 2u),
+                      kIdescS, k4 > 0 ? 1u : 0u);
+          tc_commit(sfull0 + (g * 2 + b) * 8);
+          tc_commit(kfree0 + ks * 8);
         }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(qempty0 + qi * 8);
-      gs_base += n_piece;
-      ++ic;
-    }
-    return;
-  }
-  // =============================================================================================
-  // V expanders
-  // =============================================================================================
-  if (warp >= C::kVWarp0 && warp < C::kProdWarp0) {
-    const int w4 = warp - C::kVWarp0;
-    int gs_base = 0, ic = 0;
-    while (gs_base < n_units) {
-      const int qi = ic & 1;
-      mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
-      const int n_piece = items[qi].pad0;
-      for (int u = 0; u < n_piece; ++u) {
-        const int gs = gs_base + u, g = gs & 1, slot = gs % NSTAGE;
-        mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
-        if (gs >= 2) mbar_wait(pvdone0 + g * 8, ((gs >> 1) - 1) & 1, abort_word);   // the V tile was read by unit gs - 2
-        const uint32_t st = ring_u32 + slot * C::kStageBytes;
-        i8_expand<FULL>(st + C::kOffVA, st + C::kOffVR, sbase + C::kOffVT + g * C::kTile, w4, lane);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(vready0 + g * 8);
-          mbar_arrive(empty0 + slot * 8);
-        }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(qempty0 + qi * 8);
@@ -537,86 +546,8 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
     return;
   }
 
-  // ---- tensor memory ---------------------------------------------------------------------------
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(misc + 8)),
-                 "r"((uint32_t)C::kTmCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  named_bar(8, (C::kSoftWarps + 1) * 32);
-  tc_fence_after();
-  const uint32_t tmem0 = *reinterpret_cast<volatile uint32_t*>(misc + 8);
-
   // =============================================================================================
-  // The MMA thread: issues what is ready, P.V before the next Q.K^T
-  // =============================================================================================
-  if (warp == C::kMmaWarp) {
-    if (lane == 0) {
-      int next_qk = 0, next_pv = 0, qk_end = 0, ic = 0, qk_qi = 0;
-      uint64_t t0 = globaltimer_ns();
-      uint32_t idle = 0;
-      while (next_pv < n_units) {
-        bool progress = false;
-        if (next_pv < next_qk) {
-          const int gs = next_pv, g = gs & 1;
-          const uint32_t par = (uint32_t)(gs >> 1) & 1u;
-          if (mbar_test(pready0 + g * 8, par) && mbar_test(vready0 + g * 8, par)) {
-            tc_fence_after();
-            const uint32_t acc = (uint32_t)*reinterpret_cast<volatile int*>(misc + 10 + g);
-            const uint32_t vt = sbase + C::kOffVT + g * C::kTile, pt = sbase + C::kOffPT + g * C::kTile;
-            const uint32_t d = tmem0 + g * C::kTmWg + C::kTmO;
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              i8_mma_ss(d, tc_desc(vt + (uint32_t)ks * 4096u, 16384u, 1024u),
-                        tc_desc(pt + (uint32_t)ks * 4096u, 16384u, 1024u), kIdescO, (acc || ks > 0) ? 1u : 0u);
-            tc_commit(pvdone0 + g * 8);
-            ++next_pv;
-            progress = true;
-          }
-        }
-        if (next_qk < n_units) {
-          if (next_qk == qk_end) {   // the next piece: its length, its query slot
-            if (mbar_test(qfull0 + (ic & 1) * 8, (uint32_t)(ic >> 1) & 1u)) {
-              qk_qi = ic & 1;
-              qk_end += items[qk_qi].pad0;
-              ++ic;
-              progress = true;
-            }
-          } else {
-            const int gs = next_qk, g = gs & 1;
-            if (mbar_test(kready0 + g * 8, (uint32_t)(gs >> 1) & 1u) &&
-                (gs < 2 || mbar_test(sfree0 + g * 8, (uint32_t)((gs >> 1) - 1) & 1u))) {
-              tc_fence_after();
-              const uint32_t kt = sbase + C::kOffKT + g * C::kTile;
-              const uint32_t qt = sbase + C::kOffQT + qk_qi * ((C::kQTile + 1023) / 1024 * 1024);
-              const uint32_t d = tmem0 + g * C::kTmWg + C::kTmS;
-#pragma unroll
-              for (int ks = 0; ks < 4; ++ks)
-                i8_mma_ss(d, tc_desc(kt + (uint32_t)ks * 32u, 16u, 1024u), tc_desc(qt + (uint32_t)ks * 32u, 16u, 1024u),
-                          kIdescS, ks > 0 ? 1u : 0u);
-              tc_commit(sfull0 + g * 8);
-              ++next_qk;
-              progress = true;
-            }
-          }
-        }
-        if (progress) {
-          idle = 0;
-        } else if ((++idle & 1023u) == 0) {
-          if (idle == 1024u) t0 = globaltimer_ns();
-          if (*abort_word || globaltimer_ns() - t0 > 2000000000ull) {
-            *abort_word = 1;   // give up: the waiting groups see the abort word and run out their loops
-            break;
-          }
-        }
-      }
-    }
-    return;
-  }
-
-  // =============================================================================================
-  // Softmax groups
+  // Softmax groups: V level tile, scores -> weights, P.V (issued by one thread of the group)
   // =============================================================================================
   const int wg = warp >> 2, w4 = warp & 3;
   const int r = tid & 127;                        // token of the unit (S), output dim position (O): TMEM lane
@@ -624,19 +555,26 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   const uint32_t tm_s = tmem0 + wg * C::kTmWg + C::kTmS + lane_sel;
   const uint32_t tm_o = tmem0 + wg * C::kTmWg + C::kTmO + lane_sel;
   const uint32_t tm_of = tmem0 + wg * C::kTmWg + C::kTmOF + lane_sel;
-  float* my_scal = scal + wg * 8 * CP;            // [0] qs, [1] ref, [2] factor, [3] limits (int), [4] column maxima
+  float* my_scal = scal + wg * 8 * CP;            // qs, ref, factor, limits (int)
   float* qs_s = my_scal, *ref_s = my_scal + CP, *fac_s = my_scal + 2 * CP;
   int* lim_s = reinterpret_cast<int*>(my_scal + 3 * CP);
   float* my_red = red + wg * 4 * 2 * CP;
   float* my_lz = lz + wg * 2 * CP;
   int* my_misc = misc + 64 * (1 + wg);
   const int bar_wg = 1 + wg;                      // named barrier of this group
-  const uint32_t ptile = sbase + C::kOffPT + wg * C::kTile;
-  float* mail_mine = reinterpret_cast<float*>(smem + C::kOffPT + wg * C::kTile);          // this group deposits here
-  const float* mail_other = reinterpret_cast<const float*>(smem + C::kOffPT + (wg ^ 1) * C::kTile);
+  const uint32_t vtile0 = sbase + C::kOffVT + wg * C::kVS * C::kTile;
+  const uint32_t ptile0 = sbase + C::kOffPT + wg * C::kVS * C::kPTileA;
+  float* mail_mine = reinterpret_cast<float*>(smem + C::kOffMail + wg * C::kMail);
+  const float* mail_other = reinterpret_cast<const float*>(smem + C::kOffMail + (wg ^ 1) * C::kMail);
   const int dim_out = 32 * (r >> 5) + 8 * ((r >> 2) & 3) + 2 * (r & 3) + ((r >> 4) & 1);   // head dim of lane r of O
+  // this thread's row of the P tile: 16-byte chunk j goes to position j ^ p_swz
+  const uint32_t p_swz = C::kPRow == 32 ? ((uint32_t)r >> 2) & 1u : C::kPRow == 64 ? ((uint32_t)r >> 1) & 3u : (uint32_t)r & 7u;
+  const uint32_t p_row0 = ptile0 + (uint32_t)r * C::kPRow;
   const float cb = p.sm_log2;
   bool deposit_pending = false;                   // the other group has not yet read this group's last deposit
+  // completion barrier and phase parity of the P.V of this group's unit n (units alternate between the tiles)
+  auto pv_bar = [&](uint32_t n) { return pvdone0 + (uint32_t)(wg * 2 + (C::kVS == 2 ? (int)(n & 1u) : 0)) * 8u; };
+  auto pv_par = [&](uint32_t n) { return C::kVS == 2 ? (n >> 1) & 1u : n & 1u; };
 
   int gs_base = 0, ic = 0;
   while (gs_base < n_units) {
@@ -677,11 +615,11 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
       int units_in_acc = 0;
       uint32_t n_own = (uint32_t)((gs_base + u_first) >> 1);   // index of the unit among this group's units
 
-      // Ends the current accumulation: O accumulators (int32, four byte planes per column) are added to
-      // the FP32 copy, and the sum is scaled by fac_s[] (the change of the reference exponents).
+      // Ends the current accumulation (the group's last P.V is complete): the int32 accumulators, four
+      // byte planes per column, are added to the FP32 copy and the sum is scaled by fac_s[] (the change
+      // of the reference exponents).
       auto drain = [&](bool scale) {
         if (units_in_acc > 0) {
-          mbar_wait(pvdone0 + wg * 8, (n_own - 1) & 1, abort_word);   // the group's previous P.V is complete
           tc_fence_after();
 #pragma unroll
           for (int c4 = 0; c4 < CP / 4; ++c4) {
@@ -693,7 +631,6 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
             for (int k = 0; k < 4; ++k) {
               const float v = fmaf(fmaf(fmaf((float)(int)a[4 * k + 3], 256.0f, (float)(int)a[4 * k + 2]), 256.0f,
                                         (float)(int)a[4 * k + 1]), 256.0f, (float)(int)a[4 * k]);
-              // both the copy and the accumulators are relative to the old reference exponent
               const float old = have_of ? __uint_as_float(of[k]) : 0.0f;
               of[k] = __float_as_uint((old + v) * (scale ? fac_s[c4 * 4 + k] : 1.0f));
             }
@@ -718,16 +655,22 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
 
       for (int u = u_first; u < n_piece; u += 2, ++n_own) {
         const int gs = gs_base + u, slot = gs % NSTAGE;
+        const int sb = (int)(n_own & 1u);           // S buffer of this unit
         const int unit_t0 = (item.pad1 + u) * C::kST;
         const int tok = unit_t0 + r;
         const uint32_t st = ring_u32 + slot * C::kStageBytes;
         mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
         float2 km = lds64f(st + C::kOffKM + r * 8), vm = lds64f(st + C::kOffVM + r * 8);
+        // the V and P tiles of this unit are free once the P.V that last read them is complete
+        const uint32_t tb = C::kVS == 2 ? (n_own & 1u) : 0u;
+        const uint32_t vtile = vtile0 + tb * C::kTile, ptile = ptile0 + tb * C::kPTileA;
+        if (n_own >= (uint32_t)C::kVS) mbar_wait(pv_bar(n_own - C::kVS), pv_par(n_own - C::kVS), abort_word);
+        i8_expand<FULL>(st + C::kOffVA, st + C::kOffVR, vtile, w4, lane);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + slot * 8);
         const bool valid = tok < len;
         if (!valid) { km = make_float2(0.f, 0.f); vm = make_float2(0.f, 0.f); }
-        const float sve = fmaxf(FULL ? vm.x : 16.0f * vm.x, 9.094947e-13f);   // floor 2^-40: see the header
+        const float sve = fmaxf(FULL ? vm.x : 16.0f * vm.x, 9.094947e-13f);   // floor 2^-40
         const float al = km.x * ca;
         const float be = (FULL ? km.y : fmaf(km.x, 8.0f, km.y)) * cb;
         const float lsv = lg2_approx(sve);
@@ -735,18 +678,18 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         const float ib = (FULL ? vm.y : fmaf(vm.x, 8.0f, vm.y)) * ia;
 
         // ---- scores of this thread's token -------------------------------------------------------
-        mbar_wait(sfull0 + wg * 8, n_own & 1, abort_word);
+        mbar_wait(sfull0 + (wg * 2 + sb) * 8, (n_own >> 1) & 1, abort_word);
         tc_fence_after();
         float x[CP];
         {
           uint32_t s0[CP], s1[CP], s2[CP];
-          TmemRegs<CP>::ld(tm_s, s0);
-          TmemRegs<CP>::ld(tm_s + CP, s1);
-          TmemRegs<CP>::ld(tm_s + 2 * CP, s2);
+          TmemRegs<CP>::ld(tm_s + sb * C::kNQK, s0);
+          TmemRegs<CP>::ld(tm_s + sb * C::kNQK + CP, s1);
+          TmemRegs<CP>::ld(tm_s + sb * C::kNQK + 2 * CP, s2);
           tc_wait_ld();
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(sfree0 + wg * 8);
+          if (lane == 0) mbar_arrive(sfree0 + (wg * 2 + sb) * 8);
 #pragma unroll
           for (int c = 0; c < CP; ++c) {
             const float sf = fmaf((float)((int)s2[c] * 256 + (int)s1[c]), 256.0f, (float)(int)s0[c]);
@@ -783,6 +726,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           named_bar(bar_wg, 128);
 #pragma unroll
           for (int c = 0; c < CP; ++c) { l[c] *= fac_s[c]; zs[c] *= fac_s[c]; }
+          if (C::kVS > 1 && units_in_acc > 0) mbar_wait(pv_bar(n_own - 1), pv_par(n_own - 1), abort_word);
           drain(true);
           fresh = false;
         }
@@ -795,26 +739,30 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           l[c] = fmaf(wf, ia, l[c]);
           zs[c] = fmaf(wf, ib, zs[c]);
         }
-        // the P tile is free once the group's previous P.V is complete (and the other group has read
-        // what this group deposited there at the end of the last piece)
-        if (units_in_acc > 0) mbar_wait(pvdone0 + wg * 8, (n_own - 1) & 1, abort_word);
-        if (deposit_pending) {
-          named_bar(5 + wg, 256);
-          deposit_pending = false;
-        }
 #pragma unroll
         for (int j = 0; j < CP / 4; ++j)
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(ptile + (uint32_t)r * 128u + ((uint32_t)(j ^ (r & 7)) << 4)), "r"(wi[4 * j]),
-                         "r"(wi[4 * j + 1]), "r"(wi[4 * j + 2]), "r"(wi[4 * j + 3]) : "memory");
-        if (r == 0) *reinterpret_cast<volatile int*>(misc + 10 + wg) = units_in_acc > 0 ? 1 : 0;
+                       ::"r"(p_row0 + tb * C::kPTileA + (((uint32_t)j ^ p_swz) << 4)), "r"(wi[4 * j]), "r"(wi[4 * j + 1]),
+                         "r"(wi[4 * j + 2]), "r"(wi[4 * j + 3]) : "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        tc_fence_before();
+        named_bar(bar_wg, 128);     // the P tile and the V tile are complete
+        if (r == 0) {
+          tc_fence_after();
+          const uint32_t d = tmem0 + wg * C::kTmWg + C::kTmO;
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            i8_mma_ss(d, i8_desc(vtile + (uint32_t)k4 * 4096u, 16384u, 1024u, 2u),
+                      i8_desc(ptile + (uint32_t)k4 * (32u * C::kPRow), 16384u, 8u * C::kPRow, (uint32_t)C::kPLayout),
+                      kIdescO, (units_in_acc > 0 || k4 > 0) ? 1u : 0u);
+          tc_commit(pv_bar(n_own));
+        }
         __syncwarp();
-        if (lane == 0) mbar_arrive(pready0 + wg * 8);
         ++units_in_acc;
       }
       // ---- end of the piece for this group -----------------------------------------------------------
-      drain(false);   // waits for the last P.V; the FP32 copy now holds this group's part of O
+      mbar_wait(pv_bar(n_own - 1), pv_par(n_own - 1), abort_word);   // the last P.V
+      drain(false);   // the FP32 copy now holds this group's part of O
       float of[CP];
 #pragma unroll
       for (int c4 = 0; c4 < CP / 4; ++c4) {
@@ -840,7 +788,8 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
       if (r < 2 * CP) my_lz[r] = (my_red[r] + my_red[2 * CP + r]) + (my_red[4 * CP + r] + my_red[6 * CP + r]);
       named_bar(bar_wg, 128);
       if (!finisher) {
-        // deposit (O, l, zs, ref) in this group's idle P tile for the group that owns the piece's last unit
+        // deposit (O, l, zs, ref) for the group that owns the piece's last unit
+        if (deposit_pending) named_bar(5 + wg, 256);   // the previous deposit has been read
 #pragma unroll
         for (int c = 0; c < CP; ++c) mail_mine[c * 128 + r] = of[c];
         if (r < CP) {
@@ -868,7 +817,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
             zt[c] = zt[c] * f1 + z2 * f2;
             mt[c] = M;
           }
-          bar_arrive(5 + (wg ^ 1), 256);   // its P tile may be written again
+          bar_arrive(5 + (wg ^ 1), 256);   // it may deposit again
         }
         const bool direct = item.n_contrib == 1;
         const size_t bh = (size_t)item.b * p.Hkv + item.hkv;
