@@ -38,6 +38,8 @@
 // holds dim 32 j + 8 w + 2 i + parity (what the nibble expansion yields with two logic
 // operations per word); the query planes use the same order and O is un-permuted at write-out.
 
+constexpr int kI8PieceUnits = 32;  // stage-units whose block ids a producer warp looks up at a time
+
 template <bool FULL, int CP>
 struct I8Cfg {
   static_assert(CP == 4 || CP == 8 || CP == 16, "padded column counts");
@@ -50,48 +52,46 @@ struct I8Cfg {
   static constexpr int kNPV = 4 * CP;                    // N of the P.V product
   static constexpr int kPartCols = CP < 8 ? 8 : CP;      // column stride of the partial slots
   static constexpr int kColsPad = CP;
-  // warps: softmax 0..7 (two groups), K expanders 8..11, producers 12..15
-  static constexpr int kSoftWarps = 8, kKWarps = 4, kProdWarps = 4;
-  static constexpr int kKWarp0 = kSoftWarps, kProdWarp0 = kKWarp0 + kKWarps;
+  // warps: kTeams teams of four (team t = warps 4t .. 4t+3), then the producers
+  static constexpr int kTeams = (FULL || CP == 16) ? 3 : 4;
+  static constexpr int kProdWarps = 4;
+  static constexpr int kProdWarp0 = 4 * kTeams;
   static constexpr int kThreads = (kProdWarp0 + kProdWarps) * 32;
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int kTile = 16384;                    // K and V level tiles: [128 rows][128 B]
-  static constexpr int kKSlots = (FULL && CP == 16) ? 2 : 3;
-  static constexpr int kVS = FULL ? 1 : 2;               // V and P tiles per softmax group
   static constexpr int kPRow = 4 * CP < 32 ? 32 : 4 * CP;   // bytes of a P tile row (one token)
   static constexpr int kPTile = 128 * kPRow;
   static constexpr int kPLayout = kPRow == 32 ? 6 : kPRow == 64 ? 4 : 2;   // descriptor swizzle mode of the P tile
+  // Where shared memory is short the P tile shares the K tile's memory (K is dead once Q.K^T is complete,
+  // P is written after that); the next K expansion then has to wait for the P.V.
+  static constexpr bool kPAliasK = FULL ? CP >= 8 : CP == 8;
+  static constexpr int kTeamBytes = 2 * kTile + (kPAliasK ? 0 : kPTile);  // K tile, V tile, P tile
   static constexpr int kQTile = (kNQK * 128 + 1023) / 1024 * 1024;
-  static constexpr int kMail = (CP * 128 + 3 * CP) * 4;    // end-of-piece deposit of a group: O, l, zs, ref
-  static constexpr int kOffKT = 0, kOffVT = kKSlots * kTile, kOffPT = kOffVT + 2 * kVS * kTile;
-  static constexpr int kPTileA = (kPTile + 1023) / 1024 * 1024;
-  static constexpr int kOffQT = kOffPT + 2 * kVS * kPTileA;
+  static constexpr int kMail = (CP * 128 + 3 * CP) * 4;  // end-of-piece deposit of a team (in its V tile): O, l, zs, ref
+  static_assert(kMail <= kTile, "the deposit lives in the team's V tile");
+  static constexpr int kOffQT = kTeams * kTeamBytes;
   static constexpr int kOffRing = kOffQT + 2 * kQTile;
-  static constexpr int kFixedTail = 2 * kMail + 2 * CP * 256   // deposits; raw BF16 queries, 2 slots
-                                    + 2 * 8 * CP * 4     // per group: qs, ref, factor, limits
-                                    + 2 * 4 * 2 * CP * 4 // per group: reduce scratch [4 warps][2 CP]
-                                    + 2 * 2 * CP * 4     // per group: totals of l and zs
-                                    + kProdWarps * 2 * kPieceUnits * 4 + 2 * 32 + 64 * 8 + 3 * 256 + 64;
-  static constexpr int kAvail = 227 * 1024 - 1024 - kOffRing - kFixedTail;
-  static constexpr int kNStage = kAvail / kStageBytes > 6 ? 6 : kAvail / kStageBytes;
-  static_assert(kNStage >= 2, "ring too small");
-  static constexpr int kOffMail = kOffRing + kNStage * kStageBytes;
-  static constexpr int kOffQRaw = kOffMail + 2 * kMail;
-  static constexpr int kOffScal = kOffQRaw + 2 * CP * 256;       // per group [8][CP] floats
-  static constexpr int kOffRed = kOffScal + 2 * 8 * CP * 4;      // per group [4 warps][2 CP]
-  static constexpr int kOffLz = kOffRed + 2 * 4 * 2 * CP * 4;    // per group [2 CP]
-  static constexpr int kOffBlk = kOffLz + 2 * 2 * CP * 4;
-  static constexpr int kOffItems = kOffBlk + kProdWarps * 2 * kPieceUnits * 4;
+  static constexpr int kTeamScal = (8 * CP + 4 * 2 * CP + 2 * CP) * 4;   // qs, ref, factor, limits; reduce scratch; totals
+  static constexpr int kFixedTail = 2 * CP * 256 + kTeams * kTeamScal +
+                                    kProdWarps * 2 * kI8PieceUnits * 4 + 2 * 32 + 64 * 8 + (1 + kTeams) * 256 + 64;
+  // One raw stage per team: unit gs lands in stage gs % kTeams, the stage of the team that owns it, so
+  // every team sees the phases of its stage's barriers in order.  (A waiter that is a phase ahead of
+  // an mbarrier cannot tell "not yet" from "long ago": stages shared between teams would allow that.)
+  static constexpr int kNStage = kTeams;
+  static constexpr int kOffQRaw = kOffRing + kNStage * kStageBytes;
+  static constexpr int kOffScal = kOffQRaw + 2 * CP * 256;
+  static constexpr int kOffBlk = kOffScal + kTeams * kTeamScal;
+  static constexpr int kOffItems = kOffBlk + kProdWarps * 2 * kI8PieceUnits * 4;
   static constexpr int kOffBars = kOffItems + 2 * 32;
-  static constexpr int kOffMisc = kOffBars + 64 * 8;             // [3][64] ints: common, group 0, group 1
-  static constexpr int kSmem = kOffMisc + 3 * 256 + 64 + 1024;   // + alignment slack
+  static constexpr int kOffMisc = kOffBars + 64 * 8;             // [1 + teams][64] ints
+  static constexpr int kSmem = kOffMisc + (1 + kTeams) * 256 + 64 + 1024;   // + alignment slack
   static_assert(kSmem <= 227 * 1024, "shared memory");
-  static_assert(kOffMail % 16 == 0 && kMail % 16 == 0 && kOffBars % 8 == 0, "alignment");
-  // tensor memory columns of a softmax group: two S buffers, O accumulators, FP32 copy of O
-  static constexpr int kTmS = 0, kTmO = 2 * kNQK, kTmOF = 2 * kNQK + kNPV;
-  static constexpr int kTmWg = CP == 4 ? 64 : CP == 8 ? 128 : 256;
-  static constexpr int kTmCols = 2 * kTmWg;
-  static_assert(kTmOF + CP <= kTmWg, "tensor memory");
+  static_assert(kOffScal % 16 == 0 && kTeamScal % 16 == 0 && kOffBars % 8 == 0, "alignment");
+  // tensor memory columns of a team: S, O accumulators, FP32 copy of O
+  static constexpr int kTmS = 0, kTmO = kNQK, kTmOF = kNQK + kNPV;
+  static constexpr int kTmTeam = CP == 4 ? 64 : 128;
+  static constexpr int kTmCols = kTeams * kTmTeam > 256 ? 512 : kTeams * kTmTeam > 128 ? 256 : 128;
+  static_assert(kTmOF + CP <= kTmTeam && kTeams * kTmTeam <= 512, "tensor memory");
   static constexpr int kDrainUnits = FULL ? 256 : 4096;  // own units after which the int32 sums could overflow
 };
 
@@ -270,7 +270,7 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
                                      : arr == 3 ? C::kOffVM : arr == 4 ? C::kOffKR : C::kOffVR) +
                           (uint32_t)sub * my_bytes;
   constexpr uint32_t kBytesSub = (FULL ? 4u : 2u) * 1024u + 2u * 128u;   // bytes of one sub-block
-  uint32_t* my_blk = blk_s + pw * 2 * kPieceUnits;   // [2 sub-blocks][kPieceUnits]
+  uint32_t* my_blk = blk_s + pw * 2 * kI8PieceUnits;   // [2 sub-blocks][kI8PieceUnits]
   int b = b_lo, len = clamp_len(b), U = (len + ST - 1) / ST;
   int hkv = (int)(off_lo / U), u = (int)(off_lo % U);
   int remaining = n_units, gs = 0, ic = 0;
@@ -295,8 +295,8 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
                  p.q + (((size_t)b * p.nq + j) * p.Hq + (size_t)hkv * p.G) * LYNX_D,
                  (uint32_t)(p.G * LYNX_D * 2), qfull0 + qi * 8);
     }
-    for (int c0 = 0; c0 < n; c0 += kPieceUnits) {
-      const int cn = min(kPieceUnits, n - c0);
+    for (int c0 = 0; c0 < n; c0 += kI8PieceUnits) {
+      const int cn = min(kI8PieceUnits, n - c0);
       for (int i2 = lane; i2 < 2 * cn; i2 += 32) {
         const int i = i2 >> 1;
         const int t0 = (u + c0 + i) * ST + (sub_first + (i2 & 1)) * 16;
@@ -309,13 +309,13 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
           }
           row = (uint32_t)(((size_t)blk * p.Hkv + hkv) * p.bt + (t0 % p.bt));
         }
-        my_blk[(i2 & 1) * kPieceUnits + i] = row;
+        my_blk[(i2 & 1) * kI8PieceUnits + i] = row;
       }
       __syncwarp();
       for (int k = 0; k < cn; ++k, ++gs) {
         const int slot = gs % NSTAGE;
         if (gs >= NSTAGE) mbar_wait(empty0 + slot * 8, ((gs / NSTAGE) - 1) & 1, abort_word);
-        const uint32_t row0 = my_blk[k], row1 = my_blk[kPieceUnits + k];
+        const uint32_t row0 = my_blk[k], row1 = my_blk[kI8PieceUnits + k];
         const uint32_t row = sub == sub_first ? row0 : row1;
         const uint32_t bar = full0 + slot * 8;
         if (lane == 0) {
@@ -378,17 +378,28 @@ __device__ __forceinline__ uint64_t i8_desc(uint32_t addr, uint32_t lbo_bytes, u
          ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout << 61);
 }
 
+// Bounded wait until a shared-memory sequence counter has reached `need` (a counter, unlike an mbarrier
+// phase, cannot be misread by a waiter that is ahead of the writer).  Gives up after ~2 s like mbar_wait.
+__device__ __noinline__ bool seq_wait(const volatile int* ctr, int need, volatile int* abort_word) {
+  const uint64_t t0 = globaltimer_ns();
+  for (;;) {
+    for (int i = 0; i < 64; ++i) {
+      if (*ctr >= need) { __threadfence_block(); return true; }
+      __nanosleep(40);
+    }
+    if (*abort_word) return false;
+    if (globaltimer_ns() - t0 > 2000000000ull) { *abort_word = 1; return false; }
+  }
+}
+
 template <bool FULL, int CP>
 __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(const AttnParams p) {
   using C = I8Cfg<FULL, CP>;
-  constexpr int NSTAGE = C::kNStage, KS = C::kKSlots;
+  constexpr int NSTAGE = C::kNStage, T = C::kTeams;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
   unsigned char* qraw = smem + C::kOffQRaw;
-  float* scal = reinterpret_cast<float*>(smem + C::kOffScal);
-  float* red = reinterpret_cast<float*>(smem + C::kOffRed);
-  float* lz = reinterpret_cast<float*>(smem + C::kOffLz);
   uint32_t* blk_s = reinterpret_cast<uint32_t*>(smem + C::kOffBlk);
   Item* items = reinterpret_cast<Item*>(smem + C::kOffItems);
   int* misc = reinterpret_cast<int*>(smem + C::kOffMisc);
@@ -396,29 +407,27 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   const uint32_t ring_u32 = sbase + C::kOffRing;
   const uint32_t full0 = sbase + C::kOffBars, empty0 = full0 + NSTAGE * 8;
   const uint32_t qfull0 = empty0 + NSTAGE * 8, qempty0 = qfull0 + 16;
-  const uint32_t kfree0 = qempty0 + 16;           // [KS]   Q.K^T of the unit in this K tile complete
-  const uint32_t sfull0 = kfree0 + KS * 8;        // [group][S buffer]  Q.K^T complete: scores valid
-  const uint32_t sfree0 = sfull0 + 32;            // [group][S buffer]  the group holds the scores in registers
-  const uint32_t pvdone0 = sfree0 + 32;           // [group][tile]  P.V complete: P and V tiles free, accumulators current
+  const uint32_t qready0 = qempty0 + 16;          // [query slot]  the digit planes of the piece are written
+  const uint32_t sfull0 = qready0 + 16;           // [team]  Q.K^T complete: scores valid, K tile free
+  const uint32_t pvdone0 = sfull0 + T * 8;        // [team]  P.V complete: P and V tiles free, accumulators current
   volatile int* abort_word = misc;
-  // misc[8] = tensor memory base; misc[12..15] = scratch of the K expanders
+  // misc[8] = tensor memory base; misc[16 + t] = deposits written by team t, misc[24 + t] = deposits of team t read
 
   if (tid == 0) {
     for (int i = 0; i < NSTAGE; ++i) {
       mbar_init(full0 + i * 8, C::kProdWarps);
-      mbar_init(empty0 + i * 8, C::kKWarps + 4);   // the K expanders and the softmax group that owns the unit
+      mbar_init(empty0 + i * 8, 4);               // the four warps of the team that owns the unit
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(qfull0 + i * 8, 1);
-      mbar_init(qempty0 + i * 8, C::kSoftWarps + C::kKWarps);
+      mbar_init(qempty0 + i * 8, 4 * T);
+      mbar_init(qready0 + i * 8, 4);
     }
-    for (int i = 0; i < KS; ++i) mbar_init(kfree0 + i * 8, 1);
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < T; ++i) {
       mbar_init(sfull0 + i * 8, 1);
-      mbar_init(sfree0 + i * 8, 4);
       mbar_init(pvdone0 + i * 8, 1);
     }
-    for (int i = 0; i < 3 * 64 + 16; ++i) misc[i] = 0;
+    for (int i = 0; i < (1 + T) * 64 + 16; ++i) misc[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // raw query slots (their padding columns stay zero) and query digit planes (their padding rows too)
@@ -444,137 +453,39 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
-  named_bar(8, (C::kSoftWarps + C::kKWarps) * 32);
+  named_bar(8, 4 * T * 32);
   tc_fence_after();
   const uint32_t tmem0 = *reinterpret_cast<volatile uint32_t*>(misc + 8);
   constexpr uint32_t kIdescS = i8_idesc(C::kNQK, false, true), kIdescO = i8_idesc(C::kNPV, true, false);
 
   // =============================================================================================
-  // K expanders: query digit planes at the start of a piece, K level tile of every unit, and the
-  // Q.K^T of the unit, issued by one of their threads as soon as the tile is complete
+  // Teams.  Team t takes the units gs = t, t + T, ... of the CTA's range and does everything for
+  // them: K tile, Q.K^T, V tile, scores -> weights, P.V.
   // =============================================================================================
-  if (warp >= C::kKWarp0) {
-    const int w4 = warp - C::kKWarp0, kt = tid - C::kKWarp0 * 32;
-    float* amax_s = reinterpret_cast<float*>(misc + 12);
-    int gs_base = 0, ic = 0;
-    while (gs_base < n_units) {
-      const int qi = ic & 1;
-      mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
-      const int n_piece = items[qi].pad0;
-      for (int u = 0; u < n_piece; ++u) {
-        const int gs = gs_base + u, slot = gs % NSTAGE, ks = gs % KS;
-        mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
-        // the K tile was last read by the Q.K^T of unit gs - KS
-        if (gs >= KS) mbar_wait(kfree0 + ks * 8, ((gs / KS) - 1) & 1, abort_word);
-        if (u == 0) {
-          // the query planes of the piece before last were last read by a unit up to gs - 2
-          if (gs >= 2) mbar_wait(kfree0 + ((gs - 2) % KS) * 8, ((gs - 2) / KS) & 1, abort_word);
-          // three balanced s8 digit planes of q_int = rint(q 2^e), rows plane * CP + column
-          const unsigned char* qb = qraw + qi * CP * 256;
-          const float am = i8_q_absmax<CP>(qb, kt);
-          if (lane == 0) amax_s[w4] = am;
-          named_bar(7, C::kKWarps * 32);
-          const float amax = fmaxf(fmaxf(amax_s[0], amax_s[1]), fmaxf(amax_s[2], amax_s[3]));
-          const int e = i8_q_exponent(amax);
-          const float up = __int_as_float((127 + e) << 23);
-          const uint32_t qt = sbase + C::kOffQT + qi * C::kQTile;
-          if (kt < CP * 4) {
-            const int c = kt >> 2, j = kt & 3;
-            uint32_t pl[3][2][4];   // [plane][parity][word]
-#pragma unroll
-            for (int w = 0; w < 4; ++w) {
-              const uint4 v = *reinterpret_cast<const uint4*>(qb + c * 256 + j * 64 + w * 16);
-              const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
-              uint32_t acc[3][2] = {{0, 0}, {0, 0}, {0, 0}};
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-#pragma unroll
-                for (int par = 0; par < 2; ++par) {
-                  const float f = par ? __uint_as_float(ww[i] & 0xFFFF0000u) : __uint_as_float(ww[i] << 16);
-                  int qv = __float2int_rn(f * up);
-                  qv = max(-4194303, min(4194303, qv));
-#pragma unroll
-                  for (int pln = 0; pln < 3; ++pln) {
-                    const int dgt = (int)(signed char)(qv & 0xFF);
-                    acc[pln][par] |= (uint32_t)(dgt & 0xFF) << (8 * i);
-                    qv = (qv - dgt) >> 8;
-                  }
-                }
-              }
-#pragma unroll
-              for (int pln = 0; pln < 3; ++pln) { pl[pln][0][w] = acc[pln][0]; pl[pln][1][w] = acc[pln][1]; }
-            }
-#pragma unroll
-            for (int pln = 0; pln < 3; ++pln) {
-              const int n = pln * CP + c;
-#pragma unroll
-              for (int par = 0; par < 2; ++par) {
-                const uint32_t a = qt + (uint32_t)n * 128u + ((uint32_t)((2 * j + par) ^ (n & 7)) << 4);
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pl[pln][par][0]),
-                             "r"(pl[pln][par][1]), "r"(pl[pln][par][2]), "r"(pl[pln][par][3]) : "memory");
-              }
-            }
-          }
-        }
-        const uint32_t st = ring_u32 + slot * C::kStageBytes;
-        const uint32_t ktile = sbase + C::kOffKT + ks * C::kTile;
-        i8_expand<FULL>(st + C::kOffKA, st + C::kOffKR, ktile, w4, lane);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty0 + slot * 8);
-        named_bar(7, C::kKWarps * 32);   // the tile (and the query planes) are complete; amax_s may be rewritten
-        if (kt == 0) {
-          const int g = gs & 1, n = gs >> 1, b = n & 1;   // softmax group, its unit index, its S buffer
-          if (n >= 2) mbar_wait(sfree0 + (g * 2 + b) * 8, ((n >> 1) - 1) & 1, abort_word);
-          tc_fence_after();
-          const uint32_t qt = sbase + C::kOffQT + qi * C::kQTile;
-          const uint32_t d = tmem0 + g * C::kTmWg + C::kTmS + b * C::kNQK;
-#pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4)
-            i8_mma_ss(d, i8_desc(ktile + (uint32_t)k4 * 32u, 16u, 1024u, 2u), i8_desc(qt + (uint32_t)k4 * 32u, 16u, 1024u, 2u),
-                      kIdescS, k4 > 0 ? 1u : 0u);
-          tc_commit(sfull0 + (g * 2 + b) * 8);
-          tc_commit(kfree0 + ks * 8);
-        }
-        __syncwarp();
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(qempty0 + qi * 8);
-      gs_base += n_piece;
-      ++ic;
-    }
-    return;
-  }
-
-  // =============================================================================================
-  // Softmax groups: V level tile, scores -> weights, P.V (issued by one thread of the group)
-  // =============================================================================================
-  const int wg = warp >> 2, w4 = warp & 3;
+  const int tm = warp >> 2, w4 = warp & 3;
   const int r = tid & 127;                        // token of the unit (S), output dim position (O): TMEM lane
   const uint32_t lane_sel = (uint32_t)(w4 * 32) << 16;
-  const uint32_t tm_s = tmem0 + wg * C::kTmWg + C::kTmS + lane_sel;
-  const uint32_t tm_o = tmem0 + wg * C::kTmWg + C::kTmO + lane_sel;
-  const uint32_t tm_of = tmem0 + wg * C::kTmWg + C::kTmOF + lane_sel;
-  float* my_scal = scal + wg * 8 * CP;            // qs, ref, factor, limits (int)
+  const uint32_t tm_s = tmem0 + tm * C::kTmTeam + C::kTmS + lane_sel;
+  const uint32_t tm_o = tmem0 + tm * C::kTmTeam + C::kTmO + lane_sel;
+  const uint32_t tm_of = tmem0 + tm * C::kTmTeam + C::kTmOF + lane_sel;
+  float* my_scal = reinterpret_cast<float*>(smem + C::kOffScal + tm * C::kTeamScal);
   float* qs_s = my_scal, *ref_s = my_scal + CP, *fac_s = my_scal + 2 * CP;
   int* lim_s = reinterpret_cast<int*>(my_scal + 3 * CP);
-  float* my_red = red + wg * 4 * 2 * CP;
-  float* my_lz = lz + wg * 2 * CP;
-  int* my_misc = misc + 64 * (1 + wg);
-  const int bar_wg = 1 + wg;                      // named barrier of this group
-  const uint32_t vtile0 = sbase + C::kOffVT + wg * C::kVS * C::kTile;
-  const uint32_t ptile0 = sbase + C::kOffPT + wg * C::kVS * C::kPTileA;
-  float* mail_mine = reinterpret_cast<float*>(smem + C::kOffMail + wg * C::kMail);
-  const float* mail_other = reinterpret_cast<const float*>(smem + C::kOffMail + (wg ^ 1) * C::kMail);
+  float* my_red = my_scal + 8 * CP;               // [4 warps][2 CP]
+  float* my_lz = my_scal + 16 * CP;               // [2 CP]
+  int* my_misc = misc + 64 * (1 + tm);
+  const int bar_tm = 1 + tm;                      // named barrier of this team
+  const uint32_t ktile = sbase + tm * C::kTeamBytes, vtile = ktile + C::kTile, ptile = C::kPAliasK ? ktile : vtile + C::kTile;
   const int dim_out = 32 * (r >> 5) + 8 * ((r >> 2) & 3) + 2 * (r & 3) + ((r >> 4) & 1);   // head dim of lane r of O
   // this thread's row of the P tile: 16-byte chunk j goes to position j ^ p_swz
   const uint32_t p_swz = C::kPRow == 32 ? ((uint32_t)r >> 2) & 1u : C::kPRow == 64 ? ((uint32_t)r >> 1) & 3u : (uint32_t)r & 7u;
-  const uint32_t p_row0 = ptile0 + (uint32_t)r * C::kPRow;
+  const uint32_t p_row = ptile + (uint32_t)r * C::kPRow;
   const float cb = p.sm_log2;
-  bool deposit_pending = false;                   // the other group has not yet read this group's last deposit
-  // completion barrier and phase parity of the P.V of this group's unit n (units alternate between the tiles)
-  auto pv_bar = [&](uint32_t n) { return pvdone0 + (uint32_t)(wg * 2 + (C::kVS == 2 ? (int)(n & 1u) : 0)) * 8u; };
-  auto pv_par = [&](uint32_t n) { return C::kVS == 2 ? (n >> 1) & 1u : n & 1u; };
+  uint32_t dep_cnt[T];                            // deposits made so far, per team (every team keeps the same count)
+#pragma unroll
+  for (int i = 0; i < T; ++i) dep_cnt[i] = 0;
+  uint32_t my_deps = 0;                           // this team's own deposits
+  bool ack_pending = false;                       // this team's last deposit (in its V tile) may not have been read yet
 
   int gs_base = 0, ic = 0;
   while (gs_base < n_units) {
@@ -582,10 +493,11 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
     mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
     const Item item = items[qi];
     const int len = item.len, n_piece = item.pad0;
-    const int u_first = ((gs_base & 1) == wg) ? 0 : 1;   // this group's units of the piece: u_first, u_first + 2, ...
+    const int team0 = gs_base % T;                        // team of the piece's first unit
+    const int u_first = (tm - team0 + T) % T;             // this team's units of the piece: u_first, u_first + T, ...
+    const int team_f = (gs_base + n_piece - 1) % T;       // team of the piece's last unit: it writes the piece's result
     if (u_first < n_piece) {
-      const int u_last = u_first + ((n_piece - 1 - u_first) & ~1);
-      const bool finisher = u_last == n_piece - 1;
+      const bool finisher = tm == team_f;
       const int full_lim = p.causal ? len - p.nq + 1 : len;
       // ---- the piece's queries: fixed-point exponent, sum of q per column, causal limits ----------
       const unsigned char* qb = qraw + qi * CP * 256;
@@ -601,21 +513,68 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           if (lane == 0) qs_s[c] = sum;
         }
         if (r < CP) lim_s[r] = r < p.ncols ? (p.causal ? len - p.nq + r / p.G + 1 : len) : 0;
-        named_bar(bar_wg, 128);
+        named_bar(bar_tm, 128);
       }
       const float amax = fmaxf(fmaxf(my_red[0], my_red[1]), fmaxf(my_red[2], my_red[3]));
       const int e = i8_q_exponent(amax);
       const float ca = p.sm_log2 * __int_as_float((127 - e) << 23) * (FULL ? 1.0f : 16.0f);
-      named_bar(bar_wg, 128);   // my_red is reused below
+      named_bar(bar_tm, 128);   // my_red is reused below
+      const uint32_t qt = sbase + C::kOffQT + qi * C::kQTile;
+      if (u_first == 0 && r < CP * 4) {
+        // this team owns the piece's first unit: it writes the three balanced s8 digit planes of
+        // q_int = rint(q 2^e), rows plane * CP + column.  (The slot's previous planes belong to the piece
+        // before last, which every team has left: the queries of this piece were loaded after that.)
+        const float up = __int_as_float((127 + e) << 23);
+        const int c = r >> 2, j = r & 3;
+        uint32_t pl[3][2][4];   // [plane][parity][word]
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const uint4 v = *reinterpret_cast<const uint4*>(qb + c * 256 + j * 64 + w * 16);
+          const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+          uint32_t acc[3][2] = {{0, 0}, {0, 0}, {0, 0}};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+#pragma unroll
+            for (int par = 0; par < 2; ++par) {
+              const float f = par ? __uint_as_float(ww[i] & 0xFFFF0000u) : __uint_as_float(ww[i] << 16);
+              int qv = __float2int_rn(f * up);
+              qv = max(-4194303, min(4194303, qv));
+#pragma unroll
+              for (int pln = 0; pln < 3; ++pln) {
+                const int dgt = (int)(signed char)(qv & 0xFF);
+                acc[pln][par] |= (uint32_t)(dgt & 0xFF) << (8 * i);
+                qv = (qv - dgt) >> 8;
+              }
+            }
+          }
+#pragma unroll
+          for (int pln = 0; pln < 3; ++pln) { pl[pln][0][w] = acc[pln][0]; pl[pln][1][w] = acc[pln][1]; }
+        }
+#pragma unroll
+        for (int pln = 0; pln < 3; ++pln) {
+          const int n = pln * CP + c;
+#pragma unroll
+          for (int par = 0; par < 2; ++par) {
+            const uint32_t a = qt + (uint32_t)n * 128u + ((uint32_t)((2 * j + par) ^ (n & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pl[pln][par][0]),
+                         "r"(pl[pln][par][1]), "r"(pl[pln][par][2]), "r"(pl[pln][par][3]) : "memory");
+          }
+        }
+      }
+      if (u_first == 0) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(qready0 + qi * 8);
+      }
 
       float l[CP], zs[CP];
 #pragma unroll
       for (int c = 0; c < CP; ++c) { l[c] = 0.0f; zs[c] = 0.0f; }
       bool fresh = true, have_of = false;
       int units_in_acc = 0;
-      uint32_t n_own = (uint32_t)((gs_base + u_first) >> 1);   // index of the unit among this group's units
+      uint32_t n_own = (uint32_t)((gs_base + u_first) / T);   // index of the unit among this team's units
 
-      // Ends the current accumulation (the group's last P.V is complete): the int32 accumulators, four
+      // Ends the current accumulation (the team's last P.V is complete): the int32 accumulators, four
       // byte planes per column, are added to the FP32 copy and the sum is scaled by fac_s[] (the change
       // of the reference exponents).
       auto drain = [&](bool scale) {
@@ -653,18 +612,37 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         }
       };
 
-      for (int u = u_first; u < n_piece; u += 2, ++n_own) {
+      for (int u = u_first; u < n_piece; u += T, ++n_own) {
         const int gs = gs_base + u, slot = gs % NSTAGE;
-        const int sb = (int)(n_own & 1u);           // S buffer of this unit
         const int unit_t0 = (item.pad1 + u) * C::kST;
         const int tok = unit_t0 + r;
         const uint32_t st = ring_u32 + slot * C::kStageBytes;
         mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
         float2 km = lds64f(st + C::kOffKM + r * 8), vm = lds64f(st + C::kOffVM + r * 8);
-        // the V and P tiles of this unit are free once the P.V that last read them is complete
-        const uint32_t tb = C::kVS == 2 ? (n_own & 1u) : 0u;
-        const uint32_t vtile = vtile0 + tb * C::kTile, ptile = ptile0 + tb * C::kPTileA;
-        if (n_own >= (uint32_t)C::kVS) mbar_wait(pv_bar(n_own - C::kVS), pv_par(n_own - C::kVS), abort_word);
+        // ---- K tile (free: the team's previous Q.K^T has been waited for), then Q.K^T ---------------
+        if (C::kPAliasK && n_own > 0) mbar_wait(pvdone0 + tm * 8, (n_own - 1) & 1, abort_word);   // P lives there too
+        i8_expand<FULL>(st + C::kOffKA, st + C::kOffKR, ktile, w4, lane);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        tc_fence_before();
+        named_bar(bar_tm, 128);
+        if (r == 0) {
+          mbar_wait(qready0 + qi * 8, (ic >> 1) & 1, abort_word);   // the piece's query planes
+          tc_fence_after();
+          const uint32_t d = tmem0 + tm * C::kTmTeam + C::kTmS;
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            i8_mma_ss(d, i8_desc(ktile + (uint32_t)k4 * 32u, 16u, 1024u, 2u), i8_desc(qt + (uint32_t)k4 * 32u, 16u, 1024u, 2u),
+                      kIdescS, k4 > 0 ? 1u : 0u);
+          tc_commit(sfull0 + tm * 8);
+        }
+        __syncwarp();
+        // ---- V tile: free once the team's previous P.V is complete (and its deposit there was read) ---
+        if (ack_pending) {   // uniform over the team
+          if (r == 0) seq_wait(misc + 24 + tm, (int)my_deps, abort_word);
+          named_bar(bar_tm, 128);
+          ack_pending = false;
+        }
+        if (!C::kPAliasK && n_own > 0) mbar_wait(pvdone0 + tm * 8, (n_own - 1) & 1, abort_word);
         i8_expand<FULL>(st + C::kOffVA, st + C::kOffVR, vtile, w4, lane);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + slot * 8);
@@ -678,18 +656,15 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         const float ib = (FULL ? vm.y : fmaf(vm.x, 8.0f, vm.y)) * ia;
 
         // ---- scores of this thread's token -------------------------------------------------------
-        mbar_wait(sfull0 + (wg * 2 + sb) * 8, (n_own >> 1) & 1, abort_word);
+        mbar_wait(sfull0 + tm * 8, n_own & 1, abort_word);
         tc_fence_after();
         float x[CP];
         {
           uint32_t s0[CP], s1[CP], s2[CP];
-          TmemRegs<CP>::ld(tm_s + sb * C::kNQK, s0);
-          TmemRegs<CP>::ld(tm_s + sb * C::kNQK + CP, s1);
-          TmemRegs<CP>::ld(tm_s + sb * C::kNQK + 2 * CP, s2);
+          TmemRegs<CP>::ld(tm_s, s0);
+          TmemRegs<CP>::ld(tm_s + CP, s1);
+          TmemRegs<CP>::ld(tm_s + 2 * CP, s2);
           tc_wait_ld();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(sfree0 + (wg * 2 + sb) * 8);
 #pragma unroll
           for (int c = 0; c < CP; ++c) {
             const float sf = fmaf((float)((int)s2[c] * 256 + (int)s1[c]), 256.0f, (float)(int)s0[c]);
@@ -705,7 +680,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         bool need = fresh || units_in_acc >= C::kDrainUnits;
 #pragma unroll
         for (int c = 0; c < CP; ++c) need |= x[c] - ref_s[c] > 31.5f;
-        if (bar_or(bar_wg, 128, need)) {
+        if (bar_or(bar_tm, 128, need)) {
 #pragma unroll
           for (int c = 0; c < CP; ++c) {
             float mx = x[c];
@@ -713,7 +688,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
             for (int off = 16; off >= 1; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
             if (lane == 0) my_red[w4 * CP + c] = mx;
           }
-          named_bar(bar_wg, 128);
+          named_bar(bar_tm, 128);
           if (r < CP) {
             const float mx = fmaxf(fmaxf(my_red[r], my_red[CP + r]), fmaxf(my_red[2 * CP + r], my_red[3 * CP + r]));
             const float old = ref_s[r];
@@ -723,11 +698,10 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
             ref_s[r] = nw;
             fac_s[r] = f;
           }
-          named_bar(bar_wg, 128);
+          named_bar(bar_tm, 128);
 #pragma unroll
           for (int c = 0; c < CP; ++c) { l[c] *= fac_s[c]; zs[c] *= fac_s[c]; }
-          if (C::kVS > 1 && units_in_acc > 0) mbar_wait(pv_bar(n_own - 1), pv_par(n_own - 1), abort_word);
-          drain(true);
+          drain(true);   // (the team's previous P.V was waited for before the V tile was rewritten)
           fresh = false;
         }
         // ---- weights ------------------------------------------------------------------------------
@@ -742,27 +716,27 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
 #pragma unroll
         for (int j = 0; j < CP / 4; ++j)
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(p_row0 + tb * C::kPTileA + (((uint32_t)j ^ p_swz) << 4)), "r"(wi[4 * j]), "r"(wi[4 * j + 1]),
+                       ::"r"(p_row + (((uint32_t)j ^ p_swz) << 4)), "r"(wi[4 * j]), "r"(wi[4 * j + 1]),
                          "r"(wi[4 * j + 2]), "r"(wi[4 * j + 3]) : "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         tc_fence_before();
-        named_bar(bar_wg, 128);     // the P tile and the V tile are complete
+        named_bar(bar_tm, 128);     // the P tile and the V tile are complete, S has been read
         if (r == 0) {
           tc_fence_after();
-          const uint32_t d = tmem0 + wg * C::kTmWg + C::kTmO;
+          const uint32_t d = tmem0 + tm * C::kTmTeam + C::kTmO;
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
             i8_mma_ss(d, i8_desc(vtile + (uint32_t)k4 * 4096u, 16384u, 1024u, 2u),
                       i8_desc(ptile + (uint32_t)k4 * (32u * C::kPRow), 16384u, 8u * C::kPRow, (uint32_t)C::kPLayout),
                       kIdescO, (units_in_acc > 0 || k4 > 0) ? 1u : 0u);
-          tc_commit(pv_bar(n_own));
+          tc_commit(pvdone0 + tm * 8);
         }
         __syncwarp();
         ++units_in_acc;
       }
-      // ---- end of the piece for this group -----------------------------------------------------------
-      mbar_wait(pv_bar(n_own - 1), pv_par(n_own - 1), abort_word);   // the last P.V
-      drain(false);   // the FP32 copy now holds this group's part of O
+      // ---- end of the piece for this team -----------------------------------------------------------
+      mbar_wait(pvdone0 + tm * 8, (n_own - 1) & 1, abort_word);   // the last P.V
+      drain(false);   // the FP32 copy now holds this team's part of O
       float of[CP];
 #pragma unroll
       for (int c4 = 0; c4 < CP / 4; ++c4) {
@@ -773,7 +747,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         for (int k = 0; k < 4; ++k) of[c4 * 4 + k] = __uint_as_float(t[k]);
       }
       tc_fence_before();
-      // totals of l and zs over the group's 128 token lanes
+      // totals of l and zs over the team's 128 token lanes
 #pragma unroll
       for (int c = 0; c < CP; ++c) {
         float a = l[c], b = zs[c];
@@ -784,32 +758,39 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         }
         if (lane == 0) { my_red[w4 * 2 * CP + c] = a; my_red[w4 * 2 * CP + CP + c] = b; }
       }
-      named_bar(bar_wg, 128);
+      named_bar(bar_tm, 128);
       if (r < 2 * CP) my_lz[r] = (my_red[r] + my_red[2 * CP + r]) + (my_red[4 * CP + r] + my_red[6 * CP + r]);
-      named_bar(bar_wg, 128);
+      named_bar(bar_tm, 128);
       if (!finisher) {
-        // deposit (O, l, zs, ref) for the group that owns the piece's last unit
-        if (deposit_pending) named_bar(5 + wg, 256);   // the previous deposit has been read
+        // deposit (O, l, zs, ref) in this team's V tile (idle: its last P.V is complete) for the team that
+        // owns the piece's last unit
+        float* mail = reinterpret_cast<float*>(smem + tm * C::kTeamBytes + C::kTile);
 #pragma unroll
-        for (int c = 0; c < CP; ++c) mail_mine[c * 128 + r] = of[c];
+        for (int c = 0; c < CP; ++c) mail[c * 128 + r] = of[c];
         if (r < CP) {
-          mail_mine[CP * 128 + r] = my_lz[r];
-          mail_mine[CP * 128 + CP + r] = my_lz[CP + r];
-          mail_mine[CP * 128 + 2 * CP + r] = ref_s[r];
+          mail[CP * 128 + r] = my_lz[r];
+          mail[CP * 128 + CP + r] = my_lz[CP + r];
+          mail[CP * 128 + 2 * CP + r] = ref_s[r];
         }
         __threadfence_block();
-        bar_arrive(3 + wg, 256);
-        deposit_pending = true;
+        named_bar(bar_tm, 128);
+        ++my_deps;
+        if (r == 0) *reinterpret_cast<volatile int*>(misc + 16 + tm) = (int)my_deps;
+        ack_pending = true;
       } else {
         float lt[CP], zt[CP], mt[CP];
 #pragma unroll
         for (int c = 0; c < CP; ++c) { lt[c] = my_lz[c]; zt[c] = my_lz[CP + c]; mt[c] = ref_s[c]; }
-        if (n_piece >= 2) {
-          named_bar(3 + (wg ^ 1), 256);   // the other group's deposit is complete
+#pragma unroll
+        for (int d = 0; d < T; ++d) {
+          if (d == tm || (d - team0 + T) % T >= n_piece) continue;   // itself; a team without a unit in the piece
+          if (r == 0) seq_wait(misc + 16 + d, (int)dep_cnt[d] + 1, abort_word);   // its deposit is complete
+          named_bar(bar_tm, 128);
+          const float* mo = reinterpret_cast<const float*>(smem + d * C::kTeamBytes + C::kTile);
 #pragma unroll
           for (int c = 0; c < CP; ++c) {
-            const float o2 = mail_other[c * 128 + r], l2 = mail_other[CP * 128 + c];
-            const float z2 = mail_other[CP * 128 + CP + c], m2 = mail_other[CP * 128 + 2 * CP + c];
+            const float o2 = mo[c * 128 + r], l2 = mo[CP * 128 + c];
+            const float z2 = mo[CP * 128 + CP + c], m2 = mo[CP * 128 + 2 * CP + c];
             const float M = fmaxf(mt[c], m2);
             const float f1 = ex2_full(mt[c] - M), f2 = ex2_full(m2 - M);
             of[c] = of[c] * f1 + o2 * f2;
@@ -817,7 +798,9 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
             zt[c] = zt[c] * f1 + z2 * f2;
             mt[c] = M;
           }
-          bar_arrive(5 + (wg ^ 1), 256);   // it may deposit again
+          __threadfence_block();
+          named_bar(bar_tm, 128);
+          if (r == 0) *reinterpret_cast<volatile int*>(misc + 24 + d) = (int)dep_cnt[d] + 1;   // its V tile may be written again
         }
         const bool direct = item.n_contrib == 1;
         const size_t bh = (size_t)item.b * p.Hkv + item.hkv;
@@ -836,9 +819,13 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           }
         }
         __threadfence();
-        finish_piece<FULL, C::kPartCols, 128>(p, item, direct, r, my_misc, bar_wg);
+        finish_piece<FULL, C::kPartCols, 128>(p, item, direct, r, my_misc, bar_tm);
       }
     }
+    // every team keeps count of every team's deposits (the phase of its deposit barrier)
+#pragma unroll
+    for (int d = 0; d < T; ++d)
+      if (d != team_f && (d - team0 + T) % T < n_piece) ++dep_cnt[d];
     __syncwarp();
     if (lane == 0) mbar_arrive(qempty0 + qi * 8);
     gs_base += n_piece;
@@ -846,7 +833,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   }
   // ---- release the tensor memory ---------------------------------------------------------------
   tc_fence_before();
-  named_bar(9, C::kSoftWarps * 32);
+  named_bar(9, 4 * T * 32);
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem0), "r"((uint32_t)C::kTmCols)
