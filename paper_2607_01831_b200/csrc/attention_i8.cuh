@@ -58,14 +58,11 @@ struct I8Cfg {
   static constexpr int kProdWarp0 = 4 * kTeams;
   static constexpr int kThreads = (kProdWarp0 + kProdWarps) * 32;
   // shared memory map (offsets from a 1024-byte aligned base)
-  static constexpr int kTile = 16384;                    // K and V level tiles: [128 rows][128 B]
+  static constexpr int kTile = 16384;                    // V level tile: [128 tokens][128 B]
   static constexpr int kPRow = 4 * CP < 32 ? 32 : 4 * CP;   // bytes of a P tile row (one token)
   static constexpr int kPTile = 128 * kPRow;
   static constexpr int kPLayout = kPRow == 32 ? 6 : kPRow == 64 ? 4 : 2;   // descriptor swizzle mode of the P tile
-  // Where shared memory is short the P tile shares the K tile's memory (K is dead once Q.K^T is complete,
-  // P is written after that); the next K expansion then has to wait for the P.V.
-  static constexpr bool kPAliasK = FULL ? CP >= 8 : CP == 8;
-  static constexpr int kTeamBytes = 2 * kTile + (kPAliasK ? 0 : kPTile);  // K tile, V tile, P tile
+  static constexpr int kTeamBytes = kTile + kPTile;      // V tile, P tile (the K levels live in tensor memory)
   static constexpr int kQTile = (kNQK * 128 + 1023) / 1024 * 1024;
   static constexpr int kMail = (CP * 128 + 3 * CP) * 4;  // end-of-piece deposit of a team (in its V tile): O, l, zs, ref
   static_assert(kMail <= kTile, "the deposit lives in the team's V tile");
@@ -74,10 +71,9 @@ struct I8Cfg {
   static constexpr int kTeamScal = (8 * CP + 4 * 2 * CP + 2 * CP) * 4;   // qs, ref, factor, limits; reduce scratch; totals
   static constexpr int kFixedTail = 2 * CP * 256 + kTeams * kTeamScal +
                                     kProdWarps * 2 * kI8PieceUnits * 4 + 2 * 32 + 64 * 8 + (1 + kTeams) * 256 + 64;
-  // One raw stage per team: unit gs lands in stage gs % kTeams, the stage of the team that owns it, so
-  // every team sees the phases of its stage's barriers in order.  (A waiter that is a phase ahead of
-  // an mbarrier cannot tell "not yet" from "long ago": stages shared between teams would allow that.)
-  static constexpr int kNStage = kTeams;
+  static constexpr int kAvail = 227 * 1024 - 1024 - kOffRing - kFixedTail;
+  static constexpr int kNStage = kAvail / kStageBytes > 8 ? 8 : kAvail / kStageBytes;
+  static_assert(kNStage >= 2, "ring too small");
   static constexpr int kOffQRaw = kOffRing + kNStage * kStageBytes;
   static constexpr int kOffScal = kOffQRaw + 2 * CP * 256;
   static constexpr int kOffBlk = kOffScal + kTeams * kTeamScal;
@@ -87,11 +83,11 @@ struct I8Cfg {
   static constexpr int kSmem = kOffMisc + (1 + kTeams) * 256 + 64 + 1024;   // + alignment slack
   static_assert(kSmem <= 227 * 1024, "shared memory");
   static_assert(kOffScal % 16 == 0 && kTeamScal % 16 == 0 && kOffBars % 8 == 0, "alignment");
-  // tensor memory columns of a team: S, O accumulators, FP32 copy of O
-  static constexpr int kTmS = 0, kTmO = kNQK, kTmOF = kNQK + kNPV;
-  static constexpr int kTmTeam = CP == 4 ? 64 : 128;
-  static constexpr int kTmCols = kTeams * kTmTeam > 256 ? 512 : kTeams * kTmTeam > 128 ? 256 : 128;
-  static_assert(kTmOF + CP <= kTmTeam && kTeams * kTmTeam <= 512, "tensor memory");
+  // tensor memory columns of a team: S, O accumulators, FP32 copy of O, K levels (128 bytes per token)
+  static constexpr int kTmS = 0, kTmO = kNQK, kTmOF = kNQK + kNPV, kTmK = (kTmOF + CP + 7) / 8 * 8;
+  static constexpr int kTmTeam = CP == 16 ? 160 : 128;
+  static constexpr int kTmCols = 512;
+  static_assert(kTmK + 32 <= kTmTeam && kTeams * kTmTeam <= 512, "tensor memory");
   static constexpr int kDrainUnits = FULL ? 256 : 4096;  // own units after which the int32 sums could overflow
 };
 
@@ -118,6 +114,13 @@ __device__ __forceinline__ void i8_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void i8_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
 }
 // barrier among `n` threads that also ORs a predicate over them
 __device__ __forceinline__ bool bar_or(int id, int n, bool pred) {
@@ -181,6 +184,53 @@ __device__ __forceinline__ void i8_expand(uint32_t raw_a, uint32_t raw_r, uint32
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + c1), "r"(od[0]), "r"(od[1]), "r"(od[2]),
                  "r"(od[3]) : "memory");
   }
+}
+
+// K levels of a 128-token raw stage into tensor memory: thread r owns token r (TMEM lane r) and writes
+// its 128 level bytes to 32 columns, byte 4 col + b in the order of the operand tiles (see the header).
+// The four 16-byte chunks of the row are read in a lane-dependent order (chunk i ^ s, s = (r >> 1) & 3:
+// rows are 64 bytes apart, so a fixed order would put a quarter-warp on two bank groups) and put back
+// in order with two levels of selects.
+template <bool FULL>
+__device__ __forceinline__ void i8_expand_k_tmem(uint32_t raw_a, uint32_t raw_r, int r, uint32_t tm_k) {
+  const uint32_t s = ((uint32_t)r >> 1) & 3u;
+  uint4 xa[4], xr[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t off = (uint32_t)r * 64u + (((uint32_t)i ^ s) << 4);
+    xa[i] = lds128(raw_a + off);
+    if (FULL) xr[i] = lds128(raw_r + off);
+  }
+  auto sel4 = [](bool c, const uint4& a, const uint4& b) {
+    return make_uint4(c ? a.x : b.x, c ? a.y : b.y, c ? a.z : b.z, c ? a.w : b.w);
+  };
+  uint4 ya[4], yr[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    ya[i] = sel4(s & 1u, xa[i ^ 1], xa[i]);
+    if (FULL) yr[i] = sel4(s & 1u, xr[i ^ 1], xr[i]);
+  }
+  uint32_t regs[32];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint4 a4 = sel4(s & 2u, ya[j ^ 2], ya[j]);
+    const uint32_t a[4] = {a4.x, a4.y, a4.z, a4.w};
+    uint32_t rr[4] = {0, 0, 0, 0};
+    if (FULL) {
+      const uint4 r4 = sel4(s & 2u, yr[j ^ 2], yr[j]);
+      rr[0] = r4.x; rr[1] = r4.y; rr[2] = r4.z; rr[3] = r4.w;
+    }
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      if (FULL) {
+        merge_codes(a[w], rr[w], regs[8 * j + w], regs[8 * j + 4 + w]);
+      } else {
+        regs[8 * j + w] = a[w] & 0x0F0F0F0Fu;
+        regs[8 * j + 4 + w] = (a[w] >> 4) & 0x0F0F0F0Fu;
+      }
+    }
+  }
+  TmemRegs<32>::st(tm_k, regs);
 }
 
 // One of the producer warps: the stream-K bookkeeping (every warp derives the same range and
@@ -411,7 +461,8 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   const uint32_t sfull0 = qready0 + 16;           // [team]  Q.K^T complete: scores valid, K tile free
   const uint32_t pvdone0 = sfull0 + T * 8;        // [team]  P.V complete: P and V tiles free, accumulators current
   volatile int* abort_word = misc;
-  // misc[8] = tensor memory base; misc[16 + t] = deposits written by team t, misc[24 + t] = deposits of team t read
+  // misc[8] = tensor memory base; misc[16 + t] = deposits written by team t, misc[24 + t] = deposits of team t read;
+  // misc[32 + s] = completed phases of raw stage s
 
   if (tid == 0) {
     for (int i = 0; i < NSTAGE; ++i) {
@@ -475,7 +526,8 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   float* my_lz = my_scal + 16 * CP;               // [2 CP]
   int* my_misc = misc + 64 * (1 + tm);
   const int bar_tm = 1 + tm;                      // named barrier of this team
-  const uint32_t ktile = sbase + tm * C::kTeamBytes, vtile = ktile + C::kTile, ptile = C::kPAliasK ? ktile : vtile + C::kTile;
+  const uint32_t vtile = sbase + tm * C::kTeamBytes, ptile = vtile + C::kTile;
+  const uint32_t tm_k = tmem0 + tm * C::kTmTeam + C::kTmK;
   const int dim_out = 32 * (r >> 5) + 8 * ((r >> 2) & 3) + 2 * (r & 3) + ((r >> 4) & 1);   // head dim of lane r of O
   // this thread's row of the P tile: 16-byte chunk j goes to position j ^ p_swz
   const uint32_t p_swz = C::kPRow == 32 ? ((uint32_t)r >> 2) & 1u : C::kPRow == 64 ? ((uint32_t)r >> 1) & 3u : (uint32_t)r & 7u;
@@ -617,12 +669,16 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         const int unit_t0 = (item.pad1 + u) * C::kST;
         const int tok = unit_t0 + r;
         const uint32_t st = ring_u32 + slot * C::kStageBytes;
+        // stages are shared between the teams: the wait for this stage's phase gs / NSTAGE is only well
+        // defined once the phase before it is known to be complete (its owner says so in misc[32 + slot])
+        if (gs >= NSTAGE && *reinterpret_cast<volatile int*>(misc + 32 + slot) < gs / NSTAGE)
+          seq_wait(misc + 32 + slot, gs / NSTAGE, abort_word);
         mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
+        if (r == 0) *reinterpret_cast<volatile int*>(misc + 32 + slot) = gs / NSTAGE + 1;
         float2 km = lds64f(st + C::kOffKM + r * 8), vm = lds64f(st + C::kOffVM + r * 8);
         // ---- K tile (free: the team's previous Q.K^T has been waited for), then Q.K^T ---------------
-        if (C::kPAliasK && n_own > 0) mbar_wait(pvdone0 + tm * 8, (n_own - 1) & 1, abort_word);   // P lives there too
-        i8_expand<FULL>(st + C::kOffKA, st + C::kOffKR, ktile, w4, lane);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        i8_expand_k_tmem<FULL>(st + C::kOffKA, st + C::kOffKR, r, tm_k + lane_sel);
+        tc_wait_st();
         tc_fence_before();
         named_bar(bar_tm, 128);
         if (r == 0) {
@@ -631,8 +687,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           const uint32_t d = tmem0 + tm * C::kTmTeam + C::kTmS;
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
-            i8_mma_ss(d, i8_desc(ktile + (uint32_t)k4 * 32u, 16u, 1024u, 2u), i8_desc(qt + (uint32_t)k4 * 32u, 16u, 1024u, 2u),
-                      kIdescS, k4 > 0 ? 1u : 0u);
+            i8_mma_ts(d, tm_k + (uint32_t)k4 * 8u, i8_desc(qt + (uint32_t)k4 * 32u, 16u, 1024u, 2u), kIdescS, k4 > 0 ? 1u : 0u);
           tc_commit(sfull0 + tm * 8);
         }
         __syncwarp();
@@ -642,7 +697,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           named_bar(bar_tm, 128);
           ack_pending = false;
         }
-        if (!C::kPAliasK && n_own > 0) mbar_wait(pvdone0 + tm * 8, (n_own - 1) & 1, abort_word);
+        if (n_own > 0) mbar_wait(pvdone0 + tm * 8, (n_own - 1) & 1, abort_word);
         i8_expand<FULL>(st + C::kOffVA, st + C::kOffVR, vtile, w4, lane);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + slot * 8);
@@ -764,7 +819,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
       if (!finisher) {
         // deposit (O, l, zs, ref) in this team's V tile (idle: its last P.V is complete) for the team that
         // owns the piece's last unit
-        float* mail = reinterpret_cast<float*>(smem + tm * C::kTeamBytes + C::kTile);
+        float* mail = reinterpret_cast<float*>(smem + tm * C::kTeamBytes);
 #pragma unroll
         for (int c = 0; c < CP; ++c) mail[c * 128 + r] = of[c];
         if (r < CP) {
@@ -786,7 +841,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           if (d == tm || (d - team0 + T) % T >= n_piece) continue;   // itself; a team without a unit in the piece
           if (r == 0) seq_wait(misc + 16 + d, (int)dep_cnt[d] + 1, abort_word);   // its deposit is complete
           named_bar(bar_tm, 128);
-          const float* mo = reinterpret_cast<const float*>(smem + d * C::kTeamBytes + C::kTile);
+          const float* mo = reinterpret_cast<const float*>(smem + d * C::kTeamBytes);
 #pragma unroll
           for (int c = 0; c < CP; ++c) {
             const float o2 = mo[c * 128 + r], l2 = mo[CP * 128 + c];
