@@ -44,10 +44,10 @@ template <bool FULL, int CP>
 struct I8Cfg {
   static_assert(CP == 4 || CP == 8 || CP == 16, "padded column counts");
   static constexpr int kST = 128;                   // tokens per stage-unit
-  static constexpr int kNArr = FULL ? 6 : 4;        // arrays copied per 16-token sub-block
-  static constexpr int kStageBytes = kST * (FULL ? 272 : 144);
+  static constexpr int kNArr = FULL ? 4 : 2;        // plane arrays copied per 16-token sub-block (the metadata is
+                                                    // read with plain loads: the copy engine takes ~35 cycles per copy)
+  static constexpr int kStageBytes = kST * (FULL ? 256 : 128);
   static constexpr int kOffKA = 0, kOffVA = kST * 64, kOffKR = kST * 128, kOffVR = kST * 192;
-  static constexpr int kOffKM = FULL ? kST * 256 : kST * 128, kOffVM = kOffKM + kST * 8;
   static constexpr int kNQK = (3 * CP + 15) / 16 * 16;   // N of the Q.K^T product
   static constexpr int kNPV = 4 * CP;                    // N of the P.V product
   static constexpr int kPartCols = CP < 8 ? 8 : CP;      // column stride of the partial slots
@@ -307,19 +307,15 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
   const int n_units = (int)(lo < hi ? hi - lo : 0);
   if (n_units == 0) return;
 
-  constexpr int RP = 2 * NARR;                 // roles of this warp: (sub-block, array) of two sub-blocks
+  constexpr int SPW = 8 / C::kProdWarps;       // 16-token sub-blocks per warp: 2 or 1
+  constexpr int RP = SPW * NARR;               // roles of this warp: (sub-block, array)
   const int role = pw * RP + (lane < RP ? lane : 0);
-  const int sub = role / NARR, arr = role % NARR, sub_first = 2 * pw;
-  const bool is_meta = arr == 2 || arr == 3;
-  const unsigned char* my_src = arr == 0 ? p.ka : arr == 1 ? p.va
-                              : arr == 2 ? reinterpret_cast<const unsigned char*>(p.km)
-                              : arr == 3 ? reinterpret_cast<const unsigned char*>(p.vm)
-                              : arr == 4 ? p.kr : p.vr;
-  const uint32_t my_bytes = is_meta ? 128u : 1024u, my_mul = is_meta ? 8u : 64u;
-  const uint32_t my_dst = (uint32_t)(arr == 0 ? C::kOffKA : arr == 1 ? C::kOffVA : arr == 2 ? C::kOffKM
-                                     : arr == 3 ? C::kOffVM : arr == 4 ? C::kOffKR : C::kOffVR) +
+  const int sub = role / NARR, arr = role % NARR, sub_first = SPW * pw;
+  const unsigned char* my_src = arr == 0 ? p.ka : arr == 1 ? p.va : arr == 2 ? p.kr : p.vr;
+  const uint32_t my_bytes = 1024u, my_mul = 64u;
+  const uint32_t my_dst = (uint32_t)(arr == 0 ? C::kOffKA : arr == 1 ? C::kOffVA : arr == 2 ? C::kOffKR : C::kOffVR) +
                           (uint32_t)sub * my_bytes;
-  constexpr uint32_t kBytesSub = (FULL ? 4u : 2u) * 1024u + 2u * 128u;   // bytes of one sub-block
+  constexpr uint32_t kBytesSub = (FULL ? 4u : 2u) * 1024u;   // bytes of one sub-block
   uint32_t* my_blk = blk_s + pw * 2 * kI8PieceUnits;   // [2 sub-blocks][kI8PieceUnits]
   int b = b_lo, len = clamp_len(b), U = (len + ST - 1) / ST;
   int hkv = (int)(off_lo / U), u = (int)(off_lo % U);
@@ -347,9 +343,9 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
     }
     for (int c0 = 0; c0 < n; c0 += kI8PieceUnits) {
       const int cn = min(kI8PieceUnits, n - c0);
-      for (int i2 = lane; i2 < 2 * cn; i2 += 32) {
-        const int i = i2 >> 1;
-        const int t0 = (u + c0 + i) * ST + (sub_first + (i2 & 1)) * 16;
+      for (int i2 = lane; i2 < SPW * cn; i2 += 32) {
+        const int i = i2 / SPW;
+        const int t0 = (u + c0 + i) * ST + (sub_first + (i2 % SPW)) * 16;
         uint32_t row = 0xFFFFFFFFu;  // sub-block beyond the end of the sequence: nothing to copy
         if (t0 < len) {
           int blk = __ldg(p.block_table + (size_t)b * p.max_blocks + t0 / p.bt);
@@ -359,13 +355,13 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
           }
           row = (uint32_t)(((size_t)blk * p.Hkv + hkv) * p.bt + (t0 % p.bt));
         }
-        my_blk[(i2 & 1) * kI8PieceUnits + i] = row;
+        my_blk[(i2 % SPW) * kI8PieceUnits + i] = row;
       }
       __syncwarp();
       for (int k = 0; k < cn; ++k, ++gs) {
         const int slot = gs % NSTAGE;
         if (gs >= NSTAGE) mbar_wait(empty0 + slot * 8, ((gs / NSTAGE) - 1) & 1, abort_word);
-        const uint32_t row0 = my_blk[k], row1 = my_blk[kI8PieceUnits + k];
+        const uint32_t row0 = my_blk[k], row1 = SPW == 2 ? my_blk[kI8PieceUnits + k] : 0xFFFFFFFFu;
         const uint32_t row = sub == sub_first ? row0 : row1;
         const uint32_t bar = full0 + slot * 8;
         if (lane == 0) {
@@ -664,6 +660,34 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         }
       };
 
+      // Metadata of this thread's token, read with plain loads two steps ahead: the block id of the unit
+      // after next (a block-table look-up whose result is first touched one step later, so that nothing
+      // waits for it), the (scale, zero) pairs of the next unit.
+      const int bt_shift = (p.bt & (p.bt - 1)) == 0 ? 31 - __clz(p.bt) : -1;   // block size a power of two?
+      auto blk_of = [&](int uu) -> int {      // the raw table entry (0 where there is no such token)
+        const int t = (item.pad1 + uu) * C::kST + r;
+        if (uu >= n_piece || t >= len) return 0;
+        const int bi = bt_shift >= 0 ? t >> bt_shift : t / p.bt;
+        return __ldg(p.block_table + (size_t)item.b * p.max_blocks + bi);
+      };
+      auto row_of = [&](int uu, int blk) -> uint32_t {
+        const int t = (item.pad1 + uu) * C::kST + r;
+        if (uu >= n_piece || t >= len) return 0xFFFFFFFFu;
+        const int in_blk = bt_shift >= 0 ? t & (p.bt - 1) : t % p.bt;
+        blk = min(max(blk, 0), p.num_blocks - 1);     // (out-of-range ids are reported by the producer)
+        return (uint32_t)(((size_t)blk * p.Hkv + item.hkv) * p.bt + in_blk);
+      };
+      auto meta_of = [&](uint32_t row, float2& k2, float2& v2) {
+        k2 = make_float2(0.f, 0.f); v2 = k2;
+        if (row != 0xFFFFFFFFu) {
+          k2 = __ldg(reinterpret_cast<const float2*>(p.km) + row);
+          v2 = __ldg(reinterpret_cast<const float2*>(p.vm) + row);
+        }
+      };
+      int blk_n1 = blk_of(u_first + T), blk_n2 = blk_of(u_first + 2 * T);
+      float2 km_c, vm_c;
+      meta_of(row_of(u_first, blk_of(u_first)), km_c, vm_c);
+
       for (int u = u_first; u < n_piece; u += T, ++n_own) {
         const int gs = gs_base + u, slot = gs % NSTAGE;
         const int unit_t0 = (item.pad1 + u) * C::kST;
@@ -675,7 +699,10 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           seq_wait(misc + 32 + slot, gs / NSTAGE, abort_word);
         mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
         if (r == 0) *reinterpret_cast<volatile int*>(misc + 32 + slot) = gs / NSTAGE + 1;
-        float2 km = lds64f(st + C::kOffKM + r * 8), vm = lds64f(st + C::kOffVM + r * 8);
+        float2 km = km_c, vm = vm_c;
+        meta_of(row_of(u + T, blk_n1), km_c, vm_c);   // for this team's next unit
+        blk_n1 = blk_n2;
+        blk_n2 = blk_of(u + 3 * T);                   // and the block id of the one after the one after
         // ---- K tile (free: the team's previous Q.K^T has been waited for), then Q.K^T ---------------
         i8_expand_k_tmem<FULL>(st + C::kOffKA, st + C::kOffKR, r, tm_k + lane_sel);
         tc_wait_st();
