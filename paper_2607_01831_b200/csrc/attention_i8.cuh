@@ -53,7 +53,7 @@ struct I8Cfg {
   static constexpr int kPartCols = CP < 8 ? 8 : CP;      // column stride of the partial slots
   static constexpr int kColsPad = CP;
   // warps: kTeams teams of four (team t = warps 4t .. 4t+3), then the producers
-  static constexpr int kTeams = (FULL || CP == 16) ? 3 : 4;
+  static constexpr int kTeams = (FULL || CP == 16) ? 3 : CP == 4 ? 5 : 4;
   static constexpr int kProdWarps = 4;
   static constexpr int kProdWarp0 = 4 * kTeams;
   static constexpr int kThreads = (kProdWarp0 + kProdWarps) * 32;
@@ -85,7 +85,7 @@ struct I8Cfg {
   static_assert(kOffScal % 16 == 0 && kTeamScal % 16 == 0 && kOffBars % 8 == 0, "alignment");
   // tensor memory columns of a team: S, O accumulators, FP32 copy of O, K levels (128 bytes per token)
   static constexpr int kTmS = 0, kTmO = kNQK, kTmOF = kNQK + kNPV, kTmK = (kTmOF + CP + 7) / 8 * 8;
-  static constexpr int kTmTeam = CP == 16 ? 160 : 128;
+  static constexpr int kTmTeam = CP == 16 ? 160 : CP == 4 ? 96 : 128;
   static constexpr int kTmCols = 512;
   static_assert(kTmK + 32 <= kTmTeam && kTeams * kTmTeam <= 512, "tensor memory");
   static constexpr int kDrainUnits = FULL ? 256 : 4096;  // own units after which the int32 sums could overflow
@@ -418,6 +418,20 @@ __device__ __forceinline__ int i8_q_exponent(float amax) {
   return max(-100, min(100, e));
 }
 
+// The two halves of a shared-memory matrix descriptor (the MMA-issuing thread keeps the low words of
+// its operands in registers and adds the K-step offset: building descriptors is a chain of dependent
+// instructions in the one thread everybody waits for).
+__host__ __device__ constexpr uint32_t i8_desc_hi(uint32_t sbo_bytes, uint32_t layout) {
+  return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (layout << 29);
+}
+__device__ __forceinline__ uint32_t i8_desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+  return ((addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+__device__ __forceinline__ uint64_t i8_pack(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
 // Shared-memory matrix descriptor with the swizzle mode given (2 = 128 B, 4 = 64 B, 6 = 32 B).
 __device__ __forceinline__ uint64_t i8_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
   return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
@@ -529,6 +543,10 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   const uint32_t p_swz = C::kPRow == 32 ? ((uint32_t)r >> 2) & 1u : C::kPRow == 64 ? ((uint32_t)r >> 1) & 3u : (uint32_t)r & 7u;
   const uint32_t p_row = ptile + (uint32_t)r * C::kPRow;
   const float cb = p.sm_log2;
+  // descriptor low words of the MMA operands (used by the team's issuing thread)
+  const uint32_t qd_lo0 = i8_desc_lo(sbase + C::kOffQT, 16u), vd_lo = i8_desc_lo(vtile, 16384u), pd_lo = i8_desc_lo(ptile, 16384u);
+  constexpr uint32_t kQdHi = i8_desc_hi(1024u, 2u), kVdHi = i8_desc_hi(1024u, 2u),
+                     kPdHi = i8_desc_hi(8u * C::kPRow, (uint32_t)C::kPLayout);
   uint32_t dep_cnt[T];                            // deposits made so far, per team (every team keeps the same count)
 #pragma unroll
   for (int i = 0; i < T; ++i) dep_cnt[i] = 0;
@@ -712,9 +730,10 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           mbar_wait(qready0 + qi * 8, (ic >> 1) & 1, abort_word);   // the piece's query planes
           tc_fence_after();
           const uint32_t d = tmem0 + tm * C::kTmTeam + C::kTmS;
+          const uint32_t qd_lo = qd_lo0 + (uint32_t)qi * (C::kQTile >> 4);
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
-            i8_mma_ts(d, tm_k + (uint32_t)k4 * 8u, i8_desc(qt + (uint32_t)k4 * 32u, 16u, 1024u, 2u), kIdescS, k4 > 0 ? 1u : 0u);
+            i8_mma_ts(d, tm_k + (uint32_t)k4 * 8u, i8_pack(qd_lo + (uint32_t)k4 * 2u, kQdHi), kIdescS, k4 > 0 ? 1u : 0u);
           tc_commit(sfull0 + tm * 8);
         }
         __syncwarp();
@@ -808,8 +827,8 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           const uint32_t d = tmem0 + tm * C::kTmTeam + C::kTmO;
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
-            i8_mma_ss(d, i8_desc(vtile + (uint32_t)k4 * 4096u, 16384u, 1024u, 2u),
-                      i8_desc(ptile + (uint32_t)k4 * (32u * C::kPRow), 16384u, 8u * C::kPRow, (uint32_t)C::kPLayout),
+            i8_mma_ss(d, i8_pack(vd_lo + (uint32_t)k4 * (4096u >> 4), kVdHi),
+                      i8_pack(pd_lo + (uint32_t)k4 * ((32u * C::kPRow) >> 4), kPdHi),
                       kIdescO, (units_in_acc > 0 || k4 > 0) ? 1u : 0u);
           tc_commit(pvdone0 + tm * 8);
         }
