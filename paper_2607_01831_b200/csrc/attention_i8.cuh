@@ -727,7 +727,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         tc_fence_before();
         named_bar(bar_tm, 128);
         if (r == 0) {
-          mbar_wait(qready0 + qi * 8, (ic >> 1) & 1, abort_word);   // the piece's query planes
+          if (u == u_first) mbar_wait(qready0 + qi * 8, (ic >> 1) & 1, abort_word);   // the piece's query planes
           tc_fence_after();
           const uint32_t d = tmem0 + tm * C::kTmTeam + C::kTmS;
           const uint32_t qd_lo = qd_lo0 + (uint32_t)qi * (C::kQTile >> 4);
