@@ -1385,16 +1385,18 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   p.bt = shape->block_tokens; p.num_blocks = shape->num_blocks; p.max_blocks = shape->max_blocks_per_seq;
   p.ncols = pl.ncols;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // up to 16 columns: the integer tcgen05 kernels
-  if (pl.ncols <= 16) {
+  // up to 32 columns: the integer tcgen05 kernels
+  if (pl.ncols <= 32) {
     if (!full) {
       if (pl.ncols <= 4) return launch_i8<false, 4>(p, st);
       if (pl.ncols <= 8) return launch_i8<false, 8>(p, st);
-      return launch_i8<false, 16>(p, st);
+      if (pl.ncols <= 16) return launch_i8<false, 16>(p, st);
+      return launch_i8<false, 32>(p, st);
     }
     if (pl.ncols <= 4) return launch_i8<true, 4>(p, st);
     if (pl.ncols <= 8) return launch_i8<true, 8>(p, st);
-    return launch_i8<true, 16>(p, st);
+    if (pl.ncols <= 16) return launch_i8<true, 16>(p, st);
+    return launch_i8<true, 32>(p, st);
   }
   // <FULL, NT, DS, TEAMS, stages, CTAs/SM>
   if (!full) {

@@ -42,7 +42,7 @@ constexpr int kI8PieceUnits = 32;  // stage-units whose block ids a producer war
 
 template <bool FULL, int CP>
 struct I8Cfg {
-  static_assert(CP == 4 || CP == 8 || CP == 16, "padded column counts");
+  static_assert(CP == 4 || CP == 8 || CP == 16 || CP == 32, "padded column counts");
   static constexpr int kST = 128;                   // tokens per stage-unit
   static constexpr int kNArr = FULL ? 4 : 2;        // plane arrays copied per 16-token sub-block (the metadata is
                                                     // read with plain loads: the copy engine takes ~35 cycles per copy)
@@ -52,10 +52,14 @@ struct I8Cfg {
   static constexpr int kNPV = 4 * CP;                    // N of the P.V product
   static constexpr int kPartCols = CP < 8 ? 8 : CP;      // column stride of the partial slots
   static constexpr int kColsPad = CP;
-  // warps: kTeams teams of four (team t = warps 4t .. 4t+3), then the producers
-  static constexpr int kTeams = (FULL || CP == 16) ? 3 : CP == 4 ? 5 : 4;
-  static constexpr int kProdWarps = 4;
-  static constexpr int kProdWarp0 = 4 * kTeams;
+  // warps: kTeams teams, then the producers.  A team is one warpgroup per column group: with 32 columns
+  // two warpgroups share the tokens of a unit, each scoring 16 columns (and one expanding K, the other V).
+  static constexpr int kGroups = CP == 32 ? 2 : 1;
+  static constexpr int kCG = CP / kGroups;               // columns of a column group
+  static constexpr int kTeamWarps = 4 * kGroups, kTeamThreads = 32 * kTeamWarps;
+  static constexpr int kTeams = CP == 32 ? 2 : (FULL || CP == 16) ? 3 : CP == 4 ? 5 : 4;
+  static constexpr int kProdWarps = CP == 32 ? 2 : 4;
+  static constexpr int kProdWarp0 = kTeamWarps * kTeams;
   static constexpr int kThreads = (kProdWarp0 + kProdWarps) * 32;
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int kTile = 16384;                    // V level tile: [128 tokens][128 B]
@@ -64,28 +68,30 @@ struct I8Cfg {
   static constexpr int kPLayout = kPRow == 32 ? 6 : kPRow == 64 ? 4 : 2;   // descriptor swizzle mode of the P tile
   static constexpr int kTeamBytes = kTile + kPTile;      // V tile, P tile (the K levels live in tensor memory)
   static constexpr int kQTile = (kNQK * 128 + 1023) / 1024 * 1024;
-  static constexpr int kMail = (CP * 128 + 3 * CP) * 4;  // end-of-piece deposit of a team (in its V tile): O, l, zs, ref
+  static constexpr int kMail = CP * 128 * 4;             // end-of-piece deposit of a team: O in its V tile (l, zs, ref beside its scalars)
   static_assert(kMail <= kTile, "the deposit lives in the team's V tile");
   static constexpr int kOffQT = kTeams * kTeamBytes;
   static constexpr int kOffRing = kOffQT + 2 * kQTile;
-  static constexpr int kTeamScal = (8 * CP + 4 * 2 * CP + 2 * CP) * 4;   // qs, ref, factor, limits; reduce scratch; totals
+  static constexpr int kTeamScal = (8 * CP + 4 * 2 * CP + 2 * CP + 3 * CP) * 4;   // qs, ref, factor, limits, maxima; reduce scratch; totals; deposit header
   static constexpr int kFixedTail = 2 * CP * 256 + kTeams * kTeamScal +
-                                    kProdWarps * 2 * kI8PieceUnits * 4 + 2 * 32 + 64 * 8 + (1 + kTeams) * 256 + 64;
+                                    8 * kI8PieceUnits * 4 + 2 * 32 + 64 * 8 + (1 + kTeams) * 256 + 64;
   static constexpr int kAvail = 227 * 1024 - 1024 - kOffRing - kFixedTail;
   static constexpr int kNStage = kAvail / kStageBytes > 8 ? 8 : kAvail / kStageBytes;
   static_assert(kNStage >= 2, "ring too small");
   static constexpr int kOffQRaw = kOffRing + kNStage * kStageBytes;
   static constexpr int kOffScal = kOffQRaw + 2 * CP * 256;
   static constexpr int kOffBlk = kOffScal + kTeams * kTeamScal;
-  static constexpr int kOffItems = kOffBlk + kProdWarps * 2 * kI8PieceUnits * 4;
+  static constexpr int kOffItems = kOffBlk + 8 * kI8PieceUnits * 4;
   static constexpr int kOffBars = kOffItems + 2 * 32;
   static constexpr int kOffMisc = kOffBars + 64 * 8;             // [1 + teams][64] ints
   static constexpr int kSmem = kOffMisc + (1 + kTeams) * 256 + 64 + 1024;   // + alignment slack
   static_assert(kSmem <= 227 * 1024, "shared memory");
   static_assert(kOffScal % 16 == 0 && kTeamScal % 16 == 0 && kOffBars % 8 == 0, "alignment");
   // tensor memory columns of a team: S, O accumulators, FP32 copy of O, K levels (128 bytes per token)
-  static constexpr int kTmS = 0, kTmO = kNQK, kTmOF = kNQK + kNPV, kTmK = (kTmOF + CP + 7) / 8 * 8;
-  static constexpr int kTmTeam = CP == 16 ? 160 : CP == 4 ? 96 : 128;
+  // (with 32 columns there is no room for the copy: it stays in registers)
+  static constexpr bool kOfInTmem = CP <= 16;
+  static constexpr int kTmS = 0, kTmO = kNQK, kTmOF = kNQK + kNPV, kTmK = kOfInTmem ? (kTmOF + CP + 7) / 8 * 8 : kTmOF;
+  static constexpr int kTmTeam = CP == 32 ? 256 : CP == 16 ? 160 : CP == 4 ? 96 : 128;
   static constexpr int kTmCols = 512;
   static_assert(kTmK + 32 <= kTmTeam && kTeams * kTmTeam <= 512, "tensor memory");
   static constexpr int kDrainUnits = FULL ? 256 : 4096;  // own units after which the int32 sums could overflow
@@ -307,7 +313,7 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
   const int n_units = (int)(lo < hi ? hi - lo : 0);
   if (n_units == 0) return;
 
-  constexpr int SPW = 8 / C::kProdWarps;       // 16-token sub-blocks per warp: 2 or 1
+  constexpr int SPW = 8 / C::kProdWarps;       // 16-token sub-blocks per warp: 1, 2 or 4
   constexpr int RP = SPW * NARR;               // roles of this warp: (sub-block, array)
   const int role = pw * RP + (lane < RP ? lane : 0);
   const int sub = role / NARR, arr = role % NARR, sub_first = SPW * pw;
@@ -316,7 +322,7 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
   const uint32_t my_dst = (uint32_t)(arr == 0 ? C::kOffKA : arr == 1 ? C::kOffVA : arr == 2 ? C::kOffKR : C::kOffVR) +
                           (uint32_t)sub * my_bytes;
   constexpr uint32_t kBytesSub = (FULL ? 4u : 2u) * 1024u;   // bytes of one sub-block
-  uint32_t* my_blk = blk_s + pw * 2 * kI8PieceUnits;   // [2 sub-blocks][kI8PieceUnits]
+  uint32_t* my_blk = blk_s + pw * SPW * kI8PieceUnits;   // [SPW sub-blocks][kI8PieceUnits]
   int b = b_lo, len = clamp_len(b), U = (len + ST - 1) / ST;
   int hkv = (int)(off_lo / U), u = (int)(off_lo % U);
   int remaining = n_units, gs = 0, ic = 0;
@@ -361,11 +367,12 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
       for (int k = 0; k < cn; ++k, ++gs) {
         const int slot = gs % NSTAGE;
         if (gs >= NSTAGE) mbar_wait(empty0 + slot * 8, ((gs / NSTAGE) - 1) & 1, abort_word);
-        const uint32_t row0 = my_blk[k], row1 = SPW == 2 ? my_blk[kI8PieceUnits + k] : 0xFFFFFFFFu;
-        const uint32_t row = sub == sub_first ? row0 : row1;
+        const uint32_t row = my_blk[(sub - sub_first) * kI8PieceUnits + k];
         const uint32_t bar = full0 + slot * 8;
         if (lane == 0) {
-          const uint32_t bytes = (row0 != 0xFFFFFFFFu ? kBytesSub : 0u) + (row1 != 0xFFFFFFFFu ? kBytesSub : 0u);
+          uint32_t bytes = 0;
+#pragma unroll
+          for (int i = 0; i < SPW; ++i) bytes += my_blk[i * kI8PieceUnits + k] != 0xFFFFFFFFu ? kBytesSub : 0u;
           if (bytes) mbar_expect_tx(bar, bytes);
           else mbar_arrive(bar);
         }
@@ -396,9 +403,9 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
 // Largest |q| of a piece's raw queries, by 128 threads (index i of 0..127), reduced over the
 // warp; the caller combines the warps.
 template <int CP>
-__device__ __forceinline__ float i8_q_absmax(const unsigned char* qraw, int i) {
+__device__ __forceinline__ float i8_q_absmax(const unsigned char* qraw, int i, int nthr) {
   float amax = 0.0f;
-  for (int k = i; k < CP * 16; k += 128) {
+  for (int k = i; k < CP * 16; k += nthr) {
     const uint4 v = reinterpret_cast<const uint4*>(qraw)[k];
     const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -455,7 +462,7 @@ __device__ __noinline__ bool seq_wait(const volatile int* ctr, int need, volatil
 template <bool FULL, int CP>
 __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(const AttnParams p) {
   using C = I8Cfg<FULL, CP>;
-  constexpr int NSTAGE = C::kNStage, T = C::kTeams;
+  constexpr int NSTAGE = C::kNStage, T = C::kTeams, G = C::kGroups, CG = C::kCG, TT = C::kTeamThreads;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
@@ -477,12 +484,12 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   if (tid == 0) {
     for (int i = 0; i < NSTAGE; ++i) {
       mbar_init(full0 + i * 8, C::kProdWarps);
-      mbar_init(empty0 + i * 8, 4);               // the four warps of the team that owns the unit
+      mbar_init(empty0 + i * 8, C::kTeamWarps);   // the warps of the team that owns the unit
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(qfull0 + i * 8, 1);
-      mbar_init(qempty0 + i * 8, 4 * T);
-      mbar_init(qready0 + i * 8, 4);
+      mbar_init(qempty0 + i * 8, C::kTeamWarps * T);
+      mbar_init(qready0 + i * 8, C::kTeamWarps);
     }
     for (int i = 0; i < T; ++i) {
       mbar_init(sfull0 + i * 8, 1);
@@ -514,7 +521,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
-  named_bar(8, 4 * T * 32);
+  named_bar(8, T * TT);
   tc_fence_after();
   const uint32_t tmem0 = *reinterpret_cast<volatile uint32_t*>(misc + 8);
   constexpr uint32_t kIdescS = i8_idesc(C::kNQK, false, true), kIdescO = i8_idesc(C::kNPV, true, false);
@@ -523,17 +530,22 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   // Teams.  Team t takes the units gs = t, t + T, ... of the CTA's range and does everything for
   // them: K tile, Q.K^T, V tile, scores -> weights, P.V.
   // =============================================================================================
-  const int tm = warp >> 2, w4 = warp & 3;
+  const int tm = warp / C::kTeamWarps, grp = (warp >> 2) % G, w4 = warp & 3;
   const int r = tid & 127;                        // token of the unit (S), output dim position (O): TMEM lane
+  const int tt = r + 128 * grp;                   // thread of the team
+  const int c0 = grp * CG;                        // first column of this thread's column group
   const uint32_t lane_sel = (uint32_t)(w4 * 32) << 16;
-  const uint32_t tm_s = tmem0 + tm * C::kTmTeam + C::kTmS + lane_sel;
-  const uint32_t tm_o = tmem0 + tm * C::kTmTeam + C::kTmO + lane_sel;
-  const uint32_t tm_of = tmem0 + tm * C::kTmTeam + C::kTmOF + lane_sel;
+  const uint32_t tm_s = tmem0 + tm * C::kTmTeam + C::kTmS + c0 + lane_sel;        // + plane * CP
+  const uint32_t tm_o = tmem0 + tm * C::kTmTeam + C::kTmO + 4 * c0 + lane_sel;
+  const uint32_t tm_of = tmem0 + tm * C::kTmTeam + C::kTmOF + c0 + lane_sel;
   float* my_scal = reinterpret_cast<float*>(smem + C::kOffScal + tm * C::kTeamScal);
   float* qs_s = my_scal, *ref_s = my_scal + CP, *fac_s = my_scal + 2 * CP;
   int* lim_s = reinterpret_cast<int*>(my_scal + 3 * CP);
-  float* my_red = my_scal + 8 * CP;               // [4 warps][2 CP]
+  float* amax_s = my_scal + 4 * CP;               // [team warps]
+  float* my_red = my_scal + 8 * CP;               // [team warps][2 CG]
   float* my_lz = my_scal + 16 * CP;               // [2 CP]
+  float* my_hdr = my_scal + 18 * CP;              // [3 CP] l, zs, ref of this team's deposit
+  const int tw = grp * 4 + w4;                    // warp of the team
   int* my_misc = misc + 64 * (1 + tm);
   const int bar_tm = 1 + tm;                      // named barrier of this team
   const uint32_t vtile = sbase + tm * C::kTeamBytes, ptile = vtile + C::kTile;
@@ -568,9 +580,9 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
       // ---- the piece's queries: fixed-point exponent, sum of q per column, causal limits ----------
       const unsigned char* qb = qraw + qi * CP * 256;
       {
-        const float am = i8_q_absmax<CP>(qb, r);
-        if (lane == 0) my_red[w4] = am;
-        for (int c = w4; c < CP; c += 4) {
+        const float am = i8_q_absmax<CP>(qb, tt, TT);
+        if (lane == 0) amax_s[tw] = am;
+        for (int c = tw; c < CP; c += C::kTeamWarps) {
           const uint2 v = *reinterpret_cast<const uint2*>(qb + c * 256 + lane * 8);
           float sum = (__uint_as_float(v.x << 16) + __uint_as_float(v.x & 0xFFFF0000u)) +
                       (__uint_as_float(v.y << 16) + __uint_as_float(v.y & 0xFFFF0000u));
@@ -578,20 +590,21 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           for (int off = 16; off >= 1; off >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, off);
           if (lane == 0) qs_s[c] = sum;
         }
-        if (r < CP) lim_s[r] = r < p.ncols ? (p.causal ? len - p.nq + r / p.G + 1 : len) : 0;
-        named_bar(bar_tm, 128);
+        if (tt < CP) lim_s[tt] = tt < p.ncols ? (p.causal ? len - p.nq + tt / p.G + 1 : len) : 0;
+        named_bar(bar_tm, TT);
       }
-      const float amax = fmaxf(fmaxf(my_red[0], my_red[1]), fmaxf(my_red[2], my_red[3]));
+      float amax = 0.0f;
+#pragma unroll
+      for (int i = 0; i < C::kTeamWarps; ++i) amax = fmaxf(amax, amax_s[i]);
       const int e = i8_q_exponent(amax);
       const float ca = p.sm_log2 * __int_as_float((127 - e) << 23) * (FULL ? 1.0f : 16.0f);
-      named_bar(bar_tm, 128);   // my_red is reused below
       const uint32_t qt = sbase + C::kOffQT + qi * C::kQTile;
-      if (u_first == 0 && r < CP * 4) {
+      if (u_first == 0 && tt < CP * 4) {
         // this team owns the piece's first unit: it writes the three balanced s8 digit planes of
         // q_int = rint(q 2^e), rows plane * CP + column.  (The slot's previous planes belong to the piece
         // before last, which every team has left: the queries of this piece were loaded after that.)
         const float up = __int_as_float((127 + e) << 23);
-        const int c = r >> 2, j = r & 3;
+        const int c = tt >> 2, j = tt & 3;
         uint32_t pl[3][2][4];   // [plane][parity][word]
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
@@ -633,9 +646,10 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         if (lane == 0) mbar_arrive(qready0 + qi * 8);
       }
 
-      float l[CP], zs[CP];
+      float l[CG], zs[CG];
+      float of_r[C::kOfInTmem ? 1 : CG];   // FP32 copy of O where tensor memory has no room for it
 #pragma unroll
-      for (int c = 0; c < CP; ++c) { l[c] = 0.0f; zs[c] = 0.0f; }
+      for (int c = 0; c < CG; ++c) { l[c] = 0.0f; zs[c] = 0.0f; }
       bool fresh = true, have_of = false;
       int units_in_acc = 0;
       uint32_t n_own = (uint32_t)((gs_base + u_first) / T);   // index of the unit among this team's units
@@ -647,34 +661,41 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         if (units_in_acc > 0) {
           tc_fence_after();
 #pragma unroll
-          for (int c4 = 0; c4 < CP / 4; ++c4) {
+          for (int c4 = 0; c4 < CG / 4; ++c4) {
             uint32_t a[16], of[4];
             TmemRegs<16>::ld(tm_o + c4 * 16, a);
-            if (have_of) TmemRegs<4>::ld(tm_of + c4 * 4, of);
+            if (C::kOfInTmem && have_of) TmemRegs<4>::ld(tm_of + c4 * 4, of);
             tc_wait_ld();
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
               const float v = fmaf(fmaf(fmaf((float)(int)a[4 * k + 3], 256.0f, (float)(int)a[4 * k + 2]), 256.0f,
                                         (float)(int)a[4 * k + 1]), 256.0f, (float)(int)a[4 * k]);
-              const float old = have_of ? __uint_as_float(of[k]) : 0.0f;
-              of[k] = __float_as_uint((old + v) * (scale ? fac_s[c4 * 4 + k] : 1.0f));
+              const float old = !have_of ? 0.0f : C::kOfInTmem ? __uint_as_float(of[k]) : of_r[C::kOfInTmem ? 0 : c4 * 4 + k];
+              const float nw = (old + v) * (scale ? fac_s[c0 + c4 * 4 + k] : 1.0f);
+              of[k] = __float_as_uint(nw);
+              if (!C::kOfInTmem) of_r[C::kOfInTmem ? 0 : c4 * 4 + k] = nw;
             }
-            TmemRegs<4>::st(tm_of + c4 * 4, of);
+            if (C::kOfInTmem) TmemRegs<4>::st(tm_of + c4 * 4, of);
           }
-          tc_wait_st();
+          if (C::kOfInTmem) tc_wait_st();
           have_of = true;
           units_in_acc = 0;
         } else if (have_of && scale) {
 #pragma unroll
-          for (int c4 = 0; c4 < CP / 4; ++c4) {
-            uint32_t of[4];
-            TmemRegs<4>::ld(tm_of + c4 * 4, of);
-            tc_wait_ld();
+          for (int c4 = 0; c4 < CG / 4; ++c4) {
+            if (C::kOfInTmem) {
+              uint32_t of[4];
+              TmemRegs<4>::ld(tm_of + c4 * 4, of);
+              tc_wait_ld();
 #pragma unroll
-            for (int k = 0; k < 4; ++k) of[k] = __float_as_uint(__uint_as_float(of[k]) * fac_s[c4 * 4 + k]);
-            TmemRegs<4>::st(tm_of + c4 * 4, of);
+              for (int k = 0; k < 4; ++k) of[k] = __float_as_uint(__uint_as_float(of[k]) * fac_s[c0 + c4 * 4 + k]);
+              TmemRegs<4>::st(tm_of + c4 * 4, of);
+            } else {
+#pragma unroll
+              for (int k = 0; k < 4; ++k) of_r[C::kOfInTmem ? 0 : c4 * 4 + k] *= fac_s[c0 + c4 * 4 + k];
+            }
           }
-          tc_wait_st();
+          if (C::kOfInTmem) tc_wait_st();
         }
       };
 
@@ -716,17 +737,28 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         if (gs >= NSTAGE && *reinterpret_cast<volatile int*>(misc + 32 + slot) < gs / NSTAGE)
           seq_wait(misc + 32 + slot, gs / NSTAGE, abort_word);
         mbar_wait(full0 + slot * 8, (gs / NSTAGE) & 1, abort_word);
-        if (r == 0) *reinterpret_cast<volatile int*>(misc + 32 + slot) = gs / NSTAGE + 1;
+        if (tt == 0) *reinterpret_cast<volatile int*>(misc + 32 + slot) = gs / NSTAGE + 1;
         float2 km = km_c, vm = vm_c;
         meta_of(row_of(u + T, blk_n1), km_c, vm_c);   // for this team's next unit
         blk_n1 = blk_n2;
         blk_n2 = blk_of(u + 3 * T);                   // and the block id of the one after the one after
-        // ---- K tile (free: the team's previous Q.K^T has been waited for), then Q.K^T ---------------
-        i8_expand_k_tmem<FULL>(st + C::kOffKA, st + C::kOffKR, r, tm_k + lane_sel);
-        tc_wait_st();
+        if (ack_pending) {   // uniform over the team: its last deposit (in the V tile) has been read
+          if (tt == 0) seq_wait(misc + 24 + tm, (int)my_deps, abort_word);
+          named_bar(bar_tm, TT);
+          ack_pending = false;
+        }
+        // ---- K levels (free: the team's previous Q.K^T has been waited for), then Q.K^T; V tile (free
+        // once the team's previous P.V is complete).  With two column groups one expands K, the other V.
+        if (G == 1 || grp == 0) {
+          i8_expand_k_tmem<FULL>(st + C::kOffKA, st + C::kOffKR, r, tm_k + lane_sel);
+          tc_wait_st();
+        } else {
+          if (n_own > 0) mbar_wait(pvdone0 + tm * 8, (n_own - 1) & 1, abort_word);
+          i8_expand<FULL>(st + C::kOffVA, st + C::kOffVR, vtile, w4, lane);
+        }
         tc_fence_before();
-        named_bar(bar_tm, 128);
-        if (r == 0) {
+        named_bar(bar_tm, TT);
+        if (tt == 0) {
           if (u == u_first) mbar_wait(qready0 + qi * 8, (ic >> 1) & 1, abort_word);   // the piece's query planes
           tc_fence_after();
           const uint32_t d = tmem0 + tm * C::kTmTeam + C::kTmS;
@@ -737,14 +769,10 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           tc_commit(sfull0 + tm * 8);
         }
         __syncwarp();
-        // ---- V tile: free once the team's previous P.V is complete (and its deposit there was read) ---
-        if (ack_pending) {   // uniform over the team
-          if (r == 0) seq_wait(misc + 24 + tm, (int)my_deps, abort_word);
-          named_bar(bar_tm, 128);
-          ack_pending = false;
+        if (G == 1 || grp == 0) {   // (the other group has waited already)
+          if (n_own > 0) mbar_wait(pvdone0 + tm * 8, (n_own - 1) & 1, abort_word);
         }
-        if (n_own > 0) mbar_wait(pvdone0 + tm * 8, (n_own - 1) & 1, abort_word);
-        i8_expand<FULL>(st + C::kOffVA, st + C::kOffVR, vtile, w4, lane);
+        if (G == 1) i8_expand<FULL>(st + C::kOffVA, st + C::kOffVR, vtile, w4, lane);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + slot * 8);
         const bool valid = tok < len;
@@ -759,70 +787,71 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         // ---- scores of this thread's token -------------------------------------------------------
         mbar_wait(sfull0 + tm * 8, n_own & 1, abort_word);
         tc_fence_after();
-        float x[CP];
+        float x[CG];
         {
-          uint32_t s0[CP], s1[CP], s2[CP];
-          TmemRegs<CP>::ld(tm_s, s0);
-          TmemRegs<CP>::ld(tm_s + CP, s1);
-          TmemRegs<CP>::ld(tm_s + 2 * CP, s2);
+          uint32_t s0[CG], s1[CG], s2[CG];
+          TmemRegs<CG>::ld(tm_s, s0);
+          TmemRegs<CG>::ld(tm_s + CP, s1);
+          TmemRegs<CG>::ld(tm_s + 2 * CP, s2);
           tc_wait_ld();
 #pragma unroll
-          for (int c = 0; c < CP; ++c) {
+          for (int c = 0; c < CG; ++c) {
             const float sf = fmaf((float)((int)s2[c] * 256 + (int)s1[c]), 256.0f, (float)(int)s0[c]);
-            x[c] = fmaf(sf, al, fmaf(be, qs_s[c], lsv));
+            x[c] = fmaf(sf, al, fmaf(be, qs_s[c0 + c], lsv));
           }
         }
         if (unit_t0 + C::kST > full_lim) {
 #pragma unroll
-          for (int c = 0; c < CP; ++c)
-            if (tok >= lim_s[c]) x[c] = -INFINITY;
+          for (int c = 0; c < CG; ++c)
+            if (tok >= lim_s[c0 + c]) x[c] = -INFINITY;
         }
         // ---- reference exponents: raised when a weight would leave the u32 range -----------------------
         bool need = fresh || units_in_acc >= C::kDrainUnits;
 #pragma unroll
-        for (int c = 0; c < CP; ++c) need |= x[c] - ref_s[c] > 31.5f;
-        if (bar_or(bar_tm, 128, need)) {
+        for (int c = 0; c < CG; ++c) need |= x[c] - ref_s[c0 + c] > 31.5f;
+        if (bar_or(bar_tm, TT, need)) {   // (team-wide: one P.V covers all columns, so they all restart together)
 #pragma unroll
-          for (int c = 0; c < CP; ++c) {
+          for (int c = 0; c < CG; ++c) {
             float mx = x[c];
 #pragma unroll
             for (int off = 16; off >= 1; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
-            if (lane == 0) my_red[w4 * CP + c] = mx;
+            if (lane == 0) my_red[tw * CG + c] = mx;
           }
-          named_bar(bar_tm, 128);
-          if (r < CP) {
-            const float mx = fmaxf(fmaxf(my_red[r], my_red[CP + r]), fmaxf(my_red[2 * CP + r], my_red[3 * CP + r]));
-            const float old = ref_s[r];
+          named_bar(bar_tm, TT);
+          if (tt < CP) {
+            const float* mr = my_red + (tt / CG) * 4 * CG + (tt % CG);   // the four warps of the column's group
+            const float mx = fmaxf(fmaxf(mr[0], mr[CG]), fmaxf(mr[2 * CG], mr[3 * CG]));
+            const float old = ref_s[tt];
             float nw = old, f = 1.0f;
             if (fresh) { nw = fmaxf(mx, -1.0e4f) - 28.0f; f = 0.0f; }
             else if (mx - old > 31.5f) { nw = mx - 28.0f; f = ex2_full(old - nw); }
-            ref_s[r] = nw;
-            fac_s[r] = f;
+            ref_s[tt] = nw;
+            fac_s[tt] = f;
           }
-          named_bar(bar_tm, 128);
+          named_bar(bar_tm, TT);
 #pragma unroll
-          for (int c = 0; c < CP; ++c) { l[c] *= fac_s[c]; zs[c] *= fac_s[c]; }
-          drain(true);   // (the team's previous P.V was waited for before the V tile was rewritten)
+          for (int c = 0; c < CG; ++c) { l[c] *= fac_s[c0 + c]; zs[c] *= fac_s[c0 + c]; }
+          drain(true);   // (the team's previous P.V has been waited for)
           fresh = false;
         }
         // ---- weights ------------------------------------------------------------------------------
-        uint32_t wi[CP];
+        uint32_t wi[CG];
 #pragma unroll
-        for (int c = 0; c < CP; ++c) {
-          const float wf = ex2_full(x[c] - ref_s[c]);
+        for (int c = 0; c < CG; ++c) {
+          const float wf = ex2_full(x[c] - ref_s[c0 + c]);
           asm("cvt.rni.u32.f32 %0, %1;" : "=r"(wi[c]) : "f"(wf));
           l[c] = fmaf(wf, ia, l[c]);
           zs[c] = fmaf(wf, ib, zs[c]);
         }
 #pragma unroll
-        for (int j = 0; j < CP / 4; ++j)
+        for (int j = 0; j < CG / 4; ++j)
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(p_row + (((uint32_t)j ^ p_swz) << 4)), "r"(wi[4 * j]), "r"(wi[4 * j + 1]),
+                       ::"r"(p_row + (((uint32_t)(grp * (CG / 4) + j) ^ p_swz) << 4)), "r"(wi[4 * j]), "r"(wi[4 * j + 1]),
                          "r"(wi[4 * j + 2]), "r"(wi[4 * j + 3]) : "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         tc_fence_before();
-        named_bar(bar_tm, 128);     // the P tile and the V tile are complete, S has been read
-        if (r == 0) {
+        named_bar(bar_tm, TT);     // the P tile and the V tile are complete, S has been read
+        if (tt == 0) {
           tc_fence_after();
           const uint32_t d = tmem0 + tm * C::kTmTeam + C::kTmO;
 #pragma unroll
@@ -838,60 +867,70 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
       // ---- end of the piece for this team -----------------------------------------------------------
       mbar_wait(pvdone0 + tm * 8, (n_own - 1) & 1, abort_word);   // the last P.V
       drain(false);   // the FP32 copy now holds this team's part of O
-      float of[CP];
+      float of[CG];
 #pragma unroll
-      for (int c4 = 0; c4 < CP / 4; ++c4) {
-        uint32_t t[4];
-        TmemRegs<4>::ld(tm_of + c4 * 4, t);
-        tc_wait_ld();
+      for (int c4 = 0; c4 < CG / 4; ++c4) {
+        if (C::kOfInTmem) {
+          uint32_t t[4];
+          TmemRegs<4>::ld(tm_of + c4 * 4, t);
+          tc_wait_ld();
 #pragma unroll
-        for (int k = 0; k < 4; ++k) of[c4 * 4 + k] = __uint_as_float(t[k]);
+          for (int k = 0; k < 4; ++k) of[c4 * 4 + k] = __uint_as_float(t[k]);
+        } else {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) of[c4 * 4 + k] = of_r[C::kOfInTmem ? 0 : c4 * 4 + k];
+        }
       }
       tc_fence_before();
-      // totals of l and zs over the team's 128 token lanes
+      // totals of l and zs over the 128 token lanes of every column group
 #pragma unroll
-      for (int c = 0; c < CP; ++c) {
+      for (int c = 0; c < CG; ++c) {
         float a = l[c], b = zs[c];
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) {
           a += __shfl_xor_sync(0xFFFFFFFFu, a, off);
           b += __shfl_xor_sync(0xFFFFFFFFu, b, off);
         }
-        if (lane == 0) { my_red[w4 * 2 * CP + c] = a; my_red[w4 * 2 * CP + CP + c] = b; }
+        if (lane == 0) { my_red[tw * 2 * CG + c] = a; my_red[tw * 2 * CG + CG + c] = b; }
       }
-      named_bar(bar_tm, 128);
-      if (r < 2 * CP) my_lz[r] = (my_red[r] + my_red[2 * CP + r]) + (my_red[4 * CP + r] + my_red[6 * CP + r]);
-      named_bar(bar_tm, 128);
+      named_bar(bar_tm, TT);
+      if (tt < 2 * CP) {   // my_lz: l of the CP columns, then zs
+        const int which = tt / CP, c = tt % CP;
+        const float* mr = my_red + (c / CG) * 4 * 2 * CG + which * CG + (c % CG);   // the four warps of the column's group
+        my_lz[tt] = (mr[0] + mr[2 * CG]) + (mr[4 * CG] + mr[6 * CG]);
+      }
+      named_bar(bar_tm, TT);
       if (!finisher) {
-        // deposit (O, l, zs, ref) in this team's V tile (idle: its last P.V is complete) for the team that
-        // owns the piece's last unit
+        // deposit O in this team's V tile (idle: its last P.V is complete) and (l, zs, ref) beside its
+        // scalars, for the team that owns the piece's last unit
         float* mail = reinterpret_cast<float*>(smem + tm * C::kTeamBytes);
 #pragma unroll
-        for (int c = 0; c < CP; ++c) mail[c * 128 + r] = of[c];
-        if (r < CP) {
-          mail[CP * 128 + r] = my_lz[r];
-          mail[CP * 128 + CP + r] = my_lz[CP + r];
-          mail[CP * 128 + 2 * CP + r] = ref_s[r];
+        for (int c = 0; c < CG; ++c) mail[(c0 + c) * 128 + r] = of[c];
+        if (tt < CP) {
+          my_hdr[tt] = my_lz[tt];
+          my_hdr[CP + tt] = my_lz[CP + tt];
+          my_hdr[2 * CP + tt] = ref_s[tt];
         }
         __threadfence_block();
-        named_bar(bar_tm, 128);
+        named_bar(bar_tm, TT);
         ++my_deps;
-        if (r == 0) *reinterpret_cast<volatile int*>(misc + 16 + tm) = (int)my_deps;
+        if (tt == 0) *reinterpret_cast<volatile int*>(misc + 16 + tm) = (int)my_deps;
         ack_pending = true;
       } else {
-        float lt[CP], zt[CP], mt[CP];
+        float lt[CG], zt[CG], mt[CG];
 #pragma unroll
-        for (int c = 0; c < CP; ++c) { lt[c] = my_lz[c]; zt[c] = my_lz[CP + c]; mt[c] = ref_s[c]; }
+        for (int c = 0; c < CG; ++c) { lt[c] = my_lz[c0 + c]; zt[c] = my_lz[CP + c0 + c]; mt[c] = ref_s[c0 + c]; }
 #pragma unroll
         for (int d = 0; d < T; ++d) {
           if (d == tm || (d - team0 + T) % T >= n_piece) continue;   // itself; a team without a unit in the piece
-          if (r == 0) seq_wait(misc + 16 + d, (int)dep_cnt[d] + 1, abort_word);   // its deposit is complete
-          named_bar(bar_tm, 128);
+          if (tt == 0) seq_wait(misc + 16 + d, (int)dep_cnt[d] + 1, abort_word);   // its deposit is complete
+          named_bar(bar_tm, TT);
           const float* mo = reinterpret_cast<const float*>(smem + d * C::kTeamBytes);
+          const float* mh = reinterpret_cast<const float*>(smem + C::kOffScal + d * C::kTeamScal) + 18 * CP;
 #pragma unroll
-          for (int c = 0; c < CP; ++c) {
-            const float o2 = mo[c * 128 + r], l2 = mo[CP * 128 + c];
-            const float z2 = mo[CP * 128 + CP + c], m2 = mo[CP * 128 + 2 * CP + c];
+          for (int c = 0; c < CG; ++c) {
+            const float o2 = mo[(c0 + c) * 128 + r], l2 = mh[c0 + c];
+            const float z2 = mh[CP + c0 + c], m2 = mh[2 * CP + c0 + c];
             const float M = fmaxf(mt[c], m2);
             const float f1 = ex2_full(mt[c] - M), f2 = ex2_full(m2 - M);
             of[c] = of[c] * f1 + o2 * f2;
@@ -900,27 +939,28 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
             mt[c] = M;
           }
           __threadfence_block();
-          named_bar(bar_tm, 128);
-          if (r == 0) *reinterpret_cast<volatile int*>(misc + 24 + d) = (int)dep_cnt[d] + 1;   // its V tile may be written again
+          named_bar(bar_tm, TT);
+          if (tt == 0) *reinterpret_cast<volatile int*>(misc + 24 + d) = (int)dep_cnt[d] + 1;   // it may deposit again
         }
         const bool direct = item.n_contrib == 1;
         const size_t bh = (size_t)item.b * p.Hkv + item.hkv;
         float* part = p.ws_part + (bh + (size_t)blockIdx.x) * (size_t)C::kPartCols * kPartStride;
 #pragma unroll
-        for (int c = 0; c < CP; ++c) {
+        for (int cc = 0; cc < CG; ++cc) {
+          const int c = c0 + cc;
           if (c >= p.ncols) break;
-          const float v = of[c] + zt[c];
+          const float v = of[cc] + zt[cc];
           if (direct) {
             const int j = c / p.G, hh = c % p.G;
             p.out[(((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + dim_out] =
-                lt[c] > 0.0f ? v / lt[c] : 0.0f;
+                lt[cc] > 0.0f ? v / lt[cc] : 0.0f;
           } else {
             part[(size_t)c * kPartStride + dim_out] = v;
-            if (r == 0) { part[(size_t)c * kPartStride + 128] = mt[c]; part[(size_t)c * kPartStride + 129] = lt[c]; }
+            if (r == 0) { part[(size_t)c * kPartStride + 128] = mt[cc]; part[(size_t)c * kPartStride + 129] = lt[cc]; }
           }
         }
         __threadfence();
-        finish_piece<FULL, C::kPartCols, 128>(p, item, direct, r, my_misc, bar_tm);
+        finish_piece<FULL, C::kPartCols, TT>(p, item, direct, tt, my_misc, bar_tm);
       }
     }
     // every team keeps count of every team's deposits (the phase of its deposit barrier)
@@ -934,7 +974,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   }
   // ---- release the tensor memory ---------------------------------------------------------------
   tc_fence_before();
-  named_bar(9, 4 * T * 32);
+  named_bar(9, T * TT);
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem0), "r"((uint32_t)C::kTmCols)
