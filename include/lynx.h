@@ -62,7 +62,8 @@ typedef enum {
   LYNX_ERR_WORKSPACE = 5,       /* workspace too small (see lynx_workspace_bytes) */
   LYNX_ERR_CUDA = 6,            /* a CUDA runtime call failed */
   LYNX_ERR_BAD_BLOCK_TABLE = 7, /* (lynx_check) a kernel saw a block id out of range */
-  LYNX_ERR_TIMEOUT = 8          /* (lynx_check) a bounded on-chip wait ran out */
+  LYNX_ERR_TIMEOUT = 8,         /* (lynx_check) a bounded on-chip wait ran out */
+  LYNX_ERR_RANGE = 9            /* (lynx_check) a value row outside the range a kernel can represent */
 } lynx_status;
 
 /* One of K or V of one layer (or of several flattened layers), quantised and paged. */

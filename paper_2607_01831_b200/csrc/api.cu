@@ -29,6 +29,7 @@ extern "C" const char* lynx_status_string(lynx_status s) {
     case LYNX_ERR_CUDA: return "CUDA runtime error";
     case LYNX_ERR_BAD_BLOCK_TABLE: return "block id out of range seen by a kernel";
     case LYNX_ERR_TIMEOUT: return "a bounded on-chip wait ran out";
+    case LYNX_ERR_RANGE: return "a value row has a range beyond what the kernel represents";
   }
   return "unknown status";
 }
@@ -56,5 +57,6 @@ extern "C" lynx_status lynx_check(void* workspace, void* stream) {
   }
   if (flags & lynx::kFlagTimeout) return LYNX_ERR_TIMEOUT;
   if (flags & lynx::kFlagBadBlock) return LYNX_ERR_BAD_BLOCK_TABLE;
+  if (flags & lynx::kFlagRange) return LYNX_ERR_RANGE;
   return LYNX_OK;
 }

@@ -6,13 +6,13 @@
 // With one (scale, zero) per token row the two contractions of Section 2's attention run on the
 // integer levels themselves (see attention.cu).  Here both are exact integer tensor-core
 // products over a 128-token stage-unit:
-//   S^T[128 tokens x 3 CP]   = level(K)[128 x 128 dims] . Qd^T     A = K tile (u8, K-major),
+//   S^T[128 tokens x 3 CP]   = level(K)[128 x 128 dims] . Qd^T     A = K levels (u8, in tensor memory),
 //                                                                   B = three balanced s8 digit planes
 //                                                                       of the fixed-point query
 //   O^T[128 dims x 4 CP]    += level(V)^T[128 x 128 tokens] . Wd    A = V tile (u8, MN-major),
 //                                                                   B = the four bytes of the u32
 //                                                                       fixed-point weights (MN-major)
-// CP = query columns (n_q * G) padded to 4, 8, 16 or 32.  The int32 accumulators are exact, so
+// CP = query columns (n_q * G) padded to 4, 8, 16 or 32 (anchor calls with more are run in slices).  The int32 accumulators are exact, so
 // there is no rounding in either product: the query is good to 2^-22 of its largest entry and a
 // weight to 2^-28 of the largest weight seen so far.
 //
@@ -24,15 +24,22 @@
 // W / scale_v, so a single attended token reproduces its value row to FP32 rounding.
 //
 // Warp roles of a CTA (one CTA per SM):
-//   2 softmax warpgroups take alternate units; each has its own S, O and FP32 copy in tensor
-//     memory, its own reference exponents and its own P tile.  A thread owns one token of the
-//     unit (TMEM lane = token for S) and, when accumulators are read back, one output dim.
-//   4 + 4 expander warps turn the nibble planes of a raw stage into the u8 level tiles of K and
-//     of V (128-byte-swizzled canonical layout, the same bytes K-major for K and MN-major for V);
-//     the K expanders also build the query digit planes of a piece.
-//   4 producer warps stream the raw planes into a shared-memory ring (cp.async.bulk).
-//   1 thread issues every tcgen05.mma and commit.
-// All hand-offs are mbarriers with bounded waits; nothing waits on another CTA.
+//   Teams of four warps (eight with 32 columns) each take every kTeams-th unit of the CTA's range
+//     and do everything for it, so that no hand-off between warps with different jobs lies on the
+//     path of a unit and the teams hide one another's latencies:
+//       K levels into tensor memory (a thread owns a token = a TMEM lane; Q.K^T takes its A
+//         operand from there, so the K levels never pass through shared memory again);
+//       Q.K^T (one thread issues four tcgen05.mma and a commit);
+//       V level tile into shared memory (128-byte-swizzled canonical layout, MN-major);
+//       scores -> weights: S read back (TMEM lane = token), per-token scale / zero point / causal
+//         limit applied, weights written to the team's P tile;
+//       P.V (one thread issues), accumulators and their FP32 copy in the team's tensor memory.
+//     The team that owns a piece's first unit also writes the piece's query digit planes; at the
+//     end of a piece the teams' partial results are merged by the team that owns its last unit.
+//   Producer warps stream the raw planes into a shared-memory ring (cp.async.bulk).  The per-token
+//     (scale, zero) pairs do not travel with them (the copy engine takes ~35 cycles per copy
+//     whatever its size): every thread reads its own, two units ahead.
+// All hand-offs are mbarriers or sequence counters with bounded waits; nothing waits on another CTA.
 //
 // Element order along head_dim inside operand tiles: byte 16 (2 j + parity) + 4 w + i of a row
 // holds dim 32 j + 8 w + 2 i + parity (what the nibble expansion yields with two logic
@@ -293,7 +300,7 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
     for (int b = cta; b < p.B; b += n_cta) {
       if (clamp_len(b) != 0) continue;
       const size_t n = (size_t)p.nq * p.Hq * LYNX_D;
-      for (size_t i = lane; i < n; i += 32) p.out[(size_t)b * n + i] = 0.0f;
+      for (size_t i = lane; i < n; i += 32) p.out[(size_t)b * p.nq_stride * p.Hq * LYNX_D + i] = 0.0f;
       if (FULL && p.draft != nullptr) {
         int fr = p.nq;
         for (int j = p.nq - 1; j >= 0; --j) {
@@ -344,7 +351,7 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
       __syncwarp();
       for (int j = lane; j < p.nq; j += 32)
         bulk_g2s(qraw_u32 + (uint32_t)((qi * C::kColsPad + j * p.G) * LYNX_D * 2),
-                 p.q + (((size_t)b * p.nq + j) * p.Hq + (size_t)hkv * p.G) * LYNX_D,
+                 p.q + (((size_t)b * p.nq_stride + j) * p.Hq + (size_t)hkv * p.G) * LYNX_D,
                  (uint32_t)(p.G * LYNX_D * 2), qfull0 + qi * 8);
     }
     for (int c0 = 0; c0 < n; c0 += kI8PieceUnits) {
@@ -576,7 +583,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
     const int team_f = (gs_base + n_piece - 1) % T;       // team of the piece's last unit: it writes the piece's result
     if (u_first < n_piece) {
       const bool finisher = tm == team_f;
-      const int full_lim = p.causal ? len - p.nq + 1 : len;
+      const int full_lim = p.causal ? len - p.tail + 1 : len;
       // ---- the piece's queries: fixed-point exponent, sum of q per column, causal limits ----------
       const unsigned char* qb = qraw + qi * CP * 256;
       {
@@ -590,7 +597,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           for (int off = 16; off >= 1; off >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, off);
           if (lane == 0) qs_s[c] = sum;
         }
-        if (tt < CP) lim_s[tt] = tt < p.ncols ? (p.causal ? len - p.nq + tt / p.G + 1 : len) : 0;
+        if (tt < CP) lim_s[tt] = tt < p.ncols ? (p.causal ? len - p.tail + tt / p.G + 1 : len) : 0;
         named_bar(bar_tm, TT);
       }
       float amax = 0.0f;
@@ -952,7 +959,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           const float v = of[cc] + zt[cc];
           if (direct) {
             const int j = c / p.G, hh = c % p.G;
-            p.out[(((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + dim_out] =
+            p.out[(((size_t)item.b * p.nq_stride + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + dim_out] =
                 lt[cc] > 0.0f ? v / lt[cc] : 0.0f;
           } else {
             part[(size_t)c * kPartStride + dim_out] = v;

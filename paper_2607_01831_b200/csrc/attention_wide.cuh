@@ -722,6 +722,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
         sc[2] = in ? km.y * cb : 0.0f;     // beta: score per unit of sum(q)
         sc[128] = in ? vm.y : 0.0f;        // zero point of the V row
         sc[130] = in ? vm.x * kWideWeightUp : 0.0f;   // scale of the V row, times the weights' factor
+        if (in && !(vm.x < 16.0f)) atomicOr(p.ws_flags, kFlagRange);   // FP16 weights would overflow: reported, not hidden
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();

@@ -29,5 +29,6 @@ __host__ int sm_count();
 constexpr int kWsHeaderBytes = 256;
 constexpr uint32_t kFlagBadBlock = 1u;
 constexpr uint32_t kFlagTimeout = 2u;
+constexpr uint32_t kFlagRange = 4u;
 
 }  // namespace lynx

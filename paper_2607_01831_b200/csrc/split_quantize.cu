@@ -22,10 +22,7 @@ constexpr int kLanesPerRow = 8;   // a quarter-warp owns a row: 2 x 16 B per lan
 // rows per quarter-warp per loop trip: dense rows 8 (2: 0.84, 4: 0.87, 8: 0.90 of the copy rate; 12:
 // spills); rows of listed blocks 4 (2: 0.81, 4: 0.87, 8: 0.77: the block lookups cost registers)
 constexpr int kRowsInFlight = 8;
-#ifndef LYNX_SQ_IDS_ROWS
-#define LYNX_SQ_IDS_ROWS 4
-#endif
-constexpr int kRowsInFlightIds = LYNX_SQ_IDS_ROWS;
+constexpr int kRowsInFlightIds = 4;
 
 // Round-half-even of the exact product u*inv, as the low byte of an FP32 whose ulp is 1:
 // fma(u, inv, 1.5 * 2^23) rounds the exact sum once, to an integer, ties to even.
