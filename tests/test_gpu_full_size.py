@@ -37,6 +37,7 @@ def test_config_full_size_sampled_layers(cfg):
     nbl, Hkv, bt = wlk.nb_layer, wl.num_kv_heads, wl.block_tokens
     table = torch.arange(nbl, dtype=torch.int32).view(1, nbl).numpy()
     lens = np.array([wl.context], np.int32)
+    exercised = 0
     for layer in (0, wl.layers - 1):
         sl = slice(layer * nbl, (layer + 1) * nbl)
         planes = {}
@@ -48,7 +49,8 @@ def test_config_full_size_sampled_layers(cfg):
             assert np.array_equal(got.meta[sl].cpu().numpy().view(np.uint32), want[2].view(np.uint32))
             planes[which] = want
         for win in wlk.windows:                # k = 2, 4, 8: 8, 16 and 32 columns
-            _check_window(oracle, win, layer, planes, table, lens, Hkv, bt)
+            exercised += _check_window(oracle, win, layer, planes, table, lens, Hkv, bt)
+    assert exercised >= 1, "no accept/reject index was compared: every deviation fell inside the guard band"
 
 
 def _check_window(oracle, win, b, planes, table, lens, Hkv, bt):
@@ -61,24 +63,26 @@ def _check_window(oracle, win, b, planes, table, lens, Hkv, bt):
         g = got.astype(np.float64)
         assert np.all(np.abs(g - ref) <= ATOL + RTOL * np.abs(ref)), (win["k"], float(np.abs(g - ref).max()))
     want_fr, want_dev = oracle.verify_decision(ref_f, draft, 0.5, 0.1)
+    assert np.allclose(win["dev"][b].cpu().numpy(), want_dev[0], rtol=0.05, atol=1e-3)
     if np.all(np.abs(want_dev - 1.0) > 0.05):
         assert int(win["first_reject"][b]) == int(want_fr[0])
-    assert np.allclose(win["dev"][b].cpu().numpy(), want_dev[0], rtol=0.05, atol=1e-3)
+        return 1        # an index was compared
+    return 0            # a deviation within 5 % of the threshold: the index may legitimately differ
 
 
-@pytest.mark.parametrize("cfg,layers", [(5, 2), (4, 2), (5, 0)])
+@pytest.mark.parametrize("cfg,layers", [(5, 2), (4, 2), (5, 0), (4, 0)])
 def test_config_shape_sampled(cfg, layers):
     """The 70B-class shape (config 5: GQA group 8, batch 2, k = 8: 64 verify columns) at two layers
     and at its full 80 (a CTA then works through whole 131072-token heads: the longest accumulation
     chains of any configuration), and two layers of the ragged serving mix (config 4: 16 sequences
     of 8192..65536 tokens, lengths that are no multiples of 16, shuffled 16-token blocks,
-    quantisation of listed blocks, k = 4), through the same Workload class and launches as bench.py:
-    sampled (layer, sequence) pairs."""
+    quantisation of listed blocks, k = 4) and its full 32 layers, through the same Workload class and
+    launches as bench.py: sampled (layer, sequence) pairs."""
     import bench
     import oracle
     torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
-    need = 150 if layers == 0 else 16
+    need = (150 if cfg == 5 else 135) if layers == 0 else 16
     if free < need * 2 ** 30:
         pytest.skip(f"needs ~{need} GB of device memory")
     wlk = bench.Workload(cfg, torch.device("cuda", 0), layers=layers)
@@ -89,6 +93,7 @@ def test_config_shape_sampled(cfg, layers):
         wlk.lynx.check(w["ws"])
     nbl, Hkv, bt = wlk.nb_layer, wl.num_kv_heads, wl.block_tokens
     table_all = wlk.table.cpu().numpy()
+    exercised = 0
     for b in (0, wlk.B // 2 + 1, wlk.B - 1)[::(1 if cfg == 4 else 2)]:   # flattened (layer, sequence) index
         layer, seq = divmod(b, wl.batch)
         sl = slice(layer * nbl, (layer + 1) * nbl)
@@ -104,7 +109,8 @@ def test_config_shape_sampled(cfg, layers):
             assert np.array_equal(got.meta[sl].cpu().numpy().view(np.uint32)[used], want[2].view(np.uint32)[used])
             planes[which] = want
         for win in wlk.windows:
-            _check_window(oracle, win, b, planes, table, lens, Hkv, bt)
+            exercised += _check_window(oracle, win, b, planes, table, lens, Hkv, bt)
+    assert exercised >= 1, "no accept/reject index was compared: every deviation fell inside the guard band"
 
 
 @pytest.mark.parametrize("G,k", [(4, 2), (4, 8), (8, 8)])

@@ -189,9 +189,11 @@ def test_merge_verify_matches_oracle_and_decides_identically(lynx, case, causal)
     ref = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(),
                            c["lens"].numpy(), Hkv, bt, causal=causal)
     # thresholds: pick (atol, rtol) so that every oracle dev is outside the guard band around 1
+    exercised = 0
     for atol, rtol in [(2e-2, 2e-2), (5e-2, 5e-2), (1e-1, 1e-1), (3e-1, 1e-1), (1.0, 0.0), (3e-3, 0.0)]:
         want_fr, want_dev = oracle.verify_decision(ref, draft_np, atol, rtol)
         if np.all(np.abs(want_dev - 1.0) > 0.05):
+            exercised += 1
             out, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"],
                                                        draft_out=draft, atol=atol, rtol=rtol,
                                                        causal=causal)
@@ -199,6 +201,7 @@ def test_merge_verify_matches_oracle_and_decides_identically(lynx, case, causal)
             _close(out.cpu().numpy().astype(np.float64), ref, "merge-verify attention")
             assert np.array_equal(fr.cpu().numpy(), want_fr), (atol, rtol, want_dev)
             assert np.allclose(dev.cpu().numpy(), want_dev, rtol=0.05, atol=1e-3)
+    assert exercised >= 1, "every threshold set fell inside the guard band: no index was compared"
     # the full result fed back as its own draft is accepted everywhere
     out, _, _ = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=causal)
     _close(out.cpu().numpy().astype(np.float64), ref, "merge-verify attention (no draft)")
@@ -356,15 +359,18 @@ def test_wide_verify_matches_oracle_and_decides_identically(lynx, case, causal):
     rng = np.random.default_rng(7)
     draft = torch.from_numpy((ref + rng.normal(0.0, 0.02, ref.shape)).astype(np.float32))
     draft[0, k // 2] += 0.5
+    exercised = 0
     for atol, rtol in [(0.2, 0.0), (0.1, 0.1), (0.3, 0.1), (1.0, 0.0)]:
         want_fr, want_dev = oracle.verify_decision(ref, draft.numpy(), atol, rtol)
         if np.all(np.abs(want_dev - 1.0) > 0.05):
+            exercised += 1
             _, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"],
                                                      draft_out=draft.cuda(), atol=atol, rtol=rtol,
                                                      causal=causal)
             lynx.check(c["ws"])
             assert np.array_equal(fr.cpu().numpy(), want_fr), (atol, rtol, want_dev)
             assert np.allclose(dev.cpu().numpy(), want_dev, rtol=0.05, atol=2e-3)
+    assert exercised >= 1, "every threshold set fell inside the guard band: no index was compared"
 
 
 def test_wide_verify_long_context_many_pieces(lynx):
@@ -437,6 +443,7 @@ def test_seeded_random_shapes_all_variants(lynx, long_batches):
     pool = [0, 1, 17, 300, 5000, 12345, 20000, 33333, 47001] if long_batches else \
         [0, 1, 5, 16, 63, 64, 65, 200, 777, 1500, 3100]
     done = 0
+    exercised = 0
     while done < (8 if long_batches else 14):
         Hkv = int(rng.choice([1, 2, 3]))
         G = int(rng.choice([1, 2, 3, 4, 6, 8, 16]))
@@ -464,7 +471,9 @@ def test_seeded_random_shapes_all_variants(lynx, long_batches):
         want_fr, want_dev = oracle.verify_decision(ref_f, out_a.cpu().numpy(), 0.25, 0.05)
         if np.all(np.abs(want_dev - 1.0) > 0.05):
             assert np.array_equal(fr.cpu().numpy(), want_fr), what
+            exercised += 1
         done += 1
+    assert exercised >= done // 2, f"only {exercised} of {done} shapes had their indices compared"
 
 
 @pytest.mark.parametrize("bt,G,k,lens", [(48, 4, 4, (1000, 5, 48, 49)), (112, 2, 16, (4000,)),
@@ -507,3 +516,85 @@ def test_custom_softmax_scale(lynx, scale):
         lynx.check(c["ws"])
         _close(out_a.cpu().numpy().astype(np.float64), ref_a, f"anchor scale={scale} k={k}")
         _close(out_f.cpu().numpy().astype(np.float64), ref_f, f"verify scale={scale} k={k}")
+
+
+# ------------------------------------------------------------------ input ranges at the edges
+@pytest.mark.parametrize("qscale", [8.0, 32.0, 128.0])
+@pytest.mark.parametrize("recipe", ["student_t4", "normal"])
+def test_scaled_queries(lynx, qscale, recipe):
+    # queries far larger than the N(0,1) ones of the other tests (max |q| up to ~500): attention
+    # becomes one-hot-like and any error in the logits shows.  The integer kernels carry the query
+    # as 22-bit fixed point relative to its largest entry, the FP16 kernels as exact FP16 after a
+    # power-of-two scale: 4, 16, 32 and 64 columns, anchor and merge-verify.
+    Hkv = 2
+    for G, k in ((4, 1), (4, 4), (4, 8), (8, 8)):
+        c = _case(lynx, 8100 + k + G, 2, Hkv, G, k, (1500, 333), 16, True, recipe)
+        q = (c["q"].float() * qscale).to(torch.bfloat16)
+        qd, td, ld = q.cuda(), c["table"].cuda(), c["lens"].cuda()
+        for full in (False, True):
+            ref = oracle.attention(full, bf16_bits(q), c["kp"], c["vp"], c["table"].numpy(), c["lens"].numpy(),
+                                   Hkv, 16, causal=True)
+            if full:
+                got = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True)[0]
+            else:
+                got = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True)
+            lynx.check(c["ws"])
+            _close(got.cpu().numpy().astype(np.float64), ref, f"qscale={qscale} {recipe} cols={k * G} full={full}")
+
+
+def _scaled_value_case(lynx, seed, G, k, vscale):
+    """A case whose V rows are scaled by `vscale` before quantisation (K unchanged)."""
+    B, Hkv, bt, lens = 2, 2, 16, (700, 65)
+    lens_t = torch.tensor(lens, dtype=torch.int32)
+    table, nb = synth.block_table(lens_t, bt, True, "vr", seed)
+    kx = synth.kv_block_values("normal", nb, Hkv, bt, "cpu", "vrK", seed)
+    vx = (synth.kv_block_values("normal", nb, Hkv, bt, "cpu", "vrV", seed).float() * vscale).to(torch.bfloat16)
+    q = synth.queries(B, k, Hkv * G, "cpu", "vrQ", seed)
+    K, V = lynx.split_quantize(kx.cuda()), lynx.split_quantize(vx.cuda())
+    kp, vp = oracle.split_quantize(bf16_bits(kx)), oracle.split_quantize(bf16_bits(vx))
+    geo = lynx.Geometry(Hkv * G, Hkv, bt, nb, table.shape[1])
+    return dict(geo=geo, ws=lynx.make_workspace(geo, B, k, "cuda"), q=q, K=K, V=V, kp=kp, vp=vp, table=table,
+                lens=lens_t, Hkv=Hkv, bt=bt)
+
+
+@pytest.mark.parametrize("vscale", [1.0e-3, 400.0, 1.0e30])
+def test_value_rows_of_any_range_on_the_integer_kernels(lynx, vscale):
+    # the integer kernels fold log2(scale_v) into the weights' exponent, so the magnitude of the V rows
+    # (here ranges of ~1e-2, ~3000 and ~1e31) does not matter: relative accuracy as for ordinary rows
+    for G, k, full in ((4, 1, False), (4, 4, False), (8, 8, False), (4, 2, True), (4, 4, True)):
+        c = _scaled_value_case(lynx, 8300 + k, G, k, vscale)
+        qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+        ref = oracle.attention(full, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(), c["lens"].numpy(),
+                               c["Hkv"], 16, causal=True)
+        if full:
+            got = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True)[0]
+        else:
+            got = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True)
+        lynx.check(c["ws"])
+        got = got.cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(got))
+        err = np.abs(got - ref) / (ATOL * vscale + RTOL * np.abs(ref))     # the tolerance scaled with the rows
+        assert float(err.max()) <= 1.0, (vscale, G, k, full, float(err.max()))
+
+
+def test_value_range_limit_of_the_fp16_verify_kernels_is_reported(lynx):
+    # merge-verify with 17..64 columns carries the weights in FP16: value rows whose scale reaches 16 (a
+    # range above 4080) would overflow them.  Just below the limit the result is within tolerance; above
+    # it lynx_check reports LYNX_ERR_RANGE instead of a silent Inf / NaN.
+    G, k = 4, 8
+    c = _scaled_value_case(lynx, 8400, G, k, 400.0)      # ranges ~3000: scale_v ~ 12
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    assert float(c["vp"][2][..., 0].max()) < 16.0
+    ref = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(), c["lens"].numpy(),
+                           c["Hkv"], 16, causal=True)
+    got = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True)[0]
+    lynx.check(c["ws"])
+    err = np.abs(got.cpu().numpy().astype(np.float64) - ref) / (ATOL * 400.0 + RTOL * np.abs(ref))
+    assert float(err.max()) <= 1.0
+    c = _scaled_value_case(lynx, 8401, G, k, 4000.0)     # ranges ~30000: scale_v ~ 120
+    assert float(c["vp"][2][..., 0].max()) > 16.0
+    lynx.merge_verify_attention(c["geo"], c["q"].cuda(), c["K"], c["V"], c["table"].cuda(), c["lens"].cuda(),
+                                c["ws"], causal=True)
+    with pytest.raises(lynx.LynxError, match="range"):
+        lynx.check(c["ws"])
+    lynx.check(c["ws"])                                   # the status word was cleared
