@@ -161,6 +161,22 @@ lynx_status lynx_anchor_attention_static(const lynx_shape* shape, const void* q_
                                          const int32_t* block_table, const int32_t* seq_lens,
                                          float softmax_scale, float* out, void* stream);
 
+/* Decode attention over dequantised BF16 pages: the path the paper itself describes (Section 4.2: the
+ * dequantisation kernel scatters BF16 pages into the paged KV memory, the engine's attention reads
+ * them; Section 2 attention equation), here as the baseline the fused calls above are measured
+ * against (256 bytes per row of K or V instead of 72 / 136).
+ * k_pages_bf16, v_pages_bf16 : BF16 [num_blocks][Hkv][block_tokens][128], as lynx_recombine writes
+ * them (dequant_bf16).  q_bf16, block_table, seq_lens, causal, softmax_scale, out as for
+ * lynx_anchor_attention.  n_q * (Hq/Hkv) must be <= 8 (decode and short windows); any block_tokens.
+ * workspace : lynx_bf16_workspace_bytes(shape, batch, n_q) bytes of scratch (split-K partials), no
+ * initialisation needed.  Out-of-range block ids are clamped and not reported. */
+size_t lynx_bf16_workspace_bytes(const lynx_shape* shape, int32_t batch, int32_t n_q);
+lynx_status lynx_bf16_attention(const lynx_shape* shape, const void* q_bf16, int32_t batch, int32_t n_q,
+                                int32_t causal, const void* k_pages_bf16, const void* v_pages_bf16,
+                                const int32_t* block_table, const int32_t* seq_lens,
+                                float softmax_scale, float* out, void* workspace,
+                                size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, reads and clears the workspace's status word.  Test / debug use. */
 lynx_status lynx_check(void* workspace, void* stream);
 

@@ -137,3 +137,43 @@ def verify_decision(out_full: np.ndarray, draft_f32: np.ndarray, atol: float, rt
                                         ctypes.c_int32(Hq), ctypes.c_double(atol),
                                         ctypes.c_double(rtol), _p(fr), _p(dev))
     return fr, dev
+
+
+def attention_bf16_pages(q_bf16_bits: np.ndarray, k_pages_bits: np.ndarray, v_pages_bits: np.ndarray,
+                         block_table: np.ndarray, seq_lens: np.ndarray, causal: bool = False,
+                         softmax_scale: float | None = None) -> np.ndarray:
+    """Attention over dequantised BF16 pages in binary64: the decode path the paper describes
+    (Section 4.2: the dequantisation kernel scatters BF16 pages, the engine's attention reads them;
+    Section 2: softmax(Q K^T / sqrt(d)) V).  Plain numpy, one (sequence, query, head) at a time.
+
+    q_bf16_bits uint16 [B][n_q][Hq][128]; k/v_pages_bits uint16 [num_blocks][Hkv][block_tokens][128]
+    (BF16 bit patterns); block_table int32 [B][max_blocks]; seq_lens int32 [B].  Query j of
+    sequence b sees tokens [0, len) or, causal, [0, len - n_q + j + 1).  Returns float64
+    [B][n_q][Hq][128]; a query that sees nothing gets zeros.
+    """
+    def f64(bits):
+        return (np.ascontiguousarray(bits, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    q, kp, vp = f64(q_bf16_bits), f64(k_pages_bits), f64(v_pages_bits)
+    B, n_q, Hq, d = q.shape
+    _, Hkv, bt, _ = kp.shape
+    assert d == D and Hq % Hkv == 0
+    G = Hq // Hkv
+    if softmax_scale is None:
+        softmax_scale = 1.0 / np.sqrt(np.float64(D))
+    scale = np.float64(np.float32(softmax_scale))
+    out = np.zeros((B, n_q, Hq, D), np.float64)
+    for b in range(B):
+        length = min(max(int(seq_lens[b]), 0), block_table.shape[1] * bt)
+        nblk = (length + bt - 1) // bt
+        blocks = np.asarray(block_table[b, :nblk], np.int64)
+        for h in range(Hq):
+            k_rows = kp[blocks, h // G].reshape(-1, D)[:length]      # token t = row t % bt of block t / bt
+            v_rows = vp[blocks, h // G].reshape(-1, D)[:length]
+            for j in range(n_q):
+                lim = length - n_q + j + 1 if causal else length
+                if lim <= 0:
+                    continue
+                s = (k_rows[:lim] @ q[b, j, h]) * scale
+                w = np.exp(s - s.max())
+                out[b, j, h] = (w / w.sum()) @ v_rows[:lim]
+    return out

@@ -38,7 +38,7 @@ class _Shape(ctypes.Structure):
 
 EXPORTS = ["lynx_split_quantize", "lynx_recombine", "lynx_workspace_bytes", "lynx_workspace_init",
            "lynx_anchor_attention", "lynx_merge_verify_attention", "lynx_anchor_attention_static",
-           "lynx_check",
+           "lynx_bf16_workspace_bytes", "lynx_bf16_attention", "lynx_check",
            "lynx_status_string", "lynx_version"]
 
 
@@ -74,6 +74,11 @@ def load():
     lib.lynx_anchor_attention_static.argtypes = [ctypes.POINTER(_Shape), vp, i32, i32, i32, _Plane,
                                                  _Plane, vp, vp, f32, vp, vp]
     lib.lynx_anchor_attention_static.restype = ctypes.c_int
+    lib.lynx_bf16_workspace_bytes.argtypes = [ctypes.POINTER(_Shape), i32, i32]
+    lib.lynx_bf16_workspace_bytes.restype = ctypes.c_size_t
+    lib.lynx_bf16_attention.argtypes = [ctypes.POINTER(_Shape), vp, i32, i32, i32, vp, vp, vp, vp, f32, vp, vp,
+                                        ctypes.c_size_t, vp]
+    lib.lynx_bf16_attention.restype = ctypes.c_int
     lib.lynx_check.argtypes = [vp, vp]
     lib.lynx_check.restype = ctypes.c_int
     lib.lynx_status_string.argtypes = [ctypes.c_int]
@@ -243,3 +248,26 @@ def merge_verify_attention(geo: Geometry, q: torch.Tensor, K: Planes, V: Planes,
                                            workspace.numel(), _stream()),
         "lynx_merge_verify_attention")
     return out_full, first_reject, dev
+
+
+def bf16_attention(geo: Geometry, q: torch.Tensor, k_pages: torch.Tensor, v_pages: torch.Tensor,
+                   block_table: torch.Tensor, seq_lens: torch.Tensor, workspace: torch.Tensor | None = None,
+                   causal: bool = False, softmax_scale: float = 0.0, out: torch.Tensor | None = None) -> torch.Tensor:
+    """lynx_bf16_attention: decode attention over dequantised BF16 pages [num_blocks][Hkv][bt][128]
+    (what recombine(want_bf16=True) writes).  q BF16 [B][n_q][Hq][128] -> float32 [B][n_q][Hq][128]."""
+    B, n_q, Hq, d = q.shape
+    if q.dtype != torch.bfloat16 or d != D or Hq != geo.num_q_heads:
+        raise LynxError("q must be BF16 [B][n_q][Hq][128]")
+    if k_pages.dtype != torch.bfloat16 or v_pages.dtype != torch.bfloat16:
+        raise LynxError("pages must be BF16")
+    if out is None:
+        out = torch.empty(B, n_q, Hq, D, dtype=torch.float32, device=q.device)
+    if workspace is None:
+        n = int(load().lynx_bf16_workspace_bytes(ctypes.byref(geo._c()), B, n_q))
+        if n == 0:
+            raise LynxError("unsupported attention shape")
+        workspace = torch.empty(n, dtype=torch.uint8, device=q.device)
+    _ok(load().lynx_bf16_attention(ctypes.byref(geo._c()), _ptr(q), B, n_q, int(causal), _ptr(k_pages),
+                                   _ptr(v_pages), _ptr(block_table), _ptr(seq_lens), softmax_scale, _ptr(out),
+                                   _ptr(workspace), workspace.numel(), _stream()), "lynx_bf16_attention")
+    return out

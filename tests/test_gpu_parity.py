@@ -598,3 +598,26 @@ def test_value_range_limit_of_the_fp16_verify_kernels_is_reported(lynx):
     with pytest.raises(lynx.LynxError, match="range"):
         lynx.check(c["ws"])
     lynx.check(c["ws"])                                   # the status word was cleared
+
+
+# ------------------------------------------------- the paper's own flow: BF16 pages + attention on them
+@pytest.mark.parametrize("G,n_q,lens,bt", [(4, 1, (4099, 37), 16), (8, 1, (2500, 0), 32), (4, 2, (777, 1), 16),
+                                           (1, 1, (300, 5000), 16), (2, 1, (70,), 48)])
+def test_bf16_pages_attention_matches_oracle(lynx, G, n_q, lens, bt):
+    # lynx_recombine writes the dequantised BF16 pages (bit-exact against the oracle's), lynx_bf16_attention
+    # attends on them: compared with the float64 oracle on the same pages
+    Hkv = 2
+    c = _case(lynx, 9000 + G + n_q, len(lens), Hkv, G, n_q, lens, bt, True, "lognormal_channels")
+    _, k_pages = lynx.recombine(c["K"], want_codes=False, want_bf16=True)
+    _, v_pages = lynx.recombine(c["V"], want_codes=False, want_bf16=True)
+    ok_pages, ov_pages = oracle.recombine(*c["kp"])[1], oracle.recombine(*c["vp"])[1]
+    assert np.array_equal(bf16_bits(k_pages), ok_pages) and np.array_equal(bf16_bits(v_pages), ov_pages)
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    for causal in (False, True):
+        got = lynx.bf16_attention(c["geo"], qd, k_pages, v_pages, td, ld, causal=causal)
+        ref = oracle.attention_bf16_pages(bf16_bits(c["q"]), ok_pages, ov_pages, c["table"].numpy(),
+                                          c["lens"].numpy(), causal=causal)
+        _close(got.cpu().numpy().astype(np.float64), ref, f"bf16 pages G={G} n_q={n_q} causal={causal}")
+    with pytest.raises(lynx.LynxError):        # more than 8 query columns
+        lynx.bf16_attention(c["geo"], torch.zeros(len(lens), 16, Hkv * G, 128, dtype=torch.bfloat16, device="cuda"),
+                            k_pages, v_pages, td, ld)

@@ -347,3 +347,43 @@ def test_anchor_state_is_a_worse_draft_than_full_state():
     nm = lambda o: np.mean(np.sum((o - ref) ** 2, -1) / np.sum(ref ** 2, -1))
     assert nm(oa[0, 0]) > 20 * nm(of[0, 0])
     assert nm(of[0, 0]) < 1e-2
+
+
+def test_attention_on_bf16_pages_equals_torch_sdpa_and_the_plane_oracle():
+    """oracle.attention_bf16_pages (the paper's dequantise-to-pages decode path) against torch's float64
+    scaled_dot_product_attention on the same rows (paged shuffled table, GQA, causal), and against the
+    plane oracle up to the BF16 rounding of the dequantised rows."""
+    import torch
+    rng = np.random.default_rng(5)
+    B, Hkv, G, n_q, bt, lens = 2, 2, 4, 3, 16, (50, 21)
+    nb = sum((l + bt - 1) // bt for l in lens)
+    x = rng.normal(0.0, 1.0, (2, nb, Hkv, bt, 128)).astype(np.float32)
+    kb, vb = (np.asarray(bf16_bits(f32_to_bf16_tensor(x[i]))) for i in range(2))
+    q = rng.normal(0.0, 1.0, (B, n_q, Hkv * G, 128)).astype(np.float32)
+    qb = np.asarray(bf16_bits(f32_to_bf16_tensor(q)))
+    perm = rng.permutation(nb).astype(np.int32)
+    table = np.zeros((B, 4), np.int32)
+    table[0, :4] = perm[:4]
+    table[1, :2] = perm[4:6]
+    lens_a = np.array(lens, np.int32)
+    # quantise, recombine to BF16 pages with the oracle, attend on the pages
+    kp, vp = oracle.split_quantize(kb), oracle.split_quantize(vb)
+    k_pages, v_pages = oracle.recombine(*kp)[1], oracle.recombine(*vp)[1]
+    for causal in (False, True):
+        got = oracle.attention_bf16_pages(qb, k_pages, v_pages, table, lens_a, causal=causal)
+        qf, kf, vf = (torch.from_numpy(bits_to_f64(a)) for a in (qb, k_pages, v_pages))
+        for b in range(B):
+            L = int(lens[b])
+            rows = lambda pages: pages[torch.from_numpy(table[b, :(L + bt - 1) // bt].astype(np.int64))].permute(1, 0, 2, 3).reshape(Hkv, -1, 128)[:, :L]
+            kk, vv = rows(kf), rows(vf)
+            mask = torch.ones(n_q, L, dtype=torch.bool)
+            if causal:
+                for j in range(n_q):
+                    mask[j, max(L - n_q + j + 1, 0):] = False
+            want = torch.nn.functional.scaled_dot_product_attention(
+                qf[b].permute(1, 0, 2)[None], kk[None], vv[None], attn_mask=mask, enable_gqa=True,
+                scale=float(np.float32(1.0 / np.sqrt(128.0))))[0].permute(1, 0, 2)   # (the scale crosses the C ABI as binary32)
+            assert np.allclose(got[b], want.numpy(), rtol=1e-9, atol=1e-12)
+        # the BF16 rounding of the pages (2^-9 relative per element) is the only difference from the plane oracle
+        ref = oracle.attention(True, qb, kp, vp, table, lens_a, Hkv, bt, causal=causal)
+        assert np.max(np.abs(got - ref)) < 0.05 and np.max(np.abs(got - ref)) > 0.0
