@@ -444,6 +444,7 @@ def main():
     if rank == 0 and world == 1:
         line["per_layer_launches"] = run_per_layer(wlk, peak)
         line["recombine"] = run_recombine(wlk, peak)
+        line["bf16_pages"] = run_bf16_pages(wlk, peak)
     if rank == 0 and world == 1 and not args.no_e2e:
         line["e2e"] = run_e2e(wlk, args.e2e_steps, step_bytes)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -455,6 +456,78 @@ def main():
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(line))
+
+
+def run_bf16_pages(wlk: "Workload", peak: float, max_layers: int = 8):
+    """Context: the decode path the paper describes (Section 4.2: dequantise to BF16 pages, the engine's
+    attention reads 256 bytes per row) against the fused call on the same full-precision state (136
+    bytes per row), one decode step (n_q = 1) on up to 8 layers of the workload: lynx_recombine of K
+    and V to pages, lynx_bf16_attention on them, lynx_merge_verify_attention with k = 1.  Not part of
+    `value`."""
+    lynx, wl = wlk.lynx, wlk.wl
+    layers = min(wl.layers, max_layers)
+    Bs = layers * wl.batch
+    nb = layers * wlk.nb_layer
+    dev = wlk.device
+
+    def first(pl):
+        return lynx.Planes(pl.anchor[:nb], pl.residual[:nb], pl.meta[:nb])
+    K, V = first(wlk.planes["K"]), first(wlk.planes["V"])
+    geo = lynx.Geometry(wl.num_q_heads, wl.num_kv_heads, wl.block_tokens, nb, wlk.table.shape[1])
+    table, lens = wlk.table[:Bs].contiguous(), wlk.lens_flat[:Bs].contiguous()
+    q = wlk.windows[0]["qs"][0][:Bs].contiguous()
+    ws = lynx.make_workspace(geo, Bs, 1, dev)
+    pages = {w: torch.empty(nb, wl.num_kv_heads, wl.block_tokens, 128, dtype=torch.bfloat16, device=dev) for w in "KV"}
+    import ctypes
+    wsb = torch.empty(int(lynx.load().lynx_bf16_workspace_bytes(ctypes.byref(geo._c()), Bs, 1)),
+                      dtype=torch.uint8, device=dev)
+    out_a = torch.empty(Bs, 1, wl.num_q_heads, 128, dtype=torch.float32, device=dev)
+    out_b = torch.empty_like(out_a)
+    lib = lynx.load()
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def recombine():
+        for w, pl in (("K", K), ("V", V)):
+            st = lib.lynx_recombine(pl.anchor.data_ptr(), pl.residual.data_ptr(), pl.meta.data_ptr(),
+                                    pl.anchor.numel() // 64, None, pages[w].data_ptr(), stream)
+            if st != 0:
+                raise RuntimeError(f"lynx_recombine: status {st}")
+
+    def bf16():
+        lynx.bf16_attention(geo, q, pages["K"], pages["V"], table, lens, workspace=wsb, out=out_b)
+
+    def fused():
+        lynx.merge_verify_attention(geo, q, K, V, table, lens, ws, causal=True, out_full=out_a)
+
+    def time_ms(fn, reps=5):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+    rows = 2 * wl.num_kv_heads * int(wlk.lens_flat_cpu[:Bs].sum())     # K rows + V rows the step attends to
+    rows_pool = 2 * nb * wl.num_kv_heads * wl.block_tokens
+    t_rec, t_bf, t_fu = time_ms(recombine), time_ms(bf16), time_ms(fused)
+    lynx.check(ws)
+    diff = float((out_a - out_b).abs().max())
+
+    def entry(ms, bytes_):
+        g = bytes_ / (ms * 1e-3) / 1e9
+        return {"ms": ms, "bytes": bytes_, "GBps": g, "frac_of_measured": g / peak}
+    return {"layers": layers, "rows": rows,
+            "recombine_to_pages": entry(t_rec, rows_pool * (136 + 256)),
+            "bf16_attention": entry(t_bf, rows * 256),
+            "fused_full_state_decode": entry(t_fu, rows * 136),
+            "roofline": {"bound": "hbm", "kernel": "bf16_attention", "achieved": rows * 256 / (t_bf * 1e-3) / 1e9,
+                         "peak": peak, "unit": "GB/s", "frac": rows * 256 / (t_bf * 1e-3) / 1e9 / peak},
+            "speedup_fused_vs_bf16_attention": t_bf / t_fu,
+            "speedup_fused_vs_recombine_plus_bf16_attention": (t_rec + t_bf) / t_fu,
+            "max_abs_difference_of_outputs": diff}
 
 
 def run_recombine(wlk: "Workload", peak: float, max_rows: int = 4 << 20):

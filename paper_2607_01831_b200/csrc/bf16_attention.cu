@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(kWarps * 32, COLS <= 4 ? 2 : 1) bf16_decode_ke
 
   // tokens of this warp: t_begin + warp * 256 + pass * TPP + grp
   const int w_begin = t_begin + warp * (kChunk / kWarps), w_end = min(t_end, w_begin + kChunk / kWarps);
-  constexpr int U = 2;                   // passes whose loads are issued together
+  constexpr int U = COLS <= 4 ? 4 : 2;   // passes whose loads are issued together
   for (int t00 = w_begin; t00 < w_end; t00 += U * TPP) {
     uint4 kxu[U][NV], vxu[U][NV];
     bool validu[U];
@@ -127,15 +127,24 @@ __global__ void __launch_bounds__(kWarps * 32, COLS <= 4 ? 2 : 1) bf16_decode_ke
     }
     // online softmax of the token group, O accumulation
     float pw[COLS];
+    bool grew = false;
+#pragma unroll
+    for (int c = 0; c < COLS; ++c) grew |= s[c] > m[c];
+    if (__any_sync(0xFFFFFFFFu, grew)) {   // the running maxima rise rarely: rescale only then
+#pragma unroll
+      for (int c = 0; c < COLS; ++c) {
+        const float mn = fmaxf(m[c], s[c]);
+        const float f = ex2f(m[c] - mn);
+        l[c] *= f;
+        m[c] = mn;
+#pragma unroll
+        for (int d = 0; d < DPL; ++d) o[c][d] *= f;
+      }
+    }
 #pragma unroll
     for (int c = 0; c < COLS; ++c) {
-      const float mn = fmaxf(m[c], s[c]);
-      const float f = ex2f(m[c] - mn);
-      pw[c] = ex2f(s[c] - mn);
-      l[c] = fmaf(l[c], f, pw[c]);
-      m[c] = mn;
-#pragma unroll
-      for (int d = 0; d < DPL; ++d) o[c][d] *= f;
+      pw[c] = ex2f(s[c] - m[c]);
+      l[c] += pw[c];
     }
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
