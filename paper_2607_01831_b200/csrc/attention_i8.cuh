@@ -75,11 +75,11 @@ struct I8Cfg {
   static constexpr int kPLayout = kPRow == 32 ? 6 : kPRow == 64 ? 4 : 2;   // descriptor swizzle mode of the P tile
   static constexpr int kTeamBytes = kTile + kPTile;      // V tile, P tile (the K levels live in tensor memory)
   static constexpr int kQTile = (kNQK * 128 + 1023) / 1024 * 1024;
-  static constexpr int kMail = CP * 128 * 4;             // end-of-piece deposit of a team: O in its V tile (l, zs, ref beside its scalars)
+  static constexpr int kMail = CP * 128 * 4;             // end-of-piece deposit of a team: O in its V tile, (l, zs, ref) in its P tile
   static_assert(kMail <= kTile, "the deposit lives in the team's V tile");
   static constexpr int kOffQT = kTeams * kTeamBytes;
   static constexpr int kOffRing = kOffQT + 2 * kQTile;
-  static constexpr int kTeamScal = (8 * CP + 4 * 2 * CP + 2 * CP + 3 * CP) * 4;   // qs, ref, factor, limits, maxima; reduce scratch; totals; deposit header
+  static constexpr int kTeamScal = (8 * CP + 4 * 2 * CP + 2 * CP) * 4;   // qs, ref, factor, limits, maxima; reduce scratch; totals
   static constexpr int kFixedTail = 2 * CP * 256 + kTeams * kTeamScal +
                                     8 * kI8PieceUnits * 4 + 2 * 32 + 64 * 8 + (1 + kTeams) * 256 + 64;
   static constexpr int kAvail = 227 * 1024 - 1024 - kOffRing - kFixedTail;
@@ -551,11 +551,11 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   float* amax_s = my_scal + 4 * CP;               // [team warps]
   float* my_red = my_scal + 8 * CP;               // [team warps][2 CG]
   float* my_lz = my_scal + 16 * CP;               // [2 CP]
-  float* my_hdr = my_scal + 18 * CP;              // [3 CP] l, zs, ref of this team's deposit
   const int tw = grp * 4 + w4;                    // warp of the team
   int* my_misc = misc + 64 * (1 + tm);
   const int bar_tm = 1 + tm;                      // named barrier of this team
   const uint32_t vtile = sbase + tm * C::kTeamBytes, ptile = vtile + C::kTile;
+  float* my_hdr = reinterpret_cast<float*>(smem + tm * C::kTeamBytes + C::kTile);   // [3 CP] l, zs, ref of this team's deposit (in its idle P tile)
   const uint32_t tm_k = tmem0 + tm * C::kTmTeam + C::kTmK;
   const int dim_out = 32 * (r >> 5) + 8 * ((r >> 2) & 3) + 2 * (r & 3) + ((r >> 4) & 1);   // head dim of lane r of O
   // this thread's row of the P tile: 16-byte chunk j goes to position j ^ p_swz
@@ -908,8 +908,8 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
       }
       named_bar(bar_tm, TT);
       if (!finisher) {
-        // deposit O in this team's V tile (idle: its last P.V is complete) and (l, zs, ref) beside its
-        // scalars, for the team that owns the piece's last unit
+        // deposit O in this team's V tile and (l, zs, ref) in its P tile (both idle: its last P.V is
+        // complete), for the team that owns the piece's last unit
         float* mail = reinterpret_cast<float*>(smem + tm * C::kTeamBytes);
 #pragma unroll
         for (int c = 0; c < CG; ++c) mail[(c0 + c) * 128 + r] = of[c];
@@ -933,7 +933,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           if (tt == 0) seq_wait(misc + 16 + d, (int)dep_cnt[d] + 1, abort_word);   // its deposit is complete
           named_bar(bar_tm, TT);
           const float* mo = reinterpret_cast<const float*>(smem + d * C::kTeamBytes);
-          const float* mh = reinterpret_cast<const float*>(smem + C::kOffScal + d * C::kTeamScal) + 18 * CP;
+          const float* mh = reinterpret_cast<const float*>(smem + d * C::kTeamBytes + C::kTile);
 #pragma unroll
           for (int c = 0; c < CG; ++c) {
             const float o2 = mo[(c0 + c) * 128 + r], l2 = mh[c0 + c];
