@@ -161,6 +161,25 @@ lynx_status lynx_anchor_attention_static(const lynx_shape* shape, const void* q_
                                          const int32_t* block_table, const int32_t* seq_lens,
                                          float softmax_scale, float* out, void* stream);
 
+/* The paper's own quantiser (Section 4.1, Algorithm 1 "Lynx Hierarchical Quantization"; inverse: the
+ * inverse alpha-law of its stage 3, eq. 4) as a second scheme beside the linear one above.
+ * src_bf16 : BF16 [n_pages][256][128]: pages of P = 256 consecutive tokens of one KV head (contiguous).
+ * Per channel: page minimum and range (gamma_min, gamma_scale: float [n_pages][128]); per chunk of
+ * C = 32 consecutive tokens its mean and largest deviation (mu, sigma: float [n_pages][8][128]);
+ * magnitudes companded with the alpha-law (alpha = 255) to integers 0..120, split into a 4-bit
+ * sign-aware two's-complement Anchor and a 4-bit centred Residual, packed two per byte like the linear
+ * planes (q_anc, q_res: uint8 [n_pages][256][64], byte j = channel 2j | channel 2j+1 << 4).
+ * Arithmetic is binary32; the readings of the algorithm's open points (alpha, epsilon = 1e-6, the scale
+ * 120, the sign taken from the centred value) are stated in the library's design notes.
+ * lynx_hier_dequantize reconstructs BF16 pages [n_pages][256][128] from both streams, or from the
+ * Anchor alone when q_res is NULL (the Residual, a centred correction, taken as zero); the pages can be
+ * attended to with lynx_bf16_attention (block_tokens = 256). */
+lynx_status lynx_hier_quantize(const void* src_bf16, int64_t n_pages, uint8_t* q_anc, uint8_t* q_res,
+                               float* gamma_min, float* gamma_scale, float* mu, float* sigma, void* stream);
+lynx_status lynx_hier_dequantize(const uint8_t* q_anc, const uint8_t* q_res, int64_t n_pages,
+                                 const float* gamma_min, const float* gamma_scale, const float* mu,
+                                 const float* sigma, void* dst_bf16, void* stream);
+
 /* Decode attention over dequantised BF16 pages: the path the paper itself describes (Section 4.2: the
  * dequantisation kernel scatters BF16 pages into the paged KV memory, the engine's attention reads
  * them; Section 2 attention equation), here as the baseline the fused calls above are measured

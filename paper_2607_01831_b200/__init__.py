@@ -38,7 +38,8 @@ class _Shape(ctypes.Structure):
 
 EXPORTS = ["lynx_split_quantize", "lynx_recombine", "lynx_workspace_bytes", "lynx_workspace_init",
            "lynx_anchor_attention", "lynx_merge_verify_attention", "lynx_anchor_attention_static",
-           "lynx_bf16_workspace_bytes", "lynx_bf16_attention", "lynx_check",
+           "lynx_bf16_workspace_bytes", "lynx_bf16_attention", "lynx_hier_quantize", "lynx_hier_dequantize",
+           "lynx_check",
            "lynx_status_string", "lynx_version"]
 
 
@@ -79,6 +80,10 @@ def load():
     lib.lynx_bf16_attention.argtypes = [ctypes.POINTER(_Shape), vp, i32, i32, i32, vp, vp, vp, vp, f32, vp, vp,
                                         ctypes.c_size_t, vp]
     lib.lynx_bf16_attention.restype = ctypes.c_int
+    lib.lynx_hier_quantize.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp]
+    lib.lynx_hier_quantize.restype = ctypes.c_int
+    lib.lynx_hier_dequantize.argtypes = [vp, vp, i64, vp, vp, vp, vp, vp, vp]
+    lib.lynx_hier_dequantize.restype = ctypes.c_int
     lib.lynx_check.argtypes = [vp, vp]
     lib.lynx_check.restype = ctypes.c_int
     lib.lynx_status_string.argtypes = [ctypes.c_int]
@@ -270,4 +275,39 @@ def bf16_attention(geo: Geometry, q: torch.Tensor, k_pages: torch.Tensor, v_page
     _ok(load().lynx_bf16_attention(ctypes.byref(geo._c()), _ptr(q), B, n_q, int(causal), _ptr(k_pages),
                                    _ptr(v_pages), _ptr(block_table), _ptr(seq_lens), softmax_scale, _ptr(out),
                                    _ptr(workspace), workspace.numel(), _stream()), "lynx_bf16_attention")
+    return out
+
+
+@dataclass
+class HierPlanes:
+    """Algorithm 1 output for pages of 256 tokens: packed nibbles and the per-channel metadata."""
+    q_anc: torch.Tensor        # u8 [n_pages][256][64]
+    q_res: torch.Tensor        # u8 [n_pages][256][64]
+    gamma_min: torch.Tensor    # f32 [n_pages][128]
+    gamma_scale: torch.Tensor  # f32 [n_pages][128]
+    mu: torch.Tensor           # f32 [n_pages][8][128]
+    sigma: torch.Tensor        # f32 [n_pages][8][128]
+
+
+def hier_quantize(src: torch.Tensor) -> HierPlanes:
+    """lynx_hier_quantize: src BF16 [n_pages][256][128] -> HierPlanes."""
+    if src.dtype != torch.bfloat16 or src.dim() != 3 or tuple(src.shape[1:]) != (256, D):
+        raise LynxError("src must be BF16 [n_pages][256][128]")
+    n, dev = src.shape[0], src.device
+    out = HierPlanes(torch.empty(n, 256, 64, dtype=torch.uint8, device=dev), torch.empty(n, 256, 64, dtype=torch.uint8, device=dev),
+                     torch.empty(n, D, dtype=torch.float32, device=dev), torch.empty(n, D, dtype=torch.float32, device=dev),
+                     torch.empty(n, 8, D, dtype=torch.float32, device=dev), torch.empty(n, 8, D, dtype=torch.float32, device=dev))
+    _ok(load().lynx_hier_quantize(_ptr(src), n, _ptr(out.q_anc), _ptr(out.q_res), _ptr(out.gamma_min),
+                                  _ptr(out.gamma_scale), _ptr(out.mu), _ptr(out.sigma), _stream()), "lynx_hier_quantize")
+    return out
+
+
+def hier_dequantize(h: HierPlanes, anchor_only: bool = False, out: torch.Tensor | None = None) -> torch.Tensor:
+    """lynx_hier_dequantize -> BF16 [n_pages][256][128] (from the Anchor stream alone if asked)."""
+    n = h.q_anc.shape[0]
+    if out is None:
+        out = torch.empty(n, 256, D, dtype=torch.bfloat16, device=h.q_anc.device)
+    _ok(load().lynx_hier_dequantize(_ptr(h.q_anc), None if anchor_only else _ptr(h.q_res), n, _ptr(h.gamma_min),
+                                    _ptr(h.gamma_scale), _ptr(h.mu), _ptr(h.sigma), _ptr(out), _stream()),
+        "lynx_hier_dequantize")
     return out
