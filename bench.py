@@ -445,6 +445,8 @@ def main():
         line["per_layer_launches"] = run_per_layer(wlk, peak)
         line["recombine"] = run_recombine(wlk, peak)
         line["bf16_pages"] = run_bf16_pages(wlk, peak)
+        line["hierarchical"] = run_hier(wlk, peak)
+        line["progressive"] = run_progressive(wlk)
     if rank == 0 and world == 1 and not args.no_e2e:
         line["e2e"] = run_e2e(wlk, args.e2e_steps, step_bytes)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -456,6 +458,127 @@ def main():
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(line))
+
+
+def run_progressive(wlk: "Workload", max_layers: int = 8, cap: int = 64, k: int = 4):
+    """Context: progressive arrival (Section 4.2, Residual Phase; Section 4.2 "Speculative Decoder").  The
+    Anchor planes of up to 8 layers are resident; their Residual planes arrive from pinned host memory on
+    a second stream, layer by layer (the stand-in for the NIC queue of lower priority), while the decoder
+    drafts on the Anchor state: one anchor decode step over all layers per token, the host polling the
+    Residual's arrival before each next token as the paper's decoder does, up to `cap` drafts.  When the
+    Residual is in, one merge-verify pass checks the last k drafted positions.  Reported against the same
+    work done one after the other.  Not part of `value`."""
+    lynx, wl, dev = wlk.lynx, wlk.wl, wlk.device
+    layers = min(wl.layers, max_layers)
+    Bs, nb = layers * wl.batch, layers * wlk.nb_layer
+    K, V = wlk.planes["K"], wlk.planes["V"]
+    host = {w: pl.residual[:nb].cpu().pin_memory() for w, pl in (("K", K), ("V", V))}
+    late = {w: torch.zeros_like(pl.residual[:nb]) for w, pl in (("K", K), ("V", V))}     # where the Residual lands
+    Ka, Va = (lynx.Planes(pl.anchor[:nb], late[w], pl.meta[:nb]) for w, pl in (("K", K), ("V", V)))
+    geo = lynx.Geometry(wl.num_q_heads, wl.num_kv_heads, wl.block_tokens, nb, wlk.table.shape[1])
+    table = wlk.table[:Bs].contiguous()
+    lens_full = wlk.lens_flat[:Bs].contiguous()
+    win = next(w for w in wlk.windows if w["k"] == k) if any(w["k"] == k for w in wlk.windows) else wlk.windows[0]
+    k = win["k"]
+    q1 = win["qs"][0][:Bs].contiguous()
+    qk = win["q"][:Bs].contiguous()
+    ws1, wsk = lynx.make_workspace(geo, Bs, 1, dev), lynx.make_workspace(geo, Bs, k, dev)
+    out1 = torch.empty(Bs, 1, wl.num_q_heads, 128, dtype=torch.float32, device=dev)
+    draft = torch.zeros(Bs, k, wl.num_q_heads, 128, dtype=torch.float32, device=dev)
+    outk = torch.empty_like(draft)
+    fr = torch.empty(Bs, dtype=torch.int32, device=dev)
+    dv = torch.empty(Bs, k, dtype=torch.float32, device=dev)
+    step_lens = [(lens_full - cap + j + 1).contiguous() for j in range(cap)]
+    copy_stream = torch.cuda.Stream(device=dev)
+    per_layer = wlk.nb_layer
+
+    def transfer():
+        with torch.cuda.stream(copy_stream):
+            for l in range(layers):
+                sl = slice(l * per_layer, (l + 1) * per_layer)
+                for w in "KV":
+                    late[w][sl].copy_(host[w][sl], non_blocking=True)
+            ev = torch.cuda.Event()
+            ev.record(copy_stream)
+        return ev
+
+    def anchor_step(j):
+        lynx.anchor_attention(geo, q1, Ka, Va, table, step_lens[j], ws1, out=out1)
+
+    def verify():
+        lynx.merge_verify_attention(geo, qk, Ka, Va, table, lens_full, wsk, draft_out=draft, atol=0.5, rtol=0.1,
+                                    causal=True, out_full=outk, first_reject=fr, dev=dv)
+    import time
+    for _ in range(2):          # warm-up of every piece
+        transfer().synchronize(); anchor_step(0); verify(); torch.cuda.synchronize()
+    t0 = time.perf_counter(); transfer().synchronize(); t_h2d = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    for j in range(8):
+        anchor_step(j); torch.cuda.synchronize()
+    t_step = (time.perf_counter() - t0) / 8
+    t0 = time.perf_counter(); verify(); torch.cuda.synchronize(); t_ver = time.perf_counter() - t0
+    # overlapped: drafts run while the Residual arrives
+    for w in "KV":
+        late[w].zero_()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    ev = transfer()
+    n = 0
+    while n < cap and not ev.query():
+        anchor_step(n); torch.cuda.current_stream().synchronize()     # (a decoder needs the token before the next step)
+        n += 1
+    t_draft_end = time.perf_counter() - t0
+    ev.synchronize()
+    verify(); torch.cuda.synchronize()
+    t_total = time.perf_counter() - t0
+    lynx.check(wsk); lynx.check(ws1)
+    ok = bool(torch.equal(late["K"], K.residual[:nb]) and torch.equal(late["V"], V.residual[:nb]))
+    serial = t_h2d + n * t_step + t_ver
+    return {"layers": layers, "residual_bytes": int(2 * late["K"].numel()), "h2d_alone_ms": t_h2d * 1e3,
+            "anchor_step_ms": t_step * 1e3, "verify_ms": t_ver * 1e3, "drafts_while_waiting": n, "draft_cap": cap,
+            "drafting_ended_ms": t_draft_end * 1e3, "overlapped_total_ms": t_total * 1e3, "one_after_the_other_ms": serial * 1e3,
+            "transfer_hidden_frac": min(1.0, n * t_step / t_h2d) if t_h2d > 0 else None,
+            "residual_arrived_intact": ok, "timing": "host wall clock around synchronised steps (context only)"}
+
+
+def run_hier(wlk: "Workload", peak: float, max_pages: int = 16384):
+    """Context: the paper's own quantiser (Algorithm 1) and its inverse on the first rows of the BF16
+    K source viewed as pages of 256 tokens (1 GiB at most).  Not part of `value`."""
+    lynx = wlk.lynx
+    src = wlk.src["K"].view(-1, 128)
+    n = min(src.shape[0] // 256, max_pages)
+    x = src[: n * 256].view(n, 256, 128)
+    h = lynx.hier_quantize(x)
+    out = torch.empty(n, 256, 128, dtype=torch.bfloat16, device=wlk.device)
+
+    def time_ms(fn, reps=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+    lib, stream = lynx.load(), torch.cuda.current_stream().cuda_stream
+
+    def quant():
+        st = lib.lynx_hier_quantize(x.data_ptr(), n, h.q_anc.data_ptr(), h.q_res.data_ptr(), h.gamma_min.data_ptr(),
+                                    h.gamma_scale.data_ptr(), h.mu.data_ptr(), h.sigma.data_ptr(), stream)
+        if st != 0:
+            raise RuntimeError(f"lynx_hier_quantize: status {st}")
+    res = {"pages": n}
+    meta = (2 * 128 + 2 * 8 * 128) * 4
+    for name, fn, bytes_pp in (("quantize", quant, 256 * 256 + 2 * 256 * 64 + meta),
+                               ("dequantize", lambda: lynx.hier_dequantize(h, out=out), 2 * 256 * 64 + meta + 256 * 256),
+                               ("dequantize_anchor_only", lambda: lynx.hier_dequantize(h, anchor_only=True, out=out),
+                                256 * 64 + meta + 256 * 256)):
+        ms = time_ms(fn)
+        g = n * bytes_pp / (ms * 1e-3) / 1e9
+        res[name] = {"ms": ms, "bytes_per_page": bytes_pp, "GBps": g, "frac_of_measured": g / peak}
+    return res
 
 
 def run_bf16_pages(wlk: "Workload", peak: float, max_layers: int = 8):
