@@ -273,7 +273,7 @@ def oracle_sample(cfg_id: int, k_list=None):
 # (dram__bytes_read.sum + dram__bytes_write.sum over 72 / 136 / 392 B per row; captures on an
 # 8-layer copy of config 3, summarised under profiles/).  Traffic grows in proportion to the
 # rows a launch processes, so a full launch is scaled by the rows.
-TRAFFIC_RATIO = {"anchor_attention": 1.005, "merge_verify_attention": 1.003, "split_quantize": 0.990}
+TRAFFIC_RATIO = {"anchor_attention": 1.016, "merge_verify_attention": 1.004, "split_quantize": 0.990}
 
 
 def base_kind(kind: str) -> str:
@@ -348,6 +348,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-context", action="store_true", help="skip the context measurements after the timed steps")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "lynx" else args.warmup
     if args.impl == "reference":
@@ -422,14 +423,14 @@ def main():
             "peak_source": "measured copy rate (MEASURED_PEAKS.json hbm_gbs)" if peak_kind == "measured"
             else "fallback 6.65 TB/s (MEASURED_PEAKS.json absent)",
             "traffic": launch_bytes[dom] * TRAFFIC_RATIO[dom],
-            "traffic_source": "ncu dram__bytes_read+write on an 8-layer copy of config 3, scaled by rows",
+            "traffic_source": "ncu dram__bytes_read+write on a 6-layer copy of config 3, scaled by rows",
             "algorithmic_bytes_per_launch": launch_bytes[dom], "share_of_step": share[dom],
             "launches": len(dom_ts), "avg_launch_ms": sum(dom_ts) / len(dom_ts)}
 
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "u8 x s8 -> s32 (Q.K^T; f16 on tcgen05), f16 x f16 -> f32 (P.V), f32 softmax and quantiser",
+        "vs_baseline": None, "dtype": "u8 x s8 -> s32 (Q.K^T) and u8 x u8 -> s32 (P.V) on tcgen05 kind::i8; f16 -> f32 on tcgen05 for verify with 17..64 columns; f32 softmax and quantiser",
         "data": "synthetic",
         "config": {"workload": wl.name, "layers": wl.layers, "batch": wl.batch, "context": wl.context,
                    "num_kv_heads": wl.num_kv_heads, "num_q_heads": wl.num_q_heads, "k": list(wl.k_list),
@@ -441,7 +442,7 @@ def main():
         "kernels": kernels, "roofline": roof, "clocks": clocks,
     }
 
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.no_context:
         line["per_layer_launches"] = run_per_layer(wlk, peak)
         line["recombine"] = run_recombine(wlk, peak)
         line["bf16_pages"] = run_bf16_pages(wlk, peak)
