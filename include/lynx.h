@@ -105,11 +105,12 @@ lynx_status lynx_recombine(const uint8_t* anchor, const uint8_t* residual, const
  * Returns 0 for an unsupported shape.  The workspace must be zero-filled once before its first
  * use (lynx_workspace_init, or cudaMemsetAsync of the whole buffer); each call leaves it ready
  * for the next.  Calls sharing a workspace must be ordered on one stream.
- * The figure includes 10 to 20 MB for FP32 copies of the kernels' accumulators, into which long
- * accumulation chains are cut (what the tensor cores lose by truncating when they accumulate is
- * then bounded whatever the context length).  A call given less than the full figure, but enough
- * for the rest, runs without that cut: fine for value rows with a modest range, up to a few 1e-3
- * of absolute error for rows whose range is in the hundreds and contexts of 100k tokens. */
+ * A buffer smaller than this figure is rejected by the attention calls (LYNX_ERR_WORKSPACE): nothing
+ * degrades silently.  For verification with more than 16 columns (k * Hq/Hkv in 17..64) the figure
+ * includes about 19 MB for FP32 copies of the accumulators of the FP16 tensor-core kernels used there
+ * (their accumulation chains are cut every 256 units of 64 tokens, which bounds what the tensor
+ * cores lose by truncating when they accumulate, whatever the context length).  Anchor attention and
+ * verification with up to 16 columns run on exact integer tensor-core products and need no such copies. */
 size_t lynx_workspace_bytes(const lynx_shape* shape, int32_t batch, int32_t n_cols_q);
 lynx_status lynx_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
@@ -118,7 +119,9 @@ lynx_status lynx_workspace_init(void* workspace, size_t workspace_bytes, void* s
  * Query j of sequence b attends tokens [0, seq_lens[b]) (causal == 0) or
  * [0, seq_lens[b] - n_q + j + 1) (causal != 0); a query that sees no token gets zeros.
  * softmax_scale 0 means 1/sqrt(128).  out : [batch][n_q][Hq][128] float.
- * n_q * (Hq/Hkv) must be <= 64.  seq_lens[b] is clamped to the table's capacity. */
+ * n_q must be <= 16 and n_q * (Hq/Hkv) <= 64.  seq_lens[b] is clamped to the table's capacity.
+ * Value rows of any finite scale are handled (the weights are fixed-point numbers relative to a
+ * per-column reference exponent). */
 lynx_status lynx_anchor_attention(const lynx_shape* shape, const void* q_bf16, int32_t batch,
                                   int32_t n_q, int32_t causal, lynx_plane K, lynx_plane V,
                                   const int32_t* block_table, const int32_t* seq_lens,
@@ -131,7 +134,11 @@ lynx_status lynx_anchor_attention(const lynx_shape* shape, const void* q_bf16, i
  * and first_reject[b] = smallest j with dev[b][j] > 1, or k if none (the longest agreeing
  * prefix; out_full at that position is the correction).
  * draft_out : [batch][k][Hq][128] float, the Anchor-state results being verified; may be NULL,
- * then dev / first_reject are not written (and may be NULL).  out_full : same shape, float. */
+ * then dev / first_reject are not written (and may be NULL).  out_full : same shape, float.
+ * k must be <= 16 and k * (Hq/Hkv) <= 64.  With 17..64 columns the weights are FP16 numbers: a value
+ * row whose scale reaches 16 (a range of 4080 or more) would overflow them; such rows are recorded
+ * in the status word and lynx_check returns LYNX_ERR_RANGE (the outputs of that call are then not
+ * to be used).  Up to 16 columns there is no such limit. */
 lynx_status lynx_merge_verify_attention(const lynx_shape* shape, const void* q_bf16,
                                         int32_t batch, int32_t k, int32_t causal, lynx_plane K,
                                         lynx_plane V, const int32_t* block_table,
@@ -147,8 +154,8 @@ lynx_status lynx_merge_verify_attention(const lynx_shape* shape, const void* q_b
  * captured).  Same computation, arguments and result as lynx_anchor_attention, but the scratch
  * memory is a fixed 8 MiB array inside the library image (every GPU that loads the library
  * holds it until the process exits); the call itself allocates nothing.
- *  - Problems whose scratch need (lynx_workspace_bytes less the accumulator copies, which this
- *    call does without) exceeds 8 MiB are rejected with LYNX_ERR_WORKSPACE and nothing is launched.
+ *  - Problems whose scratch need (lynx_workspace_bytes for the same shape) exceeds 8 MiB are rejected
+ *    with LYNX_ERR_WORKSPACE; nothing is launched and the array is not touched.
  *  - The first call on each device looks up the array's device address (a one-time set-up,
  *    done with that device current); make that first call before any stream capture begins.
  *  - All calls share the one array.  Each call clears the words that must start at zero, on

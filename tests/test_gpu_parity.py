@@ -600,6 +600,22 @@ def test_value_range_limit_of_the_fp16_verify_kernels_is_reported(lynx):
     lynx.check(c["ws"])                                   # the status word was cleared
 
 
+def test_status_word_bits_map_to_their_statuses(lynx):
+    # what a kernel records when a bounded wait runs out (or a block id / value range is bad) is one bit
+    # of the workspace's status word; no wait is made to run out on the GPU here: the bits are written
+    # from the host and lynx_check must report, in order of severity, and clear them
+    c = _case(lynx, 8500, 1, 2, 4, 1, (100,), 16, True, "normal")
+    word = c["ws"][:4].view(torch.int32)
+    for bits, name in ((2, "status 8"), (1, "status 7"), (4, "status 9"), (7, "status 8"), (5, "status 7")):
+        word.fill_(bits)
+        with pytest.raises(lynx.LynxError, match=name):
+            lynx.check(c["ws"])
+        lynx.check(c["ws"])                                   # cleared by the report
+    out = lynx.anchor_attention(c["geo"], c["q"].cuda(), c["K"], c["V"], c["table"].cuda(), c["lens"].cuda(), c["ws"])
+    lynx.check(c["ws"])                                       # and the workspace is still usable
+    assert bool(torch.isfinite(out).all())
+
+
 # ------------------------------------------------- the paper's own flow: BF16 pages + attention on them
 @pytest.mark.parametrize("G,n_q,lens,bt", [(4, 1, (4099, 37), 16), (8, 1, (2500, 0), 32), (4, 2, (777, 1), 16),
                                            (1, 1, (300, 5000), 16), (2, 1, (70,), 48)])
