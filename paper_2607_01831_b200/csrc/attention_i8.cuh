@@ -157,6 +157,40 @@ __device__ __forceinline__ float rcp_approx(float x) {
   asm("rcp.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float ex2_ftz(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Packed pairs of FP32 values (one 64-bit register pair, one instruction per pair of operations)
+__device__ __forceinline__ uint64_t f2_pack(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ float ex2_full(float x) {   // no flush of small results
   float y;
   asm("ex2.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -477,7 +511,10 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   uint32_t* blk_s = reinterpret_cast<uint32_t*>(smem + C::kOffBlk);
   Item* items = reinterpret_cast<Item*>(smem + C::kOffItems);
   int* misc = reinterpret_cast<int*>(smem + C::kOffMisc);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31;
+  // (broadcast from lane 0 so that the compiler knows the warp index, and all that follows from it -- team, tiles,
+  // operand descriptors -- to be the same for every lane: such values can live in uniform registers)
+  const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);
   const uint32_t ring_u32 = sbase + C::kOffRing;
   const uint32_t full0 = sbase + C::kOffBars, empty0 = full0 + NSTAGE * 8;
   const uint32_t qfull0 = empty0 + NSTAGE * 8, qempty0 = qfull0 + 16;
@@ -509,6 +546,8 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   for (int i = tid; i < 2 * CP * 256 / 16; i += C::kThreads) reinterpret_cast<uint4*>(qraw)[i] = make_uint4(0, 0, 0, 0);
   for (int i = tid; i < 2 * C::kQTile / 16; i += C::kThreads)
     reinterpret_cast<uint4*>(smem + C::kOffQT)[i] = make_uint4(0, 0, 0, 0);
+  // the teams' scalars (the reference exponents must be finite numbers before their first use)
+  for (int i = tid; i < T * C::kTeamScal / 4; i += C::kThreads) reinterpret_cast<float*>(smem + C::kOffScal)[i] = 0.0f;
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
 
@@ -549,6 +588,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   float* qs_s = my_scal, *ref_s = my_scal + CP, *fac_s = my_scal + 2 * CP;
   int* lim_s = reinterpret_cast<int*>(my_scal + 3 * CP);
   float* amax_s = my_scal + 4 * CP;               // [team warps]
+  const float* zero_s = my_scal + 5 * CP;         // [CP] zeros (never written after the set-up)
   float* my_red = my_scal + 8 * CP;               // [team warps][2 CG]
   float* my_lz = my_scal + 16 * CP;               // [2 CP]
   const int tw = grp * 4 + w4;                    // warp of the team
@@ -653,10 +693,10 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         if (lane == 0) mbar_arrive(qready0 + qi * 8);
       }
 
-      float l[CG], zs[CG];
+      uint64_t l2[CG / 2], zs2[CG / 2];   // softmax sums, two columns per register pair
       float of_r[C::kOfInTmem ? 1 : CG];   // FP32 copy of O where tensor memory has no room for it
 #pragma unroll
-      for (int c = 0; c < CG; ++c) { l[c] = 0.0f; zs[c] = 0.0f; }
+      for (int c = 0; c < CG / 2; ++c) { l2[c] = 0ull; zs2[c] = 0ull; }
       bool fresh = true, have_of = false;
       int units_in_acc = 0;
       uint32_t n_own = (uint32_t)((gs_base + u_first) / T);   // index of the unit among this team's units
@@ -794,32 +834,52 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         // ---- scores of this thread's token -------------------------------------------------------
         mbar_wait(sfull0 + tm * 8, n_own & 1, abort_word);
         tc_fence_after();
-        float x[CG];
+        // y = log2 of the weight relative to the column's reference exponent, two columns per register pair
+        uint64_t y2[CG / 2];
         {
           uint32_t s0[CG], s1[CG], s2[CG];
           TmemRegs<CG>::ld(tm_s, s0);
           TmemRegs<CG>::ld(tm_s + CP, s1);
           TmemRegs<CG>::ld(tm_s + 2 * CP, s2);
           tc_wait_ld();
+          const uint64_t al2 = f2_pack(al, al), be2 = f2_pack(be, be), lsv2 = f2_pack(lsv, lsv);
+          const uint64_t k256 = f2_pack(256.0f, 256.0f);
+          const float* ref_r = fresh ? zero_s : ref_s;   // (a piece's first unit: relative to zero)
 #pragma unroll
-          for (int c = 0; c < CG; ++c) {
-            const float sf = fmaf((float)((int)s2[c] * 256 + (int)s1[c]), 256.0f, (float)(int)s0[c]);
-            x[c] = fmaf(sf, al, fmaf(be, qs_s[c0 + c], lsv));
+          for (int c = 0; c < CG / 2; ++c) {
+            const uint64_t hi = f2_pack((float)((int)s2[2 * c] * 256 + (int)s1[2 * c]),
+                                        (float)((int)s2[2 * c + 1] * 256 + (int)s1[2 * c + 1]));
+            const uint64_t lo = f2_pack((float)(int)s0[2 * c], (float)(int)s0[2 * c + 1]);
+            const uint64_t qs2 = *reinterpret_cast<const uint64_t*>(qs_s + c0 + 2 * c);
+            const uint64_t rf2 = *reinterpret_cast<const uint64_t*>(ref_r + c0 + 2 * c);
+            y2[c] = f2_fma(f2_fma(hi, k256, lo), al2, f2_fma(be2, qs2, f2_sub(lsv2, rf2)));
           }
         }
         if (unit_t0 + C::kST > full_lim) {
 #pragma unroll
-          for (int c = 0; c < CG; ++c)
-            if (tok >= lim_s[c0 + c]) x[c] = -INFINITY;
+          for (int c = 0; c < CG / 2; ++c) {
+            float a, b;
+            f2_unpack(y2[c], a, b);
+            if (tok >= lim_s[c0 + 2 * c]) a = -INFINITY;
+            if (tok >= lim_s[c0 + 2 * c + 1]) b = -INFINITY;
+            y2[c] = f2_pack(a, b);
+          }
         }
         // ---- reference exponents: raised when a weight would leave the u32 range -----------------------
-        bool need = fresh || units_in_acc >= C::kDrainUnits;
+        float ymax = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < CG; ++c) need |= x[c] - ref_s[c0 + c] > 31.5f;
+        for (int c = 0; c < CG / 2; ++c) {
+          float a, b;
+          f2_unpack(y2[c], a, b);
+          ymax = max3(ymax, a, b);
+        }
+        const bool need = fresh || units_in_acc >= C::kDrainUnits || ymax > 31.5f;
         if (bar_or(bar_tm, TT, need)) {   // (team-wide: one P.V covers all columns, so they all restart together)
 #pragma unroll
-          for (int c = 0; c < CG; ++c) {
-            float mx = x[c];
+          for (int c = 0; c < CG; ++c) {   // (rare path: back to absolute exponents x = y + ref)
+            float a, b;
+            f2_unpack(y2[c >> 1], a, b);
+            float mx = ((c & 1) ? b : a) + (fresh ? 0.0f : ref_s[c0 + c]);
 #pragma unroll
             for (int off = 16; off >= 1; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
             if (lane == 0) my_red[tw * CG + c] = mx;
@@ -828,27 +888,42 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           if (tt < CP) {
             const float* mr = my_red + (tt / CG) * 4 * CG + (tt % CG);   // the four warps of the column's group
             const float mx = fmaxf(fmaxf(mr[0], mr[CG]), fmaxf(mr[2 * CG], mr[3 * CG]));
-            const float old = ref_s[tt];
+            const float old = fresh ? 0.0f : ref_s[tt];
             float nw = old, f = 1.0f;
             if (fresh) { nw = fmaxf(mx, -1.0e4f) - 28.0f; f = 0.0f; }
             else if (mx - old > 31.5f) { nw = mx - 28.0f; f = ex2_full(old - nw); }
             ref_s[tt] = nw;
             fac_s[tt] = f;
+            my_red[C::kTeamWarps * CG + tt] = nw - old;   // what the change takes off every exponent of the column
           }
           named_bar(bar_tm, TT);
 #pragma unroll
-          for (int c = 0; c < CG; ++c) { l[c] *= fac_s[c0 + c]; zs[c] *= fac_s[c0 + c]; }
+          for (int c = 0; c < CG / 2; ++c) {
+            const uint64_t f2 = *reinterpret_cast<const uint64_t*>(fac_s + c0 + 2 * c);
+            l2[c] = f2_mul(l2[c], f2);
+            zs2[c] = f2_mul(zs2[c], f2);
+            // the exponents again, relative to the new references
+            const uint64_t od = *reinterpret_cast<const uint64_t*>(my_red + C::kTeamWarps * CG + c0 + 2 * c);
+            y2[c] = f2_sub(y2[c], od);
+          }
           drain(true);   // (the team's previous P.V has been waited for)
           fresh = false;
         }
         // ---- weights ------------------------------------------------------------------------------
         uint32_t wi[CG];
+        {
+          const uint64_t ia2 = f2_pack(ia, ia), ib2 = f2_pack(ib, ib);
 #pragma unroll
-        for (int c = 0; c < CG; ++c) {
-          const float wf = ex2_full(x[c] - ref_s[c0 + c]);
-          asm("cvt.rni.u32.f32 %0, %1;" : "=r"(wi[c]) : "f"(wf));
-          l[c] = fmaf(wf, ia, l[c]);
-          zs[c] = fmaf(wf, ib, zs[c]);
+          for (int c = 0; c < CG / 2; ++c) {
+            float a, b;
+            f2_unpack(y2[c], a, b);
+            const float wa = ex2_ftz(a), wb = ex2_ftz(b);
+            asm("cvt.rni.u32.f32 %0, %1;" : "=r"(wi[2 * c]) : "f"(wa));
+            asm("cvt.rni.u32.f32 %0, %1;" : "=r"(wi[2 * c + 1]) : "f"(wb));
+            const uint64_t w2 = f2_pack(wa, wb);
+            l2[c] = f2_fma(w2, ia2, l2[c]);
+            zs2[c] = f2_fma(w2, ib2, zs2[c]);
+          }
         }
 #pragma unroll
         for (int j = 0; j < CG / 4; ++j)
@@ -892,7 +967,14 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
       // totals of l and zs over the 128 token lanes of every column group
 #pragma unroll
       for (int c = 0; c < CG; ++c) {
-        float a = l[c], b = zs[c];
+        float a, b;
+        {
+          float l_lo, l_hi, z_lo, z_hi;
+          f2_unpack(l2[c >> 1], l_lo, l_hi);
+          f2_unpack(zs2[c >> 1], z_lo, z_hi);
+          a = (c & 1) ? l_hi : l_lo;
+          b = (c & 1) ? z_hi : z_lo;
+        }
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) {
           a += __shfl_xor_sync(0xFFFFFFFFu, a, off);
