@@ -351,6 +351,83 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
   }
 }
 
+
+// The stream-K cut of the work list (units of ST tokens in (sequence, KV head, position) order) for
+// CTA `cta` of `n_cta`, derived by one warp from the sequence lengths on the device.  Normally every
+// CTA takes q = ceil(total / n_cta) consecutive units, wherever the (sequence, head) boundaries fall.
+// When all sequences have the same number of units U and the B * Hkv segments are few enough to give
+// each of them c >= 1 CTAs of its own (one layer of a long context per launch), the cut is aligned
+// instead: q = ceil(U / c), and CTA i takes part i % c of segment i / c.  No CTA then pays for the
+// end of one piece and the start of another, at the cost of n_cta - c * segments idle CTAs (accepted
+// up to 15 %).  lo, hi index a list in which every segment occupies c * q entries, so that the
+// contributors of a segment and their partial slots follow from lo and q as in the plain cut.
+struct SkRange {
+  long long q, lo, hi, off_lo;   // off_lo: offset of `lo` among the Hkv * U units of sequence b_lo
+  int b_lo;
+};
+template <int ST, class ClampLen>
+__device__ __forceinline__ SkRange sk_range(const AttnParams& p, int n_cta, int cta, int lane, ClampLen clamp_len) {
+  SkRange r;
+  long long tot = 0;
+  int umin = 0x7FFFFFFF, umax = 0;
+  for (int b = lane; b < p.B; b += 32) {
+    const int u = (clamp_len(b) + ST - 1) / ST;
+    tot += u;
+    umin = min(umin, u);
+    umax = max(umax, u);
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    tot += __shfl_xor_sync(0xFFFFFFFFu, tot, off);
+    umin = min(umin, __shfl_xor_sync(0xFFFFFFFFu, umin, off));
+    umax = max(umax, __shfl_xor_sync(0xFFFFFFFFu, umax, off));
+  }
+  const long long T = tot * p.Hkv;
+  const long long segs = (long long)p.B * p.Hkv;
+  if (umin == umax && umax > 0 && segs <= n_cta && (n_cta / segs) * segs * 100 >= 85LL * n_cta) {
+    const int c = (int)(n_cta / segs), U = umax;
+    r.q = (U + c - 1) / c;
+    const int s = cta / c, part = cta % c;
+    r.lo = r.hi = 0; r.b_lo = 0; r.off_lo = 0;
+    if (s < segs && (long long)part * r.q < U) {
+      r.b_lo = s / p.Hkv;
+      r.off_lo = (long long)(s % p.Hkv) * U + (long long)part * r.q;
+      r.lo = ((long long)s * c + part) * r.q;
+      r.hi = r.lo + min(r.q, (long long)U - (long long)part * r.q);
+    }
+    return r;
+  }
+  r.q = (T + n_cta - 1) / n_cta;
+  r.lo = (long long)cta * r.q;
+  r.hi = (r.lo + r.q < T) ? r.lo + r.q : T;
+  r.b_lo = 0;
+  r.off_lo = 0;
+  if (r.lo < r.hi) {
+    long long running = 0;
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+      const int b = b0 + lane;
+      const long long u = b < p.B ? (long long)p.Hkv * ((clamp_len(b) + ST - 1) / ST) : 0;
+      long long incl = u;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const long long v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      const long long excl = running + incl - u;
+      const bool hit = u > 0 && r.lo >= excl && r.lo < excl + u;
+      const unsigned mk = __ballot_sync(0xFFFFFFFFu, hit);
+      if (mk) {
+        const int src = __ffs(mk) - 1;
+        r.b_lo = b0 + src;
+        r.off_lo = r.lo - __shfl_sync(0xFFFFFFFFu, excl, src);
+        break;
+      }
+      running += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+  }
+  return r;
+}
+
 #include "attention_wide.cuh"
 #include "attention_i8.cuh"
 

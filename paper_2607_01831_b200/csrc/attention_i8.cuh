@@ -296,38 +296,9 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
     int len = __ldg(p.seq_lens + b);
     return len < 0 ? 0 : (len > cap ? cap : len);
   };
-  long long tot = 0;
-  for (int b = lane; b < p.B; b += 32) tot += (clamp_len(b) + ST - 1) / ST;
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) tot += __shfl_xor_sync(0xFFFFFFFFu, tot, off);
-  const long long T = tot * p.Hkv;
-  const long long q = (T + n_cta - 1) / n_cta;
-  const long long lo = (long long)cta * q, hi = (lo + q < T) ? lo + q : T;
-  int b_lo = 0;
-  long long off_lo = 0;
-  if (lo < hi) {
-    long long running = 0;
-    for (int b0 = 0; b0 < p.B; b0 += 32) {
-      const int b = b0 + lane;
-      const long long u = b < p.B ? (long long)p.Hkv * ((clamp_len(b) + ST - 1) / ST) : 0;
-      long long incl = u;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const long long v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += v;
-      }
-      const long long excl = running + incl - u;
-      const bool hit = u > 0 && lo >= excl && lo < excl + u;
-      const unsigned mk = __ballot_sync(0xFFFFFFFFu, hit);
-      if (mk) {
-        const int src = __ffs(mk) - 1;
-        b_lo = b0 + src;
-        off_lo = lo - __shfl_sync(0xFFFFFFFFu, excl, src);
-        break;
-      }
-      running += __shfl_sync(0xFFFFFFFFu, incl, 31);
-    }
-  }
+  const SkRange rng = sk_range<ST>(p, n_cta, cta, lane, clamp_len);
+  const long long q = rng.q, lo = rng.lo, hi = rng.hi, off_lo = rng.off_lo;
+  const int b_lo = rng.b_lo;
   if (pw == 0) {
     if (lane == 0) misc[7] = lo < hi ? (int)(hi - lo) : 0;
     // sequences with no token: outputs are zero, nothing is rejected unless the draft is not zero
@@ -569,7 +540,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   tc_fence_before();
   named_bar(8, T * TT);
   tc_fence_after();
-  const uint32_t tmem0 = *reinterpret_cast<volatile uint32_t*>(misc + 8);
+  const uint32_t tmem0 = __shfl_sync(0xFFFFFFFFu, *reinterpret_cast<volatile uint32_t*>(misc + 8), 0);   // (known to be uniform)
   constexpr uint32_t kIdescS = i8_idesc(C::kNQK, false, true), kIdescO = i8_idesc(C::kNPV, true, false);
 
   // =============================================================================================

@@ -216,38 +216,9 @@ __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int l
     int len = __ldg(p.seq_lens + b);
     return len < 0 ? 0 : (len > cap ? cap : len);
   };
-  long long tot = 0;
-  for (int b = lane; b < p.B; b += 32) tot += (clamp_len(b) + ST - 1) / ST;
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) tot += __shfl_xor_sync(0xFFFFFFFFu, tot, off);
-  const long long T = tot * p.Hkv;
-  const long long q = (T + n_cta - 1) / n_cta;
-  const long long lo = (long long)cta * q, hi = (lo + q < T) ? lo + q : T;
-  int b_lo = 0;
-  long long off_lo = 0;
-  if (lo < hi) {
-    long long running = 0;
-    for (int b0 = 0; b0 < p.B; b0 += 32) {
-      const int b = b0 + lane;
-      const long long u = b < p.B ? (long long)p.Hkv * ((clamp_len(b) + ST - 1) / ST) : 0;
-      long long incl = u;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const long long v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += v;
-      }
-      const long long excl = running + incl - u;
-      const bool hit = u > 0 && lo >= excl && lo < excl + u;
-      const unsigned mk = __ballot_sync(0xFFFFFFFFu, hit);
-      if (mk) {
-        const int src = __ffs(mk) - 1;
-        b_lo = b0 + src;
-        off_lo = lo - __shfl_sync(0xFFFFFFFFu, excl, src);
-        break;
-      }
-      running += __shfl_sync(0xFFFFFFFFu, incl, 31);
-    }
-  }
+  const SkRange rng = sk_range<ST>(p, n_cta, cta, lane, clamp_len);
+  const long long q = rng.q, lo = rng.lo, hi = rng.hi, off_lo = rng.off_lo;
+  const int b_lo = rng.b_lo;
   if (pw == 0) {
     if (lane == 0) misc[7] = lo < hi ? (int)(hi - lo) : 0;
     // sequences with no token: outputs are zero, nothing is rejected unless the draft is not zero
@@ -416,7 +387,8 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
   int4* info_s = reinterpret_cast<int4*>(smem + C::kOffInfo);
   Item* items = reinterpret_cast<Item*>(info_s + NSTAGE);
   int* misc = reinterpret_cast<int*>(smem + C::kOffMisc);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);   // (broadcast: the compiler may keep what follows from it in uniform registers)
   const int cta = blockIdx.x;
   const uint32_t ring_u32 = sbase + C::kOffRing;
   const uint32_t full0 = sbase + C::kOffBars, empty0 = full0 + NSTAGE * 8;
@@ -471,7 +443,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
     tc_fence_before();
     named_bar(5, C::kConsThreads + 32);
     tc_fence_after();
-    tmem0 = *reinterpret_cast<volatile uint32_t*>(misc + 8);
+    tmem0 = __shfl_sync(0xFFFFFFFFu, *reinterpret_cast<volatile uint32_t*>(misc + 8), 0);
   }
   // =============================================================================================
   // V converters (4 warps): expand the V planes of every unit into the V tile of the group that
