@@ -226,7 +226,8 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
     // 592 CTAs: 20 us at the tail of the launch).  The last CTA to arrive of each group of kGroup
     // neighbouring contributors merges the group into its first slot; the last group to finish
     // merges the group results into the output.  Every ticket resets itself; nobody waits.
-    constexpr int kGroup = 8, kOneLevel = 16;   // up to kOneLevel slots are merged in one go
+    constexpr int kGroup = 8, kOneLevel = 24;   // up to kOneLevel slots are merged in one go
+    constexpr int kAhead = 6;                    // loads in flight per thread
     const int n = item.n_contrib;
     const int ng = (n + kGroup - 1) / kGroup;
     const int g = ((int)blockIdx.x - item.first_cta) / kGroup;
@@ -256,17 +257,17 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
       const int first = top ? 0 : g * kGroup;
       const int count = top ? (n <= kOneLevel ? n : ng) : gsize;
       const size_t sstride = (top && n > kOneLevel ? (size_t)kGroup : (size_t)1) * cstride;
-      // a warp per column, a lane per 4 dims; `count` slots from `first` on, merged online, four
+      // a warp per column, a lane per 4 dims; `count` slots from `first` on, merged online, kAhead
       // loads ahead; the result goes to the output (normalised) or back to slot `first`
       for (int c = tid >> 5; c < p.ncols; c += kConsThreads / 32) {
         float* col = seg + (size_t)first * cstride + (size_t)c * kPartStride;
         float M = -INFINITY, L = 0.0f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int i0 = 0; i0 < count; i0 += 4) {
-          float mi[4], li[4];
-          float4 oi[4];
+        for (int i0 = 0; i0 < count; i0 += kAhead) {
+          float mi[kAhead], li[kAhead];
+          float4 oi[kAhead];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
+          for (int u = 0; u < kAhead; ++u) {
             const bool in = i0 + u < count;
             const float* src = col + (size_t)(in ? i0 + u : i0) * sstride;
             mi[u] = in ? __ldcg(src + 128) : -INFINITY;
@@ -274,7 +275,7 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
             oi[u] = __ldcg(reinterpret_cast<const float4*>(src) + lane);
           }
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
+          for (int u = 0; u < kAhead; ++u) {
             const float Mn = fmaxf(M, mi[u]);
             // an absent slot (mi = -inf) keeps fa = 1, fb = 0 once M is finite; while M is still
             // -inf both factors are forced to 0 / taken from the slot without forming inf - inf

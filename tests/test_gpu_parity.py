@@ -394,7 +394,7 @@ def test_wide_verify_long_context_many_pieces(lynx):
 def test_long_context_partial_slots_merge_in_two_levels(lynx):
     # 40k tokens on two KV heads: every head is split over some 40 CTAs, more than one group of
     # partial slots, so the group tickets and the merge of the group results are exercised (anchor
-    # and merge-verify at 4, 8 and 16 columns on the mma.sync kernels)
+    # and merge-verify at 4, 8 and 16 columns); the lengths differ, so the plain cut of the work is used
     B, Hkv, G, L = 2, 2, 4, 40_003
     for k in (1, 2, 4):
         c = _case(lynx, 740 + k, B, Hkv, G, k, (L, 9_000), 16, True, "lognormal_channels")
@@ -413,6 +413,30 @@ def test_long_context_partial_slots_merge_in_two_levels(lynx):
             lynx.check(c["ws"])
             _close(out.cpu().numpy().astype(np.float64), rf, f"verify 40k, {k * G} columns, call {rep}")
             assert fr.cpu().tolist() == [k] * B
+
+
+@pytest.mark.parametrize("B,Hkv,G,k,L", [(1, 8, 4, 1, 40_003), (1, 8, 4, 4, 20_001), (1, 2, 4, 2, 40_003),
+                                         (2, 4, 8, 1, 33_000), (1, 8, 4, 8, 12_345), (3, 8, 2, 2, 7_777)])
+def test_equal_length_sequences_use_the_aligned_cut(lynx, B, Hkv, G, k, L):
+    # all sequences equally long and few (sequence, head) segments: every segment gets whole CTAs of its
+    # own (18 per head for one layer of 8 heads; 74 per head with 2 heads: two merge levels; 6 for 24
+    # segments).  Anchor and merge-verify, twice on the same workspace (tickets reset themselves).
+    c = _case(lynx, 7600 + Hkv * k, B, Hkv, G, k, (L,) * B, 16, True, "lognormal_channels")
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    ra = oracle.attention(False, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(), c["lens"].numpy(),
+                          Hkv, 16, causal=True)
+    rf = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(), c["lens"].numpy(),
+                          Hkv, 16, causal=True)
+    for rep in range(2):
+        a = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True)
+        lynx.check(c["ws"])
+        _close(a.cpu().numpy().astype(np.float64), ra, f"anchor, aligned cut, call {rep}")
+        out, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True,
+                                                   draft_out=torch.from_numpy(rf.astype(np.float32)).cuda(),
+                                                   atol=0.05, rtol=0.0)
+        lynx.check(c["ws"])
+        _close(out.cpu().numpy().astype(np.float64), rf, f"verify, aligned cut, call {rep}")
+        assert fr.cpu().tolist() == [k] * B
 
 
 def test_wide_verify_single_token_returns_its_value_row(lynx):
