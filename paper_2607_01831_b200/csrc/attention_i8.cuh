@@ -493,6 +493,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   const uint32_t sfull0 = qready0 + 16;           // [team]  Q.K^T complete: scores valid, K tile free
   const uint32_t pvdone0 = sfull0 + T * 8;        // [team]  P.V complete: P and V tiles free, accumulators current
   volatile int* abort_word = misc;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent grid may be scheduled as SMs become free
   // misc[8] = tensor memory base; misc[16 + t] = deposits written by team t, misc[24 + t] = deposits of team t read;
   // misc[32 + s] = completed phases of raw stage s
 
@@ -521,6 +522,8 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
   for (int i = tid; i < T * C::kTeamScal / 4; i += C::kThreads) reinterpret_cast<float*>(smem + C::kOffScal)[i] = 0.0f;
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
+  // nothing in global memory has been touched so far: wait for the grids this one depends on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (warp >= C::kProdWarp0) {
     i8_producer<C, FULL>(p, warp - C::kProdWarp0, lane, ring_u32, full0, empty0, qfull0, qempty0,
@@ -1059,6 +1062,20 @@ lynx_status launch_i8(const AttnParams& p, cudaStream_t st) {
   long long grid = (cap_units + 3) / 4;
   const long long full = sm_count();   // one CTA per SM
   grid = grid < 1 ? 1 : (grid > full ? full : grid);
-  kern<<<(unsigned)grid, C::kThreads, C::kSmem, st>>>(p);
+  // Programmatic dependent launch: when the kernel before this one in the stream is of the same kind (one
+  // launch per layer of a decoder), this grid's CTAs may become resident, and set up their shared and tensor
+  // memory, while the last CTAs of that kernel are still merging; they read nothing before
+  // griddepcontrol.wait, i.e. before that kernel has completed and its memory is visible.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(C::kThreads);
+  cfg.dynamicSmemBytes = C::kSmem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) return LYNX_ERR_CUDA;
   return launch_status();
 }
