@@ -64,7 +64,7 @@ struct I8Cfg {
   static constexpr int kGroups = CP == 32 ? 2 : 1;
   static constexpr int kCG = CP / kGroups;               // columns of a column group
   static constexpr int kTeamWarps = 4 * kGroups, kTeamThreads = 32 * kTeamWarps;
-  static constexpr int kTeams = CP == 32 ? 2 : (FULL || CP == 16) ? 3 : CP == 4 ? 5 : 4;
+  static constexpr int kTeams = CP == 32 ? 2 : (FULL || CP == 16) ? 3 : 5;
   static constexpr int kProdWarps = CP == 32 ? 2 : 4;
   static constexpr int kProdWarp0 = kTeamWarps * kTeams;
   static constexpr int kThreads = (kProdWarp0 + kProdWarps) * 32;
@@ -96,9 +96,9 @@ struct I8Cfg {
   static_assert(kOffScal % 16 == 0 && kTeamScal % 16 == 0 && kOffBars % 8 == 0, "alignment");
   // tensor memory columns of a team: S, O accumulators, FP32 copy of O, K levels (128 bytes per token)
   // (with 32 columns there is no room for the copy: it stays in registers)
-  static constexpr bool kOfInTmem = CP <= 16;
+  static constexpr bool kOfInTmem = CP <= 16 && !(CP == 8 && !FULL);
   static constexpr int kTmS = 0, kTmO = kNQK, kTmOF = kNQK + kNPV, kTmK = kOfInTmem ? (kTmOF + CP + 7) / 8 * 8 : kTmOF;
-  static constexpr int kTmTeam = CP == 32 ? 256 : CP == 16 ? 160 : CP == 4 ? 96 : 128;
+  static constexpr int kTmTeam = CP == 32 ? 256 : CP == 16 ? 160 : (CP == 4 || !FULL) ? 96 : 128;
   static constexpr int kTmCols = 512;
   static_assert(kTmK + 32 <= kTmTeam && kTeams * kTmTeam <= 512, "tensor memory");
   static constexpr int kDrainUnits = FULL ? 256 : 4096;  // own units after which the int32 sums could overflow
