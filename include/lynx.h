@@ -177,7 +177,8 @@ lynx_status lynx_anchor_attention_static(const lynx_shape* shape, const void* q_
  * sign-aware two's-complement Anchor and a 4-bit centred Residual, packed two per byte like the linear
  * planes (q_anc, q_res: uint8 [n_pages][256][64], byte j = channel 2j | channel 2j+1 << 4).
  * Arithmetic is binary32; the readings of the algorithm's open points (alpha, epsilon = 1e-6, the scale
- * 120, the sign taken from the centred value) are stated in the library's design notes.
+ * 120, the sign taken from the centred value) are stated in the library's design notes.  All pointers
+ * 16-byte aligned (LYNX_ERR_ALIGN otherwise); n_pages == 0 is a valid no-op.
  * lynx_hier_dequantize reconstructs BF16 pages [n_pages][256][128] from both streams, or from the
  * Anchor alone when q_res is NULL (the Residual, a centred correction, taken as zero); the pages can be
  * attended to with lynx_bf16_attention (block_tokens = 256). */
