@@ -847,8 +847,16 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           f2_unpack(y2[c], a, b);
           ymax = max3(ymax, a, b);
         }
-        const bool need = fresh || units_in_acc >= C::kDrainUnits || ymax > 31.5f;
-        if (bar_or(bar_tm, TT, need)) {   // (team-wide: one P.V covers all columns, so they all restart together)
+        // A restart of the accumulation (new reference exponents, the int32 sums drained into the FP32 copy)
+        // is a decision of the whole team: one P.V covers all columns.  Where it is known beforehand (first
+        // unit of a piece, sums about to overflow) it is taken first.  Otherwise every thread writes its
+        // weights at once and a thread whose weight would leave the u32 range raises a flag, which all
+        // look at after the barrier that completes the P tile anyway: the common case has no barrier of
+        // its own for the question.
+        const bool forced = fresh || units_in_acc >= C::kDrainUnits;   // uniform over the team
+        const bool over = ymax > 31.5f;
+        volatile int* raise_flag = my_misc + 2;
+        auto restart = [&]() {
 #pragma unroll
           for (int c = 0; c < CG; ++c) {   // (rare path: back to absolute exponents x = y + ref)
             float a, b;
@@ -859,6 +867,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
             if (lane == 0) my_red[tw * CG + c] = mx;
           }
           named_bar(bar_tm, TT);
+          if (tt == 0) *raise_flag = 0;
           if (tt < CP) {
             const float* mr = my_red + (tt / CG) * 4 * CG + (tt % CG);   // the four warps of the column's group
             const float mx = fmaxf(fmaxf(mr[0], mr[CG]), fmaxf(mr[2 * CG], mr[3 * CG]));
@@ -882,10 +891,10 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           }
           drain(true);   // (the team's previous P.V has been waited for)
           fresh = false;
-        }
-        // ---- weights ------------------------------------------------------------------------------
-        uint32_t wi[CG];
-        {
+        };
+        // weights of this thread's token into its row of the P tile; `commit`: add them to the softmax sums
+        auto weights = [&](bool commit) {
+          uint32_t wi[CG];
           const uint64_t ia2 = f2_pack(ia, ia), ib2 = f2_pack(ib, ib);
 #pragma unroll
           for (int c = 0; c < CG / 2; ++c) {
@@ -894,19 +903,34 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
             const float wa = ex2_ftz(a), wb = ex2_ftz(b);
             asm("cvt.rni.u32.f32 %0, %1;" : "=r"(wi[2 * c]) : "f"(wa));
             asm("cvt.rni.u32.f32 %0, %1;" : "=r"(wi[2 * c + 1]) : "f"(wb));
-            const uint64_t w2 = f2_pack(wa, wb);
-            l2[c] = f2_fma(w2, ia2, l2[c]);
-            zs2[c] = f2_fma(w2, ib2, zs2[c]);
+            if (commit) {   // (not for weights beyond the range: they may be infinite)
+              const uint64_t w2 = f2_pack(wa, wb);
+              l2[c] = f2_fma(w2, ia2, l2[c]);
+              zs2[c] = f2_fma(w2, ib2, zs2[c]);
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < CG / 4; ++j)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                         ::"r"(p_row + (((uint32_t)(grp * (CG / 4) + j) ^ p_swz) << 4)), "r"(wi[4 * j]), "r"(wi[4 * j + 1]),
+                           "r"(wi[4 * j + 2]), "r"(wi[4 * j + 3]) : "memory");
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          tc_fence_before();
+          named_bar(bar_tm, TT);     // the P tile and the V tile are complete, S has been read
+        };
+        if (FULL) {   // (the merge-verify instances measure faster with the question asked first: one more barrier)
+          if (bar_or(bar_tm, TT, forced || over)) restart();
+          weights(true);
+        } else {
+          if (forced) restart();
+          else if (over) *raise_flag = 1;
+          // (a thread beyond the range keeps its weights out of the sums: after the restart they are different ones)
+          weights(forced || !over);
+          if (!forced && *raise_flag != 0) {   // uniform: read after the barrier; cleared inside restart()
+            restart();
+            weights(over);
           }
         }
-#pragma unroll
-        for (int j = 0; j < CG / 4; ++j)
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(p_row + (((uint32_t)(grp * (CG / 4) + j) ^ p_swz) << 4)), "r"(wi[4 * j]), "r"(wi[4 * j + 1]),
-                         "r"(wi[4 * j + 2]), "r"(wi[4 * j + 3]) : "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        tc_fence_before();
-        named_bar(bar_tm, TT);     // the P tile and the V tile are complete, S has been read
         if (tt == 0) {
           tc_fence_after();
           const uint32_t d = tmem0 + tm * C::kTmTeam + C::kTmO;
