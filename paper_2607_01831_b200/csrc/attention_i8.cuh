@@ -55,7 +55,13 @@ struct I8Cfg {
                                                     // read with plain loads: the copy engine takes ~35 cycles per copy)
   static constexpr int kStageBytes = kST * (FULL ? 256 : 128);
   static constexpr int kOffKA = 0, kOffVA = kST * 64, kOffKR = kST * 128, kOffVR = kST * 192;
-  static constexpr int kNQK = (3 * CP + 15) / 16 * 16;   // N of the Q.K^T product
+  // Anchor decode with up to 8 columns feeds the K planes to Q.K^T as they are: a token's 64 raw bytes
+  // b_m = a_2m + 16 a_2m+1 followed by the 64 masked bytes a_2m, against the query values Q_2m+1 and
+  // 16 Q_2m - Q_2m+1 (four digit planes instead of three: they fit the padding of N), which gives
+  // 16 sum_d Q_d a_d with a third of the logic operations of a full nibble expansion.
+  static constexpr bool kRawK = !FULL && CP <= 8;
+  static constexpr int kQPlanes = kRawK ? 4 : 3;
+  static constexpr int kNQK = (kQPlanes * CP + 15) / 16 * 16;   // N of the Q.K^T product
   static constexpr int kNPV = 4 * CP;                    // N of the P.V product
   static constexpr int kPartCols = CP < 8 ? 8 : CP;      // column stride of the partial slots
   static constexpr int kColsPad = CP;
@@ -238,7 +244,7 @@ __device__ __forceinline__ void i8_expand(uint32_t raw_a, uint32_t raw_r, uint32
 // The four 16-byte chunks of the row are read in a lane-dependent order (chunk i ^ s, s = (r >> 1) & 3:
 // rows are 64 bytes apart, so a fixed order would put a quarter-warp on two bank groups) and put back
 // in order with two levels of selects.
-template <bool FULL>
+template <bool FULL, bool RAW>
 __device__ __forceinline__ void i8_expand_k_tmem(uint32_t raw_a, uint32_t raw_r, int r, uint32_t tm_k) {
   const uint32_t s = ((uint32_t)r >> 1) & 3u;
   uint4 xa[4], xr[4];
@@ -271,6 +277,9 @@ __device__ __forceinline__ void i8_expand_k_tmem(uint32_t raw_a, uint32_t raw_r,
     for (int w = 0; w < 4; ++w) {
       if (FULL) {
         merge_codes(a[w], rr[w], regs[8 * j + w], regs[8 * j + 4 + w]);
+      } else if (RAW) {   // bytes 16 j + 4 w .. + 3 of the row as they are, and their low nibbles 64 bytes further on
+        regs[4 * j + w] = a[w];
+        regs[16 + 4 * j + w] = a[w] & 0x0F0F0F0Fu;
       } else {
         regs[8 * j + w] = a[w] & 0x0F0F0F0Fu;
         regs[8 * j + 4 + w] = (a[w] >> 4) & 0x0F0F0F0Fu;
@@ -618,7 +627,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
 #pragma unroll
       for (int i = 0; i < C::kTeamWarps; ++i) amax = fmaxf(amax, amax_s[i]);
       const int e = i8_q_exponent(amax);
-      const float ca = p.sm_log2 * __int_as_float((127 - e) << 23) * (FULL ? 1.0f : 16.0f);
+      const float ca = p.sm_log2 * __int_as_float((127 - e) << 23) * ((FULL || C::kRawK) ? 1.0f : 16.0f);
       const uint32_t qt = sbase + C::kOffQT + qi * C::kQTile;
       if (u_first == 0 && tt < CP * 4) {
         // this team owns the piece's first unit: it writes the three balanced s8 digit planes of
@@ -626,21 +635,33 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         // before last, which every team has left: the queries of this piece were loaded after that.)
         const float up = __int_as_float((127 + e) << 23);
         const int c = tt >> 2, j = tt & 3;
-        uint32_t pl[3][2][4];   // [plane][parity][word]
+        constexpr int NP = C::kQPlanes;
+        uint32_t pl[NP][2][4];   // [plane][half][word]
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
           const uint4 v = *reinterpret_cast<const uint4*>(qb + c * 256 + j * 64 + w * 16);
           const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
-          uint32_t acc[3][2] = {{0, 0}, {0, 0}, {0, 0}};
+          uint32_t acc[NP][2];
+#pragma unroll
+          for (int pln = 0; pln < NP; ++pln) { acc[pln][0] = 0; acc[pln][1] = 0; }
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
+            int qv2[2];
 #pragma unroll
             for (int par = 0; par < 2; ++par) {
               const float f = par ? __uint_as_float(ww[i] & 0xFFFF0000u) : __uint_as_float(ww[i] << 16);
-              int qv = __float2int_rn(f * up);
-              qv = max(-4194303, min(4194303, qv));
+              const int qv = __float2int_rn(f * up);
+              qv2[par] = max(-4194303, min(4194303, qv));
+            }
+            // half 0 / 1 of the row: even / odd dims -- or, where K goes in as raw bytes, what multiplies the
+            // byte pair m (dims 2m, 2m+1; odd value) and its low nibble (16 x even value - odd value)
+            int val[2] = {qv2[0], qv2[1]};
+            if (C::kRawK) { val[0] = qv2[1]; val[1] = 16 * qv2[0] - qv2[1]; }
 #pragma unroll
-              for (int pln = 0; pln < 3; ++pln) {
+            for (int par = 0; par < 2; ++par) {
+              int qv = val[par];
+#pragma unroll
+              for (int pln = 0; pln < NP; ++pln) {
                 const int dgt = (int)(signed char)(qv & 0xFF);
                 acc[pln][par] |= (uint32_t)(dgt & 0xFF) << (8 * i);
                 qv = (qv - dgt) >> 8;
@@ -648,14 +669,15 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
             }
           }
 #pragma unroll
-          for (int pln = 0; pln < 3; ++pln) { pl[pln][0][w] = acc[pln][0]; pl[pln][1][w] = acc[pln][1]; }
+          for (int pln = 0; pln < NP; ++pln) { pl[pln][0][w] = acc[pln][0]; pl[pln][1][w] = acc[pln][1]; }
         }
 #pragma unroll
-        for (int pln = 0; pln < 3; ++pln) {
+        for (int pln = 0; pln < NP; ++pln) {
           const int n = pln * CP + c;
 #pragma unroll
           for (int par = 0; par < 2; ++par) {
-            const uint32_t a = qt + (uint32_t)n * 128u + ((uint32_t)((2 * j + par) ^ (n & 7)) << 4);
+            const int chunk = C::kRawK ? 4 * par + j : 2 * j + par;   // 16 bytes of the row's 128
+            const uint32_t a = qt + (uint32_t)n * 128u + ((uint32_t)(chunk ^ (n & 7)) << 4);
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pl[pln][par][0]),
                          "r"(pl[pln][par][1]), "r"(pl[pln][par][2]), "r"(pl[pln][par][3]) : "memory");
           }
@@ -771,7 +793,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         // ---- K levels (free: the team's previous Q.K^T has been waited for), then Q.K^T; V tile (free
         // once the team's previous P.V is complete).  With two column groups one expands K, the other V.
         if (G == 1 || grp == 0) {
-          i8_expand_k_tmem<FULL>(st + C::kOffKA, st + C::kOffKR, r, tm_k + lane_sel);
+          i8_expand_k_tmem<FULL, C::kRawK>(st + C::kOffKA, st + C::kOffKR, r, tm_k + lane_sel);
           tc_wait_st();
         } else {
           if (n_own > 0) mbar_wait(pvdone0 + tm * 8, (n_own - 1) & 1, abort_word);
@@ -811,19 +833,25 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
         // y = log2 of the weight relative to the column's reference exponent, two columns per register pair
         uint64_t y2[CG / 2];
         {
-          uint32_t s0[CG], s1[CG], s2[CG];
+          uint32_t s0[CG], s1[CG], s2[CG], s3[C::kRawK ? CG : 1];
           TmemRegs<CG>::ld(tm_s, s0);
           TmemRegs<CG>::ld(tm_s + CP, s1);
           TmemRegs<CG>::ld(tm_s + 2 * CP, s2);
+          if (C::kRawK) TmemRegs<CG>::ld(tm_s + 3 * CP, s3);
           tc_wait_ld();
           const uint64_t al2 = f2_pack(al, al), be2 = f2_pack(be, be), lsv2 = f2_pack(lsv, lsv);
-          const uint64_t k256 = f2_pack(256.0f, 256.0f);
+          const uint64_t k256 = C::kRawK ? f2_pack(65536.0f, 65536.0f) : f2_pack(256.0f, 256.0f);
           const float* ref_r = fresh ? zero_s : ref_s;   // (a piece's first unit: relative to zero)
 #pragma unroll
           for (int c = 0; c < CG / 2; ++c) {
-            const uint64_t hi = f2_pack((float)((int)s2[2 * c] * 256 + (int)s1[2 * c]),
-                                        (float)((int)s2[2 * c + 1] * 256 + (int)s1[2 * c + 1]));
-            const uint64_t lo = f2_pack((float)(int)s0[2 * c], (float)(int)s0[2 * c + 1]);
+            uint64_t hi, lo;   // the digit-plane sums put together: exact in int32 two planes at a time
+            if (C::kRawK) {
+              hi = f2_pack((float)((int)s3[2 * c] * 256 + (int)s2[2 * c]), (float)((int)s3[2 * c + 1] * 256 + (int)s2[2 * c + 1]));
+              lo = f2_pack((float)((int)s1[2 * c] * 256 + (int)s0[2 * c]), (float)((int)s1[2 * c + 1] * 256 + (int)s0[2 * c + 1]));
+            } else {
+              hi = f2_pack((float)((int)s2[2 * c] * 256 + (int)s1[2 * c]), (float)((int)s2[2 * c + 1] * 256 + (int)s1[2 * c + 1]));
+              lo = f2_pack((float)(int)s0[2 * c], (float)(int)s0[2 * c + 1]);
+            }
             const uint64_t qs2 = *reinterpret_cast<const uint64_t*>(qs_s + c0 + 2 * c);
             const uint64_t rf2 = *reinterpret_cast<const uint64_t*>(ref_r + c0 + 2 * c);
             y2[c] = f2_fma(f2_fma(hi, k256, lo), al2, f2_fma(be2, qs2, f2_sub(lsv2, rf2)));
