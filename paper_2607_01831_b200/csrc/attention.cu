@@ -25,6 +25,7 @@
 // partial (m, l, O) goes to the workspace and the last contributor (atomic ticket, no waiting)
 // merges them; for verification the last CTA of a sequence also takes the accept/reject
 // decision.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 

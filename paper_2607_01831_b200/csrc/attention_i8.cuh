@@ -45,6 +45,44 @@
 // holds dim 32 j + 8 w + 2 i + parity (what the nibble expansion yields with two logic
 // operations per word); the query planes use the same order and O is un-permuted at write-out.
 
+// Tensor maps of the K planes ([rows][64 bytes] u8, box = one 16-token sub-block, 64-byte swizzle): the
+// copy engine stores 16-byte chunk c of row r at position c ^ ((r >> 1) & 3), which is the order in which
+// the threads of a quarter-warp can read their rows (64 bytes apart) without bank conflicts; read back at
+// position i ^ ((r >> 1) & 3), chunk i arrives in place with no reordering in registers.
+// The V planes go through maps of the same shape without swizzle, so that one instruction of a producer warp
+// issues all its copies of a unit (the map is a per-lane operand).
+struct alignas(64) I8Maps {
+  CUtensorMap m[4];   // K Anchor, V Anchor, K Residual, V Residual (the order of the stage's arrays)
+};
+inline bool i8_plane_map(CUtensorMap* m, const uint8_t* base, uint64_t rows, bool swizzle) {
+  using Fn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                          const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                          CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static Fn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<Fn>(f);
+  }();
+  if (!fn || !base || rows == 0) return false;
+  const cuuint64_t dims[2] = {64, rows};
+  const cuuint64_t strides[1] = {64};
+  const cuuint32_t box[2] = {64, 16}, es[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// one 16-row box of a plane (rows row .. row + 15, all 64 bytes) into shared memory
+__device__ __forceinline__ void tma_rows16(uint32_t dst, const CUtensorMap* map, int row, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(bar)
+      : "memory");
+}
+
 constexpr int kI8PieceUnits = 32;  // stage-units whose block ids a producer warp looks up at a time
 
 template <bool FULL, int CP>
@@ -254,25 +292,12 @@ __device__ __forceinline__ void i8_expand_k_tmem(uint32_t raw_a, uint32_t raw_r,
     xa[i] = lds128(raw_a + off);
     if (FULL) xr[i] = lds128(raw_r + off);
   }
-  auto sel4 = [](bool c, const uint4& a, const uint4& b) {
-    return make_uint4(c ? a.x : b.x, c ? a.y : b.y, c ? a.z : b.z, c ? a.w : b.w);
-  };
-  uint4 ya[4], yr[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    ya[i] = sel4(s & 1u, xa[i ^ 1], xa[i]);
-    if (FULL) yr[i] = sel4(s & 1u, xr[i ^ 1], xr[i]);
-  }
   uint32_t regs[32];
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const uint4 a4 = sel4(s & 2u, ya[j ^ 2], ya[j]);
-    const uint32_t a[4] = {a4.x, a4.y, a4.z, a4.w};
+  for (int j = 0; j < 4; ++j) {   // (position j ^ s holds chunk j: the copy engine's 64-byte swizzle)
+    const uint32_t a[4] = {xa[j].x, xa[j].y, xa[j].z, xa[j].w};
     uint32_t rr[4] = {0, 0, 0, 0};
-    if (FULL) {
-      const uint4 r4 = sel4(s & 2u, yr[j ^ 2], yr[j]);
-      rr[0] = r4.x; rr[1] = r4.y; rr[2] = r4.z; rr[3] = r4.w;
-    }
+    if (FULL) { rr[0] = xr[j].x; rr[1] = xr[j].y; rr[2] = xr[j].z; rr[3] = xr[j].w; }
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
       if (FULL) {
@@ -297,7 +322,7 @@ template <class C, bool FULL>
 __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lane, uint32_t ring_u32,
                                             uint32_t full0, uint32_t empty0, uint32_t qfull0, uint32_t qempty0,
                                             uint32_t qraw_u32, uint32_t* blk_s, Item* items, int* misc,
-                                            volatile int* abort_word) {
+                                            volatile int* abort_word, const I8Maps* maps) {
   constexpr int ST = C::kST, NSTAGE = C::kNStage, NARR = C::kNArr;
   const int n_cta = gridDim.x, cta = blockIdx.x;
   const int cap = p.max_blocks * p.bt;
@@ -338,8 +363,7 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
   constexpr int RP = SPW * NARR;               // roles of this warp: (sub-block, array)
   const int role = pw * RP + (lane < RP ? lane : 0);
   const int sub = role / NARR, arr = role % NARR, sub_first = SPW * pw;
-  const unsigned char* my_src = arr == 0 ? p.ka : arr == 1 ? p.va : arr == 2 ? p.kr : p.vr;
-  const uint32_t my_bytes = 1024u, my_mul = 64u;
+  const uint32_t my_bytes = 1024u;
   const uint32_t my_dst = (uint32_t)(arr == 0 ? C::kOffKA : arr == 1 ? C::kOffVA : arr == 2 ? C::kOffKR : C::kOffVR) +
                           (uint32_t)sub * my_bytes;
   constexpr uint32_t kBytesSub = (FULL ? 4u : 2u) * 1024u;   // bytes of one sub-block
@@ -399,7 +423,7 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
         }
         __syncwarp();
         if (lane < RP && row != 0xFFFFFFFFu)
-          bulk_g2s(ring_u32 + slot * C::kStageBytes + my_dst, my_src + (size_t)row * my_mul, my_bytes, bar);
+          tma_rows16(ring_u32 + slot * C::kStageBytes + my_dst, &maps->m[arr], (int)row, bar);
       }
       __syncwarp();  // my_blk is rewritten by the next round
     }
@@ -481,7 +505,8 @@ __device__ __noinline__ bool seq_wait(const volatile int* ctr, int need, volatil
 }
 
 template <bool FULL, int CP>
-__global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(const AttnParams p,
+                                                                               const __grid_constant__ I8Maps maps) {
   using C = I8Cfg<FULL, CP>;
   constexpr int NSTAGE = C::kNStage, T = C::kTeams, G = C::kGroups, CG = C::kCG, TT = C::kTeamThreads;
   extern __shared__ unsigned char smem_raw[];
@@ -536,7 +561,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
 
   if (warp >= C::kProdWarp0) {
     i8_producer<C, FULL>(p, warp - C::kProdWarp0, lane, ring_u32, full0, empty0, qfull0, qempty0,
-                         sbase + C::kOffQRaw, blk_s, items, misc, abort_word);
+                         sbase + C::kOffQRaw, blk_s, items, misc, abort_word, &maps);
     return;
   }
   __syncthreads();  // (A)
@@ -1128,6 +1153,17 @@ lynx_status launch_i8(const AttnParams& p, cudaStream_t st) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) return LYNX_ERR_CUDA;
+  I8Maps maps;
+  const uint64_t plane_rows = (uint64_t)p.num_blocks * p.Hkv * p.bt;
+  if (!i8_plane_map(&maps.m[0], p.ka, plane_rows, true) || !i8_plane_map(&maps.m[1], p.va, plane_rows, false))
+    return LYNX_ERR_CUDA;
+  if (FULL) {
+    if (!i8_plane_map(&maps.m[2], p.kr, plane_rows, true) || !i8_plane_map(&maps.m[3], p.vr, plane_rows, false))
+      return LYNX_ERR_CUDA;
+  } else {
+    maps.m[2] = maps.m[0];
+    maps.m[3] = maps.m[1];
+  }
+  if (cudaLaunchKernelEx(&cfg, kern, p, maps) != cudaSuccess) return LYNX_ERR_CUDA;
   return launch_status();
 }
