@@ -121,7 +121,9 @@ lynx_status lynx_workspace_init(void* workspace, size_t workspace_bytes, void* s
  * softmax_scale 0 means 1/sqrt(128).  out : [batch][n_q][Hq][128] float.
  * n_q must be <= 16 and n_q * (Hq/Hkv) <= 64.  seq_lens[b] is clamped to the table's capacity.
  * Value rows of any finite scale are handled (the weights are fixed-point numbers relative to a
- * per-column reference exponent). */
+ * per-column reference exponent).  Queries enter as fixed-point numbers with 22 bits below the largest
+ * |q| among the columns of a (sequence, KV head): whatever their magnitude, entries are exact to
+ * 2^-22 of that largest one. */
 lynx_status lynx_anchor_attention(const lynx_shape* shape, const void* q_bf16, int32_t batch,
                                   int32_t n_q, int32_t causal, lynx_plane K, lynx_plane V,
                                   const int32_t* block_table, const int32_t* seq_lens,
