@@ -93,11 +93,14 @@ struct I8Cfg {
                                                     // read with plain loads: the copy engine takes ~35 cycles per copy)
   static constexpr int kStageBytes = kST * (FULL ? 256 : 128);
   static constexpr int kOffKA = 0, kOffVA = kST * 64, kOffKR = kST * 128, kOffVR = kST * 192;
-  // Anchor decode with up to 8 columns feeds the K planes to Q.K^T as they are: a token's 64 raw bytes
+  // Anchor decode with 4 columns feeds the K planes to Q.K^T as they are: a token's 64 raw bytes
   // b_m = a_2m + 16 a_2m+1 followed by the 64 masked bytes a_2m, against the query values Q_2m+1 and
   // 16 Q_2m - Q_2m+1 (four digit planes instead of three: they fit the padding of N), which gives
   // 16 sum_d Q_d a_d with a third of the logic operations of a full nibble expansion.
-  static constexpr bool kRawK = !FULL && CP <= 8;
+  // (with more columns the fourth plane's share of the score arithmetic costs more registers than the
+  // expansion saves: 8 columns measured 20 % slower with it)
+  static constexpr bool kRawK = !FULL && CP == 4;
+  static constexpr bool kVoteFirst = FULL || CP > 4;   // restart question before the weights (see the unit loop)
   static constexpr int kQPlanes = kRawK ? 4 : 3;
   static constexpr int kNQK = (kQPlanes * CP + 15) / 16 * 16;   // N of the Q.K^T product
   static constexpr int kNPV = 4 * CP;                    // N of the P.V product
@@ -971,7 +974,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
           tc_fence_before();
           named_bar(bar_tm, TT);     // the P tile and the V tile are complete, S has been read
         };
-        if (FULL) {   // (the merge-verify instances measure faster with the question asked first: one more barrier)
+        if (C::kVoteFirst) {   // (every instance but the 4-column anchor one measures faster with the question asked first)
           if (bar_or(bar_tm, TT, forced || over)) restart();
           weights(true);
         } else {
