@@ -119,7 +119,9 @@ lynx_status lynx_workspace_init(void* workspace, size_t workspace_bytes, void* s
  * Query j of sequence b attends tokens [0, seq_lens[b]) (causal == 0) or
  * [0, seq_lens[b] - n_q + j + 1) (causal != 0); a query that sees no token gets zeros.
  * softmax_scale 0 means 1/sqrt(128).  out : [batch][n_q][Hq][128] float.
- * n_q must be <= 16 and n_q * (Hq/Hkv) <= 64.  seq_lens[b] is clamped to the table's capacity.
+ * n_q must be <= 64 (the cap on speculated positions of Section 5.1).  A kernel launch takes up to 32
+ * query columns n_q * (Hq/Hkv); a call with more runs as slices of whole positions, each a pass of its own
+ * over the planes, one after the other on the stream.  seq_lens[b] is clamped to the table's capacity.
  * Value rows of any finite scale are handled (the weights are fixed-point numbers relative to a
  * per-column reference exponent).  Queries enter as fixed-point numbers with 22 bits below the largest
  * |q| among the columns of a (sequence, KV head): whatever their magnitude, entries are exact to
@@ -137,7 +139,9 @@ lynx_status lynx_anchor_attention(const lynx_shape* shape, const void* q_bf16, i
  * prefix; out_full at that position is the correction).
  * draft_out : [batch][k][Hq][128] float, the Anchor-state results being verified; may be NULL,
  * then dev / first_reject are not written (and may be NULL).  out_full : same shape, float.
- * k must be <= 16 and k * (Hq/Hkv) <= 64.  With 17..64 columns the weights are FP16 numbers: a value
+ * k must be <= 64.  A launch takes up to 16 positions and 64 columns k * (Hq/Hkv); a longer window runs as
+ * slices of whole positions (a pass over the planes each), and first_reject is then taken over the whole
+ * window from the deviations.  With 17..64 columns per launch the weights are FP16 numbers: a value
  * row whose scale reaches 16 (a range of 4080 or more) would overflow them; such rows are recorded
  * in the status word and lynx_check returns LYNX_ERR_RANGE (the outputs of that call are then not
  * to be used).  Up to 16 columns there is no such limit. */

@@ -34,8 +34,10 @@
 namespace lynx {
 namespace {
 
-constexpr int kMaxQ = 16;          // query positions per call
-constexpr int kMaxCols = 64;       // n_q * G
+constexpr int kMaxQ = 16;          // query positions per launch
+constexpr int kMaxWindow = 64;     // query positions per call (Section 5.1: at most 64 speculative tokens); more than
+                                   // kMaxQ positions or kMaxCols columns run as slices, one pass over the planes each
+constexpr int kMaxCols = 64;       // n_q * G per launch
 constexpr int kPartStride = 132;   // floats per (chunk, column) partial: O[128], m, l, pad
 
 struct AttnParams {
@@ -343,7 +345,7 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
           float worst = 0.0f;
           for (int h = 0; h < p.Hkv; ++h)
             worst = fmaxf(worst, __ldcg(p.ws_dev + ((size_t)item.b * p.Hkv + h) * kMaxQ + j));
-          p.dev[(size_t)item.b * p.nq + j] = worst;
+          p.dev[(size_t)item.b * p.nq_stride + j] = worst;
           if (worst > 1.0f) fr = j;
         }
         p.first_reject[item.b] = fr;
@@ -436,7 +438,16 @@ __device__ __forceinline__ SkRange sk_range(const AttnParams& p, int n_cta, int 
 // ------------------------------------------------------------------ host side
 constexpr int kMaxCtasPerSm = 4;
 
+// Query positions per launch of a verification call: all of them up to kMaxQ positions and kMaxCols
+// columns, else as many whole positions as fit both.
+inline int verify_slice(int nq, int G) {
+  if (nq <= kMaxQ && nq * G <= kMaxCols) return nq;
+  const int by_cols = kMaxCols / G > 0 ? kMaxCols / G : 1;
+  return by_cols < kMaxQ ? by_cols : kMaxQ;
+}
+
 struct Plan {
+  int per;             // query positions per verification launch
   int ncols, variant;  // variant: 0: NT1 TW4 CG1; 1: NT2 TW4 CG1; 2: NT2 TW4 CG2; 3: NT2 TW2 CG4
   int cols_pad;
   size_t off_chunk_ctr, off_seq_ctr, off_group_ctr, off_dev, off_part, bytes;
@@ -446,11 +457,14 @@ struct Plan {
 bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   if (!s || s->head_dim != LYNX_D || s->num_kv_heads <= 0 || s->num_q_heads <= 0 ||
       s->num_q_heads % s->num_kv_heads != 0 || s->block_tokens <= 0 || s->block_tokens % 16 != 0 ||
-      s->num_blocks <= 0 || s->max_blocks_per_seq <= 0 || B <= 0 || nq <= 0 || nq > kMaxQ)
+      s->num_blocks <= 0 || s->max_blocks_per_seq <= 0 || B <= 0 || nq <= 0 || nq > kMaxWindow)
     return false;
   const int G = s->num_q_heads / s->num_kv_heads;
-  const int ncols = nq * G;
-  if (ncols > kMaxCols) return false;
+  if (G > 16) return false;
+  // positions per launch of a verification call (anchor calls slice further, to 32 columns); the scratch is
+  // sized for the widest launch
+  pl->per = verify_slice(nq, G);
+  const int ncols = pl->per * G;
   const int64_t cap = (int64_t)s->max_blocks_per_seq * s->block_tokens;
   if (cap >= (1ll << 31)) return false;
   if ((int64_t)s->num_blocks * s->num_kv_heads * s->block_tokens >= (1ll << 32)) return false;
@@ -472,6 +486,17 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   // (only the FP16 kernels have them: verification with 17..64 columns, anchor attention with 33..64)
   pl->shadow_bytes = ncols > 16 ? (size_t)sm_count() * 131072 : 0;
   return true;
+}
+
+// Section 4.3's longest agreeing prefix over a window that was verified in slices: the smallest position
+// whose deviation exceeds 1, or the number of positions.
+__global__ void first_reject_kernel(const float* __restrict__ dev, int B, int nq, int32_t* __restrict__ first_reject) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  int fr = nq;
+  for (int j = nq - 1; j >= 0; --j)
+    if (dev[(size_t)b * nq + j] > 1.0f) fr = j;
+  first_reject[b] = fr;
 }
 
 lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int B, int nq, int causal,
@@ -496,7 +521,7 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
     return LYNX_ERR_ALIGN;
   // the FP16 kernels cut their accumulation chains into FP32 copies at the end of the workspace; the
   // fixed-scratch entry point has no room for them and says so in its contract
-  const bool fp16_kernel = full && pl.ncols > 16;
+  const bool fp16_kernel = full && pl.ncols > 16;   // (pl.ncols: the columns of the widest launch)
   const bool use_shadow = fp16_kernel && !fixed_scratch;
   if (workspace_bytes < pl.bytes + (use_shadow ? pl.shadow_bytes : 0)) return LYNX_ERR_WORKSPACE;
   if (full && draft && !(atol > 0.0f && rtol >= 0.0f)) return LYNX_ERR_SHAPE;
@@ -529,7 +554,7 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
     // Anchor attention: the integer tcgen05 kernels take up to 32 columns.  A call with more (33..64) is
     // run as slices of whole query positions, each a pass of its own over the planes, one after the
     // other on the stream (they share the workspace).
-    const int per = pl.ncols <= 32 ? nq : (32 / p.G > 0 ? 32 / p.G : 1);
+    const int per = nq * p.G <= 32 ? nq : (32 / p.G > 0 ? 32 / p.G : 1);
     for (int j0 = 0; j0 < nq; j0 += per) {
       AttnParams ps = p;
       ps.nq = nq - j0 < per ? nq - j0 : per;
@@ -543,12 +568,28 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
     }
     return LYNX_OK;
   }
-  // verification: the integer kernels up to 16 columns, tcgen05 with FP16 operands (attention_wide.cuh) above
-  if (pl.ncols <= 4) return launch_i8<true, 4>(p, st);
-  if (pl.ncols <= 8) return launch_i8<true, 8>(p, st);
-  if (pl.ncols <= 16) return launch_i8<true, 16>(p, st);
-  if (pl.ncols <= 32) return launch_wide<2, 2>(p, st);
-  return launch_wide<2, 1>(p, st);
+  // verification: the integer kernels up to 16 columns, tcgen05 with FP16 operands (attention_wide.cuh) above.
+  // A window of more than kMaxQ positions or kMaxCols columns runs as slices of whole positions, each a pass
+  // of its own over the planes that writes its outputs and deviations; the index of the first rejected
+  // position over the whole window then follows from the deviations.
+  for (int j0 = 0; j0 < nq; j0 += pl.per) {
+    AttnParams ps = p;
+    ps.nq = nq - j0 < pl.per ? nq - j0 : pl.per;
+    ps.ncols = ps.nq * p.G;
+    ps.tail = nq - j0;
+    ps.q = p.q + (size_t)j0 * p.Hq * LYNX_D;
+    ps.out = p.out + (size_t)j0 * p.Hq * LYNX_D;
+    if (p.draft) { ps.draft = p.draft + (size_t)j0 * p.Hq * LYNX_D; ps.dev = p.dev + j0; }
+    const lynx_status rc = ps.ncols <= 4 ? launch_i8<true, 4>(ps, st) : ps.ncols <= 8 ? launch_i8<true, 8>(ps, st)
+                         : ps.ncols <= 16 ? launch_i8<true, 16>(ps, st)
+                         : ps.ncols <= 32 ? launch_wide<2, 2>(ps, st) : launch_wide<2, 1>(ps, st);
+    if (rc != LYNX_OK) return rc;
+  }
+  if (p.draft && pl.per < nq) {
+    first_reject_kernel<<<(unsigned)((B + 127) / 128), 128, 0, st>>>(p.dev, B, nq, p.first_reject);
+    return launch_status();
+  }
+  return LYNX_OK;
 }
 
 }  // namespace

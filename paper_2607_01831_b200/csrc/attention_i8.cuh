@@ -348,10 +348,10 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
         for (int j = p.nq - 1; j >= 0; --j) {
           float worst = 0.0f;
           for (int i = lane; i < p.Hq * LYNX_D; i += 32)
-            worst = fmaxf(worst, fabsf(__ldg(p.draft + ((size_t)b * p.nq + j) * p.Hq * LYNX_D + i)) / p.atol);
+            worst = fmaxf(worst, fabsf(__ldg(p.draft + ((size_t)b * p.nq_stride + j) * p.Hq * LYNX_D + i)) / p.atol);
 #pragma unroll
           for (int off = 16; off >= 1; off >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xFFFFFFFFu, worst, off));
-          if (lane == 0) p.dev[(size_t)b * p.nq + j] = worst;
+          if (lane == 0) p.dev[(size_t)b * p.nq_stride + j] = worst;
           if (worst > 1.0f) fr = j;
         }
         if (lane == 0) p.first_reject[b] = fr;

@@ -225,16 +225,16 @@ __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int l
     for (int b = cta; b < p.B; b += n_cta) {
       if (clamp_len(b) != 0) continue;
       const size_t n = (size_t)p.nq * p.Hq * LYNX_D;
-      for (size_t i = lane; i < n; i += 32) p.out[(size_t)b * n + i] = 0.0f;
+      for (size_t i = lane; i < n; i += 32) p.out[(size_t)b * p.nq_stride * p.Hq * LYNX_D + i] = 0.0f;
       if (p.draft != nullptr) {
         int fr = p.nq;
         for (int j = p.nq - 1; j >= 0; --j) {
           float worst = 0.0f;
           for (int i = lane; i < p.Hq * LYNX_D; i += 32)
-            worst = fmaxf(worst, fabsf(__ldg(p.draft + ((size_t)b * p.nq + j) * p.Hq * LYNX_D + i)) / p.atol);
+            worst = fmaxf(worst, fabsf(__ldg(p.draft + ((size_t)b * p.nq_stride + j) * p.Hq * LYNX_D + i)) / p.atol);
 #pragma unroll
           for (int off = 16; off >= 1; off >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xFFFFFFFFu, worst, off));
-          if (lane == 0) p.dev[(size_t)b * p.nq + j] = worst;
+          if (lane == 0) p.dev[(size_t)b * p.nq_stride + j] = worst;
           if (worst > 1.0f) fr = j;
         }
         if (lane == 0) p.first_reject[b] = fr;
@@ -288,7 +288,7 @@ __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int l
       __syncwarp();
       for (int j = lane; j < p.nq; j += 32)
         bulk_g2s(smem_u32(q_s + ((size_t)qi * C::kColsPad + j * p.G) * LYNX_D),
-                 p.q + (((size_t)b * p.nq + j) * p.Hq + (size_t)hkv * p.G) * LYNX_D,
+                 p.q + (((size_t)b * p.nq_stride + j) * p.Hq + (size_t)hkv * p.G) * LYNX_D,
                  (uint32_t)(p.G * LYNX_D * 2), qfull0 + qi * 8);
     }
     for (int c0 = 0; c0 < n; c0 += kPieceUnits) {
@@ -595,8 +595,8 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
     mbar_wait(qfull0 + qi * 8, (ic >> 1) & 1, abort_word);
     const Item item = items[qi];
     const int len = item.len, n_piece = item.pad0;
-    const int full_lim = p.causal ? len - p.nq + 1 : len;
-    const int lim_c = c < p.ncols ? (p.causal ? len - p.nq + c / p.G + 1 : len) : 0;
+    const int full_lim = p.causal ? len - p.tail + 1 : len;   // (a slice of a longer window: tail positions to its end)
+    const int lim_c = c < p.ncols ? (p.causal ? len - p.tail + c / p.G + 1 : len) : 0;
     const __nv_bfloat16* qb = q_s + (size_t)qi * CP * LYNX_D;
     // ---- the piece's queries: common power-of-two scale, FP16 A operand, sum of q ------------
     float amax = 0.0f;
@@ -927,7 +927,7 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
         const float v = msc[cc * C::kMergeStride + d] + z;
         if (direct) {
           const int j = cc / p.G, hh = cc % p.G;
-          p.out[(((size_t)item.b * p.nq + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + d] =
+          p.out[(((size_t)item.b * p.nq_stride + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + d] =
               lt > 0.0f ? v / lt : 0.0f;
         } else {
           part_dst[(size_t)cc * kPartStride + d] = v;

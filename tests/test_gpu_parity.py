@@ -439,6 +439,46 @@ def test_equal_length_sequences_use_the_aligned_cut(lynx, B, Hkv, G, k, L):
         assert fr.cpu().tolist() == [k] * B
 
 
+@pytest.mark.parametrize("B,Hkv,G,k,lens", [(2, 2, 4, 24, (1500, 37)), (1, 2, 1, 40, (900,)), (2, 1, 8, 20, (300, 0)),
+                                            (1, 1, 2, 64, (2100,)), (1, 2, 16, 5, (700,))])
+def test_windows_beyond_one_launch_run_as_slices(lynx, B, Hkv, G, k, lens):
+    # up to 64 drafted positions per call (the cap Section 5.1 states): more than 16 positions or 64 columns
+    # are verified in slices of whole positions, anchor calls likewise; outputs against the oracle, and the
+    # first rejected position over the WHOLE window identical to the oracle's
+    c = _case(lynx, 9100 + k, B, Hkv, G, k, lens, 16, True, "lognormal_channels")
+    qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
+    ra = oracle.attention(False, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(), c["lens"].numpy(),
+                          Hkv, 16, causal=True)
+    rf = oracle.attention(True, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(), c["lens"].numpy(),
+                          Hkv, 16, causal=True)
+    draft = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True)
+    lynx.check(c["ws"])
+    _close(draft.cpu().numpy().astype(np.float64), ra, "anchor attention, sliced window")
+    draft_np = draft.cpu().numpy()
+    exercised = 0
+    for atol, rtol in [(2e-2, 2e-2), (5e-2, 5e-2), (1e-1, 1e-1), (3e-1, 1e-1), (1.0, 0.0), (3e-3, 0.0)]:
+        want_fr, want_dev = oracle.verify_decision(rf, draft_np, atol, rtol)
+        if np.all(np.abs(want_dev - 1.0) > 0.05):
+            exercised += 1
+            out, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"],
+                                                       draft_out=draft, atol=atol, rtol=rtol, causal=True)
+            lynx.check(c["ws"])
+            _close(out.cpu().numpy().astype(np.float64), rf, "merge-verify attention, sliced window")
+            assert np.array_equal(fr.cpu().numpy(), want_fr), (atol, rtol, want_dev)
+            assert np.allclose(dev.cpu().numpy(), want_dev, rtol=0.05, atol=1e-3)
+    assert exercised >= 1
+    # a perturbation in a later slice is found as the first rejection of the whole window
+    out, _, _ = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], causal=True)
+    j = k - 2
+    bad = out.clone()
+    bad[0, j, 0, 5] += 1.0
+    _, fr, dev = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], td, ld, c["ws"], draft_out=bad,
+                                             atol=1e-2, rtol=1e-2, causal=True)
+    assert fr.cpu().tolist()[0] == j and fr.cpu().tolist()[1:] == [k] * (B - 1)
+    with pytest.raises(lynx.LynxError):   # beyond the window cap
+        lynx.workspace_bytes(c["geo"], B, 65) or lynx.make_workspace(c["geo"], B, 65, "cuda")
+
+
 def test_wide_verify_single_token_returns_its_value_row(lynx):
     # the two weight terms on the tcgen05 path: one attended token gives its V row to FP32 rounding
     B, Hkv, G, k = 3, 1, 8, 8
