@@ -140,11 +140,26 @@ class Workload:
                     self.geo, win["q"], K, V, self.table, self.lens_flat, win["ws"], draft_out=win["draft"],
                     atol=0.5, rtol=0.1, causal=True, out_full=win["out_full"],
                     first_reject=win["first_reject"], dev=win["dev"]))
-                n += win["k"] + 1
+                n += win["k"] + self.verify_kernels(win["k"])
         return n
 
+    def verify_kernels(self, k):
+        """Kernels of one merge-verify call: one attention launch per slice of the window (the library takes up
+        to 16 columns per launch on the integer kernel and runs 17..32 columns as two such passes; up to 16
+        positions and 64 columns on the FP16 kernel), plus the decision kernel when there is more than one."""
+        G = self.wl.num_q_heads // self.wl.num_kv_heads
+        cols = k * G
+        if 16 < cols <= 32 and 16 // G > 0:
+            per = 16 // G
+        elif k <= 16 and cols <= 64:
+            per = k
+        else:
+            per = min(16, max(1, 64 // G))
+        slices = -(-k // per)
+        return slices + (1 if slices > 1 else 0)
+
     def launches_per_step(self):
-        return 2 + sum(w["reps"] * (w["k"] + 1) for w in self.windows)
+        return 2 + sum(w["reps"] * (w["k"] + self.verify_kernels(w["k"])) for w in self.windows)
 
     def bytes_per_step(self):
         b = 2 * self.launch_rows["split_quantize"] * BYTES_PER_ROW["split_quantize"]

@@ -106,7 +106,7 @@ lynx_status lynx_recombine(const uint8_t* anchor, const uint8_t* residual, const
  * use (lynx_workspace_init, or cudaMemsetAsync of the whole buffer); each call leaves it ready
  * for the next.  Calls sharing a workspace must be ordered on one stream.
  * A buffer smaller than this figure is rejected by the attention calls (LYNX_ERR_WORKSPACE): nothing
- * degrades silently.  For verification with more than 16 columns (k * Hq/Hkv in 17..64) the figure
+ * degrades silently.  For verification with more than 32 columns (k * Hq/Hkv in 33..64) the figure
  * includes about 19 MB for FP32 copies of the accumulators of the FP16 tensor-core kernels used there
  * (their accumulation chains are cut every 256 units of 64 tokens, which bounds what the tensor
  * cores lose by truncating when they accumulate, whatever the context length).  Anchor attention and
@@ -139,12 +139,13 @@ lynx_status lynx_anchor_attention(const lynx_shape* shape, const void* q_bf16, i
  * prefix; out_full at that position is the correction).
  * draft_out : [batch][k][Hq][128] float, the Anchor-state results being verified; may be NULL,
  * then dev / first_reject are not written (and may be NULL).  out_full : same shape, float.
- * k must be <= 64.  A launch takes up to 16 positions and 64 columns k * (Hq/Hkv); a longer window runs as
- * slices of whole positions (a pass over the planes each), and first_reject is then taken over the whole
- * window from the deviations.  With 17..64 columns per launch the weights are FP16 numbers: a value
- * row whose scale reaches 16 (a range of 4080 or more) would overflow them; such rows are recorded
+ * k must be <= 64.  Up to 16 columns k * (Hq/Hkv) are one launch of the exact integer kernel and 17..32 two
+ * passes of it; 33..64 columns (up to 16 positions) are one launch of a kernel whose weights are FP16
+ * numbers; a longer window runs as slices of whole positions (a pass over the planes each).  With several
+ * launches first_reject is taken over the whole window from the deviations.  In the FP16 kernel a value
+ * row whose scale reaches 16 (a range of 4080 or more) would overflow the weights; such rows are recorded
  * in the status word and lynx_check returns LYNX_ERR_RANGE (the outputs of that call are then not
- * to be used).  Up to 16 columns there is no such limit. */
+ * to be used).  Up to 32 columns there is no such limit. */
 lynx_status lynx_merge_verify_attention(const lynx_shape* shape, const void* q_bf16,
                                         int32_t batch, int32_t k, int32_t causal, lynx_plane K,
                                         lynx_plane V, const int32_t* block_table,

@@ -11,15 +11,15 @@
 //     q . K^_t        = scale_t * (q . level_t) + zero_t * sum_d q_d
 //     sum_t p_t V^_t  = sum_t (p_t scale_t) level_t + (sum_t p_t zero_t) * 1
 // so the two contractions run on the integer levels and the scalars are applied per token
-// outside.  Anchor attention (any column count) and verification with up to 16 columns run both
-// contractions as exact integer products on tcgen05.mma kind::i8 (attention_i8.cuh);
-// verification with 17..64 columns runs them on tcgen05.mma kind::f16 with two-term FP16
-// weights (attention_wide.cuh).
+// outside.  Anchor attention (any column count) and verification with up to 16 columns per launch
+// (17..32 columns: two such launches) run both contractions as exact integer products on
+// tcgen05.mma kind::i8 (attention_i8.cuh); verification with 33..64 columns per launch runs them on
+// tcgen05.mma kind::f16 with two-term FP16 weights (attention_wide.cuh).
 //
 // Common shape.  Persistent grid, one CTA per SM, flash-decoding split-K in stream-K form: the
 // (sequence, KV head, stage-unit) list is cut into equal contiguous ranges, one per CTA.
 // Producer warps stream 16-token sub-blocks of the planes (1 KiB each, contiguous in the paged
-// layout) into a shared-memory ring with cp.async.bulk (TMA, 1-D) completing on mbarriers, and
+// layout) into a shared-memory ring with bulk copies (TMA) completing on mbarriers, and
 // the queries of each piece into one of two slots.
 // A range that covers a whole (sequence, KV head) writes the output directly, otherwise the
 // partial (m, l, O) goes to the workspace and the last contributor (atomic ticket, no waiting)
@@ -441,6 +441,9 @@ constexpr int kMaxCtasPerSm = 4;
 // Query positions per launch of a verification call: all of them up to kMaxQ positions and kMaxCols
 // columns, else as many whole positions as fit both.
 inline int verify_slice(int nq, int G) {
+  // (17..32 columns: two passes of the exact integer kernel at 16 columns measure as fast as one pass of the
+  // FP16 kernel at 32, without its limits on the value range)
+  if (nq * G > 16 && nq * G <= 32 && 16 / G > 0) return 16 / G;
   if (nq <= kMaxQ && nq * G <= kMaxCols) return nq;
   const int by_cols = kMaxCols / G > 0 ? kMaxCols / G : 1;
   return by_cols < kMaxQ ? by_cols : kMaxQ;
@@ -470,7 +473,10 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   if ((int64_t)s->num_blocks * s->num_kv_heads * s->block_tokens >= (1ll << 32)) return false;
   pl->ncols = ncols;
   pl->variant = ncols <= 8 ? 0 : ncols <= 16 ? 1 : ncols <= 32 ? 2 : 3;
-  pl->cols_pad = ncols <= 8 ? 8 : ncols <= 16 ? 16 : ncols <= 32 ? 32 : 64;
+  // (the partial slots also serve anchor calls on the same workspace, which take up to 32 columns per launch)
+  const int cols_anchor = nq * G <= 32 ? nq * G : (32 / G > 0 ? 32 / G : 1) * G;
+  const int cols_max = ncols > cols_anchor ? ncols : cols_anchor;
+  pl->cols_pad = cols_max <= 8 ? 8 : cols_max <= 16 ? 16 : cols_max <= 32 ? 32 : 64;
   size_t off = kWsHeaderBytes;
   pl->off_chunk_ctr = off; off += (size_t)B * s->num_kv_heads * 4;
   pl->off_seq_ctr = off;   off += (size_t)B * 4;
@@ -481,10 +487,9 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   pl->off_part = off;
   off += ((size_t)B * s->num_kv_heads + (size_t)sm_count() * kMaxCtasPerSm) * pl->cols_pad * kPartStride * 4;
   pl->bytes = (off + 255) & ~(size_t)255;
-  // mma.sync kernels: one O slice per consumer warp, 16 KB per CTA (64 KB with 64 columns, one CTA per
-  // SM); tcgen05 kernels: 2 groups x 128 rows x 128 dims per CTA
-  // (only the FP16 kernels have them: verification with 17..64 columns, anchor attention with 33..64)
-  pl->shadow_bytes = ncols > 16 ? (size_t)sm_count() * 131072 : 0;
+  // FP32 copies of the accumulators of the FP16 kernel (verification with 33..64 columns per launch):
+  // 2 groups x 128 rows x 128 dims per CTA
+  pl->shadow_bytes = ncols > 32 ? (size_t)sm_count() * 131072 : 0;
   return true;
 }
 
@@ -521,7 +526,7 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
     return LYNX_ERR_ALIGN;
   // the FP16 kernels cut their accumulation chains into FP32 copies at the end of the workspace; the
   // fixed-scratch entry point has no room for them and says so in its contract
-  const bool fp16_kernel = full && pl.ncols > 16;   // (pl.ncols: the columns of the widest launch)
+  const bool fp16_kernel = full && pl.ncols > 32;   // (pl.ncols: the columns of the widest launch)
   const bool use_shadow = fp16_kernel && !fixed_scratch;
   if (workspace_bytes < pl.bytes + (use_shadow ? pl.shadow_bytes : 0)) return LYNX_ERR_WORKSPACE;
   if (full && draft && !(atol > 0.0f && rtol >= 0.0f)) return LYNX_ERR_SHAPE;
@@ -581,8 +586,7 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
     ps.out = p.out + (size_t)j0 * p.Hq * LYNX_D;
     if (p.draft) { ps.draft = p.draft + (size_t)j0 * p.Hq * LYNX_D; ps.dev = p.dev + j0; }
     const lynx_status rc = ps.ncols <= 4 ? launch_i8<true, 4>(ps, st) : ps.ncols <= 8 ? launch_i8<true, 8>(ps, st)
-                         : ps.ncols <= 16 ? launch_i8<true, 16>(ps, st)
-                         : ps.ncols <= 32 ? launch_wide<2, 2>(ps, st) : launch_wide<2, 1>(ps, st);
+                         : ps.ncols <= 16 ? launch_i8<true, 16>(ps, st) : launch_wide<2, 1>(ps, st);
     if (rc != LYNX_OK) return rc;
   }
   if (p.draft && pl.per < nq) {

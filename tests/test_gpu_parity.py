@@ -330,12 +330,12 @@ def test_long_context_multi_chunk_sampled(lynx):
     _close(out_v.cpu().numpy().astype(np.float64), ref_v, "verify 40k")
 
 
-# ------------------------------------------------------ verify with 17..64 columns (tcgen05 path)
+# ----------- verify with 17..64 columns (17..32: two passes of the integer kernel; 33..64: the FP16 tcgen05 kernel)
 WIDE_CASES = [
     # B, Hkv, G, k, lens, bt, recipe
-    (4, 2, 4, 8, (1, 15, 17, 0), 16, "student_t4"),              # 32 columns: tiny, ragged and empty sequences
+    (4, 2, 4, 8, (1, 15, 17, 0), 16, "student_t4"),              # 32 columns (two slices): tiny, ragged and empty sequences
     (2, 2, 8, 8, (63, 130), 16, "normal_outlier2pct_x10"),       # 64 columns around one and two 64-token units
-    (1, 2, 4, 5, (700,), 32, "lognormal_channels"),              # 20 columns, padded to 32
+    (1, 2, 4, 5, (700,), 32, "lognormal_channels"),              # 20 columns: slices of 4 positions + 1
     (1, 2, 8, 5, (333,), 16, "normal_outlier4x8"),               # 40 columns, padded to 64
     (1, 1, 3, 11, (513,), 16, "normal"),                         # 33 columns, group of 3, 11 positions
     (3, 1, 16, 4, (64, 128, 65), 64, "student_t4"),              # 64 columns from G = 16, exact unit multiples
@@ -625,7 +625,7 @@ def _scaled_value_case(lynx, seed, G, k, vscale):
 def test_value_rows_of_any_range_on_the_integer_kernels(lynx, vscale):
     # the integer kernels fold log2(scale_v) into the weights' exponent, so the magnitude of the V rows
     # (here ranges of ~1e-2, ~3000 and ~1e31) does not matter: relative accuracy as for ordinary rows
-    for G, k, full in ((4, 1, False), (4, 4, False), (8, 8, False), (4, 2, True), (4, 4, True)):
+    for G, k, full in ((4, 1, False), (4, 4, False), (8, 8, False), (4, 2, True), (4, 4, True), (4, 8, True)):
         c = _scaled_value_case(lynx, 8300 + k, G, k, vscale)
         qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
         ref = oracle.attention(full, bf16_bits(c["q"]), c["kp"], c["vp"], c["table"].numpy(), c["lens"].numpy(),
@@ -642,10 +642,10 @@ def test_value_rows_of_any_range_on_the_integer_kernels(lynx, vscale):
 
 
 def test_value_range_limit_of_the_fp16_verify_kernels_is_reported(lynx):
-    # merge-verify with 17..64 columns carries the weights in FP16: value rows whose scale reaches 16 (a
-    # range above 4080) would overflow them.  Just below the limit the result is within tolerance; above
-    # it lynx_check reports LYNX_ERR_RANGE instead of a silent Inf / NaN.
-    G, k = 4, 8
+    # merge-verify with 33..64 columns per launch carries the weights in FP16: value rows whose scale reaches
+    # 16 (a range above 4080) would overflow them.  Just below the limit the result is within tolerance;
+    # above it lynx_check reports LYNX_ERR_RANGE instead of a silent Inf / NaN.
+    G, k = 8, 8
     c = _scaled_value_case(lynx, 8400, G, k, 400.0)      # ranges ~3000: scale_v ~ 12
     qd, td, ld = c["q"].cuda(), c["table"].cuda(), c["lens"].cuda()
     assert float(c["vp"][2][..., 0].max()) < 16.0
