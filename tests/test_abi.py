@@ -39,6 +39,8 @@ def test_host_side_validation_needs_no_gpu():
     assert lynx.workspace_bytes(geo, 1, 4) > lynx.workspace_bytes(geo, 1, 1)
     assert lynx.workspace_bytes(lynx.Geometry(32, 8, 16, 1024, 64, head_dim=64), 1, 1) == 0
     assert lynx.workspace_bytes(lynx.Geometry(32, 8, 24, 1024, 64), 1, 1) == 0      # block_tokens % 16
-    assert lynx.workspace_bytes(lynx.Geometry(32, 8, 16, 1024, 64), 1, 17) == 0     # too many positions
-    assert lynx.workspace_bytes(lynx.Geometry(64, 8, 16, 1024, 64), 1, 16) == 0     # 128 columns
+    assert lynx.workspace_bytes(lynx.Geometry(32, 8, 16, 1024, 64), 1, 65) == 0     # too many positions
+    assert lynx.workspace_bytes(lynx.Geometry(32, 8, 16, 1024, 64), 1, 64) > 0      # the window cap (in slices)
+    assert lynx.workspace_bytes(lynx.Geometry(64, 8, 16, 1024, 64), 1, 16) > 0      # 128 columns: two slices
+    assert lynx.workspace_bytes(lynx.Geometry(8 * 17, 8, 16, 1024, 64), 1, 1) == 0  # more than 16 q heads per KV head
     assert lynx.workspace_bytes(lynx.Geometry(30, 8, 16, 1024, 64), 1, 1) == 0      # Hq % Hkv
