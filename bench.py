@@ -288,7 +288,7 @@ def oracle_sample(cfg_id: int, k_list=None):
 # (dram__bytes_read.sum + dram__bytes_write.sum over 72 / 136 / 392 B per row; captures on an
 # 8-layer copy of config 3, summarised under profiles/).  Traffic grows in proportion to the
 # rows a launch processes, so a full launch is scaled by the rows.
-TRAFFIC_RATIO = {"anchor_attention": 1.010, "merge_verify_attention": 1.005, "split_quantize": 0.990}
+TRAFFIC_RATIO = {"anchor_attention": 1.005, "merge_verify_attention": 1.005, "split_quantize": 0.990}
 
 
 def base_kind(kind: str) -> str:
