@@ -463,6 +463,7 @@ def main():
         line["bf16_pages"] = run_bf16_pages(wlk, peak)
         line["hierarchical"] = run_hier(wlk, peak)
         line["progressive"] = run_progressive(wlk)
+        line["token_verify"] = run_token_verify(wlk, peak)
     if rank == 0 and world == 1 and not args.no_e2e:
         line["e2e"] = run_e2e(wlk, args.e2e_steps, step_bytes)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -555,6 +556,38 @@ def run_progressive(wlk: "Workload", max_layers: int = 8, cap: int = 64, k: int 
             "drafting_ended_ms": t_draft_end * 1e3, "overlapped_total_ms": t_total * 1e3, "one_after_the_other_ms": serial * 1e3,
             "transfer_hidden_frac": min(1.0, n * t_step / t_h2d) if t_h2d > 0 else None,
             "residual_arrived_intact": ok, "timing": "host wall clock around synchronised steps (context only)"}
+
+
+def run_token_verify(wlk: "Workload", peak: float, batch: int = 256, k: int = 8, vocab: int = 128256):
+    """Context: token-level verification (Section 4.3) of `batch` windows of k drafts over a Llama-3-sized
+    vocabulary; synthetic distributions, the uniforms supplied.  Not part of `value`."""
+    lynx = wlk.lynx
+    g = torch.Generator(device=wlk.device)
+    g.manual_seed(1234)
+    logits = torch.randn(batch, k + 1, vocab, generator=g, device=wlk.device) * 3.0
+    q = torch.softmax(logits, -1)
+    p = torch.softmax(logits[:, :k] + 0.3 * torch.randn(batch, k, vocab, generator=g, device=wlk.device), -1)
+    del logits
+    s = torch.multinomial(p.view(-1, vocab), 1, generator=g).view(batch, k).to(torch.int32)
+    u = torch.rand(batch, k, generator=g, device=wlk.device)
+    r = torch.rand(batch, generator=g, device=wlk.device)
+    for _ in range(3):
+        n_acc, nxt = lynx.token_verify(p, q, s, u, r)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 20
+    e0.record()
+    for _ in range(reps):
+        n_acc, nxt = lynx.token_verify(p, q, s, u, r)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    # bytes that must move: one or two vocabulary rows per window (the correction or the bonus row), read twice
+    # at worst by the slice sums and the walk of one slice; counted once
+    rows = int((n_acc < k).sum().item()) * 2 + int((n_acc == k).sum().item())
+    gb = rows * vocab * 4 / (ms * 1e-3) / 1e9
+    return {"windows": batch, "k": k, "vocab": vocab, "ms": ms, "mean_accepted": float(n_acc.float().mean().item()),
+            "bytes": rows * vocab * 4, "GBps": gb, "frac_of_measured": gb / peak}
 
 
 def run_hier(wlk: "Workload", peak: float, max_pages: int = 16384):

@@ -195,6 +195,22 @@ lynx_status lynx_hier_dequantize(const uint8_t* q_anc, const uint8_t* q_res, int
                                  const float* gamma_min, const float* gamma_scale, const float* mu,
                                  const float* sigma, void* dst_bf16, void* stream);
 
+/* Token-level verification of a speculated window (Section 4.3; the acceptance rule of speculative sampling
+ * the paper builds on, Section 2.4).  The k draft tokens s_i were drawn from the Anchor-state distributions
+ * p_i; the verification pass yields the distributions q_1 .. q_{k+1}.  Token i is accepted iff
+ * u_i * p_i(s_i) < q_i(s_i), i.e. with probability min(1, q_i(s_i) / p_i(s_i)); n_accepted[b] is the length of
+ * the accepted prefix.  next_token[b] is the correction drawn from norm(max(0, q_j - p_j)) at the first
+ * rejected position j (from q_j itself should that residual be zero everywhere), or the bonus token drawn
+ * from q_{k+1} when all k are accepted: the smallest vocabulary index whose cumulative weight exceeds
+ * r[b] * total.  The outputs are then distributed as samples of q alone.
+ * p_probs : float [batch][k][vocab]; q_probs : float [batch][k+1][vocab]; draft_tokens : int32 [batch][k]
+ * (clamped to the vocabulary); u : float [batch][k] and r : float [batch], uniform in [0, 1), supplied by the
+ * caller; n_accepted, next_token : int32 [batch].  1 <= k <= 64.  Sums are FP32: a decision within rounding
+ * of its threshold may differ from a higher-precision evaluation. */
+lynx_status lynx_token_verify(const float* p_probs, const float* q_probs, const int32_t* draft_tokens,
+                              const float* u, const float* r, int32_t batch, int32_t k, int32_t vocab,
+                              int32_t* n_accepted, int32_t* next_token, void* stream);
+
 /* Decode attention over dequantised BF16 pages: the path the paper itself describes (Section 4.2: the
  * dequantisation kernel scatters BF16 pages into the paged KV memory, the engine's attention reads
  * them; Section 2 attention equation), here as the baseline the fused calls above are measured

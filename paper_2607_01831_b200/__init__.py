@@ -39,6 +39,7 @@ class _Shape(ctypes.Structure):
 EXPORTS = ["lynx_split_quantize", "lynx_recombine", "lynx_workspace_bytes", "lynx_workspace_init",
            "lynx_anchor_attention", "lynx_merge_verify_attention", "lynx_anchor_attention_static",
            "lynx_bf16_workspace_bytes", "lynx_bf16_attention", "lynx_hier_quantize", "lynx_hier_dequantize",
+           "lynx_token_verify",
            "lynx_check",
            "lynx_status_string", "lynx_version"]
 
@@ -84,6 +85,8 @@ def load():
     lib.lynx_hier_quantize.restype = ctypes.c_int
     lib.lynx_hier_dequantize.argtypes = [vp, vp, i64, vp, vp, vp, vp, vp, vp]
     lib.lynx_hier_dequantize.restype = ctypes.c_int
+    lib.lynx_token_verify.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
+    lib.lynx_token_verify.restype = ctypes.c_int
     lib.lynx_check.argtypes = [vp, vp]
     lib.lynx_check.restype = ctypes.c_int
     lib.lynx_status_string.argtypes = [ctypes.c_int]
@@ -311,3 +314,24 @@ def hier_dequantize(h: HierPlanes, anchor_only: bool = False, out: torch.Tensor 
                                     _ptr(h.gamma_scale), _ptr(h.mu), _ptr(h.sigma), _ptr(out), _stream()),
         "lynx_hier_dequantize")
     return out
+
+
+def token_verify(p_probs: torch.Tensor, q_probs: torch.Tensor, draft_tokens: torch.Tensor, u: torch.Tensor,
+                 r: torch.Tensor):
+    """lynx_token_verify: p_probs f32 [B][k][V], q_probs f32 [B][k+1][V], draft_tokens i32 [B][k], u f32 [B][k],
+    r f32 [B] -> (n_accepted i32 [B], next_token i32 [B])."""
+    B, k, V = p_probs.shape
+    if tuple(q_probs.shape) != (B, k + 1, V) or p_probs.dtype != torch.float32 or q_probs.dtype != torch.float32:
+        raise LynxError("p_probs must be float32 [B][k][V], q_probs float32 [B][k+1][V]")
+    if draft_tokens.dtype != torch.int32 or tuple(draft_tokens.shape) != (B, k):
+        raise LynxError("draft_tokens must be int32 [B][k]")
+    if u.dtype != torch.float32 or tuple(u.shape) != (B, k) or r.dtype != torch.float32 or tuple(r.shape) != (B,):
+        raise LynxError("u must be float32 [B][k], r float32 [B]")
+    for t in (p_probs, q_probs, draft_tokens, u, r):
+        if not t.is_contiguous():
+            raise LynxError("contiguous tensors required")
+    n_acc = torch.empty(B, dtype=torch.int32, device=p_probs.device)
+    nxt = torch.empty(B, dtype=torch.int32, device=p_probs.device)
+    _ok(load().lynx_token_verify(_ptr(p_probs), _ptr(q_probs), _ptr(draft_tokens), _ptr(u), _ptr(r), B, k, V,
+                                 _ptr(n_acc), _ptr(nxt), _stream()), "lynx_token_verify")
+    return n_acc, nxt
