@@ -445,7 +445,7 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "u8 x s8 -> s32 (Q.K^T) and u8 x u8 -> s32 (P.V) on tcgen05 kind::i8; f16 -> f32 on tcgen05 for verify with 17..64 columns; f32 softmax and quantiser",
+        "vs_baseline": None, "dtype": "u8 x s8 -> s32 (Q.K^T) and u8 x u8 -> s32 (P.V) on tcgen05 kind::i8; f16 -> f32 on tcgen05 for verify with 33..64 columns per launch; f32 softmax and quantiser",
         "data": "synthetic",
         "config": {"workload": wl.name, "layers": wl.layers, "batch": wl.batch, "context": wl.context,
                    "num_kv_heads": wl.num_kv_heads, "num_q_heads": wl.num_q_heads, "k": list(wl.k_list),
