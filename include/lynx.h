@@ -205,8 +205,9 @@ lynx_status lynx_hier_dequantize(const uint8_t* q_anc, const uint8_t* q_res, int
  * r[b] * total.  The outputs are then distributed as samples of q alone.
  * p_probs : float [batch][k][vocab]; q_probs : float [batch][k+1][vocab]; draft_tokens : int32 [batch][k]
  * (clamped to the vocabulary); u : float [batch][k] and r : float [batch], uniform in [0, 1), supplied by the
- * caller; n_accepted, next_token : int32 [batch].  1 <= k <= 64.  Sums are FP32: a decision within rounding
- * of its threshold may differ from a higher-precision evaluation. */
+ * caller; n_accepted, next_token : int32 [batch].  1 <= k <= 64; vocab <= 1572864 (LYNX_ERR_UNSUPPORTED
+ * beyond).  Sums are FP32: a decision within rounding of its threshold may differ from a higher-precision
+ * evaluation. */
 lynx_status lynx_token_verify(const float* p_probs, const float* q_probs, const int32_t* draft_tokens,
                               const float* u, const float* r, int32_t batch, int32_t k, int32_t vocab,
                               int32_t* n_accepted, int32_t* next_token, void* stream);
