@@ -40,14 +40,26 @@ __device__ __forceinline__ uint32_t bf2max(uint32_t a, uint32_t b) {
   return d;
 }
 
+// Two FP32 values in a register pair, one instruction for both (IEEE round-to-nearest per element, as the
+// scalar forms)
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
 // Codes of 8 consecutive elements (4 BF16 pairs in w) -> 4 bytes of each nibble plane.
 __device__ __forceinline__ void codes8(const uint32_t (&w)[4], float mn, float inv, uint32_t& a,
                                        uint32_t& r) {
   uint32_t c[8];
+  const uint64_t mn2 = pack2(mn, mn), inv2 = pack2(inv, inv), magic2 = pack2(12582912.0f, 12582912.0f);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    c[2 * i] = code_bits(__uint_as_float(w[i] << 16), mn, inv);
-    c[2 * i + 1] = code_bits(__uint_as_float(w[i] & 0xFFFF0000u), mn, inv);
+    // (x - mn) rounded, then fma(u, inv, 1.5 * 2^23): the two elements of a word at once
+    const uint64_t x2 = pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u));
+    uint64_t u2, y2;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(u2) : "l"(x2), "l"(mn2));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(y2) : "l"(u2), "l"(inv2), "l"(magic2));
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(c[2 * i]), "=r"(c[2 * i + 1]) : "l"(y2));
   }
   // low bytes gathered: w0 = codes 0..3, w1 = codes 4..7
   const uint32_t w0 = __byte_perm(__byte_perm(c[0], c[1], 0x0040), __byte_perm(c[2], c[3], 0x0040), 0x5410);
