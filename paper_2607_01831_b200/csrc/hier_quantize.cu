@@ -45,18 +45,36 @@ __device__ __forceinline__ uint32_t bf2_max(uint32_t a, uint32_t b) {
   return d;
 }
 
-// Stages 3 and 4 for one element: x_final = fma(x, A, B) (stages 1 and 2 folded into one multiply-add), the
-// alpha-law magnitude y = log2(1 + 255 |x_final|) * 15 rounded to the nearest even integer I (0..120) by the
-// magic-number addition, whose sum keeps I in its low mantissa bits.  Returned: (I + 7) ^ sign mask, whose
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+// Stages 3 and 4 for the two channels of a word (the multiply-adds as packed FP32 pairs):
+// x_final = fma(x, A, B) (stages 1 and 2 folded into one multiply-add), the alpha-law magnitude
+// y = log2(1 + 255 |x_final|) * 15 rounded to the nearest even integer I (0..120) by the magic-number
+// addition, whose sum keeps I in its low mantissa bits.  Returned per channel: (I + 7) ^ sign mask, whose
 // bits 4..7 are the Anchor nibble (v_mag = (I + 7) >> 4; two's complement -v_mag - 1 = ~v_mag for negative
 // values), and -I, whose low nibble is the Residual (16 v_mag - I modulo 16).
-__device__ __forceinline__ void hier_code(float x, float A, float B, uint32_t& anc4, uint32_t& negI) {
-  const float t = fmaf(x, A, B);
-  float lg;
-  asm("lg2.approx.f32 %0, %1;" : "=f"(lg) : "f"(fmaf(kAlpha, fabsf(t), 1.0f)));
-  const uint32_t r = __float_as_uint(fmaf(lg, kYmax / kLog2_1pAlpha, 12582912.0f));   // 0x4B400000 + I
-  anc4 = (r + 7u) ^ (uint32_t)(__float_as_int(t) >> 31);
-  negI = 0u - r;                                                                       // low byte: -I modulo 256
+__device__ __forceinline__ void hier_code2(uint32_t w, uint64_t A2, uint64_t B2, uint32_t& anc4_0, uint32_t& negI_0,
+                                           uint32_t& anc4_1, uint32_t& negI_1) {
+  const uint64_t x2 = pack2(lo_bf16(w), hi_bf16(w));
+  uint64_t t2;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(t2) : "l"(x2), "l"(A2), "l"(B2));
+  float t0, t1;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(t0), "=f"(t1) : "l"(t2));
+  float l0, l1;
+  asm("lg2.approx.f32 %0, %1;" : "=f"(l0) : "f"(fmaf(kAlpha, fabsf(t0), 1.0f)));
+  asm("lg2.approx.f32 %0, %1;" : "=f"(l1) : "f"(fmaf(kAlpha, fabsf(t1), 1.0f)));
+  uint64_t r2;
+  const uint64_t k2 = pack2(kYmax / kLog2_1pAlpha, kYmax / kLog2_1pAlpha), m2 = pack2(12582912.0f, 12582912.0f);
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r2) : "l"(pack2(l0, l1)), "l"(k2), "l"(m2));
+  uint32_t r0, r1;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(r0), "=r"(r1) : "l"(r2));   // 0x4B400000 + I
+  anc4_0 = (r0 + 7u) ^ (uint32_t)(__float_as_int(t0) >> 31);
+  anc4_1 = (r1 + 7u) ^ (uint32_t)(__float_as_int(t1) >> 31);
+  negI_0 = 0u - r0;
+  negI_1 = 0u - r1;
 }
 
 // One CTA per page: the page (64 KB) is staged in shared memory; a thread owns a channel pair (one 32-bit word
@@ -131,14 +149,14 @@ __global__ void __launch_bounds__(256, 3) hier_quantize_kernel(const __nv_bfloat
       // x_final = ((x - gmin) inv - mu) / (sigma + eps) = (x - mean) * A
       const float A0 = inv.x / (sg0 + kEps), A1 = inv.y / (sg1 + kEps);
       const float B0 = -mean0 * A0, B1 = -mean1 * A1;
+      const uint64_t A2 = pack2(A0, A1), B2 = pack2(B0, B1);
       uint8_t* pa = q_anc + ((size_t)pg * kP + ch * kC) * 64 + pr;
       uint8_t* pr_ = q_res + ((size_t)pg * kP + ch * kC) * 64 + pr;
 #pragma unroll 8
       for (int t = 0; t < kC; ++t) {
         const uint32_t w = page[(ch * kC + t) * 64 + pr];
         uint32_t a0, n0, a1, n1;
-        hier_code(lo_bf16(w), A0, B0, a0, n0);
-        hier_code(hi_bf16(w), A1, B1, a1, n1);
+        hier_code2(w, A2, B2, a0, n0, a1, n1);
         pa[(size_t)t * 64] = (uint8_t)lop3_sel(a0 >> 4, a1, 0x0Fu);
         pr_[(size_t)t * 64] = (uint8_t)lop3_sel(n0, n1 << 4, 0x0Fu);
       }
