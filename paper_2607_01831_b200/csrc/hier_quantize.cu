@@ -87,8 +87,8 @@ __device__ __forceinline__ void hier_code2(uint32_t w, uint64_t A2, uint64_t B2,
   float f0, f1;
   unpack2(t2, f0, f1);
   float l0, l1;
-  asm("lg2.approx.f32 %0, %1;" : "=f"(l0) : "f"(fmaf(kAlpha, fabsf(f0), 1.0f)));
-  asm("lg2.approx.f32 %0, %1;" : "=f"(l1) : "f"(fmaf(kAlpha, fabsf(f1), 1.0f)));
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l0) : "f"(fmaf(kAlpha, fabsf(f0), 1.0f)));
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l1) : "f"(fmaf(kAlpha, fabsf(f1), 1.0f)));
   const uint64_t k2 = pack2(kYmax / kLog2_1pAlpha, kYmax / kLog2_1pAlpha), m2 = pack2(12582919.0f, 12582919.0f);
   const uint64_t r2 = f2_fma(pack2(l0, l1), k2, m2);   // 0x4B400007 + I
   asm("mov.b64 {%0, %1}, %2;" : "=r"(r0), "=r"(r1) : "l"(r2));
@@ -269,15 +269,17 @@ __global__ void __launch_bounds__(256, 3) hier_quantize_kernel(const __nv_bfloat
 // the table indices of four channels at a time by one bit-select, eight look-ups, four packed multiply-adds, one
 // 16-byte store.
 template <bool FULL>
-__global__ void __launch_bounds__(128) hier_dequantize_kernel(const uint8_t* __restrict__ q_anc,
+__global__ void __launch_bounds__(128, FULL ? 4 : 6) hier_dequantize_kernel(const uint8_t* __restrict__ q_anc,
                                                               const uint8_t* __restrict__ q_res, int n_pages,
                                                               const float* __restrict__ g_min,
                                                               const float* __restrict__ g_scale,
                                                               const float* __restrict__ mu,
                                                               const float* __restrict__ sigma,
                                                               __nv_bfloat16* __restrict__ dst) {
-  constexpr int kEntries = FULL ? 256 : 16;
-  __shared__ float table[kEntries];
+  // FULL: every lane has its own copy of the 256 entries (entry e of lane l at e * 32 + l), so that the eight
+  // look-ups of a token never meet in a bank; the 16 entries of the Anchor-only case sit in 16 banks anyway.
+  constexpr int kEntries = FULL ? 256 : 16, kCopies = FULL ? 32 : 1;
+  __shared__ float table[kEntries * kCopies];
   const int tid = threadIdx.x;
   for (int e = tid; e < kEntries; e += 128) {
     const int i = FULL ? e : e << 4;
@@ -285,9 +287,14 @@ __global__ void __launch_bounds__(128) hier_dequantize_kernel(const uint8_t* __r
     const int v_mag = qa < 0 ? -qa - 1 : qa;
     const int I = (v_mag << 4) - qr;
     const float mag = (exp2f((float)I * (kLog2_1pAlpha / kYmax)) - 1.0f) * (1.0f / kAlpha);
-    table[e] = qa < 0 ? -mag : mag;
+    table[e * kCopies] = qa < 0 ? -mag : mag;
   }
   __syncthreads();
+  if (FULL) {
+    for (int i = tid; i < kEntries * kCopies; i += 128) table[i] = table[i & ~(kCopies - 1)];
+    __syncthreads();
+  }
+  const uint32_t lane4 = (uint32_t)(tid & 31) << 2;
   const int ch = tid >> 4, oc = tid & 15;                                     // chunk, octet of channels
   constexpr int kB = 8;                                                       // tokens per batch of loads
   for (int pg = blockIdx.x; pg < n_pages; pg += gridDim.x) {
@@ -335,7 +342,16 @@ __global__ void __launch_bounds__(128) hier_dequantize_kernel(const uint8_t* __r
         uint32_t o[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const float x0 = table[(L >> (8 * j)) & 0xFFu], x1 = table[(H >> (8 * j)) & 0xFFu];
+          float x0, x1;
+          if (FULL) {   // byte offset of entry e of this lane: e * 128 + lane * 4, one shift and one bit-select
+            const uint32_t o0 = lop3_sel(j == 0 ? L << 7 : L >> (8 * j - 7), lane4, 0x7F80u);
+            const uint32_t o1 = lop3_sel(j == 0 ? H << 7 : H >> (8 * j - 7), lane4, 0x7F80u);
+            x0 = *reinterpret_cast<const float*>(reinterpret_cast<const char*>(table) + o0);
+            x1 = *reinterpret_cast<const float*>(reinterpret_cast<const char*>(table) + o1);
+          } else {
+            x0 = table[(L >> (8 * j)) & 0xFFu];
+            x1 = table[(H >> (8 * j)) & 0xFFu];
+          }
           float y0, y1;
           unpack2(f2_fma(pack2(x0, x1), S2[j], T2[j]), y0, y1);
           asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[j]) : "f"(y1), "f"(y0));
