@@ -64,7 +64,7 @@ __device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
 }
 __device__ __forceinline__ float rcp_fast(float x) {
   float r;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
   return r;
 }
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
@@ -76,14 +76,17 @@ __device__ __forceinline__ void cp_async16(uint32_t saddr, const void* g) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(saddr), "l"(g) : "memory");
 }
 
-// Stages 3 and 4 for the two channels of a word (the multiply-adds as packed FP32 pairs):
-// x_final = fma(x, A, B) (stages 1 and 2 folded into one multiply-add), the alpha-law magnitude
+// Stages 3 and 4 for the two channels of a word (packed FP32 pairs): x_final = (x - mean) * A (stages 1 and 2
+// folded: the difference first, which is exact where it is small; one multiply-add x * A - mean * A would carry the
+// rounding of mean * A, a large error for a channel whose offset dwarfs its chunk deviation), the alpha-law magnitude
 // y = log2(1 + 255 |x_final|) * 15 rounded to the nearest even integer I (0..120) by the magic-number
 // addition, whose sum keeps the integer in its low mantissa bits; the magic number carries the +7 of stage 4,
 // so the low byte of r is J = I + 7 (7..127).  t keeps the sign of x_final.
-__device__ __forceinline__ void hier_code2(uint32_t w, uint64_t A2, uint64_t B2, uint32_t& r0, uint32_t& r1,
+__device__ __forceinline__ void hier_code2(uint32_t w, uint64_t A2, uint64_t M2, uint32_t& r0, uint32_t& r1,
                                            uint32_t& t0, uint32_t& t1) {
-  const uint64_t t2 = f2_fma(pack2(lo_bf16(w), hi_bf16(w)), A2, B2);
+  uint64_t d2, t2;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d2) : "l"(pack2(lo_bf16(w), hi_bf16(w))), "l"(M2));
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(t2) : "l"(d2), "l"(A2));
   float f0, f1;
   unpack2(t2, f0, f1);
   float l0, l1;
@@ -224,7 +227,7 @@ __global__ void __launch_bounds__(256, 3) hier_quantize_kernel(const __nv_bfloat
       reinterpret_cast<float4*>(dstp)[1] = make_float4(o[4], o[5], o[6], o[7]);
     }
     // x_final = ((x - gmin) inv - mu) / (sigma + eps) = (x - mean) * A,  A = inv / (sigma + eps)
-    uint64_t A2[4], B2[4];
+    uint64_t A2[4], M2[4];
     {
       float A[8];
 #pragma unroll
@@ -237,7 +240,7 @@ __global__ void __launch_bounds__(256, 3) hier_quantize_kernel(const __nv_bfloat
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         A2[j] = pack2(A[2 * j], A[2 * j + 1]);
-        B2[j] = pack2(-mean[2 * j] * A[2 * j], -mean[2 * j + 1] * A[2 * j + 1]);
+        M2[j] = pack2(mean[2 * j], mean[2 * j + 1]);
       }
     }
     // ---- stages 3 and 4: the codes of the thread's 16 tokens x 8 channels ---------------------------------------
@@ -249,7 +252,7 @@ __global__ void __launch_bounds__(256, 3) hier_quantize_kernel(const __nv_bfloat
       const uint32_t w[4] = {v.x, v.y, v.z, v.w};
       uint32_t r[8], s[8];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) hier_code2(w[j], A2[j], B2[j], r[2 * j], r[2 * j + 1], s[2 * j], s[2 * j + 1]);
+      for (int j = 0; j < 4; ++j) hier_code2(w[j], A2[j], M2[j], r[2 * j], r[2 * j + 1], s[2 * j], s[2 * j + 1]);
       uint32_t a_lo, r_lo, a_hi, r_hi;
       hier_nibbles4(r, s, a_lo, r_lo);
       hier_nibbles4(r + 4, s + 4, a_hi, r_hi);

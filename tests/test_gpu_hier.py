@@ -19,12 +19,38 @@ def _nib(packed):         # u8 [...,64] -> signed 4-bit values int [...,128]
     return np.where(v > 7, v - 16, v)
 
 
-@pytest.mark.parametrize("recipe,n_pages", [("normal_outlier4x8", 5), ("student_t4", 37), ("lognormal_channels", 300)])
+# 1000 pages: more than the quantiser's grid (three CTAs per SM), so CTAs walk through several pages
+@pytest.mark.parametrize("recipe,n_pages", [("normal_outlier4x8", 5), ("student_t4", 37), ("lognormal_channels", 300),
+                                            ("normal_outlier4x8", 1000)])
 def test_hier_quantize_and_dequantize_match_the_oracle(recipe, n_pages):
-    import paper_2607_01831_b200 as lynx
-    lynx.load()
     # pages of 256 tokens x 128 channels (one KV head each)
     x = synth.kv_block_values(recipe, n_pages, 1, 256, "cpu", "hier", n_pages).reshape(n_pages, 256, 128)
+    _check_against_oracle(x)
+
+
+def test_hier_degenerate_pages():
+    """Channels that are constant over a page or over a chunk (range / deviation 0: only epsilon keeps the
+    divisions finite), a single outlier in an otherwise constant channel, a page of zeros, negative zero,
+    values of very different magnitude in neighbouring channels."""
+    g = torch.Generator().manual_seed(11)
+    x = torch.randn(6, 256, 128, generator=g)
+    x[0, :, 0:8] = 3.25                      # constant over the page
+    x[0, :, 8] = -0.0
+    x[1, 64:96, 16:24] = -1.5                # constant over one chunk
+    x[1, :, 24] = 0.0
+    x[1, 200, 24] = 7.0                      # one outlier in a constant channel
+    x[2] = 0.0                               # a page of zeros
+    x[3, :, 0::2] *= 1.0e-3                  # small next to large: the two channels of a word
+    x[3, :, 1::2] *= 1.0e3
+    x[4] = torch.round(x[4] * 2.0) / 2.0     # many equal values, ties in the statistics
+    x[5, :, 40] = torch.linspace(-1.0, 1.0, 256)
+    _check_against_oracle(x.to(torch.bfloat16))
+
+
+def _check_against_oracle(x):
+    import paper_2607_01831_b200 as lynx
+    lynx.load()
+    n_pages = x.shape[0]
     got = lynx.hier_quantize(x.cuda())
     torch.cuda.synchronize()
     xf = bits_to_f64(bf16_bits(x))
