@@ -219,14 +219,35 @@ lynx_status lynx_token_verify(const float* p_probs, const float* q_probs, const 
  * k_pages_bf16, v_pages_bf16 : BF16 [num_blocks][Hkv][block_tokens][128], as lynx_recombine writes
  * them (dequant_bf16).  q_bf16, block_table, seq_lens, causal, softmax_scale, out as for
  * lynx_anchor_attention.  n_q * (Hq/Hkv) must be <= 8 (decode and short windows); any block_tokens.
- * workspace : lynx_bf16_workspace_bytes(shape, batch, n_q) bytes of scratch (split-K partials), no
- * initialisation needed.  Out-of-range block ids are clamped and not reported. */
+ * workspace : lynx_bf16_workspace_bytes(shape, batch, n_q) bytes of scratch (split-K partials and the rows'
+ * log-sum-exps), no initialisation needed.  Out-of-range block ids are clamped and not reported. */
 size_t lynx_bf16_workspace_bytes(const lynx_shape* shape, int32_t batch, int32_t n_q);
 lynx_status lynx_bf16_attention(const lynx_shape* shape, const void* q_bf16, int32_t batch, int32_t n_q,
                                 int32_t causal, const void* k_pages_bf16, const void* v_pages_bf16,
                                 const int32_t* block_table, const int32_t* seq_lens,
                                 float softmax_scale, float* out, void* workspace,
                                 size_t workspace_bytes, void* stream);
+
+/* A quantised prefix followed by a BF16 tail (no paper counterpart as a call; Section 4.2 keeps the tokens the
+ * decode node generates itself out of the quantiser, and Section 2's softmax runs over prefix and tail alike).
+ * Every attention call above leaves, next to its output, the natural-log log-sum-exp of each output row's scaled
+ * scores in its workspace: lse[b][j][h] = log sum_t exp(softmax_scale * q[b][j][h] . K_hat[t]) over the tokens the
+ * query saw, -inf where it saw none.  lynx_workspace_lse / lynx_bf16_workspace_lse return the DEVICE address of
+ * that array, float [batch][n_q][Hq], inside `workspace`, for the (shape, batch, n_q) of the call that wrote it
+ * (NULL for an unsupported shape or a NULL workspace); it is valid once that call has completed on its stream and
+ * until the next call on the workspace.  Nothing is launched, allocated or copied.
+ *
+ * lynx_lse_merge joins two results over disjoint key sets into the attention over their union:
+ *   out[r] = (e^lse_a[r] out_a[r] + e^lse_b[r] out_b[r]) / (e^lse_a[r] + e^lse_b[r]),  lse_out[r] = log of that sum,
+ * for n_rows rows of 128 floats (n_rows = batch * n_q * Hq for two attention calls on the same queries: the
+ * prefix through lynx_anchor_attention or lynx_merge_verify_attention, non-causal, the tail through
+ * lynx_bf16_attention, causal among the tail's own tokens).  A row with lse = -inf contributes nothing, whatever
+ * its out row holds; two such rows give zeros and -inf.  All pointers are DEVICE pointers; out_* and out 16-byte
+ * aligned; out may be out_a or out_b; lse_out may be NULL.  Asynchronous on `stream`. */
+const float* lynx_workspace_lse(const lynx_shape* shape, int32_t batch, int32_t n_q, const void* workspace);
+const float* lynx_bf16_workspace_lse(const lynx_shape* shape, int32_t batch, int32_t n_q, const void* workspace);
+lynx_status lynx_lse_merge(const float* out_a, const float* lse_a, const float* out_b, const float* lse_b,
+                           int64_t n_rows, float* out, float* lse_out, void* stream);
 
 /* Synchronises `stream`, reads and clears the workspace's status word.  Test / debug use. */
 lynx_status lynx_check(void* workspace, void* stream);

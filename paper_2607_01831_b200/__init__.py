@@ -39,7 +39,7 @@ class _Shape(ctypes.Structure):
 EXPORTS = ["lynx_split_quantize", "lynx_recombine", "lynx_workspace_bytes", "lynx_workspace_init",
            "lynx_anchor_attention", "lynx_merge_verify_attention", "lynx_anchor_attention_static",
            "lynx_bf16_workspace_bytes", "lynx_bf16_attention", "lynx_hier_quantize", "lynx_hier_dequantize",
-           "lynx_token_verify",
+           "lynx_token_verify", "lynx_workspace_lse", "lynx_bf16_workspace_lse", "lynx_lse_merge",
            "lynx_check",
            "lynx_status_string", "lynx_version"]
 
@@ -87,6 +87,12 @@ def load():
     lib.lynx_hier_dequantize.restype = ctypes.c_int
     lib.lynx_token_verify.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
     lib.lynx_token_verify.restype = ctypes.c_int
+    lib.lynx_workspace_lse.argtypes = [ctypes.POINTER(_Shape), i32, i32, vp]
+    lib.lynx_workspace_lse.restype = ctypes.c_void_p
+    lib.lynx_bf16_workspace_lse.argtypes = [ctypes.POINTER(_Shape), i32, i32, vp]
+    lib.lynx_bf16_workspace_lse.restype = ctypes.c_void_p
+    lib.lynx_lse_merge.argtypes = [vp, vp, vp, vp, i64, vp, vp, vp]
+    lib.lynx_lse_merge.restype = ctypes.c_int
     lib.lynx_check.argtypes = [vp, vp]
     lib.lynx_check.restype = ctypes.c_int
     lib.lynx_status_string.argtypes = [ctypes.c_int]
@@ -279,6 +285,46 @@ def bf16_attention(geo: Geometry, q: torch.Tensor, k_pages: torch.Tensor, v_page
                                    _ptr(v_pages), _ptr(block_table), _ptr(seq_lens), softmax_scale, _ptr(out),
                                    _ptr(workspace), workspace.numel(), _stream()), "lynx_bf16_attention")
     return out
+
+
+def _lse_view(addr, workspace: torch.Tensor, B: int, n_q: int, Hq: int, what: str) -> torch.Tensor:
+    if not addr:
+        raise LynxError(f"{what}: unsupported shape")
+    off = int(addr) - workspace.data_ptr()
+    n = B * n_q * Hq * 4
+    if workspace.dtype != torch.uint8 or off < 0 or off + n > workspace.numel():
+        raise LynxError(f"{what}: the workspace is smaller than the call's")
+    return workspace[off:off + n].view(torch.float32).view(B, n_q, Hq)
+
+
+def workspace_lse(geo: Geometry, B: int, n_q: int, workspace: torch.Tensor) -> torch.Tensor:
+    """lynx_workspace_lse: float32 [B][n_q][Hq] view, inside `workspace`, of the natural-log log-sum-exps the last
+    anchor_attention / merge_verify_attention call with this (B, n_q) left there."""
+    return _lse_view(load().lynx_workspace_lse(ctypes.byref(geo._c()), B, n_q, _ptr(workspace)), workspace, B, n_q,
+                     geo.num_q_heads, "lynx_workspace_lse")
+
+
+def bf16_workspace_lse(geo: Geometry, B: int, n_q: int, workspace: torch.Tensor) -> torch.Tensor:
+    """lynx_bf16_workspace_lse: the same for the workspace of a bf16_attention call."""
+    return _lse_view(load().lynx_bf16_workspace_lse(ctypes.byref(geo._c()), B, n_q, _ptr(workspace)), workspace, B,
+                     n_q, geo.num_q_heads, "lynx_bf16_workspace_lse")
+
+
+def lse_merge(out_a: torch.Tensor, lse_a: torch.Tensor, out_b: torch.Tensor, lse_b: torch.Tensor,
+              out: torch.Tensor | None = None, want_lse: bool = False):
+    """lynx_lse_merge: two attention results float32 [...][128] over disjoint key sets, with their log-sum-exps
+    float32 [...], joined into the attention over the union.  Returns out, or (out, lse) with want_lse."""
+    if out_a.dtype != torch.float32 or out_b.dtype != torch.float32 or out_a.shape != out_b.shape or out_a.shape[-1] != D:
+        raise LynxError("out_a, out_b must be float32 [...][128] of one shape")
+    rows = out_a.numel() // D
+    if lse_a.dtype != torch.float32 or lse_b.dtype != torch.float32 or lse_a.numel() != rows or lse_b.numel() != rows:
+        raise LynxError("lse_a, lse_b must be float32 with one value per row")
+    if out is None:
+        out = torch.empty_like(out_a)
+    lse = torch.empty(out_a.shape[:-1], dtype=torch.float32, device=out_a.device) if want_lse else None
+    _ok(load().lynx_lse_merge(_ptr(out_a), _ptr(lse_a), _ptr(out_b), _ptr(lse_b), rows, _ptr(out), _ptr(lse), _stream()),
+        "lynx_lse_merge")
+    return (out, lse) if want_lse else out
 
 
 @dataclass

@@ -56,6 +56,7 @@ struct AttnParams {
   uint32_t* ws_group_ctr;  // [2 * CTAs of the largest grid]: tickets of the groups of partial slots
   float* ws_shadow;        // FP32 copies of the O accumulators (see kFlushMmas), or null
   float* ws_dev;           // [B*Hkv][kMaxQ]
+  float* ws_lse;           // [B][nq_stride][Hq] natural-log log-sum-exp of every output row's scores
   float* ws_part;          // [B*Hkv + CTAs][ncols_pad][kPartStride], slot = segment + CTA index
   float atol, rtol;
   float sm_log2;           // softmax_scale * log2(e)
@@ -204,6 +205,11 @@ __device__ __forceinline__ void merge_codes(uint32_t xa, uint32_t xr, uint32_t& 
   ev = bit_select(xa << 4, xr, 0xF0F0F0F0u);
   od = bit_select(xa, xr >> 4, 0xF0F0F0F0u);
 }
+// Natural-log log-sum-exp of a row's scores from its running maximum (or reference exponent) M, in log2 units,
+// and the sum L of 2^(score - M); -inf for a row that saw no token.
+__device__ __forceinline__ float lse_of(float M, float L) {
+  return L > 0.0f ? (M + __log2f(L)) * 0.6931471805599453f : -INFINITY;
+}
 constexpr int kPieceUnits = 64;  // stage-units whose block ids are looked up at a time
 
 struct Item {  // one piece: a run of stage-units of one (sequence, KV head) given to one CTA
@@ -298,6 +304,7 @@ __device__ __forceinline__ void finish_piece(const AttnParams& p, const Item& it
           float4* dst = reinterpret_cast<float4*>(
               p.out + (((size_t)item.b * p.nq_stride + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D);
           dst[lane] = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+          if (lane == 0) p.ws_lse[((size_t)item.b * p.nq_stride + j) * p.Hq + item.hkv * p.G + hh] = lse_of(M, L);
         } else {
           reinterpret_cast<float4*>(col)[lane] = acc;
           if (lane == 0) { col[128] = M; col[129] = L; }
@@ -453,7 +460,7 @@ struct Plan {
   int per;             // query positions per verification launch
   int ncols, variant;  // variant: 0: NT1 TW4 CG1; 1: NT2 TW4 CG1; 2: NT2 TW4 CG2; 3: NT2 TW2 CG4
   int cols_pad;
-  size_t off_chunk_ctr, off_seq_ctr, off_group_ctr, off_dev, off_part, bytes;
+  size_t off_chunk_ctr, off_seq_ctr, off_group_ctr, off_dev, off_lse, off_part, bytes;
   size_t shadow_bytes;   // optional tail of the workspace: FP32 copies of the accumulators (see kFlushMmas)
 };
 
@@ -483,6 +490,8 @@ bool make_plan(const lynx_shape* s, int B, int nq, Plan* pl) {
   pl->off_group_ctr = off; off += (size_t)2 * sm_count() * kMaxCtasPerSm * 4;
   off = (off + 255) & ~(size_t)255;
   pl->off_dev = off;       off += (size_t)B * s->num_kv_heads * kMaxQ * 4;
+  off = (off + 255) & ~(size_t)255;
+  pl->off_lse = off;       off += (size_t)B * nq * s->num_q_heads * 4;
   off = (off + 255) & ~(size_t)255;
   pl->off_part = off;
   off += ((size_t)B * s->num_kv_heads + (size_t)sm_count() * kMaxCtasPerSm) * pl->cols_pad * kPartStride * 4;
@@ -544,6 +553,7 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
   p.ws_group_ctr = reinterpret_cast<uint32_t*>(ws + pl.off_group_ctr);
   p.ws_shadow = use_shadow ? reinterpret_cast<float*>(ws + pl.bytes) : nullptr;
   p.ws_dev = reinterpret_cast<float*>(ws + pl.off_dev);
+  p.ws_lse = reinterpret_cast<float*>(ws + pl.off_lse);
   p.ws_part = reinterpret_cast<float*>(ws + pl.off_part);
   p.atol = atol; p.rtol = rtol;
   const float sc = softmax_scale == 0.0f ? 0.08838834764831845f : softmax_scale;
@@ -567,6 +577,7 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
       ps.tail = nq - j0;
       ps.q = p.q + (size_t)j0 * p.Hq * LYNX_D;
       ps.out = p.out + (size_t)j0 * p.Hq * LYNX_D;
+      ps.ws_lse = p.ws_lse + (size_t)j0 * p.Hq;
       const lynx_status rc = ps.ncols <= 4 ? launch_i8<false, 4>(ps, st) : ps.ncols <= 8 ? launch_i8<false, 8>(ps, st)
                            : ps.ncols <= 16 ? launch_i8<false, 16>(ps, st) : launch_i8<false, 32>(ps, st);
       if (rc != LYNX_OK) return rc;
@@ -584,6 +595,7 @@ lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int
     ps.tail = nq - j0;
     ps.q = p.q + (size_t)j0 * p.Hq * LYNX_D;
     ps.out = p.out + (size_t)j0 * p.Hq * LYNX_D;
+    ps.ws_lse = p.ws_lse + (size_t)j0 * p.Hq;
     if (p.draft) { ps.draft = p.draft + (size_t)j0 * p.Hq * LYNX_D; ps.dev = p.dev + j0; }
     const lynx_status rc = ps.ncols <= 4 ? launch_i8<true, 4>(ps, st) : ps.ncols <= 8 ? launch_i8<true, 8>(ps, st)
                          : ps.ncols <= 16 ? launch_i8<true, 16>(ps, st) : launch_wide<2, 1>(ps, st);
@@ -603,6 +615,12 @@ extern "C" size_t lynx_workspace_bytes(const lynx_shape* shape, int32_t batch, i
   lynx::Plan pl;
   if (!lynx::make_plan(shape, batch, n_cols_q, &pl)) return 0;
   return pl.bytes + pl.shadow_bytes;
+}
+
+extern "C" const float* lynx_workspace_lse(const lynx_shape* shape, int32_t batch, int32_t n_q, const void* workspace) {
+  lynx::Plan pl;
+  if (!workspace || !lynx::make_plan(shape, batch, n_q, &pl)) return nullptr;
+  return reinterpret_cast<const float*>(static_cast<const unsigned char*>(workspace) + pl.off_lse);
 }
 
 extern "C" lynx_status lynx_anchor_attention(const lynx_shape* shape, const void* q_bf16, int32_t batch,

@@ -346,6 +346,7 @@ __device__ __forceinline__ void i8_producer(const AttnParams& p, int pw, int lan
       if (clamp_len(b) != 0) continue;
       const size_t n = (size_t)p.nq * p.Hq * LYNX_D;
       for (size_t i = lane; i < n; i += 32) p.out[(size_t)b * p.nq_stride * p.Hq * LYNX_D + i] = 0.0f;
+      for (int i = lane; i < p.nq * p.Hq; i += 32) p.ws_lse[(size_t)b * p.nq_stride * p.Hq + i] = -INFINITY;
       if (FULL && p.draft != nullptr) {
         int fr = p.nq;
         for (int j = p.nq - 1; j >= 0; --j) {
@@ -1100,6 +1101,7 @@ __global__ void __launch_bounds__(I8Cfg<FULL, CP>::kThreads, 1) attn_i8_kernel(c
             const int j = c / p.G, hh = c % p.G;
             p.out[(((size_t)item.b * p.nq_stride + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + dim_out] =
                 lt[cc] > 0.0f ? v / lt[cc] : 0.0f;
+            if (r == 0) p.ws_lse[((size_t)item.b * p.nq_stride + j) * p.Hq + item.hkv * p.G + hh] = lse_of(mt[cc], lt[cc]);
           } else {
             part[(size_t)c * kPartStride + dim_out] = v;
             if (r == 0) { part[(size_t)c * kPartStride + 128] = mt[cc]; part[(size_t)c * kPartStride + 129] = lt[cc]; }

@@ -226,6 +226,7 @@ __device__ __forceinline__ void wide_producer(const AttnParams& p, int pw, int l
       if (clamp_len(b) != 0) continue;
       const size_t n = (size_t)p.nq * p.Hq * LYNX_D;
       for (size_t i = lane; i < n; i += 32) p.out[(size_t)b * p.nq_stride * p.Hq * LYNX_D + i] = 0.0f;
+      for (int i = lane; i < p.nq * p.Hq; i += 32) p.ws_lse[(size_t)b * p.nq_stride * p.Hq + i] = -INFINITY;
       if (p.draft != nullptr) {
         int fr = p.nq;
         for (int j = p.nq - 1; j >= 0; --j) {
@@ -929,6 +930,12 @@ __global__ void __launch_bounds__(WideCfg<NCOPY, TERMS>::kThreads, 1) attn_wide_
           const int j = cc / p.G, hh = cc % p.G;
           p.out[(((size_t)item.b * p.nq_stride + j) * p.Hq + item.hkv * p.G + hh) * LYNX_D + d] =
               lt > 0.0f ? v / lt : 0.0f;
+          if (d == 0) {
+            float Mc = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 2 * NR; ++i) Mc = fmaxf(Mc, sc_m[(i / NR) * 128 + (i % NR) * CP + cc]);
+            p.ws_lse[((size_t)item.b * p.nq_stride + j) * p.Hq + item.hkv * p.G + hh] = lse_of(Mc, lt);
+          }
         } else {
           part_dst[(size_t)cc * kPartStride + d] = v;
           if (d == 0) {

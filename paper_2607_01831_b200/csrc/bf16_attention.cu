@@ -30,6 +30,7 @@ struct BfParams {
   const int32_t* seq_lens;
   float* out;
   float* part;      // [B][Hkv][chunks][cols][kPartStrideB]
+  float* lse;       // [B][nq][Hq] natural-log log-sum-exp of every output row's scores
   float sm_log2;
   int B, nq, causal, Hq, Hkv, G, bt, num_blocks, max_blocks, ncols, chunks;
 };
@@ -421,6 +422,7 @@ __global__ void __launch_bounds__(LYNX_D) bf16_combine_kernel(const BfParams p) 
   }
   const int j = c / p.G, hh = c % p.G;
   p.out[(((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
+  if (d == 0) p.lse[((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh] = L > 0.0f ? (M + __log2f(L)) * 0.6931471805599453f : -INFINITY;
 }
 
 template <int COLS, int LPT>
@@ -451,6 +453,13 @@ lynx_status launch_bf16_tc(const BfParams& p, cudaStream_t st) {
   return launch_status();
 }
 
+// bytes of the chunk partials, rounded up to 256: the log-sum-exps follow them in the workspace
+size_t bf16_part_bytes(const lynx_shape* s, int B, int ncols, int chunks) {
+  const int cols_pad = ncols <= 1 ? 1 : ncols <= 2 ? 2 : ncols <= 4 ? 4 : 8;
+  const size_t b = (size_t)B * s->num_kv_heads * chunks * cols_pad * kPartStrideB * sizeof(float);
+  return (b + 255) & ~(size_t)255;
+}
+
 bool bf16_shape_ok(const lynx_shape* s, int B, int nq, int* ncols, int* chunks) {
   if (!s || s->head_dim != LYNX_D || s->num_kv_heads <= 0 || s->num_q_heads <= 0 ||
       s->num_q_heads % s->num_kv_heads != 0 || s->block_tokens <= 0 || s->num_blocks <= 0 ||
@@ -471,8 +480,14 @@ bool bf16_shape_ok(const lynx_shape* s, int B, int nq, int* ncols, int* chunks) 
 extern "C" size_t lynx_bf16_workspace_bytes(const lynx_shape* shape, int32_t batch, int32_t n_q) {
   int ncols = 0, chunks = 0;
   if (!lynx::bf16_shape_ok(shape, batch, n_q, &ncols, &chunks)) return 0;
-  const int cols_pad = ncols <= 1 ? 1 : ncols <= 2 ? 2 : ncols <= 4 ? 4 : 8;
-  return (size_t)batch * shape->num_kv_heads * chunks * cols_pad * lynx::kPartStrideB * sizeof(float);
+  return lynx::bf16_part_bytes(shape, batch, ncols, chunks) + (size_t)batch * n_q * shape->num_q_heads * sizeof(float);
+}
+
+extern "C" const float* lynx_bf16_workspace_lse(const lynx_shape* shape, int32_t batch, int32_t n_q, const void* workspace) {
+  int ncols = 0, chunks = 0;
+  if (!workspace || !lynx::bf16_shape_ok(shape, batch, n_q, &ncols, &chunks)) return nullptr;
+  return reinterpret_cast<const float*>(static_cast<const unsigned char*>(workspace) +
+                                        lynx::bf16_part_bytes(shape, batch, ncols, chunks));
 }
 
 extern "C" lynx_status lynx_bf16_attention(const lynx_shape* shape, const void* q_bf16, int32_t batch, int32_t n_q,
@@ -495,6 +510,7 @@ extern "C" lynx_status lynx_bf16_attention(const lynx_shape* shape, const void* 
   p.v = static_cast<const __nv_bfloat16*>(v_pages_bf16);
   p.block_table = block_table; p.seq_lens = seq_lens; p.out = out;
   p.part = static_cast<float*>(workspace);
+  p.lse = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + bf16_part_bytes(shape, batch, p.ncols, p.chunks));
   const float sc = softmax_scale == 0.0f ? 0.08838834764831845f : softmax_scale;
   p.sm_log2 = sc * 1.4426950408889634f;
   p.B = batch; p.nq = n_q; p.causal = causal ? 1 : 0;
