@@ -464,6 +464,7 @@ def main():
         line["hierarchical"] = run_hier(wlk, peak)
         line["progressive"] = run_progressive(wlk)
         line["token_verify"] = run_token_verify(wlk, peak)
+        line["bf16_tail"] = run_tail(wlk)
     if rank == 0 and world == 1 and not args.no_e2e:
         line["e2e"] = run_e2e(wlk, args.e2e_steps, step_bytes)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -700,6 +701,67 @@ def run_bf16_pages(wlk: "Workload", peak: float, max_layers: int = 8):
             "speedup_fused_vs_bf16_attention": t_bf / t_fu,
             "speedup_fused_vs_recombine_plus_bf16_attention": (t_rec + t_bf) / t_fu,
             "max_abs_difference_of_outputs": diff}
+
+
+def run_tail(wlk: "Workload", max_layers: int = 8, tail_tokens: int = 1024):
+    """Context: one decode step (n_q = 1) on the Anchor state of up to 8 layers of the workload when every
+    sequence is followed by `tail_tokens` tokens the decode node generated itself (BF16 pages, Section 4.2
+    keeps them out of the quantiser): lynx_anchor_attention on the prefix, lynx_bf16_attention on the tail,
+    lynx_lse_merge of the two by the log-sum-exps the calls leave in their workspaces.  Reports what the tail
+    adds to the prefix call.  Not part of `value`."""
+    import ctypes
+    lynx, wl = wlk.lynx, wlk.wl
+    layers = min(wl.layers, max_layers)
+    Bs, nb, dev = layers * wl.batch, layers * wlk.nb_layer, wlk.device
+    K = lynx.Planes(wlk.planes["K"].anchor[:nb], None, wlk.planes["K"].meta[:nb])
+    V = lynx.Planes(wlk.planes["V"].anchor[:nb], None, wlk.planes["V"].meta[:nb])
+    geo = lynx.Geometry(wl.num_q_heads, wl.num_kv_heads, wl.block_tokens, nb, wlk.table.shape[1])
+    table, lens = wlk.table[:Bs].contiguous(), wlk.lens_flat[:Bs].contiguous()
+    q = wlk.windows[0]["qs"][0][:Bs].contiguous()
+    ws = lynx.make_workspace(geo, Bs, 1, dev)
+    # the tail: `tail_tokens` BF16 tokens per sequence in pages of the workload's block size (seeded values)
+    bt = wl.block_tokens
+    per = (tail_tokens + bt - 1) // bt
+    geo_t = lynx.Geometry(wl.num_q_heads, wl.num_kv_heads, bt, Bs * per, per)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(20260701)
+    pages = [torch.randn(Bs * per, wl.num_kv_heads, bt, 128, device=dev, generator=gen).to(torch.bfloat16) for _ in "KV"]
+    ttable = torch.arange(Bs * per, dtype=torch.int32, device=dev).view(Bs, per)
+    tlens = torch.full((Bs,), tail_tokens, dtype=torch.int32, device=dev)
+    ws_t = torch.empty(int(lynx.load().lynx_bf16_workspace_bytes(ctypes.byref(geo_t._c()), Bs, 1)), dtype=torch.uint8, device=dev)
+    out_p = torch.empty(Bs, 1, wl.num_q_heads, 128, dtype=torch.float32, device=dev)
+    out_t, out = torch.empty_like(out_p), torch.empty_like(out_p)
+    lse_p, lse_t = lynx.workspace_lse(geo, Bs, 1, ws), lynx.bf16_workspace_lse(geo_t, Bs, 1, ws_t)
+
+    def prefix():
+        lynx.anchor_attention(geo, q, K, V, table, lens, ws, out=out_p)
+
+    def tail():
+        lynx.bf16_attention(geo_t, q, pages[0], pages[1], ttable, tlens, workspace=ws_t, causal=True, out=out_t)
+
+    def merge():
+        lynx.lse_merge(out_p, lse_p, out_t, lse_t, out=out)
+
+    def all3():
+        prefix(); tail(); merge()
+
+    def time_ms(fn, reps=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+    t = {name: time_ms(fn) for name, fn in (("prefix_anchor_attention", prefix), ("tail_bf16_attention", tail),
+                                             ("lse_merge", merge), ("all_three", all3))}
+    lynx.check(ws)
+    share = float(torch.exp(lse_t - torch.logaddexp(lse_p, lse_t)).mean())
+    return {"layers": layers, "sequences": Bs, "tail_tokens": tail_tokens, "ms": t,
+            "tail_adds": t["all_three"] / t["prefix_anchor_attention"] - 1.0, "mean_softmax_mass_on_tail": share}
 
 
 def run_recombine(wlk: "Workload", peak: float, max_rows: int = 4 << 20):
