@@ -701,3 +701,69 @@ def test_bf16_pages_attention_matches_oracle(lynx, G, n_q, lens, bt):
     with pytest.raises(lynx.LynxError):        # more than 8 query columns
         lynx.bf16_attention(c["geo"], torch.zeros(len(lens), 16, Hkv * G, 128, dtype=torch.bfloat16, device="cuda"),
                             k_pages, v_pages, td, ld)
+
+
+# ------------------------------------------------------------------------ degenerate key / value rows
+@pytest.mark.parametrize("G,n_q", [(4, 1), (4, 2), (4, 4), (8, 8), (2, 1)])
+def test_degenerate_key_and_value_rows(lynx, G, n_q):
+    """Rows the quantiser and the kernels treat specially, mixed into ordinary ones: constant rows (scale 0: the
+    row is its zero point), rows of zeros and of -0, rows 10^-4 times and 50 times the ordinary size (the large
+    keys take nearly all the softmax mass), large value rows, a run of identical keys (uniform weights among
+    them), and a sequence whose queries are zero (uniform weights over everything).  Anchor and full state at
+    4 / 8 / 16 / 64 columns, the BF16-page kernel on the dequantised pages where it takes the shape."""
+    Hkv, bt, lens = 2, 16, (300, 45)
+    B = len(lens)
+    lens_t = torch.tensor(lens, dtype=torch.int32)
+    table, nb = synth.block_table(lens_t, bt, True, "dg", G * n_q)
+    g = torch.Generator().manual_seed(77 + G * n_q)
+    k = torch.randn(nb, Hkv, bt, 128, generator=g)
+    v = torch.randn(nb, Hkv, bt, 128, generator=g)
+
+    def rows(x, b, t0, t1):          # view of tokens [t0, t1) of sequence b: list of (block, row) slices
+        return [(int(table[b, t // bt]), t % bt) for t in range(t0, min(t1, lens[b]))]
+    for b in range(B):
+        for blk, r in rows(k, b, 0, 10):
+            k[blk, :, r] = 2.5
+            v[blk, :, r] = -1.25
+        for blk, r in rows(k, b, 10, 20):
+            k[blk, :, r] = 0.0
+            v[blk, :, r] = 0.0
+        for blk, r in rows(k, b, 20, 25):
+            k[blk, :, r] = -0.0
+            v[blk, :, r] = -0.0
+        for blk, r in rows(k, b, 30, 40):
+            k[blk, :, r] *= 1.0e-4
+            v[blk, :, r] *= 1.0e-4
+        for blk, r in rows(k, b, 40, 44):
+            k[blk, :, r] *= 50.0
+        for blk, r in rows(k, b, 50, 60):
+            v[blk, :, r] *= 100.0
+        same = torch.randn(Hkv, 128, generator=g)
+        for blk, r in rows(k, b, 100, 200):
+            k[blk, :, r] = same
+    k, v = k.to(torch.bfloat16), v.to(torch.bfloat16)
+    q = synth.queries(B, n_q, Hkv * G, "cpu", "dgQ", G)
+    q[1] = 0.0
+    K, V = lynx.split_quantize(k.cuda()), lynx.split_quantize(v.cuda())
+    kp, vp = oracle.split_quantize(bf16_bits(k)), oracle.split_quantize(bf16_bits(v))
+    _assert_planes_equal(_planes_np(K), kp)
+    _assert_planes_equal(_planes_np(V), vp)
+    geo = lynx.Geometry(Hkv * G, Hkv, bt, nb, table.shape[1])
+    ws = lynx.make_workspace(geo, B, n_q, "cuda")
+    qd, td, ld = q.cuda(), table.cuda(), lens_t.cuda()
+    for causal in (False, True):
+        out = lynx.anchor_attention(geo, qd, K, V, td, ld, ws, causal=causal)
+        lynx.check(ws)
+        ref = oracle.attention(False, bf16_bits(q), kp, vp, table.numpy(), lens_t.numpy(), Hkv, bt, causal=causal)
+        _close(out.cpu().numpy().astype(np.float64), ref, f"anchor, degenerate rows, causal={causal}")
+        full, _, _ = lynx.merge_verify_attention(geo, qd, K, V, td, ld, ws, causal=causal)
+        lynx.check(ws)
+        ref = oracle.attention(True, bf16_bits(q), kp, vp, table.numpy(), lens_t.numpy(), Hkv, bt, causal=causal)
+        _close(full.cpu().numpy().astype(np.float64), ref, f"full state, degenerate rows, causal={causal}")
+        if n_q * G <= 8:
+            _, k_pages = lynx.recombine(K, want_codes=False, want_bf16=True)
+            _, v_pages = lynx.recombine(V, want_codes=False, want_bf16=True)
+            got = lynx.bf16_attention(geo, qd, k_pages, v_pages, td, ld, causal=causal)
+            ref = oracle.attention_bf16_pages(bf16_bits(q), oracle.recombine(*kp)[1], oracle.recombine(*vp)[1],
+                                              table.numpy(), lens_t.numpy(), causal=causal)
+            _close(got.cpu().numpy().astype(np.float64), ref, f"BF16 pages, degenerate rows, causal={causal}")
