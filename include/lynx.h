@@ -218,7 +218,9 @@ lynx_status lynx_token_verify(const float* p_probs, const float* q_probs, const 
  * against (256 bytes per row of K or V instead of 72 / 136).
  * k_pages_bf16, v_pages_bf16 : BF16 [num_blocks][Hkv][block_tokens][128], as lynx_recombine writes
  * them (dequant_bf16).  q_bf16, block_table, seq_lens, causal, softmax_scale, out as for
- * lynx_anchor_attention.  n_q * (Hq/Hkv) must be <= 8 (decode and short windows); any block_tokens.
+ * lynx_anchor_attention.  Hq/Hkv must be <= 8 and n_q <= 64; a launch takes up to 8 query columns
+ * n_q * (Hq/Hkv), a call with more runs as slices of whole positions, each a pass of its own over the pages.
+ * Any block_tokens.
  * workspace : lynx_bf16_workspace_bytes(shape, batch, n_q) bytes of scratch (split-K partials and the rows'
  * log-sum-exps), no initialisation needed.  Out-of-range block ids are clamped and not reported. */
 size_t lynx_bf16_workspace_bytes(const lynx_shape* shape, int32_t batch, int32_t n_q);
@@ -243,11 +245,20 @@ lynx_status lynx_bf16_attention(const lynx_shape* shape, const void* q_bf16, int
  * prefix through lynx_anchor_attention or lynx_merge_verify_attention, non-causal, the tail through
  * lynx_bf16_attention, causal among the tail's own tokens).  A row with lse = -inf contributes nothing, whatever
  * its out row holds; two such rows give zeros and -inf.  All pointers are DEVICE pointers; out_* and out 16-byte
- * aligned; out may be out_a or out_b; lse_out may be NULL.  Asynchronous on `stream`. */
+ * aligned; out may be out_a or out_b; lse_out may be NULL.  Asynchronous on `stream`.
+ *
+ * lynx_verify_decision is Section 4.3's agreement test on outputs that are already in memory -- the full-state
+ * result of a window after it has been joined with the tail: out_full, draft_out float [batch][k][Hq][128],
+ * dev[b][j] = max over heads and dims of |f - d| / (atol + rtol |f|), first_reject[b] = the smallest j with
+ * dev[b][j] > 1, else k: the decision lynx_merge_verify_attention takes when it is given a draft.  k <= 64,
+ * atol > 0, rtol >= 0; out_full and draft_out 16-byte aligned.  Asynchronous on `stream`. */
 const float* lynx_workspace_lse(const lynx_shape* shape, int32_t batch, int32_t n_q, const void* workspace);
 const float* lynx_bf16_workspace_lse(const lynx_shape* shape, int32_t batch, int32_t n_q, const void* workspace);
 lynx_status lynx_lse_merge(const float* out_a, const float* lse_a, const float* out_b, const float* lse_b,
                            int64_t n_rows, float* out, float* lse_out, void* stream);
+lynx_status lynx_verify_decision(const float* out_full, const float* draft_out, int32_t batch, int32_t k,
+                                 int32_t num_q_heads, float atol, float rtol, int32_t* first_reject, float* dev,
+                                 void* stream);
 
 /* Synchronises `stream`, reads and clears the workspace's status word.  Test / debug use. */
 lynx_status lynx_check(void* workspace, void* stream);

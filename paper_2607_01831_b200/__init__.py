@@ -39,7 +39,7 @@ class _Shape(ctypes.Structure):
 EXPORTS = ["lynx_split_quantize", "lynx_recombine", "lynx_workspace_bytes", "lynx_workspace_init",
            "lynx_anchor_attention", "lynx_merge_verify_attention", "lynx_anchor_attention_static",
            "lynx_bf16_workspace_bytes", "lynx_bf16_attention", "lynx_hier_quantize", "lynx_hier_dequantize",
-           "lynx_token_verify", "lynx_workspace_lse", "lynx_bf16_workspace_lse", "lynx_lse_merge",
+           "lynx_token_verify", "lynx_workspace_lse", "lynx_bf16_workspace_lse", "lynx_lse_merge", "lynx_verify_decision",
            "lynx_check",
            "lynx_status_string", "lynx_version"]
 
@@ -93,6 +93,8 @@ def load():
     lib.lynx_bf16_workspace_lse.restype = ctypes.c_void_p
     lib.lynx_lse_merge.argtypes = [vp, vp, vp, vp, i64, vp, vp, vp]
     lib.lynx_lse_merge.restype = ctypes.c_int
+    lib.lynx_verify_decision.argtypes = [vp, vp, i32, i32, i32, f32, f32, vp, vp, vp]
+    lib.lynx_verify_decision.restype = ctypes.c_int
     lib.lynx_check.argtypes = [vp, vp]
     lib.lynx_check.restype = ctypes.c_int
     lib.lynx_status_string.argtypes = [ctypes.c_int]
@@ -325,6 +327,19 @@ def lse_merge(out_a: torch.Tensor, lse_a: torch.Tensor, out_b: torch.Tensor, lse
     _ok(load().lynx_lse_merge(_ptr(out_a), _ptr(lse_a), _ptr(out_b), _ptr(lse_b), rows, _ptr(out), _ptr(lse), _stream()),
         "lynx_lse_merge")
     return (out, lse) if want_lse else out
+
+
+def verify_decision(out_full: torch.Tensor, draft_out: torch.Tensor, atol: float, rtol: float):
+    """lynx_verify_decision: out_full, draft_out float32 [B][k][Hq][128] -> (first_reject i32 [B], dev f32 [B][k])."""
+    if out_full.dtype != torch.float32 or draft_out.dtype != torch.float32 or out_full.shape != draft_out.shape \
+            or out_full.dim() != 4 or out_full.shape[-1] != D:
+        raise LynxError("out_full, draft_out must be float32 [B][k][Hq][128]")
+    B, k, Hq, _ = out_full.shape
+    first_reject = torch.empty(B, dtype=torch.int32, device=out_full.device)
+    dev = torch.empty(B, k, dtype=torch.float32, device=out_full.device)
+    _ok(load().lynx_verify_decision(_ptr(out_full), _ptr(draft_out), B, k, Hq, atol, rtol, _ptr(first_reject), _ptr(dev),
+                                    _stream()), "lynx_verify_decision")
+    return first_reject, dev
 
 
 @dataclass

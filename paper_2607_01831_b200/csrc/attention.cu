@@ -513,6 +513,33 @@ __global__ void first_reject_kernel(const float* __restrict__ dev, int B, int nq
   first_reject[b] = fr;
 }
 
+// Section 4.3's agreement test on outputs that are already in memory (a verification pass whose result was joined
+// with a BF16 tail first): dev[b][j] = max over heads and dims of |f - d| / (atol + rtol |f|), the arithmetic of
+// the decision fused into the verification kernels.  One CTA per (sequence, position).
+__global__ void __launch_bounds__(256) deviation_kernel(const float4* __restrict__ out_full, const float4* __restrict__ draft,
+                                                        int row_f4, float atol, float rtol, float* __restrict__ dev) {
+  const float4* f = out_full + (size_t)blockIdx.x * row_f4;
+  const float4* d = draft + (size_t)blockIdx.x * row_f4;
+  float worst = 0.0f;
+  for (int i = threadIdx.x; i < row_f4; i += 256) {
+    const float4 a = f[i], b = __ldg(d + i);
+    worst = fmaxf(worst, fabsf(a.x - b.x) / (atol + rtol * fabsf(a.x)));
+    worst = fmaxf(worst, fabsf(a.y - b.y) / (atol + rtol * fabsf(a.y)));
+    worst = fmaxf(worst, fabsf(a.z - b.z) / (atol + rtol * fabsf(a.z)));
+    worst = fmaxf(worst, fabsf(a.w - b.w) / (atol + rtol * fabsf(a.w)));
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) worst = fmaxf(worst, __shfl_xor_sync(0xFFFFFFFFu, worst, off));
+  __shared__ float red[8];
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = worst;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int w = 1; w < 8; ++w) worst = fmaxf(worst, red[w]);
+    dev[blockIdx.x] = worst;
+  }
+}
+
 lynx_status run_attention(bool full, const lynx_shape* shape, const void* q, int B, int nq, int causal,
                           lynx_plane K, lynx_plane V, const int32_t* block_table,
                           const int32_t* seq_lens, float softmax_scale, const float* draft,
@@ -615,6 +642,25 @@ extern "C" size_t lynx_workspace_bytes(const lynx_shape* shape, int32_t batch, i
   lynx::Plan pl;
   if (!lynx::make_plan(shape, batch, n_cols_q, &pl)) return 0;
   return pl.bytes + pl.shadow_bytes;
+}
+
+extern "C" lynx_status lynx_verify_decision(const float* out_full, const float* draft_out, int32_t batch, int32_t k,
+                                            int32_t num_q_heads, float atol, float rtol, int32_t* first_reject,
+                                            float* dev, void* stream) {
+  using namespace lynx;
+  if (batch == 0) return LYNX_OK;
+  if (batch < 0 || k <= 0 || k > kMaxWindow || num_q_heads <= 0 || (int64_t)batch * k >= (1ll << 31)) return LYNX_ERR_SHAPE;
+  if (!out_full || !draft_out || !first_reject || !dev) return LYNX_ERR_NULL;
+  if (!aligned16(out_full) || !aligned16(draft_out)) return LYNX_ERR_ALIGN;
+  if (!(atol > 0.0f && rtol >= 0.0f)) return LYNX_ERR_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  deviation_kernel<<<(unsigned)(batch * k), 256, 0, st>>>(reinterpret_cast<const float4*>(out_full),
+                                                         reinterpret_cast<const float4*>(draft_out),
+                                                         num_q_heads * (LYNX_D / 4), atol, rtol, dev);
+  lynx_status rc = launch_status();
+  if (rc != LYNX_OK) return rc;
+  first_reject_kernel<<<(unsigned)((batch + 127) / 128), 128, 0, st>>>(dev, batch, k, first_reject);
+  return launch_status();
 }
 
 extern "C" const float* lynx_workspace_lse(const lynx_shape* shape, int32_t batch, int32_t n_q, const void* workspace) {

@@ -33,6 +33,10 @@ struct BfParams {
   float* lse;       // [B][nq][Hq] natural-log log-sum-exp of every output row's scores
   float sm_log2;
   int B, nq, causal, Hq, Hkv, G, bt, num_blocks, max_blocks, ncols, chunks;
+  // A launch may be one slice [j0, j0 + nq) of the caller's n_q query positions (q, out and lse then point at
+  // position j0): nq_stride = the caller's n_q, tail = n_q - j0 (the causal limit of position j of the slice is
+  // len - tail + j + 1).  Unsliced: both equal nq.
+  int nq_stride, tail;
 };
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -65,8 +69,8 @@ __global__ void __launch_bounds__(kWarps * 32, COLS <= 4 ? 2 : 1) bf16_decode_ke
   for (int c = 0; c < COLS; ++c) {
     const int j = c / p.G, hh = c % p.G;
     const bool in = c < p.ncols;
-    lim[c] = in ? (p.causal ? len - p.nq + j + 1 : len) : 0;
-    const __nv_bfloat16* qp = p.q + (((size_t)b * p.nq + (in ? j : 0)) * p.Hq + hkv * p.G + (in ? hh : 0)) * LYNX_D + sl * DPL;
+    lim[c] = in ? (p.causal ? len - p.tail + j + 1 : len) : 0;
+    const __nv_bfloat16* qp = p.q + (((size_t)b * p.nq_stride + (in ? j : 0)) * p.Hq + hkv * p.G + (in ? hh : 0)) * LYNX_D + sl * DPL;
 #pragma unroll
     for (int d = 0; d < DPL; ++d) q[c][d] = in ? __bfloat162float(qp[d]) * p.sm_log2 : 0.0f;
   }
@@ -257,9 +261,9 @@ __global__ void __launch_bounds__(kTcWarps * 32, 2) bf16_decode_tc_kernel(const 
   {
     const int c = g, j = c / p.G, hh = c % p.G;
     const bool in = c < p.ncols;
-    lim = in ? (p.causal ? len - p.nq + j + 1 : len) : 0;
+    lim = in ? (p.causal ? len - p.tail + j + 1 : len) : 0;
     const uint32_t* qp = reinterpret_cast<const uint32_t*>(
-        p.q + (((size_t)b * p.nq + (in ? j : 0)) * p.Hq + hkv * p.G + (in ? hh : 0)) * LYNX_D);
+        p.q + (((size_t)b * p.nq_stride + (in ? j : 0)) * p.Hq + hkv * p.G + (in ? hh : 0)) * LYNX_D);
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
       qa[ks][0] = in ? __ldg(qp + 8 * ks + t) : 0u;
@@ -421,8 +425,8 @@ __global__ void __launch_bounds__(LYNX_D) bf16_combine_kernel(const BfParams p) 
     M = mn;
   }
   const int j = c / p.G, hh = c % p.G;
-  p.out[(((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
-  if (d == 0) p.lse[((size_t)b * p.nq + j) * p.Hq + hkv * p.G + hh] = L > 0.0f ? (M + __log2f(L)) * 0.6931471805599453f : -INFINITY;
+  p.out[(((size_t)b * p.nq_stride + j) * p.Hq + hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
+  if (d == 0) p.lse[((size_t)b * p.nq_stride + j) * p.Hq + hkv * p.G + hh] = L > 0.0f ? (M + __log2f(L)) * 0.6931471805599453f : -INFINITY;
 }
 
 template <int COLS, int LPT>
@@ -466,10 +470,10 @@ bool bf16_shape_ok(const lynx_shape* s, int B, int nq, int* ncols, int* chunks) 
       s->max_blocks_per_seq <= 0 || B <= 0 || nq <= 0)
     return false;
   const int G = s->num_q_heads / s->num_kv_heads;
-  if ((int64_t)nq * G > 8) return false;
+  if (G > 8 || nq > 64) return false;
   const int64_t cap = (int64_t)s->max_blocks_per_seq * s->block_tokens;
   if (cap >= (1ll << 31) || (int64_t)B * s->num_kv_heads * ((cap + kChunk - 1) / kChunk) >= (1ll << 31)) return false;
-  *ncols = nq * G;
+  *ncols = nq * G <= 8 ? nq * G : (8 / G) * G;   // columns of the widest launch: whole positions, 8 columns at most
   *chunks = (int)((cap + kChunk - 1) / kChunk);
   return true;
 }
@@ -517,14 +521,27 @@ extern "C" lynx_status lynx_bf16_attention(const lynx_shape* shape, const void* 
   p.Hq = shape->num_q_heads; p.Hkv = shape->num_kv_heads; p.G = p.Hq / p.Hkv;
   p.bt = shape->block_tokens; p.num_blocks = shape->num_blocks; p.max_blocks = shape->max_blocks_per_seq;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (p.bt % 16 == 0) {   // the tensor-core kernel (tiles of 16 tokens inside a block)
-    if (p.ncols <= 1) return launch_bf16_tc<1>(p, st);
-    if (p.ncols <= 2) return launch_bf16_tc<2>(p, st);
-    if (p.ncols <= 4) return launch_bf16_tc<4>(p, st);
-    return launch_bf16_tc<8>(p, st);
+  // a launch takes up to 8 query columns; a call with more runs as slices of whole positions, each a pass of its
+  // own over the pages, one after the other on the stream (they share the partials)
+  const int per = n_q * p.G <= 8 ? n_q : 8 / p.G;
+  for (int j0 = 0; j0 < n_q; j0 += per) {
+    BfParams ps = p;
+    ps.nq = n_q - j0 < per ? n_q - j0 : per;
+    ps.ncols = ps.nq * p.G;
+    ps.nq_stride = n_q;
+    ps.tail = n_q - j0;
+    ps.q = p.q + (size_t)j0 * p.Hq * LYNX_D;
+    ps.out = p.out + (size_t)j0 * p.Hq * LYNX_D;
+    ps.lse = p.lse + (size_t)j0 * p.Hq;
+    lynx_status rc;
+    if (p.bt % 16 == 0) {   // the tensor-core kernel (tiles of 16 tokens inside a block)
+      rc = ps.ncols <= 1 ? launch_bf16_tc<1>(ps, st) : ps.ncols <= 2 ? launch_bf16_tc<2>(ps, st)
+         : ps.ncols <= 4 ? launch_bf16_tc<4>(ps, st) : launch_bf16_tc<8>(ps, st);
+    } else {
+      rc = ps.ncols <= 1 ? launch_bf16<1, 8>(ps, st) : ps.ncols <= 2 ? launch_bf16<2, 8>(ps, st)
+         : ps.ncols <= 4 ? launch_bf16<4, 16>(ps, st) : launch_bf16<8, 16>(ps, st);
+    }
+    if (rc != LYNX_OK) return rc;
   }
-  if (p.ncols <= 1) return launch_bf16<1, 8>(p, st);
-  if (p.ncols <= 2) return launch_bf16<2, 8>(p, st);
-  if (p.ncols <= 4) return launch_bf16<4, 16>(p, st);
-  return launch_bf16<8, 16>(p, st);
+  return LYNX_OK;
 }

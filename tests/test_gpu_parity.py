@@ -698,9 +698,22 @@ def test_bf16_pages_attention_matches_oracle(lynx, G, n_q, lens, bt):
         ref = oracle.attention_bf16_pages(bf16_bits(c["q"]), ok_pages, ov_pages, c["table"].numpy(),
                                           c["lens"].numpy(), causal=causal)
         _close(got.cpu().numpy().astype(np.float64), ref, f"bf16 pages G={G} n_q={n_q} causal={causal}")
-    with pytest.raises(lynx.LynxError):        # more than 8 query columns
-        lynx.bf16_attention(c["geo"], torch.zeros(len(lens), 16, Hkv * G, 128, dtype=torch.bfloat16, device="cuda"),
+    with pytest.raises(lynx.LynxError):        # more than 64 query positions
+        lynx.bf16_attention(c["geo"], torch.zeros(len(lens), 65, Hkv * G, 128, dtype=torch.bfloat16, device="cuda"),
                             k_pages, v_pages, td, ld)
+
+
+def test_bf16_pages_attention_windows_run_as_slices(lynx):
+    # 5 positions x 4 heads per KV head = 20 columns: slices of 2, 2 and 1 positions; causal limits per position
+    Hkv, G, n_q, lens, bt = 2, 4, 5, (700, 3, 0), 16
+    c = _case(lynx, 9100, len(lens), Hkv, G, n_q, lens, bt, True, "student_t4")
+    _, k_pages = lynx.recombine(c["K"], want_codes=False, want_bf16=True)
+    _, v_pages = lynx.recombine(c["V"], want_codes=False, want_bf16=True)
+    for causal in (False, True):
+        got = lynx.bf16_attention(c["geo"], c["q"].cuda(), k_pages, v_pages, c["table"].cuda(), c["lens"].cuda(), causal=causal)
+        ref = oracle.attention_bf16_pages(bf16_bits(c["q"]), oracle.recombine(*c["kp"])[1], oracle.recombine(*c["vp"])[1],
+                                          c["table"].numpy(), c["lens"].numpy(), causal=causal)
+        _close(got.cpu().numpy().astype(np.float64), ref, f"bf16 pages in slices, causal={causal}")
 
 
 # ------------------------------------------------------------------------ degenerate key / value rows

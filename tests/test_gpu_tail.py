@@ -153,3 +153,60 @@ def test_lse_merge_against_the_oracle_rule_and_its_edge_cases(lynx):
     assert L.lynx_lse_merge(x.data_ptr() + 4, la.cuda().data_ptr(), x.data_ptr(), la.cuda().data_ptr(), 4, x.data_ptr(), None, None) == 3
     assert L.lynx_lse_merge(x.data_ptr(), la.cuda().data_ptr(), x.data_ptr(), la.cuda().data_ptr(), -1, x.data_ptr(), None, None) == 2
     assert L.lynx_lse_merge(None, None, None, None, 0, None, None, None) == 0
+
+
+def test_verify_decision_on_outputs_in_memory(lynx):
+    g = torch.Generator().manual_seed(9)
+    B, k, Hq = 37, 5, 12
+    f = torch.randn(B, k, Hq, 128, generator=g)
+    d = f + 0.02 * torch.randn(B, k, Hq, 128, generator=g) * (torch.rand(B, k, 1, 1, generator=g) < 0.5)
+    d[3] = f[3]                                  # a window that agrees everywhere
+    d[4, 0, 2, 7] += 5.0                         # and one rejected at its first position
+    exercised = 0
+    for atol, rtol in [(0.05, 0.05), (0.1, 0.0), (0.2, 0.1), (1e-3, 1e-2)]:
+        want_fr, want_dev = oracle.verify_decision(f.numpy().astype(np.float64), d.numpy(), atol, rtol)
+        fr, dev = lynx.verify_decision(f.cuda(), d.cuda(), atol, rtol)
+        assert np.allclose(dev.cpu().numpy(), want_dev, rtol=1e-5, atol=1e-7)
+        clear = np.all(np.abs(want_dev - 1.0) > 1e-4, axis=1)      # (binary32 against binary64 at the threshold)
+        exercised += int(clear.sum())
+        assert np.array_equal(fr.cpu().numpy()[clear], want_fr[clear])
+        assert int(fr[3]) == k and int(fr[4]) == 0
+    assert exercised >= 100
+    L = lynx.load()
+    x = f.cuda()
+    fr = torch.empty(B, dtype=torch.int32, device="cuda")
+    dv = torch.empty(B, k, device="cuda")
+    assert L.lynx_verify_decision(x.data_ptr(), None, B, k, Hq, 0.1, 0.1, fr.data_ptr(), dv.data_ptr(), None) == 1
+    assert L.lynx_verify_decision(x.data_ptr(), x.data_ptr(), B, 65, Hq, 0.1, 0.1, fr.data_ptr(), dv.data_ptr(), None) == 2
+    assert L.lynx_verify_decision(x.data_ptr(), x.data_ptr(), B, k, Hq, 0.0, 0.1, fr.data_ptr(), dv.data_ptr(), None) == 2
+    assert L.lynx_verify_decision(x.data_ptr() + 4, x.data_ptr(), B, k, Hq, 0.1, 0.1, fr.data_ptr(), dv.data_ptr(), None) == 3
+    assert L.lynx_verify_decision(None, None, 0, k, Hq, 0.1, 0.1, None, None, None) == 0
+
+
+def test_a_window_is_verified_over_prefix_and_tail(lynx):
+    """Section 4.3 with a BF16 tail: drafts on the Anchor prefix + tail, the full-state pass on prefix + tail, the
+    agreement test on the joined outputs -- against the oracle's decision on its own joined outputs."""
+    G, k = 4, 4      # 16 columns: one launch of the integer kernels, two slices of the BF16-page kernel
+    c = _case(lynx, 321, 2, G, k, (1800, 90, 0), (6, 40, 9), recipe="student_t4")
+    qd = c["q"].cuda()
+    ws = lynx.make_workspace(c["geo"], c["B"], k, "cuda")
+    ws_t = torch.empty(int(lynx.load().lynx_bf16_workspace_bytes(c["geo_t"]._c(), c["B"], k)), dtype=torch.uint8, device="cuda")
+    tl = lynx.bf16_attention(c["geo_t"], qd, c["kt"].cuda(), c["vt"].cuda(), c["ttable"].cuda(), c["tlens"].cuda(),
+                             workspace=ws_t, causal=True)
+    lse_tl = lynx.bf16_workspace_lse(c["geo_t"], c["B"], k, ws_t).clone()
+    lse_pre = lynx.workspace_lse(c["geo"], c["B"], k, ws)
+    anchor = lynx.anchor_attention(c["geo"], qd, c["K"], c["V"], c["table"].cuda(), c["lens"].cuda(), ws, causal=False)
+    draft = lynx.lse_merge(anchor, lse_pre, tl, lse_tl)
+    full, _, _ = lynx.merge_verify_attention(c["geo"], qd, c["K"], c["V"], c["table"].cuda(), c["lens"].cuda(), ws, causal=False)
+    joined = lynx.lse_merge(full, lse_pre, tl, lse_tl)
+    ref_a, ref_f = _oracle(c, False, True)["out"], _oracle(c, True, True)["out"]
+    _close(draft.cpu().numpy().astype(np.float64), ref_a, "draft over prefix + tail")
+    _close(joined.cpu().numpy().astype(np.float64), ref_f, "full state over prefix + tail")
+    exercised = 0
+    for atol, rtol in [(2e-2, 2e-2), (5e-2, 5e-2), (1e-1, 1e-1), (3e-1, 1e-1), (1.0, 0.0), (3e-3, 0.0)]:
+        want_fr, want_dev = oracle.verify_decision(ref_f, ref_a.astype(np.float32), atol, rtol)
+        if np.all(np.abs(want_dev - 1.0) > 0.05):
+            exercised += 1
+            fr, dev = lynx.verify_decision(joined, draft, atol, rtol)
+            assert np.array_equal(fr.cpu().numpy(), want_fr), (atol, rtol, want_dev)
+    assert exercised >= 1
