@@ -7,7 +7,7 @@
 // norm(max(0, q_j - p_j)), and if all are accepted a bonus token is drawn from q_{k+1} -- both by inverse CDF
 // in vocabulary order with the uniform r.  The random numbers are inputs.
 //
-// One CTA per sequence.  The acceptance scan touches k values; the correction reads one or two vocabulary rows
+// One CTA per sequence.  The acceptance scan touches k values (a lane per position); the correction reads one or two vocabulary rows
 // (4 or 8 bytes per entry) once, with coalesced loads: the 32 warps sum the row in chunks of 128 entries
 // (entry 32 e + lane of a chunk in step e) into shared memory, one warp scans the chunk sums for the chunk that
 // holds r * total and walks that chunk with a warp scan per step.  HBM-bound by construction, and small: the
@@ -31,15 +31,23 @@ __global__ void __launch_bounds__(kTvThreads) token_verify_kernel(const float* _
   const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const float* p = p_probs + (size_t)b * k * V;
   const float* q = q_probs + (size_t)b * (k + 1) * V;
-  if (tid == 0) {
+  if (warp == 0) {   // the acceptance scan: a lane per position, all loads in flight together (k <= 64: two rounds)
     int j = k;
-    for (int i = 0; i < k; ++i) {
-      int s = draft[(size_t)b * k + i];
-      s = s < 0 ? 0 : (s >= V ? V - 1 : s);
-      if (!(u[(size_t)b * k + i] * p[(size_t)i * V + s] < q[(size_t)i * V + s])) { j = i; break; }
+    for (int base = 0; base < k && j == k; base += 32) {
+      const int i = base + lane;
+      bool reject = false;
+      if (i < k) {
+        int s = draft[(size_t)b * k + i];
+        s = s < 0 ? 0 : (s >= V ? V - 1 : s);
+        reject = !(u[(size_t)b * k + i] * p[(size_t)i * V + s] < q[(size_t)i * V + s]);
+      }
+      const unsigned hit = __ballot_sync(0xFFFFFFFFu, reject);
+      if (hit != 0u) j = base + __ffs(hit) - 1;
     }
-    j_s = j;
-    n_accepted[b] = j;
+    if (lane == 0) {
+      j_s = j;
+      n_accepted[b] = j;
+    }
   }
   __syncthreads();
   const int j = j_s;
