@@ -465,6 +465,7 @@ def main():
         line["progressive"] = run_progressive(wlk)
         line["token_verify"] = run_token_verify(wlk, peak)
         line["bf16_tail"] = run_tail(wlk)
+        line["bit_splits"] = run_bit_splits(wlk, peak)
     if rank == 0 and world == 1 and not args.no_e2e:
         line["e2e"] = run_e2e(wlk, args.e2e_steps, step_bytes)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -762,6 +763,51 @@ def run_tail(wlk: "Workload", max_layers: int = 8, tail_tokens: int = 1024):
     share = float(torch.exp(lse_t - torch.logaddexp(lse_p, lse_t)).mean())
     return {"layers": layers, "sequences": Bs, "tail_tokens": tail_tokens, "ms": t,
             "tail_adds": t["all_three"] / t["prefix_anchor_attention"] - 1.0, "mean_softmax_mass_on_tail": share}
+
+
+def run_bit_splits(wlk: "Workload", peak: float, max_rows: int = 4 << 20):
+    """Context: the Anchor / Residual split at other bit positions (Conclusion: splits other than INT4 + INT4) on
+    the first rows of the BF16 K source, at most 4 Mi rows: lynx_split_quantize_bits for 2 + 6 and 6 + 2 bits
+    (392 bytes per row, as for 4 + 4), lynx_recombine_bits to BF16 pages from both streams and from the Anchor
+    alone.  Not part of `value`."""
+    lynx = wlk.lynx
+    src = wlk.src["K"].view(-1, 128)
+    rows = min(src.shape[0], max_rows)
+    x = src[:rows]
+    lib, stream = lynx.load(), torch.cuda.current_stream().cuda_stream
+    deq = torch.empty(rows, 128, dtype=torch.bfloat16, device=wlk.device)
+
+    def time_ms(fn, reps=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+    out = {"rows": rows}
+    for A in (2, 6):
+        a, r, m = lynx.split_quantize_bits(x, A)
+
+        def quant():
+            st = lib.lynx_split_quantize_bits(x.data_ptr(), rows, A, a.data_ptr(), r.data_ptr(), m.data_ptr(), stream)
+            if st != 0:
+                raise RuntimeError(f"lynx_split_quantize_bits: status {st}")
+
+        def pages(res):
+            st = lib.lynx_recombine_bits(a.data_ptr(), res.data_ptr() if res is not None else None, m.data_ptr(), rows, A,
+                                         None, deq.data_ptr(), stream)
+            if st != 0:
+                raise RuntimeError(f"lynx_recombine_bits: status {st}")
+        for name, fn, bpr in (("split_quantize", quant, 256 + 128 + 8), ("pages_from_both_streams", lambda: pages(r), 136 + 256),
+                              ("pages_from_the_anchor", lambda: pages(None), 16 * A + 8 + 256)):
+            ms = time_ms(fn)
+            g = rows * bpr / (ms * 1e-3) / 1e9
+            out[f"{A}+{8 - A} {name}"] = {"ms": ms, "bytes_per_row": bpr, "GBps": g, "frac_of_measured": g / peak}
+    return out
 
 
 def run_recombine(wlk: "Workload", peak: float, max_rows: int = 4 << 20):

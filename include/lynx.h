@@ -260,6 +260,24 @@ lynx_status lynx_verify_decision(const float* out_full, const float* draft_out, 
                                  int32_t num_q_heads, float atol, float rtol, int32_t* first_reject, float* dev,
                                  void* stream);
 
+/* The Anchor / Residual split at other bit positions (Conclusion: splits other than INT4 + INT4; Section 4.1
+ * stage 4 for the split itself, Section 2.3 for the code).  anchor_bits = A in {2, 4, 6}; R = 8 - A.  The 8-bit
+ * code, scale and zero are exactly those of lynx_split_quantize; the Anchor plane holds the top A bits of every
+ * code, the Residual plane the bottom R bits: (anchor << R) | residual is the code, and A = 4 writes the planes
+ * lynx_split_quantize writes.  Packing per 128-element row and stream: element e's field occupies bits
+ * [e w, (e + 1) w) of the row's 16 w bytes, least significant bit first (w = A or R).
+ *   src_bf16 : [n_rows][128] BF16;  anchor : [n_rows][16 A] bytes;  residual : [n_rows][16 R] bytes;
+ *   meta : [n_rows][2] float (scale, zero).  All DEVICE pointers, 16-byte aligned (meta: 8).
+ * lynx_recombine_bits: levels = (anchor << R) | residual, or with residual NULL the middle of the Anchor's
+ * bucket, (anchor << R) + 2^(R-1) (Section 4.2, Anchor phase); codes_u8 [n_rows][128] and / or dequant_bf16
+ * [n_rows][128] BF16 = bf16(fl(level * scale + zero)), as lynx_recombine; at least one output.  The pages it
+ * writes feed lynx_bf16_attention: that is how these splits reach attention (the fused attention calls read
+ * the 4 + 4 planes only).  LYNX_ERR_UNSUPPORTED for any other anchor_bits. */
+lynx_status lynx_split_quantize_bits(const void* src_bf16, int64_t n_rows, int32_t anchor_bits, uint8_t* anchor,
+                                     uint8_t* residual, float* meta, void* stream);
+lynx_status lynx_recombine_bits(const uint8_t* anchor, const uint8_t* residual, const float* meta, int64_t n_rows,
+                                int32_t anchor_bits, uint8_t* codes_u8, void* dequant_bf16, void* stream);
+
 /* Synchronises `stream`, reads and clears the workspace's status word.  Test / debug use. */
 lynx_status lynx_check(void* workspace, void* stream);
 

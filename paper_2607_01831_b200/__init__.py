@@ -39,7 +39,7 @@ class _Shape(ctypes.Structure):
 EXPORTS = ["lynx_split_quantize", "lynx_recombine", "lynx_workspace_bytes", "lynx_workspace_init",
            "lynx_anchor_attention", "lynx_merge_verify_attention", "lynx_anchor_attention_static",
            "lynx_bf16_workspace_bytes", "lynx_bf16_attention", "lynx_hier_quantize", "lynx_hier_dequantize",
-           "lynx_token_verify", "lynx_workspace_lse", "lynx_bf16_workspace_lse", "lynx_lse_merge", "lynx_verify_decision",
+           "lynx_token_verify", "lynx_workspace_lse", "lynx_bf16_workspace_lse", "lynx_lse_merge", "lynx_verify_decision", "lynx_split_quantize_bits", "lynx_recombine_bits",
            "lynx_check",
            "lynx_status_string", "lynx_version"]
 
@@ -95,6 +95,10 @@ def load():
     lib.lynx_lse_merge.restype = ctypes.c_int
     lib.lynx_verify_decision.argtypes = [vp, vp, i32, i32, i32, f32, f32, vp, vp, vp]
     lib.lynx_verify_decision.restype = ctypes.c_int
+    lib.lynx_split_quantize_bits.argtypes = [vp, i64, i32, vp, vp, vp, vp]
+    lib.lynx_split_quantize_bits.restype = ctypes.c_int
+    lib.lynx_recombine_bits.argtypes = [vp, vp, vp, i64, i32, vp, vp, vp]
+    lib.lynx_recombine_bits.restype = ctypes.c_int
     lib.lynx_check.argtypes = [vp, vp]
     lib.lynx_check.restype = ctypes.c_int
     lib.lynx_status_string.argtypes = [ctypes.c_int]
@@ -327,6 +331,32 @@ def lse_merge(out_a: torch.Tensor, lse_a: torch.Tensor, out_b: torch.Tensor, lse
     _ok(load().lynx_lse_merge(_ptr(out_a), _ptr(lse_a), _ptr(out_b), _ptr(lse_b), rows, _ptr(out), _ptr(lse), _stream()),
         "lynx_lse_merge")
     return (out, lse) if want_lse else out
+
+
+def split_quantize_bits(src: torch.Tensor, anchor_bits: int):
+    """lynx_split_quantize_bits: src BF16 [...][128] -> (anchor u8 [...][16 A], residual u8 [...][16 (8 - A)],
+    meta f32 [...][2]) for the split with A = anchor_bits top bits in the Anchor."""
+    if src.dtype != torch.bfloat16 or src.shape[-1] != D:
+        raise LynxError("src must be BF16 [...][128]")
+    lead, rows = tuple(src.shape[:-1]), src.numel() // D
+    anchor = torch.empty(lead + (16 * anchor_bits,), dtype=torch.uint8, device=src.device)
+    residual = torch.empty(lead + (16 * (8 - anchor_bits),), dtype=torch.uint8, device=src.device)
+    meta = torch.empty(lead + (2,), dtype=torch.float32, device=src.device)
+    _ok(load().lynx_split_quantize_bits(_ptr(src), rows, anchor_bits, _ptr(anchor), _ptr(residual), _ptr(meta), _stream()),
+        "lynx_split_quantize_bits")
+    return anchor, residual, meta
+
+
+def recombine_bits(anchor: torch.Tensor, residual: torch.Tensor | None, meta: torch.Tensor, anchor_bits: int,
+                   want_codes: bool = True, want_bf16: bool = True):
+    """lynx_recombine_bits -> (codes u8 [...][128] or None, dequantised BF16 [...][128] or None); residual None:
+    the Anchor alone (bucket mid-points)."""
+    lead, rows = tuple(anchor.shape[:-1]), anchor.numel() // (16 * anchor_bits)
+    codes = torch.empty(lead + (D,), dtype=torch.uint8, device=anchor.device) if want_codes else None
+    deq = torch.empty(lead + (D,), dtype=torch.bfloat16, device=anchor.device) if want_bf16 else None
+    _ok(load().lynx_recombine_bits(_ptr(anchor), _ptr(residual), _ptr(meta), rows, anchor_bits, _ptr(codes), _ptr(deq),
+                                   _stream()), "lynx_recombine_bits")
+    return codes, deq
 
 
 def verify_decision(out_full: torch.Tensor, draft_out: torch.Tensor, atol: float, rtol: float):

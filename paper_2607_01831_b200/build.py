@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "liblynx.so")
-SOURCES = ["api.cu", "split_quantize.cu", "attention.cu", "bf16_attention.cu", "hier_quantize.cu", "token_verify.cu", "lse_merge.cu"]
+SOURCES = ["api.cu", "split_quantize.cu", "attention.cu", "bf16_attention.cu", "hier_quantize.cu", "token_verify.cu", "lse_merge.cu", "bit_split.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 
