@@ -9,7 +9,7 @@
 //
 // One CTA per sequence.  The acceptance scan touches k values (a lane per position); the correction reads one or two vocabulary rows
 // (4 or 8 bytes per entry) once, with coalesced loads: the 32 warps sum the row in chunks of 128 entries
-// (entry 32 e + lane of a chunk in step e) into shared memory, one warp scans the chunk sums for the chunk that
+// (four chunks of a warp in flight) into shared memory, one warp scans the chunk sums for the chunk that
 // holds r * total and walks that chunk with a warp scan per step.  HBM-bound by construction, and small: the
 // point of this kernel is that the decision stays on the device.
 #include "lynx_common.cuh"
@@ -17,7 +17,8 @@
 namespace lynx {
 namespace {
 
-constexpr int kTvThreads = 1024, kTvWarps = kTvThreads / 32;   // (many warps: the row sums are latency-bound per warp)
+constexpr int kTvThreads = 512, kTvWarps = kTvThreads / 32;
+constexpr int kCh = 4;   // chunks of a warp in flight
 
 __global__ void __launch_bounds__(kTvThreads) token_verify_kernel(const float* __restrict__ p_probs,
                                                                   const float* __restrict__ q_probs,
@@ -55,22 +56,53 @@ __global__ void __launch_bounds__(kTvThreads) token_verify_kernel(const float* _
   const float* pj = j < k ? p + (size_t)j * V : nullptr;
   const int n_chunks = (V + 127) / 128;
   bool residual = pj != nullptr;
+  // rows start on 16-byte boundaries when the arrays do and V is a multiple of 4
+  const bool vec = (V & 3) == 0 && ((reinterpret_cast<uintptr_t>(p_probs) | reinterpret_cast<uintptr_t>(q_probs)) & 15u) == 0;
   auto weight = [&](int x) -> float {
     if (x >= V) return 0.0f;
     return residual ? fmaxf(__ldg(qj + x) - __ldg(pj + x), 0.0f) : __ldg(qj + x);
   };
   for (int pass = 0; pass < 2; ++pass) {   // a second pass only if the residual is zero everywhere: w = q_j
-    // chunk sums: four chunks of a warp in flight at a time
-    for (int c = warp * 4; c < n_chunks; c += kTvWarps * 4) {
-      float s[4];
+    // chunk sums: four chunks of a warp in flight at a time, all their loads issued before the first use
+    // (branch-free: an index beyond the row is clamped and its value masked).  With 16-byte alignment a lane takes
+    // four consecutive entries of a chunk in one load, else entry 32 e + lane in step e.
+    for (int c = warp * kCh; c < n_chunks; c += kTvWarps * kCh) {
+      float s[kCh];
+      if (vec) {
+        float4 a[kCh], d[kCh];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        s[i] = 0.0f;
+        for (int i = 0; i < kCh; ++i) {
+          const int x = (c + i) * 128 + lane * 4;
+          const int xx = x < V ? x : 0;
+          a[i] = __ldg(reinterpret_cast<const float4*>(qj + xx));
+          d[i] = residual ? __ldg(reinterpret_cast<const float4*>(pj + xx)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
 #pragma unroll
-        for (int e = 0; e < 4; ++e) s[i] += c + i < n_chunks ? weight((c + i) * 128 + e * 32 + lane) : 0.0f;
+        for (int i = 0; i < kCh; ++i) {
+          const float v = residual ? (fmaxf(a[i].x - d[i].x, 0.0f) + fmaxf(a[i].y - d[i].y, 0.0f)) +
+                                         (fmaxf(a[i].z - d[i].z, 0.0f) + fmaxf(a[i].w - d[i].w, 0.0f))
+                                   : (a[i].x + a[i].y) + (a[i].z + a[i].w);
+          s[i] = (c + i) * 128 + lane * 4 < V ? v : 0.0f;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < kCh; ++i) {
+          float a[4], d[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int x = (c + i) * 128 + e * 32 + lane;
+            const int xx = x < V ? x : 0;
+            a[e] = __ldg(qj + xx);
+            d[e] = residual ? __ldg(pj + xx) : 0.0f;
+          }
+          s[i] = 0.0f;
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            s[i] += (c + i) * 128 + e * 32 + lane < V ? (residual ? fmaxf(a[e] - d[e], 0.0f) : a[e]) : 0.0f;
+        }
       }
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < kCh; ++i) {
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) s[i] += __shfl_xor_sync(0xFFFFFFFFu, s[i], off);
         if (lane == 0 && c + i < n_chunks) csum[c + i] = s[i];
