@@ -415,14 +415,25 @@ __global__ void __launch_bounds__(LYNX_D) bf16_combine_kernel(const BfParams p) 
   const int n = (len + kChunk - 1) / kChunk;
   const float* part = p.part + (size_t)bh * p.chunks * (size_t)COLS * kPartStrideB + (size_t)c * kPartStrideB;
   float M = -1.0e30f, L = 0.0f, acc = 0.0f;
-  for (int i = 0; i < n; ++i) {
-    const float* src = part + (size_t)i * COLS * kPartStrideB;
-    const float mi = src[128], li = src[129], oi = src[d];
-    const float mn = fmaxf(M, mi);
-    const float fa = ex2f(M - mn), fb = ex2f(mi - mn);
-    acc = acc * fa + oi * fb;
-    L = L * fa + li * fb;
-    M = mn;
+  constexpr int kAhead = 8;   // partials whose loads are issued together (one L2 round trip per batch, not per chunk)
+  for (int i0 = 0; i0 < n; i0 += kAhead) {
+    float mi[kAhead], li[kAhead], oi[kAhead];
+#pragma unroll
+    for (int u = 0; u < kAhead; ++u) {
+      const bool in = i0 + u < n;
+      const float* src = part + (size_t)(in ? i0 + u : i0) * COLS * kPartStrideB;
+      mi[u] = in ? src[128] : -1.0e30f;
+      li[u] = in ? src[129] : 0.0f;
+      oi[u] = in ? src[d] : 0.0f;
+    }
+#pragma unroll
+    for (int u = 0; u < kAhead; ++u) {
+      const float mn = fmaxf(M, mi[u]);
+      const float fa = ex2f(M - mn), fb = ex2f(mi[u] - mn);
+      acc = acc * fa + oi[u] * fb;
+      L = L * fa + li[u] * fb;
+      M = mn;
+    }
   }
   const int j = c / p.G, hh = c % p.G;
   p.out[(((size_t)b * p.nq_stride + j) * p.Hq + hkv * p.G + hh) * LYNX_D + d] = L > 0.0f ? acc / L : 0.0f;
